@@ -1,0 +1,169 @@
+"""Sequential fp64 CPU oracle for Gated Slot Attention -- TEST INFRASTRUCTURE ONLY.
+
+Only the tests, the smoke check and the benchmark's CPU-baseline leg may import
+this package; the CUDA library and its Python binding never do, and the two
+share no code.
+
+``fwd`` / ``bwd`` / ``decode_step`` marshal numpy arrays into the plain C
+recurrence of ``gsa_oracle.c`` (Eq. 6 of arXiv 2409.07146, evaluated one token
+at a time in double precision) and spread the independent (batch, head) pairs
+over host threads.  ``unrolled.py`` and ``chunkwise.py`` hold second and third
+statements of the same function that the CPU tests use to pin this one.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+import threading
+from concurrent.futures import ThreadPoolExecutor
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "gsa_oracle.c")
+_SO = os.path.join(_HERE, "libgsa_oracle.so")
+_lock = threading.Lock()
+_lib = None
+
+_D = ctypes.POINTER(ctypes.c_double)
+
+
+def build(force: bool = False) -> str:
+    """Compile the C oracle with gcc (no CUDA involved) and return the .so path."""
+    with _lock:
+        if force or not os.path.exists(_SO) or os.path.getmtime(_SO) < os.path.getmtime(_SRC):
+            tmp = _SO + ".tmp.%d" % os.getpid()
+            subprocess.check_call(
+                ["gcc", "-O2", "-std=c11", "-fPIC", "-shared", "-o", tmp, _SRC, "-lm"])
+            os.replace(tmp, _SO)
+    return _SO
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        lib = ctypes.CDLL(build())
+        i, d = ctypes.c_int, ctypes.c_double
+        lib.gsa_oracle_fwd.argtypes = [i] * 7 + [d] + [_D] * 10 + [i, i]
+        lib.gsa_oracle_fwd.restype = i
+        lib.gsa_oracle_decode_step.argtypes = [i] * 6 + [d] + [_D] * 7 + [i, i]
+        lib.gsa_oracle_decode_step.restype = i
+        lib.gsa_oracle_bwd.argtypes = [i] * 7 + [d] + [_D] * 15 + [i, i]
+        lib.gsa_oracle_bwd.restype = i
+        _lib = lib
+    return _lib
+
+
+def _f64(x, shape=None):
+    if x is None:
+        return None
+    a = np.ascontiguousarray(np.asarray(x, dtype=np.float64))
+    if shape is not None and tuple(a.shape) != tuple(shape):
+        raise ValueError(f"expected shape {shape}, got {a.shape}")
+    return a
+
+
+def _p(a):
+    return None if a is None else a.ctypes.data_as(_D)
+
+
+def default_threads() -> int:
+    return max(1, len(os.sched_getaffinity(0)))
+
+
+def _run_split(fn, n_items: int, threads: int | None):
+    """Call fn(begin, end) over a partition of range(n_items) on host threads."""
+    nt = max(1, min(threads or default_threads(), n_items))
+    bounds = [(n_items * j // nt, n_items * (j + 1) // nt) for j in range(nt)]
+    if nt == 1:
+        rcs = [fn(*bounds[0])]
+    else:
+        with ThreadPoolExecutor(nt) as ex:
+            rcs = list(ex.map(lambda be: fn(*be), bounds))
+    if any(rc != 0 for rc in rcs):
+        raise RuntimeError(f"oracle returned {rcs}")
+    return nt
+
+
+def fwd(q, k, v, gate, *, gate_is_log=False, scale=1.0, K0=None, V0=None,
+        bh_range=None, threads=None):
+    """Eq. 6 over whole sequences.
+
+    q,k [B,T,H,d_k]; v [B,T,H,d_v]; gate [B,T,H,m] (a, or log a when
+    gate_is_log).  Returns dict(o, ok, KT, VT): outputs, scaled pre-softmax slot
+    logits [B,T,H,m], final memories [B,H,m,d].  ``bh_range=(lo, hi)`` restricts
+    the work to those flattened (b,h) pairs; the other entries stay zero.
+    """
+    lib = _load()
+    q = _f64(q); B, T, H, dk = q.shape
+    k = _f64(k, (B, T, H, dk))
+    v = _f64(v); dv = v.shape[-1]
+    gate = _f64(gate); m = gate.shape[-1]
+    K0 = _f64(K0, (B, H, m, dk)) if K0 is not None else None
+    V0 = _f64(V0, (B, H, m, dv)) if V0 is not None else None
+    o = np.zeros((B, T, H, dv)); ok = np.zeros((B, T, H, m))
+    KT = np.zeros((B, H, m, dk)); VT = np.zeros((B, H, m, dv))
+    lo, hi = bh_range if bh_range is not None else (0, B * H)
+
+    def run(b0, b1):
+        return lib.gsa_oracle_fwd(B, T, H, dk, dv, m, int(gate_is_log), float(scale),
+                                  _p(q), _p(k), _p(v), _p(gate), _p(K0), _p(V0),
+                                  _p(o), _p(ok), _p(KT), _p(VT), lo + b0, lo + b1)
+
+    nt = _run_split(run, hi - lo, threads)
+    return dict(o=o, ok=ok, KT=KT, VT=VT, threads=nt)
+
+
+def bwd(q, k, v, gate, dO, *, gate_is_log=False, scale=1.0, K0=None, V0=None,
+        dKT=None, dVT=None, bh_range=None, threads=None):
+    """Reverse sweep of Eq. 6.  Returns dict(dq, dk, dv, dgate, dK0, dV0);
+    dgate is the total derivative w.r.t. the gate tensor as passed."""
+    lib = _load()
+    q = _f64(q); B, T, H, dk = q.shape
+    k = _f64(k, (B, T, H, dk))
+    v = _f64(v); dv = v.shape[-1]
+    gate = _f64(gate); m = gate.shape[-1]
+    dO = _f64(dO, (B, T, H, dv))
+    K0 = _f64(K0, (B, H, m, dk)) if K0 is not None else None
+    V0 = _f64(V0, (B, H, m, dv)) if V0 is not None else None
+    dKT = _f64(dKT, (B, H, m, dk)) if dKT is not None else None
+    dVT = _f64(dVT, (B, H, m, dv)) if dVT is not None else None
+    dq = np.zeros_like(q); dk_ = np.zeros_like(k); dv_ = np.zeros_like(v)
+    dgate = np.zeros_like(gate)
+    dK0 = np.zeros((B, H, m, dk)); dV0 = np.zeros((B, H, m, dv))
+    lo, hi = bh_range if bh_range is not None else (0, B * H)
+
+    def run(b0, b1):
+        return lib.gsa_oracle_bwd(B, T, H, dk, dv, m, int(gate_is_log), float(scale),
+                                  _p(q), _p(k), _p(v), _p(gate), _p(K0), _p(V0),
+                                  _p(dO), _p(dKT), _p(dVT), _p(dq), _p(dk_), _p(dv_),
+                                  _p(dgate), _p(dK0), _p(dV0), lo + b0, lo + b1)
+
+    nt = _run_split(run, hi - lo, threads)
+    return dict(dq=dq, dk=dk_, dv=dv_, dgate=dgate, dK0=dK0, dV0=dV0, threads=nt)
+
+
+def decode_step(q, k, v, gate, Kstate, Vstate, *, gate_is_log=False, scale=1.0,
+                threads=None):
+    """One recurrent step of Eq. 6 for S sequences; q,k [S,H,d_k], v [S,H,d_v],
+    gate [S,H,m]; Kstate/Vstate [S,H,m,d] float64 C-contiguous arrays updated IN
+    PLACE.  Returns o [S,H,d_v]."""
+    lib = _load()
+    q = _f64(q); S, H, dk = q.shape
+    k = _f64(k, (S, H, dk))
+    v = _f64(v); dv = v.shape[-1]
+    gate = _f64(gate); m = gate.shape[-1]
+    for st, d in ((Kstate, dk), (Vstate, dv)):
+        if not (isinstance(st, np.ndarray) and st.dtype == np.float64
+                and st.flags.c_contiguous and st.shape == (S, H, m, d)):
+            raise ValueError("states must be C-contiguous float64 [S,H,m,d] arrays")
+    o = np.zeros((S, H, dv))
+
+    def run(s0, s1):
+        return lib.gsa_oracle_decode_step(S, H, dk, dv, m, int(gate_is_log), float(scale),
+                                          _p(q), _p(k), _p(v), _p(gate), _p(Kstate),
+                                          _p(Vstate), _p(o), s0, s1)
+
+    _run_split(run, S * H, threads)
+    return o
