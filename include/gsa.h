@@ -1,0 +1,146 @@
+/*
+ * libgsa -- Gated Slot Attention layer for NVIDIA B200 (sm_100a), C ABI.
+ *
+ * The layer (arXiv 2409.07146, Sec. 3.2, Eq. 6), per (batch b, head h):
+ *     K~_t = Diag(a_t) K~_{t-1} + (1 - a_t) (x) k_t          (m x d_k)
+ *     V~_t = Diag(a_t) V~_{t-1} + (1 - a_t) (x) v_t          (m x d_v)
+ *     o_t  = V~_t^T softmax(scale * K~_t q_t)
+ * with both memories updated by token t before they are read.  Training and
+ * prefill evaluate it in the chunkwise two-pass form of Eq. 7 / Algorithm 1
+ * (two gated-linear-attention passes joined by a softmax over the m slots);
+ * decoding applies one step of Eq. 6.
+ *
+ * Conventions for every entry point
+ *   - All tensor pointers are DEVICE pointers owned by the caller, contiguous,
+ *     16-byte aligned.  Layouts: q,k,dq,dk [B,T,H,d_k]; v,o,dO,dv [B,T,H,d_v];
+ *     gate,dgate,ok [B,T,H,m]; memories and their gradients [B,H,m,d].
+ *   - q,k,v,o,dO,dq,dk,dv have the element type `io` (fp32 or bf16); gate, the
+ *     slot logits and all memories are always fp32; accumulation is fp32.
+ *   - The gate tensor holds a in [0,1] (GSA_GATE_A) or log a <= 0
+ *     (GSA_GATE_LOG_A).  Internally log a is clamped to >= -100.
+ *   - `params` is a HOST pointer.  `stream` is a cudaStream_t passed as void*
+ *     (NULL = the legacy default stream).  Work is only enqueued; nothing
+ *     synchronises with the host, allocates or frees device memory.
+ *   - `ws` is caller-provided device scratch of at least
+ *     gsa_workspace_bytes() bytes, 256-byte aligned; its contents are
+ *     undefined afterwards.  Calls that run concurrently need distinct
+ *     workspaces.
+ *   - Supported: d_k, d_v in {64,128,256,512}; m in {32,64}; B,T,H >= 1
+ *     (T need not be a multiple of the chunk; the tail chunk is masked).
+ *   - Errors are return codes; arguments are validated before anything is
+ *     launched and outputs are untouched when a call fails validation.
+ *     No entry point throws, aborts or prints.
+ */
+#ifndef GSA_H_
+#define GSA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define GSA_API __attribute__((visibility("default")))
+#else
+#define GSA_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    GSA_OK = 0,
+    GSA_ERR_INVALID_ARG = 1,  /* null/misaligned pointer, non-positive size, bad enum */
+    GSA_ERR_UNSUPPORTED = 2,  /* valid request outside the supported (d, m, dtype) set */
+    GSA_ERR_WORKSPACE = 3,    /* ws is NULL or smaller than gsa_workspace_bytes() */
+    GSA_ERR_CUDA = 4,         /* a CUDA runtime call or launch failed */
+    GSA_ERR_TIMEOUT = 5       /* a bounded device-side wait expired (see dev_status) */
+} gsa_status_t;
+
+typedef enum { GSA_F32 = 0, GSA_BF16 = 1 } gsa_dtype_t;
+typedef enum { GSA_GATE_A = 0, GSA_GATE_LOG_A = 1 } gsa_gate_t;
+
+/* Which kernels serve the d-sized contractions of the chunk passes. */
+typedef enum {
+    GSA_IMPL_AUTO = 0,   /* bf16 io: tensor-core kernels; fp32 io: fp32 CUDA-core kernels */
+    GSA_IMPL_SIMT = 1,   /* fp32 CUDA-core kernels for either io type */
+    GSA_IMPL_TC = 2      /* tcgen05 bf16 tensor-core kernels (bf16 io only) */
+} gsa_impl_t;
+
+typedef struct {
+    int32_t B, T, H, d_k, d_v, m;
+    int32_t io;         /* gsa_dtype_t */
+    int32_t gate_kind;  /* gsa_gate_t */
+    float scale;        /* multiplies the slot logits; 1.0f is the paper's layer */
+    int32_t impl;       /* gsa_impl_t */
+} gsa_params_t;
+
+enum { GSA_WS_FWD = 0, GSA_WS_BWD = 1, GSA_WS_DECODE = 2 };
+
+/* Chunk length C of the chunkwise form (Algorithm 1 leaves C open). */
+GSA_API int32_t gsa_chunk_size(void);
+
+/* Bytes of scratch `which` (GSA_WS_*) needs for these params; 0 for decode and
+ * for invalid params. */
+GSA_API size_t gsa_workspace_bytes(const gsa_params_t* params, int32_t which);
+
+GSA_API const char* gsa_status_string(gsa_status_t status);
+
+/*
+ * chunk_cumsum of Algorithm 1 (its "preprocessing" step), in log space: for
+ * each chunk of C tokens, G[i] = sum_{j <= i in chunk} log a_j (log a clamped
+ * to >= -100), and the input gate I = 1 - a.  gate, G, I: [B,T,H,m] fp32; G and
+ * I are written in full.  Uses no workspace.
+ */
+GSA_API gsa_status_t gsa_gate_cumsum(const gsa_params_t* params, const float* gate,
+                             float* G, float* I, void* stream);
+
+/*
+ * ForwardPass of Algorithm 1 == Eq. 6 over whole sequences.
+ *   in : q, k, v, gate; K0, V0 initial memories (NULL = zeros)
+ *   out: o; ok_save (nullable) the scaled pre-softmax slot logits
+ *        scale * K~_t q_t (the "output of the first GLA pass" that the paper
+ *        keeps for the backward); KT, VT (nullable) the final memories.
+ * dev_status (nullable, device int32): set non-zero by a kernel whose bounded
+ * wait expired; read it after synchronising the stream.
+ */
+GSA_API gsa_status_t gsa_fwd(const gsa_params_t* params, const void* q, const void* k,
+                     const void* v, const float* gate, const float* K0,
+                     const float* V0, void* o, float* ok_save, float* KT,
+                     float* VT, void* ws, size_t ws_bytes, void* stream,
+                     int32_t* dev_status);
+
+/*
+ * BackwardPass of Algorithm 1: gradients of gsa_fwd's o (and, optionally, of
+ * its final memories) w.r.t. every input.  The memories and the softmax are
+ * recomputed from the inputs (the paper's recomputation scheme); ok_saved
+ * (nullable) is gsa_fwd's ok_save and spares the recomputation of pass 1.
+ *   in : q, k, v, gate, K0, V0 (nullable) as given to gsa_fwd; dO;
+ *        dKT, dVT gradients w.r.t. the final memories (NULL = zeros)
+ *   out: dq, dk, dv; dgate = total derivative w.r.t. the gate tensor as
+ *        passed (through the decay and through the coupled input gate 1 - a);
+ *        dK0, dV0 (nullable).
+ * With GSA_GATE_A the decay part of dgate is d(log a)/a and loses accuracy as
+ * a -> 0; GSA_GATE_LOG_A has no such division.
+ */
+GSA_API gsa_status_t gsa_bwd(const gsa_params_t* params, const void* q, const void* k,
+                     const void* v, const float* gate, const float* K0,
+                     const float* V0, const float* ok_saved, const void* dO,
+                     const float* dKT, const float* dVT, void* dq, void* dk,
+                     void* dv, float* dgate, float* dK0, float* dV0, void* ws,
+                     size_t ws_bytes, void* stream, int32_t* dev_status);
+
+/*
+ * One recurrent step of Eq. 6 for B independent sequences (params->T is
+ * ignored): q,k [B,H,d_k], v,o [B,H,d_v] of type io, gate [B,H,m] fp32;
+ * Kstate [B,H,m,d_k] and Vstate [B,H,m,d_v] fp32 are updated IN PLACE (same
+ * layout as gsa_fwd's KT/VT, so a prefill hands its memories straight to the
+ * decoder).  Works in linear space: a = 0 and a = 1 are exact.  No workspace.
+ */
+GSA_API gsa_status_t gsa_decode_step(const gsa_params_t* params, const void* q,
+                             const void* k, const void* v, const float* gate,
+                             float* Kstate, float* Vstate, void* o, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GSA_H_ */

@@ -1,0 +1,207 @@
+"""ctypes binding of libgsa.so: same names and argument order as include/gsa.h."""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "libgsa.so")
+_lib = None
+
+GSA_F32, GSA_BF16 = 0, 1
+GSA_GATE_A, GSA_GATE_LOG_A = 0, 1
+GSA_IMPL_AUTO, GSA_IMPL_SIMT, GSA_IMPL_TC = 0, 1, 2
+GSA_WS_FWD, GSA_WS_BWD, GSA_WS_DECODE = 0, 1, 2
+
+_IMPL = {"auto": GSA_IMPL_AUTO, "simt": GSA_IMPL_SIMT, "tc": GSA_IMPL_TC}
+
+
+class GsaError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        msg = load_library().gsa_status_string(code).decode()
+        super().__init__(f"{where}: {msg} (status {code})")
+
+
+class _CParams(ctypes.Structure):
+    _fields_ = [("B", ctypes.c_int32), ("T", ctypes.c_int32), ("H", ctypes.c_int32),
+                ("d_k", ctypes.c_int32), ("d_v", ctypes.c_int32), ("m", ctypes.c_int32),
+                ("io", ctypes.c_int32), ("gate_kind", ctypes.c_int32),
+                ("scale", ctypes.c_float), ("impl", ctypes.c_int32)]
+
+
+@dataclass(frozen=True)
+class Params:
+    """Mirror of gsa_params_t."""
+    B: int
+    T: int
+    H: int
+    d_k: int
+    d_v: int
+    m: int
+    io: str = "bf16"          # "f32" | "bf16"
+    gate_is_log: bool = False
+    scale: float = 1.0
+    impl: str = "auto"        # "auto" | "simt" | "tc"
+
+    def c(self) -> _CParams:
+        return _CParams(self.B, self.T, self.H, self.d_k, self.d_v, self.m,
+                        GSA_BF16 if self.io == "bf16" else GSA_F32,
+                        GSA_GATE_LOG_A if self.gate_is_log else GSA_GATE_A,
+                        float(self.scale), _IMPL[self.impl])
+
+    @property
+    def io_dtype(self) -> torch.dtype:
+        return torch.bfloat16 if self.io == "bf16" else torch.float32
+
+
+def lib_path() -> str:
+    return _LIB_PATH
+
+
+def exported_symbols():
+    return ["gsa_chunk_size", "gsa_workspace_bytes", "gsa_status_string", "gsa_gate_cumsum",
+            "gsa_fwd", "gsa_bwd", "gsa_decode_step"]
+
+
+def load_library():
+    """Load libgsa.so; there is no fallback if it has not been built."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(_LIB_PATH):
+        raise ImportError(
+            f"{_LIB_PATH} is missing: build it with `python -m paper_2409_07146_b200.build` "
+            "(nvcc, sm_100a).  The GSA layer has no non-CUDA path.")
+    lib = ctypes.CDLL(_LIB_PATH)
+    vp, sz, i32 = ctypes.c_void_p, ctypes.c_size_t, ctypes.c_int32
+    pp = ctypes.POINTER(_CParams)
+    lib.gsa_chunk_size.argtypes = []
+    lib.gsa_chunk_size.restype = i32
+    lib.gsa_workspace_bytes.argtypes = [pp, i32]
+    lib.gsa_workspace_bytes.restype = sz
+    lib.gsa_status_string.argtypes = [ctypes.c_int]
+    lib.gsa_status_string.restype = ctypes.c_char_p
+    lib.gsa_gate_cumsum.argtypes = [pp, vp, vp, vp, vp]
+    lib.gsa_gate_cumsum.restype = ctypes.c_int
+    lib.gsa_fwd.argtypes = [pp] + [vp] * 10 + [vp, sz, vp, vp]
+    lib.gsa_fwd.restype = ctypes.c_int
+    lib.gsa_bwd.argtypes = [pp] + [vp] * 16 + [vp, sz, vp, vp]
+    lib.gsa_bwd.restype = ctypes.c_int
+    lib.gsa_decode_step.argtypes = [pp] + [vp] * 8
+    lib.gsa_decode_step.restype = ctypes.c_int
+    _lib = lib
+    return lib
+
+
+def _ptr(t, dtype=None, shape=None, name="tensor"):
+    if t is None:
+        return None
+    if not isinstance(t, torch.Tensor) or not t.is_cuda:
+        raise TypeError(f"{name}: expected a CUDA tensor (the library has no CPU path)")
+    if not t.is_contiguous():
+        raise ValueError(f"{name}: must be contiguous")
+    if dtype is not None and t.dtype != dtype:
+        raise TypeError(f"{name}: expected {dtype}, got {t.dtype}")
+    if shape is not None and tuple(t.shape) != tuple(shape):
+        raise ValueError(f"{name}: expected shape {tuple(shape)}, got {tuple(t.shape)}")
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def _stream():
+    return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _check(code: int, where: str):
+    if code != 0:
+        raise GsaError(code, where)
+
+
+def gsa_chunk_size() -> int:
+    return int(load_library().gsa_chunk_size())
+
+
+def gsa_workspace_bytes(p: Params, which: int) -> int:
+    cp = p.c()
+    return int(load_library().gsa_workspace_bytes(ctypes.byref(cp), which))
+
+
+def _workspace(p: Params, which: int, ws, device):
+    need = gsa_workspace_bytes(p, which)
+    if ws is None:
+        ws = torch.empty(max(need, 256), dtype=torch.uint8, device=device)
+    return ws, ws.numel() * ws.element_size()
+
+
+def gsa_gate_cumsum(p: Params, gate, G, I):
+    shp = (p.B, p.T, p.H, p.m)
+    cp = p.c()
+    _check(load_library().gsa_gate_cumsum(
+        ctypes.byref(cp), _ptr(gate, torch.float32, shp, "gate"), _ptr(G, torch.float32, shp, "G"),
+        _ptr(I, torch.float32, shp, "I"), _stream()), "gsa_gate_cumsum")
+
+
+def gsa_fwd(p: Params, q, k, v, gate, K0=None, V0=None, o=None, ok_save=None, KT=None, VT=None,
+            ws=None, dev_status=None):
+    """Enqueue the forward on the current stream.  `o` (and `ws`) are allocated with torch when
+    not given.  Returns o."""
+    io = p.io_dtype
+    qk, vv, mm = (p.B, p.T, p.H, p.d_k), (p.B, p.T, p.H, p.d_v), (p.B, p.T, p.H, p.m)
+    sk, sv = (p.B, p.H, p.m, p.d_k), (p.B, p.H, p.m, p.d_v)
+    if o is None:
+        o = torch.empty(vv, dtype=io, device=q.device)
+    ws, ws_bytes = _workspace(p, GSA_WS_FWD, ws, q.device)
+    cp = p.c()
+    _check(load_library().gsa_fwd(
+        ctypes.byref(cp), _ptr(q, io, qk, "q"), _ptr(k, io, qk, "k"), _ptr(v, io, vv, "v"),
+        _ptr(gate, torch.float32, mm, "gate"), _ptr(K0, torch.float32, sk, "K0"),
+        _ptr(V0, torch.float32, sv, "V0"), _ptr(o, io, vv, "o"),
+        _ptr(ok_save, torch.float32, mm, "ok_save"), _ptr(KT, torch.float32, sk, "KT"),
+        _ptr(VT, torch.float32, sv, "VT"), _ptr(ws, None, None, "ws"), ws_bytes, _stream(),
+        _ptr(dev_status, torch.int32, None, "dev_status")), "gsa_fwd")
+    return o
+
+
+def gsa_bwd(p: Params, q, k, v, gate, dO, K0=None, V0=None, ok_saved=None, dKT=None, dVT=None,
+            dq=None, dk=None, dv=None, dgate=None, dK0=None, dV0=None, ws=None, dev_status=None):
+    """Enqueue the backward on the current stream.  Returns (dq, dk, dv, dgate)."""
+    io = p.io_dtype
+    qk, vv, mm = (p.B, p.T, p.H, p.d_k), (p.B, p.T, p.H, p.d_v), (p.B, p.T, p.H, p.m)
+    sk, sv = (p.B, p.H, p.m, p.d_k), (p.B, p.H, p.m, p.d_v)
+    dev = q.device
+    dq = torch.empty(qk, dtype=io, device=dev) if dq is None else dq
+    dk = torch.empty(qk, dtype=io, device=dev) if dk is None else dk
+    dv = torch.empty(vv, dtype=io, device=dev) if dv is None else dv
+    dgate = torch.empty(mm, dtype=torch.float32, device=dev) if dgate is None else dgate
+    ws, ws_bytes = _workspace(p, GSA_WS_BWD, ws, dev)
+    cp = p.c()
+    _check(load_library().gsa_bwd(
+        ctypes.byref(cp), _ptr(q, io, qk, "q"), _ptr(k, io, qk, "k"), _ptr(v, io, vv, "v"),
+        _ptr(gate, torch.float32, mm, "gate"), _ptr(K0, torch.float32, sk, "K0"),
+        _ptr(V0, torch.float32, sv, "V0"), _ptr(ok_saved, torch.float32, mm, "ok_saved"),
+        _ptr(dO, io, vv, "dO"), _ptr(dKT, torch.float32, sk, "dKT"),
+        _ptr(dVT, torch.float32, sv, "dVT"), _ptr(dq, io, qk, "dq"), _ptr(dk, io, qk, "dk"),
+        _ptr(dv, io, vv, "dv"), _ptr(dgate, torch.float32, mm, "dgate"),
+        _ptr(dK0, torch.float32, sk, "dK0"), _ptr(dV0, torch.float32, sv, "dV0"),
+        _ptr(ws, None, None, "ws"), ws_bytes, _stream(),
+        _ptr(dev_status, torch.int32, None, "dev_status")), "gsa_bwd")
+    return dq, dk, dv, dgate
+
+
+def gsa_decode_step(p: Params, q, k, v, gate, Kstate, Vstate, o=None):
+    """One recurrent step for p.B sequences; Kstate/Vstate are updated in place.  Returns o."""
+    io = p.io_dtype
+    qk, vv, mm = (p.B, p.H, p.d_k), (p.B, p.H, p.d_v), (p.B, p.H, p.m)
+    if o is None:
+        o = torch.empty(vv, dtype=io, device=q.device)
+    cp = p.c()
+    _check(load_library().gsa_decode_step(
+        ctypes.byref(cp), _ptr(q, io, qk, "q"), _ptr(k, io, qk, "k"), _ptr(v, io, vv, "v"),
+        _ptr(gate, torch.float32, mm, "gate"),
+        _ptr(Kstate, torch.float32, (p.B, p.H, p.m, p.d_k), "Kstate"),
+        _ptr(Vstate, torch.float32, (p.B, p.H, p.m, p.d_v), "Vstate"), _ptr(o, io, vv, "o"),
+        _stream()), "gsa_decode_step")
+    return o

@@ -1,0 +1,231 @@
+// C ABI of the GSA library: argument validation, workspace carving and the order in which
+// the kernels of one forward / backward call are enqueued.  No kernel lives here.
+#include <string.h>
+
+#include "common.cuh"
+
+using namespace gsa;
+
+namespace {
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+bool ok_ptr(const void* p) { return p != nullptr && aligned16(p); }
+bool ok_opt(const void* p) { return p == nullptr || aligned16(p); }
+bool dim_ok(int d) { return d == 64 || d == 128 || d == 256 || d == 512; }
+
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+gsa_status_t check_params(const gsa_params_t* p, bool need_T) {
+    if (p == nullptr) return GSA_ERR_INVALID_ARG;
+    if (p->B < 1 || p->H < 1 || p->d_k < 1 || p->d_v < 1 || p->m < 1) return GSA_ERR_INVALID_ARG;
+    if (need_T && p->T < 1) return GSA_ERR_INVALID_ARG;
+    if (p->io != GSA_F32 && p->io != GSA_BF16) return GSA_ERR_INVALID_ARG;
+    if (p->gate_kind != GSA_GATE_A && p->gate_kind != GSA_GATE_LOG_A) return GSA_ERR_INVALID_ARG;
+    if (p->impl != GSA_IMPL_AUTO && p->impl != GSA_IMPL_SIMT && p->impl != GSA_IMPL_TC)
+        return GSA_ERR_INVALID_ARG;
+    if (!(p->scale == p->scale)) return GSA_ERR_INVALID_ARG;
+    if (!dim_ok(p->d_k) || !dim_ok(p->d_v)) return GSA_ERR_UNSUPPORTED;
+    if (p->m != 32 && p->m != 64) return GSA_ERR_UNSUPPORTED;
+    if ((long long)p->B * p->H > 0x7fffffffLL / 4) return GSA_ERR_UNSUPPORTED;
+    if (p->impl == GSA_IMPL_TC && p->io != GSA_BF16) return GSA_ERR_UNSUPPORTED;
+    return GSA_OK;
+}
+
+// Does this call run the tensor-core chunk kernels?
+bool use_tc(const gsa_params_t& p) {
+    if (p.impl == GSA_IMPL_SIMT) return false;
+    return p.io == GSA_BF16 && tc_supported(p.d_k, p.d_v, p.m);
+}
+
+struct Slices { int k, v; };
+Slices slices(const gsa_params_t& p) {
+    if (use_tc(p)) return {tc_value_side_slices(p.d_k), tc_value_side_slices(p.d_v)};
+    return {p.d_k / 64, p.d_v / 64};
+}
+
+struct Carver {
+    char* base; size_t off;
+    float* take(size_t nfloat) {
+        float* r = reinterpret_cast<float*>(base + off);
+        off += align_up(nfloat * sizeof(float), 256);
+        return r;
+    }
+};
+
+struct Workspace {
+    float *G, *I, *okpart, *ok, *p, *dz, *u, *dppart, *dIk, *dIv, *chunk_tot, *KT, *VT;
+    size_t bytes;
+};
+
+Workspace carve(const gsa_params_t& p, int which, void* ws) {
+    Workspace w;
+    memset(&w, 0, sizeof(w));
+    const size_t mt = (size_t)p.B * p.T * p.H * p.m;
+    const Slices s = slices(p);
+    Carver c{static_cast<char*>(ws), 0};
+    w.G = c.take(mt);
+    w.I = c.take(mt);
+    w.okpart = c.take(mt * s.k);
+    w.ok = c.take(mt);
+    w.p = c.take(mt);
+    if (which == GSA_WS_BWD) {
+        w.dz = c.take(mt);
+        w.u = c.take(mt);
+        w.dppart = c.take(mt * s.v);
+        w.dIk = c.take(mt * s.k);
+        w.dIv = c.take(mt * s.v);
+        w.chunk_tot = c.take((size_t)p.B * p.H * ((p.T + kChunk - 1) / kChunk) * p.m);
+        w.KT = c.take((size_t)p.B * p.H * p.m * p.d_k);
+        w.VT = c.take((size_t)p.B * p.H * p.m * p.d_v);
+    }
+    w.bytes = c.off;
+    return w;
+}
+
+cudaError_t value_side(const gsa_params_t& p, const ValueSideArgs& a, int reverse, cudaStream_t st,
+                       int32_t* dev_status) {
+    if (use_tc(p)) return launch_value_side_tc(a, p.m, reverse, st, dev_status);
+    return launch_value_side_simt(a, p.io, p.m, reverse, st);
+}
+cudaError_t key_side(const gsa_params_t& p, const KeySideArgs& a, int reverse, cudaStream_t st,
+                     int32_t* dev_status) {
+    if (use_tc(p)) return launch_key_side_tc(a, p.m, reverse, st, dev_status);
+    return launch_key_side_simt(a, p.io, p.m, reverse, st);
+}
+
+#define GSA_CUDA(expr)                                  \
+    do {                                                \
+        cudaError_t e__ = (expr);                       \
+        if (e__ != cudaSuccess) return GSA_ERR_CUDA;    \
+    } while (0)
+
+}  // namespace
+
+extern "C" {
+
+int32_t gsa_chunk_size(void) { return kChunk; }
+
+const char* gsa_status_string(gsa_status_t status) {
+    switch (status) {
+        case GSA_OK: return "ok";
+        case GSA_ERR_INVALID_ARG: return "invalid argument";
+        case GSA_ERR_UNSUPPORTED: return "unsupported shape or dtype";
+        case GSA_ERR_WORKSPACE: return "workspace missing or too small";
+        case GSA_ERR_CUDA: return "CUDA error";
+        case GSA_ERR_TIMEOUT: return "bounded device-side wait expired";
+    }
+    return "unknown status";
+}
+
+size_t gsa_workspace_bytes(const gsa_params_t* params, int32_t which) {
+    if (which == GSA_WS_DECODE) return 0;
+    if (which != GSA_WS_FWD && which != GSA_WS_BWD) return 0;
+    if (check_params(params, true) != GSA_OK) return 0;
+    return carve(*params, which, nullptr).bytes;
+}
+
+gsa_status_t gsa_gate_cumsum(const gsa_params_t* params, const float* gate, float* G, float* I,
+                             void* stream) {
+    gsa_status_t st = check_params(params, true);
+    if (st != GSA_OK) return st;
+    if (!ok_ptr(gate) || !ok_ptr(G) || !ok_ptr(I)) return GSA_ERR_INVALID_ARG;
+    const gsa_params_t& p = *params;
+    GSA_CUDA(launch_gate_cumsum(gate, p.gate_kind == GSA_GATE_LOG_A, G, I, p.B, p.T, p.H, p.m,
+                                static_cast<cudaStream_t>(stream)));
+    return GSA_OK;
+}
+
+gsa_status_t gsa_fwd(const gsa_params_t* params, const void* q, const void* k, const void* v,
+                     const float* gate, const float* K0, const float* V0, void* o,
+                     float* ok_save, float* KT, float* VT, void* ws, size_t ws_bytes,
+                     void* stream, int32_t* dev_status) {
+    gsa_status_t rc = check_params(params, true);
+    if (rc != GSA_OK) return rc;
+    if (!ok_ptr(q) || !ok_ptr(k) || !ok_ptr(v) || !ok_ptr(gate) || !ok_ptr(o)) return GSA_ERR_INVALID_ARG;
+    if (!ok_opt(K0) || !ok_opt(V0) || !ok_opt(ok_save) || !ok_opt(KT) || !ok_opt(VT))
+        return GSA_ERR_INVALID_ARG;
+    const gsa_params_t& p = *params;
+    if (ws == nullptr || (reinterpret_cast<uintptr_t>(ws) & 255u) != 0) return GSA_ERR_WORKSPACE;
+    const Workspace w = carve(p, GSA_WS_FWD, ws);
+    if (ws_bytes < w.bytes) return GSA_ERR_WORKSPACE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const Slices s = slices(p);
+    const size_t rows = (size_t)p.B * p.T * p.H;
+
+    GSA_CUDA(launch_gate_cumsum(gate, p.gate_kind == GSA_GATE_LOG_A, w.G, w.I, p.B, p.T, p.H, p.m, st));
+    // pass 1: o' = GLA(q, k, 1-a) with the decay on the slot (value) side
+    ValueSideArgs a1{q, k, w.I, w.G, K0, KT, w.okpart, p.B, p.T, p.H, p.d_k};
+    GSA_CUDA(value_side(p, a1, 0, st, dev_status));
+    float* ok = ok_save ? ok_save : w.ok;
+    GSA_CUDA(launch_slot_softmax_fwd(w.okpart, s.k, p.scale, ok, w.p, rows, p.m, st));
+    // pass 2: o = GLA(softmax(o'), 1-a, v) with the decay on the slot (key) side
+    KeySideArgs a2{w.p, w.I, w.G, v, V0, VT, o, p.B, p.T, p.H, p.d_v};
+    GSA_CUDA(key_side(p, a2, 0, st, dev_status));
+    return GSA_OK;
+}
+
+gsa_status_t gsa_bwd(const gsa_params_t* params, const void* q, const void* k, const void* v,
+                     const float* gate, const float* K0, const float* V0, const float* ok_saved,
+                     const void* dO, const float* dKT, const float* dVT, void* dq, void* dk,
+                     void* dv, float* dgate, float* dK0, float* dV0, void* ws, size_t ws_bytes,
+                     void* stream, int32_t* dev_status) {
+    gsa_status_t rc = check_params(params, true);
+    if (rc != GSA_OK) return rc;
+    if (!ok_ptr(q) || !ok_ptr(k) || !ok_ptr(v) || !ok_ptr(gate) || !ok_ptr(dO) || !ok_ptr(dq) ||
+        !ok_ptr(dk) || !ok_ptr(dv) || !ok_ptr(dgate))
+        return GSA_ERR_INVALID_ARG;
+    if (!ok_opt(K0) || !ok_opt(V0) || !ok_opt(ok_saved) || !ok_opt(dKT) || !ok_opt(dVT) ||
+        !ok_opt(dK0) || !ok_opt(dV0))
+        return GSA_ERR_INVALID_ARG;
+    const gsa_params_t& p = *params;
+    if (ws == nullptr || (reinterpret_cast<uintptr_t>(ws) & 255u) != 0) return GSA_ERR_WORKSPACE;
+    const Workspace w = carve(p, GSA_WS_BWD, ws);
+    if (ws_bytes < w.bytes) return GSA_ERR_WORKSPACE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const Slices s = slices(p);
+    const size_t rows = (size_t)p.B * p.T * p.H;
+
+    GSA_CUDA(launch_gate_cumsum(gate, p.gate_kind == GSA_GATE_LOG_A, w.G, w.I, p.B, p.T, p.H, p.m, st));
+    const float* ok = ok_saved;
+    if (ok == nullptr) {  // recompute pass 1 and its logits
+        ValueSideArgs a1{q, k, w.I, w.G, K0, nullptr, w.okpart, p.B, p.T, p.H, p.d_k};
+        GSA_CUDA(value_side(p, a1, 0, st, dev_status));
+        GSA_CUDA(launch_slot_softmax_fwd(w.okpart, s.k, p.scale, w.ok, w.p, rows, p.m, st));
+        ok = w.ok;
+    }
+    // gradient w.r.t. the pass-2 queries p: the pass-1 form on (dO, v, 1-a); carries V~
+    ValueSideArgs adp{dO, v, w.I, w.G, V0, dVT ? w.VT : nullptr, w.dppart, p.B, p.T, p.H, p.d_v};
+    GSA_CUDA(value_side(p, adp, 0, st, dev_status));
+    GSA_CUDA(launch_slot_softmax_bwd(ok, w.dppart, s.v, p.scale, w.p, w.dz, w.u, rows, p.m, st));
+    // dq: the pass-2 form on (dz, 1-a, k); carries K~
+    KeySideArgs adq{w.dz, w.I, w.G, k, K0, dKT ? w.KT : nullptr, dq, p.B, p.T, p.H, p.d_k};
+    GSA_CUDA(key_side(p, adq, 0, st, dev_status));
+    // time-reversed runs: dv and dI^v share the state dV~; dk and dI^k share dK~
+    KeySideArgs adv{w.I, w.p, w.G, dO, dVT, dV0, dv, p.B, p.T, p.H, p.d_v};
+    GSA_CUDA(key_side(p, adv, 1, st, dev_status));
+    ValueSideArgs adIv{v, dO, w.p, w.G, dVT, nullptr, w.dIv, p.B, p.T, p.H, p.d_v};
+    GSA_CUDA(value_side(p, adIv, 1, st, dev_status));
+    KeySideArgs adk{w.I, w.dz, w.G, q, dKT, dK0, dk, p.B, p.T, p.H, p.d_k};
+    GSA_CUDA(key_side(p, adk, 1, st, dev_status));
+    ValueSideArgs adIk{k, q, w.dz, w.G, dKT, nullptr, w.dIk, p.B, p.T, p.H, p.d_k};
+    GSA_CUDA(value_side(p, adIk, 1, st, dev_status));
+    // forget-gate gradient: reversed cumulative sum over the whole sequence
+    GSA_CUDA(launch_gate_grad(w.u, w.I, w.dIk, s.k, w.dIv, s.v, gate, p.gate_kind == GSA_GATE_LOG_A,
+                              dKT, w.KT, dVT, w.VT, p.d_k, p.d_v, w.chunk_tot, dgate, p.B, p.T,
+                              p.H, p.m, st));
+    return GSA_OK;
+}
+
+gsa_status_t gsa_decode_step(const gsa_params_t* params, const void* q, const void* k,
+                             const void* v, const float* gate, float* Kstate, float* Vstate,
+                             void* o, void* stream) {
+    gsa_status_t rc = check_params(params, false);
+    if (rc != GSA_OK) return rc;
+    if (!ok_ptr(q) || !ok_ptr(k) || !ok_ptr(v) || !ok_ptr(gate) || !ok_ptr(Kstate) ||
+        !ok_ptr(Vstate) || !ok_ptr(o))
+        return GSA_ERR_INVALID_ARG;
+    GSA_CUDA(launch_decode(*params, q, k, v, gate, Kstate, Vstate, o, static_cast<cudaStream_t>(stream)));
+    return GSA_OK;
+}
+
+}  // extern "C"

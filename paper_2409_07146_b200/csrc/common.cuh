@@ -1,0 +1,121 @@
+// Shared declarations of the GSA CUDA library (internal; the public surface is include/gsa.h).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "gsa.h"
+
+namespace gsa {
+
+constexpr int kChunk = 64;            // C of the chunkwise form
+constexpr float kLogGateMin = -100.f; // clamp of log a (exp(-100) == 0 in fp32)
+// A chunk whose total log-decay stays above this bound uses the factorised
+// decay exp(G_i) * exp(-G_j) (one reference point per chunk); below it the
+// exponent differences are taken explicitly so nothing can overflow.
+constexpr float kFactorisedDecayMin = -60.f;
+
+template <typename T> struct IoTraits;
+template <> struct IoTraits<float> {
+    static constexpr int kVec = 4;  // elements per 16-byte access
+};
+template <> struct IoTraits<__nv_bfloat16> {
+    static constexpr int kVec = 8;
+};
+
+// 16-byte global load of kVec consecutive elements, widened to fp32.
+__device__ __forceinline__ void load_vec(const float* p, float (&out)[4]) {
+    float4 v = *reinterpret_cast<const float4*>(p);
+    out[0] = v.x; out[1] = v.y; out[2] = v.z; out[3] = v.w;
+}
+__device__ __forceinline__ void load_vec(const __nv_bfloat16* p, float (&out)[8]) {
+    uint4 v = *reinterpret_cast<const uint4*>(p);
+    const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&v);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        float2 f = __bfloat1622float2(h[i]);
+        out[2 * i] = f.x; out[2 * i + 1] = f.y;
+    }
+}
+__device__ __forceinline__ void store_vec(float* p, const float (&in)[4]) {
+    *reinterpret_cast<float4*>(p) = make_float4(in[0], in[1], in[2], in[3]);
+}
+__device__ __forceinline__ void store_vec(__nv_bfloat16* p, const float (&in)[8]) {
+    uint4 v;
+    __nv_bfloat162* h = reinterpret_cast<__nv_bfloat162*>(&v);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) h[i] = __floats2bfloat162_rn(in[2 * i], in[2 * i + 1]);
+    *reinterpret_cast<uint4*>(p) = v;
+}
+__device__ __forceinline__ void store_vec4(float* p, const float (&in)[4]) {
+    *reinterpret_cast<float4*>(p) = make_float4(in[0], in[1], in[2], in[3]);
+}
+__device__ __forceinline__ void store_vec4(__nv_bfloat16* p, const float (&in)[4]) {
+    uint2 v;
+    __nv_bfloat162* h = reinterpret_cast<__nv_bfloat162*>(&v);
+    h[0] = __floats2bfloat162_rn(in[0], in[1]);
+    h[1] = __floats2bfloat162_rn(in[2], in[3]);
+    *reinterpret_cast<uint2*>(p) = v;
+}
+
+// ---- arguments of the two chunk primitives (both passes, forward and time-reversed) ----
+//
+// value_side ("gsa_fwd" of Algorithm 1 with GATE_K = False, the pass-1 form):
+//     out_i[s] = sum_{j<=i} <xq_i, xk_j> w_j[s] prod_{r=j+1..i} a_r[s]   (+ state term)
+//   xq, xk: [B,T,H,D] io; w, G: [B,T,H,M] fp32; state S (D x M), given/returned in the
+//   memory layout [B,H,M,D].  The contraction over D is split into `nslice` slices of
+//   width D/nslice; slice z writes its partial sums to out + z * B*T*H*M.
+//
+// key_side ("gsa_fwd" with GATE_K = True, the pass-2 form):
+//     out_i = sum_{j<=i} (sum_s uq_i[s] uk_j[s] prod_{r=j+1..i} a_r[s]) xv_j   (+ state term)
+//   uq, uk, G: [B,T,H,M] fp32; xv, out: [B,T,H,D] io; state S (M x D) in [B,H,M,D].
+//
+// reverse = 1 sums over i >= j instead (same decay product): the gradients w.r.t. keys,
+// values and the input gate are such time-reversed runs.
+struct ValueSideArgs {
+    const void* xq; const void* xk;   // io
+    const float* w; const float* G;
+    const float* S0;                  // nullable
+    float* Send;                      // nullable
+    float* out;                       // [nslice][B,T,H,M]
+    int B, T, H, D;
+};
+struct KeySideArgs {
+    const float* uq; const float* uk; const float* G;
+    const void* xv;                   // io
+    const float* S0;                  // nullable
+    float* Send;                      // nullable
+    void* out;                        // io [B,T,H,D]
+    int B, T, H, D;
+};
+
+// launchers (definitions in the .cu files); all return cudaGetLastError() of the launch
+cudaError_t launch_gate_cumsum(const float* gate, int gate_is_log, float* G, float* I,
+                               int B, int T, int H, int M, cudaStream_t st);
+cudaError_t launch_slot_softmax_fwd(const float* part, int nslice, float scale, float* ok,
+                                    float* p, size_t rows, int M, cudaStream_t st);
+cudaError_t launch_slot_softmax_bwd(const float* ok, const float* dp_part, int nslice,
+                                    float scale, float* p, float* dz, float* u, size_t rows,
+                                    int M, cudaStream_t st);
+cudaError_t launch_gate_grad(const float* u, const float* I, const float* dIk_part, int nsk,
+                             const float* dIv_part, int nsv, const float* gate,
+                             int gate_is_log, const float* dKT, const float* KT,
+                             const float* dVT, const float* VT, int d_k, int d_v,
+                             float* chunk_tot, float* dgate, int B, int T, int H, int M,
+                             cudaStream_t st);
+cudaError_t launch_value_side_simt(const ValueSideArgs& a, int io, int M, int reverse,
+                                   cudaStream_t st);
+cudaError_t launch_key_side_simt(const KeySideArgs& a, int io, int M, int reverse,
+                                 cudaStream_t st);
+// tcgen05 (bf16 tensor-core) versions of the two primitives; bf16 io only.
+bool tc_supported(int d_k, int d_v, int M);
+int tc_value_side_slices(int D);   // how many partial-sum slices value_side writes for width D
+cudaError_t launch_value_side_tc(const ValueSideArgs& a, int M, int reverse, cudaStream_t st,
+                                 int32_t* dev_status);
+cudaError_t launch_key_side_tc(const KeySideArgs& a, int M, int reverse, cudaStream_t st,
+                               int32_t* dev_status);
+cudaError_t launch_decode(const gsa_params_t& p, const void* q, const void* k, const void* v,
+                          const float* gate, float* Ks, float* Vs, void* o, cudaStream_t st);
+
+}  // namespace gsa

@@ -1,0 +1,213 @@
+"""GPU parity: every entry point of libgsa.so, called through the C ABI binding, against
+the sequential fp64 oracle on the same seeded inputs (element by element)."""
+import numpy as np
+import pytest
+import torch
+
+import gsa_workloads as W
+import oracle
+import paper_2409_07146_b200 as gsa
+from util import TOL, rand_inputs, rel_err, to_dev, to_np
+
+pytestmark = pytest.mark.gpu
+
+
+def run_fwd(d, B, T, H, dk, dv, m, io, impl="auto", scale=1.0, log=False, want_states=True):
+    p = gsa.Params(B, T, H, dk, dv, m, io=io, impl=impl, scale=scale, gate_is_log=log)
+    gate = np.log(np.maximum(d["gate"].astype(np.float64), 1e-300)).astype(np.float32) if log else d["gate"]
+    K0, V0 = to_dev(d.get("K0")), to_dev(d.get("V0"))
+    KT = torch.empty(B, H, m, dk, device="cuda") if want_states else None
+    VT = torch.empty(B, H, m, dv, device="cuda") if want_states else None
+    ok = torch.empty(B, T, H, m, device="cuda")
+    o = gsa.gsa_fwd(p, to_dev(d["q"], io), to_dev(d["k"], io), to_dev(d["v"], io), to_dev(gate),
+                    K0, V0, ok_save=ok, KT=KT, VT=VT)
+    torch.cuda.synchronize()
+    return dict(o=to_np(o), ok=to_np(ok), KT=None if KT is None else to_np(KT),
+                VT=None if VT is None else to_np(VT)), gate
+
+
+def check_fwd(d, got, gate, io, scale=1.0, log=False, tol=None):
+    ref = oracle.fwd(d["q"], d["k"], d["v"], gate, gate_is_log=log, scale=scale,
+                     K0=d.get("K0"), V0=d.get("V0"))
+    tol = tol or TOL[io]
+    errs = {n: rel_err(got[n], ref[n]) for n in ("o", "ok", "KT", "VT") if got[n] is not None}
+    assert all(np.isfinite(got[n]).all() for n in errs), "non-finite output"
+    assert all(e <= tol for e in errs.values()), errs
+    return errs
+
+
+# ------------------------------------------------------------------ gate kernel
+@pytest.mark.parametrize("T,m,log", [(256, 64, False), (100, 32, True), (1, 64, False)])
+def test_gate_cumsum(T, m, log):
+    B, H = 2, 3
+    r = np.random.default_rng(T + m)
+    a = (1 / (1 + np.exp(-r.standard_normal((B, T, H, m))))).astype(np.float32)
+    a[0, T // 2, 0, 0] = 0.0
+    gate = np.log(np.maximum(a.astype(np.float64), 1e-300)).astype(np.float32) if log else a
+    p = gsa.Params(B, T, H, 64, 64, m, gate_is_log=log)
+    G = torch.empty(B, T, H, m, device="cuda"); I = torch.empty_like(G)
+    gsa.gsa_gate_cumsum(p, to_dev(gate), G, I)
+    g64 = np.maximum(gate.astype(np.float64) if log else np.log(np.maximum(a.astype(np.float64), 1e-300)), -100.0)
+    ref = np.zeros_like(g64)
+    C = gsa.gsa_chunk_size()
+    for t0 in range(0, T, C):
+        ref[:, t0:t0 + C] = np.cumsum(g64[:, t0:t0 + C], axis=1)
+    np.testing.assert_allclose(to_np(G), ref, rtol=2e-6, atol=2e-6)
+    iref = -np.expm1(gate.astype(np.float64)) if log else 1.0 - a.astype(np.float64)
+    np.testing.assert_allclose(to_np(I), iref, rtol=1e-6, atol=1e-7)
+
+
+# ------------------------------------------------------------------ forward
+@pytest.mark.parametrize("io", ["f32", "bf16"])
+@pytest.mark.parametrize("T", [1, 15, 17, 64, 65, 100, 256])
+def test_fwd_ragged_lengths_simt(io, T):
+    B, H, dk, dv, m = 2, 2, 64, 128, 32
+    d = rand_inputs(100 + T, B, T, H, dk, dv, m, io, init=True)
+    got, gate = run_fwd(d, B, T, H, dk, dv, m, io, impl="simt", scale=0.9)
+    check_fwd(d, got, gate, io, scale=0.9)
+
+
+@pytest.mark.parametrize("io", ["f32", "bf16"])
+@pytest.mark.parametrize("dk,dv,m", [(64, 64, 64), (128, 64, 64), (256, 128, 32), (512, 512, 64)])
+def test_fwd_shapes_simt(io, dk, dv, m):
+    B, T, H = 1, 200, 2
+    d = rand_inputs(7, B, T, H, dk, dv, m, io)
+    got, gate = run_fwd(d, B, T, H, dk, dv, m, io, impl="simt")
+    check_fwd(d, got, gate, io)
+
+
+@pytest.mark.parametrize("impl", ["simt", "auto"])
+@pytest.mark.parametrize("gate", ["strong", "mixed"])
+@pytest.mark.parametrize("log", [False, True])
+def test_fwd_strong_forgetting_and_exact_zero_one_gates(impl, gate, log):
+    # chunks whose decay underflows take the explicit-exponent path; a == 0 and a == 1 exactly
+    B, T, H, dk, dv, m = 1, 192, 2, 64, 64, 32
+    io = "bf16" if impl == "auto" else "f32"
+    d = rand_inputs(11, B, T, H, dk, dv, m, io, init=True, gate=gate)
+    got, g = run_fwd(d, B, T, H, dk, dv, m, io, impl=impl, log=log)
+    gref = np.maximum(g.astype(np.float64), -100.0) if log else g
+    check_fwd(d, got, gref, io, log=log)
+
+
+def test_fwd_tiny_config_fp32():
+    # configuration 1: B=1 H=2 T=256 d=64 m=32, fp32, seed 0
+    w = W.CONFIGS["tiny_f32"]
+    d = W.make_inputs(w)
+    got, gate = run_fwd(d, w.B, w.T, w.H, w.d_k, w.d_v, w.m, "f32")
+    errs = check_fwd(d, got, gate, "f32")
+    print("tiny_f32 fwd errors", errs)
+    # a == 0 => o = v on the same shape
+    d0 = dict(d, gate=np.zeros_like(d["gate"]))
+    got0, _ = run_fwd(d0, w.B, w.T, w.H, w.d_k, w.d_v, w.m, "f32")
+    assert rel_err(got0["o"], d["v"]) <= 1e-6
+
+
+def test_fwd_is_deterministic_and_leaves_inputs_alone():
+    B, T, H, dk, dv, m = 2, 130, 2, 64, 64, 64
+    d = rand_inputs(5, B, T, H, dk, dv, m, "bf16")
+    a, _ = run_fwd(d, B, T, H, dk, dv, m, "bf16")
+    b, _ = run_fwd(d, B, T, H, dk, dv, m, "bf16")
+    for n in ("o", "ok", "KT", "VT"):
+        np.testing.assert_array_equal(a[n], b[n])
+
+
+def test_fwd_state_carry_matches_one_call():
+    B, T, H, dk, dv, m = 1, 192, 2, 64, 64, 32
+    d = rand_inputs(21, B, T, H, dk, dv, m, "f32")
+    full, gate = run_fwd(d, B, T, H, dk, dv, m, "f32")
+    cut = 100
+    d1 = {n: (x[:, :cut] if x.shape[1] == T else x) for n, x in d.items()}
+    first, _ = run_fwd(d1, B, cut, H, dk, dv, m, "f32")
+    d2 = {n: (x[:, cut:] if x.shape[1] == T else x) for n, x in d.items()}
+    d2["K0"], d2["V0"] = first["KT"].astype(np.float32), first["VT"].astype(np.float32)
+    second, _ = run_fwd(d2, B, T - cut, H, dk, dv, m, "f32")
+    assert rel_err(np.concatenate([first["o"], second["o"]], 1), full["o"]) <= 1e-5
+    assert rel_err(second["KT"], full["KT"]) <= 1e-5
+
+
+# ------------------------------------------------------------------ backward
+def run_bwd(d, B, T, H, dk, dv, m, io, impl="auto", scale=1.0, log=False, saved=False):
+    p = gsa.Params(B, T, H, dk, dv, m, io=io, impl=impl, scale=scale, gate_is_log=log)
+    gate = np.log(d["gate"].astype(np.float64)).astype(np.float32) if log else d["gate"]
+    q, k, v, dO = (to_dev(d[n], io) for n in ("q", "k", "v", "dO"))
+    K0, V0, dKT, dVT = (to_dev(d.get(n)) for n in ("K0", "V0", "dKT", "dVT"))
+    ok = None
+    if saved:
+        ok = torch.empty(B, T, H, m, device="cuda")
+        gsa.gsa_fwd(p, q, k, v, to_dev(gate), K0, V0, ok_save=ok)
+    dK0 = torch.empty(B, H, m, dk, device="cuda"); dV0 = torch.empty(B, H, m, dv, device="cuda")
+    dq, dk_, dv_, dg = gsa.gsa_bwd(p, q, k, v, to_dev(gate), dO, K0, V0, ok_saved=ok, dKT=dKT,
+                                   dVT=dVT, dK0=dK0, dV0=dV0)
+    torch.cuda.synchronize()
+    got = dict(dq=to_np(dq), dk=to_np(dk_), dv=to_np(dv_), dgate=to_np(dg), dK0=to_np(dK0), dV0=to_np(dV0))
+    ref = oracle.bwd(d["q"], d["k"], d["v"], gate, d["dO"], gate_is_log=log, scale=scale,
+                     K0=d.get("K0"), V0=d.get("V0"), dKT=d.get("dKT"), dVT=d.get("dVT"))
+    return got, ref
+
+
+def check_bwd(got, ref, tol):
+    errs = {n: rel_err(got[n], ref[n]) for n in got}
+    assert all(np.isfinite(got[n]).all() for n in got), "non-finite gradient"
+    assert all(e <= tol for e in errs.values()), errs
+    return errs
+
+
+@pytest.mark.parametrize("io", ["f32", "bf16"])
+@pytest.mark.parametrize("T", [17, 64, 150])
+@pytest.mark.parametrize("log", [False, True])
+def test_bwd_simt(io, T, log):
+    B, H, dk, dv, m = 2, 2, 64, 128, 32
+    d = rand_inputs(300 + T, B, T, H, dk, dv, m, io, init=True, final_grads=True)
+    got, ref = run_bwd(d, B, T, H, dk, dv, m, io, impl="simt", scale=1.1, log=log)
+    check_bwd(got, ref, TOL[io])
+
+
+@pytest.mark.parametrize("saved", [False, True])
+def test_bwd_zero_init_with_and_without_saved_logits(saved):
+    B, T, H, dk, dv, m = 1, 200, 2, 128, 64, 64
+    d = rand_inputs(41, B, T, H, dk, dv, m, "f32")
+    got, ref = run_bwd(d, B, T, H, dk, dv, m, "f32", saved=saved)
+    check_bwd(got, ref, TOL["f32"])
+
+
+def test_bwd_strong_forgetting():
+    B, T, H, dk, dv, m = 1, 160, 1, 64, 64, 32
+    d = rand_inputs(43, B, T, H, dk, dv, m, "f32", init=True, gate="strong")
+    got, ref = run_bwd(d, B, T, H, dk, dv, m, "f32", log=True)
+    check_bwd(got, ref, TOL["f32"])
+
+
+# ------------------------------------------------------------------ decode
+@pytest.mark.parametrize("io", ["f32", "bf16"])
+@pytest.mark.parametrize("dk,dv,m", [(64, 64, 32), (128, 128, 64), (256, 512, 64), (512, 64, 32)])
+def test_decode_steps(io, dk, dv, m):
+    S, H, steps = 3, 5, 4
+    w = W.CONFIGS["decode"].scaled(B=S, H=H, d_k=dk, d_v=dv, m=m, io=io)
+    st = W.make_decode_states(w)
+    Ks, Vs = to_dev(st["K"]), to_dev(st["V"])
+    Kr, Vr = st["K"].astype(np.float64), st["V"].astype(np.float64)
+    p = gsa.Params(S, 1, H, dk, dv, m, io=io, scale=0.8)
+    for step in range(steps):
+        x = W.make_decode_step_inputs(w, step)
+        if step == 2:   # exact 0 and 1 gates are handled in linear space
+            x["gate"][:, :, 0] = 0.0
+            x["gate"][:, :, 1] = 1.0
+        o = gsa.gsa_decode_step(p, to_dev(x["q"], io), to_dev(x["k"], io), to_dev(x["v"], io),
+                                to_dev(x["gate"]), Ks, Vs)
+        ro = oracle.decode_step(x["q"], x["k"], x["v"], x["gate"], Kr, Vr, scale=0.8)
+        assert rel_err(to_np(o), ro) <= TOL[io]
+    assert rel_err(to_np(Ks), Kr) <= 1e-5 and rel_err(to_np(Vs), Vr) <= 1e-5
+
+
+def test_decode_continues_a_prefill():
+    # prefill with gsa_fwd, hand KT/VT to the decoder, compare with one long forward
+    B, T, H, dk, dv, m = 2, 70, 2, 64, 64, 32
+    d = rand_inputs(51, B, T + 3, H, dk, dv, m, "f32")
+    ref = oracle.fwd(d["q"], d["k"], d["v"], d["gate"])
+    d1 = {n: x[:, :T] for n, x in d.items()}
+    got, _ = run_fwd(d1, B, T, H, dk, dv, m, "f32")
+    Ks, Vs = to_dev(got["KT"].astype(np.float32)), to_dev(got["VT"].astype(np.float32))
+    p = gsa.Params(B, 1, H, dk, dv, m, io="f32")
+    for t in range(T, T + 3):
+        o = gsa.gsa_decode_step(p, *(to_dev(d[n][:, t]) for n in ("q", "k", "v", "gate")), Ks, Vs)
+        assert rel_err(to_np(o), ref["o"][:, t]) <= 1e-4

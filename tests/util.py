@@ -1,0 +1,65 @@
+"""Helpers shared by the GPU parity tests: moving seeded numpy inputs to the device,
+the error metric, and running the fp64 oracle on the values the GPU saw."""
+import numpy as np
+import torch
+
+import oracle
+
+TOL = {"f32": 1e-4, "bf16": 2e-2}   # max |x - ref| / rms(ref), outputs and gradients
+
+
+def to_dev(x, io=None):
+    """numpy float32 array -> CUDA tensor; io in {"f32","bf16"} picks the element type of
+    q/k/v-like tensors (values are already representable), None keeps float32."""
+    if x is None:
+        return None
+    t = torch.from_numpy(np.ascontiguousarray(x, dtype=np.float32)).cuda()
+    if io == "bf16":
+        t = t.to(torch.bfloat16)
+    return t.contiguous()
+
+
+def to_np(t):
+    return t.detach().to(torch.float32).cpu().numpy().astype(np.float64)
+
+
+def rel_err(x, ref):
+    """max |x - ref| / rms(ref): the normalisation used for every tolerance."""
+    x = np.asarray(x, dtype=np.float64)
+    ref = np.asarray(ref, dtype=np.float64)
+    rms = np.sqrt(np.mean(ref ** 2))
+    if rms == 0:
+        return float(np.abs(x - ref).max())
+    return float(np.abs(x - ref).max() / rms)
+
+
+def rand_inputs(seed, B, T, H, dk, dv, m, io, init=False, final_grads=False, gate="tau8"):
+    r = np.random.default_rng(seed)
+    f = lambda *s: r.standard_normal(s).astype(np.float32)
+    d = dict(q=f(B, T, H, dk) * np.float32(dk ** -0.5), k=f(B, T, H, dk), v=f(B, T, H, dv),
+             dO=f(B, T, H, dv))
+    x = r.standard_normal((B, T, H, m))
+    sig = 1 / (1 + np.exp(-x))
+    if gate == "tau8":
+        a = sig ** 0.125
+    elif gate == "strong":
+        a = 1 / (1 + np.exp(-(x - 3.0)))
+    elif gate == "mixed":        # some slots forget hard, some keep everything, exact 0 and 1
+        a = sig ** 0.125
+        a[..., 0] = 0.0
+        a[..., 1] = 1.0
+        a[..., 2] = 1 / (1 + np.exp(-(x[..., 2] - 4.0)))
+    else:
+        raise ValueError(gate)
+    d["gate"] = a.astype(np.float32)
+    if init:
+        d["K0"] = f(B, H, m, dk) * np.float32(0.3)
+        d["V0"] = f(B, H, m, dv) * np.float32(0.3)
+    if final_grads:
+        d["dKT"] = f(B, H, m, dk) * np.float32(0.3)
+        d["dVT"] = f(B, H, m, dv) * np.float32(0.3)
+    if io == "bf16":
+        import gsa_workloads as W
+        for n in ("q", "k", "v", "dO"):
+            d[n] = W.round_to_bf16(d[n])
+    return d
