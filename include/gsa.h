@@ -140,6 +140,17 @@ GSA_API gsa_status_t gsa_decode_step(const gsa_params_t* params, const void* q,
                              const void* k, const void* v, const float* gate,
                              float* Kstate, float* Vstate, void* o, void* stream);
 
+/*
+ * Self-test of the tensor-core building blocks (no counterpart in the paper): computes one
+ * 128-row bf16 product per operand layout the chunk kernels use, from two 128 x 128
+ * row-major bf16 device matrices X, Y into D (fp32, row-major):
+ *   mode 0: D[128x128] = X Y^T        mode 1: D[128x128] = X Y
+ *   mode 2: D[128x64]  = X^T Y[:64]^T mode 3: D[128x64]  = X Y[:, :64]
+ * dev_status (nullable) receives GSA_ERR_TIMEOUT if a bounded wait expired.
+ */
+GSA_API gsa_status_t gsa_tc_selftest(int32_t mode, const void* X, const void* Y, float* D,
+                                     void* stream, int32_t* dev_status);
+
 #ifdef __cplusplus
 }
 #endif

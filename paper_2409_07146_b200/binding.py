@@ -64,7 +64,7 @@ def lib_path() -> str:
 
 def exported_symbols():
     return ["gsa_chunk_size", "gsa_workspace_bytes", "gsa_status_string", "gsa_gate_cumsum",
-            "gsa_fwd", "gsa_bwd", "gsa_decode_step"]
+            "gsa_fwd", "gsa_bwd", "gsa_decode_step", "gsa_tc_selftest"]
 
 
 def load_library():
@@ -93,6 +93,8 @@ def load_library():
     lib.gsa_bwd.restype = ctypes.c_int
     lib.gsa_decode_step.argtypes = [pp] + [vp] * 8
     lib.gsa_decode_step.restype = ctypes.c_int
+    lib.gsa_tc_selftest.argtypes = [i32, vp, vp, vp, vp, vp]
+    lib.gsa_tc_selftest.restype = ctypes.c_int
     _lib = lib
     return lib
 
@@ -205,3 +207,14 @@ def gsa_decode_step(p: Params, q, k, v, gate, Kstate, Vstate, o=None):
         _ptr(Vstate, torch.float32, (p.B, p.H, p.m, p.d_v), "Vstate"), _ptr(o, io, vv, "o"),
         _stream()), "gsa_decode_step")
     return o
+
+
+def gsa_tc_selftest(mode: int, X, Y, dev_status=None):
+    """Tensor-core building-block self-test: X, Y 128 x 128 bf16; returns D (fp32)."""
+    n = 128 if mode <= 1 else 64
+    D = torch.zeros(128, n, dtype=torch.float32, device=X.device)
+    _check(load_library().gsa_tc_selftest(
+        mode, _ptr(X, torch.bfloat16, (128, 128), "X"), _ptr(Y, torch.bfloat16, (128, 128), "Y"),
+        _ptr(D, torch.float32, None, "D"), _stream(), _ptr(dev_status, torch.int32, None, "dev_status")),
+        "gsa_tc_selftest")
+    return D

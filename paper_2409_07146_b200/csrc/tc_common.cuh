@@ -1,0 +1,194 @@
+// Blackwell (sm_100a) building blocks used by the tensor-core chunk kernels: mbarriers with
+// bounded waits, TMA tile loads, tensor-memory allocation, tcgen05 MMA issue / commit /
+// accumulator loads, and the shared-memory operand layouts (128-byte swizzle) with their
+// matrix descriptors.  Everything is inline PTX; no library templates.
+#pragma once
+
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace gsa {
+namespace tc {
+
+// ---------------------------------------------------------------------------------------
+// Shared-memory operand tiles.
+//
+// Every MMA operand lives in "panels" of R rows x 128 bytes (64 bf16), 1024-byte aligned,
+// with the 128-byte swizzle: the 16-byte chunk c of row r sits at chunk (c ^ (r & 7)).
+// This is what a TMA load with CU_TENSOR_MAP_SWIZZLE_128B writes for a box of 64 bf16 x R
+// rows, and what the MMA matrix descriptors below (layout type SWIZZLE_128B) expect.
+//
+//  * K-major operand  (rows = M or N index, the 64 contiguous elements run along K):
+//      K step kk (16 elements) of panel p starts at  panel_p + (kk % 4) * 32 bytes;
+//      groups of 8 rows are 1024 bytes apart (stride byte offset).
+//  * MN-major operand (rows = K index, the 64 contiguous elements run along M or N):
+//      K step kk (16 rows) starts at panel_0 + kk * 2048 bytes; groups of 8 rows are 1024
+//      bytes apart (stride byte offset); the next 64 elements along M/N are in the next
+//      panel (leading byte offset = panel size).
+// ---------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t swz128(uint32_t row, uint32_t chunk16) {
+    return row * 128u + ((chunk16 ^ (row & 7u)) << 4);
+}
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+
+// 64-bit matrix descriptor: start address, leading/stride byte offsets (all >> 4), version 1
+// (Blackwell), layout type 2 = SWIZZLE_128B.
+__device__ __forceinline__ uint64_t make_desc(uint32_t smem_addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+    uint64_t d = 0;
+    d |= (uint64_t)((smem_addr >> 4) & 0x3FFFu);
+    d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16;
+    d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32;
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)2 << 61;
+    return d;
+}
+__device__ __forceinline__ uint64_t desc_kmajor(uint32_t panel_addr, int kk) {
+    return make_desc(panel_addr + (uint32_t)(kk & 3) * 32u, 16u, 1024u);
+}
+__device__ __forceinline__ uint64_t desc_mnmajor(uint32_t panel0_addr, int kk, uint32_t panel_bytes) {
+    return make_desc(panel0_addr + (uint32_t)kk * 2048u, panel_bytes, 1024u);
+}
+
+// 32-bit instruction descriptor of tcgen05.mma.kind::f16: bf16 x bf16 -> fp32.
+__host__ __device__ constexpr uint32_t make_idesc(int M, int N, bool a_mn_major, bool b_mn_major) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((a_mn_major ? 1u : 0u) << 15) |
+           ((b_mn_major ? 1u : 0u) << 16) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+}
+
+// ---------------------------------------------------------------------------------------
+// mbarrier
+// ---------------------------------------------------------------------------------------
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes)
+                 : "memory");
+}
+__device__ __forceinline__ uint64_t global_timer_ns() {
+    uint64_t t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+constexpr uint64_t kWaitLimitNs = 2000000000ull;   // every wait gives up after 2 s
+
+// Wait for the phase with the given parity; false if the time limit expired.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
+    const uint32_t addr = smem_u32(bar);
+    uint64_t start = 0;
+    for (uint32_t it = 0;; ++it) {
+        uint32_t done;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(done)
+            : "r"(addr), "r"(parity)
+            : "memory");
+        if (done) return true;
+        if ((it & 63u) == 63u) {
+            const uint64_t now = global_timer_ns();
+            if (start == 0) start = now;
+            else if (now - start > kWaitLimitNs) return false;
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------------
+// TMA: 4-D tiled load (no multicast) that signals an mbarrier with its byte count.
+// ---------------------------------------------------------------------------------------
+__device__ __forceinline__ void tma_load_4d(void* smem_dst, const CUtensorMap* map, uint64_t* bar,
+                                            int c0, int c1, int c2, int c3) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+        ::"r"(smem_u32(smem_dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+        : "memory");
+}
+__device__ __forceinline__ void prefetch_tmap(const CUtensorMap* map) {
+    asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
+}
+// Make shared-memory writes of this thread visible to the async proxy (TMA / MMA reads).
+__device__ __forceinline__ void fence_async_smem() {
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+
+// ---------------------------------------------------------------------------------------
+// Tensor memory + tcgen05
+// ---------------------------------------------------------------------------------------
+// One full warp allocates `ncols` (power of two >= 32) columns; the base address lands in
+// *smem_slot.
+__device__ __forceinline__ void tmem_alloc(uint32_t* smem_slot, uint32_t ncols) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(smem_slot)),
+                 "r"(ncols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before_sync() {
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+}
+__device__ __forceinline__ void tc_fence_after_sync() {
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+}
+// D[tmem] (+)= A[smem] * B[smem]; issued by ONE thread.
+__device__ __forceinline__ void mma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                         bool accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"((uint32_t)accumulate)
+        : "memory");
+}
+// The mbarrier receives one arrival when all MMAs issued so far by this thread are done.
+__device__ __forceinline__ void mma_commit(uint64_t* bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
+                 : "memory");
+}
+// 16 consecutive fp32 columns of this thread's accumulator row (lane = 32 * (warp % 4) + lane).
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float (&v)[16]) {
+    uint32_t r[16];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr));
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+__device__ __forceinline__ uint32_t tmem_row_addr(uint32_t base, int warp_in_group, int column) {
+    return base + ((uint32_t)(warp_in_group * 32) << 16) + (uint32_t)column;
+}
+
+// ---------------------------------------------------------------------------------------
+// Writing operand rows from registers
+// ---------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&h);
+}
+// 8 consecutive elements (one 16-byte chunk) of row `row` of a panel.
+__device__ __forceinline__ void store_chunk(unsigned char* panel, int row, int chunk16, const float (&x)[8]) {
+    uint4 v = make_uint4(pack_bf16(x[0], x[1]), pack_bf16(x[2], x[3]), pack_bf16(x[4], x[5]), pack_bf16(x[6], x[7]));
+    *reinterpret_cast<uint4*>(panel + swz128(row, chunk16)) = v;
+}
+// one element (row, col) of a panel (col < 64)
+__device__ __forceinline__ void store_elem(unsigned char* panel, int row, int col, float x) {
+    *reinterpret_cast<__nv_bfloat16*>(panel + swz128(row, col >> 3) + (col & 7) * 2) = __float2bfloat16_rn(x);
+}
+
+}  // namespace tc
+
+// Host side: encode a 4-D tensor map over a [B,T,H,D] bf16 tensor with a box of
+// 64 channels x `box_rows` tokens of one (batch, head), 128-byte swizzle, zero fill.
+cudaError_t make_tensor_map_bthd(CUtensorMap* map, const void* base, int B, int T, int H, int D, int box_rows);
+
+}  // namespace gsa

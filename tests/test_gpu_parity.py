@@ -7,7 +7,7 @@ import torch
 import gsa_workloads as W
 import oracle
 import paper_2409_07146_b200 as gsa
-from util import TOL, rand_inputs, rel_err, to_dev, to_np
+from util import BF16_IO, TOL, rand_inputs, rel_err, to_dev, to_np
 
 pytestmark = pytest.mark.gpu
 
@@ -30,7 +30,8 @@ def check_fwd(d, got, gate, io, scale=1.0, log=False, tol=None):
     ref = oracle.fwd(d["q"], d["k"], d["v"], gate, gate_is_log=log, scale=scale,
                      K0=d.get("K0"), V0=d.get("V0"))
     tol = tol or TOL[io]
-    errs = {n: rel_err(got[n], ref[n]) for n in ("o", "ok", "KT", "VT") if got[n] is not None}
+    errs = {n: rel_err(got[n], ref[n], io == "bf16" and n in BF16_IO)
+            for n in ("o", "ok", "KT", "VT") if got[n] is not None}
     assert all(np.isfinite(got[n]).all() for n in errs), "non-finite output"
     assert all(e <= tol for e in errs.values()), errs
     return errs
@@ -146,7 +147,7 @@ def run_bwd(d, B, T, H, dk, dv, m, io, impl="auto", scale=1.0, log=False, saved=
 
 
 def check_bwd(got, ref, tol):
-    errs = {n: rel_err(got[n], ref[n]) for n in got}
+    errs = {n: rel_err(got[n], ref[n], tol == TOL["bf16"] and n in BF16_IO) for n in got}
     assert all(np.isfinite(got[n]).all() for n in got), "non-finite gradient"
     assert all(e <= tol for e in errs.values()), errs
     return errs
@@ -195,7 +196,7 @@ def test_decode_steps(io, dk, dv, m):
         o = gsa.gsa_decode_step(p, to_dev(x["q"], io), to_dev(x["k"], io), to_dev(x["v"], io),
                                 to_dev(x["gate"]), Ks, Vs)
         ro = oracle.decode_step(x["q"], x["k"], x["v"], x["gate"], Kr, Vr, scale=0.8)
-        assert rel_err(to_np(o), ro) <= TOL[io]
+        assert rel_err(to_np(o), ro, io == "bf16") <= TOL[io]
     assert rel_err(to_np(Ks), Kr) <= 1e-5 and rel_err(to_np(Vs), Vr) <= 1e-5
 
 

@@ -23,14 +23,25 @@ def to_np(t):
     return t.detach().to(torch.float32).cpu().numpy().astype(np.float64)
 
 
-def rel_err(x, ref):
-    """max |x - ref| / rms(ref): the normalisation used for every tolerance."""
+BF16_IO = {"o", "dq", "dk", "dv"}   # tensors stored in the io type (bf16 when io == "bf16")
+
+
+def rel_err(x, ref, stored_bf16=False):
+    """max |x - ref| / rms(ref): the normalisation used for every tolerance.
+
+    For a tensor that the library stores as bfloat16, the half-ulp rounding of the result
+    itself (2^-9 |ref| per element) is taken off first: with heavy-tailed gradients
+    max|ref| / rms reaches 15-20, and the output format alone would then exceed the 2e-2
+    bound however exact the arithmetic."""
     x = np.asarray(x, dtype=np.float64)
     ref = np.asarray(ref, dtype=np.float64)
+    diff = np.abs(x - ref)
+    if stored_bf16:
+        diff = np.maximum(diff - 2.0 ** -9 * np.abs(ref), 0.0)
     rms = np.sqrt(np.mean(ref ** 2))
     if rms == 0:
-        return float(np.abs(x - ref).max())
-    return float(np.abs(x - ref).max() / rms)
+        return float(diff.max())
+    return float(diff.max() / rms)
 
 
 def rand_inputs(seed, B, T, H, dk, dv, m, io, init=False, final_grads=False, gate="tau8"):
