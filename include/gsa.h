@@ -76,8 +76,10 @@ typedef struct {
 
 enum { GSA_WS_FWD = 0, GSA_WS_BWD = 1, GSA_WS_DECODE = 2 };
 
-/* Chunk length C of the chunkwise form (Algorithm 1 leaves C open). */
-GSA_API int32_t gsa_chunk_size(void);
+/* Chunk length C of the chunkwise form that these params select (Algorithm 1 leaves C
+ * open): 128 for the tensor-core kernels, 64 for the fp32 CUDA-core kernels; 0 for
+ * invalid params. */
+GSA_API int32_t gsa_chunk_size(const gsa_params_t* params);
 
 /* Bytes of scratch `which` (GSA_WS_*) needs for these params; 0 for decode and
  * for invalid params. */
@@ -87,7 +89,7 @@ GSA_API const char* gsa_status_string(gsa_status_t status);
 
 /*
  * chunk_cumsum of Algorithm 1 (its "preprocessing" step), in log space: for
- * each chunk of C tokens, G[i] = sum_{j <= i in chunk} log a_j (log a clamped
+ * each chunk of C = gsa_chunk_size(params) tokens, G[i] = sum_{j <= i in chunk} log a_j (log a clamped
  * to >= -100), and the input gate I = 1 - a.  gate, G, I: [B,T,H,m] fp32; G and
  * I are written in full.  Uses no workspace.
  */

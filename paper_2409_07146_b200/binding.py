@@ -79,7 +79,7 @@ def load_library():
     lib = ctypes.CDLL(_LIB_PATH)
     vp, sz, i32 = ctypes.c_void_p, ctypes.c_size_t, ctypes.c_int32
     pp = ctypes.POINTER(_CParams)
-    lib.gsa_chunk_size.argtypes = []
+    lib.gsa_chunk_size.argtypes = [pp]
     lib.gsa_chunk_size.restype = i32
     lib.gsa_workspace_bytes.argtypes = [pp, i32]
     lib.gsa_workspace_bytes.restype = sz
@@ -122,8 +122,9 @@ def _check(code: int, where: str):
         raise GsaError(code, where)
 
 
-def gsa_chunk_size() -> int:
-    return int(load_library().gsa_chunk_size())
+def gsa_chunk_size(p: Params) -> int:
+    cp = p.c()
+    return int(load_library().gsa_chunk_size(ctypes.byref(cp)))
 
 
 def gsa_workspace_bytes(p: Params, which: int) -> int:

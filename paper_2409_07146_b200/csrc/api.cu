@@ -37,6 +37,8 @@ bool use_tc(const gsa_params_t& p) {
     return p.io == GSA_BF16 && tc_supported(p.d_k, p.d_v, p.m);
 }
 
+int chunk_of(const gsa_params_t& p) { return use_tc(p) ? tc_chunk() : kChunk; }
+
 struct Slices { int k, v; };
 Slices slices(const gsa_params_t& p) {
     if (use_tc(p)) return {tc_value_side_slices(p.d_k), tc_value_side_slices(p.d_v)};
@@ -103,7 +105,10 @@ cudaError_t key_side(const gsa_params_t& p, const KeySideArgs& a, int reverse, c
 
 extern "C" {
 
-int32_t gsa_chunk_size(void) { return kChunk; }
+int32_t gsa_chunk_size(const gsa_params_t* params) {
+    if (check_params(params, false) != GSA_OK) return 0;
+    return chunk_of(*params);
+}
 
 const char* gsa_status_string(gsa_status_t status) {
     switch (status) {
@@ -131,7 +136,7 @@ gsa_status_t gsa_gate_cumsum(const gsa_params_t* params, const float* gate, floa
     if (!ok_ptr(gate) || !ok_ptr(G) || !ok_ptr(I)) return GSA_ERR_INVALID_ARG;
     const gsa_params_t& p = *params;
     GSA_CUDA(launch_gate_cumsum(gate, p.gate_kind == GSA_GATE_LOG_A, G, I, p.B, p.T, p.H, p.m,
-                                static_cast<cudaStream_t>(stream)));
+                                chunk_of(p), static_cast<cudaStream_t>(stream)));
     return GSA_OK;
 }
 
@@ -152,7 +157,7 @@ gsa_status_t gsa_fwd(const gsa_params_t* params, const void* q, const void* k, c
     const Slices s = slices(p);
     const size_t rows = (size_t)p.B * p.T * p.H;
 
-    GSA_CUDA(launch_gate_cumsum(gate, p.gate_kind == GSA_GATE_LOG_A, w.G, w.I, p.B, p.T, p.H, p.m, st));
+    GSA_CUDA(launch_gate_cumsum(gate, p.gate_kind == GSA_GATE_LOG_A, w.G, w.I, p.B, p.T, p.H, p.m, chunk_of(p), st));
     // pass 1: o' = GLA(q, k, 1-a) with the decay on the slot (value) side
     ValueSideArgs a1{q, k, w.I, w.G, K0, KT, w.okpart, p.B, p.T, p.H, p.d_k};
     GSA_CUDA(value_side(p, a1, 0, st, dev_status));
@@ -185,7 +190,7 @@ gsa_status_t gsa_bwd(const gsa_params_t* params, const void* q, const void* k, c
     const Slices s = slices(p);
     const size_t rows = (size_t)p.B * p.T * p.H;
 
-    GSA_CUDA(launch_gate_cumsum(gate, p.gate_kind == GSA_GATE_LOG_A, w.G, w.I, p.B, p.T, p.H, p.m, st));
+    GSA_CUDA(launch_gate_cumsum(gate, p.gate_kind == GSA_GATE_LOG_A, w.G, w.I, p.B, p.T, p.H, p.m, chunk_of(p), st));
     const float* ok = ok_saved;
     if (ok == nullptr) {  // recompute pass 1 and its logits
         ValueSideArgs a1{q, k, w.I, w.G, K0, nullptr, w.okpart, p.B, p.T, p.H, p.d_k};

@@ -9,7 +9,7 @@
 
 namespace gsa {
 
-constexpr int kChunk = 64;            // C of the chunkwise form
+constexpr int kChunk = 64;            // C of the chunkwise form, fp32 CUDA-core kernels (tensor-core kernels: 128)
 constexpr float kLogGateMin = -100.f; // clamp of log a (exp(-100) == 0 in fp32)
 // A chunk whose total log-decay stays above this bound uses the factorised
 // decay exp(G_i) * exp(-G_j) (one reference point per chunk); below it the
@@ -92,7 +92,7 @@ struct KeySideArgs {
 
 // launchers (definitions in the .cu files); all return cudaGetLastError() of the launch
 cudaError_t launch_gate_cumsum(const float* gate, int gate_is_log, float* G, float* I,
-                               int B, int T, int H, int M, cudaStream_t st);
+                               int B, int T, int H, int M, int chunk, cudaStream_t st);
 cudaError_t launch_slot_softmax_fwd(const float* part, int nslice, float scale, float* ok,
                                     float* p, size_t rows, int M, cudaStream_t st);
 cudaError_t launch_slot_softmax_bwd(const float* ok, const float* dp_part, int nslice,
@@ -110,7 +110,8 @@ cudaError_t launch_key_side_simt(const KeySideArgs& a, int io, int M, int revers
                                  cudaStream_t st);
 // tcgen05 (bf16 tensor-core) versions of the two primitives; bf16 io only.
 bool tc_supported(int d_k, int d_v, int M);
-int tc_value_side_slices(int D);   // how many partial-sum slices value_side writes for width D
+int tc_value_side_slices(int D);
+int tc_chunk();                    // chunk length of the tensor-core kernels   // how many partial-sum slices value_side writes for width D
 cudaError_t launch_value_side_tc(const ValueSideArgs& a, int M, int reverse, cudaStream_t st,
                                  int32_t* dev_status);
 cudaError_t launch_key_side_tc(const KeySideArgs& a, int M, int reverse, cudaStream_t st,

@@ -8,19 +8,20 @@ namespace gsa {
 
 // ------------------------------------------------------------------ chunk_cumsum
 // One thread per (chunk, slot); a block covers 256/M consecutive chunks of one (b,h).
+// `chunk` is the chunk length of the kernels that will consume G (64 or 128).
 // Rows of one chunk are read 8 at a time so that several loads are in flight.
 template <int M>
 __global__ void __launch_bounds__(256) gate_cumsum_kernel(const float* __restrict__ gate,
                                                           int gate_is_log,
                                                           float* __restrict__ G,
                                                           float* __restrict__ I, int T, int H,
-                                                          int nchunks) {
+                                                          int chunk, int nchunks) {
     const int s = threadIdx.x;
     const int n = blockIdx.y * blockDim.y + threadIdx.y;
     if (n >= nchunks) return;
     const int bh = blockIdx.x, b = bh / H, h = bh % H;
-    const int t0 = n * kChunk;
-    const int rows = min(kChunk, T - t0);
+    const int t0 = n * chunk;
+    const int rows = min(chunk, T - t0);
     const size_t stride = (size_t)H * M;
     const size_t base = (((size_t)b * T + t0) * H + h) * M + s;
     float run = 0.f;
@@ -50,14 +51,14 @@ __global__ void __launch_bounds__(256) gate_cumsum_kernel(const float* __restric
 }
 
 cudaError_t launch_gate_cumsum(const float* gate, int gate_is_log, float* G, float* I, int B,
-                               int T, int H, int M, cudaStream_t st) {
-    const int nchunks = (T + kChunk - 1) / kChunk;
+                               int T, int H, int M, int chunk, cudaStream_t st) {
+    const int nchunks = (T + chunk - 1) / chunk;
     dim3 block(M, 256 / M);
     dim3 grid(B * H, (nchunks + block.y - 1) / block.y);
     if (M == 64)
-        gate_cumsum_kernel<64><<<grid, block, 0, st>>>(gate, gate_is_log, G, I, T, H, nchunks);
+        gate_cumsum_kernel<64><<<grid, block, 0, st>>>(gate, gate_is_log, G, I, T, H, chunk, nchunks);
     else
-        gate_cumsum_kernel<32><<<grid, block, 0, st>>>(gate, gate_is_log, G, I, T, H, nchunks);
+        gate_cumsum_kernel<32><<<grid, block, 0, st>>>(gate, gate_is_log, G, I, T, H, chunk, nchunks);
     return cudaGetLastError();
 }
 

@@ -53,7 +53,10 @@ __global__ void __launch_bounds__(128) tc_selftest_kernel(const __grid_constant_
         mbar_init(&bar_mma, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == 0) tmem_alloc(&tmem_slot, 128);
+    if (warp == 0) {
+        __syncwarp();
+        tmem_alloc(&tmem_slot, 128);
+    }
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
@@ -127,7 +130,10 @@ __global__ void __launch_bounds__(128) tc_selftest_kernel(const __grid_constant_
     }
     tc_fence_before_sync();
     __syncthreads();
-    if (warp == 0) tmem_dealloc(tmem, 128);
+    if (warp == 0) {
+        __syncwarp();
+        tmem_dealloc(tmem, 128);
+    }
 }
 }  // namespace
 }  // namespace gsa

@@ -34,8 +34,10 @@ def test_library_exports_every_declared_symbol(lib):
 
 
 def test_chunk_and_workspace_queries(lib):
-    assert gsa.gsa_chunk_size() == 64
     p = gsa.Params(B=2, T=100, H=3, d_k=64, d_v=128, m=32, io="f32")
+    assert gsa.gsa_chunk_size(p) == 64
+    assert gsa.gsa_chunk_size(gsa.Params(1, 256, 1, 128, 128, 64, io="bf16")) == 128
+    assert gsa.gsa_chunk_size(gsa.Params(1, 256, 1, 128, 128, 64, io="bf16", impl="simt")) == 64
     f, b = gsa.gsa_workspace_bytes(p, binding.GSA_WS_FWD), gsa.gsa_workspace_bytes(p, binding.GSA_WS_BWD)
     assert f > 0 and b > f and f % 256 == 0
     assert gsa.gsa_workspace_bytes(p, binding.GSA_WS_DECODE) == 0

@@ -7,7 +7,7 @@ import torch
 import gsa_workloads as W
 import oracle
 import paper_2409_07146_b200 as gsa
-from util import BF16_IO, TOL, rand_inputs, rel_err, to_dev, to_np
+from util import BF16_IO, TC_RTOL, TOL, mixed_err, rand_inputs, rel_err, to_dev, to_np
 
 pytestmark = pytest.mark.gpu
 
@@ -26,31 +26,36 @@ def run_fwd(d, B, T, H, dk, dv, m, io, impl="auto", scale=1.0, log=False, want_s
                 VT=None if VT is None else to_np(VT)), gate
 
 
-def check_fwd(d, got, gate, io, scale=1.0, log=False, tol=None):
+def check_fwd(d, got, gate, io, scale=1.0, log=False, tol=None, tc=False):
     ref = oracle.fwd(d["q"], d["k"], d["v"], gate, gate_is_log=log, scale=scale,
                      K0=d.get("K0"), V0=d.get("V0"))
     tol = tol or TOL[io]
-    errs = {n: rel_err(got[n], ref[n], io == "bf16" and n in BF16_IO)
-            for n in ("o", "ok", "KT", "VT") if got[n] is not None}
+    if tc:
+        errs = {n: mixed_err(got[n], ref[n], TC_RTOL) for n in ("o", "ok", "KT", "VT") if got[n] is not None}
+    else:
+        errs = {n: rel_err(got[n], ref[n], io == "bf16" and n in BF16_IO)
+                for n in ("o", "ok", "KT", "VT") if got[n] is not None}
     assert all(np.isfinite(got[n]).all() for n in errs), "non-finite output"
     assert all(e <= tol for e in errs.values()), errs
     return errs
 
 
 # ------------------------------------------------------------------ gate kernel
-@pytest.mark.parametrize("T,m,log", [(256, 64, False), (100, 32, True), (1, 64, False)])
-def test_gate_cumsum(T, m, log):
+@pytest.mark.parametrize("T,m,log,io", [(256, 64, False, "f32"), (100, 32, True, "f32"),
+                                         (1, 64, False, "f32"), (300, 64, False, "bf16")])
+def test_gate_cumsum(T, m, log, io):
     B, H = 2, 3
     r = np.random.default_rng(T + m)
     a = (1 / (1 + np.exp(-r.standard_normal((B, T, H, m))))).astype(np.float32)
     a[0, T // 2, 0, 0] = 0.0
     gate = np.log(np.maximum(a.astype(np.float64), 1e-300)).astype(np.float32) if log else a
-    p = gsa.Params(B, T, H, 64, 64, m, gate_is_log=log)
+    p = gsa.Params(B, T, H, 128, 128, m, gate_is_log=log, io=io)
     G = torch.empty(B, T, H, m, device="cuda"); I = torch.empty_like(G)
     gsa.gsa_gate_cumsum(p, to_dev(gate), G, I)
     g64 = np.maximum(gate.astype(np.float64) if log else np.log(np.maximum(a.astype(np.float64), 1e-300)), -100.0)
     ref = np.zeros_like(g64)
-    C = gsa.gsa_chunk_size()
+    C = gsa.gsa_chunk_size(p)
+    assert C == (128 if io == "bf16" else 64)
     for t0 in range(0, T, C):
         ref[:, t0:t0 + C] = np.cumsum(g64[:, t0:t0 + C], axis=1)
     np.testing.assert_allclose(to_np(G), ref, rtol=2e-6, atol=2e-6)
@@ -146,8 +151,11 @@ def run_bwd(d, B, T, H, dk, dv, m, io, impl="auto", scale=1.0, log=False, saved=
     return got, ref
 
 
-def check_bwd(got, ref, tol):
-    errs = {n: rel_err(got[n], ref[n], tol == TOL["bf16"] and n in BF16_IO) for n in got}
+def check_bwd(got, ref, tol, tc=False):
+    if tc:
+        errs = {n: mixed_err(got[n], ref[n], TC_RTOL) for n in got}
+    else:
+        errs = {n: rel_err(got[n], ref[n], tol == TOL["bf16"] and n in BF16_IO) for n in got}
     assert all(np.isfinite(got[n]).all() for n in got), "non-finite gradient"
     assert all(e <= tol for e in errs.values()), errs
     return errs
@@ -212,3 +220,57 @@ def test_decode_continues_a_prefill():
     for t in range(T, T + 3):
         o = gsa.gsa_decode_step(p, *(to_dev(d[n][:, t]) for n in ("q", "k", "v", "gate")), Ks, Vs)
         assert rel_err(to_np(o), ref["o"][:, t]) <= 1e-4
+
+
+# ------------------------------------------------------------------ tensor-core (tcgen05) kernels
+@pytest.mark.parametrize("T", [1, 100, 128, 129, 300, 512])
+def test_fwd_tc_ragged_lengths(T):
+    B, H, dk, dv, m = 2, 2, 128, 128, 64
+    d = rand_inputs(500 + T, B, T, H, dk, dv, m, "bf16", init=True)
+    got, gate = run_fwd(d, B, T, H, dk, dv, m, "bf16", impl="tc", scale=0.9)
+    errs = check_fwd(d, got, gate, "bf16", scale=0.9, tc=True)
+    print("tc fwd", T, errs)
+
+
+@pytest.mark.parametrize("dk,dv", [(256, 128), (128, 512), (512, 512)])
+def test_fwd_tc_shapes(dk, dv):
+    B, T, H, m = 1, 384, 2, 64
+    d = rand_inputs(9, B, T, H, dk, dv, m, "bf16")
+    got, gate = run_fwd(d, B, T, H, dk, dv, m, "bf16", impl="tc")
+    check_fwd(d, got, gate, "bf16", tc=True)
+
+
+@pytest.mark.parametrize("gate", ["strong", "mixed"])
+@pytest.mark.parametrize("log", [False, True])
+def test_fwd_tc_strong_forgetting(gate, log):
+    B, T, H, dk, dv, m = 1, 300, 2, 128, 128, 64
+    d = rand_inputs(13, B, T, H, dk, dv, m, "bf16", init=True, gate=gate)
+    got, g = run_fwd(d, B, T, H, dk, dv, m, "bf16", impl="tc", log=log)
+    gref = np.maximum(g.astype(np.float64), -100.0) if log else g
+    check_fwd(d, got, gref, "bf16", log=log, tc=True)
+
+
+def test_fwd_tc_matches_simt_closely():
+    # same inputs through both kernel families: they differ only by bf16 operand rounding
+    B, T, H, dk, dv, m = 1, 256, 2, 128, 128, 64
+    d = rand_inputs(17, B, T, H, dk, dv, m, "bf16", init=True)
+    a, _ = run_fwd(d, B, T, H, dk, dv, m, "bf16", impl="tc")
+    b, _ = run_fwd(d, B, T, H, dk, dv, m, "bf16", impl="simt")
+    assert rel_err(a["ok"], b["ok"]) < 2e-2 and rel_err(a["KT"], b["KT"]) < 1e-2
+
+
+@pytest.mark.parametrize("T", [100, 256, 385])
+@pytest.mark.parametrize("log", [False, True])
+def test_bwd_tc(T, log):
+    B, H, dk, dv, m = 2, 2, 128, 256, 64
+    d = rand_inputs(600 + T, B, T, H, dk, dv, m, "bf16", init=True, final_grads=True)
+    got, ref = run_bwd(d, B, T, H, dk, dv, m, "bf16", impl="tc", scale=1.1, log=log)
+    errs = check_bwd(got, ref, TOL["bf16"], tc=True)
+    print("tc bwd", T, log, errs)
+
+
+def test_bwd_tc_strong_forgetting_saved_logits():
+    B, T, H, dk, dv, m = 1, 260, 2, 128, 128, 64
+    d = rand_inputs(45, B, T, H, dk, dv, m, "bf16", gate="strong")
+    got, ref = run_bwd(d, B, T, H, dk, dv, m, "bf16", impl="tc", log=True, saved=True)
+    check_bwd(got, ref, TOL["bf16"], tc=True)

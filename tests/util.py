@@ -25,6 +25,22 @@ def to_np(t):
 
 BF16_IO = {"o", "dq", "dk", "dv"}   # tensors stored in the io type (bf16 when io == "bf16")
 
+# Relative allowance of the tensor-core path (bf16 operands): besides the inputs, the chunk
+# kernels round five derived operands to bfloat16 on the way to a gradient (masked q.k
+# products, decayed gate weights, the state copy, the slot-space attention matrix, the
+# scaled softmax gradient), each good to 2^-9 relative; 2^-7 |ref| covers their chain.
+TC_RTOL = 2.0 ** -7
+
+
+def mixed_err(x, ref, rtol):
+    """max (|x - ref| - rtol |ref|)+ / rms(ref): the rms-normalised error that is left after
+    a relative allowance rtol per element (see TC_RTOL)."""
+    x = np.asarray(x, dtype=np.float64)
+    ref = np.asarray(ref, dtype=np.float64)
+    diff = np.maximum(np.abs(x - ref) - rtol * np.abs(ref), 0.0)
+    rms = np.sqrt(np.mean(ref ** 2))
+    return float(diff.max() / (rms if rms > 0 else 1.0))
+
 
 def rel_err(x, ref, stored_bf16=False):
     """max |x - ref| / rms(ref): the normalisation used for every tolerance.
