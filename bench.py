@@ -1,0 +1,410 @@
+#!/usr/bin/env python
+"""Benchmark of the GSA layer hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+A step is one pass of the whole training hot path over one batch of the 1.3B-model layer
+shape (B=8, H=4, T=2048, d_k=d_v=512, m=64, bf16): gsa_fwd (gate cumsum, pass 1, slot
+softmax, pass 2, logits saved) followed by gsa_bwd (all gradients).  One JSON line is
+printed by rank 0.  With N > 1 (torchrun) every rank runs its own batch (weak scaling, no
+data-path collective: (batch, head) pairs are independent recurrences).
+
+--impl reference times the fp64 CPU oracle on the host cores on a bounded sample of the
+same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import gsa_workloads as W  # noqa: E402
+
+METRIC = "GSA layer fwd+bwd tokens/s (bf16, T=2048, m=64)"
+UNIT = "tokens/s"
+WORKLOAD = "train_1p3b"
+
+
+def peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        d = json.load(open(path))
+        return dict(hbm_gbs=float(d["hbm_gbs"]), source="measured (MEASURED_PEAKS.json)")
+    return dict(hbm_gbs=6650.0, source="fallback (profiling recipe)")
+
+
+# ----------------------------------------------------------------------------- byte model
+def step_algorithmic_bytes(w: W.Workload) -> int:
+    """Bytes one fwd+bwd step must move if every tensor crossed HBM exactly once: forward
+    reads q,k,v,gate and writes o and the saved logits; backward reads q,k,v,dO,gate and the
+    saved logits and writes dq,dk,dv,dgate."""
+    e = 2 if w.io == "bf16" else 4
+    R = w.B * w.T * w.H
+    fwd = e * (2 * w.d_k + 2 * w.d_v) + 4 * w.m + 4 * w.m
+    bwd = e * (2 * w.d_k + 2 * w.d_v) + e * (2 * w.d_k + w.d_v) + 4 * w.m * 3
+    return R * (fwd + bwd)
+
+
+def kernel_algorithmic_bytes(label: str, w: W.Workload) -> int:
+    """Inputs read once plus outputs written once, per launch of each kernel."""
+    e = 2 if w.io == "bf16" else 4
+    R = w.B * w.T * w.H
+    m = w.m
+    nsk, nsv = w.d_k // 128, w.d_v // 128
+    table = {
+        "gate_cumsum": 12 * m,
+        "pass1_value_side": 2 * w.d_k * e + 8 * m + 4 * m * nsk,
+        "slot_softmax": 4 * m * nsk + 8 * m,
+        "pass2_key_side": 12 * m + 2 * w.d_v * e,
+        "bwd_dp_value_side": 2 * w.d_v * e + 8 * m + 4 * m * nsv,
+        "slot_softmax_bwd": 4 * m * (1 + nsv) + 12 * m,
+        "bwd_dq_key_side": 12 * m + 2 * w.d_k * e,
+        "bwd_dv_key_side_rev": 12 * m + 2 * w.d_v * e,
+        "bwd_dIv_value_side_rev": 2 * w.d_v * e + 8 * m + 4 * m * nsv,
+        "bwd_dk_key_side_rev": 12 * m + 2 * w.d_k * e,
+        "bwd_dIk_value_side_rev": 2 * w.d_k * e + 8 * m + 4 * m * nsk,
+        "gate_grad": 2 * (8 * m + 4 * m * (nsk + nsv)) + 4 * m + 4 * m,
+    }
+    return R * table[label]
+
+
+def step_flops(w: W.Workload) -> float:
+    """Chunkwise forward flops per token-head at C = 128 (causal half counted),
+    F = 4m(dk+dv) + C(dk+dv) + 2Cm, and 3.5x that for forward + backward."""
+    C = 128
+    f = 4 * w.m * (w.d_k + w.d_v) + C * (w.d_k + w.d_v) + 2 * C * w.m
+    return 3.5 * f * w.B * w.T * w.H
+
+
+# ----------------------------------------------------------------------------- clocks
+class ClockSampler:
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.idx = gpu_index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.idx}", f"--query-gpu={self.QUERY}",
+                 "--format=csv,noheader,nounits", "-lms", "200"],
+                stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self) -> dict:
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        try:
+            for line in open(self.path):
+                f = [x.strip() for x in line.split(",")]
+                if len(f) < 9:
+                    continue
+                try:
+                    sm.append(float(f[1])); mx.append(float(f[2]))
+                except ValueError:
+                    continue
+                for n, v in zip(names, f[5:9]):
+                    if v.lower() == "active":
+                        reasons.add(n)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if sm:
+            out.update(sm_mhz=float(np.median(sm)), sm_max_mhz=float(max(mx)), samples=len(sm))
+        out["reasons"] = sorted(reasons)
+        return out
+
+
+# ----------------------------------------------------------------------------- reference arm
+def oracle_step(x, w, pairs, threads):
+    import oracle
+    rng = (0, pairs)
+    oracle.fwd(x["q"], x["k"], x["v"], x["gate"], bh_range=rng, threads=threads)
+    oracle.bwd(x["q"], x["k"], x["v"], x["gate"], x["dO"], bh_range=rng, threads=threads)
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    oracle.build()
+    w = W.CONFIGS[WORKLOAD]
+    x = W.make_inputs(w)
+    threads = min(oracle.default_threads(), 16, w.B * w.H)
+    pairs = threads
+    for _ in range(args.warmup):
+        oracle_step(x, w, pairs, threads)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle_step(x, w, pairs, threads)
+    dt = (time.perf_counter() - t0) / args.steps
+    tokens = pairs * w.T / w.H          # a token counts once all H heads are done
+    val = tokens / dt
+    sample = (f"{pairs} of {w.B * w.H} (batch, head) pairs of the {WORKLOAD} workload per step, "
+              f"forward + reverse sweep in fp64; tokens = pairs * T / H")
+    line = {
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic (seeded, bf16-rounded inputs)",
+        "config": {"workload": WORKLOAD, "B": w.B, "T": w.T, "H": w.H, "d_k": w.d_k, "d_v": w.d_v,
+                   "m": w.m, "sample": sample},
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ----------------------------------------------------------------------------- our arm
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    import __graft_entry__ as entry
+    entry.build()
+    import paper_2409_07146_b200 as gsa
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the GSA library has no CPU path")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    dev = torch.device("cuda", local)
+
+    w = W.CONFIGS[WORKLOAD].scaled(seed=W.CONFIGS[WORKLOAD].seed + 1000 * rank)
+    x = W.make_inputs(w)
+    p = gsa.Params(w.B, w.T, w.H, w.d_k, w.d_v, w.m, io=w.io)
+
+    def host(a, bf16):
+        t = torch.from_numpy(np.ascontiguousarray(a))
+        if bf16:
+            t = t.to(torch.bfloat16)
+        return t.pin_memory()
+
+    h_in = {n: host(x[n], n != "gate") for n in ("q", "k", "v", "gate", "dO")}
+    d_in = {n: t.to(dev) for n, t in h_in.items()}
+    io = torch.bfloat16
+    o = torch.empty(w.B, w.T, w.H, w.d_v, dtype=io, device=dev)
+    ok = torch.empty(w.B, w.T, w.H, w.m, dtype=torch.float32, device=dev)
+    dq = torch.empty(w.B, w.T, w.H, w.d_k, dtype=io, device=dev)
+    dk = torch.empty_like(dq)
+    dv = torch.empty_like(o)
+    dg = torch.empty_like(ok)
+    ws_f = torch.empty(gsa.gsa_workspace_bytes(p, 0), dtype=torch.uint8, device=dev)
+    ws_b = torch.empty(gsa.gsa_workspace_bytes(p, 1), dtype=torch.uint8, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    h_out = {n: torch.empty(t.shape, dtype=t.dtype).pin_memory()
+             for n, t in (("o", o), ("dq", dq), ("dk", dk), ("dv", dv), ("dgate", dg))}
+
+    def step(src):
+        gsa.gsa_fwd(p, src["q"], src["k"], src["v"], src["gate"], o=o, ok_save=ok, ws=ws_f,
+                    dev_status=status)
+        gsa.gsa_bwd(p, src["q"], src["k"], src["v"], src["gate"], src["dO"], ok_saved=ok, dq=dq,
+                    dk=dk, dv=dv, dgate=dg, ws=ws_b, dev_status=status)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(fn, steps):
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(steps):
+            fn()
+        e1.record()
+        barrier()
+        ms = torch.tensor([e0.elapsed_time(e1)], device=dev)
+        if world > 1:
+            dist.all_reduce(ms, op=dist.ReduceOp.MAX)
+        return float(ms.item())
+
+    for _ in range(max(args.warmup, 3)):
+        step(d_in)
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    total_ms = timed(lambda: step(d_in), args.steps)
+    clocks = sampler.stop() if rank == 0 else {}
+    ms_step = total_ms / args.steps
+    value = world * w.tokens / (ms_step * 1e-3)
+    if int(status.item()) != 0:
+        raise SystemExit("a bounded device-side wait expired during the benchmark")
+    if not bool(torch.isfinite(dq.float()).all()):
+        raise SystemExit("non-finite gradients")
+
+    # ---- end to end: host buffers in, host buffers out, copies inside the timed region
+    def e2e_step():
+        for n in h_in:
+            d_in[n].copy_(h_in[n], non_blocking=True)
+        step(d_in)
+        for n, t in (("o", o), ("dq", dq), ("dk", dk), ("dv", dv), ("dgate", dg)):
+            h_out[n].copy_(t, non_blocking=True)
+
+    e2e_step()
+    e2e_steps = max(3, args.steps // 4)
+    e2e_ms = timed(e2e_step, e2e_steps) / e2e_steps
+    h2d = sum(t.numel() * t.element_size() for t in h_in.values())
+    d2h = sum(t.numel() * t.element_size() for t in h_out.values())
+
+    line = None
+    if rank == 0:
+        # ---- per-kernel durations (a second pass over the same steps, kernels bracketed by events)
+        pk = peaks()
+        reps = max(3, min(args.steps, 10))
+        gsa.gsa_timing_begin(64 * reps)
+        for _ in range(reps):
+            step(d_in)
+        recs = gsa.gsa_timing_end(64 * reps)
+        per = {}
+        for lab, ms in recs:
+            per.setdefault(lab, []).append(ms)
+        launches = (len(recs) + 2 * len(per.get("gate_grad", []))) // reps
+        kernels = []
+        tot = sum(sum(v) for v in per.values())
+        for lab, v in per.items():
+            avg = sum(v) / len(v)
+            by = kernel_algorithmic_bytes(lab, w)
+            kernels.append({"kernel": lab, "launches_per_step": len(v) // reps, "avg_ms": avg,
+                            "share": sum(v) / tot, "alg_bytes": by,
+                            "achieved_gbs": by / (avg * 1e-3) / 1e9,
+                            "frac_of_hbm_peak": by / (avg * 1e-3) / 1e9 / pk["hbm_gbs"]})
+        kernels.sort(key=lambda k: -k["share"])
+        top = kernels[0]
+        traffic = None
+        tpath = os.path.join(ROOT, "profiles", "traffic.json")
+        if os.path.exists(tpath):
+            traffic = json.load(open(tpath)).get(top["kernel"])
+        roofline = {"bound": "hbm", "kernel": top["kernel"], "achieved": top["achieved_gbs"],
+                    "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": top["frac_of_hbm_peak"],
+                    "traffic": traffic, "peak_source": pk["source"],
+                    "share_of_step": top["share"]}
+        step_bytes = step_algorithmic_bytes(w)
+        whole = {"alg_bytes_per_step": step_bytes,
+                 "achieved_gbs": step_bytes / (ms_step * 1e-3) / 1e9,
+                 "frac_of_hbm_peak": step_bytes / (ms_step * 1e-3) / 1e9 / pk["hbm_gbs"],
+                 "tflops": step_flops(w) / (ms_step * 1e-3) / 1e12}
+
+        # ---- decode step (the recurrent form), reported beside the training number
+        decode = bench_decode(gsa, torch, dev, pk)
+
+        # ---- the oracle on the host cores, bounded sample
+        cpu = None
+        if world == 1 and not args.no_cpu_baseline:
+            import oracle
+            x0 = x
+            threads = min(oracle.default_threads(), 16, w.B * w.H)
+            pairs = min(w.B * w.H, 2 * threads)
+            t0 = time.perf_counter()
+            oracle_step(x0, w, pairs, threads)
+            dt = time.perf_counter() - t0
+            cpu = {"value": pairs * w.T / w.H / dt, "unit": UNIT, "cores": threads, "kind": "oracle",
+                   "sample": f"{pairs} of {w.B * w.H} (batch, head) pairs of one {WORKLOAD} step, "
+                             f"fp64 forward + reverse sweep, {dt:.1f} s wall"}
+
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+            "data": "synthetic (seeded N(0,1) q,k,v,dO; gate sigmoid(N(0,1))^(1/8))",
+            "config": {"workload": WORKLOAD, "B": w.B, "T": w.T, "H": w.H, "d_k": w.d_k,
+                       "d_v": w.d_v, "m": w.m, "io": w.io, "chunk": gsa.gsa_chunk_size(p),
+                       "step": "gsa_fwd (logits saved) + gsa_bwd",
+                       "l2": "inputs larger than L2 (1.1 GB touched per step vs 126 MB)",
+                       "parallelism": f"dp{world} over batch, no collective"},
+            "clocks": clocks,
+            "e2e": {"value": world * w.tokens / (e2e_ms * 1e-3), "unit": UNIT,
+                    "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms},
+            "gpu_launches": launches * args.steps,
+            "gpu_launches_per_step": launches,
+            "roofline": roofline,
+            "whole_step": whole,
+            "kernels": kernels,
+            "decode": decode,
+            "cpu_baseline": cpu,
+        }
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+    if line is not None:
+        print(json.dumps(line), flush=True)
+
+
+def bench_decode(gsa, torch, dev, pk):
+    """gsa_decode_step on the batched-decoding workload (256 sequences x 32 heads, d=128,
+    m=64, fp32 memories): achieved HBM GB/s on the bytes one step must move."""
+    w = W.CONFIGS["decode"]
+    p = gsa.Params(w.B, 1, w.H, w.d_k, w.d_v, w.m, io="bf16")
+    st = W.make_decode_states(w)
+    Ks = torch.from_numpy(st["K"]).to(dev)
+    Vs = torch.from_numpy(st["V"]).to(dev)
+    xs = W.make_decode_step_inputs(w, 0)
+    q, k, v = (torch.from_numpy(xs[n]).to(dev).to(torch.bfloat16) for n in ("q", "k", "v"))
+    gate = torch.from_numpy(xs["gate"]).to(dev)
+    o = torch.empty(w.B, w.H, w.d_v, dtype=torch.bfloat16, device=dev)
+    for _ in range(10):
+        gsa.gsa_decode_step(p, q, k, v, gate, Ks, Vs, o=o)
+    torch.cuda.synchronize()
+    steps = 100
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        gsa.gsa_decode_step(p, q, k, v, gate, Ks, Vs, o=o)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    pairs = w.B * w.H
+    by = pairs * (2 * 4 * w.m * (w.d_k + w.d_v) + 2 * (2 * w.d_k + 2 * w.d_v) + 4 * w.m)
+    return {"workload": "decode (256 seqs x 32 heads, d=128, m=64)", "us_per_step": ms * 1e3,
+            "tokens_per_s": w.B / (ms * 1e-3), "alg_bytes_per_step": by,
+            "achieved_gbs": by / (ms * 1e-3) / 1e9,
+            "frac_of_hbm_peak": by / (ms * 1e-3) / 1e9 / pk["hbm_gbs"],
+            "note": "states (1.07 GB read+write per step) exceed L2"}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -153,6 +153,19 @@ GSA_API gsa_status_t gsa_decode_step(const gsa_params_t* params, const void* q,
 GSA_API gsa_status_t gsa_tc_selftest(int32_t mode, const void* X, const void* Y, float* D,
                                      void* stream, int32_t* dev_status);
 
+/*
+ * Per-kernel timing for benchmarks (no counterpart in the paper).  Between
+ * gsa_timing_begin(capacity) and gsa_timing_end() on the same HOST thread, every kernel
+ * that this thread's gsa_* calls enqueue is bracketed by a pair of CUDA events on its
+ * stream (up to `capacity` kernels).  gsa_timing_end waits for the last one, writes the
+ * duration in milliseconds and a static label of each timed kernel, in launch order, to
+ * ms[0..n) / labels[0..n), and returns n (-1 on error or if timing was not active).  These
+ * two calls create and destroy events and synchronise with the host: keep them out of
+ * production paths.
+ */
+GSA_API gsa_status_t gsa_timing_begin(int32_t capacity);
+GSA_API int32_t gsa_timing_end(float* ms, const char** labels, int32_t capacity);
+
 #ifdef __cplusplus
 }
 #endif

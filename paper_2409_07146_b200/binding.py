@@ -64,7 +64,8 @@ def lib_path() -> str:
 
 def exported_symbols():
     return ["gsa_chunk_size", "gsa_workspace_bytes", "gsa_status_string", "gsa_gate_cumsum",
-            "gsa_fwd", "gsa_bwd", "gsa_decode_step", "gsa_tc_selftest"]
+            "gsa_fwd", "gsa_bwd", "gsa_decode_step", "gsa_tc_selftest", "gsa_timing_begin",
+            "gsa_timing_end"]
 
 
 def load_library():
@@ -93,6 +94,10 @@ def load_library():
     lib.gsa_bwd.restype = ctypes.c_int
     lib.gsa_decode_step.argtypes = [pp] + [vp] * 8
     lib.gsa_decode_step.restype = ctypes.c_int
+    lib.gsa_timing_begin.argtypes = [i32]
+    lib.gsa_timing_begin.restype = ctypes.c_int
+    lib.gsa_timing_end.argtypes = [ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_char_p), i32]
+    lib.gsa_timing_end.restype = i32
     lib.gsa_tc_selftest.argtypes = [i32, vp, vp, vp, vp, vp]
     lib.gsa_tc_selftest.restype = ctypes.c_int
     _lib = lib
@@ -219,3 +224,17 @@ def gsa_tc_selftest(mode: int, X, Y, dev_status=None):
         _ptr(D, torch.float32, None, "D"), _stream(), _ptr(dev_status, torch.int32, None, "dev_status")),
         "gsa_tc_selftest")
     return D
+
+
+def gsa_timing_begin(capacity: int = 4096):
+    _check(load_library().gsa_timing_begin(capacity), "gsa_timing_begin")
+
+
+def gsa_timing_end(capacity: int = 4096):
+    """Returns [(label, milliseconds)] of the kernels timed since gsa_timing_begin."""
+    ms = (ctypes.c_float * capacity)()
+    labels = (ctypes.c_char_p * capacity)()
+    n = load_library().gsa_timing_end(ms, labels, capacity)
+    if n < 0:
+        raise RuntimeError("gsa_timing_end failed")
+    return [(labels[i].decode(), float(ms[i])) for i in range(n)]

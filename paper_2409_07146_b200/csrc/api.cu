@@ -2,6 +2,8 @@
 // the kernels of one forward / backward call are enqueued.  No kernel lives here.
 #include <string.h>
 
+#include <vector>
+
 #include "common.cuh"
 
 using namespace gsa;
@@ -95,10 +97,39 @@ cudaError_t key_side(const gsa_params_t& p, const KeySideArgs& a, int reverse, c
     return launch_key_side_simt(a, p.io, p.m, reverse, st);
 }
 
+// ---- optional per-kernel timing (benchmarks only): while a sink is active on the calling
+// host thread, every kernel launch is bracketed by a pair of events on its stream.
+struct TimingSink {
+    bool active = false;
+    int capacity = 0, count = 0;
+    std::vector<cudaEvent_t> ev;       // 2 per launch
+    std::vector<const char*> labels;
+};
+thread_local TimingSink g_sink;
+
+void timing_before(cudaStream_t st) {
+    if (g_sink.active && g_sink.count < g_sink.capacity) cudaEventRecord(g_sink.ev[2 * g_sink.count], st);
+}
+void timing_after(const char* label, cudaStream_t st) {
+    if (g_sink.active && g_sink.count < g_sink.capacity) {
+        cudaEventRecord(g_sink.ev[2 * g_sink.count + 1], st);
+        g_sink.labels[g_sink.count] = label;
+        ++g_sink.count;
+    }
+}
+
 #define GSA_CUDA(expr)                                  \
     do {                                                \
         cudaError_t e__ = (expr);                       \
         if (e__ != cudaSuccess) return GSA_ERR_CUDA;    \
+    } while (0)
+// a kernel launch on stream `st`, timed when a sink is active
+#define GSA_LAUNCH(label, expr)                         \
+    do {                                                \
+        timing_before(st);                              \
+        cudaError_t e__ = (expr);                       \
+        if (e__ != cudaSuccess) return GSA_ERR_CUDA;    \
+        timing_after(label, st);                        \
     } while (0)
 
 }  // namespace
@@ -131,12 +162,13 @@ size_t gsa_workspace_bytes(const gsa_params_t* params, int32_t which) {
 
 gsa_status_t gsa_gate_cumsum(const gsa_params_t* params, const float* gate, float* G, float* I,
                              void* stream) {
-    gsa_status_t st = check_params(params, true);
-    if (st != GSA_OK) return st;
+    gsa_status_t rc = check_params(params, true);
+    if (rc != GSA_OK) return rc;
     if (!ok_ptr(gate) || !ok_ptr(G) || !ok_ptr(I)) return GSA_ERR_INVALID_ARG;
     const gsa_params_t& p = *params;
-    GSA_CUDA(launch_gate_cumsum(gate, p.gate_kind == GSA_GATE_LOG_A, G, I, p.B, p.T, p.H, p.m,
-                                chunk_of(p), static_cast<cudaStream_t>(stream)));
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    GSA_LAUNCH("gate_cumsum", launch_gate_cumsum(gate, p.gate_kind == GSA_GATE_LOG_A, G, I, p.B, p.T,
+                                                 p.H, p.m, chunk_of(p), st));
     return GSA_OK;
 }
 
@@ -157,15 +189,16 @@ gsa_status_t gsa_fwd(const gsa_params_t* params, const void* q, const void* k, c
     const Slices s = slices(p);
     const size_t rows = (size_t)p.B * p.T * p.H;
 
-    GSA_CUDA(launch_gate_cumsum(gate, p.gate_kind == GSA_GATE_LOG_A, w.G, w.I, p.B, p.T, p.H, p.m, chunk_of(p), st));
+    GSA_LAUNCH("gate_cumsum", launch_gate_cumsum(gate, p.gate_kind == GSA_GATE_LOG_A, w.G, w.I, p.B, p.T,
+                                                 p.H, p.m, chunk_of(p), st));
     // pass 1: o' = GLA(q, k, 1-a) with the decay on the slot (value) side
     ValueSideArgs a1{q, k, w.I, w.G, K0, KT, w.okpart, p.B, p.T, p.H, p.d_k};
-    GSA_CUDA(value_side(p, a1, 0, st, dev_status));
+    GSA_LAUNCH("pass1_value_side", value_side(p, a1, 0, st, dev_status));
     float* ok = ok_save ? ok_save : w.ok;
-    GSA_CUDA(launch_slot_softmax_fwd(w.okpart, s.k, p.scale, ok, w.p, rows, p.m, st));
+    GSA_LAUNCH("slot_softmax", launch_slot_softmax_fwd(w.okpart, s.k, p.scale, ok, w.p, rows, p.m, st));
     // pass 2: o = GLA(softmax(o'), 1-a, v) with the decay on the slot (key) side
     KeySideArgs a2{w.p, w.I, w.G, v, V0, VT, o, p.B, p.T, p.H, p.d_v};
-    GSA_CUDA(key_side(p, a2, 0, st, dev_status));
+    GSA_LAUNCH("pass2_key_side", key_side(p, a2, 0, st, dev_status));
     return GSA_OK;
 }
 
@@ -190,32 +223,33 @@ gsa_status_t gsa_bwd(const gsa_params_t* params, const void* q, const void* k, c
     const Slices s = slices(p);
     const size_t rows = (size_t)p.B * p.T * p.H;
 
-    GSA_CUDA(launch_gate_cumsum(gate, p.gate_kind == GSA_GATE_LOG_A, w.G, w.I, p.B, p.T, p.H, p.m, chunk_of(p), st));
+    GSA_LAUNCH("gate_cumsum", launch_gate_cumsum(gate, p.gate_kind == GSA_GATE_LOG_A, w.G, w.I, p.B, p.T,
+                                                 p.H, p.m, chunk_of(p), st));
     const float* ok = ok_saved;
     if (ok == nullptr) {  // recompute pass 1 and its logits
         ValueSideArgs a1{q, k, w.I, w.G, K0, nullptr, w.okpart, p.B, p.T, p.H, p.d_k};
-        GSA_CUDA(value_side(p, a1, 0, st, dev_status));
-        GSA_CUDA(launch_slot_softmax_fwd(w.okpart, s.k, p.scale, w.ok, w.p, rows, p.m, st));
+        GSA_LAUNCH("pass1_value_side", value_side(p, a1, 0, st, dev_status));
+        GSA_LAUNCH("slot_softmax", launch_slot_softmax_fwd(w.okpart, s.k, p.scale, w.ok, w.p, rows, p.m, st));
         ok = w.ok;
     }
     // gradient w.r.t. the pass-2 queries p: the pass-1 form on (dO, v, 1-a); carries V~
     ValueSideArgs adp{dO, v, w.I, w.G, V0, dVT ? w.VT : nullptr, w.dppart, p.B, p.T, p.H, p.d_v};
-    GSA_CUDA(value_side(p, adp, 0, st, dev_status));
-    GSA_CUDA(launch_slot_softmax_bwd(ok, w.dppart, s.v, p.scale, w.p, w.dz, w.u, rows, p.m, st));
+    GSA_LAUNCH("bwd_dp_value_side", value_side(p, adp, 0, st, dev_status));
+    GSA_LAUNCH("slot_softmax_bwd", launch_slot_softmax_bwd(ok, w.dppart, s.v, p.scale, w.p, w.dz, w.u, rows, p.m, st));
     // dq: the pass-2 form on (dz, 1-a, k); carries K~
     KeySideArgs adq{w.dz, w.I, w.G, k, K0, dKT ? w.KT : nullptr, dq, p.B, p.T, p.H, p.d_k};
-    GSA_CUDA(key_side(p, adq, 0, st, dev_status));
+    GSA_LAUNCH("bwd_dq_key_side", key_side(p, adq, 0, st, dev_status));
     // time-reversed runs: dv and dI^v share the state dV~; dk and dI^k share dK~
     KeySideArgs adv{w.I, w.p, w.G, dO, dVT, dV0, dv, p.B, p.T, p.H, p.d_v};
-    GSA_CUDA(key_side(p, adv, 1, st, dev_status));
+    GSA_LAUNCH("bwd_dv_key_side_rev", key_side(p, adv, 1, st, dev_status));
     ValueSideArgs adIv{v, dO, w.p, w.G, dVT, nullptr, w.dIv, p.B, p.T, p.H, p.d_v};
-    GSA_CUDA(value_side(p, adIv, 1, st, dev_status));
+    GSA_LAUNCH("bwd_dIv_value_side_rev", value_side(p, adIv, 1, st, dev_status));
     KeySideArgs adk{w.I, w.dz, w.G, q, dKT, dK0, dk, p.B, p.T, p.H, p.d_k};
-    GSA_CUDA(key_side(p, adk, 1, st, dev_status));
+    GSA_LAUNCH("bwd_dk_key_side_rev", key_side(p, adk, 1, st, dev_status));
     ValueSideArgs adIk{k, q, w.dz, w.G, dKT, nullptr, w.dIk, p.B, p.T, p.H, p.d_k};
-    GSA_CUDA(value_side(p, adIk, 1, st, dev_status));
+    GSA_LAUNCH("bwd_dIk_value_side_rev", value_side(p, adIk, 1, st, dev_status));
     // forget-gate gradient: reversed cumulative sum over the whole sequence
-    GSA_CUDA(launch_gate_grad(w.u, w.I, w.dIk, s.k, w.dIv, s.v, gate, p.gate_kind == GSA_GATE_LOG_A,
+    GSA_LAUNCH("gate_grad", launch_gate_grad(w.u, w.I, w.dIk, s.k, w.dIv, s.v, gate, p.gate_kind == GSA_GATE_LOG_A,
                               dKT, w.KT, dVT, w.VT, p.d_k, p.d_v, w.chunk_tot, dgate, p.B, p.T,
                               p.H, p.m, st));
     return GSA_OK;
@@ -229,8 +263,38 @@ gsa_status_t gsa_decode_step(const gsa_params_t* params, const void* q, const vo
     if (!ok_ptr(q) || !ok_ptr(k) || !ok_ptr(v) || !ok_ptr(gate) || !ok_ptr(Kstate) ||
         !ok_ptr(Vstate) || !ok_ptr(o))
         return GSA_ERR_INVALID_ARG;
-    GSA_CUDA(launch_decode(*params, q, k, v, gate, Kstate, Vstate, o, static_cast<cudaStream_t>(stream)));
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    GSA_LAUNCH("decode_step", launch_decode(*params, q, k, v, gate, Kstate, Vstate, o, st));
     return GSA_OK;
+}
+
+gsa_status_t gsa_timing_begin(int32_t capacity) {
+    if (capacity < 1 || capacity > (1 << 20) || g_sink.active) return GSA_ERR_INVALID_ARG;
+    g_sink.ev.assign(2 * (size_t)capacity, nullptr);
+    g_sink.labels.assign(capacity, nullptr);
+    for (auto& e : g_sink.ev)
+        if (cudaEventCreate(&e) != cudaSuccess) return GSA_ERR_CUDA;
+    g_sink.capacity = capacity;
+    g_sink.count = 0;
+    g_sink.active = true;
+    return GSA_OK;
+}
+
+int32_t gsa_timing_end(float* ms, const char** labels, int32_t capacity) {
+    if (!g_sink.active) return -1;
+    g_sink.active = false;
+    const int n = g_sink.count < capacity ? g_sink.count : capacity;
+    int rc = n;
+    if (g_sink.count > 0 && cudaEventSynchronize(g_sink.ev[2 * g_sink.count - 1]) != cudaSuccess) rc = -1;
+    for (int i = 0; i < n && rc >= 0; ++i) {
+        if (cudaEventElapsedTime(&ms[i], g_sink.ev[2 * i], g_sink.ev[2 * i + 1]) != cudaSuccess) rc = -1;
+        labels[i] = g_sink.labels[i];
+    }
+    for (auto& e : g_sink.ev)
+        if (e) cudaEventDestroy(e);
+    g_sink.ev.clear();
+    g_sink.labels.clear();
+    return rc;
 }
 
 }  // extern "C"
