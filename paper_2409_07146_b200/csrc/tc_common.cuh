@@ -187,8 +187,10 @@ __device__ __forceinline__ void store_elem(unsigned char* panel, int row, int co
 
 }  // namespace tc
 
-// Host side: encode a 4-D tensor map over a [B,T,H,D] bf16 tensor with a box of
-// 64 channels x `box_rows` tokens of one (batch, head), 128-byte swizzle, zero fill.
-cudaError_t make_tensor_map_bthd(CUtensorMap* map, const void* base, int B, int T, int H, int D, int box_rows);
+// Host side: encode a 4-D tensor map over a [B,T,H,D] tensor of bf16 (elem_bytes 2) or fp32
+// (elem_bytes 4) with a box of 128 bytes of channels x `box_rows` tokens of one (batch,
+// head), 128-byte swizzle, zero fill beyond the tensor.
+cudaError_t make_tensor_map_bthd(CUtensorMap* map, const void* base, int B, int T, int H, int D, int box_rows,
+                                 int elem_bytes);
 
 }  // namespace gsa

@@ -6,7 +6,8 @@
 
 namespace gsa {
 
-cudaError_t make_tensor_map_bthd(CUtensorMap* map, const void* base, int B, int T, int H, int D, int box_rows) {
+cudaError_t make_tensor_map_bthd(CUtensorMap* map, const void* base, int B, int T, int H, int D, int box_rows,
+                                 int elem_bytes) {
     typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -20,10 +21,11 @@ cudaError_t make_tensor_map_bthd(CUtensorMap* map, const void* base, int B, int 
         encode = reinterpret_cast<EncodeFn>(fn);
     }
     const cuuint64_t dims[4] = {(cuuint64_t)D, (cuuint64_t)H, (cuuint64_t)T, (cuuint64_t)B};
-    const cuuint64_t strides[3] = {(cuuint64_t)D * 2, (cuuint64_t)H * D * 2, (cuuint64_t)T * H * D * 2};
-    const cuuint32_t box[4] = {64, 1, (cuuint32_t)box_rows, 1};
+    const cuuint64_t eb = (cuuint64_t)elem_bytes;
+    const cuuint64_t strides[3] = {(cuuint64_t)D * eb, (cuuint64_t)H * D * eb, (cuuint64_t)T * H * D * eb};
+    const cuuint32_t box[4] = {(cuuint32_t)(128 / elem_bytes), 1, (cuuint32_t)box_rows, 1};
     const cuuint32_t estr[4] = {1, 1, 1, 1};
-    CUresult r = encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
+    CUresult r = encode(map, elem_bytes == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, const_cast<void*>(base), dims, strides, box, estr,
                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
@@ -143,8 +145,8 @@ extern "C" GSA_API gsa_status_t gsa_tc_selftest(int32_t mode, const void* X, con
     using namespace gsa;
     if (mode < 0 || mode > 3 || X == nullptr || Y == nullptr || D == nullptr) return GSA_ERR_INVALID_ARG;
     CUtensorMap mx, my;
-    if (make_tensor_map_bthd(&mx, X, 1, 128, 1, 128, 128) != cudaSuccess) return GSA_ERR_CUDA;
-    if (make_tensor_map_bthd(&my, Y, 1, 128, 1, 128, 128) != cudaSuccess) return GSA_ERR_CUDA;
+    if (make_tensor_map_bthd(&mx, X, 1, 128, 1, 128, 128, 2) != cudaSuccess) return GSA_ERR_CUDA;
+    if (make_tensor_map_bthd(&my, Y, 1, 128, 1, 128, 128, 2) != cudaSuccess) return GSA_ERR_CUDA;
     const size_t smem = 6 * kPanel + 1024;
     if (cudaFuncSetAttribute(tc_selftest_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return GSA_ERR_CUDA;
