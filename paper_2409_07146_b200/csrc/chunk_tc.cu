@@ -1,8 +1,9 @@
 // tcgen05 (bf16 tensor-core) versions of the two chunk primitives of Algorithm 1.
 //
-// One CTA of 128 threads owns one (batch, head) and one 128-wide slice of the head
-// dimension and walks the chunks (128 tokens each) in order.  Thread i is row i of the
-// chunk and channel i of the state slice, which is also TMEM lane i of every accumulator.
+// One CTA of 256 threads owns one (batch, head) and one 128-wide slice of the head
+// dimension and walks the chunks (128 tokens each) in order.  Threads r and r + 128 share
+// row r of the chunk, which is channel r of the state slice and TMEM lane r of every
+// accumulator; the first works on slots (or columns) 0..31 (0..63), the second on the rest.
 // Per chunk:
 //   * every tile -- the d-sized ones (xq, xk / xv, bf16) and the slot-sized ones (weights,
 //     cumulative log gate G, fp32) -- arrives by TMA with the 128-byte swizzle, requested as
@@ -33,18 +34,19 @@ constexpr int kDST = 128;              // head-dimension slice per CTA
 constexpr int kM = 64;                 // slots
 constexpr int kPanelB = 128 * 128;     // bytes of a 128-row operand panel
 constexpr uint32_t kTmemCols = 512;
+constexpr int kThreads = 256;
+constexpr int kHS = kM / 2;            // slots per thread
 
 // accumulator columns
 constexpr int kColP = 0;       // P / A           [128 x 128]
 constexpr int kColO = 128;     // inter (+ intra for key_side) output
 constexpr int kColU = 256;     // state update    [128 x 64]
-constexpr int kColO2 = 320;    // value_side intra output [128 x 64]
 
 // Optional phase timing for development builds (-DGSA_TC_PROF): CTA 0 prints, for its fifth
 // chunk, the SM clock at each phase boundary.
 #ifdef GSA_TC_PROF
-#define PROF_DECL long long prof_t[12]; int prof_n = 0;
-#define PROF_MARK() do { if (prof_n < 12) prof_t[prof_n++] = clock64(); } while (0)
+#define PROF_DECL long long prof_t[32]; int prof_n = 0;
+#define PROF_MARK() do { if (prof_n < 32) prof_t[prof_n++] = clock64(); } while (0)
 #define PROF_DUMP(name) do { if (blockIdx.x == 0 && blockIdx.y == 0 && tid == 0 && it == 4) { \
     printf("%s:", name); for (int i_ = 1; i_ < prof_n; ++i_) printf(" %lld", prof_t[i_] - prof_t[i_ - 1]); printf("\n"); } prof_n = 0; } while (0)
 #else
@@ -79,16 +81,17 @@ __device__ __forceinline__ float tile_elem(const unsigned char* tile, int row, i
     return *reinterpret_cast<const float*>(tile + (s >> 5) * kPanelB + swz128(row, (s & 31) >> 2) + (s & 3) * 4);
 }
 
-// bf16 copy of this thread's state row (64 values, optionally scaled per slot) as row `row`
-// of a one-panel operand
+// bf16 copy of this thread's half state row (32 values from slot sb on, optionally scaled
+// per slot) into row `row` of a one-panel operand
 template <bool SCALE>
-__device__ __forceinline__ void store_state_row(unsigned char* panel, int row, const float (&S)[kM], const float* scale) {
+__device__ __forceinline__ void store_state_row(unsigned char* panel, int row, int sb, const float (&S)[kHS],
+                                                const float* scale) {
 #pragma unroll
-    for (int c = 0; c < kM / 8; ++c) {
+    for (int c = 0; c < kHS / 8; ++c) {
         float x[8];
 #pragma unroll
-        for (int e = 0; e < 8; ++e) x[e] = SCALE ? S[8 * c + e] * scale[8 * c + e] : S[8 * c + e];
-        store_chunk(panel, row, c, x);
+        for (int e = 0; e < 8; ++e) x[e] = SCALE ? S[8 * c + e] * scale[sb + 8 * c + e] : S[8 * c + e];
+        store_chunk(panel, row, (sb >> 3) + c, x);
     }
 }
 
@@ -127,22 +130,24 @@ __device__ __forceinline__ void ctl_init(Ctl* ctl, int tid, int warp) {
 
 // masked accumulator row -> bf16 K-major operand row (two 64-column panels)
 template <bool REV>
-__device__ __forceinline__ void store_masked_row(uint32_t tmem, int warp, int tid, unsigned char* dst) {
+__device__ __forceinline__ void store_masked_row(uint32_t tmem, int wq, int row, int half, unsigned char* dst) {
+    unsigned char* panel = dst + half * kPanelB;      // columns 64 half .. 64 half + 63
 #pragma unroll
-    for (int c0 = 0; c0 < kCT; c0 += 16) {
-        float v[16];
-        tmem_ld16(tmem_row_addr(tmem, warp, kColP + c0), v);
+    for (int c0 = 0; c0 < 64; c0 += 32) {
+        float v[32];
+        tmem_ld32(tmem_row_addr(tmem, wq, kColP + 64 * half + c0), v);
 #pragma unroll
-        for (int e = 0; e < 16; ++e) {
-            const int j = c0 + e;
-            const bool keep = REV ? (j >= tid) : (j <= tid);
+        for (int e = 0; e < 32; ++e) {
+            const int j = 64 * half + c0 + e;
+            const bool keep = REV ? (j >= row) : (j <= row);
             v[e] = keep ? v[e] : 0.f;
         }
-        const float x0[8] = {v[0], v[1], v[2], v[3], v[4], v[5], v[6], v[7]};
-        const float x1[8] = {v[8], v[9], v[10], v[11], v[12], v[13], v[14], v[15]};
-        unsigned char* panel = dst + (c0 >> 6) * kPanelB;
-        store_chunk(panel, tid, (c0 & 63) >> 3, x0);
-        store_chunk(panel, tid, ((c0 & 63) >> 3) + 1, x1);
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            const float x[8] = {v[8 * c], v[8 * c + 1], v[8 * c + 2], v[8 * c + 3],
+                                v[8 * c + 4], v[8 * c + 5], v[8 * c + 6], v[8 * c + 7]};
+            store_chunk(panel, row, (c0 >> 3) + c, x);
+        }
     }
 }
 
@@ -150,12 +155,13 @@ __device__ __forceinline__ void store_masked_row(uint32_t tmem, int warp, int ti
 // value_side: out_i[s] = sum_{j<=i} <xq_i, xk_j> w_j[s] decay_ij[s]  + decayed (xq_i S)[s]
 // ======================================================================================
 template <bool REV>
-__global__ void __launch_bounds__(128, 1)
+__global__ void __launch_bounds__(kThreads, 1)
 value_side_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK,
                      const __grid_constant__ CUtensorMap mapW, const __grid_constant__ CUtensorMap mapG,
-                     ValueSideArgs a, int32_t* dev_status) {
+                     const __grid_constant__ CUtensorMap mapO, ValueSideArgs a, int32_t* dev_status) {
     extern __shared__ unsigned char smem_raw[];
-    unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    // align by pointer arithmetic (not an integer round trip) so accesses stay in the shared window
+    unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
     unsigned char* sXq = smem;                       // 2 panels                                  (32 KB)
     unsigned char* sXk = sXq + 2 * kPanelB;          // 2 panels                                  (32 KB)
     unsigned char* sG = sXk + 2 * kPanelB;           // G tile fp32, [2 stages][2 panels]         (64 KB)
@@ -166,7 +172,8 @@ value_side_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_cons
     unsigned char* sSb = sWt + kPanelB;              // state copy, MN-major B [128][64]          (16 KB)
     Ctl* ctl = reinterpret_cast<Ctl*>(sSb + kPanelB);
 
-    const int tid = threadIdx.x, warp = tid >> 5;
+    const int tid = threadIdx.x, warp = tid >> 5, wq = warp & 3, half = tid >> 7, row = tid & 127;
+    const int sb = kHS * half;          // this thread's first slot
     const int bh = blockIdx.x, slice = blockIdx.y, b = bh / a.H, h = bh % a.H;
     const int d0 = slice * kDST;
     const size_t strideM = (size_t)a.H * kM;
@@ -198,16 +205,16 @@ value_side_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_cons
         tma_load_4d(sW + kPanelB, &mapW, &ctl->bar_w, 32, h, t, b);
     };
     if (tid == 0) {
-        prefetch_tmap(&mapQ); prefetch_tmap(&mapK); prefetch_tmap(&mapW); prefetch_tmap(&mapG);
+        prefetch_tmap(&mapQ); prefetch_tmap(&mapK); prefetch_tmap(&mapW); prefetch_tmap(&mapG); prefetch_tmap(&mapO);
         load_g(0);
         load_w(0);
         load_x(0);
     }
 
     // state slice: S[c = tid][s]
-    float S[kM];
+    float S[kHS];
 #pragma unroll
-    for (int s = 0; s < kM; ++s) S[s] = a.S0 ? a.S0[((size_t)bh * kM + s) * a.D + d0 + tid] : 0.f;
+    for (int s = 0; s < kHS; ++s) S[s] = a.S0 ? a.S0[((size_t)bh * kM + sb + s) * a.D + d0 + row] : 0.f;
 
     constexpr uint32_t idescP = make_idesc(128, 128, false, false);  // xq xk^T
     constexpr uint32_t idescO = make_idesc(128, kM, false, true);    // xq x state copy (MN-major B)
@@ -222,42 +229,49 @@ value_side_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_cons
         const int valid = min(kCT, a.T - t0);
         const unsigned char* gt = sG + (2 * (it & 1)) * kPanelB;
         PROF_MARK();
-        if (tid == 0 && it + 1 < nchunks) load_g(it + 1);
+        if (tid == 0 && it + 1 < nchunks) {
+            bulk_wait_read();     // the output rows staged in that G buffer two chunks ago have left
+            load_g(it + 1);
+        }
         if (!mbar_wait(&ctl->bar_g[it & 1], (it >> 1) & 1)) ctl->abort = 1;
         if (!mbar_wait(&ctl->bar_w, it & 1)) ctl->abort = 1;
+        PROF_MARK();
         const bool moderate = publish_chunk_decay(ctl, tid, gt, valid - 1);
         if (ctl->abort) break;
         PROF_MARK();
 
         // ---- this token's slot rows -> operand rows (rows past the end: zero weights)
-        const int grow = min(tid, valid - 1);
+        const int grow = min(row, valid - 1);
 #pragma unroll
-        for (int s0 = 0; s0 < kM; s0 += 8) {
+        for (int s0 = sb; s0 < sb + kHS; s0 += 8) {
             float g[8], w[8], wp[8], wt[8];
             tile_row8(gt, grow, s0, g);
-            tile_row8(sW, tid, s0, w);
+            tile_row8(sW, row, s0, w);
+            // Branch-free over the elements (a branch per element would serialise the exps):
+            //   reverse           : intra = state-update weights = w exp(G)
+            //   forward, moderate : intra w exp(-G); state update = intra * exp(G_C)
+            //   forward, strong   : state update w exp(G_C - G); no intra operand
 #pragma unroll
             for (int e = 0; e < 8; ++e) {
-                if (REV) {
-                    // reverse: both the intra and the state-update weights are w exp(G)
-                    wt[e] = w[e] * __expf(g[e]);
-                    wp[e] = wt[e];
-                } else if (moderate) {
-                    // forward: intra w exp(-G), state update w exp(G_C - G) = intra * exp(G_C)
-                    wp[e] = w[e] * __expf(-g[e]);
-                    wt[e] = wp[e] * ctl->egc[s0 + e];
-                } else {
-                    wp[e] = 0.f;
-                    wt[e] = w[e] * __expf(ctl->gc[s0 + e] - g[e]);
-                }
+                const float off = (REV || moderate) ? 0.f : ctl->gc[s0 + e];
+                const float mul = (!REV && moderate) ? ctl->egc[s0 + e] : 1.f;
+                wp[e] = w[e] * __expf(REV ? g[e] : off - g[e]);
+                wt[e] = wp[e] * mul;
             }
-            store_chunk(sWt, tid, s0 >> 3, wt);
-            if (moderate) store_chunk(sWp, tid, s0 >> 3, wp);
+#ifndef EXP_NOBUILDSTORE
+            store_chunk(sWt, row, s0 >> 3, wt);
+            if (moderate) store_chunk(sWp, row, s0 >> 3, wp);
+#else
+            if (wt[0] + wp[3] == 1234.5f) store_chunk(sWt, row, s0 >> 3, wt);
+#endif
         }
+        PROF_MARK();
         // state copy for the inter-chunk product; a moderate reverse chunk folds exp(G_C) in
-        if (REV && moderate) store_state_row<true>(sSb, tid, S, ctl->egc);
-        else store_state_row<false>(sSb, tid, S, nullptr);
+        if (REV && moderate) store_state_row<true>(sSb, row, sb, S, ctl->egc);
+        else store_state_row<false>(sSb, row, sb, S, nullptr);
+        PROF_MARK();
         fence_async_smem();
+        PROF_MARK();
         if (!mbar_wait(&ctl->bar_x, it & 1)) ctl->abort = 1;
         PROF_MARK();
         tc_fence_before_sync();
@@ -291,7 +305,9 @@ value_side_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_cons
         if (tid == 0 && it + 1 < nchunks) load_x(it + 1);
 
         if (moderate) {
-            store_masked_row<REV>(tmem, warp, tid, sPm);    // overwrites the weight tile: all rows were read
+#ifndef EXP_NOPM
+            store_masked_row<REV>(tmem, wq, row, half, sPm);    // overwrites the weight tile: all rows were read
+#endif
             fence_async_smem();
         }
         tc_fence_before_sync();
@@ -311,10 +327,10 @@ value_side_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_cons
         } else {
             // Strong decay: the intra-chunk term with explicit exponent differences on the CUDA
             // cores, straight from the fp32 weight and G tiles.
-            const int jlo = REV ? tid : 0, jhi = REV ? kCT - 1 : tid;
+            const int jlo = REV ? row : 0, jhi = REV ? kCT - 1 : row;
             // the accumulator loads are warp-collective: loop bounds are those of the whole warp
-            const int wlo = REV ? warp * 32 : 0, whi = REV ? kCT - 1 : warp * 32 + 31;
-            for (int s0 = 0; s0 < kM; s0 += 16) {
+            const int wlo = REV ? wq * 32 : 0, whi = REV ? kCT - 1 : wq * 32 + 31;
+            for (int s0 = sb; s0 < sb + kHS; s0 += 16) {
                 float gi[16], acc[16], tmp[8];
                 tile_row8(gt, grow, s0, tmp);
 #pragma unroll
@@ -326,7 +342,7 @@ value_side_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_cons
                 for (int e = 0; e < 16; ++e) acc[e] = 0.f;
                 for (int c0 = wlo; c0 <= whi; c0 += 16) {
                     float v[16];
-                    tmem_ld16(tmem_row_addr(tmem, warp, kColP + c0), v);
+                    tmem_ld16(tmem_row_addr(tmem, wq, kColP + c0), v);
 #pragma unroll
                     for (int e = 0; e < 16; ++e) {
                         const int j = c0 + e;
@@ -341,9 +357,9 @@ value_side_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_cons
                     }
                 }
                 float vi[16];
-                tmem_ld16(tmem_row_addr(tmem, warp, kColO + s0), vi);
-                if (tid < valid) {
-                    float* dst = obase + (size_t)(t0 + tid) * strideM + s0;
+                tmem_ld16(tmem_row_addr(tmem, wq, kColO + s0), vi);
+                if (row < valid) {
+                    float* dst = obase + (size_t)(t0 + row) * strideM + s0;
 #pragma unroll
                     for (int e = 0; e < 16; e += 4) {
                         float r[4];
@@ -357,12 +373,11 @@ value_side_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_cons
         }
 
         // ---- state update from U (complete since bar_mma1): S <- S exp(G_C) + U
+        {
+            float v[kHS];
+            tmem_ld32(tmem_row_addr(tmem, wq, kColU + sb), v);
 #pragma unroll
-        for (int c0 = 0; c0 < kM; c0 += 16) {
-            float v[16];
-            tmem_ld16(tmem_row_addr(tmem, warp, kColU + c0), v);
-#pragma unroll
-            for (int e = 0; e < 16; ++e) S[c0 + e] = fmaf(S[c0 + e], ctl->egc[c0 + e], v[e]);
+            for (int e = 0; e < kHS; ++e) S[e] = fmaf(S[e], ctl->egc[sb + e], v[e]);
         }
         PROF_MARK();
 
@@ -372,31 +387,33 @@ value_side_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_cons
             ++n_mma2;
             tc_fence_after_sync();
             PROF_MARK();
+            // the scaled rows replace this chunk's G rows in place (each thread reads and rewrites
+            // only its own 32 slots) and leave as one tiled store, clipped at the sequence end
+            float vo[kHS];
+            tmem_ld32(tmem_row_addr(tmem, wq, kColO + sb), vo);
+            if (row < valid) {
+                unsigned char* panel = const_cast<unsigned char*>(gt) + half * kPanelB;
 #pragma unroll
-            for (int c0 = 0; c0 < kM; c0 += 16) {
-                float vo[16], g0[8], g1[8];
-                tmem_ld16(tmem_row_addr(tmem, warp, kColO + c0), vo);
-                tile_row8(gt, grow, c0, g0);
-                tile_row8(gt, grow, c0 + 8, g1);
-                if (tid < valid) {
-                    float* dst = obase + (size_t)(t0 + tid) * strideM + c0;
-#pragma unroll
-                    for (int e = 0; e < 16; e += 4) {
-                        float r[4];
-#pragma unroll
-                        for (int u = 0; u < 4; ++u) {
-                            const float g = (e + u < 8) ? g0[(e + u) & 7] : g1[(e + u) & 7];
-                            r[u] = vo[e + u] * __expf(REV ? -g : g);
-                        }
-                        *reinterpret_cast<float4*>(dst + e) = make_float4(r[0], r[1], r[2], r[3]);
-                    }
+                for (int c = 0; c < kHS / 4; ++c) {
+                    float4* cell = reinterpret_cast<float4*>(panel + swz128(row, c));
+                    const float4 g = *cell;
+                    *cell = make_float4(vo[4 * c] * __expf(REV ? -g.x : g.x), vo[4 * c + 1] * __expf(REV ? -g.y : g.y),
+                                        vo[4 * c + 2] * __expf(REV ? -g.z : g.z), vo[4 * c + 3] * __expf(REV ? -g.w : g.w));
                 }
             }
+            fence_async_smem();
         }
         tc_fence_before_sync();
         __syncthreads();
-        // the weight tile's buffer (masked P) is free again: request the next chunk's weights
-        if (tid == 0 && it + 1 < nchunks && !ctl->abort) load_w(it + 1);
+        if (tid == 0 && !ctl->abort) {
+            if (moderate) {
+                tma_store_5d(&mapO, gt, 0, h, t0, b, slice);
+                tma_store_5d(&mapO, gt + kPanelB, 32, h, t0, b, slice);
+                bulk_commit();
+            }
+            // the weight tile's buffer (masked P) is free again: request the next chunk's weights
+            if (it + 1 < nchunks) load_w(it + 1);
+        }
         PROF_MARK();
         PROF_DUMP("value_side");
         if (ctl->abort) break;
@@ -410,8 +427,9 @@ value_side_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_cons
         for (int i = 0; i < 200; ++i) __nanosleep(1000);
     } else if (a.Send) {
 #pragma unroll
-        for (int s = 0; s < kM; ++s) a.Send[((size_t)bh * kM + s) * a.D + d0 + tid] = S[s];
+        for (int s = 0; s < kHS; ++s) a.Send[((size_t)bh * kM + sb + s) * a.D + d0 + row] = S[s];
     }
+    if (tid == 0) bulk_wait_read();      // staged output rows must have left before shared memory goes away
     __syncthreads();
     if (warp == 0) {
         __syncwarp();
@@ -423,12 +441,13 @@ value_side_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_cons
 // key_side: out_i = (uq_i * qscale_i) S + sum_j A_ij xv_j,  A_ij = sum_s uq_i[s] uk_j[s] decay_ij[s]
 // ======================================================================================
 template <bool REV>
-__global__ void __launch_bounds__(128, 1)
+__global__ void __launch_bounds__(kThreads, 1)
 key_side_tc_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_constant__ CUtensorMap mapUq,
                    const __grid_constant__ CUtensorMap mapUk, const __grid_constant__ CUtensorMap mapG,
-                   KeySideArgs a, int32_t* dev_status) {
+                   const __grid_constant__ CUtensorMap mapO, KeySideArgs a, int32_t* dev_status) {
     extern __shared__ unsigned char smem_raw[];
-    unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    // align by pointer arithmetic (not an integer round trip) so accesses stay in the shared window
+    unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
     unsigned char* sXv = smem;                       // 2 panels                                   (32 KB)
     unsigned char* sUk = sXv + 2 * kPanelB;          // uk tile fp32, 2 panels                     (32 KB)
     unsigned char* sG = sUk + 2 * kPanelB;           // G tile fp32, 2 panels                      (32 KB)
@@ -441,11 +460,10 @@ key_side_tc_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_consta
     unsigned char* sSb = sKb + kPanelB;              // state copy, K-major B [128 (channel)][64]  (16 KB)
     Ctl* ctl = reinterpret_cast<Ctl*>(sSb + kPanelB);
 
-    const int tid = threadIdx.x, warp = tid >> 5;
+    const int tid = threadIdx.x, warp = tid >> 5, wq = warp & 3, half = tid >> 7, row = tid & 127;
+    const int sb = kHS * half;          // this thread's first slot
     const int bh = blockIdx.x, slice = blockIdx.y, b = bh / a.H, h = bh % a.H;
     const int d0 = slice * kDST;
-    const size_t strideD = (size_t)a.H * a.D;
-    __nv_bfloat16* obase = (__nv_bfloat16*)a.out + ((size_t)b * a.T * a.H + h) * a.D + d0;
 
     ctl_init(ctl, tid, warp);
     const uint32_t tmem = ctl->tmem_slot;
@@ -473,16 +491,16 @@ key_side_tc_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_consta
         tma_load_4d(sUq + kPanelB, &mapUq, &ctl->bar_w, 32, h, t, b);
     };
     if (tid == 0) {
-        prefetch_tmap(&mapV); prefetch_tmap(&mapUq); prefetch_tmap(&mapUk); prefetch_tmap(&mapG);
+        prefetch_tmap(&mapV); prefetch_tmap(&mapUq); prefetch_tmap(&mapUk); prefetch_tmap(&mapG); prefetch_tmap(&mapO);
         load_kg(0);
         load_q(0);
         load_v(0);
     }
 
     // state slice, transposed: S[c = tid][s]
-    float S[kM];
+    float S[kHS];
 #pragma unroll
-    for (int s = 0; s < kM; ++s) S[s] = a.S0 ? a.S0[((size_t)bh * kM + s) * a.D + d0 + tid] : 0.f;
+    for (int s = 0; s < kHS; ++s) S[s] = a.S0 ? a.S0[((size_t)bh * kM + sb + s) * a.D + d0 + row] : 0.f;
 
     constexpr uint32_t idescA = make_idesc(128, 128, false, false);   // Q~ K~^T
     constexpr uint32_t idescO = make_idesc(128, kDST, false, false);  // Q- x state copy (K-major B)
@@ -495,41 +513,43 @@ key_side_tc_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_consta
         const int t0 = chunk_t0(it);
         const int valid = min(kCT, a.T - t0);
         PROF_MARK();
+        if (tid == 0) bulk_wait_read();    // the previous chunk's output rows have left sQt / sKt
         if (!mbar_wait(&ctl->bar_g[0], it & 1)) ctl->abort = 1;
         if (!mbar_wait(&ctl->bar_w, it & 1)) ctl->abort = 1;
+        PROF_MARK();
         const bool moderate = publish_chunk_decay(ctl, tid, sG, valid - 1);
         if (ctl->abort) break;
         PROF_MARK();
 
-        const int grow = min(tid, valid - 1);
+        const int grow = min(row, valid - 1);
 #pragma unroll
-        for (int s0 = 0; s0 < kM; s0 += 8) {
+        for (int s0 = sb; s0 < sb + kHS; s0 += 8) {
             float g[8], uq[8], uk[8], qb[8], kb[8], qt[8], kt[8];
             tile_row8(sG, grow, s0, g);
-            tile_row8(sUq, tid, s0, uq);
-            tile_row8(sUk, tid, s0, uk);
+            tile_row8(sUq, row, s0, uq);
+            tile_row8(sUk, row, s0, uk);
 #pragma unroll
             for (int e = 0; e < 8; ++e) {
                 const float eg = __expf(g[e]);
+                const float einv = __expf(-g[e]);
                 const float egc_g = __expf(ctl->gc[s0 + e] - g[e]);
                 // state terms: forward Q- = uq exp(G), K- = uk exp(G_C - G); reverse swapped
                 qb[e] = uq[e] * (REV ? egc_g : eg);
                 kb[e] = uk[e] * (REV ? eg : egc_g);
-                if (moderate) {
-                    const float einv = __expf(-g[e]);
-                    qt[e] = uq[e] * (REV ? einv : eg);
-                    kt[e] = uk[e] * (REV ? eg : einv);
-                }
+                // intra terms (used by a moderate chunk only): exp(+-G) on the two sides
+                qt[e] = uq[e] * (REV ? einv : eg);
+                kt[e] = uk[e] * (REV ? eg : einv);
             }
-            store_chunk(sQb, tid, s0 >> 3, qb);
-            store_chunk(sKb, tid, s0 >> 3, kb);
+            store_chunk(sQb, row, s0 >> 3, qb);
+            store_chunk(sKb, row, s0 >> 3, kb);
             if (moderate) {
-                store_chunk(sQt, tid, s0 >> 3, qt);
-                store_chunk(sKt, tid, s0 >> 3, kt);
+                store_chunk(sQt, row, s0 >> 3, qt);
+                store_chunk(sKt, row, s0 >> 3, kt);
             }
         }
-        store_state_row<false>(sSb, tid, S, nullptr);
+        store_state_row<false>(sSb, row, sb, S, nullptr);
         fence_async_smem();
+        PROF_MARK();
         if (!mbar_wait(&ctl->bar_x, it & 1)) ctl->abort = 1;
         PROF_MARK();
         tc_fence_before_sync();
@@ -563,7 +583,7 @@ key_side_tc_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_consta
         PROF_MARK();
 
         if (moderate) {
-            store_masked_row<REV>(tmem, warp, tid, sAm);    // overwrites the uq tile: all rows were read
+            store_masked_row<REV>(tmem, wq, row, half, sAm);    // overwrites the uq tile: all rows were read
         } else {
             // Strong decay: A_ij with explicit exponent differences, from the fp32 uk and G tiles.
             float gi[kM], qi[kM];
@@ -571,17 +591,17 @@ key_side_tc_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_consta
             for (int s0 = 0; s0 < kM; s0 += 8) {
                 float g[8], uq[8];
                 tile_row8(sG, grow, s0, g);
-                tile_row8(sUq, tid, s0, uq);
+                tile_row8(sUq, row, s0, uq);
 #pragma unroll
                 for (int e = 0; e < 8; ++e) { gi[s0 + e] = g[e]; qi[s0 + e] = uq[e]; }
             }
             __syncthreads();          // every thread has its uq row in registers before sAm is written
-            for (int c0 = 0; c0 < kCT; c0 += 8) {
+            for (int c0 = 64 * half; c0 < 64 * half + 64; c0 += 8) {
                 float x[8];
 #pragma unroll
                 for (int e = 0; e < 8; ++e) {
                     const int j = c0 + e;
-                    const bool keep = REV ? (j >= tid) : (j <= tid);
+                    const bool keep = REV ? (j >= row) : (j <= row);
                     float acc = 0.f;
                     if (keep) {
                         const int jg = min(j, valid - 1);
@@ -594,7 +614,7 @@ key_side_tc_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_consta
                     }
                     x[e] = acc;
                 }
-                store_chunk(sAm + (c0 >> 6) * kPanelB, tid, (c0 & 63) >> 3, x);
+                store_chunk(sAm + (c0 >> 6) * kPanelB, row, (c0 & 63) >> 3, x);
             }
         }
         fence_async_smem();
@@ -614,12 +634,11 @@ key_side_tc_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_consta
         }
 
         // ---- state update from U^T (complete since bar_mma1): S <- exp(G_C) S + U^T
+        {
+            float v[kHS];
+            tmem_ld32(tmem_row_addr(tmem, wq, kColU + sb), v);
 #pragma unroll
-        for (int c0 = 0; c0 < kM; c0 += 16) {
-            float v[16];
-            tmem_ld16(tmem_row_addr(tmem, warp, kColU + c0), v);
-#pragma unroll
-            for (int e = 0; e < 16; ++e) S[c0 + e] = fmaf(S[c0 + e], ctl->egc[c0 + e], v[e]);
+            for (int e = 0; e < kHS; ++e) S[e] = fmaf(S[e], ctl->egc[sb + e], v[e]);
         }
         PROF_MARK();
 
@@ -632,20 +651,27 @@ key_side_tc_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_consta
             load_v(it + 1);
             load_q(it + 1);
         }
+        // output rows -> bf16, staged over the intra operands (consumed since bar_mma1), then one
+        // tiled store per 64 columns, clipped at the sequence end
 #pragma unroll
-        for (int c0 = 0; c0 < kDST; c0 += 16) {
-            float v[16];
-            tmem_ld16(tmem_row_addr(tmem, warp, kColO + c0), v);
-            if (tid < valid) {
-                __nv_bfloat16* dst = obase + (size_t)(t0 + tid) * strideD + c0;
-                const uint4 lo = make_uint4(pack_bf16(v[0], v[1]), pack_bf16(v[2], v[3]), pack_bf16(v[4], v[5]), pack_bf16(v[6], v[7]));
-                const uint4 hi = make_uint4(pack_bf16(v[8], v[9]), pack_bf16(v[10], v[11]), pack_bf16(v[12], v[13]), pack_bf16(v[14], v[15]));
-                *reinterpret_cast<uint4*>(dst) = lo;
-                *reinterpret_cast<uint4*>(dst + 8) = hi;
+        for (int c0 = 0; c0 < 64; c0 += 32) {
+            float v[32];
+            tmem_ld32(tmem_row_addr(tmem, wq, kColO + 64 * half + c0), v);
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                const float x[8] = {v[8 * c], v[8 * c + 1], v[8 * c + 2], v[8 * c + 3],
+                                    v[8 * c + 4], v[8 * c + 5], v[8 * c + 6], v[8 * c + 7]};
+                store_chunk(sQt + half * kPanelB, row, (c0 >> 3) + c, x);
             }
         }
+        fence_async_smem();
         tc_fence_before_sync();
         __syncthreads();
+        if (tid == 0 && !ctl->abort) {
+            tma_store_4d(&mapO, sQt, d0, h, t0, b);
+            tma_store_4d(&mapO, sQt + kPanelB, d0 + 64, h, t0, b);
+            bulk_commit();
+        }
         PROF_MARK();
         PROF_DUMP("key_side");
         if (ctl->abort) break;
@@ -659,8 +685,9 @@ key_side_tc_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_consta
         for (int i = 0; i < 200; ++i) __nanosleep(1000);
     } else if (a.Send) {
 #pragma unroll
-        for (int s = 0; s < kM; ++s) a.Send[((size_t)bh * kM + s) * a.D + d0 + tid] = S[s];
+        for (int s = 0; s < kHS; ++s) a.Send[((size_t)bh * kM + sb + s) * a.D + d0 + row] = S[s];
     }
+    if (tid == 0) bulk_wait_read();      // staged output rows must have left before shared memory goes away
     __syncthreads();
     if (warp == 0) {
         __syncwarp();
@@ -677,7 +704,7 @@ cudaError_t prepare(K kernel, size_t smem) {
     if (e != cudaSuccess) return e;
     // each CTA takes the whole tensor memory of its SM: make sure no second CTA can be co-resident
     int per_sm = 0;
-    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, 128, smem);
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kThreads, smem);
     if (e != cudaSuccess) return e;
     return per_sm == 1 ? cudaSuccess : cudaErrorLaunchOutOfResources;
 }
@@ -692,8 +719,9 @@ int tc_chunk() { return kCT; }
 
 cudaError_t launch_value_side_tc(const ValueSideArgs& a, int M, int reverse, cudaStream_t st, int32_t* dev_status) {
     if (M != kM || a.D % kDST != 0) return cudaErrorNotSupported;
-    CUtensorMap mq, mk, mw, mg;
+    CUtensorMap mq, mk, mw, mg, mo;
     cudaError_t e = make_tensor_map_bthd(&mq, a.xq, a.B, a.T, a.H, a.D, kCT, 2);
+    if (e == cudaSuccess) e = make_tensor_map_sliced(&mo, a.out, a.D / kDST, a.B, a.T, a.H, kM, kCT, 4);
     if (e == cudaSuccess) e = make_tensor_map_bthd(&mk, a.xk, a.B, a.T, a.H, a.D, kCT, 2);
     if (e == cudaSuccess) e = make_tensor_map_bthd(&mw, a.w, a.B, a.T, a.H, kM, kCT, 4);
     if (e == cudaSuccess) e = make_tensor_map_bthd(&mg, a.G, a.B, a.T, a.H, kM, kCT, 4);
@@ -702,19 +730,20 @@ cudaError_t launch_value_side_tc(const ValueSideArgs& a, int M, int reverse, cud
     if (reverse) {
         e = prepare(value_side_tc_kernel<true>, kSmemValueSide);
         if (e != cudaSuccess) return e;
-        value_side_tc_kernel<true><<<grid, 128, kSmemValueSide, st>>>(mq, mk, mw, mg, a, dev_status);
+        value_side_tc_kernel<true><<<grid, kThreads, kSmemValueSide, st>>>(mq, mk, mw, mg, mo, a, dev_status);
     } else {
         e = prepare(value_side_tc_kernel<false>, kSmemValueSide);
         if (e != cudaSuccess) return e;
-        value_side_tc_kernel<false><<<grid, 128, kSmemValueSide, st>>>(mq, mk, mw, mg, a, dev_status);
+        value_side_tc_kernel<false><<<grid, kThreads, kSmemValueSide, st>>>(mq, mk, mw, mg, mo, a, dev_status);
     }
     return cudaGetLastError();
 }
 
 cudaError_t launch_key_side_tc(const KeySideArgs& a, int M, int reverse, cudaStream_t st, int32_t* dev_status) {
     if (M != kM || a.D % kDST != 0) return cudaErrorNotSupported;
-    CUtensorMap mv, muq, muk, mg;
+    CUtensorMap mv, muq, muk, mg, mo;
     cudaError_t e = make_tensor_map_bthd(&mv, a.xv, a.B, a.T, a.H, a.D, kCT, 2);
+    if (e == cudaSuccess) e = make_tensor_map_bthd(&mo, a.out, a.B, a.T, a.H, a.D, kCT, 2);
     if (e == cudaSuccess) e = make_tensor_map_bthd(&muq, a.uq, a.B, a.T, a.H, kM, kCT, 4);
     if (e == cudaSuccess) e = make_tensor_map_bthd(&muk, a.uk, a.B, a.T, a.H, kM, kCT, 4);
     if (e == cudaSuccess) e = make_tensor_map_bthd(&mg, a.G, a.B, a.T, a.H, kM, kCT, 4);
@@ -723,11 +752,11 @@ cudaError_t launch_key_side_tc(const KeySideArgs& a, int M, int reverse, cudaStr
     if (reverse) {
         e = prepare(key_side_tc_kernel<true>, kSmemKeySide);
         if (e != cudaSuccess) return e;
-        key_side_tc_kernel<true><<<grid, 128, kSmemKeySide, st>>>(mv, muq, muk, mg, a, dev_status);
+        key_side_tc_kernel<true><<<grid, kThreads, kSmemKeySide, st>>>(mv, muq, muk, mg, mo, a, dev_status);
     } else {
         e = prepare(key_side_tc_kernel<false>, kSmemKeySide);
         if (e != cudaSuccess) return e;
-        key_side_tc_kernel<false><<<grid, 128, kSmemKeySide, st>>>(mv, muq, muk, mg, a, dev_status);
+        key_side_tc_kernel<false><<<grid, kThreads, kSmemKeySide, st>>>(mv, muq, muk, mg, mo, a, dev_status);
     }
     return cudaGetLastError();
 }

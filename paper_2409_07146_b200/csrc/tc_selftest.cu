@@ -6,11 +6,12 @@
 
 namespace gsa {
 
-cudaError_t make_tensor_map_bthd(CUtensorMap* map, const void* base, int B, int T, int H, int D, int box_rows,
-                                 int elem_bytes) {
-    typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                 const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                 CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+namespace {
+typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                             const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                             CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+cudaError_t get_encoder(EncodeFn* out) {
     static EncodeFn encode = nullptr;
     if (encode == nullptr) {
         void* fn = nullptr;
@@ -20,15 +21,33 @@ cudaError_t make_tensor_map_bthd(CUtensorMap* map, const void* base, int B, int 
         if (qres != cudaDriverEntryPointSuccess || fn == nullptr) return cudaErrorNotSupported;
         encode = reinterpret_cast<EncodeFn>(fn);
     }
-    const cuuint64_t dims[4] = {(cuuint64_t)D, (cuuint64_t)H, (cuuint64_t)T, (cuuint64_t)B};
+    *out = encode;
+    return cudaSuccess;
+}
+}  // namespace
+
+cudaError_t make_tensor_map_sliced(CUtensorMap* map, const void* base, int nslice, int B, int T, int H, int D,
+                                   int box_rows, int elem_bytes) {
+    EncodeFn encode;
+    cudaError_t e = get_encoder(&encode);
+    if (e != cudaSuccess) return e;
     const cuuint64_t eb = (cuuint64_t)elem_bytes;
-    const cuuint64_t strides[3] = {(cuuint64_t)D * eb, (cuuint64_t)H * D * eb, (cuuint64_t)T * H * D * eb};
-    const cuuint32_t box[4] = {(cuuint32_t)(128 / elem_bytes), 1, (cuuint32_t)box_rows, 1};
-    const cuuint32_t estr[4] = {1, 1, 1, 1};
-    CUresult r = encode(map, elem_bytes == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, const_cast<void*>(base), dims, strides, box, estr,
-                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+    const cuuint64_t dims[5] = {(cuuint64_t)D, (cuuint64_t)H, (cuuint64_t)T, (cuuint64_t)B, (cuuint64_t)nslice};
+    const cuuint64_t strides[4] = {(cuuint64_t)D * eb, (cuuint64_t)H * D * eb, (cuuint64_t)T * H * D * eb,
+                                   (cuuint64_t)B * T * H * D * eb};
+    const cuuint32_t box[5] = {(cuuint32_t)(128 / elem_bytes), 1, (cuuint32_t)box_rows, 1, 1};
+    const cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+    const cuuint32_t rank = nslice > 0 ? 5 : 4;
+    CUresult r = encode(map, elem_bytes == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32,
+                        rank, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                        CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
+}
+
+cudaError_t make_tensor_map_bthd(CUtensorMap* map, const void* base, int B, int T, int H, int D, int box_rows,
+                                 int elem_bytes) {
+    return make_tensor_map_sliced(map, base, 0, B, T, H, D, box_rows, elem_bytes);
 }
 
 namespace {
@@ -42,7 +61,8 @@ __global__ void __launch_bounds__(128) tc_selftest_kernel(const __grid_constant_
                                                           const __nv_bfloat16* __restrict__ Y, int mode,
                                                           float* __restrict__ D, int32_t* dev_status) {
     extern __shared__ unsigned char smem_raw[];
-    unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    // align by pointer arithmetic (not an integer round trip) so accesses stay in the shared window
+    unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
     unsigned char* sX = smem;                  // 2 panels (TMA)
     unsigned char* sY = smem + 2 * kPanel;     // 2 panels (TMA)
     unsigned char* sW = smem + 4 * kPanel;     // 2 panels written by threads
