@@ -59,8 +59,9 @@ struct Ctl {
     uint64_t bar_x;        // d-sized tiles of the current chunk
     uint64_t bar_g[2];     // value_side: G tile, two stages; key_side: [0] = uk + G tiles
     uint64_t bar_w;        // value_side: weight tile; key_side: uq tile
-    uint64_t bar_mma1;
-    uint64_t bar_mma2;
+    uint64_t bar_p;        // first product of the chunk (P or A) complete
+    uint64_t bar_mma1;     // state and inter-chunk products complete
+    uint64_t bar_mma2;     // intra-chunk product complete
     uint32_t tmem_slot;
     volatile int abort;
     float gc[kM];        // G of the chunk's last valid row
@@ -114,6 +115,7 @@ __device__ __forceinline__ void ctl_init(Ctl* ctl, int tid, int warp) {
         mbar_init(&ctl->bar_g[0], 1);
         mbar_init(&ctl->bar_g[1], 1);
         mbar_init(&ctl->bar_w, 1);
+        mbar_init(&ctl->bar_p, 1);
         mbar_init(&ctl->bar_mma1, 1);
         mbar_init(&ctl->bar_mma2, 1);
         ctl->abort = 0;
@@ -132,22 +134,18 @@ __device__ __forceinline__ void ctl_init(Ctl* ctl, int tid, int warp) {
 template <bool REV>
 __device__ __forceinline__ void store_masked_row(uint32_t tmem, int wq, int row, int half, unsigned char* dst) {
     unsigned char* panel = dst + half * kPanelB;      // columns 64 half .. 64 half + 63
+    float v[64];
+    tmem_ld64(tmem_row_addr(tmem, wq, kColP + 64 * half), v);
 #pragma unroll
-    for (int c0 = 0; c0 < 64; c0 += 32) {
-        float v[32];
-        tmem_ld32(tmem_row_addr(tmem, wq, kColP + 64 * half + c0), v);
+    for (int c = 0; c < 8; ++c) {
+        float x[8];
 #pragma unroll
-        for (int e = 0; e < 32; ++e) {
-            const int j = 64 * half + c0 + e;
+        for (int e = 0; e < 8; ++e) {
+            const int j = 64 * half + 8 * c + e;
             const bool keep = REV ? (j >= row) : (j <= row);
-            v[e] = keep ? v[e] : 0.f;
+            x[e] = keep ? v[8 * c + e] : 0.f;
         }
-#pragma unroll
-        for (int c = 0; c < 4; ++c) {
-            const float x[8] = {v[8 * c], v[8 * c + 1], v[8 * c + 2], v[8 * c + 3],
-                                v[8 * c + 4], v[8 * c + 5], v[8 * c + 6], v[8 * c + 7]};
-            store_chunk(panel, row, (c0 >> 3) + c, x);
-        }
+        store_chunk(panel, row, c, x);
     }
 }
 
@@ -229,9 +227,20 @@ value_side_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_cons
         const int valid = min(kCT, a.T - t0);
         const unsigned char* gt = sG + (2 * (it & 1)) * kPanelB;
         PROF_MARK();
-        if (tid == 0 && it + 1 < nchunks) {
-            bulk_wait_read();     // the output rows staged in that G buffer two chunks ago have left
-            load_g(it + 1);
+        if (tid == 0) {
+            // P = xq xk^T needs nothing but the d-sized tiles: it runs under the operand build
+            if (!mbar_wait(&ctl->bar_x, it & 1)) ctl->abort = 1;
+            tc_fence_after_sync();
+            const uint32_t aQ = smem_u32(sXq), aK = smem_u32(sXk);
+#pragma unroll
+            for (int kk = 0; kk < kDST / 16; ++kk)
+                mma_bf16(tmem + kColP, desc_kmajor(aQ + (kk >> 2) * kPanelB, kk),
+                         desc_kmajor(aK + (kk >> 2) * kPanelB, kk), idescP, kk > 0);
+            mma_commit(&ctl->bar_p);
+            if (it + 1 < nchunks) {
+                bulk_wait_read();     // the output rows staged in that G buffer two chunks ago have left
+                load_g(it + 1);
+            }
         }
         if (!mbar_wait(&ctl->bar_g[it & 1], (it >> 1) & 1)) ctl->abort = 1;
         if (!mbar_wait(&ctl->bar_w, it & 1)) ctl->abort = 1;
@@ -272,22 +281,16 @@ value_side_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_cons
         PROF_MARK();
         fence_async_smem();
         PROF_MARK();
-        if (!mbar_wait(&ctl->bar_x, it & 1)) ctl->abort = 1;
-        PROF_MARK();
         tc_fence_before_sync();
         __syncthreads();
         if (ctl->abort) break;
         PROF_MARK();
 
-        // ---- P = xq xk^T, O = xq S, U = xk^T W~
+        // ---- U = xk^T W~ and O = xq S (they run under the read-out of P)
         if (tid == 0) {
             tc_fence_after_sync();
             const uint32_t aQ = smem_u32(sXq), aK = smem_u32(sXk);
             const uint32_t aS = smem_u32(sSb), aWt = smem_u32(sWt);
-#pragma unroll
-            for (int kk = 0; kk < kDST / 16; ++kk)
-                mma_bf16(tmem + kColP, desc_kmajor(aQ + (kk >> 2) * kPanelB, kk),
-                         desc_kmajor(aK + (kk >> 2) * kPanelB, kk), idescP, kk > 0);
 #pragma unroll
             for (int kk = 0; kk < kCT / 16; ++kk)
                 mma_bf16(tmem + kColU, desc_mnmajor(aK, kk, kPanelB), desc_mnmajor(aWt, kk, kPanelB), idescU, kk > 0);
@@ -298,11 +301,9 @@ value_side_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_cons
             mma_commit(&ctl->bar_mma1);
         }
         PROF_MARK();
-        if (!mbar_wait(&ctl->bar_mma1, it & 1)) ctl->abort = 1;
+        if (!mbar_wait(&ctl->bar_p, it & 1)) ctl->abort = 1;
         tc_fence_after_sync();
         PROF_MARK();
-        // the d-sized tiles are consumed: request the next chunk's
-        if (tid == 0 && it + 1 < nchunks) load_x(it + 1);
 
         if (moderate) {
 #ifndef EXP_NOPM
@@ -327,6 +328,8 @@ value_side_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_cons
         } else {
             // Strong decay: the intra-chunk term with explicit exponent differences on the CUDA
             // cores, straight from the fp32 weight and G tiles.
+            if (!mbar_wait(&ctl->bar_mma1, it & 1)) ctl->abort = 1;    // the inter-chunk product
+            tc_fence_after_sync();
             const int jlo = REV ? row : 0, jhi = REV ? kCT - 1 : row;
             // the accumulator loads are warp-collective: loop bounds are those of the whole warp
             const int wlo = REV ? wq * 32 : 0, whi = REV ? kCT - 1 : wq * 32 + 31;
@@ -372,7 +375,11 @@ value_side_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_cons
             }
         }
 
-        // ---- state update from U (complete since bar_mma1): S <- S exp(G_C) + U
+        // ---- state update from U: S <- S exp(G_C) + U
+        if (!mbar_wait(&ctl->bar_mma1, it & 1)) ctl->abort = 1;
+        tc_fence_after_sync();
+        // the d-sized tiles are consumed: request the next chunk's
+        if (tid == 0 && it + 1 < nchunks) load_x(it + 1);
         {
             float v[kHS];
             tmem_ld32(tmem_row_addr(tmem, wq, kColU + sb), v);
@@ -387,6 +394,8 @@ value_side_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_cons
             ++n_mma2;
             tc_fence_after_sync();
             PROF_MARK();
+            // the masked P is consumed: its buffer takes the next chunk's weight tile
+            if (tid == 0 && it + 1 < nchunks) load_w(it + 1);
             // the scaled rows replace this chunk's G rows in place (each thread reads and rewrites
             // only its own 32 slots) and leave as one tiled store, clipped at the sequence end
             float vo[kHS];
@@ -411,8 +420,8 @@ value_side_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_cons
                 tma_store_5d(&mapO, gt + kPanelB, 32, h, t0, b, slice);
                 bulk_commit();
             }
-            // the weight tile's buffer (masked P) is free again: request the next chunk's weights
-            if (it + 1 < nchunks) load_w(it + 1);
+            // a strong-decay chunk read the weight tile until now
+            if (!moderate && it + 1 < nchunks) load_w(it + 1);
         }
         PROF_MARK();
         PROF_DUMP("value_side");
@@ -508,6 +517,7 @@ key_side_tc_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_consta
     constexpr uint32_t idescV = make_idesc(128, kDST, false, true);   // A x xv (MN-major B)
 
     int it = 0;
+    int n_p = 0;       // completed phases of bar_p (only moderate chunks use it)
     PROF_DECL
     for (; it < nchunks; ++it) {
         const int t0 = chunk_t0(it);
@@ -522,30 +532,38 @@ key_side_tc_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_consta
         PROF_MARK();
 
         const int grow = min(row, valid - 1);
+        // key side first: it needs the uk and G tiles only; the uq tile (which shares its buffer
+        // with the previous chunk's masked A) arrives last
 #pragma unroll
         for (int s0 = sb; s0 < sb + kHS; s0 += 8) {
-            float g[8], uq[8], uk[8], qb[8], kb[8], qt[8], kt[8];
+            float g[8], uk[8], kb[8], kt[8];
             tile_row8(sG, grow, s0, g);
-            tile_row8(sUq, row, s0, uq);
             tile_row8(sUk, row, s0, uk);
 #pragma unroll
             for (int e = 0; e < 8; ++e) {
+                // state term: forward K- = uk exp(G_C - G), reverse uk exp(G); intra term: uk exp(-+G)
                 const float eg = __expf(g[e]);
-                const float einv = __expf(-g[e]);
-                const float egc_g = __expf(ctl->gc[s0 + e] - g[e]);
-                // state terms: forward Q- = uq exp(G), K- = uk exp(G_C - G); reverse swapped
-                qb[e] = uq[e] * (REV ? egc_g : eg);
-                kb[e] = uk[e] * (REV ? eg : egc_g);
-                // intra terms (used by a moderate chunk only): exp(+-G) on the two sides
-                qt[e] = uq[e] * (REV ? einv : eg);
-                kt[e] = uk[e] * (REV ? eg : einv);
+                kb[e] = uk[e] * (REV ? eg : __expf(ctl->gc[s0 + e] - g[e]));
+                kt[e] = uk[e] * (REV ? eg : __expf(-g[e]));
+            }
+            store_chunk(sKb, row, s0 >> 3, kb);
+            if (moderate) store_chunk(sKt, row, s0 >> 3, kt);
+        }
+        if (!mbar_wait(&ctl->bar_w, it & 1)) ctl->abort = 1;
+#pragma unroll
+        for (int s0 = sb; s0 < sb + kHS; s0 += 8) {
+            float g[8], uq[8], qb[8], qt[8];
+            tile_row8(sG, grow, s0, g);
+            tile_row8(sUq, row, s0, uq);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                // state term: forward Q- = uq exp(G), reverse uq exp(G_C - G); intra term: uq exp(+-G)
+                const float eg = __expf(g[e]);
+                qb[e] = uq[e] * (REV ? __expf(ctl->gc[s0 + e] - g[e]) : eg);
+                qt[e] = uq[e] * (REV ? __expf(-g[e]) : eg);
             }
             store_chunk(sQb, row, s0 >> 3, qb);
-            store_chunk(sKb, row, s0 >> 3, kb);
-            if (moderate) {
-                store_chunk(sQt, row, s0 >> 3, qt);
-                store_chunk(sKt, row, s0 >> 3, kt);
-            }
+            if (moderate) store_chunk(sQt, row, s0 >> 3, qt);
         }
         store_state_row<false>(sSb, row, sb, S, nullptr);
         fence_async_smem();
@@ -566,6 +584,7 @@ key_side_tc_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_consta
 #pragma unroll
                 for (int kk = 0; kk < kM / 16; ++kk)
                     mma_bf16(tmem + kColP, desc_kmajor(aQt, kk), desc_kmajor(aKt, kk), idescA, kk > 0);
+                mma_commit(&ctl->bar_p);     // the state products below run under the read-out of A
             }
 #pragma unroll
             for (int kk = 0; kk < kCT / 16; ++kk)
@@ -578,7 +597,10 @@ key_side_tc_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_consta
             if (moderate && it + 1 < nchunks) load_kg(it + 1);
         }
         PROF_MARK();
-        if (!mbar_wait(&ctl->bar_mma1, it & 1)) ctl->abort = 1;
+        if (moderate) {
+            if (!mbar_wait(&ctl->bar_p, n_p & 1)) ctl->abort = 1;
+            ++n_p;
+        }
         tc_fence_after_sync();
         PROF_MARK();
 
@@ -633,7 +655,9 @@ key_side_tc_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_consta
             if (!moderate && it + 1 < nchunks) load_kg(it + 1);
         }
 
-        // ---- state update from U^T (complete since bar_mma1): S <- exp(G_C) S + U^T
+        // ---- state update from U^T: S <- exp(G_C) S + U^T
+        if (!mbar_wait(&ctl->bar_mma1, it & 1)) ctl->abort = 1;
+        tc_fence_after_sync();
         {
             float v[kHS];
             tmem_ld32(tmem_row_addr(tmem, wq, kColU + sb), v);
