@@ -88,7 +88,7 @@ def step_flops(w: W.Workload) -> float:
 
 # ----------------------------------------------------------------------------- clocks
 class ClockSampler:
-    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+    QUERY = ("index,clocks.sm,clocks.max.sm,utilization.gpu,clocks_event_reasons.active,"
              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
@@ -103,7 +103,7 @@ class ClockSampler:
             os.close(fd)
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--id={self.idx}", f"--query-gpu={self.QUERY}",
-                 "--format=csv,noheader,nounits", "-lms", "200"],
+                 "--format=csv,noheader,nounits", "-lms", "50"],
                 stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
         except Exception:
             self.proc = None
@@ -125,6 +125,8 @@ class ClockSampler:
                 if len(f) < 9:
                     continue
                 try:
+                    if float(f[3]) < 50.0:      # keep samples taken under load only
+                        continue
                     sm.append(float(f[1])); mx.append(float(f[2]))
                 except ValueError:
                     continue
@@ -249,13 +251,23 @@ def run_ours(args):
             dist.all_reduce(ms, op=dist.ReduceOp.MAX)
         return float(ms.item())
 
-    for _ in range(max(args.warmup, 3)):
-        step(d_in)
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
+    for _ in range(max(args.warmup, 3)):
+        step(d_in)
     total_ms = timed(lambda: step(d_in), args.steps)
+    # The timed region lasts a few tens of milliseconds, shorter than nvidia-smi's sampling
+    # period: keep the same steps running (untimed) for about a second so that the sampler
+    # sees the clocks of exactly this load.
+    t_end = time.perf_counter() + 1.2
+    while time.perf_counter() < t_end:
+        for _ in range(20):
+            step(d_in)
+        torch.cuda.synchronize()
     clocks = sampler.stop() if rank == 0 else {}
+    if rank == 0:
+        clocks["note"] = "nvidia-smi samples (50 ms period, utilisation >= 50%) over warm-up, the timed steps and 1.2 s more of the same steps"
     ms_step = total_ms / args.steps
     value = world * w.tokens / (ms_step * 1e-3)
     if int(status.item()) != 0:

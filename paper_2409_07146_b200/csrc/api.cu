@@ -78,7 +78,7 @@ Workspace carve(const gsa_params_t& p, int which, void* ws) {
         w.dppart = c.take(mt * s.v);
         w.dIk = c.take(mt * s.k);
         w.dIv = c.take(mt * s.v);
-        w.chunk_tot = c.take((size_t)p.B * p.H * ((p.T + kChunk - 1) / kChunk) * p.m);
+        w.chunk_tot = c.take((size_t)p.B * p.H * gate_grad_blocks(p.T) * p.m);
         w.KT = c.take((size_t)p.B * p.H * p.m * p.d_k);
         w.VT = c.take((size_t)p.B * p.H * p.m * p.d_v);
     }

@@ -1,9 +1,12 @@
 // tcgen05 (bf16 tensor-core) versions of the two chunk primitives of Algorithm 1.
 //
-// One CTA of 256 threads owns one (batch, head) and one 128-wide slice of the head
-// dimension and walks the chunks (128 tokens each) in order.  Threads r and r + 128 share
-// row r of the chunk, which is channel r of the state slice and TMEM lane r of every
-// accumulator; the first works on slots (or columns) 0..31 (0..63), the second on the rest.
+// One CTA owns one (batch, head) and one 128-wide slice of the head dimension and walks the
+// chunks (128 tokens each) in order.  It has 256 compute threads and one issuing warp.
+// Compute threads r and r + 128 share row r of the chunk, which is channel r of the state
+// slice and TMEM lane r of every accumulator; the first works on slots (or columns) 0..31
+// (0..63), the second on the rest.  One lane of the issuing warp requests every tile copy
+// and issues every MMA, running ahead of the compute threads; the two sides meet on
+// mbarriers only.
 // Per chunk:
 //   * every tile -- the d-sized ones (xq, xk / xv, bf16) and the slot-sized ones (weights,
 //     cumulative log gate G, fp32) -- arrives by TMA with the 128-byte swizzle, requested as
@@ -12,7 +15,7 @@
 //   * each thread reads its own row of the slot-sized tiles (conflict-free under the
 //     swizzle), scales it by the decay factors and writes bf16 operand rows;
 //   * all contractions run as tcgen05.mma (M = 128) with fp32 accumulators in tensor
-//     memory; thread 0 issues them and commits to an mbarrier that everybody waits on;
+//     memory, committed to mbarriers that the compute threads wait on;
 //   * the fp32 master copy of the state slice stays in registers (64 per thread); its bf16
 //     copy for the next chunk's state product is rewritten every chunk.
 // Decay inside a chunk is factorised as exp(G_i) * exp(-G_j) while the chunk's total
@@ -34,20 +37,22 @@ constexpr int kDST = 128;              // head-dimension slice per CTA
 constexpr int kM = 64;                 // slots
 constexpr int kPanelB = 128 * 128;     // bytes of a 128-row operand panel
 constexpr uint32_t kTmemCols = 512;
-constexpr int kThreads = 256;
+constexpr int kComputeThreads = 256;   // 8 warps: two threads per chunk row
+constexpr int kThreads = kComputeThreads + 32;   // + the issuing warp (TMA and MMA), one lane active
 constexpr int kHS = kM / 2;            // slots per thread
 
 // accumulator columns
 constexpr int kColP = 0;       // P / A           [128 x 128]
 constexpr int kColO = 128;     // inter (+ intra for key_side) output
 constexpr int kColU = 256;     // state update    [128 x 64]
+constexpr int kColO2 = 320;    // value_side: intra-chunk output [128 x 64]
 
 // Optional phase timing for development builds (-DGSA_TC_PROF): CTA 0 prints, for its fifth
 // chunk, the SM clock at each phase boundary.
 #ifdef GSA_TC_PROF
 #define PROF_DECL long long prof_t[32]; int prof_n = 0;
 #define PROF_MARK() do { if (prof_n < 32) prof_t[prof_n++] = clock64(); } while (0)
-#define PROF_DUMP(name) do { if (blockIdx.x == 0 && blockIdx.y == 0 && tid == 0 && it == 4) { \
+#define PROF_DUMP(name) do { if (blockIdx.x == 0 && blockIdx.y == 0 && ((tid == 0 && it == 6) || (tid == 256 && it == 4))) { \
     printf("%s:", name); for (int i_ = 1; i_ < prof_n; ++i_) printf(" %lld", prof_t[i_] - prof_t[i_ - 1]); printf("\n"); } prof_n = 0; } while (0)
 #else
 #define PROF_DECL
@@ -56,14 +61,23 @@ constexpr int kColU = 256;     // state update    [128 x 64]
 #endif
 
 struct Ctl {
+    // filled by TMA
     uint64_t bar_x;        // d-sized tiles of the current chunk
     uint64_t bar_g[2];     // value_side: G tile, two stages; key_side: [0] = uk + G tiles
     uint64_t bar_w;        // value_side: weight tile; key_side: uq tile
+    // signalled by tcgen05.commit
     uint64_t bar_p;        // first product of the chunk (P or A) complete
     uint64_t bar_mma1;     // state and inter-chunk products complete
     uint64_t bar_mma2;     // intra-chunk product complete
+    // signalled by the compute threads (one arrival after their barrier)
+    uint64_t bar_ops;      // operand rows of the chunk are in shared memory
+    uint64_t bar_pm;       // masked P / A rows are in shared memory
+    uint64_t bar_out;      // output rows are staged (or the chunk is otherwise done)
+    uint64_t bar_sb;       // value_side: the state copy for the next chunk is written
+                           // key_side: (issuing warp ->) the output staging buffer is free again
     uint32_t tmem_slot;
     volatile int abort;
+    volatile int moderate[2];   // decision of the chunk, by chunk parity
     float gc[kM];        // G of the chunk's last valid row
     float egc[kM];       // exp(gc)
 };
@@ -96,8 +110,26 @@ __device__ __forceinline__ void store_state_row(unsigned char* panel, int row, i
     }
 }
 
+// Barrier over the 256 compute threads only (the issuing warp runs ahead on its own).
+__device__ __forceinline__ void compute_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
+__device__ __forceinline__ bool compute_sync_and(bool pred) {
+    uint32_t out;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.b32 q, %1, 0;\n\t"
+        "bar.red.and.pred p, 1, 256, q;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(out)
+        : "r"((uint32_t)pred)
+        : "memory");
+    return out != 0;
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+
 // Publish the G row of the chunk's last valid token, its exponential and decide whether the
-// chunk's decay is moderate.  One __syncthreads inside; the result is uniform.
+// chunk's decay is moderate.  One compute-thread barrier inside; the result is uniform.
 __device__ __forceinline__ bool publish_chunk_decay(Ctl* ctl, int tid, const unsigned char* gtile, int last_row) {
     bool fine = true;
     if (tid < kM) {
@@ -106,7 +138,7 @@ __device__ __forceinline__ bool publish_chunk_decay(Ctl* ctl, int tid, const uns
         ctl->egc[tid] = __expf(g);
         fine = g >= kFactorisedDecayMin;
     }
-    return __syncthreads_and(fine) != 0;
+    return compute_sync_and(fine);
 }
 
 __device__ __forceinline__ void ctl_init(Ctl* ctl, int tid, int warp) {
@@ -118,6 +150,10 @@ __device__ __forceinline__ void ctl_init(Ctl* ctl, int tid, int warp) {
         mbar_init(&ctl->bar_p, 1);
         mbar_init(&ctl->bar_mma1, 1);
         mbar_init(&ctl->bar_mma2, 1);
+        mbar_init(&ctl->bar_ops, 1);
+        mbar_init(&ctl->bar_pm, 1);
+        mbar_init(&ctl->bar_out, 1);
+        mbar_init(&ctl->bar_sb, 1);
         ctl->abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -149,6 +185,12 @@ __device__ __forceinline__ void store_masked_row(uint32_t tmem, int wq, int row,
     }
 }
 
+// wait helper of the loops below: a wait that expires flags the CTA
+#define WAIT_OR_ABORT(bar, parity)                          \
+    do {                                                    \
+        if (!mbar_wait(bar, parity)) ctl->abort = 1;        \
+    } while (0)
+
 // ======================================================================================
 // value_side: out_i[s] = sum_{j<=i} <xq_i, xk_j> w_j[s] decay_ij[s]  + decayed (xq_i S)[s]
 // ======================================================================================
@@ -170,7 +212,7 @@ value_side_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_cons
     unsigned char* sSb = sWt + kPanelB;              // state copy, MN-major B [128][64]          (16 KB)
     Ctl* ctl = reinterpret_cast<Ctl*>(sSb + kPanelB);
 
-    const int tid = threadIdx.x, warp = tid >> 5, wq = warp & 3, half = tid >> 7, row = tid & 127;
+    const int tid = threadIdx.x, warp = tid >> 5, wq = warp & 3, half = (tid >> 7) & 1, row = tid & 127;
     const int sb = kHS * half;          // this thread's first slot
     const int bh = blockIdx.x, slice = blockIdx.y, b = bh / a.H, h = bh % a.H;
     const int d0 = slice * kDST;
@@ -179,253 +221,298 @@ value_side_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_cons
 
     ctl_init(ctl, tid, warp);
     const uint32_t tmem = ctl->tmem_slot;
-
     const int nchunks = (a.T + kCT - 1) / kCT;
     auto chunk_t0 = [&](int it) { return (REV ? nchunks - 1 - it : it) * kCT; };
-    auto load_x = [&](int it) {
-        const int t = chunk_t0(it);
-        mbar_expect_tx(&ctl->bar_x, 4 * kPanelB);
-        tma_load_4d(sXq, &mapQ, &ctl->bar_x, d0, h, t, b);
-        tma_load_4d(sXq + kPanelB, &mapQ, &ctl->bar_x, d0 + 64, h, t, b);
-        tma_load_4d(sXk, &mapK, &ctl->bar_x, d0, h, t, b);
-        tma_load_4d(sXk + kPanelB, &mapK, &ctl->bar_x, d0 + 64, h, t, b);
-    };
-    auto load_g = [&](int it) {
-        const int t = chunk_t0(it), st = it & 1;
-        mbar_expect_tx(&ctl->bar_g[st], 2 * kPanelB);
-        tma_load_4d(sG + (2 * st) * kPanelB, &mapG, &ctl->bar_g[st], 0, h, t, b);
-        tma_load_4d(sG + (2 * st + 1) * kPanelB, &mapG, &ctl->bar_g[st], 32, h, t, b);
-    };
-    auto load_w = [&](int it) {
-        const int t = chunk_t0(it);
-        mbar_expect_tx(&ctl->bar_w, 2 * kPanelB);
-        tma_load_4d(sW, &mapW, &ctl->bar_w, 0, h, t, b);
-        tma_load_4d(sW + kPanelB, &mapW, &ctl->bar_w, 32, h, t, b);
-    };
-    if (tid == 0) {
-        prefetch_tmap(&mapQ); prefetch_tmap(&mapK); prefetch_tmap(&mapW); prefetch_tmap(&mapG); prefetch_tmap(&mapO);
-        load_g(0);
-        load_w(0);
-        load_x(0);
-    }
 
-    // state slice: S[c = tid][s]
-    float S[kHS];
-#pragma unroll
-    for (int s = 0; s < kHS; ++s) S[s] = a.S0 ? a.S0[((size_t)bh * kM + sb + s) * a.D + d0 + row] : 0.f;
-
-    constexpr uint32_t idescP = make_idesc(128, 128, false, false);  // xq xk^T
-    constexpr uint32_t idescO = make_idesc(128, kM, false, true);    // xq x state copy (MN-major B)
-    constexpr uint32_t idescU = make_idesc(128, kM, true, true);     // xk^T (MN-major A) x W~ (MN-major B)
-    constexpr uint32_t idescI = make_idesc(128, kM, false, true);    // Pm x W' (MN-major B)
-
-    int it = 0;
-    int n_mma2 = 0;    // completed phases of bar_mma2 (only moderate chunks use it)
-    PROF_DECL
-    for (; it < nchunks; ++it) {
-        const int t0 = chunk_t0(it);
-        const int valid = min(kCT, a.T - t0);
-        const unsigned char* gt = sG + (2 * (it & 1)) * kPanelB;
-        PROF_MARK();
-        if (tid == 0) {
-            // P = xq xk^T needs nothing but the d-sized tiles: it runs under the operand build
-            if (!mbar_wait(&ctl->bar_x, it & 1)) ctl->abort = 1;
-            tc_fence_after_sync();
-            const uint32_t aQ = smem_u32(sXq), aK = smem_u32(sXk);
-#pragma unroll
-            for (int kk = 0; kk < kDST / 16; ++kk)
-                mma_bf16(tmem + kColP, desc_kmajor(aQ + (kk >> 2) * kPanelB, kk),
-                         desc_kmajor(aK + (kk >> 2) * kPanelB, kk), idescP, kk > 0);
-            mma_commit(&ctl->bar_p);
-            if (it + 1 < nchunks) {
-                bulk_wait_read();     // the output rows staged in that G buffer two chunks ago have left
-                load_g(it + 1);
-            }
-        }
-        if (!mbar_wait(&ctl->bar_g[it & 1], (it >> 1) & 1)) ctl->abort = 1;
-        if (!mbar_wait(&ctl->bar_w, it & 1)) ctl->abort = 1;
-        PROF_MARK();
-        const bool moderate = publish_chunk_decay(ctl, tid, gt, valid - 1);
-        if (ctl->abort) break;
-        PROF_MARK();
-
-        // ---- this token's slot rows -> operand rows (rows past the end: zero weights)
-        const int grow = min(row, valid - 1);
-#pragma unroll
-        for (int s0 = sb; s0 < sb + kHS; s0 += 8) {
-            float g[8], w[8], wp[8], wt[8];
-            tile_row8(gt, grow, s0, g);
-            tile_row8(sW, row, s0, w);
-            // Branch-free over the elements (a branch per element would serialise the exps):
-            //   reverse           : intra = state-update weights = w exp(G)
-            //   forward, moderate : intra w exp(-G); state update = intra * exp(G_C)
-            //   forward, strong   : state update w exp(G_C - G); no intra operand
-#pragma unroll
-            for (int e = 0; e < 8; ++e) {
-                const float off = (REV || moderate) ? 0.f : ctl->gc[s0 + e];
-                const float mul = (!REV && moderate) ? ctl->egc[s0 + e] : 1.f;
-                wp[e] = w[e] * __expf(REV ? g[e] : off - g[e]);
-                wt[e] = wp[e] * mul;
-            }
-#ifndef EXP_NOBUILDSTORE
-            store_chunk(sWt, row, s0 >> 3, wt);
-            if (moderate) store_chunk(sWp, row, s0 >> 3, wp);
-#else
-            if (wt[0] + wp[3] == 1234.5f) store_chunk(sWt, row, s0 >> 3, wt);
-#endif
-        }
-        PROF_MARK();
-        // state copy for the inter-chunk product; a moderate reverse chunk folds exp(G_C) in
-        if (REV && moderate) store_state_row<true>(sSb, row, sb, S, ctl->egc);
-        else store_state_row<false>(sSb, row, sb, S, nullptr);
-        PROF_MARK();
-        fence_async_smem();
-        PROF_MARK();
-        tc_fence_before_sync();
-        __syncthreads();
-        if (ctl->abort) break;
-        PROF_MARK();
-
-        // ---- U = xk^T W~ and O = xq S (they run under the read-out of P)
-        if (tid == 0) {
-            tc_fence_after_sync();
-            const uint32_t aQ = smem_u32(sXq), aK = smem_u32(sXk);
-            const uint32_t aS = smem_u32(sSb), aWt = smem_u32(sWt);
-#pragma unroll
-            for (int kk = 0; kk < kCT / 16; ++kk)
-                mma_bf16(tmem + kColU, desc_mnmajor(aK, kk, kPanelB), desc_mnmajor(aWt, kk, kPanelB), idescU, kk > 0);
-#pragma unroll
-            for (int kk = 0; kk < kDST / 16; ++kk)
-                mma_bf16(tmem + kColO, desc_kmajor(aQ + (kk >> 2) * kPanelB, kk),
-                         desc_mnmajor(aS, kk, kPanelB), idescO, kk > 0);
-            mma_commit(&ctl->bar_mma1);
-        }
-        PROF_MARK();
-        if (!mbar_wait(&ctl->bar_p, it & 1)) ctl->abort = 1;
-        tc_fence_after_sync();
-        PROF_MARK();
-
-        if (moderate) {
-#ifndef EXP_NOPM
-            store_masked_row<REV>(tmem, wq, row, half, sPm);    // overwrites the weight tile: all rows were read
-#endif
-            fence_async_smem();
-        }
-        tc_fence_before_sync();
-        __syncthreads();
-        if (ctl->abort) break;
-        PROF_MARK();
-        if (moderate) {
-            if (tid == 0) {
+    if (warp == kComputeThreads / 32) {
+        // =============================== issuing warp: TMA loads / stores and all MMAs
+        if (tid == kComputeThreads) {
+            auto load_x = [&](int it) {
+                const int t = chunk_t0(it);
+                mbar_expect_tx(&ctl->bar_x, 4 * kPanelB);
+                tma_load_4d(sXq, &mapQ, &ctl->bar_x, d0, h, t, b);
+                tma_load_4d(sXq + kPanelB, &mapQ, &ctl->bar_x, d0 + 64, h, t, b);
+                tma_load_4d(sXk, &mapK, &ctl->bar_x, d0, h, t, b);
+                tma_load_4d(sXk + kPanelB, &mapK, &ctl->bar_x, d0 + 64, h, t, b);
+            };
+            auto load_g = [&](int it) {
+                const int t = chunk_t0(it), st = it & 1;
+                mbar_expect_tx(&ctl->bar_g[st], 2 * kPanelB);
+                tma_load_4d(sG + (2 * st) * kPanelB, &mapG, &ctl->bar_g[st], 0, h, t, b);
+                tma_load_4d(sG + (2 * st + 1) * kPanelB, &mapG, &ctl->bar_g[st], 32, h, t, b);
+            };
+            auto load_w = [&](int it) {
+                const int t = chunk_t0(it);
+                mbar_expect_tx(&ctl->bar_w, 2 * kPanelB);
+                tma_load_4d(sW, &mapW, &ctl->bar_w, 0, h, t, b);
+                tma_load_4d(sW + kPanelB, &mapW, &ctl->bar_w, 32, h, t, b);
+            };
+            prefetch_tmap(&mapQ); prefetch_tmap(&mapK); prefetch_tmap(&mapW); prefetch_tmap(&mapG); prefetch_tmap(&mapO);
+            load_g(0);
+            load_w(0);
+            load_x(0);
+            constexpr uint32_t idescP = make_idesc(128, 128, false, false);  // xq xk^T
+            constexpr uint32_t idescO = make_idesc(128, kM, false, true);    // xq x state copy (MN-major B)
+            constexpr uint32_t idescU = make_idesc(128, kM, true, true);     // xk^T (MN-major A) x W~ (MN-major B)
+            constexpr uint32_t idescI = make_idesc(128, kM, false, true);    // Pm x W' (MN-major B)
+            // base descriptors of every operand (K step 0); advancing along K is one add each
+            const uint64_t dQk = desc_kmajor(smem_u32(sXq), 0), dKk = desc_kmajor(smem_u32(sXk), 0);
+            const uint64_t dKm = desc_mnmajor(smem_u32(sXk), 0, kPanelB), dWt = desc_mnmajor(smem_u32(sWt), 0, kPanelB);
+            const uint64_t dS = desc_mnmajor(smem_u32(sSb), 0, kPanelB), dWp = desc_mnmajor(smem_u32(sWp), 0, kPanelB);
+            const uint64_t dP = desc_kmajor(smem_u32(sPm), 0);
+            // byte offset of K step kk: K-major operands walk 32 bytes inside a 64-column panel,
+            // MN-major operands walk 16 rows (2048 bytes)
+            auto kmaj = [](int kk) { return (uint32_t)((kk >> 2) * kPanelB + (kk & 3) * 32); };
+            auto mnmaj = [](int kk) { return (uint32_t)(kk * 2048); };
+            int n_mod = 0;      // moderate chunks so far (phases of bar_pm / bar_mma2)
+            PROF_DECL
+            for (int it = 0; it < nchunks && !ctl->abort; ++it) {
+                const int t0 = chunk_t0(it);
+                PROF_MARK();
+                const unsigned char* gt = sG + (2 * (it & 1)) * kPanelB;
+                // P = xq xk^T needs nothing but the d-sized tiles: it runs under the operand build
+                WAIT_OR_ABORT(&ctl->bar_x, it & 1);
                 tc_fence_after_sync();
-                const uint32_t aP = smem_u32(sPm), aWp = smem_u32(sWp);
+                PROF_MARK();
+#pragma unroll
+                for (int kk = 0; kk < kDST / 16; ++kk)
+                    mma_bf16(tmem + kColP, desc_advance(dQk, kmaj(kk)), desc_advance(dKk, kmaj(kk)), idescP, kk > 0);
+                mma_commit(&ctl->bar_p);
+                // so does the inter-chunk product O = xq S: the state copy was written at the end
+                // of the previous chunk
+                WAIT_OR_ABORT(&ctl->bar_sb, it & 1);
+                tc_fence_after_sync();
+#pragma unroll
+                for (int kk = 0; kk < kDST / 16; ++kk)
+                    mma_bf16(tmem + kColO, desc_advance(dQk, kmaj(kk)), desc_advance(dS, mnmaj(kk)), idescO, kk > 0);
+                PROF_MARK();
+                if (it + 1 < nchunks) {
+                    bulk_wait_read();     // the output rows staged in that G buffer one chunk ago have left
+                    load_g(it + 1);
+                }
+                // U = xk^T W~ once the operand rows are there
+                PROF_MARK();
+                WAIT_OR_ABORT(&ctl->bar_ops, it & 1);
+                tc_fence_after_sync();
+                PROF_MARK();
+                const bool moderate = ctl->moderate[it & 1] != 0;
 #pragma unroll
                 for (int kk = 0; kk < kCT / 16; ++kk)
-                    mma_bf16(tmem + kColO, desc_kmajor(aP + (kk >> 2) * kPanelB, kk),
-                             desc_mnmajor(aWp, kk, kPanelB), idescI, true);
-                mma_commit(&ctl->bar_mma2);
+                    mma_bf16(tmem + kColU, desc_advance(dKm, mnmaj(kk)), desc_advance(dWt, mnmaj(kk)), idescU, kk > 0);
+                mma_commit(&ctl->bar_mma1);
+                PROF_MARK();
+                if (moderate) {
+                    WAIT_OR_ABORT(&ctl->bar_pm, n_mod & 1);
+                    tc_fence_after_sync();
+                    PROF_MARK();
+#pragma unroll
+                    for (int kk = 0; kk < kCT / 16; ++kk)
+                        mma_bf16(tmem + kColO2, desc_advance(dP, kmaj(kk)), desc_advance(dWp, mnmaj(kk)), idescI, kk > 0);
+                    mma_commit(&ctl->bar_mma2);
+                    PROF_MARK();
+                }
+                // the d-sized tiles are consumed once U and O are done: request the next chunk's
+                WAIT_OR_ABORT(&ctl->bar_mma1, it & 1);
+                PROF_MARK();
+                if (it + 1 < nchunks) load_x(it + 1);
+                if (moderate) {
+                    // the masked P is consumed: its buffer takes the next chunk's weight tile
+                    WAIT_OR_ABORT(&ctl->bar_mma2, n_mod & 1);
+                    ++n_mod;
+                    if (it + 1 < nchunks) load_w(it + 1);
+                }
+                PROF_MARK();
+                WAIT_OR_ABORT(&ctl->bar_out, it & 1);
+                PROF_MARK();
+                PROF_DUMP("value_side issue");
+                if (ctl->abort) break;
+                if (moderate) {
+                    tma_store_5d(&mapO, gt, 0, h, t0, b, slice);
+                    tma_store_5d(&mapO, gt + kPanelB, 32, h, t0, b, slice);
+                    bulk_commit();
+                } else if (it + 1 < nchunks) {
+                    load_w(it + 1);       // a strong-decay chunk read the weight tile until now
+                }
             }
-        } else {
-            // Strong decay: the intra-chunk term with explicit exponent differences on the CUDA
-            // cores, straight from the fp32 weight and G tiles.
-            if (!mbar_wait(&ctl->bar_mma1, it & 1)) ctl->abort = 1;    // the inter-chunk product
+            bulk_wait_read();      // staged output rows must have left before shared memory goes away
+        }
+    } else {
+        // =============================== compute threads
+        // state slice: S[c = row][s], slots sb .. sb+31
+        float S[kHS];
+#pragma unroll
+        for (int s = 0; s < kHS; ++s) S[s] = a.S0 ? a.S0[((size_t)bh * kM + sb + s) * a.D + d0 + row] : 0.f;
+
+        // bf16 copy of the state for the first chunk's inter-chunk product
+        store_state_row<false>(sSb, row, sb, S, nullptr);
+        fence_async_smem();
+        compute_sync();
+        if (tid == 0) mbar_arrive(&ctl->bar_sb);
+
+        int n_mod = 0;
+        PROF_DECL
+        for (int it = 0; it < nchunks; ++it) {
+            const int t0 = chunk_t0(it);
+            const int valid = min(kCT, a.T - t0);
+            PROF_MARK();
+            const unsigned char* gt = sG + (2 * (it & 1)) * kPanelB;
+            WAIT_OR_ABORT(&ctl->bar_g[it & 1], (it >> 1) & 1);
+            WAIT_OR_ABORT(&ctl->bar_w, it & 1);
+            PROF_MARK();
+            const bool moderate = publish_chunk_decay(ctl, tid, gt, valid - 1);
+            if (ctl->abort) break;
+            PROF_MARK();
+
+            // ---- this token's slot rows -> operand rows (rows past the end: zero weights)
+            const int grow = min(row, valid - 1);
+#pragma unroll
+            for (int s0 = sb; s0 < sb + kHS; s0 += 8) {
+                float g[8], w[8], wp[8], wt[8];
+                tile_row8(gt, grow, s0, g);
+                tile_row8(sW, row, s0, w);
+                // Branch-free over the elements (a branch per element would serialise the exps):
+                //   reverse           : intra = state-update weights = w exp(G)
+                //   forward, moderate : intra w exp(-G); state update = intra * exp(G_C)
+                //   forward, strong   : state update w exp(G_C - G); no intra operand
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                    const float off = (REV || moderate) ? 0.f : ctl->gc[s0 + e];
+                    const float mul = (!REV && moderate) ? ctl->egc[s0 + e] : 1.f;
+#ifdef EXP_NOEXP
+                    wp[e] = w[e] * (REV ? g[e] : off - g[e]);
+#else
+                    wp[e] = w[e] * __expf(REV ? g[e] : off - g[e]);
+#endif
+                    wt[e] = wp[e] * mul;
+                }
+#ifndef EXP_NOBUILDSTORE
+                store_chunk(sWt, row, s0 >> 3, wt);
+                if (moderate) store_chunk(sWp, row, s0 >> 3, wp);
+#else
+                if (wt[0] + wp[3] == 1234.5f) store_chunk(sWt, row, s0 >> 3, wt);
+#endif
+            }
+            fence_async_smem();
+            if (tid == 0) ctl->moderate[it & 1] = moderate;
+            compute_sync();                     // every row is written and the weight tile is read
+            if (tid == 0) mbar_arrive(&ctl->bar_ops);
+            PROF_MARK();
+
+            WAIT_OR_ABORT(&ctl->bar_p, it & 1);
             tc_fence_after_sync();
-            const int jlo = REV ? row : 0, jhi = REV ? kCT - 1 : row;
-            // the accumulator loads are warp-collective: loop bounds are those of the whole warp
-            const int wlo = REV ? wq * 32 : 0, whi = REV ? kCT - 1 : wq * 32 + 31;
-            for (int s0 = sb; s0 < sb + kHS; s0 += 16) {
-                float gi[16], acc[16], tmp[8];
-                tile_row8(gt, grow, s0, tmp);
+            PROF_MARK();
+            if (moderate) {
+                store_masked_row<REV>(tmem, wq, row, half, sPm);    // overwrites the weight tile
+                fence_async_smem();
+                tc_fence_before_sync();
+                compute_sync();
+                if (tid == 0) mbar_arrive(&ctl->bar_pm);
+            } else {
+                // Strong decay: the intra-chunk term with explicit exponent differences on the CUDA
+                // cores, straight from the fp32 weight and G tiles.
+                WAIT_OR_ABORT(&ctl->bar_mma1, it & 1);    // the inter-chunk product
+                tc_fence_after_sync();
+                const int jlo = REV ? row : 0, jhi = REV ? kCT - 1 : row;
+                // the accumulator loads are warp-collective: loop bounds are those of the whole warp
+                const int wlo = REV ? wq * 32 : 0, whi = REV ? kCT - 1 : wq * 32 + 31;
+                for (int s0 = sb; s0 < sb + kHS; s0 += 16) {
+                    float gi[16], acc[16], tmp[8];
+                    tile_row8(gt, grow, s0, tmp);
 #pragma unroll
-                for (int e = 0; e < 8; ++e) gi[e] = tmp[e];
-                tile_row8(gt, grow, s0 + 8, tmp);
+                    for (int e = 0; e < 8; ++e) gi[e] = tmp[e];
+                    tile_row8(gt, grow, s0 + 8, tmp);
 #pragma unroll
-                for (int e = 0; e < 8; ++e) gi[8 + e] = tmp[e];
+                    for (int e = 0; e < 8; ++e) gi[8 + e] = tmp[e];
 #pragma unroll
-                for (int e = 0; e < 16; ++e) acc[e] = 0.f;
-                for (int c0 = wlo; c0 <= whi; c0 += 16) {
-                    float v[16];
-                    tmem_ld16(tmem_row_addr(tmem, wq, kColP + c0), v);
+                    for (int e = 0; e < 16; ++e) acc[e] = 0.f;
+                    for (int c0 = wlo; c0 <= whi; c0 += 16) {
+                        float v[16];
+                        tmem_ld16(tmem_row_addr(tmem, wq, kColP + c0), v);
 #pragma unroll
-                    for (int e = 0; e < 16; ++e) {
-                        const int j = c0 + e;
-                        if (j < jlo || j > jhi) continue;
-                        const int jg = min(j, valid - 1);
+                        for (int e = 0; e < 16; ++e) {
+                            const int j = c0 + e;
+                            if (j < jlo || j > jhi) continue;
+                            const int jg = min(j, valid - 1);
 #pragma unroll
-                        for (int u = 0; u < 16; ++u) {
-                            const float gj = tile_elem(gt, jg, s0 + u);
-                            const float ex = REV ? gj - gi[u] : gi[u] - gj;
-                            acc[u] = fmaf(v[e] * tile_elem(sW, j, s0 + u), __expf(fminf(ex, 0.f)), acc[u]);
+                            for (int u = 0; u < 16; ++u) {
+                                const float gj = tile_elem(gt, jg, s0 + u);
+                                const float ex = REV ? gj - gi[u] : gi[u] - gj;
+                                acc[u] = fmaf(v[e] * tile_elem(sW, j, s0 + u), __expf(fminf(ex, 0.f)), acc[u]);
+                            }
+                        }
+                    }
+                    float vi[16];
+                    tmem_ld16(tmem_row_addr(tmem, wq, kColO + s0), vi);
+                    if (row < valid) {
+                        float* dst = obase + (size_t)(t0 + row) * strideM + s0;
+#pragma unroll
+                        for (int e = 0; e < 16; e += 4) {
+                            float r[4];
+#pragma unroll
+                            for (int u = 0; u < 4; ++u)
+                                r[u] = fmaf(vi[e + u], __expf(REV ? ctl->gc[s0 + e + u] - gi[e + u] : gi[e + u]), acc[e + u]);
+                            *reinterpret_cast<float4*>(dst + e) = make_float4(r[0], r[1], r[2], r[3]);
                         }
                     }
                 }
-                float vi[16];
-                tmem_ld16(tmem_row_addr(tmem, wq, kColO + s0), vi);
+            }
+
+            // ---- state update from U: S <- S exp(G_C) + U
+            PROF_MARK();
+            WAIT_OR_ABORT(&ctl->bar_mma1, it & 1);
+            tc_fence_after_sync();
+            PROF_MARK();
+            {
+                float v[kHS];
+                tmem_ld32(tmem_row_addr(tmem, wq, kColU + sb), v);
+#pragma unroll
+                for (int e = 0; e < kHS; ++e) S[e] = fmaf(S[e], ctl->egc[sb + e], v[e]);
+            }
+            // its bf16 copy feeds the next chunk's inter-chunk product (issued as soon as the next
+            // tiles are there); the product of this chunk that read the old copy is complete
+            store_state_row<false>(sSb, row, sb, S, nullptr);
+
+            // ---- output rows of a moderate chunk: exp(+-G_i) * (inter + intra)
+            PROF_MARK();
+            if (moderate) {
+                WAIT_OR_ABORT(&ctl->bar_mma2, n_mod & 1);
+                ++n_mod;
+                tc_fence_after_sync();
+                PROF_MARK();
+                // the scaled rows replace this chunk's G rows in place (each thread reads and rewrites
+                // only its own 32 slots) and leave as one tiled store, clipped at the sequence end
+                float vo[kHS], vi[kHS];
+                tmem_ld32(tmem_row_addr(tmem, wq, kColO + sb), vi);
+                tmem_ld32(tmem_row_addr(tmem, wq, kColO2 + sb), vo);
+                // forward: exp(G) (inter + intra); reverse: exp(-G) (exp(G_C) inter + intra)
+#pragma unroll
+                for (int e = 0; e < kHS; ++e) vo[e] = REV ? fmaf(vi[e], ctl->egc[sb + e], vo[e]) : vo[e] + vi[e];
                 if (row < valid) {
-                    float* dst = obase + (size_t)(t0 + row) * strideM + s0;
+                    unsigned char* panel = const_cast<unsigned char*>(gt) + half * kPanelB;
 #pragma unroll
-                    for (int e = 0; e < 16; e += 4) {
-                        float r[4];
-#pragma unroll
-                        for (int u = 0; u < 4; ++u)
-                            r[u] = fmaf(vi[e + u], __expf(REV ? ctl->gc[s0 + e + u] - gi[e + u] : gi[e + u]), acc[e + u]);
-                        *reinterpret_cast<float4*>(dst + e) = make_float4(r[0], r[1], r[2], r[3]);
+                    for (int c = 0; c < kHS / 4; ++c) {
+                        float4* cell = reinterpret_cast<float4*>(panel + swz128(row, c));
+                        const float4 g = *cell;
+                        *cell = make_float4(vo[4 * c] * __expf(REV ? -g.x : g.x), vo[4 * c + 1] * __expf(REV ? -g.y : g.y),
+                                            vo[4 * c + 2] * __expf(REV ? -g.z : g.z), vo[4 * c + 3] * __expf(REV ? -g.w : g.w));
                     }
                 }
             }
-        }
-
-        // ---- state update from U: S <- S exp(G_C) + U
-        if (!mbar_wait(&ctl->bar_mma1, it & 1)) ctl->abort = 1;
-        tc_fence_after_sync();
-        // the d-sized tiles are consumed: request the next chunk's
-        if (tid == 0 && it + 1 < nchunks) load_x(it + 1);
-        {
-            float v[kHS];
-            tmem_ld32(tmem_row_addr(tmem, wq, kColU + sb), v);
-#pragma unroll
-            for (int e = 0; e < kHS; ++e) S[e] = fmaf(S[e], ctl->egc[sb + e], v[e]);
-        }
-        PROF_MARK();
-
-        // ---- output rows of a moderate chunk: exp(+-G_i) * (inter + intra)
-        if (moderate) {
-            if (!mbar_wait(&ctl->bar_mma2, n_mma2 & 1)) ctl->abort = 1;
-            ++n_mma2;
-            tc_fence_after_sync();
-            PROF_MARK();
-            // the masked P is consumed: its buffer takes the next chunk's weight tile
-            if (tid == 0 && it + 1 < nchunks) load_w(it + 1);
-            // the scaled rows replace this chunk's G rows in place (each thread reads and rewrites
-            // only its own 32 slots) and leave as one tiled store, clipped at the sequence end
-            float vo[kHS];
-            tmem_ld32(tmem_row_addr(tmem, wq, kColO + sb), vo);
-            if (row < valid) {
-                unsigned char* panel = const_cast<unsigned char*>(gt) + half * kPanelB;
-#pragma unroll
-                for (int c = 0; c < kHS / 4; ++c) {
-                    float4* cell = reinterpret_cast<float4*>(panel + swz128(row, c));
-                    const float4 g = *cell;
-                    *cell = make_float4(vo[4 * c] * __expf(REV ? -g.x : g.x), vo[4 * c + 1] * __expf(REV ? -g.y : g.y),
-                                        vo[4 * c + 2] * __expf(REV ? -g.z : g.z), vo[4 * c + 3] * __expf(REV ? -g.w : g.w));
-                }
-            }
             fence_async_smem();
-        }
-        tc_fence_before_sync();
-        __syncthreads();
-        if (tid == 0 && !ctl->abort) {
-            if (moderate) {
-                tma_store_5d(&mapO, gt, 0, h, t0, b, slice);
-                tma_store_5d(&mapO, gt + kPanelB, 32, h, t0, b, slice);
-                bulk_commit();
+            tc_fence_before_sync();
+            compute_sync();                 // rows staged; gc / egc and the accumulators may be reused
+            if (tid == 0) {
+                mbar_arrive(&ctl->bar_sb);
+                mbar_arrive(&ctl->bar_out);
             }
-            // a strong-decay chunk read the weight tile until now
-            if (!moderate && it + 1 < nchunks) load_w(it + 1);
+            PROF_MARK();
+            PROF_DUMP("value_side compute");
+            if (ctl->abort) break;
         }
-        PROF_MARK();
-        PROF_DUMP("value_side");
-        if (ctl->abort) break;
+        if (!ctl->abort && a.Send) {
+#pragma unroll
+            for (int s = 0; s < kHS; ++s) a.Send[((size_t)bh * kM + sb + s) * a.D + d0 + row] = S[s];
+        }
     }
 
     tc_fence_before_sync();
@@ -434,11 +521,7 @@ value_side_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_cons
         if (tid == 0 && dev_status != nullptr) *dev_status = GSA_ERR_TIMEOUT;
         // bounded grace period for tile copies still in flight before shared memory goes away
         for (int i = 0; i < 200; ++i) __nanosleep(1000);
-    } else if (a.Send) {
-#pragma unroll
-        for (int s = 0; s < kHS; ++s) a.Send[((size_t)bh * kM + sb + s) * a.D + d0 + row] = S[s];
     }
-    if (tid == 0) bulk_wait_read();      // staged output rows must have left before shared memory goes away
     __syncthreads();
     if (warp == 0) {
         __syncwarp();
@@ -464,254 +547,248 @@ key_side_tc_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_consta
     unsigned char* sUq = sAm;                        //   ... shared with the uq tile fp32, 2 panels
     unsigned char* sQt = sAm + 2 * kPanelB;          // uq, intra scaling, K-major A [128][64]     (16 KB)
     unsigned char* sKt = sQt + kPanelB;              // uk, intra scaling, K-major B [128][64]     (16 KB)
+                                                     //   ... sQt + sKt also stage the output rows
     unsigned char* sQb = sKt + kPanelB;              // uq, state scaling, K-major A [128][64]     (16 KB)
     unsigned char* sKb = sQb + kPanelB;              // uk, state scaling, MN-major B [128][64]    (16 KB)
     unsigned char* sSb = sKb + kPanelB;              // state copy, K-major B [128 (channel)][64]  (16 KB)
     Ctl* ctl = reinterpret_cast<Ctl*>(sSb + kPanelB);
 
-    const int tid = threadIdx.x, warp = tid >> 5, wq = warp & 3, half = tid >> 7, row = tid & 127;
+    const int tid = threadIdx.x, warp = tid >> 5, wq = warp & 3, half = (tid >> 7) & 1, row = tid & 127;
     const int sb = kHS * half;          // this thread's first slot
     const int bh = blockIdx.x, slice = blockIdx.y, b = bh / a.H, h = bh % a.H;
     const int d0 = slice * kDST;
 
     ctl_init(ctl, tid, warp);
     const uint32_t tmem = ctl->tmem_slot;
-
     const int nchunks = (a.T + kCT - 1) / kCT;
     auto chunk_t0 = [&](int it) { return (REV ? nchunks - 1 - it : it) * kCT; };
-    auto load_v = [&](int it) {
-        const int t = chunk_t0(it);
-        mbar_expect_tx(&ctl->bar_x, 2 * kPanelB);
-        tma_load_4d(sXv, &mapV, &ctl->bar_x, d0, h, t, b);
-        tma_load_4d(sXv + kPanelB, &mapV, &ctl->bar_x, d0 + 64, h, t, b);
-    };
-    auto load_kg = [&](int it) {
-        const int t = chunk_t0(it);
-        mbar_expect_tx(&ctl->bar_g[0], 4 * kPanelB);
-        tma_load_4d(sUk, &mapUk, &ctl->bar_g[0], 0, h, t, b);
-        tma_load_4d(sUk + kPanelB, &mapUk, &ctl->bar_g[0], 32, h, t, b);
-        tma_load_4d(sG, &mapG, &ctl->bar_g[0], 0, h, t, b);
-        tma_load_4d(sG + kPanelB, &mapG, &ctl->bar_g[0], 32, h, t, b);
-    };
-    auto load_q = [&](int it) {
-        const int t = chunk_t0(it);
-        mbar_expect_tx(&ctl->bar_w, 2 * kPanelB);
-        tma_load_4d(sUq, &mapUq, &ctl->bar_w, 0, h, t, b);
-        tma_load_4d(sUq + kPanelB, &mapUq, &ctl->bar_w, 32, h, t, b);
-    };
-    if (tid == 0) {
-        prefetch_tmap(&mapV); prefetch_tmap(&mapUq); prefetch_tmap(&mapUk); prefetch_tmap(&mapG); prefetch_tmap(&mapO);
-        load_kg(0);
-        load_q(0);
-        load_v(0);
-    }
 
-    // state slice, transposed: S[c = tid][s]
-    float S[kHS];
+    if (warp == kComputeThreads / 32) {
+        // =============================== issuing warp: TMA loads / stores and all MMAs
+        if (tid == kComputeThreads) {
+            auto load_v = [&](int it) {
+                const int t = chunk_t0(it);
+                mbar_expect_tx(&ctl->bar_x, 2 * kPanelB);
+                tma_load_4d(sXv, &mapV, &ctl->bar_x, d0, h, t, b);
+                tma_load_4d(sXv + kPanelB, &mapV, &ctl->bar_x, d0 + 64, h, t, b);
+            };
+            auto load_kg = [&](int it) {
+                const int t = chunk_t0(it);
+                mbar_expect_tx(&ctl->bar_g[0], 4 * kPanelB);
+                tma_load_4d(sUk, &mapUk, &ctl->bar_g[0], 0, h, t, b);
+                tma_load_4d(sUk + kPanelB, &mapUk, &ctl->bar_g[0], 32, h, t, b);
+                tma_load_4d(sG, &mapG, &ctl->bar_g[0], 0, h, t, b);
+                tma_load_4d(sG + kPanelB, &mapG, &ctl->bar_g[0], 32, h, t, b);
+            };
+            auto load_q = [&](int it) {
+                const int t = chunk_t0(it);
+                mbar_expect_tx(&ctl->bar_w, 2 * kPanelB);
+                tma_load_4d(sUq, &mapUq, &ctl->bar_w, 0, h, t, b);
+                tma_load_4d(sUq + kPanelB, &mapUq, &ctl->bar_w, 32, h, t, b);
+            };
+            prefetch_tmap(&mapV); prefetch_tmap(&mapUq); prefetch_tmap(&mapUk); prefetch_tmap(&mapG); prefetch_tmap(&mapO);
+            load_kg(0);
+            load_q(0);
+            load_v(0);
+            constexpr uint32_t idescA = make_idesc(128, 128, false, false);   // Q~ K~^T
+            constexpr uint32_t idescO = make_idesc(128, kDST, false, false);  // Q- x state copy (K-major B)
+            constexpr uint32_t idescU = make_idesc(128, kM, true, true);      // xv^T (MN-major A) x K- (MN-major B)
+            constexpr uint32_t idescV = make_idesc(128, kDST, false, true);   // A x xv (MN-major B)
+            // base descriptors of every operand (K step 0); advancing along K is one add each
+            const uint64_t dV = desc_mnmajor(smem_u32(sXv), 0, kPanelB), dKb = desc_mnmajor(smem_u32(sKb), 0, kPanelB);
+            const uint64_t dQt = desc_kmajor(smem_u32(sQt), 0), dKt = desc_kmajor(smem_u32(sKt), 0);
+            const uint64_t dQb = desc_kmajor(smem_u32(sQb), 0), dS = desc_kmajor(smem_u32(sSb), 0);
+            const uint64_t dA = desc_kmajor(smem_u32(sAm), 0);
+            auto kmaj = [](int kk) { return (uint32_t)((kk >> 2) * kPanelB + (kk & 3) * 32); };
+            auto mnmaj = [](int kk) { return (uint32_t)(kk * 2048); };
+            for (int it = 0; it < nchunks && !ctl->abort; ++it) {
+                const int t0 = chunk_t0(it);
+                WAIT_OR_ABORT(&ctl->bar_ops, it & 1);
+                WAIT_OR_ABORT(&ctl->bar_x, it & 1);
+                tc_fence_after_sync();
+                const bool moderate = ctl->moderate[it & 1] != 0;
+                if (moderate) {
 #pragma unroll
-    for (int s = 0; s < kHS; ++s) S[s] = a.S0 ? a.S0[((size_t)bh * kM + sb + s) * a.D + d0 + row] : 0.f;
-
-    constexpr uint32_t idescA = make_idesc(128, 128, false, false);   // Q~ K~^T
-    constexpr uint32_t idescO = make_idesc(128, kDST, false, false);  // Q- x state copy (K-major B)
-    constexpr uint32_t idescU = make_idesc(128, kM, true, true);      // xv^T (MN-major A) x K- (MN-major B)
-    constexpr uint32_t idescV = make_idesc(128, kDST, false, true);   // A x xv (MN-major B)
-
-    int it = 0;
-    int n_p = 0;       // completed phases of bar_p (only moderate chunks use it)
-    PROF_DECL
-    for (; it < nchunks; ++it) {
-        const int t0 = chunk_t0(it);
-        const int valid = min(kCT, a.T - t0);
-        PROF_MARK();
-        if (tid == 0) bulk_wait_read();    // the previous chunk's output rows have left sQt / sKt
-        if (!mbar_wait(&ctl->bar_g[0], it & 1)) ctl->abort = 1;
-        if (!mbar_wait(&ctl->bar_w, it & 1)) ctl->abort = 1;
-        PROF_MARK();
-        const bool moderate = publish_chunk_decay(ctl, tid, sG, valid - 1);
-        if (ctl->abort) break;
-        PROF_MARK();
-
-        const int grow = min(row, valid - 1);
-        // key side first: it needs the uk and G tiles only; the uq tile (which shares its buffer
-        // with the previous chunk's masked A) arrives last
+                    for (int kk = 0; kk < kM / 16; ++kk)
+                        mma_bf16(tmem + kColP, desc_advance(dQt, kmaj(kk)), desc_advance(dKt, kmaj(kk)), idescA, kk > 0);
+                    mma_commit(&ctl->bar_p);     // the state products below run under the read-out of A
+                }
 #pragma unroll
-        for (int s0 = sb; s0 < sb + kHS; s0 += 8) {
-            float g[8], uk[8], kb[8], kt[8];
-            tile_row8(sG, grow, s0, g);
-            tile_row8(sUk, row, s0, uk);
-#pragma unroll
-            for (int e = 0; e < 8; ++e) {
-                // state term: forward K- = uk exp(G_C - G), reverse uk exp(G); intra term: uk exp(-+G)
-                const float eg = __expf(g[e]);
-                kb[e] = uk[e] * (REV ? eg : __expf(ctl->gc[s0 + e] - g[e]));
-                kt[e] = uk[e] * (REV ? eg : __expf(-g[e]));
-            }
-            store_chunk(sKb, row, s0 >> 3, kb);
-            if (moderate) store_chunk(sKt, row, s0 >> 3, kt);
-        }
-        if (!mbar_wait(&ctl->bar_w, it & 1)) ctl->abort = 1;
-#pragma unroll
-        for (int s0 = sb; s0 < sb + kHS; s0 += 8) {
-            float g[8], uq[8], qb[8], qt[8];
-            tile_row8(sG, grow, s0, g);
-            tile_row8(sUq, row, s0, uq);
-#pragma unroll
-            for (int e = 0; e < 8; ++e) {
-                // state term: forward Q- = uq exp(G), reverse uq exp(G_C - G); intra term: uq exp(+-G)
-                const float eg = __expf(g[e]);
-                qb[e] = uq[e] * (REV ? __expf(ctl->gc[s0 + e] - g[e]) : eg);
-                qt[e] = uq[e] * (REV ? __expf(-g[e]) : eg);
-            }
-            store_chunk(sQb, row, s0 >> 3, qb);
-            if (moderate) store_chunk(sQt, row, s0 >> 3, qt);
-        }
-        store_state_row<false>(sSb, row, sb, S, nullptr);
-        fence_async_smem();
-        PROF_MARK();
-        if (!mbar_wait(&ctl->bar_x, it & 1)) ctl->abort = 1;
-        PROF_MARK();
-        tc_fence_before_sync();
-        __syncthreads();
-        if (ctl->abort) break;
-        PROF_MARK();
-
-        const uint32_t aV = smem_u32(sXv);
-        if (tid == 0) {
-            tc_fence_after_sync();
-            const uint32_t aQt = smem_u32(sQt), aKt = smem_u32(sKt), aQb = smem_u32(sQb);
-            const uint32_t aKb = smem_u32(sKb), aS = smem_u32(sSb);
-            if (moderate) {
+                for (int kk = 0; kk < kCT / 16; ++kk)
+                    mma_bf16(tmem + kColU, desc_advance(dV, mnmaj(kk)), desc_advance(dKb, mnmaj(kk)), idescU, kk > 0);
 #pragma unroll
                 for (int kk = 0; kk < kM / 16; ++kk)
-                    mma_bf16(tmem + kColP, desc_kmajor(aQt, kk), desc_kmajor(aKt, kk), idescA, kk > 0);
-                mma_commit(&ctl->bar_p);     // the state products below run under the read-out of A
+                    mma_bf16(tmem + kColO, desc_advance(dQb, kmaj(kk)), desc_advance(dS, kmaj(kk)), idescO, kk > 0);
+                mma_commit(&ctl->bar_mma1);
+                // a moderate chunk is done with the uk and G tiles: request the next chunk's
+                if (moderate && it + 1 < nchunks) load_kg(it + 1);
+                WAIT_OR_ABORT(&ctl->bar_pm, it & 1);
+                tc_fence_after_sync();
+#pragma unroll
+                for (int kk = 0; kk < kCT / 16; ++kk)
+                    mma_bf16(tmem + kColO, desc_advance(dA, kmaj(kk)), desc_advance(dV, mnmaj(kk)), idescV, true);
+                mma_commit(&ctl->bar_mma2);
+                if (!moderate && it + 1 < nchunks) load_kg(it + 1);
+                // the masked A is consumed: its buffer takes the next chunk's uq tile
+                WAIT_OR_ABORT(&ctl->bar_mma2, it & 1);
+                if (it + 1 < nchunks) {
+                    load_q(it + 1);
+                    load_v(it + 1);
+                }
+                // the output rows are staged over the intra operands: store them, then tell the
+                // compute threads that those buffers may be rewritten
+                WAIT_OR_ABORT(&ctl->bar_out, it & 1);
+                if (ctl->abort) break;
+                tma_store_4d(&mapO, sQt, d0, h, t0, b);
+                tma_store_4d(&mapO, sQt + kPanelB, d0 + 64, h, t0, b);
+                bulk_commit();
+                bulk_wait_read();
+                mbar_arrive(&ctl->bar_sb);
             }
-#pragma unroll
-            for (int kk = 0; kk < kCT / 16; ++kk)
-                mma_bf16(tmem + kColU, desc_mnmajor(aV, kk, kPanelB), desc_mnmajor(aKb, kk, kPanelB), idescU, kk > 0);
-#pragma unroll
-            for (int kk = 0; kk < kM / 16; ++kk)
-                mma_bf16(tmem + kColO, desc_kmajor(aQb, kk), desc_kmajor(aS, kk), idescO, kk > 0);
-            mma_commit(&ctl->bar_mma1);
-            // a moderate chunk is done with the uk and G tiles: request the next chunk's
-            if (moderate && it + 1 < nchunks) load_kg(it + 1);
         }
-        PROF_MARK();
-        if (moderate) {
-            if (!mbar_wait(&ctl->bar_p, n_p & 1)) ctl->abort = 1;
-            ++n_p;
-        }
-        tc_fence_after_sync();
-        PROF_MARK();
+    } else {
+        // =============================== compute threads
+        // state slice, transposed: S[c = row][s], slots sb .. sb+31
+        float S[kHS];
+#pragma unroll
+        for (int s = 0; s < kHS; ++s) S[s] = a.S0 ? a.S0[((size_t)bh * kM + sb + s) * a.D + d0 + row] : 0.f;
 
-        if (moderate) {
-            store_masked_row<REV>(tmem, wq, row, half, sAm);    // overwrites the uq tile: all rows were read
-        } else {
-            // Strong decay: A_ij with explicit exponent differences, from the fp32 uk and G tiles.
-            float gi[kM], qi[kM];
+        int n_mod = 0;     // moderate chunks so far (phases of bar_p)
+        for (int it = 0; it < nchunks; ++it) {
+            const int t0 = chunk_t0(it);
+            const int valid = min(kCT, a.T - t0);
+            (void)t0;
+            WAIT_OR_ABORT(&ctl->bar_g[0], it & 1);
+            const bool moderate = publish_chunk_decay(ctl, tid, sG, valid - 1);
+            if (ctl->abort) break;
+
+            const int grow = min(row, valid - 1);
+            // the previous chunk's output rows must have left sQt / sKt before they are rewritten
+            if (it > 0) WAIT_OR_ABORT(&ctl->bar_sb, (it - 1) & 1);
+            // key side first: it needs the uk and G tiles only; the uq tile (which shares its buffer
+            // with the previous chunk's masked A) arrives last
 #pragma unroll
-            for (int s0 = 0; s0 < kM; s0 += 8) {
-                float g[8], uq[8];
+            for (int s0 = sb; s0 < sb + kHS; s0 += 8) {
+                float g[8], uk[8], kb[8], kt[8];
+                tile_row8(sG, grow, s0, g);
+                tile_row8(sUk, row, s0, uk);
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                    // state term: forward K- = uk exp(G_C - G), reverse uk exp(G); intra term: uk exp(-+G)
+                    const float eg = __expf(g[e]);
+                    kb[e] = uk[e] * (REV ? eg : __expf(ctl->gc[s0 + e] - g[e]));
+                    kt[e] = uk[e] * (REV ? eg : __expf(-g[e]));
+                }
+                store_chunk(sKb, row, s0 >> 3, kb);
+                if (moderate) store_chunk(sKt, row, s0 >> 3, kt);
+            }
+            WAIT_OR_ABORT(&ctl->bar_w, it & 1);
+#pragma unroll
+            for (int s0 = sb; s0 < sb + kHS; s0 += 8) {
+                float g[8], uq[8], qb[8], qt[8];
                 tile_row8(sG, grow, s0, g);
                 tile_row8(sUq, row, s0, uq);
 #pragma unroll
-                for (int e = 0; e < 8; ++e) { gi[s0 + e] = g[e]; qi[s0 + e] = uq[e]; }
-            }
-            __syncthreads();          // every thread has its uq row in registers before sAm is written
-            for (int c0 = 64 * half; c0 < 64 * half + 64; c0 += 8) {
-                float x[8];
-#pragma unroll
                 for (int e = 0; e < 8; ++e) {
-                    const int j = c0 + e;
-                    const bool keep = REV ? (j >= row) : (j <= row);
-                    float acc = 0.f;
-                    if (keep) {
-                        const int jg = min(j, valid - 1);
-#pragma unroll
-                        for (int s = 0; s < kM; ++s) {
-                            const float gj = tile_elem(sG, jg, s);
-                            const float ex = REV ? gj - gi[s] : gi[s] - gj;
-                            acc = fmaf(qi[s] * tile_elem(sUk, j, s), __expf(fminf(ex, 0.f)), acc);
-                        }
-                    }
-                    x[e] = acc;
+                    // state term: forward Q- = uq exp(G), reverse uq exp(G_C - G); intra term: uq exp(+-G)
+                    const float eg = __expf(g[e]);
+                    qb[e] = uq[e] * (REV ? __expf(ctl->gc[s0 + e] - g[e]) : eg);
+                    qt[e] = uq[e] * (REV ? __expf(-g[e]) : eg);
                 }
-                store_chunk(sAm + (c0 >> 6) * kPanelB, row, (c0 & 63) >> 3, x);
+                store_chunk(sQb, row, s0 >> 3, qb);
+                if (moderate) store_chunk(sQt, row, s0 >> 3, qt);
             }
-        }
-        fence_async_smem();
-        tc_fence_before_sync();
-        __syncthreads();
-        if (ctl->abort) break;
-        PROF_MARK();
-        if (tid == 0) {
+            store_state_row<false>(sSb, row, sb, S, nullptr);
+            fence_async_smem();
+            if (tid == 0) ctl->moderate[it & 1] = moderate;
+            compute_sync();
+            if (tid == 0) mbar_arrive(&ctl->bar_ops);
+
+            if (moderate) {
+                WAIT_OR_ABORT(&ctl->bar_p, n_mod & 1);
+                ++n_mod;
+                tc_fence_after_sync();
+                store_masked_row<REV>(tmem, wq, row, half, sAm);    // overwrites the uq tile: all rows were read
+            } else {
+                // Strong decay: A_ij with explicit exponent differences, from the fp32 uk and G tiles.
+                float gi[kM], qi[kM];
+#pragma unroll
+                for (int s0 = 0; s0 < kM; s0 += 8) {
+                    float g[8], uq[8];
+                    tile_row8(sG, grow, s0, g);
+                    tile_row8(sUq, row, s0, uq);
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) { gi[s0 + e] = g[e]; qi[s0 + e] = uq[e]; }
+                }
+                compute_sync();           // every thread has its uq row in registers before sAm is written
+                for (int c0 = 64 * half; c0 < 64 * half + 64; c0 += 8) {
+                    float x[8];
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) {
+                        const int j = c0 + e;
+                        const bool keep = REV ? (j >= row) : (j <= row);
+                        float acc = 0.f;
+                        if (keep) {
+                            const int jg = min(j, valid - 1);
+#pragma unroll
+                            for (int s = 0; s < kM; ++s) {
+                                const float gj = tile_elem(sG, jg, s);
+                                const float ex = REV ? gj - gi[s] : gi[s] - gj;
+                                acc = fmaf(qi[s] * tile_elem(sUk, j, s), __expf(fminf(ex, 0.f)), acc);
+                            }
+                        }
+                        x[e] = acc;
+                    }
+                    store_chunk(sAm + (c0 >> 6) * kPanelB, row, (c0 & 63) >> 3, x);
+                }
+            }
+            fence_async_smem();
+            tc_fence_before_sync();
+            compute_sync();
+            if (tid == 0) mbar_arrive(&ctl->bar_pm);
+
+            // ---- state update from U^T: S <- exp(G_C) S + U^T
+            WAIT_OR_ABORT(&ctl->bar_mma1, it & 1);
             tc_fence_after_sync();
-            const uint32_t aA = smem_u32(sAm);
+            {
+                float v[kHS];
+                tmem_ld32(tmem_row_addr(tmem, wq, kColU + sb), v);
 #pragma unroll
-            for (int kk = 0; kk < kCT / 16; ++kk)
-                mma_bf16(tmem + kColO, desc_kmajor(aA + (kk >> 2) * kPanelB, kk),
-                         desc_mnmajor(aV, kk, kPanelB), idescV, true);
-            mma_commit(&ctl->bar_mma2);
-            if (!moderate && it + 1 < nchunks) load_kg(it + 1);
-        }
-
-        // ---- state update from U^T: S <- exp(G_C) S + U^T
-        if (!mbar_wait(&ctl->bar_mma1, it & 1)) ctl->abort = 1;
-        tc_fence_after_sync();
-        {
-            float v[kHS];
-            tmem_ld32(tmem_row_addr(tmem, wq, kColU + sb), v);
-#pragma unroll
-            for (int e = 0; e < kHS; ++e) S[e] = fmaf(S[e], ctl->egc[sb + e], v[e]);
-        }
-        PROF_MARK();
-
-        // ---- output rows
-        if (!mbar_wait(&ctl->bar_mma2, it & 1)) ctl->abort = 1;
-        tc_fence_after_sync();
-        PROF_MARK();
-        // xv and the masked A are consumed: request the next chunk's xv and uq tiles
-        if (tid == 0 && it + 1 < nchunks && !ctl->abort) {
-            load_v(it + 1);
-            load_q(it + 1);
-        }
-        // output rows -> bf16, staged over the intra operands (consumed since bar_mma1), then one
-        // tiled store per 64 columns, clipped at the sequence end
-#pragma unroll
-        for (int c0 = 0; c0 < 64; c0 += 32) {
-            float v[32];
-            tmem_ld32(tmem_row_addr(tmem, wq, kColO + 64 * half + c0), v);
-#pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                const float x[8] = {v[8 * c], v[8 * c + 1], v[8 * c + 2], v[8 * c + 3],
-                                    v[8 * c + 4], v[8 * c + 5], v[8 * c + 6], v[8 * c + 7]};
-                store_chunk(sQt + half * kPanelB, row, (c0 >> 3) + c, x);
+                for (int e = 0; e < kHS; ++e) S[e] = fmaf(S[e], ctl->egc[sb + e], v[e]);
             }
+
+            // ---- output rows -> bf16, staged over the intra operands (consumed since bar_p), stored
+            // by the issuing warp, clipped at the sequence end
+            WAIT_OR_ABORT(&ctl->bar_mma2, it & 1);
+            tc_fence_after_sync();
+            {
+                float v[64];
+                tmem_ld64(tmem_row_addr(tmem, wq, kColO + 64 * half), v);
+#pragma unroll
+                for (int c = 0; c < 8; ++c) {
+                    const float x[8] = {v[8 * c], v[8 * c + 1], v[8 * c + 2], v[8 * c + 3],
+                                        v[8 * c + 4], v[8 * c + 5], v[8 * c + 6], v[8 * c + 7]};
+                    store_chunk(sQt + half * kPanelB, row, c, x);
+                }
+            }
+            fence_async_smem();
+            tc_fence_before_sync();
+            compute_sync();
+            if (tid == 0) mbar_arrive(&ctl->bar_out);
+            if (ctl->abort) break;
         }
-        fence_async_smem();
-        tc_fence_before_sync();
-        __syncthreads();
-        if (tid == 0 && !ctl->abort) {
-            tma_store_4d(&mapO, sQt, d0, h, t0, b);
-            tma_store_4d(&mapO, sQt + kPanelB, d0 + 64, h, t0, b);
-            bulk_commit();
+        if (!ctl->abort && a.Send) {
+#pragma unroll
+            for (int s = 0; s < kHS; ++s) a.Send[((size_t)bh * kM + sb + s) * a.D + d0 + row] = S[s];
         }
-        PROF_MARK();
-        PROF_DUMP("key_side");
-        if (ctl->abort) break;
     }
 
     tc_fence_before_sync();
     __syncthreads();
     if (ctl->abort) {
         if (tid == 0 && dev_status != nullptr) *dev_status = GSA_ERR_TIMEOUT;
-        // bounded grace period for tile copies still in flight before shared memory goes away
         for (int i = 0; i < 200; ++i) __nanosleep(1000);
-    } else if (a.Send) {
-#pragma unroll
-        for (int s = 0; s < kHS; ++s) a.Send[((size_t)bh * kM + sb + s) * a.D + d0 + row] = S[s];
     }
-    if (tid == 0) bulk_wait_read();      // staged output rows must have left before shared memory goes away
     __syncthreads();
     if (warp == 0) {
         __syncwarp();

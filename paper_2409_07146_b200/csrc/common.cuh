@@ -104,6 +104,7 @@ cudaError_t launch_gate_grad(const float* u, const float* I, const float* dIk_pa
                              const float* dVT, const float* VT, int d_k, int d_v,
                              float* chunk_tot, float* dgate, int B, int T, int H, int M,
                              cudaStream_t st);
+int gate_grad_blocks(int T);       // entries per (b,h,slot) of launch_gate_grad's scratch
 cudaError_t launch_value_side_simt(const ValueSideArgs& a, int io, int M, int reverse,
                                    cudaStream_t st);
 cudaError_t launch_key_side_simt(const KeySideArgs& a, int io, int M, int reverse,

@@ -179,43 +179,76 @@ cudaError_t launch_slot_softmax_bwd(const float* ok, const float* dp_part, int n
 // (the reversed cumulative sum of App. B, taken over the whole sequence), then
 //   gate holds a     : dgate = d(log a)|decay / a - dI
 //   gate holds log a : dgate = d(log a)|decay - a * dI
-// Three steps: per-chunk totals, an exclusive suffix scan over the chunk totals (fp64),
-// and the chunk-local reversed sums started from that carry.
-template <int M>
-__device__ __forceinline__ float sum_parts(const float* part, int nslice, size_t idx, size_t total) {
-    float acc = 0.f;
-    for (int sl = 0; sl < nslice; ++sl) acc += part[idx + (size_t)sl * total];
-    return acc;
+// Three steps: totals of 16-row blocks, an exclusive suffix scan over the block totals (fp64),
+// and the block-local reversed sums started from that carry.
+
+constexpr int kGG = 16;   // rows per thread of the gate-gradient kernels
+
+// dI[i] = sum over the d_k and d_v slices of the input-gate gradient partial sums, for the
+// kGG rows of this thread; the rows of one slice are loaded together (16 loads in flight).
+__device__ __forceinline__ void load_dI(const float* __restrict__ dIk, int nsk, const float* __restrict__ dIv,
+                                        int nsv, size_t base, size_t stride, size_t total, int rows,
+                                        float (&dI)[kGG]) {
+#pragma unroll
+    for (int i = 0; i < kGG; ++i) dI[i] = 0.f;
+    for (int sl = 0; sl < nsk; ++sl) {
+        float t[kGG];
+#pragma unroll
+        for (int i = 0; i < kGG; ++i) t[i] = (i < rows) ? dIk[base + (size_t)i * stride + (size_t)sl * total] : 0.f;
+#pragma unroll
+        for (int i = 0; i < kGG; ++i) dI[i] += t[i];
+    }
+    for (int sl = 0; sl < nsv; ++sl) {
+        float t[kGG];
+#pragma unroll
+        for (int i = 0; i < kGG; ++i) t[i] = (i < rows) ? dIv[base + (size_t)i * stride + (size_t)sl * total] : 0.f;
+#pragma unroll
+        for (int i = 0; i < kGG; ++i) dI[i] += t[i];
+    }
 }
 
 template <int M>
 __global__ void __launch_bounds__(256) gate_grad_totals_kernel(
     const float* __restrict__ u, const float* __restrict__ I, const float* __restrict__ dIk, int nsk,
-    const float* __restrict__ dIv, int nsv, float* __restrict__ chunk_tot, int B, int T, int H,
-    int nchunks) {
+    const float* __restrict__ dIv, int nsv, float* __restrict__ blk_tot, int B, int T, int H,
+    int nblk) {
     const int s = threadIdx.x;
     const int n = blockIdx.y * blockDim.y + threadIdx.y;
-    if (n >= nchunks) return;
+    if (n >= nblk) return;
     const int bh = blockIdx.x, b = bh / H, h = bh % H;
-    const int t0 = n * kChunk;
-    const int rows = min(kChunk, T - t0);
+    const int t0 = n * kGG;
+    const int rows = min(kGG, T - t0);
     const size_t stride = (size_t)H * M, total = (size_t)B * T * H * M;
     const size_t base = (((size_t)b * T + t0) * H + h) * M + s;
-    float tot = 0.f;
-    for (int i = 0; i < rows; ++i) {
-        const size_t idx = base + (size_t)i * stride;
-        const float dI = sum_parts<M>(dIk, nsk, idx, total) + sum_parts<M>(dIv, nsv, idx, total);
-        tot += u[idx] - I[idx] * dI;
+    float x[kGG], dI[kGG], uu[kGG], ii[kGG];
+#pragma unroll
+    for (int i = 0; i < kGG; ++i) {
+        uu[i] = (i < rows) ? u[base + (size_t)i * stride] : 0.f;
+        ii[i] = (i < rows) ? I[base + (size_t)i * stride] : 0.f;
     }
-    chunk_tot[((size_t)bh * nchunks + n) * M + s] = tot;
+    load_dI(dIk, nsk, dIv, nsv, base, stride, total, rows, dI);
+#pragma unroll
+    for (int i = 0; i < kGG; ++i) x[i] = uu[i] - ii[i] * dI[i];
+    float tot = 0.f;
+#pragma unroll
+    for (int i = kGG - 1; i >= 0; --i) tot += x[i];
+    blk_tot[((size_t)bh * nblk + n) * M + s] = tot;
 }
 
-// chunk_tot[bh][n][s] <- sum over chunks n' > n of the totals, plus the final-memory term.
+// blk_tot[bh][n][s] <- sum over blocks n' > n of the totals, plus the final-memory term.
+// One CTA per (b,h): M slots x 16 segments of consecutive blocks; fp64 running sums.
 template <int M>
-__global__ void gate_grad_scan_kernel(float* __restrict__ chunk_tot, const float* __restrict__ dKT,
-                                      const float* __restrict__ KT, const float* __restrict__ dVT,
-                                      const float* __restrict__ VT, int d_k, int d_v, int nchunks) {
-    const int s = threadIdx.x, bh = blockIdx.x;
+__global__ void __launch_bounds__(M * 16) gate_grad_scan_kernel(
+    float* __restrict__ blk_tot, const float* __restrict__ dKT, const float* __restrict__ KT,
+    const float* __restrict__ dVT, const float* __restrict__ VT, int d_k, int d_v, int nblk) {
+    __shared__ double seg_sum[16][M];
+    const int s = threadIdx.x, seg = threadIdx.y, bh = blockIdx.x;
+    const int per = (nblk + 15) / 16;
+    const int lo = seg * per, hi = min(nblk, lo + per);
+    double sum = 0.0;
+    for (int n = lo; n < hi; ++n) sum += (double)blk_tot[((size_t)bh * nblk + n) * M + s];
+    seg_sum[seg][s] = sum;
+    __syncthreads();
     double carry = 0.0;
     if (dKT != nullptr) {
         const float* a = dKT + ((size_t)bh * M + s) * d_k;
@@ -227,10 +260,11 @@ __global__ void gate_grad_scan_kernel(float* __restrict__ chunk_tot, const float
         const float* bb = VT + ((size_t)bh * M + s) * d_v;
         for (int c = 0; c < d_v; ++c) carry += (double)a[c] * (double)bb[c];
     }
-    for (int n = nchunks - 1; n >= 0; --n) {
-        const size_t idx = ((size_t)bh * nchunks + n) * M + s;
-        const float t = chunk_tot[idx];
-        chunk_tot[idx] = (float)carry;
+    for (int g = seg + 1; g < 16; ++g) carry += seg_sum[g][s];
+    for (int n = hi - 1; n >= lo; --n) {
+        const size_t idx = ((size_t)bh * nblk + n) * M + s;
+        const float t = blk_tot[idx];
+        blk_tot[idx] = (float)carry;
         carry += (double)t;
     }
 }
@@ -239,56 +273,66 @@ template <int M>
 __global__ void __launch_bounds__(256) gate_grad_final_kernel(
     const float* __restrict__ u, const float* __restrict__ I, const float* __restrict__ dIk, int nsk,
     const float* __restrict__ dIv, int nsv, const float* __restrict__ gate, int gate_is_log,
-    const float* __restrict__ chunk_carry, float* __restrict__ dgate, int B, int T, int H,
-    int nchunks) {
+    const float* __restrict__ blk_carry, float* __restrict__ dgate, int B, int T, int H,
+    int nblk) {
     const int s = threadIdx.x;
     const int n = blockIdx.y * blockDim.y + threadIdx.y;
-    if (n >= nchunks) return;
+    if (n >= nblk) return;
     const int bh = blockIdx.x, b = bh / H, h = bh % H;
-    const int t0 = n * kChunk;
-    const int rows = min(kChunk, T - t0);
+    const int t0 = n * kGG;
+    const int rows = min(kGG, T - t0);
     const size_t stride = (size_t)H * M, total = (size_t)B * T * H * M;
     const size_t base = (((size_t)b * T + t0) * H + h) * M + s;
-    float run = chunk_carry[((size_t)bh * nchunks + n) * M + s];
-    for (int i = rows - 1; i >= 0; --i) {
-        const size_t idx = base + (size_t)i * stride;
-        const float dI = sum_parts<M>(dIk, nsk, idx, total) + sum_parts<M>(dIv, nsv, idx, total);
-        run += u[idx] - I[idx] * dI;
-        const float gt = gate[idx];
-        float out;
-        if (gate_is_log) {
-            out = run - __expf(fmaxf(gt, kLogGateMin)) * dI;
-        } else {
-            // a == 0 leaves no way back from d(log a) to da: only the input-gate part is kept
-            out = (gt > 0.f) ? run / gt - dI : -dI;
+    float x[kGG], dI[kGG], gt[kGG], ii[kGG];
+#pragma unroll
+    for (int i = 0; i < kGG; ++i) {
+        x[i] = (i < rows) ? u[base + (size_t)i * stride] : 0.f;
+        ii[i] = (i < rows) ? I[base + (size_t)i * stride] : 0.f;
+        gt[i] = (i < rows) ? gate[base + (size_t)i * stride] : 1.f;
+    }
+    load_dI(dIk, nsk, dIv, nsv, base, stride, total, rows, dI);
+#pragma unroll
+    for (int i = 0; i < kGG; ++i) x[i] -= ii[i] * dI[i];
+    float run = blk_carry[((size_t)bh * nblk + n) * M + s];
+#pragma unroll
+    for (int i = kGG - 1; i >= 0; --i) {
+        run += x[i];
+        if (i < rows) {
+            float out;
+            if (gate_is_log) {
+                out = run - __expf(fmaxf(gt[i], kLogGateMin)) * dI[i];
+            } else {
+                // a == 0 leaves no way back from d(log a) to da: only the input-gate part is kept
+                out = (gt[i] > 0.f) ? run / gt[i] - dI[i] : -dI[i];
+            }
+            dgate[base + (size_t)i * stride] = out;
         }
-        dgate[idx] = out;
     }
 }
+
+int gate_grad_blocks(int T) { return (T + kGG - 1) / kGG; }
 
 cudaError_t launch_gate_grad(const float* u, const float* I, const float* dIk_part, int nsk,
                              const float* dIv_part, int nsv, const float* gate,
                              int gate_is_log, const float* dKT, const float* KT,
                              const float* dVT, const float* VT, int d_k, int d_v,
-                             float* chunk_tot, float* dgate, int B, int T, int H, int M,
+                             float* blk_tot, float* dgate, int B, int T, int H, int M,
                              cudaStream_t st) {
-    const int nchunks = (T + kChunk - 1) / kChunk;
+    const int nblk = gate_grad_blocks(T);
     dim3 block(M, 256 / M);
-    dim3 grid(B * H, (nchunks + block.y - 1) / block.y);
+    dim3 grid(B * H, (nblk + block.y - 1) / block.y);
     if (M == 64) {
         gate_grad_totals_kernel<64><<<grid, block, 0, st>>>(u, I, dIk_part, nsk, dIv_part, nsv,
-                                                            chunk_tot, B, T, H, nchunks);
-        gate_grad_scan_kernel<64><<<B * H, 64, 0, st>>>(chunk_tot, dKT, KT, dVT, VT, d_k, d_v, nchunks);
+                                                            blk_tot, B, T, H, nblk);
+        gate_grad_scan_kernel<64><<<B * H, dim3(64, 16), 0, st>>>(blk_tot, dKT, KT, dVT, VT, d_k, d_v, nblk);
         gate_grad_final_kernel<64><<<grid, block, 0, st>>>(u, I, dIk_part, nsk, dIv_part, nsv, gate,
-                                                           gate_is_log, chunk_tot, dgate, B, T, H,
-                                                           nchunks);
+                                                           gate_is_log, blk_tot, dgate, B, T, H, nblk);
     } else {
         gate_grad_totals_kernel<32><<<grid, block, 0, st>>>(u, I, dIk_part, nsk, dIv_part, nsv,
-                                                            chunk_tot, B, T, H, nchunks);
-        gate_grad_scan_kernel<32><<<B * H, 32, 0, st>>>(chunk_tot, dKT, KT, dVT, VT, d_k, d_v, nchunks);
+                                                            blk_tot, B, T, H, nblk);
+        gate_grad_scan_kernel<32><<<B * H, dim3(32, 16), 0, st>>>(blk_tot, dKT, KT, dVT, VT, d_k, d_v, nblk);
         gate_grad_final_kernel<32><<<grid, block, 0, st>>>(u, I, dIk_part, nsk, dIv_part, nsv, gate,
-                                                           gate_is_log, chunk_tot, dgate, B, T, H,
-                                                           nchunks);
+                                                           gate_is_log, blk_tot, dgate, B, T, H, nblk);
     }
     return cudaGetLastError();
 }

@@ -47,6 +47,11 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t smem_addr, uint32_t lbo_b
     d |= (uint64_t)2 << 61;
     return d;
 }
+// Advancing a descriptor along K only changes its start-address field: with the base
+// descriptor of an operand in registers, each MMA costs one 32-bit add per operand.
+__device__ __forceinline__ uint64_t desc_advance(uint64_t base, uint32_t byte_offset) {
+    return base + (uint64_t)(byte_offset >> 4);
+}
 __device__ __forceinline__ uint64_t desc_kmajor(uint32_t panel_addr, int kk) {
     return make_desc(panel_addr + (uint32_t)(kk & 3) * 32u, 16u, 1024u);
 }
