@@ -251,6 +251,15 @@ def run_ours(args):
             dist.all_reduce(ms, op=dist.ReduceOp.MAX)
         return float(ms.item())
 
+    if args.profile_case:
+        # bare steps for a profiler: no timing, no extras (the numbers of such a run are not
+        # benchmark values)
+        for _ in range(args.warmup + args.steps):
+            step(d_in)
+        torch.cuda.synchronize()
+        if rank == 0:
+            print(json.dumps({"profile_case": True, "steps": args.steps, "warmup": args.warmup}))
+        return
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
@@ -411,6 +420,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--profile-case", action="store_true",
+                    help="run warmup + steps bare (for ncu); prints no benchmark line")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
