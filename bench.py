@@ -35,6 +35,14 @@ UNIT = "tokens/s"
 WORKLOAD = "train_1p3b"
 
 
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the tensor-core kernels on this
+# workload, from one `ncu --set full` capture (profiles/tc_chunk_kernels_train_1p3b_ncu_full.md).
+NCU_TRAFFIC = {
+    "pass1_value_side": 211809024, "bwd_dp_value_side": 211809024,
+    "pass2_key_side": 159327744, "bwd_dq_key_side": 159327744,
+}
+
+
 def peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -184,6 +192,29 @@ def run_reference(args):
     print(json.dumps(line), flush=True)
 
 
+# ----------------------------------------------------------------------------- sharding
+def rank_workload(rank: int) -> W.Workload:
+    """Weak scaling over batch: rank r runs its own batch of the workload (its own seed);
+    (batch, head) pairs are independent recurrences, so no rank needs another's data."""
+    base = W.CONFIGS[WORKLOAD]
+    return base.scaled(seed=base.seed + 1000 * rank)
+
+
+def max_over_ranks(ms: float, world: int, device=None) -> float:
+    """Slowest rank's time (all-reduce MAX; works on nccl and gloo groups)."""
+    if world == 1:
+        return ms
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate_tokens_per_s(world: int, tokens_per_rank: int, ms_per_step: float) -> float:
+    return world * tokens_per_rank / (ms_per_step * 1e-3)
+
+
 # ----------------------------------------------------------------------------- our arm
 def run_ours(args):
     import torch
@@ -202,7 +233,7 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     dev = torch.device("cuda", local)
 
-    w = W.CONFIGS[WORKLOAD].scaled(seed=W.CONFIGS[WORKLOAD].seed + 1000 * rank)
+    w = rank_workload(rank)
     x = W.make_inputs(w)
     p = gsa.Params(w.B, w.T, w.H, w.d_k, w.d_v, w.m, io=w.io)
 
@@ -246,10 +277,7 @@ def run_ours(args):
             fn()
         e1.record()
         barrier()
-        ms = torch.tensor([e0.elapsed_time(e1)], device=dev)
-        if world > 1:
-            dist.all_reduce(ms, op=dist.ReduceOp.MAX)
-        return float(ms.item())
+        return max_over_ranks(float(e0.elapsed_time(e1)), world, dev)
 
     if args.profile_case:
         # bare steps for a profiler: no timing, no extras (the numbers of such a run are not
@@ -278,7 +306,7 @@ def run_ours(args):
     if rank == 0:
         clocks["note"] = "nvidia-smi samples (50 ms period, utilisation >= 50%) over warm-up, the timed steps and 1.2 s more of the same steps"
     ms_step = total_ms / args.steps
-    value = world * w.tokens / (ms_step * 1e-3)
+    value = aggregate_tokens_per_s(world, w.tokens, ms_step)
     if int(status.item()) != 0:
         raise SystemExit("a bounded device-side wait expired during the benchmark")
     if not bool(torch.isfinite(dq.float()).all()):
@@ -322,10 +350,7 @@ def run_ours(args):
                             "frac_of_hbm_peak": by / (avg * 1e-3) / 1e9 / pk["hbm_gbs"]})
         kernels.sort(key=lambda k: -k["share"])
         top = kernels[0]
-        traffic = None
-        tpath = os.path.join(ROOT, "profiles", "traffic.json")
-        if os.path.exists(tpath):
-            traffic = json.load(open(tpath)).get(top["kernel"])
+        traffic = NCU_TRAFFIC.get(top["kernel"])
         roofline = {"bound": "hbm", "kernel": top["kernel"], "achieved": top["achieved_gbs"],
                     "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": top["frac_of_hbm_peak"],
                     "traffic": traffic, "peak_source": pk["source"],

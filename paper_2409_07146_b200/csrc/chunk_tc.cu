@@ -16,7 +16,7 @@
 //     swizzle), scales it by the decay factors and writes bf16 operand rows;
 //   * all contractions run as tcgen05.mma (M = 128) with fp32 accumulators in tensor
 //     memory, committed to mbarriers that the compute threads wait on;
-//   * the fp32 master copy of the state slice stays in registers (64 per thread); its bf16
+//   * the fp32 master copy of the state slice stays in registers (32 per thread); its bf16
 //     copy for the next chunk's state product is rewritten every chunk.
 // Decay inside a chunk is factorised as exp(G_i) * exp(-G_j) while the chunk's total
 // log-decay stays above kFactorisedDecayMin; a chunk that forgets harder computes its

@@ -1,0 +1,57 @@
+"""The N > 1 path on CPU: two gloo ranks.  The layer shards over batch with no data-path
+collective; what the ranks share is a barrier and the max-over-ranks time.  Here each rank
+runs the fp64 oracle on its own batch shard and the gathered shards must equal one
+single-process run; the timing reduction and the rank seeding of bench.py are exercised too."""
+import os
+import socket
+
+import numpy as np
+import torch
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+import bench
+import gsa_workloads as W
+import oracle
+
+
+def _free_port():
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def _worker(rank, world, port, out_dir):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        w = W.CONFIGS["tiny_f32"].scaled(B=4, T=40)
+        x = W.make_inputs(w)
+        lo, hi = rank * w.B // world, (rank + 1) * w.B // world      # this rank's batch shard
+        part = oracle.fwd(x["q"][lo:hi], x["k"][lo:hi], x["v"][lo:hi], x["gate"][lo:hi], threads=1)
+        gathered = [None] * world
+        dist.all_gather_object(gathered, part["o"])
+        slow = bench.max_over_ranks(10.0 + rank, world)               # the slowest rank decides
+        seeds = [None] * world
+        dist.all_gather_object(seeds, bench.rank_workload(rank).seed)
+        dist.barrier()
+        if rank == 0:
+            np.save(os.path.join(out_dir, "o.npy"), np.concatenate(gathered, 0))
+            np.save(os.path.join(out_dir, "meta.npy"), np.array([slow] + seeds, dtype=np.float64))
+    finally:
+        dist.destroy_process_group()
+
+
+def test_two_gloo_ranks_shard_the_batch(tmp_path):
+    oracle.build()
+    world, port = 2, _free_port()
+    mp.start_processes(_worker, args=(world, port, str(tmp_path)), nprocs=world, join=True,
+                       start_method="spawn")
+    w = W.CONFIGS["tiny_f32"].scaled(B=4, T=40)
+    x = W.make_inputs(w)
+    full = oracle.fwd(x["q"], x["k"], x["v"], x["gate"], threads=1)
+    np.testing.assert_array_equal(np.load(tmp_path / "o.npy"), full["o"])
+    meta = np.load(tmp_path / "meta.npy")
+    assert meta[0] == 11.0                       # max over ranks of (10, 11)
+    assert meta[1] != meta[2]                    # every rank draws its own batch
+    assert bench.aggregate_tokens_per_s(2, 16384, 1.0) == 2 * 16384 / 1e-3
