@@ -143,6 +143,31 @@ GSA_API gsa_status_t gsa_decode_step(const gsa_params_t* params, const void* q,
                              float* Kstate, float* Vstate, void* o, void* stream);
 
 /*
+ * gsa_fwd without caller-provided scratch (the paper has no counterpart: this is a
+ * packaging variant of gsa_fwd, same arguments minus ws / ws_bytes, same results).
+ *
+ * For callers that cannot allocate device memory around the layer -- code running inside
+ * a server's fixed memory plan, a latency-critical loop that must avoid the allocator's
+ * lock and implicit synchronisation, a plug-in that is only handed input and output
+ * buffers.  The scratch is a fixed array inside the library image: every GPU that loads
+ * the library holds GSA_NOALLOC_MAX_WORKSPACE_BYTES (32 MiB) until the process exits.  The call allocates and frees nothing (no cudaMalloc / cudaFree, no allocating
+ * library routine).
+ *   - Shapes whose gsa_workspace_bytes(params, GSA_WS_FWD) exceeds that maximum are
+ *     rejected with GSA_ERR_WORKSPACE before anything is launched.
+ *   - The first call on each device looks up the array's device address (with that device
+ *     current); make that first call before any stream capture.
+ *   - All calls on a device share the one array: calls that overlap on the GPU (different
+ *     streams) race and give wrong results; serialise them or use gsa_fwd with separate
+ *     workspaces.  The array keeps the previous call's contents; the forward needs none of
+ *     it cleared (it writes every scratch tensor before reading it).
+ */
+#define GSA_NOALLOC_MAX_WORKSPACE_BYTES ((size_t)32 << 20)
+GSA_API gsa_status_t gsa_fwd_noalloc(const gsa_params_t* params, const void* q, const void* k,
+                                     const void* v, const float* gate, const float* K0,
+                                     const float* V0, void* o, float* ok_save, float* KT,
+                                     float* VT, void* stream, int32_t* dev_status);
+
+/*
  * Self-test of the tensor-core building blocks (no counterpart in the paper): computes one
  * 128-row bf16 product per operand layout the chunk kernels use, from two 128 x 128
  * row-major bf16 device matrices X, Y into D (fp32, row-major):

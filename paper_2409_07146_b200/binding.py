@@ -65,7 +65,7 @@ def lib_path() -> str:
 def exported_symbols():
     return ["gsa_chunk_size", "gsa_workspace_bytes", "gsa_status_string", "gsa_gate_cumsum",
             "gsa_fwd", "gsa_bwd", "gsa_decode_step", "gsa_tc_selftest", "gsa_timing_begin",
-            "gsa_timing_end"]
+            "gsa_timing_end", "gsa_fwd_noalloc"]
 
 
 def load_library():
@@ -94,6 +94,8 @@ def load_library():
     lib.gsa_bwd.restype = ctypes.c_int
     lib.gsa_decode_step.argtypes = [pp] + [vp] * 8
     lib.gsa_decode_step.restype = ctypes.c_int
+    lib.gsa_fwd_noalloc.argtypes = [pp] + [vp] * 10 + [vp, vp]
+    lib.gsa_fwd_noalloc.restype = ctypes.c_int
     lib.gsa_timing_begin.argtypes = [i32]
     lib.gsa_timing_begin.restype = ctypes.c_int
     lib.gsa_timing_end.argtypes = [ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_char_p), i32]
@@ -238,3 +240,26 @@ def gsa_timing_end(capacity: int = 4096):
     if n < 0:
         raise RuntimeError("gsa_timing_end failed")
     return [(labels[i].decode(), float(ms[i])) for i in range(n)]
+
+
+GSA_NOALLOC_MAX_WORKSPACE_BYTES = 32 << 20   # mirror of the macro in include/gsa.h
+
+
+def gsa_fwd_noalloc(p: Params, q, k, v, gate, o, K0=None, V0=None, ok_save=None, KT=None, VT=None,
+                    dev_status=None):
+    """gsa_fwd for callers that cannot allocate device memory: the scratch is a fixed array
+    inside the library (32 MiB per GPU), so the caller passes inputs and outputs only -- `o`
+    must be given, nothing is allocated here either.  Calls that overlap on the GPU share
+    that array and race; shapes that need more scratch raise GsaError (workspace)."""
+    io = p.io_dtype
+    qk, vv, mm = (p.B, p.T, p.H, p.d_k), (p.B, p.T, p.H, p.d_v), (p.B, p.T, p.H, p.m)
+    sk, sv = (p.B, p.H, p.m, p.d_k), (p.B, p.H, p.m, p.d_v)
+    cp = p.c()
+    _check(load_library().gsa_fwd_noalloc(
+        ctypes.byref(cp), _ptr(q, io, qk, "q"), _ptr(k, io, qk, "k"), _ptr(v, io, vv, "v"),
+        _ptr(gate, torch.float32, mm, "gate"), _ptr(K0, torch.float32, sk, "K0"),
+        _ptr(V0, torch.float32, sv, "V0"), _ptr(o, io, vv, "o"),
+        _ptr(ok_save, torch.float32, mm, "ok_save"), _ptr(KT, torch.float32, sk, "KT"),
+        _ptr(VT, torch.float32, sv, "VT"), _stream(),
+        _ptr(dev_status, torch.int32, None, "dev_status")), "gsa_fwd_noalloc")
+    return o
