@@ -44,8 +44,8 @@ constexpr int kHS = kM / 2;            // slots per thread
 // accumulator columns
 constexpr int kColP = 0;       // P / A           [128 x 128]
 constexpr int kColO = 128;     // inter (+ intra for key_side) output
-constexpr int kColU = 256;     // state update    [128 x 64]
-constexpr int kColO2 = 320;    // value_side: intra-chunk output [128 x 64]
+constexpr int kColU = 256;     // state update    [128 x 64] (value_side: [128 x 128], high | low weight parts)
+constexpr int kColO2 = 384;    // value_side: intra-chunk output [128 x 128], high | low weight parts
 
 // Optional phase timing for development builds (-DGSA_TC_PROF): CTA 0 prints, for its fifth
 // chunk, the SM clock at each phase boundary.
@@ -78,8 +78,8 @@ struct Ctl {
     uint32_t tmem_slot;
     volatile int abort;
     volatile int moderate[2];   // decision of the chunk, by chunk parity
-    float gc[kM];        // G of the chunk's last valid row
-    float egc[kM];       // exp(gc)
+    alignas(16) float gc[kM];    // G of the chunk's last valid row
+    alignas(16) float egc[kM];   // exp(gc)
 };
 
 // 8 consecutive fp32 values (columns s0 .. s0+7, s0 % 8 == 0) of row `row` of a slot-sized
@@ -170,18 +170,21 @@ __device__ __forceinline__ void ctl_init(Ctl* ctl, int tid, int warp) {
 template <bool REV>
 __device__ __forceinline__ void store_masked_row(uint32_t tmem, int wq, int row, int half, unsigned char* dst) {
     unsigned char* panel = dst + half * kPanelB;      // columns 64 half .. 64 half + 63
-    float v[64];
-    tmem_ld64(tmem_row_addr(tmem, wq, kColP + 64 * half), v);
+#pragma unroll 1
+    for (int c0 = 0; c0 < 64; c0 += 32) {
+        float v[32];
+        tmem_ld32(tmem_row_addr(tmem, wq, kColP + 64 * half + c0), v);
 #pragma unroll
-    for (int c = 0; c < 8; ++c) {
-        float x[8];
+        for (int c = 0; c < 4; ++c) {
+            float x[8];
 #pragma unroll
-        for (int e = 0; e < 8; ++e) {
-            const int j = 64 * half + 8 * c + e;
-            const bool keep = REV ? (j >= row) : (j <= row);
-            x[e] = keep ? v[8 * c + e] : 0.f;
+            for (int e = 0; e < 8; ++e) {
+                const int j = 64 * half + c0 + 8 * c + e;
+                const bool keep = REV ? (j >= row) : (j <= row);
+                x[e] = keep ? v[8 * c + e] : 0.f;
+            }
+            store_chunk(panel, row, (c0 >> 3) + c, x);
         }
-        store_chunk(panel, row, c, x);
     }
 }
 
@@ -190,6 +193,58 @@ __device__ __forceinline__ void store_masked_row(uint32_t tmem, int wq, int row,
     do {                                                    \
         if (!mbar_wait(bar, parity)) ctl->abort = 1;        \
     } while (0)
+
+// Strong-decay chunk of value_side: this thread's 32 output slots of row `row`,
+//   out[s] = exp(+-..) * inter[s] + sum_j P_ij w_j[s] exp(-|G_i[s] - G_j[s]|),
+// with explicit exponent differences from the fp32 weight and G tiles; P and the inter-chunk
+// product are read from the accumulators; the row goes straight to global memory.
+template <bool REV>
+__device__ __noinline__ void value_side_explicit_rows(const unsigned char* gt, const unsigned char* sW,
+                                                      const float* gc, uint32_t tmem, int wq, int row, int sb,
+                                                      int grow, int valid, float* out_row) {
+    const int jlo = REV ? row : 0, jhi = REV ? kCT - 1 : row;
+    // the accumulator loads are warp-collective: loop bounds are those of the whole warp
+    const int wlo = REV ? wq * 32 : 0, whi = REV ? kCT - 1 : wq * 32 + 31;
+    for (int s0 = sb; s0 < sb + kHS; s0 += 16) {
+        float gi[16], acc[16], tmp[8];
+        tile_row8(gt, grow, s0, tmp);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) gi[e] = tmp[e];
+        tile_row8(gt, grow, s0 + 8, tmp);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) gi[8 + e] = tmp[e];
+#pragma unroll
+        for (int e = 0; e < 16; ++e) acc[e] = 0.f;
+        for (int c0 = wlo; c0 <= whi; c0 += 16) {
+            float v[16];
+            tmem_ld16(tmem_row_addr(tmem, wq, kColP + c0), v);
+#pragma unroll
+            for (int e = 0; e < 16; ++e) {
+                const int j = c0 + e;
+                if (j < jlo || j > jhi) continue;
+                const int jg = min(j, valid - 1);
+#pragma unroll
+                for (int u = 0; u < 16; ++u) {
+                    const float gj = tile_elem(gt, jg, s0 + u);
+                    const float ex = REV ? gj - gi[u] : gi[u] - gj;
+                    acc[u] = fmaf(v[e] * tile_elem(sW, j, s0 + u), __expf(fminf(ex, 0.f)), acc[u]);
+                }
+            }
+        }
+        float vi[16];
+        tmem_ld16(tmem_row_addr(tmem, wq, kColO + s0), vi);
+        if (row < valid) {
+#pragma unroll
+            for (int e = 0; e < 16; e += 4) {
+                float r[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u)
+                    r[u] = fmaf(vi[e + u], __expf(REV ? gc[s0 + e + u] - gi[e + u] : gi[e + u]), acc[e + u]);
+                *reinterpret_cast<float4*>(out_row + s0 + e) = make_float4(r[0], r[1], r[2], r[3]);
+            }
+        }
+    }
+}
 
 // ======================================================================================
 // value_side: out_i[s] = sum_{j<=i} <xq_i, xk_j> w_j[s] decay_ij[s]  + decayed (xq_i S)[s]
@@ -207,9 +262,9 @@ value_side_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_cons
     unsigned char* sG = sXk + 2 * kPanelB;           // G tile fp32, [2 stages][2 panels]         (64 KB)
     unsigned char* sPm = sG + 4 * kPanelB;           // masked P, K-major A, 2 panels             (32 KB)
     unsigned char* sW = sPm;                         //   ... shared with the weight tile fp32, 2 panels
-    unsigned char* sWp = sPm + 2 * kPanelB;          // intra weights, MN-major B [128][64]       (16 KB)
-    unsigned char* sWt = sWp + kPanelB;              // state-update weights, MN-major B [128][64] (16 KB)
-    unsigned char* sSb = sWt + kPanelB;              // state copy, MN-major B [128][64]          (16 KB)
+    unsigned char* sWa = sPm + 2 * kPanelB;          // decayed weights, bf16 high part, MN-major B [128][64] (16 KB)
+    unsigned char* sWb = sWa + kPanelB;              // ... their bf16 rounding residual (low part)           (16 KB)
+    unsigned char* sSb = sWb + kPanelB;              // state copy, MN-major B [128][64]          (16 KB)
     Ctl* ctl = reinterpret_cast<Ctl*>(sSb + kPanelB);
 
     const int tid = threadIdx.x, warp = tid >> 5, wq = warp & 3, half = (tid >> 7) & 1, row = tid & 127;
@@ -253,12 +308,14 @@ value_side_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_cons
             load_x(0);
             constexpr uint32_t idescP = make_idesc(128, 128, false, false);  // xq xk^T
             constexpr uint32_t idescO = make_idesc(128, kM, false, true);    // xq x state copy (MN-major B)
-            constexpr uint32_t idescU = make_idesc(128, kM, true, true);     // xk^T (MN-major A) x W~ (MN-major B)
-            constexpr uint32_t idescI = make_idesc(128, kM, false, true);    // Pm x W' (MN-major B)
+            // the high and the low part of the weights are two adjacent 64-column panels of ONE
+            // MN-major B operand (N = 128): one product yields [.. W_hi | .. W_lo]
+            constexpr uint32_t idescU = make_idesc(128, 2 * kM, true, true);   // xk^T (MN-major A) x [W_hi | W_lo]
+            constexpr uint32_t idescI = make_idesc(128, 2 * kM, false, true);  // Pm x [W_hi | W_lo]
             // base descriptors of every operand (K step 0); advancing along K is one add each
             const uint64_t dQk = desc_kmajor(smem_u32(sXq), 0), dKk = desc_kmajor(smem_u32(sXk), 0);
-            const uint64_t dKm = desc_mnmajor(smem_u32(sXk), 0, kPanelB), dWt = desc_mnmajor(smem_u32(sWt), 0, kPanelB);
-            const uint64_t dS = desc_mnmajor(smem_u32(sSb), 0, kPanelB), dWp = desc_mnmajor(smem_u32(sWp), 0, kPanelB);
+            const uint64_t dKm = desc_mnmajor(smem_u32(sXk), 0, kPanelB), dWa = desc_mnmajor(smem_u32(sWa), 0, kPanelB);
+            const uint64_t dS = desc_mnmajor(smem_u32(sSb), 0, kPanelB);
             const uint64_t dP = desc_kmajor(smem_u32(sPm), 0);
             // byte offset of K step kk: K-major operands walk 32 bytes inside a 64-column panel,
             // MN-major operands walk 16 rows (2048 bytes)
@@ -290,7 +347,7 @@ value_side_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_cons
                     bulk_wait_read();     // the output rows staged in that G buffer one chunk ago have left
                     load_g(it + 1);
                 }
-                // U = xk^T W~ once the operand rows are there
+                // U = xk^T W (high + low part of the weights) once the operand rows are there
                 PROF_MARK();
                 WAIT_OR_ABORT(&ctl->bar_ops, it & 1);
                 tc_fence_after_sync();
@@ -298,7 +355,7 @@ value_side_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_cons
                 const bool moderate = ctl->moderate[it & 1] != 0;
 #pragma unroll
                 for (int kk = 0; kk < kCT / 16; ++kk)
-                    mma_bf16(tmem + kColU, desc_advance(dKm, mnmaj(kk)), desc_advance(dWt, mnmaj(kk)), idescU, kk > 0);
+                    mma_bf16(tmem + kColU, desc_advance(dKm, mnmaj(kk)), desc_advance(dWa, mnmaj(kk)), idescU, kk > 0);
                 mma_commit(&ctl->bar_mma1);
                 PROF_MARK();
                 if (moderate) {
@@ -307,7 +364,7 @@ value_side_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_cons
                     PROF_MARK();
 #pragma unroll
                     for (int kk = 0; kk < kCT / 16; ++kk)
-                        mma_bf16(tmem + kColO2, desc_advance(dP, kmaj(kk)), desc_advance(dWp, mnmaj(kk)), idescI, kk > 0);
+                        mma_bf16(tmem + kColO2, desc_advance(dP, kmaj(kk)), desc_advance(dWa, mnmaj(kk)), idescI, kk > 0);
                     mma_commit(&ctl->bar_mma2);
                     PROF_MARK();
                 }
@@ -365,32 +422,26 @@ value_side_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_cons
 
             // ---- this token's slot rows -> operand rows (rows past the end: zero weights)
             const int grow = min(row, valid - 1);
+            const float strong = moderate ? 0.f : 1.f;      // adds G_C to the exponent of a strong-decay chunk
 #pragma unroll
             for (int s0 = sb; s0 < sb + kHS; s0 += 8) {
-                float g[8], w[8], wp[8], wt[8];
+                float g[8], w[8], wd[8];
                 tile_row8(gt, grow, s0, g);
                 tile_row8(sW, row, s0, w);
-                // Branch-free over the elements (a branch per element would serialise the exps):
-                //   reverse           : intra = state-update weights = w exp(G)
-                //   forward, moderate : intra w exp(-G); state update = intra * exp(G_C)
-                //   forward, strong   : state update w exp(G_C - G); no intra operand
+                // ONE set of decayed weights serves the intra-chunk product and the state update,
+                // branch-free over the elements (a branch per element would serialise the exps):
+                //   reverse           : w exp(G)
+                //   forward, moderate : w exp(-G); the state update gets its exp(G_C) afterwards,
+                //                       S <- exp(G_C) (S + xk^T W)
+                //   forward, strong   : w exp(G_C - G) (state update only; no intra product)
+                // They are stored as a bf16 pair (value + rounding residual): the weights multiply
+                // sums that cancel in the gate gradient, where a plain bf16 rounding is too coarse.
+                const float4 gc0 = *reinterpret_cast<const float4*>(&ctl->gc[s0]);
+                const float4 gc1 = *reinterpret_cast<const float4*>(&ctl->gc[s0 + 4]);
+                const float gcv[8] = {gc0.x, gc0.y, gc0.z, gc0.w, gc1.x, gc1.y, gc1.z, gc1.w};
 #pragma unroll
-                for (int e = 0; e < 8; ++e) {
-                    const float off = (REV || moderate) ? 0.f : ctl->gc[s0 + e];
-                    const float mul = (!REV && moderate) ? ctl->egc[s0 + e] : 1.f;
-#ifdef EXP_NOEXP
-                    wp[e] = w[e] * (REV ? g[e] : off - g[e]);
-#else
-                    wp[e] = w[e] * __expf(REV ? g[e] : off - g[e]);
-#endif
-                    wt[e] = wp[e] * mul;
-                }
-#ifndef EXP_NOBUILDSTORE
-                store_chunk(sWt, row, s0 >> 3, wt);
-                if (moderate) store_chunk(sWp, row, s0 >> 3, wp);
-#else
-                if (wt[0] + wp[3] == 1234.5f) store_chunk(sWt, row, s0 >> 3, wt);
-#endif
+                for (int e = 0; e < 8; ++e) wd[e] = w[e] * __expf(REV ? g[e] : fmaf(strong, gcv[e], -g[e]));
+                store_chunk_split(sWa, sWb, row, s0 >> 3, wd);
             }
             fence_async_smem();
             if (tid == 0) ctl->moderate[it & 1] = moderate;
@@ -409,64 +460,27 @@ value_side_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_cons
                 if (tid == 0) mbar_arrive(&ctl->bar_pm);
             } else {
                 // Strong decay: the intra-chunk term with explicit exponent differences on the CUDA
-                // cores, straight from the fp32 weight and G tiles.
+                // cores (kept out of line so that its registers do not weigh on the common path).
                 WAIT_OR_ABORT(&ctl->bar_mma1, it & 1);    // the inter-chunk product
                 tc_fence_after_sync();
-                const int jlo = REV ? row : 0, jhi = REV ? kCT - 1 : row;
-                // the accumulator loads are warp-collective: loop bounds are those of the whole warp
-                const int wlo = REV ? wq * 32 : 0, whi = REV ? kCT - 1 : wq * 32 + 31;
-                for (int s0 = sb; s0 < sb + kHS; s0 += 16) {
-                    float gi[16], acc[16], tmp[8];
-                    tile_row8(gt, grow, s0, tmp);
-#pragma unroll
-                    for (int e = 0; e < 8; ++e) gi[e] = tmp[e];
-                    tile_row8(gt, grow, s0 + 8, tmp);
-#pragma unroll
-                    for (int e = 0; e < 8; ++e) gi[8 + e] = tmp[e];
-#pragma unroll
-                    for (int e = 0; e < 16; ++e) acc[e] = 0.f;
-                    for (int c0 = wlo; c0 <= whi; c0 += 16) {
-                        float v[16];
-                        tmem_ld16(tmem_row_addr(tmem, wq, kColP + c0), v);
-#pragma unroll
-                        for (int e = 0; e < 16; ++e) {
-                            const int j = c0 + e;
-                            if (j < jlo || j > jhi) continue;
-                            const int jg = min(j, valid - 1);
-#pragma unroll
-                            for (int u = 0; u < 16; ++u) {
-                                const float gj = tile_elem(gt, jg, s0 + u);
-                                const float ex = REV ? gj - gi[u] : gi[u] - gj;
-                                acc[u] = fmaf(v[e] * tile_elem(sW, j, s0 + u), __expf(fminf(ex, 0.f)), acc[u]);
-                            }
-                        }
-                    }
-                    float vi[16];
-                    tmem_ld16(tmem_row_addr(tmem, wq, kColO + s0), vi);
-                    if (row < valid) {
-                        float* dst = obase + (size_t)(t0 + row) * strideM + s0;
-#pragma unroll
-                        for (int e = 0; e < 16; e += 4) {
-                            float r[4];
-#pragma unroll
-                            for (int u = 0; u < 4; ++u)
-                                r[u] = fmaf(vi[e + u], __expf(REV ? ctl->gc[s0 + e + u] - gi[e + u] : gi[e + u]), acc[e + u]);
-                            *reinterpret_cast<float4*>(dst + e) = make_float4(r[0], r[1], r[2], r[3]);
-                        }
-                    }
-                }
+                value_side_explicit_rows<REV>(gt, sW, ctl->gc, tmem, wq, row, sb, grow, valid,
+                                              obase + (size_t)(t0 + row) * strideM);
             }
 
-            // ---- state update from U: S <- S exp(G_C) + U
+            // ---- state update from U: S <- S exp(G_C) + U  (forward moderate chunk: exp(G_C) (S + U))
             PROF_MARK();
             WAIT_OR_ABORT(&ctl->bar_mma1, it & 1);
             tc_fence_after_sync();
             PROF_MARK();
             {
-                float v[kHS];
+                float v[kHS], vl[kHS];
                 tmem_ld32(tmem_row_addr(tmem, wq, kColU + sb), v);
+                tmem_ld32(tmem_row_addr(tmem, wq, kColU + kM + sb), vl);
 #pragma unroll
-                for (int e = 0; e < kHS; ++e) S[e] = fmaf(S[e], ctl->egc[sb + e], v[e]);
+                for (int e = 0; e < kHS; ++e) {
+                    const float u = v[e] + vl[e];
+                    S[e] = (!REV && moderate) ? (S[e] + u) * ctl->egc[sb + e] : fmaf(S[e], ctl->egc[sb + e], u);
+                }
             }
             // its bf16 copy feeds the next chunk's inter-chunk product (issued as soon as the next
             // tiles are there); the product of this chunk that read the old copy is complete
@@ -482,8 +496,11 @@ value_side_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_cons
                 // the scaled rows replace this chunk's G rows in place (each thread reads and rewrites
                 // only its own 32 slots) and leave as one tiled store, clipped at the sequence end
                 float vo[kHS], vi[kHS];
-                tmem_ld32(tmem_row_addr(tmem, wq, kColO + sb), vi);
                 tmem_ld32(tmem_row_addr(tmem, wq, kColO2 + sb), vo);
+                tmem_ld32(tmem_row_addr(tmem, wq, kColO2 + kM + sb), vi);
+#pragma unroll
+                for (int e = 0; e < kHS; ++e) vo[e] += vi[e];          // high + low weight parts
+                tmem_ld32(tmem_row_addr(tmem, wq, kColO + sb), vi);
                 // forward: exp(G) (inter + intra); reverse: exp(-G) (exp(G_C) inter + intra)
 #pragma unroll
                 for (int e = 0; e < kHS; ++e) vo[e] = REV ? fmaf(vi[e], ctl->egc[sb + e], vo[e]) : vo[e] + vi[e];
@@ -526,6 +543,46 @@ value_side_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_cons
     if (warp == 0) {
         __syncwarp();
         tmem_dealloc(tmem, kTmemCols);
+    }
+}
+
+// Strong-decay chunk of key_side: A_ij = sum_s uq_i[s] uk_j[s] exp(-|G_i[s] - G_j[s]|) on the kept
+// triangle, computed with explicit exponent differences from the fp32 uq / uk / G tiles, and
+// written as the bf16 operand rows of the masked matrix (which shares its buffer with the
+// uq tile: every thread first takes its uq row into registers).
+template <bool REV>
+__device__ __noinline__ void key_side_explicit_rows(const unsigned char* sG, const unsigned char* sUq,
+                                                    const unsigned char* sUk, unsigned char* sAm, int row,
+                                                    int half, int grow, int valid) {
+    float gi[kM], qi[kM];
+#pragma unroll
+    for (int s0 = 0; s0 < kM; s0 += 8) {
+        float g[8], uq[8];
+        tile_row8(sG, grow, s0, g);
+        tile_row8(sUq, row, s0, uq);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) { gi[s0 + e] = g[e]; qi[s0 + e] = uq[e]; }
+    }
+    compute_sync();           // every thread has its uq row in registers before sAm is written
+    for (int c0 = 64 * half; c0 < 64 * half + 64; c0 += 8) {
+        float x[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+            const int j = c0 + e;
+            const bool keep = REV ? (j >= row) : (j <= row);
+            float acc = 0.f;
+            if (keep) {
+                const int jg = min(j, valid - 1);
+#pragma unroll
+                for (int s = 0; s < kM; ++s) {
+                    const float gj = tile_elem(sG, jg, s);
+                    const float ex = REV ? gj - gi[s] : gi[s] - gj;
+                    acc = fmaf(qi[s] * tile_elem(sUk, j, s), __expf(fminf(ex, 0.f)), acc);
+                }
+            }
+            x[e] = acc;
+        }
+        store_chunk(sAm + (c0 >> 6) * kPanelB, row, (c0 & 63) >> 3, x);
     }
 }
 
@@ -654,17 +711,23 @@ key_side_tc_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_consta
         for (int s = 0; s < kHS; ++s) S[s] = a.S0 ? a.S0[((size_t)bh * kM + sb + s) * a.D + d0 + row] : 0.f;
 
         int n_mod = 0;     // moderate chunks so far (phases of bar_p)
+        PROF_DECL
         for (int it = 0; it < nchunks; ++it) {
             const int t0 = chunk_t0(it);
             const int valid = min(kCT, a.T - t0);
             (void)t0;
+            PROF_MARK();
             WAIT_OR_ABORT(&ctl->bar_g[0], it & 1);
+            PROF_MARK();
             const bool moderate = publish_chunk_decay(ctl, tid, sG, valid - 1);
             if (ctl->abort) break;
+            PROF_MARK();
 
             const int grow = min(row, valid - 1);
             // the previous chunk's output rows must have left sQt / sKt before they are rewritten
             if (it > 0) WAIT_OR_ABORT(&ctl->bar_sb, (it - 1) & 1);
+            const float strong = moderate ? 0.f : 1.f;     // adds G_C to the exponent of a strong-decay chunk
+            const float modf_ = moderate ? 1.f : 0.f;      // multiplies by exp(G_C) afterwards in a moderate one
             // key side first: it needs the uk and G tiles only; the uq tile (which shares its buffer
             // with the previous chunk's masked A) arrives last
 #pragma unroll
@@ -672,28 +735,45 @@ key_side_tc_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_consta
                 float g[8], uk[8], kb[8], kt[8];
                 tile_row8(sG, grow, s0, g);
                 tile_row8(sUk, row, s0, uk);
+                // One exponential per element (the SFU is the scarce unit here), no branch:
+                //   reverse           : K- = K~ = uk exp(G)
+                //   forward, moderate : K~ = uk exp(-G), K- = K~ exp(G_C)
+                //   forward, strong   : K- = uk exp(G_C - G) (no intra operand)
+                const float4 gc0 = *reinterpret_cast<const float4*>(&ctl->gc[s0]);
+                const float4 gc1 = *reinterpret_cast<const float4*>(&ctl->gc[s0 + 4]);
+                const float4 ec0 = *reinterpret_cast<const float4*>(&ctl->egc[s0]);
+                const float4 ec1 = *reinterpret_cast<const float4*>(&ctl->egc[s0 + 4]);
+                const float gcv[8] = {gc0.x, gc0.y, gc0.z, gc0.w, gc1.x, gc1.y, gc1.z, gc1.w};
+                const float ecv[8] = {ec0.x, ec0.y, ec0.z, ec0.w, ec1.x, ec1.y, ec1.z, ec1.w};
 #pragma unroll
                 for (int e = 0; e < 8; ++e) {
-                    // state term: forward K- = uk exp(G_C - G), reverse uk exp(G); intra term: uk exp(-+G)
-                    const float eg = __expf(g[e]);
-                    kb[e] = uk[e] * (REV ? eg : __expf(ctl->gc[s0 + e] - g[e]));
-                    kt[e] = uk[e] * (REV ? eg : __expf(-g[e]));
+                    kt[e] = uk[e] * __expf(REV ? g[e] : fmaf(strong, gcv[e], -g[e]));
+                    kb[e] = kt[e] * ((!REV) ? fmaf(modf_, ecv[e], 1.f - modf_) : 1.f);
                 }
                 store_chunk(sKb, row, s0 >> 3, kb);
                 if (moderate) store_chunk(sKt, row, s0 >> 3, kt);
             }
+            PROF_MARK();
             WAIT_OR_ABORT(&ctl->bar_w, it & 1);
+            PROF_MARK();
 #pragma unroll
             for (int s0 = sb; s0 < sb + kHS; s0 += 8) {
                 float g[8], uq[8], qb[8], qt[8];
                 tile_row8(sG, grow, s0, g);
                 tile_row8(sUq, row, s0, uq);
+                //   forward           : Q- = Q~ = uq exp(G)
+                //   reverse, moderate : Q~ = uq exp(-G), Q- = Q~ exp(G_C)
+                //   reverse, strong   : Q- = uq exp(G_C - G)
+                const float4 gc0 = *reinterpret_cast<const float4*>(&ctl->gc[s0]);
+                const float4 gc1 = *reinterpret_cast<const float4*>(&ctl->gc[s0 + 4]);
+                const float4 ec0 = *reinterpret_cast<const float4*>(&ctl->egc[s0]);
+                const float4 ec1 = *reinterpret_cast<const float4*>(&ctl->egc[s0 + 4]);
+                const float gcv[8] = {gc0.x, gc0.y, gc0.z, gc0.w, gc1.x, gc1.y, gc1.z, gc1.w};
+                const float ecv[8] = {ec0.x, ec0.y, ec0.z, ec0.w, ec1.x, ec1.y, ec1.z, ec1.w};
 #pragma unroll
                 for (int e = 0; e < 8; ++e) {
-                    // state term: forward Q- = uq exp(G), reverse uq exp(G_C - G); intra term: uq exp(+-G)
-                    const float eg = __expf(g[e]);
-                    qb[e] = uq[e] * (REV ? __expf(ctl->gc[s0 + e] - g[e]) : eg);
-                    qt[e] = uq[e] * (REV ? __expf(-g[e]) : eg);
+                    qt[e] = uq[e] * __expf(REV ? fmaf(strong, gcv[e], -g[e]) : g[e]);
+                    qb[e] = qt[e] * (REV ? fmaf(modf_, ecv[e], 1.f - modf_) : 1.f);
                 }
                 store_chunk(sQb, row, s0 >> 3, qb);
                 if (moderate) store_chunk(sQt, row, s0 >> 3, qt);
@@ -703,53 +783,29 @@ key_side_tc_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_consta
             if (tid == 0) ctl->moderate[it & 1] = moderate;
             compute_sync();
             if (tid == 0) mbar_arrive(&ctl->bar_ops);
+            PROF_MARK();
 
             if (moderate) {
                 WAIT_OR_ABORT(&ctl->bar_p, n_mod & 1);
                 ++n_mod;
                 tc_fence_after_sync();
+                PROF_MARK();
                 store_masked_row<REV>(tmem, wq, row, half, sAm);    // overwrites the uq tile: all rows were read
             } else {
-                // Strong decay: A_ij with explicit exponent differences, from the fp32 uk and G tiles.
-                float gi[kM], qi[kM];
-#pragma unroll
-                for (int s0 = 0; s0 < kM; s0 += 8) {
-                    float g[8], uq[8];
-                    tile_row8(sG, grow, s0, g);
-                    tile_row8(sUq, row, s0, uq);
-#pragma unroll
-                    for (int e = 0; e < 8; ++e) { gi[s0 + e] = g[e]; qi[s0 + e] = uq[e]; }
-                }
-                compute_sync();           // every thread has its uq row in registers before sAm is written
-                for (int c0 = 64 * half; c0 < 64 * half + 64; c0 += 8) {
-                    float x[8];
-#pragma unroll
-                    for (int e = 0; e < 8; ++e) {
-                        const int j = c0 + e;
-                        const bool keep = REV ? (j >= row) : (j <= row);
-                        float acc = 0.f;
-                        if (keep) {
-                            const int jg = min(j, valid - 1);
-#pragma unroll
-                            for (int s = 0; s < kM; ++s) {
-                                const float gj = tile_elem(sG, jg, s);
-                                const float ex = REV ? gj - gi[s] : gi[s] - gj;
-                                acc = fmaf(qi[s] * tile_elem(sUk, j, s), __expf(fminf(ex, 0.f)), acc);
-                            }
-                        }
-                        x[e] = acc;
-                    }
-                    store_chunk(sAm + (c0 >> 6) * kPanelB, row, (c0 & 63) >> 3, x);
-                }
+                // Strong decay: A_ij with explicit exponent differences (kept out of line so that
+                // its registers do not weigh on the common path).
+                key_side_explicit_rows<REV>(sG, sUq, sUk, sAm, row, half, grow, valid);
             }
             fence_async_smem();
             tc_fence_before_sync();
             compute_sync();
             if (tid == 0) mbar_arrive(&ctl->bar_pm);
+            PROF_MARK();
 
             // ---- state update from U^T: S <- exp(G_C) S + U^T
             WAIT_OR_ABORT(&ctl->bar_mma1, it & 1);
             tc_fence_after_sync();
+            PROF_MARK();
             {
                 float v[kHS];
                 tmem_ld32(tmem_row_addr(tmem, wq, kColU + sb), v);
@@ -759,22 +815,27 @@ key_side_tc_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_consta
 
             // ---- output rows -> bf16, staged over the intra operands (consumed since bar_p), stored
             // by the issuing warp, clipped at the sequence end
+            PROF_MARK();
             WAIT_OR_ABORT(&ctl->bar_mma2, it & 1);
             tc_fence_after_sync();
-            {
-                float v[64];
-                tmem_ld64(tmem_row_addr(tmem, wq, kColO + 64 * half), v);
+            PROF_MARK();
+#pragma unroll 1
+            for (int c0 = 0; c0 < 64; c0 += 32) {
+                float v[32];
+                tmem_ld32(tmem_row_addr(tmem, wq, kColO + 64 * half + c0), v);
 #pragma unroll
-                for (int c = 0; c < 8; ++c) {
+                for (int c = 0; c < 4; ++c) {
                     const float x[8] = {v[8 * c], v[8 * c + 1], v[8 * c + 2], v[8 * c + 3],
                                         v[8 * c + 4], v[8 * c + 5], v[8 * c + 6], v[8 * c + 7]};
-                    store_chunk(sQt + half * kPanelB, row, c, x);
+                    store_chunk(sQt + half * kPanelB, row, (c0 >> 3) + c, x);
                 }
             }
             fence_async_smem();
             tc_fence_before_sync();
             compute_sync();
             if (tid == 0) mbar_arrive(&ctl->bar_out);
+            PROF_MARK();
+            PROF_DUMP("key_side compute");
             if (ctl->abort) break;
         }
         if (!ctl->abort && a.Send) {

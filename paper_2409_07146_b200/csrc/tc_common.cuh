@@ -226,6 +226,16 @@ __device__ __forceinline__ void store_chunk(unsigned char* panel, int row, int c
     uint4 v = make_uint4(pack_bf16(x[0], x[1]), pack_bf16(x[2], x[3]), pack_bf16(x[4], x[5]), pack_bf16(x[6], x[7]));
     *reinterpret_cast<uint4*>(panel + swz128(row, chunk16)) = v;
 }
+// The same 8 elements as a bf16 pair hi + lo (lo = the rounding residual of hi): two operand
+// rows whose products, accumulated, carry ~16 mantissa bits of the fp32 values.
+__device__ __forceinline__ void store_chunk_split(unsigned char* panel_hi, unsigned char* panel_lo, int row,
+                                                  int chunk16, const float (&x)[8]) {
+    float lo[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) lo[e] = x[e] - __bfloat162float(__float2bfloat16_rn(x[e]));
+    store_chunk(panel_hi, row, chunk16, x);
+    store_chunk(panel_lo, row, chunk16, lo);
+}
 // one element (row, col) of a panel (col < 64)
 __device__ __forceinline__ void store_elem(unsigned char* panel, int row, int col, float x) {
     *reinterpret_cast<__nv_bfloat16*>(panel + swz128(row, col >> 3) + (col & 7) * 2) = __float2bfloat16_rn(x);
