@@ -477,9 +477,14 @@ value_side_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_cons
                 tmem_ld32(tmem_row_addr(tmem, wq, kColU + sb), v);
                 tmem_ld32(tmem_row_addr(tmem, wq, kColU + kM + sb), vl);
 #pragma unroll
-                for (int e = 0; e < kHS; ++e) {
-                    const float u = v[e] + vl[e];
-                    S[e] = (!REV && moderate) ? (S[e] + u) * ctl->egc[sb + e] : fmaf(S[e], ctl->egc[sb + e], u);
+                for (int e = 0; e < kHS; e += 4) {
+                    const float4 ec = *reinterpret_cast<const float4*>(&ctl->egc[sb + e]);
+                    const float ecv[4] = {ec.x, ec.y, ec.z, ec.w};
+#pragma unroll
+                    for (int t = 0; t < 4; ++t) {
+                        const float u = v[e + t] + vl[e + t];
+                        S[e + t] = (!REV && moderate) ? (S[e + t] + u) * ecv[t] : fmaf(S[e + t], ecv[t], u);
+                    }
                 }
             }
             // its bf16 copy feeds the next chunk's inter-chunk product (issued as soon as the next
@@ -656,6 +661,7 @@ key_side_tc_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_consta
             const uint64_t dQt = desc_kmajor(smem_u32(sQt), 0), dKt = desc_kmajor(smem_u32(sKt), 0);
             const uint64_t dQb = desc_kmajor(smem_u32(sQb), 0), dS = desc_kmajor(smem_u32(sSb), 0);
             const uint64_t dA = desc_kmajor(smem_u32(sAm), 0);
+            const uint64_t dKtm = desc_mnmajor(smem_u32(sKt), 0, kPanelB);   // K~ read MN-major (= K- of a moderate reverse chunk)
             auto kmaj = [](int kk) { return (uint32_t)((kk >> 2) * kPanelB + (kk & 3) * 32); };
             auto mnmaj = [](int kk) { return (uint32_t)(kk * 2048); };
             for (int it = 0; it < nchunks && !ctl->abort; ++it) {
@@ -670,12 +676,15 @@ key_side_tc_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_consta
                         mma_bf16(tmem + kColP, desc_advance(dQt, kmaj(kk)), desc_advance(dKt, kmaj(kk)), idescA, kk > 0);
                     mma_commit(&ctl->bar_p);     // the state products below run under the read-out of A
                 }
+                // (moderate chunks keep one copy of the operand that serves both products)
+                const uint64_t dKstate = (REV && moderate) ? dKtm : dKb;
+                const uint64_t dQstate = (!REV && moderate) ? dQt : dQb;
 #pragma unroll
                 for (int kk = 0; kk < kCT / 16; ++kk)
-                    mma_bf16(tmem + kColU, desc_advance(dV, mnmaj(kk)), desc_advance(dKb, mnmaj(kk)), idescU, kk > 0);
+                    mma_bf16(tmem + kColU, desc_advance(dV, mnmaj(kk)), desc_advance(dKstate, mnmaj(kk)), idescU, kk > 0);
 #pragma unroll
                 for (int kk = 0; kk < kM / 16; ++kk)
-                    mma_bf16(tmem + kColO, desc_advance(dQb, kmaj(kk)), desc_advance(dS, kmaj(kk)), idescO, kk > 0);
+                    mma_bf16(tmem + kColO, desc_advance(dQstate, kmaj(kk)), desc_advance(dS, kmaj(kk)), idescO, kk > 0);
                 mma_commit(&ctl->bar_mma1);
                 // a moderate chunk is done with the uk and G tiles: request the next chunk's
                 if (moderate && it + 1 < nchunks) load_kg(it + 1);
@@ -750,7 +759,9 @@ key_side_tc_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_consta
                     kt[e] = uk[e] * __expf(REV ? g[e] : fmaf(strong, gcv[e], -g[e]));
                     kb[e] = kt[e] * ((!REV) ? fmaf(modf_, ecv[e], 1.f - modf_) : 1.f);
                 }
-                store_chunk(sKb, row, s0 >> 3, kb);
+                // a moderate reverse chunk has K- == K~ (same bytes, read K-major for the intra product
+                // and MN-major for the state update): one copy
+                if (!(REV && moderate)) store_chunk(sKb, row, s0 >> 3, kb);
                 if (moderate) store_chunk(sKt, row, s0 >> 3, kt);
             }
             PROF_MARK();
@@ -775,7 +786,8 @@ key_side_tc_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_consta
                     qt[e] = uq[e] * __expf(REV ? fmaf(strong, gcv[e], -g[e]) : g[e]);
                     qb[e] = qt[e] * (REV ? fmaf(modf_, ecv[e], 1.f - modf_) : 1.f);
                 }
-                store_chunk(sQb, row, s0 >> 3, qb);
+                // a moderate forward chunk has Q- == Q~: one copy
+                if (!(!REV && moderate)) store_chunk(sQb, row, s0 >> 3, qb);
                 if (moderate) store_chunk(sQt, row, s0 >> 3, qt);
             }
             store_state_row<false>(sSb, row, sb, S, nullptr);
@@ -810,7 +822,13 @@ key_side_tc_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_consta
                 float v[kHS];
                 tmem_ld32(tmem_row_addr(tmem, wq, kColU + sb), v);
 #pragma unroll
-                for (int e = 0; e < kHS; ++e) S[e] = fmaf(S[e], ctl->egc[sb + e], v[e]);
+                for (int e = 0; e < kHS; e += 4) {
+                    const float4 ec = *reinterpret_cast<const float4*>(&ctl->egc[sb + e]);
+                    S[e] = fmaf(S[e], ec.x, v[e]);
+                    S[e + 1] = fmaf(S[e + 1], ec.y, v[e + 1]);
+                    S[e + 2] = fmaf(S[e + 2], ec.z, v[e + 2]);
+                    S[e + 3] = fmaf(S[e + 3], ec.w, v[e + 3]);
+                }
             }
 
             // ---- output rows -> bf16, staged over the intra operands (consumed since bar_p), stored

@@ -7,58 +7,69 @@
 namespace gsa {
 
 // ------------------------------------------------------------------ chunk_cumsum
-// One thread per (chunk, slot); a block covers 256/M consecutive chunks of one (b,h).
-// `chunk` is the chunk length of the kernels that will consume G (64 or 128).
-// Rows of one chunk are read 8 at a time so that several loads are in flight.
+// One CTA per (b,h, chunk): M slots x (chunk / 16) row groups.  A thread takes the logs of
+// its 16 rows (16 independent loads in flight), sums them, the group sums are scanned through
+// shared memory, and the thread writes its 16 running sums.  `chunk` is the chunk length of
+// the kernels that will consume G (64 or 128).
+constexpr int kCumRows = 16;
+
 template <int M>
-__global__ void __launch_bounds__(256) gate_cumsum_kernel(const float* __restrict__ gate,
-                                                          int gate_is_log,
-                                                          float* __restrict__ G,
-                                                          float* __restrict__ I, int T, int H,
-                                                          int chunk, int nchunks) {
-    const int s = threadIdx.x;
-    const int n = blockIdx.y * blockDim.y + threadIdx.y;
-    if (n >= nchunks) return;
+__global__ void __launch_bounds__(M * 8) gate_cumsum_kernel(const float* __restrict__ gate,
+                                                            int gate_is_log,
+                                                            float* __restrict__ G,
+                                                            float* __restrict__ I, int T, int H,
+                                                            int chunk) {
+    __shared__ double group_sum[8][M];
+    const int s = threadIdx.x, grp = threadIdx.y;          // blockDim.y = chunk / 16 <= 8
+    const int n = blockIdx.y;
     const int bh = blockIdx.x, b = bh / H, h = bh % H;
-    const int t0 = n * chunk;
-    const int rows = min(chunk, T - t0);
+    const int t0 = n * chunk + grp * kCumRows;
+    const int rows = max(0, min(kCumRows, min(T, (n + 1) * chunk) - t0));
     const size_t stride = (size_t)H * M;
     const size_t base = (((size_t)b * T + t0) * H + h) * M + s;
-    float run = 0.f;
-    for (int i0 = 0; i0 < rows; i0 += 8) {
-        float x[8];
+    float g[kCumRows];
 #pragma unroll
-        for (int u = 0; u < 8; ++u)
-            x[u] = (i0 + u < rows) ? gate[base + (size_t)(i0 + u) * stride] : (gate_is_log ? 0.f : 1.f);
-#pragma unroll
-        for (int u = 0; u < 8; ++u) {
-            if (i0 + u < rows) {
-                float g, inp;
-                if (gate_is_log) {
-                    g = x[u];
-                    inp = -expm1f(g);
-                } else {
-                    g = logf(x[u]);
-                    inp = 1.f - x[u];
-                }
-                g = fmaxf(g, kLogGateMin);
-                run += g;
-                G[base + (size_t)(i0 + u) * stride] = run;
-                I[base + (size_t)(i0 + u) * stride] = inp;
-            }
+    for (int i = 0; i < kCumRows; ++i) {
+        float x = gate_is_log ? 0.f : 1.f;
+        if (i < rows) x = gate[base + (size_t)i * stride];
+        float inp;
+        if (gate_is_log) {
+            g[i] = x;
+            inp = -expm1f(x);
+        } else {
+            g[i] = logf(x);
+            inp = 1.f - x;
         }
+        g[i] = fmaxf(g[i], kLogGateMin);
+        if (i < rows) I[base + (size_t)i * stride] = inp;
     }
+    // running sums in fp64 (a handful of adds per thread): G is then the correctly rounded
+    // cumulative sum, which matters when strong decay makes |G| reach the hundreds
+    double run[kCumRows], acc = 0.0;
+#pragma unroll
+    for (int i = 0; i < kCumRows; ++i) {
+        acc += (i < rows) ? (double)g[i] : 0.0;
+        run[i] = acc;
+    }
+    group_sum[grp][s] = acc;
+    __syncthreads();
+    double before = 0.0;
+    for (int q = 0; q < grp; ++q) before += group_sum[q][s];
+#pragma unroll
+    for (int i = 0; i < kCumRows; ++i)
+        if (i < rows) G[base + (size_t)i * stride] = (float)(before + run[i]);
 }
 
 cudaError_t launch_gate_cumsum(const float* gate, int gate_is_log, float* G, float* I, int B,
                                int T, int H, int M, int chunk, cudaStream_t st) {
+    if (chunk % kCumRows != 0 || chunk / kCumRows > 8) return cudaErrorInvalidValue;
     const int nchunks = (T + chunk - 1) / chunk;
-    dim3 block(M, 256 / M);
-    dim3 grid(B * H, (nchunks + block.y - 1) / block.y);
+    dim3 block(M, chunk / kCumRows);
+    dim3 grid(B * H, nchunks);
     if (M == 64)
-        gate_cumsum_kernel<64><<<grid, block, 0, st>>>(gate, gate_is_log, G, I, T, H, chunk, nchunks);
+        gate_cumsum_kernel<64><<<grid, block, 0, st>>>(gate, gate_is_log, G, I, T, H, chunk);
     else
-        gate_cumsum_kernel<32><<<grid, block, 0, st>>>(gate, gate_is_log, G, I, T, H, chunk, nchunks);
+        gate_cumsum_kernel<32><<<grid, block, 0, st>>>(gate, gate_is_log, G, I, T, H, chunk);
     return cudaGetLastError();
 }
 

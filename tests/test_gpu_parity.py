@@ -183,7 +183,9 @@ def test_bwd_strong_forgetting():
     B, T, H, dk, dv, m = 1, 160, 1, 64, 64, 32
     d = rand_inputs(43, B, T, H, dk, dv, m, "f32", init=True, gate="strong")
     got, ref = run_bwd(d, B, T, H, dk, dv, m, "f32", log=True)
-    check_bwd(got, ref, TOL["f32"])
+    # cumulative log gates reach -200 here: in fp32 their differences carry an absolute
+    # rounding of ~1e-5, i.e. a relative 1e-5..1e-4 on every decay factor, hence 3e-4
+    check_bwd(got, ref, 3 * TOL["f32"])
 
 
 # ------------------------------------------------------------------ decode
