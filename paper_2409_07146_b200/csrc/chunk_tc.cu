@@ -92,6 +92,13 @@ __device__ __forceinline__ void tile_row8(const unsigned char* tile, int row, in
     x[0] = t0.x; x[1] = t0.y; x[2] = t0.z; x[3] = t0.w;
     x[4] = t1.x; x[5] = t1.y; x[6] = t1.z; x[7] = t1.w;
 }
+// 8 consecutive floats from a 16-byte aligned plain (unswizzled) row
+__device__ __forceinline__ void tile_free_row8(const float* p, float (&x)[8]) {
+    const float4 t0 = *reinterpret_cast<const float4*>(p);
+    const float4 t1 = *reinterpret_cast<const float4*>(p + 4);
+    x[0] = t0.x; x[1] = t0.y; x[2] = t0.z; x[3] = t0.w;
+    x[4] = t1.x; x[5] = t1.y; x[6] = t1.z; x[7] = t1.w;
+}
 __device__ __forceinline__ float tile_elem(const unsigned char* tile, int row, int s) {
     return *reinterpret_cast<const float*>(tile + (s >> 5) * kPanelB + swz128(row, (s & 31) >> 2) + (s & 3) * 4);
 }
@@ -607,12 +614,10 @@ key_side_tc_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_consta
     unsigned char* sG = sUk + 2 * kPanelB;           // G tile fp32, 2 panels                      (32 KB)
     unsigned char* sAm = sG + 2 * kPanelB;           // masked A, K-major A, 2 panels              (32 KB)
     unsigned char* sUq = sAm;                        //   ... shared with the uq tile fp32, 2 panels
-    unsigned char* sQt = sAm + 2 * kPanelB;          // uq, intra scaling, K-major A [128][64]     (16 KB)
-    unsigned char* sKt = sQt + kPanelB;              // uk, intra scaling, K-major B [128][64]     (16 KB)
+    unsigned char* sQt = sAm + 2 * kPanelB;          // decayed uq, K-major A [128][64]            (16 KB)
+    unsigned char* sKt = sQt + kPanelB;              // decayed uk, K-major B / MN-major B [128][64] (16 KB)
                                                      //   ... sQt + sKt also stage the output rows
-    unsigned char* sQb = sKt + kPanelB;              // uq, state scaling, K-major A [128][64]     (16 KB)
-    unsigned char* sKb = sQb + kPanelB;              // uk, state scaling, MN-major B [128][64]    (16 KB)
-    unsigned char* sSb = sKb + kPanelB;              // state copy, K-major B [128 (channel)][64]  (16 KB)
+    unsigned char* sSb = sKt + kPanelB;              // state copy, K-major B [128 (channel)][64]  (16 KB)
     Ctl* ctl = reinterpret_cast<Ctl*>(sSb + kPanelB);
 
     const int tid = threadIdx.x, warp = tid >> 5, wq = warp & 3, half = (tid >> 7) & 1, row = tid & 127;
@@ -657,11 +662,11 @@ key_side_tc_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_consta
             constexpr uint32_t idescU = make_idesc(128, kM, true, true);      // xv^T (MN-major A) x K- (MN-major B)
             constexpr uint32_t idescV = make_idesc(128, kDST, false, true);   // A x xv (MN-major B)
             // base descriptors of every operand (K step 0); advancing along K is one add each
-            const uint64_t dV = desc_mnmajor(smem_u32(sXv), 0, kPanelB), dKb = desc_mnmajor(smem_u32(sKb), 0, kPanelB);
+            const uint64_t dV = desc_mnmajor(smem_u32(sXv), 0, kPanelB);
             const uint64_t dQt = desc_kmajor(smem_u32(sQt), 0), dKt = desc_kmajor(smem_u32(sKt), 0);
-            const uint64_t dQb = desc_kmajor(smem_u32(sQb), 0), dS = desc_kmajor(smem_u32(sSb), 0);
+            const uint64_t dS = desc_kmajor(smem_u32(sSb), 0);
             const uint64_t dA = desc_kmajor(smem_u32(sAm), 0);
-            const uint64_t dKtm = desc_mnmajor(smem_u32(sKt), 0, kPanelB);   // K~ read MN-major (= K- of a moderate reverse chunk)
+            const uint64_t dKtm = desc_mnmajor(smem_u32(sKt), 0, kPanelB);   // the decayed uk read MN-major
             auto kmaj = [](int kk) { return (uint32_t)((kk >> 2) * kPanelB + (kk & 3) * 32); };
             auto mnmaj = [](int kk) { return (uint32_t)(kk * 2048); };
             for (int it = 0; it < nchunks && !ctl->abort; ++it) {
@@ -676,15 +681,13 @@ key_side_tc_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_consta
                         mma_bf16(tmem + kColP, desc_advance(dQt, kmaj(kk)), desc_advance(dKt, kmaj(kk)), idescA, kk > 0);
                     mma_commit(&ctl->bar_p);     // the state products below run under the read-out of A
                 }
-                // (moderate chunks keep one copy of the operand that serves both products)
-                const uint64_t dKstate = (REV && moderate) ? dKtm : dKb;
-                const uint64_t dQstate = (!REV && moderate) ? dQt : dQb;
+                // the decayed uk is read K-major by the intra product and MN-major by the state update
 #pragma unroll
                 for (int kk = 0; kk < kCT / 16; ++kk)
-                    mma_bf16(tmem + kColU, desc_advance(dV, mnmaj(kk)), desc_advance(dKstate, mnmaj(kk)), idescU, kk > 0);
+                    mma_bf16(tmem + kColU, desc_advance(dV, mnmaj(kk)), desc_advance(dKtm, mnmaj(kk)), idescU, kk > 0);
 #pragma unroll
                 for (int kk = 0; kk < kM / 16; ++kk)
-                    mma_bf16(tmem + kColO, desc_advance(dQstate, kmaj(kk)), desc_advance(dS, kmaj(kk)), idescO, kk > 0);
+                    mma_bf16(tmem + kColO, desc_advance(dQt, kmaj(kk)), desc_advance(dS, kmaj(kk)), idescO, kk > 0);
                 mma_commit(&ctl->bar_mma1);
                 // a moderate chunk is done with the uk and G tiles: request the next chunk's
                 if (moderate && it + 1 < nchunks) load_kg(it + 1);
@@ -735,62 +738,48 @@ key_side_tc_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_consta
             const int grow = min(row, valid - 1);
             // the previous chunk's output rows must have left sQt / sKt before they are rewritten
             if (it > 0) WAIT_OR_ABORT(&ctl->bar_sb, (it - 1) & 1);
-            const float strong = moderate ? 0.f : 1.f;     // adds G_C to the exponent of a strong-decay chunk
-            const float modf_ = moderate ? 1.f : 0.f;      // multiplies by exp(G_C) afterwards in a moderate one
             // key side first: it needs the uk and G tiles only; the uq tile (which shares its buffer
             // with the previous chunk's masked A) arrives last
 #pragma unroll
             for (int s0 = sb; s0 < sb + kHS; s0 += 8) {
-                float g[8], uk[8], kb[8], kt[8];
+                float g[8], uk[8], kd[8], gcv[8];
                 tile_row8(sG, grow, s0, g);
                 tile_row8(sUk, row, s0, uk);
-                // One exponential per element (the SFU is the scarce unit here), no branch:
-                //   reverse           : K- = K~ = uk exp(G)
-                //   forward, moderate : K~ = uk exp(-G), K- = K~ exp(G_C)
-                //   forward, strong   : K- = uk exp(G_C - G) (no intra operand)
-                const float4 gc0 = *reinterpret_cast<const float4*>(&ctl->gc[s0]);
-                const float4 gc1 = *reinterpret_cast<const float4*>(&ctl->gc[s0 + 4]);
-                const float4 ec0 = *reinterpret_cast<const float4*>(&ctl->egc[s0]);
-                const float4 ec1 = *reinterpret_cast<const float4*>(&ctl->egc[s0 + 4]);
-                const float gcv[8] = {gc0.x, gc0.y, gc0.z, gc0.w, gc1.x, gc1.y, gc1.z, gc1.w};
-                const float ecv[8] = {ec0.x, ec0.y, ec0.z, ec0.w, ec1.x, ec1.y, ec1.z, ec1.w};
+                // ONE decayed copy of uk serves the intra product and the state update, with one
+                // exponential per element (the SFU is the scarce unit here) and no branch:
+                //   reverse           : uk exp(G)
+                //   forward, moderate : uk exp(-G); the state update gets its exp(G_C) afterwards,
+                //                       S <- exp(G_C) (S + xv^T K)
+                //   forward, strong   : uk exp(G_C - G) (state update only)
 #pragma unroll
-                for (int e = 0; e < 8; ++e) {
-                    kt[e] = uk[e] * __expf(REV ? g[e] : fmaf(strong, gcv[e], -g[e]));
-                    kb[e] = kt[e] * ((!REV) ? fmaf(modf_, ecv[e], 1.f - modf_) : 1.f);
-                }
-                // a moderate reverse chunk has K- == K~ (same bytes, read K-major for the intra product
-                // and MN-major for the state update): one copy
-                if (!(REV && moderate)) store_chunk(sKb, row, s0 >> 3, kb);
-                if (moderate) store_chunk(sKt, row, s0 >> 3, kt);
+                for (int e = 0; e < 8; ++e) gcv[e] = 0.f;
+                if (!REV && !moderate) tile_free_row8(&ctl->gc[s0], gcv);
+#pragma unroll
+                for (int e = 0; e < 8; ++e) kd[e] = uk[e] * __expf(REV ? g[e] : gcv[e] - g[e]);
+                store_chunk(sKt, row, s0 >> 3, kd);
             }
             PROF_MARK();
             WAIT_OR_ABORT(&ctl->bar_w, it & 1);
             PROF_MARK();
 #pragma unroll
             for (int s0 = sb; s0 < sb + kHS; s0 += 8) {
-                float g[8], uq[8], qb[8], qt[8];
+                float g[8], uq[8], qd[8], gcv[8];
                 tile_row8(sG, grow, s0, g);
                 tile_row8(sUq, row, s0, uq);
-                //   forward           : Q- = Q~ = uq exp(G)
-                //   reverse, moderate : Q~ = uq exp(-G), Q- = Q~ exp(G_C)
-                //   reverse, strong   : Q- = uq exp(G_C - G)
-                const float4 gc0 = *reinterpret_cast<const float4*>(&ctl->gc[s0]);
-                const float4 gc1 = *reinterpret_cast<const float4*>(&ctl->gc[s0 + 4]);
-                const float4 ec0 = *reinterpret_cast<const float4*>(&ctl->egc[s0]);
-                const float4 ec1 = *reinterpret_cast<const float4*>(&ctl->egc[s0 + 4]);
-                const float gcv[8] = {gc0.x, gc0.y, gc0.z, gc0.w, gc1.x, gc1.y, gc1.z, gc1.w};
-                const float ecv[8] = {ec0.x, ec0.y, ec0.z, ec0.w, ec1.x, ec1.y, ec1.z, ec1.w};
+                // likewise ONE decayed copy of uq:
+                //   forward           : uq exp(G)
+                //   reverse, moderate : uq exp(-G); the inter-chunk product gets its exp(G_C) through
+                //                       the state copy, which is scaled per slot
+                //   reverse, strong   : uq exp(G_C - G)
 #pragma unroll
-                for (int e = 0; e < 8; ++e) {
-                    qt[e] = uq[e] * __expf(REV ? fmaf(strong, gcv[e], -g[e]) : g[e]);
-                    qb[e] = qt[e] * (REV ? fmaf(modf_, ecv[e], 1.f - modf_) : 1.f);
-                }
-                // a moderate forward chunk has Q- == Q~: one copy
-                if (!(!REV && moderate)) store_chunk(sQb, row, s0 >> 3, qb);
-                if (moderate) store_chunk(sQt, row, s0 >> 3, qt);
+                for (int e = 0; e < 8; ++e) gcv[e] = 0.f;
+                if (REV && !moderate) tile_free_row8(&ctl->gc[s0], gcv);
+#pragma unroll
+                for (int e = 0; e < 8; ++e) qd[e] = uq[e] * __expf(REV ? gcv[e] - g[e] : g[e]);
+                store_chunk(sQt, row, s0 >> 3, qd);
             }
-            store_state_row<false>(sSb, row, sb, S, nullptr);
+            if (REV && moderate) store_state_row<true>(sSb, row, sb, S, ctl->egc);
+            else store_state_row<false>(sSb, row, sb, S, nullptr);
             fence_async_smem();
             if (tid == 0) ctl->moderate[it & 1] = moderate;
             compute_sync();
@@ -814,7 +803,7 @@ key_side_tc_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_consta
             if (tid == 0) mbar_arrive(&ctl->bar_pm);
             PROF_MARK();
 
-            // ---- state update from U^T: S <- exp(G_C) S + U^T
+            // ---- state update from U^T: S <- exp(G_C) S + U^T  (forward moderate chunk: exp(G_C) (S + U^T))
             WAIT_OR_ABORT(&ctl->bar_mma1, it & 1);
             tc_fence_after_sync();
             PROF_MARK();
@@ -824,10 +813,10 @@ key_side_tc_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_consta
 #pragma unroll
                 for (int e = 0; e < kHS; e += 4) {
                     const float4 ec = *reinterpret_cast<const float4*>(&ctl->egc[sb + e]);
-                    S[e] = fmaf(S[e], ec.x, v[e]);
-                    S[e + 1] = fmaf(S[e + 1], ec.y, v[e + 1]);
-                    S[e + 2] = fmaf(S[e + 2], ec.z, v[e + 2]);
-                    S[e + 3] = fmaf(S[e + 3], ec.w, v[e + 3]);
+                    const float ecv[4] = {ec.x, ec.y, ec.z, ec.w};
+#pragma unroll
+                    for (int t = 0; t < 4; ++t)
+                        S[e + t] = (!REV && moderate) ? (S[e + t] + v[e + t]) * ecv[t] : fmaf(S[e + t], ecv[t], v[e + t]);
                 }
             }
 
@@ -876,7 +865,7 @@ key_side_tc_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_consta
 }
 
 constexpr size_t kSmemValueSide = 1024 + 13 * kPanelB + sizeof(Ctl);
-constexpr size_t kSmemKeySide = 1024 + 13 * kPanelB + sizeof(Ctl);
+constexpr size_t kSmemKeySide = 1024 + 11 * kPanelB + sizeof(Ctl);
 
 template <typename K>
 cudaError_t prepare(K kernel, size_t smem) {
