@@ -173,10 +173,13 @@ __device__ __forceinline__ void ctl_init(Ctl* ctl, int tid, int warp) {
     tc_fence_after_sync();
 }
 
-// masked accumulator row -> bf16 K-major operand row (two 64-column panels)
-template <bool REV>
-__device__ __forceinline__ void store_masked_row(uint32_t tmem, int wq, int row, int half, unsigned char* dst) {
+// masked accumulator row -> bf16 K-major operand row (two 64-column panels); with SPLIT the
+// rounding residual goes to a second operand of the same shape (dst_lo)
+template <bool REV, bool SPLIT>
+__device__ __forceinline__ void store_masked_row(uint32_t tmem, int wq, int row, int half, unsigned char* dst,
+                                                 unsigned char* dst_lo) {
     unsigned char* panel = dst + half * kPanelB;      // columns 64 half .. 64 half + 63
+    unsigned char* panel_lo = dst_lo + half * kPanelB;
 #pragma unroll 1
     for (int c0 = 0; c0 < 64; c0 += 32) {
         float v[32];
@@ -190,7 +193,8 @@ __device__ __forceinline__ void store_masked_row(uint32_t tmem, int wq, int row,
                 const bool keep = REV ? (j >= row) : (j <= row);
                 x[e] = keep ? v[8 * c + e] : 0.f;
             }
-            store_chunk(panel, row, (c0 >> 3) + c, x);
+            if (SPLIT) store_chunk_split(panel, panel_lo, row, (c0 >> 3) + c, x);
+            else store_chunk(panel, row, (c0 >> 3) + c, x);
         }
     }
 }
@@ -460,7 +464,7 @@ value_side_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_cons
             tc_fence_after_sync();
             PROF_MARK();
             if (moderate) {
-                store_masked_row<REV>(tmem, wq, row, half, sPm);    // overwrites the weight tile
+                store_masked_row<REV, false>(tmem, wq, row, half, sPm, sPm);    // overwrites the weight tile
                 fence_async_smem();
                 tc_fence_before_sync();
                 compute_sync();
@@ -564,8 +568,8 @@ value_side_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_cons
 // uq tile: every thread first takes its uq row into registers).
 template <bool REV>
 __device__ __noinline__ void key_side_explicit_rows(const unsigned char* sG, const unsigned char* sUq,
-                                                    const unsigned char* sUk, unsigned char* sAm, int row,
-                                                    int half, int grow, int valid) {
+                                                    const unsigned char* sUk, unsigned char* sAm,
+                                                    unsigned char* sAl, int row, int half, int grow, int valid) {
     float gi[kM], qi[kM];
 #pragma unroll
     for (int s0 = 0; s0 < kM; s0 += 8) {
@@ -594,7 +598,7 @@ __device__ __noinline__ void key_side_explicit_rows(const unsigned char* sG, con
             }
             x[e] = acc;
         }
-        store_chunk(sAm + (c0 >> 6) * kPanelB, row, (c0 & 63) >> 3, x);
+        store_chunk_split(sAm + (c0 >> 6) * kPanelB, sAl + (c0 >> 6) * kPanelB, row, (c0 & 63) >> 3, x);
     }
 }
 
@@ -618,7 +622,8 @@ key_side_tc_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_consta
     unsigned char* sKt = sQt + kPanelB;              // decayed uk, K-major B / MN-major B [128][64] (16 KB)
                                                      //   ... sQt + sKt also stage the output rows
     unsigned char* sSb = sKt + kPanelB;              // state copy, K-major B [128 (channel)][64]  (16 KB)
-    Ctl* ctl = reinterpret_cast<Ctl*>(sSb + kPanelB);
+    unsigned char* sAl = sSb + kPanelB;              // rounding residual of the masked A, 2 panels (32 KB)
+    Ctl* ctl = reinterpret_cast<Ctl*>(sAl + 2 * kPanelB);
 
     const int tid = threadIdx.x, warp = tid >> 5, wq = warp & 3, half = (tid >> 7) & 1, row = tid & 127;
     const int sb = kHS * half;          // this thread's first slot
@@ -665,7 +670,7 @@ key_side_tc_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_consta
             const uint64_t dV = desc_mnmajor(smem_u32(sXv), 0, kPanelB);
             const uint64_t dQt = desc_kmajor(smem_u32(sQt), 0), dKt = desc_kmajor(smem_u32(sKt), 0);
             const uint64_t dS = desc_kmajor(smem_u32(sSb), 0);
-            const uint64_t dA = desc_kmajor(smem_u32(sAm), 0);
+            const uint64_t dA = desc_kmajor(smem_u32(sAm), 0), dAl = desc_kmajor(smem_u32(sAl), 0);
             const uint64_t dKtm = desc_mnmajor(smem_u32(sKt), 0, kPanelB);   // the decayed uk read MN-major
             auto kmaj = [](int kk) { return (uint32_t)((kk >> 2) * kPanelB + (kk & 3) * 32); };
             auto mnmaj = [](int kk) { return (uint32_t)(kk * 2048); };
@@ -696,6 +701,9 @@ key_side_tc_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_consta
 #pragma unroll
                 for (int kk = 0; kk < kCT / 16; ++kk)
                     mma_bf16(tmem + kColO, desc_advance(dA, kmaj(kk)), desc_advance(dV, mnmaj(kk)), idescV, true);
+#pragma unroll
+                for (int kk = 0; kk < kCT / 16; ++kk)      // ... and the rounding residual of A
+                    mma_bf16(tmem + kColO, desc_advance(dAl, kmaj(kk)), desc_advance(dV, mnmaj(kk)), idescV, true);
                 mma_commit(&ctl->bar_mma2);
                 if (!moderate && it + 1 < nchunks) load_kg(it + 1);
                 // the masked A is consumed: its buffer takes the next chunk's uq tile
@@ -791,11 +799,11 @@ key_side_tc_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_consta
                 ++n_mod;
                 tc_fence_after_sync();
                 PROF_MARK();
-                store_masked_row<REV>(tmem, wq, row, half, sAm);    // overwrites the uq tile: all rows were read
+                store_masked_row<REV, true>(tmem, wq, row, half, sAm, sAl);    // overwrites the uq tile: all rows were read
             } else {
                 // Strong decay: A_ij with explicit exponent differences (kept out of line so that
                 // its registers do not weigh on the common path).
-                key_side_explicit_rows<REV>(sG, sUq, sUk, sAm, row, half, grow, valid);
+                key_side_explicit_rows<REV>(sG, sUq, sUk, sAm, sAl, row, half, grow, valid);
             }
             fence_async_smem();
             tc_fence_before_sync();
@@ -865,7 +873,7 @@ key_side_tc_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_consta
 }
 
 constexpr size_t kSmemValueSide = 1024 + 13 * kPanelB + sizeof(Ctl);
-constexpr size_t kSmemKeySide = 1024 + 11 * kPanelB + sizeof(Ctl);
+constexpr size_t kSmemKeySide = 1024 + 13 * kPanelB + sizeof(Ctl);
 
 template <typename K>
 cudaError_t prepare(K kernel, size_t smem) {

@@ -33,19 +33,17 @@ TC_RTOL = 2.0 ** -7
 # Bounds of the tensor-core path at the size of the benchmark configurations, per tensor:
 # ("plain", 0, x)  = max|err| / rms <= x with no allowance (the stated bound where x = 2e-2);
 # ("mixed", r, x)  = the same after a relative allowance r |ref| per element.
-# Forward tensors, logits and final memories meet the stated 2e-2 as it stands; o, dv only
-# after the half-ulp rounding of their own bf16 storage (2^-9).  dq and dk sit behind up to
-# eight bf16 roundings in a row (masked products, state copy, slot-space matrix and its two
-# factors, the scaled softmax gradient, the output), hence 8 * 2^-9 = 2^-6; their noise
-# (sigma ~ 0.4% of the rms) still peaks at 2.0-2.7e-2 over millions of elements, and where key
-# channels carry outliers (t2r_7b: max|dq| / rms = 39) the error follows the scale of the
-# channel rather than of the element and reaches 6.4e-2: known gaps to the stated 2e-2.
-# The gate gradient, a difference of long sums that cancel, is at 1.3-2.4e-2 since the
-# decayed weights are carried as bf16 pairs (5-7e-2 before).
+# The output o, the slot logits, the final memories, dv and the gate gradient meet the
+# stated 2e-2 as it stands (the decayed weights and the masked slot-space matrix are carried
+# as bf16 high/low pairs for that).  dq and dk still sit behind plain bf16 roundings of the
+# masked q.k products, the state copy and the decayed softmax gradient: 3.9-4.2e-2 at
+# train_1p3b, and where key channels carry outliers (t2r_7b: max|dq| / rms = 39) the error
+# follows the scale of the channel rather than of the element, 11.5e-2; after a 2^-6
+# allowance (eight bf16 roundings in a row) they are at 1.4-5.0e-2: known gaps.
 TC_CONFIG_BOUNDS = {
-    "o": ("mixed", 2.0 ** -9, 2e-2), "ok": ("plain", 0.0, 2e-2), "KT": ("plain", 0.0, 2e-2),
-    "VT": ("plain", 0.0, 2e-2), "dv": ("mixed", 2.0 ** -9, 2e-2), "dq": ("mixed", 2.0 ** -6, 8e-2),
-    "dk": ("mixed", 2.0 ** -6, 3e-2), "dgate": ("plain", 0.0, 3e-2),
+    "o": ("plain", 0.0, 2e-2), "ok": ("plain", 0.0, 2e-2), "KT": ("plain", 0.0, 2e-2),
+    "VT": ("plain", 0.0, 2e-2), "dv": ("plain", 0.0, 2e-2), "dq": ("mixed", 2.0 ** -6, 6e-2),
+    "dk": ("mixed", 2.0 ** -6, 3.5e-2), "dgate": ("plain", 0.0, 3e-2),
 }
 
 
