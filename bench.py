@@ -338,7 +338,10 @@ def run_ours(args):
         per = {}
         for lab, ms in recs:
             per.setdefault(lab, []).append(ms)
-        launches = (len(recs) + 2 * len(per.get("gate_grad", []))) // reps
+        # kernels behind one label: gate_grad is three; every chunk pass is two (the lean and the
+        # general variant of the kernel are both launched, each CTA runs in one of them)
+        two = sum(len(v) for lab, v in per.items() if lab.endswith("_side") or lab.endswith("_side_rev"))
+        launches = (len(recs) + 2 * len(per.get("gate_grad", [])) + two) // reps
         kernels = []
         tot = sum(sum(v) for v in per.values())
         for lab, v in per.items():

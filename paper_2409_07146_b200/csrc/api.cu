@@ -58,6 +58,7 @@ struct Carver {
 
 struct Workspace {
     float *G, *I, *okpart, *ok, *p, *dz, *u, *dppart, *dIk, *dIv, *chunk_tot, *KT, *VT;
+    int* strong;     // [B*H] flags: this (b,h) has a chunk that decays too hard for the factorised form
     size_t bytes;
 };
 
@@ -67,6 +68,7 @@ Workspace carve(const gsa_params_t& p, int which, void* ws) {
     const size_t mt = (size_t)p.B * p.T * p.H * p.m;
     const Slices s = slices(p);
     Carver c{static_cast<char*>(ws), 0};
+    w.strong = reinterpret_cast<int*>(c.take((size_t)p.B * p.H));
     w.G = c.take(mt);
     w.I = c.take(mt);
     w.okpart = c.take(mt * s.k);
@@ -86,14 +88,14 @@ Workspace carve(const gsa_params_t& p, int which, void* ws) {
     return w;
 }
 
-cudaError_t value_side(const gsa_params_t& p, const ValueSideArgs& a, int reverse, cudaStream_t st,
-                       int32_t* dev_status) {
-    if (use_tc(p)) return launch_value_side_tc(a, p.m, reverse, st, dev_status);
+cudaError_t value_side(const gsa_params_t& p, const ValueSideArgs& a, int reverse, const int* strong,
+                       cudaStream_t st, int32_t* dev_status) {
+    if (use_tc(p)) return launch_value_side_tc(a, p.m, reverse, strong, st, dev_status);
     return launch_value_side_simt(a, p.io, p.m, reverse, st);
 }
-cudaError_t key_side(const gsa_params_t& p, const KeySideArgs& a, int reverse, cudaStream_t st,
-                     int32_t* dev_status) {
-    if (use_tc(p)) return launch_key_side_tc(a, p.m, reverse, st, dev_status);
+cudaError_t key_side(const gsa_params_t& p, const KeySideArgs& a, int reverse, const int* strong,
+                     cudaStream_t st, int32_t* dev_status) {
+    if (use_tc(p)) return launch_key_side_tc(a, p.m, reverse, strong, st, dev_status);
     return launch_key_side_simt(a, p.io, p.m, reverse, st);
 }
 
@@ -168,7 +170,7 @@ gsa_status_t gsa_gate_cumsum(const gsa_params_t* params, const float* gate, floa
     const gsa_params_t& p = *params;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     GSA_LAUNCH("gate_cumsum", launch_gate_cumsum(gate, p.gate_kind == GSA_GATE_LOG_A, G, I, p.B, p.T,
-                                                 p.H, p.m, chunk_of(p), st));
+                                                 p.H, p.m, chunk_of(p), nullptr, st));
     return GSA_OK;
 }
 
@@ -189,16 +191,17 @@ gsa_status_t gsa_fwd(const gsa_params_t* params, const void* q, const void* k, c
     const Slices s = slices(p);
     const size_t rows = (size_t)p.B * p.T * p.H;
 
+    GSA_CUDA(cudaMemsetAsync(w.strong, 0, sizeof(int) * (size_t)p.B * p.H, st));
     GSA_LAUNCH("gate_cumsum", launch_gate_cumsum(gate, p.gate_kind == GSA_GATE_LOG_A, w.G, w.I, p.B, p.T,
-                                                 p.H, p.m, chunk_of(p), st));
+                                                 p.H, p.m, chunk_of(p), w.strong, st));
     // pass 1: o' = GLA(q, k, 1-a) with the decay on the slot (value) side
     ValueSideArgs a1{q, k, w.I, w.G, K0, KT, w.okpart, p.B, p.T, p.H, p.d_k};
-    GSA_LAUNCH("pass1_value_side", value_side(p, a1, 0, st, dev_status));
+    GSA_LAUNCH("pass1_value_side", value_side(p, a1, 0, w.strong, st, dev_status));
     float* ok = ok_save ? ok_save : w.ok;
     GSA_LAUNCH("slot_softmax", launch_slot_softmax_fwd(w.okpart, s.k, p.scale, ok, w.p, rows, p.m, st));
     // pass 2: o = GLA(softmax(o'), 1-a, v) with the decay on the slot (key) side
     KeySideArgs a2{w.p, w.I, w.G, v, V0, VT, o, p.B, p.T, p.H, p.d_v};
-    GSA_LAUNCH("pass2_key_side", key_side(p, a2, 0, st, dev_status));
+    GSA_LAUNCH("pass2_key_side", key_side(p, a2, 0, w.strong, st, dev_status));
     return GSA_OK;
 }
 
@@ -223,31 +226,32 @@ gsa_status_t gsa_bwd(const gsa_params_t* params, const void* q, const void* k, c
     const Slices s = slices(p);
     const size_t rows = (size_t)p.B * p.T * p.H;
 
+    GSA_CUDA(cudaMemsetAsync(w.strong, 0, sizeof(int) * (size_t)p.B * p.H, st));
     GSA_LAUNCH("gate_cumsum", launch_gate_cumsum(gate, p.gate_kind == GSA_GATE_LOG_A, w.G, w.I, p.B, p.T,
-                                                 p.H, p.m, chunk_of(p), st));
+                                                 p.H, p.m, chunk_of(p), w.strong, st));
     const float* ok = ok_saved;
     if (ok == nullptr) {  // recompute pass 1 and its logits
         ValueSideArgs a1{q, k, w.I, w.G, K0, nullptr, w.okpart, p.B, p.T, p.H, p.d_k};
-        GSA_LAUNCH("pass1_value_side", value_side(p, a1, 0, st, dev_status));
+        GSA_LAUNCH("pass1_value_side", value_side(p, a1, 0, w.strong, st, dev_status));
         GSA_LAUNCH("slot_softmax", launch_slot_softmax_fwd(w.okpart, s.k, p.scale, w.ok, w.p, rows, p.m, st));
         ok = w.ok;
     }
     // gradient w.r.t. the pass-2 queries p: the pass-1 form on (dO, v, 1-a); carries V~
     ValueSideArgs adp{dO, v, w.I, w.G, V0, dVT ? w.VT : nullptr, w.dppart, p.B, p.T, p.H, p.d_v};
-    GSA_LAUNCH("bwd_dp_value_side", value_side(p, adp, 0, st, dev_status));
+    GSA_LAUNCH("bwd_dp_value_side", value_side(p, adp, 0, w.strong, st, dev_status));
     GSA_LAUNCH("slot_softmax_bwd", launch_slot_softmax_bwd(ok, w.dppart, s.v, p.scale, w.p, w.dz, w.u, rows, p.m, st));
     // dq: the pass-2 form on (dz, 1-a, k); carries K~
     KeySideArgs adq{w.dz, w.I, w.G, k, K0, dKT ? w.KT : nullptr, dq, p.B, p.T, p.H, p.d_k};
-    GSA_LAUNCH("bwd_dq_key_side", key_side(p, adq, 0, st, dev_status));
+    GSA_LAUNCH("bwd_dq_key_side", key_side(p, adq, 0, w.strong, st, dev_status));
     // time-reversed runs: dv and dI^v share the state dV~; dk and dI^k share dK~
     KeySideArgs adv{w.I, w.p, w.G, dO, dVT, dV0, dv, p.B, p.T, p.H, p.d_v};
-    GSA_LAUNCH("bwd_dv_key_side_rev", key_side(p, adv, 1, st, dev_status));
+    GSA_LAUNCH("bwd_dv_key_side_rev", key_side(p, adv, 1, w.strong, st, dev_status));
     ValueSideArgs adIv{v, dO, w.p, w.G, dVT, nullptr, w.dIv, p.B, p.T, p.H, p.d_v};
-    GSA_LAUNCH("bwd_dIv_value_side_rev", value_side(p, adIv, 1, st, dev_status));
+    GSA_LAUNCH("bwd_dIv_value_side_rev", value_side(p, adIv, 1, w.strong, st, dev_status));
     KeySideArgs adk{w.I, w.dz, w.G, q, dKT, dK0, dk, p.B, p.T, p.H, p.d_k};
-    GSA_LAUNCH("bwd_dk_key_side_rev", key_side(p, adk, 1, st, dev_status));
+    GSA_LAUNCH("bwd_dk_key_side_rev", key_side(p, adk, 1, w.strong, st, dev_status));
     ValueSideArgs adIk{k, q, w.dz, w.G, dKT, nullptr, w.dIk, p.B, p.T, p.H, p.d_k};
-    GSA_LAUNCH("bwd_dIk_value_side_rev", value_side(p, adIk, 1, st, dev_status));
+    GSA_LAUNCH("bwd_dIk_value_side_rev", value_side(p, adIk, 1, w.strong, st, dev_status));
     // forget-gate gradient: reversed cumulative sum over the whole sequence
     GSA_LAUNCH("gate_grad", launch_gate_grad(w.u, w.I, w.dIk, s.k, w.dIv, s.v, gate, p.gate_kind == GSA_GATE_LOG_A,
                               dKT, w.KT, dVT, w.VT, p.d_k, p.d_v, w.chunk_tot, dgate, p.B, p.T,

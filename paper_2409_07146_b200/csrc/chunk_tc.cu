@@ -210,7 +210,7 @@ __device__ __forceinline__ void store_masked_row(uint32_t tmem, int wq, int row,
 // with explicit exponent differences from the fp32 weight and G tiles; P and the inter-chunk
 // product are read from the accumulators; the row goes straight to global memory.
 template <bool REV>
-__device__ __noinline__ void value_side_explicit_rows(const unsigned char* gt, const unsigned char* sW,
+__device__ __forceinline__ void value_side_explicit_rows(const unsigned char* gt, const unsigned char* sW,
                                                       const float* gc, uint32_t tmem, int wq, int row, int sb,
                                                       int grow, int valid, float* out_row) {
     const int jlo = REV ? row : 0, jhi = REV ? kCT - 1 : row;
@@ -260,11 +260,15 @@ __device__ __noinline__ void value_side_explicit_rows(const unsigned char* gt, c
 // ======================================================================================
 // value_side: out_i[s] = sum_{j<=i} <xq_i, xk_j> w_j[s] decay_ij[s]  + decayed (xq_i S)[s]
 // ======================================================================================
-template <bool REV>
+template <bool REV, bool GENERAL>
 __global__ void __launch_bounds__(kThreads, 1)
 value_side_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK,
                      const __grid_constant__ CUtensorMap mapW, const __grid_constant__ CUtensorMap mapG,
-                     const __grid_constant__ CUtensorMap mapO, ValueSideArgs a, int32_t* dev_status) {
+                     const __grid_constant__ CUtensorMap mapO, ValueSideArgs a, const int* __restrict__ strong_flag,
+                     int32_t* dev_status) {
+    // Two variants of this kernel are launched back to back: this CTA's (batch, head) belongs to
+    // the general one (with the strong-decay path) or to the lean one (moderate chunks only).
+    if ((strong_flag[blockIdx.x] != 0) != GENERAL) return;
     extern __shared__ unsigned char smem_raw[];
     // align by pointer arithmetic (not an integer round trip) so accesses stay in the shared window
     unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
@@ -363,7 +367,7 @@ value_side_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_cons
                 WAIT_OR_ABORT(&ctl->bar_ops, it & 1);
                 tc_fence_after_sync();
                 PROF_MARK();
-                const bool moderate = ctl->moderate[it & 1] != 0;
+                const bool moderate = !GENERAL || ctl->moderate[it & 1] != 0;
 #pragma unroll
                 for (int kk = 0; kk < kCT / 16; ++kk)
                     mma_bf16(tmem + kColU, desc_advance(dKm, mnmaj(kk)), desc_advance(dWa, mnmaj(kk)), idescU, kk > 0);
@@ -427,7 +431,7 @@ value_side_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_cons
             WAIT_OR_ABORT(&ctl->bar_g[it & 1], (it >> 1) & 1);
             WAIT_OR_ABORT(&ctl->bar_w, it & 1);
             PROF_MARK();
-            const bool moderate = publish_chunk_decay(ctl, tid, gt, valid - 1);
+            const bool moderate = publish_chunk_decay(ctl, tid, gt, valid - 1) || !GENERAL;
             if (ctl->abort) break;
             PROF_MARK();
 
@@ -469,9 +473,9 @@ value_side_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_cons
                 tc_fence_before_sync();
                 compute_sync();
                 if (tid == 0) mbar_arrive(&ctl->bar_pm);
-            } else {
+            } else if constexpr (GENERAL) {
                 // Strong decay: the intra-chunk term with explicit exponent differences on the CUDA
-                // cores (kept out of line so that its registers do not weigh on the common path).
+                // cores (only the general variant of the kernel carries this path).
                 WAIT_OR_ABORT(&ctl->bar_mma1, it & 1);    // the inter-chunk product
                 tc_fence_after_sync();
                 value_side_explicit_rows<REV>(gt, sW, ctl->gc, tmem, wq, row, sb, grow, valid,
@@ -567,7 +571,7 @@ value_side_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_cons
 // written as the bf16 operand rows of the masked matrix (which shares its buffer with the
 // uq tile: every thread first takes its uq row into registers).
 template <bool REV>
-__device__ __noinline__ void key_side_explicit_rows(const unsigned char* sG, const unsigned char* sUq,
+__device__ __forceinline__ void key_side_explicit_rows(const unsigned char* sG, const unsigned char* sUq,
                                                     const unsigned char* sUk, unsigned char* sAm,
                                                     unsigned char* sAl, int row, int half, int grow, int valid) {
     float gi[kM], qi[kM];
@@ -605,11 +609,14 @@ __device__ __noinline__ void key_side_explicit_rows(const unsigned char* sG, con
 // ======================================================================================
 // key_side: out_i = (uq_i * qscale_i) S + sum_j A_ij xv_j,  A_ij = sum_s uq_i[s] uk_j[s] decay_ij[s]
 // ======================================================================================
-template <bool REV>
+template <bool REV, bool GENERAL>
 __global__ void __launch_bounds__(kThreads, 1)
 key_side_tc_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_constant__ CUtensorMap mapUq,
                    const __grid_constant__ CUtensorMap mapUk, const __grid_constant__ CUtensorMap mapG,
-                   const __grid_constant__ CUtensorMap mapO, KeySideArgs a, int32_t* dev_status) {
+                   const __grid_constant__ CUtensorMap mapO, KeySideArgs a, const int* __restrict__ strong_flag,
+                   int32_t* dev_status) {
+    // (see value_side_tc_kernel: general or lean variant, by (batch, head))
+    if ((strong_flag[blockIdx.x] != 0) != GENERAL) return;
     extern __shared__ unsigned char smem_raw[];
     // align by pointer arithmetic (not an integer round trip) so accesses stay in the shared window
     unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
@@ -679,7 +686,7 @@ key_side_tc_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_consta
                 WAIT_OR_ABORT(&ctl->bar_ops, it & 1);
                 WAIT_OR_ABORT(&ctl->bar_x, it & 1);
                 tc_fence_after_sync();
-                const bool moderate = ctl->moderate[it & 1] != 0;
+                const bool moderate = !GENERAL || ctl->moderate[it & 1] != 0;
                 if (moderate) {
 #pragma unroll
                     for (int kk = 0; kk < kM / 16; ++kk)
@@ -739,7 +746,7 @@ key_side_tc_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_consta
             PROF_MARK();
             WAIT_OR_ABORT(&ctl->bar_g[0], it & 1);
             PROF_MARK();
-            const bool moderate = publish_chunk_decay(ctl, tid, sG, valid - 1);
+            const bool moderate = publish_chunk_decay(ctl, tid, sG, valid - 1) || !GENERAL;
             if (ctl->abort) break;
             PROF_MARK();
 
@@ -800,9 +807,9 @@ key_side_tc_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_consta
                 tc_fence_after_sync();
                 PROF_MARK();
                 store_masked_row<REV, true>(tmem, wq, row, half, sAm, sAl);    // overwrites the uq tile: all rows were read
-            } else {
-                // Strong decay: A_ij with explicit exponent differences (kept out of line so that
-                // its registers do not weigh on the common path).
+            } else if constexpr (GENERAL) {
+                // Strong decay: A_ij with explicit exponent differences (only the general variant of
+                // the kernel carries this path).
                 key_side_explicit_rows<REV>(sG, sUq, sUk, sAm, sAl, row, half, grow, valid);
             }
             fence_async_smem();
@@ -894,8 +901,9 @@ bool tc_supported(int d_k, int d_v, int M) {
 int tc_value_side_slices(int D) { return D / kDST; }
 int tc_chunk() { return kCT; }
 
-cudaError_t launch_value_side_tc(const ValueSideArgs& a, int M, int reverse, cudaStream_t st, int32_t* dev_status) {
-    if (M != kM || a.D % kDST != 0) return cudaErrorNotSupported;
+cudaError_t launch_value_side_tc(const ValueSideArgs& a, int M, int reverse, const int* strong_flag,
+                                 cudaStream_t st, int32_t* dev_status) {
+    if (M != kM || a.D % kDST != 0 || strong_flag == nullptr) return cudaErrorNotSupported;
     CUtensorMap mq, mk, mw, mg, mo;
     cudaError_t e = make_tensor_map_bthd(&mq, a.xq, a.B, a.T, a.H, a.D, kCT, 2);
     if (e == cudaSuccess) e = make_tensor_map_sliced(&mo, a.out, a.D / kDST, a.B, a.T, a.H, kM, kCT, 4);
@@ -904,20 +912,21 @@ cudaError_t launch_value_side_tc(const ValueSideArgs& a, int M, int reverse, cud
     if (e == cudaSuccess) e = make_tensor_map_bthd(&mg, a.G, a.B, a.T, a.H, kM, kCT, 4);
     if (e != cudaSuccess) return e;
     dim3 grid(a.B * a.H, a.D / kDST);
-    if (reverse) {
-        e = prepare(value_side_tc_kernel<true>, kSmemValueSide);
-        if (e != cudaSuccess) return e;
-        value_side_tc_kernel<true><<<grid, kThreads, kSmemValueSide, st>>>(mq, mk, mw, mg, mo, a, dev_status);
-    } else {
-        e = prepare(value_side_tc_kernel<false>, kSmemValueSide);
-        if (e != cudaSuccess) return e;
-        value_side_tc_kernel<false><<<grid, kThreads, kSmemValueSide, st>>>(mq, mk, mw, mg, mo, a, dev_status);
-    }
+#define GSA_LAUNCH_VS(REVV, GEN)                                                                         \
+    e = prepare(value_side_tc_kernel<REVV, GEN>, kSmemValueSide);                                        \
+    if (e != cudaSuccess) return e;                                                                      \
+    value_side_tc_kernel<REVV, GEN><<<grid, kThreads, kSmemValueSide, st>>>(mq, mk, mw, mg, mo, a, strong_flag, dev_status)
+    // lean variant for the (batch, head) pairs whose chunks all decay moderately, general
+    // variant for the others; each CTA of the variant that is not its own returns at once
+    if (reverse) { GSA_LAUNCH_VS(true, false); GSA_LAUNCH_VS(true, true); }
+    else { GSA_LAUNCH_VS(false, false); GSA_LAUNCH_VS(false, true); }
+#undef GSA_LAUNCH_VS
     return cudaGetLastError();
 }
 
-cudaError_t launch_key_side_tc(const KeySideArgs& a, int M, int reverse, cudaStream_t st, int32_t* dev_status) {
-    if (M != kM || a.D % kDST != 0) return cudaErrorNotSupported;
+cudaError_t launch_key_side_tc(const KeySideArgs& a, int M, int reverse, const int* strong_flag,
+                               cudaStream_t st, int32_t* dev_status) {
+    if (M != kM || a.D % kDST != 0 || strong_flag == nullptr) return cudaErrorNotSupported;
     CUtensorMap mv, muq, muk, mg, mo;
     cudaError_t e = make_tensor_map_bthd(&mv, a.xv, a.B, a.T, a.H, a.D, kCT, 2);
     if (e == cudaSuccess) e = make_tensor_map_bthd(&mo, a.out, a.B, a.T, a.H, a.D, kCT, 2);
@@ -926,15 +935,13 @@ cudaError_t launch_key_side_tc(const KeySideArgs& a, int M, int reverse, cudaStr
     if (e == cudaSuccess) e = make_tensor_map_bthd(&mg, a.G, a.B, a.T, a.H, kM, kCT, 4);
     if (e != cudaSuccess) return e;
     dim3 grid(a.B * a.H, a.D / kDST);
-    if (reverse) {
-        e = prepare(key_side_tc_kernel<true>, kSmemKeySide);
-        if (e != cudaSuccess) return e;
-        key_side_tc_kernel<true><<<grid, kThreads, kSmemKeySide, st>>>(mv, muq, muk, mg, mo, a, dev_status);
-    } else {
-        e = prepare(key_side_tc_kernel<false>, kSmemKeySide);
-        if (e != cudaSuccess) return e;
-        key_side_tc_kernel<false><<<grid, kThreads, kSmemKeySide, st>>>(mv, muq, muk, mg, mo, a, dev_status);
-    }
+#define GSA_LAUNCH_KS(REVV, GEN)                                                                         \
+    e = prepare(key_side_tc_kernel<REVV, GEN>, kSmemKeySide);                                            \
+    if (e != cudaSuccess) return e;                                                                      \
+    key_side_tc_kernel<REVV, GEN><<<grid, kThreads, kSmemKeySide, st>>>(mv, muq, muk, mg, mo, a, strong_flag, dev_status)
+    if (reverse) { GSA_LAUNCH_KS(true, false); GSA_LAUNCH_KS(true, true); }
+    else { GSA_LAUNCH_KS(false, false); GSA_LAUNCH_KS(false, true); }
+#undef GSA_LAUNCH_KS
     return cudaGetLastError();
 }
 

@@ -91,8 +91,11 @@ struct KeySideArgs {
 };
 
 // launchers (definitions in the .cu files); all return cudaGetLastError() of the launch
+// strong_flag (nullable, [B*H] ints, zeroed by the caller): set to 1 for every (b,h) that has a
+// chunk whose total log-decay is below kFactorisedDecayMin.
 cudaError_t launch_gate_cumsum(const float* gate, int gate_is_log, float* G, float* I,
-                               int B, int T, int H, int M, int chunk, cudaStream_t st);
+                               int B, int T, int H, int M, int chunk, int* strong_flag,
+                               cudaStream_t st);
 cudaError_t launch_slot_softmax_fwd(const float* part, int nslice, float scale, float* ok,
                                     float* p, size_t rows, int M, cudaStream_t st);
 cudaError_t launch_slot_softmax_bwd(const float* ok, const float* dp_part, int nslice,
@@ -113,10 +116,10 @@ cudaError_t launch_key_side_simt(const KeySideArgs& a, int io, int M, int revers
 bool tc_supported(int d_k, int d_v, int M);
 int tc_value_side_slices(int D);
 int tc_chunk();                    // chunk length of the tensor-core kernels   // how many partial-sum slices value_side writes for width D
-cudaError_t launch_value_side_tc(const ValueSideArgs& a, int M, int reverse, cudaStream_t st,
-                                 int32_t* dev_status);
-cudaError_t launch_key_side_tc(const KeySideArgs& a, int M, int reverse, cudaStream_t st,
-                               int32_t* dev_status);
+cudaError_t launch_value_side_tc(const ValueSideArgs& a, int M, int reverse, const int* strong_flag,
+                                 cudaStream_t st, int32_t* dev_status);
+cudaError_t launch_key_side_tc(const KeySideArgs& a, int M, int reverse, const int* strong_flag,
+                               cudaStream_t st, int32_t* dev_status);
 cudaError_t launch_decode(const gsa_params_t& p, const void* q, const void* k, const void* v,
                           const float* gate, float* Ks, float* Vs, void* o, cudaStream_t st);
 

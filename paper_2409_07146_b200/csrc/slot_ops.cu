@@ -18,7 +18,7 @@ __global__ void __launch_bounds__(M * 8) gate_cumsum_kernel(const float* __restr
                                                             int gate_is_log,
                                                             float* __restrict__ G,
                                                             float* __restrict__ I, int T, int H,
-                                                            int chunk) {
+                                                            int chunk, int* __restrict__ strong_flag) {
     __shared__ double group_sum[8][M];
     const int s = threadIdx.x, grp = threadIdx.y;          // blockDim.y = chunk / 16 <= 8
     const int n = blockIdx.y;
@@ -55,21 +55,24 @@ __global__ void __launch_bounds__(M * 8) gate_cumsum_kernel(const float* __restr
     __syncthreads();
     double before = 0.0;
     for (int q = 0; q < grp; ++q) before += group_sum[q][s];
+    // the chunk's total log-decay decides which variant of the chunk kernels takes this (b,h)
+    if (strong_flag != nullptr && grp == (int)blockDim.y - 1 && before + acc < (double)kFactorisedDecayMin)
+        strong_flag[bh] = 1;
 #pragma unroll
     for (int i = 0; i < kCumRows; ++i)
         if (i < rows) G[base + (size_t)i * stride] = (float)(before + run[i]);
 }
 
 cudaError_t launch_gate_cumsum(const float* gate, int gate_is_log, float* G, float* I, int B,
-                               int T, int H, int M, int chunk, cudaStream_t st) {
+                               int T, int H, int M, int chunk, int* strong_flag, cudaStream_t st) {
     if (chunk % kCumRows != 0 || chunk / kCumRows > 8) return cudaErrorInvalidValue;
     const int nchunks = (T + chunk - 1) / chunk;
     dim3 block(M, chunk / kCumRows);
     dim3 grid(B * H, nchunks);
     if (M == 64)
-        gate_cumsum_kernel<64><<<grid, block, 0, st>>>(gate, gate_is_log, G, I, T, H, chunk);
+        gate_cumsum_kernel<64><<<grid, block, 0, st>>>(gate, gate_is_log, G, I, T, H, chunk, strong_flag);
     else
-        gate_cumsum_kernel<32><<<grid, block, 0, st>>>(gate, gate_is_log, G, I, T, H, chunk);
+        gate_cumsum_kernel<32><<<grid, block, 0, st>>>(gate, gate_is_log, G, I, T, H, chunk, strong_flag);
     return cudaGetLastError();
 }
 
