@@ -81,7 +81,7 @@ def kernel_algorithmic_bytes(label: str, w: W.Workload) -> int:
         "bwd_dIv_value_side_rev": 2 * w.d_v * e + 8 * m + 4 * m * nsv,
         "bwd_dk_key_side_rev": 12 * m + 2 * w.d_k * e,
         "bwd_dIk_value_side_rev": 2 * w.d_k * e + 8 * m + 4 * m * nsk,
-        "gate_grad": 2 * (8 * m + 4 * m * (nsk + nsv)) + 4 * m + 4 * m,
+        "gate_grad": 4 * m * (7 + nsk + nsv),   # one pass over u, I, gate, partials -> dgate; carry pass r/w
     }
     return R * table[label]
 

@@ -193,8 +193,8 @@ cudaError_t launch_slot_softmax_bwd(const float* ok, const float* dp_part, int n
 // (the reversed cumulative sum of App. B, taken over the whole sequence), then
 //   gate holds a     : dgate = d(log a)|decay / a - dI
 //   gate holds log a : dgate = d(log a)|decay - a * dI
-// Three steps: totals of 16-row blocks, an exclusive suffix scan over the block totals (fp64),
-// and the block-local reversed sums started from that carry.
+// Three steps: block-local reversed sums of 16-row blocks (the only pass over the inputs), an
+// exclusive suffix scan over the block totals (fp64), and the addition of each block's carry.
 
 constexpr int kGG = 16;   // rows per thread of the gate-gradient kernels
 
@@ -219,34 +219,6 @@ __device__ __forceinline__ void load_dI(const float* __restrict__ dIk, int nsk, 
 #pragma unroll
         for (int i = 0; i < kGG; ++i) dI[i] += t[i];
     }
-}
-
-template <int M>
-__global__ void __launch_bounds__(256) gate_grad_totals_kernel(
-    const float* __restrict__ u, const float* __restrict__ I, const float* __restrict__ dIk, int nsk,
-    const float* __restrict__ dIv, int nsv, float* __restrict__ blk_tot, int B, int T, int H,
-    int nblk) {
-    const int s = threadIdx.x;
-    const int n = blockIdx.y * blockDim.y + threadIdx.y;
-    if (n >= nblk) return;
-    const int bh = blockIdx.x, b = bh / H, h = bh % H;
-    const int t0 = n * kGG;
-    const int rows = min(kGG, T - t0);
-    const size_t stride = (size_t)H * M, total = (size_t)B * T * H * M;
-    const size_t base = (((size_t)b * T + t0) * H + h) * M + s;
-    float x[kGG], dI[kGG], uu[kGG], ii[kGG];
-#pragma unroll
-    for (int i = 0; i < kGG; ++i) {
-        uu[i] = (i < rows) ? u[base + (size_t)i * stride] : 0.f;
-        ii[i] = (i < rows) ? I[base + (size_t)i * stride] : 0.f;
-    }
-    load_dI(dIk, nsk, dIv, nsv, base, stride, total, rows, dI);
-#pragma unroll
-    for (int i = 0; i < kGG; ++i) x[i] = uu[i] - ii[i] * dI[i];
-    float tot = 0.f;
-#pragma unroll
-    for (int i = kGG - 1; i >= 0; --i) tot += x[i];
-    blk_tot[((size_t)bh * nblk + n) * M + s] = tot;
 }
 
 // blk_tot[bh][n][s] <- sum over blocks n' > n of the totals, plus the final-memory term.
@@ -283,12 +255,14 @@ __global__ void __launch_bounds__(M * 16) gate_grad_scan_kernel(
     }
 }
 
+// Block-local pass: for each 16-row block, the reversed running sums of x = u - I dI that start
+// at the block's end, turned into the gate gradient as if nothing followed the block, plus
+// the block total for the scan.  One read of every input.
 template <int M>
-__global__ void __launch_bounds__(256) gate_grad_final_kernel(
+__global__ void __launch_bounds__(256) gate_grad_local_kernel(
     const float* __restrict__ u, const float* __restrict__ I, const float* __restrict__ dIk, int nsk,
     const float* __restrict__ dIv, int nsv, const float* __restrict__ gate, int gate_is_log,
-    const float* __restrict__ blk_carry, float* __restrict__ dgate, int B, int T, int H,
-    int nblk) {
+    float* __restrict__ blk_tot, float* __restrict__ dgate, int B, int T, int H, int nblk) {
     const int s = threadIdx.x;
     const int n = blockIdx.y * blockDim.y + threadIdx.y;
     if (n >= nblk) return;
@@ -307,7 +281,7 @@ __global__ void __launch_bounds__(256) gate_grad_final_kernel(
     load_dI(dIk, nsk, dIv, nsv, base, stride, total, rows, dI);
 #pragma unroll
     for (int i = 0; i < kGG; ++i) x[i] -= ii[i] * dI[i];
-    float run = blk_carry[((size_t)bh * nblk + n) * M + s];
+    float run = 0.f;
 #pragma unroll
     for (int i = kGG - 1; i >= 0; --i) {
         run += x[i];
@@ -322,6 +296,32 @@ __global__ void __launch_bounds__(256) gate_grad_final_kernel(
             dgate[base + (size_t)i * stride] = out;
         }
     }
+    blk_tot[((size_t)bh * nblk + n) * M + s] = run;
+}
+
+// Adds what follows the block: dgate += carry (log gate) or carry / a (linear gate).
+template <int M>
+__global__ void __launch_bounds__(256) gate_grad_carry_kernel(
+    const float* __restrict__ gate, int gate_is_log, const float* __restrict__ blk_carry,
+    float* __restrict__ dgate, int T, int H, int nblk) {
+    const int s = threadIdx.x;
+    const int n = blockIdx.y * blockDim.y + threadIdx.y;
+    if (n >= nblk) return;
+    const int bh = blockIdx.x, b = bh / H, h = bh % H;
+    const int t0 = n * kGG;
+    const int rows = min(kGG, T - t0);
+    const size_t stride = (size_t)H * M;
+    const size_t base = (((size_t)b * T + t0) * H + h) * M + s;
+    const float carry = blk_carry[((size_t)bh * nblk + n) * M + s];
+    float d[kGG], gt[kGG];
+#pragma unroll
+    for (int i = 0; i < kGG; ++i) {
+        d[i] = (i < rows) ? dgate[base + (size_t)i * stride] : 0.f;
+        gt[i] = (i < rows && !gate_is_log) ? gate[base + (size_t)i * stride] : 1.f;
+    }
+#pragma unroll
+    for (int i = 0; i < kGG; ++i)
+        if (i < rows) dgate[base + (size_t)i * stride] = d[i] + ((gate_is_log || gt[i] > 0.f) ? carry / gt[i] : 0.f);
 }
 
 int gate_grad_blocks(int T) { return (T + kGG - 1) / kGG; }
@@ -336,17 +336,15 @@ cudaError_t launch_gate_grad(const float* u, const float* I, const float* dIk_pa
     dim3 block(M, 256 / M);
     dim3 grid(B * H, (nblk + block.y - 1) / block.y);
     if (M == 64) {
-        gate_grad_totals_kernel<64><<<grid, block, 0, st>>>(u, I, dIk_part, nsk, dIv_part, nsv,
-                                                            blk_tot, B, T, H, nblk);
+        gate_grad_local_kernel<64><<<grid, block, 0, st>>>(u, I, dIk_part, nsk, dIv_part, nsv, gate, gate_is_log,
+                                                           blk_tot, dgate, B, T, H, nblk);
         gate_grad_scan_kernel<64><<<B * H, dim3(64, 16), 0, st>>>(blk_tot, dKT, KT, dVT, VT, d_k, d_v, nblk);
-        gate_grad_final_kernel<64><<<grid, block, 0, st>>>(u, I, dIk_part, nsk, dIv_part, nsv, gate,
-                                                           gate_is_log, blk_tot, dgate, B, T, H, nblk);
+        gate_grad_carry_kernel<64><<<grid, block, 0, st>>>(gate, gate_is_log, blk_tot, dgate, T, H, nblk);
     } else {
-        gate_grad_totals_kernel<32><<<grid, block, 0, st>>>(u, I, dIk_part, nsk, dIv_part, nsv,
-                                                            blk_tot, B, T, H, nblk);
+        gate_grad_local_kernel<32><<<grid, block, 0, st>>>(u, I, dIk_part, nsk, dIv_part, nsv, gate, gate_is_log,
+                                                           blk_tot, dgate, B, T, H, nblk);
         gate_grad_scan_kernel<32><<<B * H, dim3(32, 16), 0, st>>>(blk_tot, dKT, KT, dVT, VT, d_k, d_v, nblk);
-        gate_grad_final_kernel<32><<<grid, block, 0, st>>>(u, I, dIk_part, nsk, dIv_part, nsv, gate,
-                                                           gate_is_log, blk_tot, dgate, B, T, H, nblk);
+        gate_grad_carry_kernel<32><<<grid, block, 0, st>>>(gate, gate_is_log, blk_tot, dgate, T, H, nblk);
     }
     return cudaGetLastError();
 }
