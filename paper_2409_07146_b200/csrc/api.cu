@@ -47,6 +47,19 @@ Slices slices(const gsa_params_t& p) {
     return {p.d_k / 64, p.d_v / 64};
 }
 
+// Segment-parallel scheduling of the forward: when (batch, head, slice) triples cannot fill the
+// GPU, long sequences are cut into nseg segments that run as independent sequences (the
+// memories are linear in (k, v), so every segment's start memories follow from a first pass
+// that runs the segments from empty memories).  1 = off.
+int segments_of(const gsa_params_t& p) {
+    if (!use_tc(p)) return 1;
+    const int chunk = tc_chunk();
+    const long long ctas = (long long)p.B * p.H * (p.d_k < p.d_v ? p.d_k : p.d_v) / 128;
+    int nseg = 1;
+    while (ctas * nseg * 2 <= 160 && p.T % (nseg * 2 * chunk) == 0 && p.T / (nseg * 2) >= 8 * chunk) nseg *= 2;
+    return nseg;
+}
+
 struct Carver {
     char* base; size_t off;
     float* take(size_t nfloat) {
@@ -58,7 +71,8 @@ struct Carver {
 
 struct Workspace {
     float *G, *I, *okpart, *ok, *p, *dz, *u, *dppart, *dIk, *dIv, *chunk_tot, *KT, *VT;
-    int* strong;     // [B*H] flags: this (b,h) has a chunk that decays too hard for the factorised form
+    int* strong;     // [B*nseg*H] flags: this (b,h) has a chunk that decays too hard for the factorised form
+    float *seg_decay, *Kloc, *Vloc, *Kstart, *Vstart;   // segment-parallel forward only
     size_t bytes;
 };
 
@@ -68,7 +82,16 @@ Workspace carve(const gsa_params_t& p, int which, void* ws) {
     const size_t mt = (size_t)p.B * p.T * p.H * p.m;
     const Slices s = slices(p);
     Carver c{static_cast<char*>(ws), 0};
-    w.strong = reinterpret_cast<int*>(c.take((size_t)p.B * p.H));
+    const int nseg = which == GSA_WS_FWD ? segments_of(p) : 1;
+    w.strong = reinterpret_cast<int*>(c.take((size_t)p.B * p.H * nseg));
+    if (nseg > 1) {
+        const size_t pairs = (size_t)p.B * nseg * p.H;
+        w.seg_decay = c.take(pairs * p.m);
+        w.Kloc = c.take(pairs * p.m * p.d_k);
+        w.Vloc = c.take(pairs * p.m * p.d_v);
+        w.Kstart = c.take(pairs * p.m * p.d_k);
+        w.Vstart = c.take(pairs * p.m * p.d_v);
+    }
     w.G = c.take(mt);
     w.I = c.take(mt);
     w.okpart = c.take(mt * s.k);
@@ -170,7 +193,7 @@ gsa_status_t gsa_gate_cumsum(const gsa_params_t* params, const float* gate, floa
     const gsa_params_t& p = *params;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     GSA_LAUNCH("gate_cumsum", launch_gate_cumsum(gate, p.gate_kind == GSA_GATE_LOG_A, G, I, p.B, p.T,
-                                                 p.H, p.m, chunk_of(p), nullptr, st));
+                                                 p.H, p.m, chunk_of(p), nullptr, 1, st));
     return GSA_OK;
 }
 
@@ -191,16 +214,38 @@ gsa_status_t gsa_fwd(const gsa_params_t* params, const void* q, const void* k, c
     const Slices s = slices(p);
     const size_t rows = (size_t)p.B * p.T * p.H;
 
-    GSA_CUDA(cudaMemsetAsync(w.strong, 0, sizeof(int) * (size_t)p.B * p.H, st));
+    const int nseg = segments_of(p);
+    GSA_CUDA(cudaMemsetAsync(w.strong, 0, sizeof(int) * (size_t)p.B * p.H * nseg, st));
     GSA_LAUNCH("gate_cumsum", launch_gate_cumsum(gate, p.gate_kind == GSA_GATE_LOG_A, w.G, w.I, p.B, p.T,
-                                                 p.H, p.m, chunk_of(p), w.strong, st));
-    // pass 1: o' = GLA(q, k, 1-a) with the decay on the slot (value) side
-    ValueSideArgs a1{q, k, w.I, w.G, K0, KT, w.okpart, p.B, p.T, p.H, p.d_k};
-    GSA_LAUNCH("pass1_value_side", value_side(p, a1, 0, w.strong, st, dev_status));
+                                                 p.H, p.m, chunk_of(p), w.strong, nseg, st));
     float* ok = ok_save ? ok_save : w.ok;
+    // [B,T,H,.] cut into nseg segments is the same memory as [B*nseg, T/nseg, H, .]
+    const int Bs = p.B * nseg, Ts = p.T / nseg;
+    const float *Kin = K0, *Vin = V0;
+    float *Kout = KT, *Vout = VT;
+    if (nseg > 1) {
+        // first pass: every segment from empty memories, only for its end memories (the outputs
+        // land in buffers that the second pass overwrites); then the start memories of all
+        // segments, and the final memories, by a scan over the segments
+        GSA_LAUNCH("segment_logdecay", launch_segment_logdecay(w.G, w.seg_decay, p.B, p.T, p.H, p.m, nseg,
+                                                               chunk_of(p), st));
+        ValueSideArgs s1{q, k, w.I, w.G, nullptr, w.Kloc, w.okpart, Bs, Ts, p.H, p.d_k};
+        GSA_LAUNCH("segment_pass1_states", value_side(p, s1, 0, w.strong, st, dev_status));
+        KeySideArgs s2{w.I, w.I, w.G, v, nullptr, w.Vloc, o, Bs, Ts, p.H, p.d_v};
+        GSA_LAUNCH("segment_pass2_states", key_side(p, s2, 0, w.strong, st, dev_status));
+        GSA_LAUNCH("segment_combine", launch_segment_combine(w.seg_decay, w.Kloc, K0, w.Kstart, KT, p.B, p.H, p.m,
+                                                             p.d_k, nseg, st));
+        GSA_LAUNCH("segment_combine", launch_segment_combine(w.seg_decay, w.Vloc, V0, w.Vstart, VT, p.B, p.H, p.m,
+                                                             p.d_v, nseg, st));
+        Kin = w.Kstart; Vin = w.Vstart;
+        Kout = nullptr; Vout = nullptr;
+    }
+    // pass 1: o' = GLA(q, k, 1-a) with the decay on the slot (value) side
+    ValueSideArgs a1{q, k, w.I, w.G, Kin, Kout, w.okpart, Bs, Ts, p.H, p.d_k};
+    GSA_LAUNCH("pass1_value_side", value_side(p, a1, 0, w.strong, st, dev_status));
     GSA_LAUNCH("slot_softmax", launch_slot_softmax_fwd(w.okpart, s.k, p.scale, ok, w.p, rows, p.m, st));
     // pass 2: o = GLA(softmax(o'), 1-a, v) with the decay on the slot (key) side
-    KeySideArgs a2{w.p, w.I, w.G, v, V0, VT, o, p.B, p.T, p.H, p.d_v};
+    KeySideArgs a2{w.p, w.I, w.G, v, Vin, Vout, o, Bs, Ts, p.H, p.d_v};
     GSA_LAUNCH("pass2_key_side", key_side(p, a2, 0, w.strong, st, dev_status));
     return GSA_OK;
 }
@@ -228,7 +273,7 @@ gsa_status_t gsa_bwd(const gsa_params_t* params, const void* q, const void* k, c
 
     GSA_CUDA(cudaMemsetAsync(w.strong, 0, sizeof(int) * (size_t)p.B * p.H, st));
     GSA_LAUNCH("gate_cumsum", launch_gate_cumsum(gate, p.gate_kind == GSA_GATE_LOG_A, w.G, w.I, p.B, p.T,
-                                                 p.H, p.m, chunk_of(p), w.strong, st));
+                                                 p.H, p.m, chunk_of(p), w.strong, 1, st));
     const float* ok = ok_saved;
     if (ok == nullptr) {  // recompute pass 1 and its logits
         ValueSideArgs a1{q, k, w.I, w.G, K0, nullptr, w.okpart, p.B, p.T, p.H, p.d_k};

@@ -92,10 +92,18 @@ struct KeySideArgs {
 
 // launchers (definitions in the .cu files); all return cudaGetLastError() of the launch
 // strong_flag (nullable, [B*H] ints, zeroed by the caller): set to 1 for every (b,h) that has a
-// chunk whose total log-decay is below kFactorisedDecayMin.
+// chunk whose total log-decay is below kFactorisedDecayMin (nseg > 1: [B*nseg*H], per segment).
 cudaError_t launch_gate_cumsum(const float* gate, int gate_is_log, float* G, float* I,
-                               int B, int T, int H, int M, int chunk, int* strong_flag,
+                               int B, int T, int H, int M, int chunk, int* strong_flag, int nseg,
                                cudaStream_t st);
+// Segment-parallel scheduling (T cut into nseg segments run as independent sequences): per-segment
+// log-decay [B,nseg,H,M] from G, and the start memories [B,nseg,H,M,D] of every segment from the
+// end memories of the segments run from empty memories.
+cudaError_t launch_segment_logdecay(const float* G, float* seg_logdecay, int B, int T, int H, int M, int nseg,
+                                    int chunk, cudaStream_t st);
+cudaError_t launch_segment_combine(const float* seg_logdecay, const float* local_end, const float* S0,
+                                   float* start, float* final_state, int B, int H, int M, int D, int nseg,
+                                   cudaStream_t st);
 cudaError_t launch_slot_softmax_fwd(const float* part, int nslice, float scale, float* ok,
                                     float* p, size_t rows, int M, cudaStream_t st);
 cudaError_t launch_slot_softmax_bwd(const float* ok, const float* dp_part, int nslice,

@@ -18,7 +18,7 @@ __global__ void __launch_bounds__(M * 8) gate_cumsum_kernel(const float* __restr
                                                             int gate_is_log,
                                                             float* __restrict__ G,
                                                             float* __restrict__ I, int T, int H,
-                                                            int chunk, int* __restrict__ strong_flag) {
+                                                            int chunk, int* __restrict__ strong_flag, int nseg) {
     __shared__ double group_sum[8][M];
     const int s = threadIdx.x, grp = threadIdx.y;          // blockDim.y = chunk / 16 <= 8
     const int n = blockIdx.y;
@@ -56,23 +56,26 @@ __global__ void __launch_bounds__(M * 8) gate_cumsum_kernel(const float* __restr
     double before = 0.0;
     for (int q = 0; q < grp; ++q) before += group_sum[q][s];
     // the chunk's total log-decay decides which variant of the chunk kernels takes this (b,h)
-    if (strong_flag != nullptr && grp == (int)blockDim.y - 1 && before + acc < (double)kFactorisedDecayMin)
-        strong_flag[bh] = 1;
+    // (with segment-parallel scheduling the flags are per (batch, segment, head))
+    if (strong_flag != nullptr && grp == (int)blockDim.y - 1 && before + acc < (double)kFactorisedDecayMin) {
+        const int seg = (int)(((long long)n * chunk) / (T / nseg));
+        strong_flag[(b * nseg + seg) * H + h] = 1;
+    }
 #pragma unroll
     for (int i = 0; i < kCumRows; ++i)
         if (i < rows) G[base + (size_t)i * stride] = (float)(before + run[i]);
 }
 
 cudaError_t launch_gate_cumsum(const float* gate, int gate_is_log, float* G, float* I, int B,
-                               int T, int H, int M, int chunk, int* strong_flag, cudaStream_t st) {
+                               int T, int H, int M, int chunk, int* strong_flag, int nseg, cudaStream_t st) {
     if (chunk % kCumRows != 0 || chunk / kCumRows > 8) return cudaErrorInvalidValue;
     const int nchunks = (T + chunk - 1) / chunk;
     dim3 block(M, chunk / kCumRows);
     dim3 grid(B * H, nchunks);
     if (M == 64)
-        gate_cumsum_kernel<64><<<grid, block, 0, st>>>(gate, gate_is_log, G, I, T, H, chunk, strong_flag);
+        gate_cumsum_kernel<64><<<grid, block, 0, st>>>(gate, gate_is_log, G, I, T, H, chunk, strong_flag, nseg < 1 ? 1 : nseg);
     else
-        gate_cumsum_kernel<32><<<grid, block, 0, st>>>(gate, gate_is_log, G, I, T, H, chunk, strong_flag);
+        gate_cumsum_kernel<32><<<grid, block, 0, st>>>(gate, gate_is_log, G, I, T, H, chunk, strong_flag, nseg < 1 ? 1 : nseg);
     return cudaGetLastError();
 }
 
@@ -346,6 +349,63 @@ cudaError_t launch_gate_grad(const float* u, const float* I, const float* dIk_pa
         gate_grad_scan_kernel<32><<<B * H, dim3(32, 16), 0, st>>>(blk_tot, dKT, KT, dVT, VT, d_k, d_v, nblk);
         gate_grad_carry_kernel<32><<<grid, block, 0, st>>>(gate, gate_is_log, blk_tot, dgate, T, H, nblk);
     }
+    return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------ segment-parallel scheduling
+// The memories are linear in (k, v): K~ after a segment = D * K~ before + (K~ of the segment run
+// from empty memories), D = product of the gates over the segment.  A sequence cut into nseg
+// segments can therefore run as nseg independent sequences once every segment's start
+// memories are known.
+//
+// seg_logdecay[b][r][h][s] = sum over the chunks of segment r of G at the chunk's last row.
+template <int M>
+__global__ void segment_logdecay_kernel(const float* __restrict__ G, float* __restrict__ seg_logdecay, int T, int H,
+                                        int nseg, int chunk) {
+    const int s = threadIdx.x, h = blockIdx.y;
+    const int b = blockIdx.x / nseg, r = blockIdx.x % nseg;
+    const int Tseg = T / nseg;
+    double acc = 0.0;
+    for (int t = r * Tseg + chunk - 1; t < (r + 1) * Tseg; t += chunk)
+        acc += (double)G[(((size_t)b * T + t) * H + h) * M + s];
+    seg_logdecay[(((size_t)b * nseg + r) * H + h) * M + s] = (float)acc;
+}
+
+// start[b][r] = D[r-1] start[b][r-1] + local_end[b][r-1], start[b][0] = S0[b] (or 0); the memory
+// after the last segment goes to final (nullable).  Memories [.., H, M, D]; one thread per (s, c).
+template <int M>
+__global__ void segment_combine_kernel(const float* __restrict__ seg_logdecay, const float* __restrict__ local_end,
+                                       const float* __restrict__ S0, float* __restrict__ start,
+                                       float* __restrict__ final_state, int H, int D, int nseg) {
+    const int b = blockIdx.x / H, h = blockIdx.x % H;
+    const int idx = blockIdx.y * blockDim.x + threadIdx.x;
+    if (idx < M * D) {
+        const int s = idx / D;
+        float cur = S0 ? S0[((size_t)(b * H + h)) * M * D + idx] : 0.f;
+        for (int r = 0; r < nseg; ++r) {
+            const size_t pair = ((size_t)b * nseg + r) * H + h;
+            start[pair * M * D + idx] = cur;
+            cur = fmaf(cur, __expf(seg_logdecay[pair * M + s]), local_end[pair * M * D + idx]);
+        }
+        if (final_state) final_state[((size_t)(b * H + h)) * M * D + idx] = cur;
+    }
+}
+
+cudaError_t launch_segment_logdecay(const float* G, float* seg_logdecay, int B, int T, int H, int M, int nseg,
+                                    int chunk, cudaStream_t st) {
+    dim3 grid(B * nseg, H);
+    if (M == 64) segment_logdecay_kernel<64><<<grid, 64, 0, st>>>(G, seg_logdecay, T, H, nseg, chunk);
+    else segment_logdecay_kernel<32><<<grid, 32, 0, st>>>(G, seg_logdecay, T, H, nseg, chunk);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_segment_combine(const float* seg_logdecay, const float* local_end, const float* S0, float* start,
+                                   float* final_state, int B, int H, int M, int D, int nseg, cudaStream_t st) {
+    dim3 grid(B * H, (M * D + 255) / 256);
+    if (M == 64)
+        segment_combine_kernel<64><<<grid, 256, 0, st>>>(seg_logdecay, local_end, S0, start, final_state, H, D, nseg);
+    else
+        segment_combine_kernel<32><<<grid, 256, 0, st>>>(seg_logdecay, local_end, S0, start, final_state, H, D, nseg);
     return cudaGetLastError();
 }
 

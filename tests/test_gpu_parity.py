@@ -252,6 +252,21 @@ def test_fwd_tc_strong_forgetting(gate, log):
     check_fwd(d, got, gref, "bf16", log=log, tc=True)
 
 
+@pytest.mark.parametrize("gate", ["tau8", "mixed"])
+@pytest.mark.parametrize("init", [False, True])
+def test_fwd_tc_segment_parallel_schedule(gate, init):
+    # one sequence, few heads: the forward cuts T into segments that run as independent
+    # sequences (4 here), so start memories, per-segment decay and final memories all matter
+    B, T, H, dk, dv, m = 1, 4096, 2, 256, 128, 64
+    d = rand_inputs(41, B, T, H, dk, dv, m, "bf16", init=init, gate=gate)
+    if gate == "mixed":          # strong decay in the third segment only
+        d["gate"][:, :2048, :, 2] = 0.99
+        d["gate"][:, 3072:, :, 2] = 0.99
+    got, g = run_fwd(d, B, T, H, dk, dv, m, "bf16", impl="tc", scale=0.7)
+    errs = check_fwd(d, got, g, "bf16", scale=0.7, tc=True)
+    print("segment-parallel fwd", errs)
+
+
 def test_fwd_tc_matches_simt_closely():
     # same inputs through both kernel families: they differ only by bf16 operand rounding
     B, T, H, dk, dv, m = 1, 256, 2, 128, 128, 64
