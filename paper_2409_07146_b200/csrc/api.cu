@@ -73,6 +73,8 @@ struct Workspace {
     float *G, *I, *okpart, *ok, *p, *dz, *u, *dppart, *dIk, *dIv, *chunk_tot, *KT, *VT;
     int* strong;     // [B*nseg*H] flags: this (b,h) has a chunk that decays too hard for the factorised form
     float *seg_decay, *Kloc, *Vloc, *Kstart, *Vstart;   // segment-parallel forward only
+    // tensor-core path: bf16 rows [high | residual] of I exp(-G), p exp(G), dz exp(G), each [B,T,H,2m]
+    void *Id, *Pd, *Zd;
     size_t bytes;
 };
 
@@ -97,6 +99,11 @@ Workspace carve(const gsa_params_t& p, int which, void* ws) {
     w.okpart = c.take(mt * s.k);
     w.ok = c.take(mt);
     w.p = c.take(mt);
+    if (use_tc(p)) {           // 2m bf16 per row = m floats
+        w.Id = c.take(mt);
+        w.Pd = c.take(mt);
+        if (which == GSA_WS_BWD) w.Zd = c.take(mt);
+    }
     if (which == GSA_WS_BWD) {
         w.dz = c.take(mt);
         w.u = c.take(mt);
@@ -193,7 +200,7 @@ gsa_status_t gsa_gate_cumsum(const gsa_params_t* params, const float* gate, floa
     const gsa_params_t& p = *params;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     GSA_LAUNCH("gate_cumsum", launch_gate_cumsum(gate, p.gate_kind == GSA_GATE_LOG_A, G, I, p.B, p.T,
-                                                 p.H, p.m, chunk_of(p), nullptr, 1, st));
+                                                 p.H, p.m, chunk_of(p), nullptr, 1, nullptr, st));
     return GSA_OK;
 }
 
@@ -217,8 +224,10 @@ gsa_status_t gsa_fwd(const gsa_params_t* params, const void* q, const void* k, c
     const int nseg = segments_of(p);
     GSA_CUDA(cudaMemsetAsync(w.strong, 0, sizeof(int) * (size_t)p.B * p.H * nseg, st));
     GSA_LAUNCH("gate_cumsum", launch_gate_cumsum(gate, p.gate_kind == GSA_GATE_LOG_A, w.G, w.I, p.B, p.T,
-                                                 p.H, p.m, chunk_of(p), w.strong, nseg, st));
+                                                 p.H, p.m, chunk_of(p), w.strong, nseg, w.Id, st));
     float* ok = ok_save ? ok_save : w.ok;
+    // the pipelined kernels leave the row factor of the pass-1 sums to the softmax kernel
+    const PendingDecay pend = use_tc(p) ? PendingDecay{w.G, w.strong, p.T, p.H, nseg} : PendingDecay{nullptr, nullptr, 1, 1, 1};
     // [B,T,H,.] cut into nseg segments is the same memory as [B*nseg, T/nseg, H, .]
     const int Bs = p.B * nseg, Ts = p.T / nseg;
     const float *Kin = K0, *Vin = V0;
@@ -229,9 +238,9 @@ gsa_status_t gsa_fwd(const gsa_params_t* params, const void* q, const void* k, c
         // segments, and the final memories, by a scan over the segments
         GSA_LAUNCH("segment_logdecay", launch_segment_logdecay(w.G, w.seg_decay, p.B, p.T, p.H, p.m, nseg,
                                                                chunk_of(p), st));
-        ValueSideArgs s1{q, k, w.I, w.G, nullptr, w.Kloc, w.okpart, Bs, Ts, p.H, p.d_k};
+        ValueSideArgs s1{q, k, w.I, w.G, nullptr, w.Kloc, w.okpart, Bs, Ts, p.H, p.d_k, w.Id};
         GSA_LAUNCH("segment_pass1_states", value_side(p, s1, 0, w.strong, st, dev_status));
-        KeySideArgs s2{w.I, w.I, w.G, v, nullptr, w.Vloc, o, Bs, Ts, p.H, p.d_v};
+        KeySideArgs s2{w.I, w.I, w.G, v, nullptr, w.Vloc, o, Bs, Ts, p.H, p.d_v, w.Id, w.Id};
         GSA_LAUNCH("segment_pass2_states", key_side(p, s2, 0, w.strong, st, dev_status));
         GSA_LAUNCH("segment_combine", launch_segment_combine(w.seg_decay, w.Kloc, K0, w.Kstart, KT, p.B, p.H, p.m,
                                                              p.d_k, nseg, st));
@@ -241,11 +250,11 @@ gsa_status_t gsa_fwd(const gsa_params_t* params, const void* q, const void* k, c
         Kout = nullptr; Vout = nullptr;
     }
     // pass 1: o' = GLA(q, k, 1-a) with the decay on the slot (value) side
-    ValueSideArgs a1{q, k, w.I, w.G, Kin, Kout, w.okpart, Bs, Ts, p.H, p.d_k};
+    ValueSideArgs a1{q, k, w.I, w.G, Kin, Kout, w.okpart, Bs, Ts, p.H, p.d_k, w.Id};
     GSA_LAUNCH("pass1_value_side", value_side(p, a1, 0, w.strong, st, dev_status));
-    GSA_LAUNCH("slot_softmax", launch_slot_softmax_fwd(w.okpart, s.k, p.scale, ok, w.p, rows, p.m, st));
+    GSA_LAUNCH("slot_softmax", launch_slot_softmax_fwd(w.okpart, s.k, p.scale, ok, w.p, rows, p.m, pend.G, w.Pd, pend, st));
     // pass 2: o = GLA(softmax(o'), 1-a, v) with the decay on the slot (key) side
-    KeySideArgs a2{w.p, w.I, w.G, v, Vin, Vout, o, Bs, Ts, p.H, p.d_v};
+    KeySideArgs a2{w.p, w.I, w.G, v, Vin, Vout, o, Bs, Ts, p.H, p.d_v, w.Pd, w.Id};
     GSA_LAUNCH("pass2_key_side", key_side(p, a2, 0, w.strong, st, dev_status));
     return GSA_OK;
 }
@@ -273,34 +282,36 @@ gsa_status_t gsa_bwd(const gsa_params_t* params, const void* q, const void* k, c
 
     GSA_CUDA(cudaMemsetAsync(w.strong, 0, sizeof(int) * (size_t)p.B * p.H, st));
     GSA_LAUNCH("gate_cumsum", launch_gate_cumsum(gate, p.gate_kind == GSA_GATE_LOG_A, w.G, w.I, p.B, p.T,
-                                                 p.H, p.m, chunk_of(p), w.strong, 1, st));
+                                                 p.H, p.m, chunk_of(p), w.strong, 1, w.Id, st));
     const float* ok = ok_saved;
+    const PendingDecay pend = use_tc(p) ? PendingDecay{w.G, w.strong, p.T, p.H, 1} : PendingDecay{nullptr, nullptr, 1, 1, 1};
     if (ok == nullptr) {  // recompute pass 1 and its logits
-        ValueSideArgs a1{q, k, w.I, w.G, K0, nullptr, w.okpart, p.B, p.T, p.H, p.d_k};
+        ValueSideArgs a1{q, k, w.I, w.G, K0, nullptr, w.okpart, p.B, p.T, p.H, p.d_k, w.Id};
         GSA_LAUNCH("pass1_value_side", value_side(p, a1, 0, w.strong, st, dev_status));
-        GSA_LAUNCH("slot_softmax", launch_slot_softmax_fwd(w.okpart, s.k, p.scale, w.ok, w.p, rows, p.m, st));
+        GSA_LAUNCH("slot_softmax", launch_slot_softmax_fwd(w.okpart, s.k, p.scale, w.ok, w.p, rows, p.m, pend.G, nullptr, pend, st));
         ok = w.ok;
     }
     // gradient w.r.t. the pass-2 queries p: the pass-1 form on (dO, v, 1-a); carries V~
-    ValueSideArgs adp{dO, v, w.I, w.G, V0, dVT ? w.VT : nullptr, w.dppart, p.B, p.T, p.H, p.d_v};
+    ValueSideArgs adp{dO, v, w.I, w.G, V0, dVT ? w.VT : nullptr, w.dppart, p.B, p.T, p.H, p.d_v, w.Id};
     GSA_LAUNCH("bwd_dp_value_side", value_side(p, adp, 0, w.strong, st, dev_status));
-    GSA_LAUNCH("slot_softmax_bwd", launch_slot_softmax_bwd(ok, w.dppart, s.v, p.scale, w.p, w.dz, w.u, rows, p.m, st));
+    GSA_LAUNCH("slot_softmax_bwd", launch_slot_softmax_bwd(ok, w.dppart, s.v, p.scale, w.p, w.dz, w.u, rows, p.m, pend.G, w.Pd,
+                                                           w.Zd, pend, st));
     // dq: the pass-2 form on (dz, 1-a, k); carries K~
-    KeySideArgs adq{w.dz, w.I, w.G, k, K0, dKT ? w.KT : nullptr, dq, p.B, p.T, p.H, p.d_k};
+    KeySideArgs adq{w.dz, w.I, w.G, k, K0, dKT ? w.KT : nullptr, dq, p.B, p.T, p.H, p.d_k, w.Zd, w.Id};
     GSA_LAUNCH("bwd_dq_key_side", key_side(p, adq, 0, w.strong, st, dev_status));
     // time-reversed runs: dv and dI^v share the state dV~; dk and dI^k share dK~
-    KeySideArgs adv{w.I, w.p, w.G, dO, dVT, dV0, dv, p.B, p.T, p.H, p.d_v};
+    KeySideArgs adv{w.I, w.p, w.G, dO, dVT, dV0, dv, p.B, p.T, p.H, p.d_v, w.Id, w.Pd};
     GSA_LAUNCH("bwd_dv_key_side_rev", key_side(p, adv, 1, w.strong, st, dev_status));
-    ValueSideArgs adIv{v, dO, w.p, w.G, dVT, nullptr, w.dIv, p.B, p.T, p.H, p.d_v};
+    ValueSideArgs adIv{v, dO, w.p, w.G, dVT, nullptr, w.dIv, p.B, p.T, p.H, p.d_v, w.Pd};
     GSA_LAUNCH("bwd_dIv_value_side_rev", value_side(p, adIv, 1, w.strong, st, dev_status));
-    KeySideArgs adk{w.I, w.dz, w.G, q, dKT, dK0, dk, p.B, p.T, p.H, p.d_k};
+    KeySideArgs adk{w.I, w.dz, w.G, q, dKT, dK0, dk, p.B, p.T, p.H, p.d_k, w.Id, w.Zd};
     GSA_LAUNCH("bwd_dk_key_side_rev", key_side(p, adk, 1, w.strong, st, dev_status));
-    ValueSideArgs adIk{k, q, w.dz, w.G, dKT, nullptr, w.dIk, p.B, p.T, p.H, p.d_k};
+    ValueSideArgs adIk{k, q, w.dz, w.G, dKT, nullptr, w.dIk, p.B, p.T, p.H, p.d_k, w.Zd};
     GSA_LAUNCH("bwd_dIk_value_side_rev", value_side(p, adIk, 1, w.strong, st, dev_status));
     // forget-gate gradient: reversed cumulative sum over the whole sequence
     GSA_LAUNCH("gate_grad", launch_gate_grad(w.u, w.I, w.dIk, s.k, w.dIv, s.v, gate, p.gate_kind == GSA_GATE_LOG_A,
                               dKT, w.KT, dVT, w.VT, p.d_k, p.d_v, w.chunk_tot, dgate, p.B, p.T,
-                              p.H, p.m, st));
+                              p.H, p.m, pend, st));
     return GSA_OK;
 }
 

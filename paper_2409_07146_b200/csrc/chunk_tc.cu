@@ -23,42 +23,12 @@
 // intra-chunk term with explicit exponent differences on the CUDA cores instead.
 // Every wait is bounded: on expiry the CTA flags dev_status, frees its tensor memory and
 // returns.
-#include <stdio.h>
-
-#include "common.cuh"
-#include "tc_common.cuh"
+#include "chunk_tc_shared.cuh"
 
 namespace gsa {
 namespace {
 using namespace tc;
-
-constexpr int kCT = 128;               // chunk length of the tensor-core kernels
-constexpr int kDST = 128;              // head-dimension slice per CTA
-constexpr int kM = 64;                 // slots
-constexpr int kPanelB = 128 * 128;     // bytes of a 128-row operand panel
-constexpr uint32_t kTmemCols = 512;
-constexpr int kComputeThreads = 256;   // 8 warps: two threads per chunk row
-constexpr int kThreads = kComputeThreads + 32;   // + the issuing warp (TMA and MMA), one lane active
-constexpr int kHS = kM / 2;            // slots per thread
-
-// accumulator columns
-constexpr int kColP = 0;       // P / A           [128 x 128]
-constexpr int kColO = 128;     // inter (+ intra for key_side) output
-constexpr int kColU = 256;     // state update    [128 x 64] (value_side: [128 x 128], high | low weight parts)
-constexpr int kColO2 = 384;    // value_side: intra-chunk output [128 x 128], high | low weight parts
-
-// Optional phase timing for development builds (-DGSA_TC_PROF): CTA 0 prints, for its fifth
-// chunk, the SM clock at each phase boundary.
-#ifdef GSA_TC_PROF
-#define PROF_DECL long long prof_t[32]; int prof_n = 0;
-#define PROF_MARK() do { if (prof_n < 32) prof_t[prof_n++] = clock64(); } while (0)
-#define PROF_DUMP(name) do { if (blockIdx.x == 0 && blockIdx.y == 0 && ((tid == 0 && it == 6) || (tid == 256 && it == 4))) { \
-    printf("%s:", name); for (int i_ = 1; i_ < prof_n; ++i_) printf(" %lld", prof_t[i_] - prof_t[i_ - 1]); printf("\n"); } prof_n = 0; } while (0)
-#else
-#define PROF_DECL
-#define PROF_MARK() do {} while (0)
-#define PROF_DUMP(name) do {} while (0)
-#endif
+using namespace tcchunk;
 
 struct Ctl {
     // filled by TMA
@@ -81,59 +51,6 @@ struct Ctl {
     alignas(16) float gc[kM];    // G of the chunk's last valid row
     alignas(16) float egc[kM];   // exp(gc)
 };
-
-// 8 consecutive fp32 values (columns s0 .. s0+7, s0 % 8 == 0) of row `row` of a slot-sized
-// fp32 tile: two panels of 32 columns, 128-byte swizzle.
-__device__ __forceinline__ void tile_row8(const unsigned char* tile, int row, int s0, float (&x)[8]) {
-    const unsigned char* panel = tile + (s0 >> 5) * kPanelB;
-    const int c = (s0 & 31) >> 2;
-    const float4 t0 = *reinterpret_cast<const float4*>(panel + swz128(row, c));
-    const float4 t1 = *reinterpret_cast<const float4*>(panel + swz128(row, c + 1));
-    x[0] = t0.x; x[1] = t0.y; x[2] = t0.z; x[3] = t0.w;
-    x[4] = t1.x; x[5] = t1.y; x[6] = t1.z; x[7] = t1.w;
-}
-// 8 consecutive floats from a 16-byte aligned plain (unswizzled) row
-__device__ __forceinline__ void tile_free_row8(const float* p, float (&x)[8]) {
-    const float4 t0 = *reinterpret_cast<const float4*>(p);
-    const float4 t1 = *reinterpret_cast<const float4*>(p + 4);
-    x[0] = t0.x; x[1] = t0.y; x[2] = t0.z; x[3] = t0.w;
-    x[4] = t1.x; x[5] = t1.y; x[6] = t1.z; x[7] = t1.w;
-}
-__device__ __forceinline__ float tile_elem(const unsigned char* tile, int row, int s) {
-    return *reinterpret_cast<const float*>(tile + (s >> 5) * kPanelB + swz128(row, (s & 31) >> 2) + (s & 3) * 4);
-}
-
-// bf16 copy of this thread's half state row (32 values from slot sb on, optionally scaled
-// per slot) into row `row` of a one-panel operand
-template <bool SCALE>
-__device__ __forceinline__ void store_state_row(unsigned char* panel, int row, int sb, const float (&S)[kHS],
-                                                const float* scale) {
-#pragma unroll
-    for (int c = 0; c < kHS / 8; ++c) {
-        float x[8];
-#pragma unroll
-        for (int e = 0; e < 8; ++e) x[e] = SCALE ? S[8 * c + e] * scale[sb + 8 * c + e] : S[8 * c + e];
-        store_chunk(panel, row, (sb >> 3) + c, x);
-    }
-}
-
-// Barrier over the 256 compute threads only (the issuing warp runs ahead on its own).
-__device__ __forceinline__ void compute_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
-__device__ __forceinline__ bool compute_sync_and(bool pred) {
-    uint32_t out;
-    asm volatile(
-        "{\n\t.reg .pred p, q;\n\t"
-        "setp.ne.b32 q, %1, 0;\n\t"
-        "bar.red.and.pred p, 1, 256, q;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(out)
-        : "r"((uint32_t)pred)
-        : "memory");
-    return out != 0;
-}
-__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
 
 // Publish the G row of the chunk's last valid token, its exponential and decide whether the
 // chunk's decay is moderate.  One compute-thread barrier inside; the result is uniform.
@@ -172,38 +89,6 @@ __device__ __forceinline__ void ctl_init(Ctl* ctl, int tid, int warp) {
     __syncthreads();
     tc_fence_after_sync();
 }
-
-// masked accumulator row -> bf16 K-major operand row (two 64-column panels); with SPLIT the
-// rounding residual goes to a second operand of the same shape (dst_lo)
-template <bool REV, bool SPLIT>
-__device__ __forceinline__ void store_masked_row(uint32_t tmem, int wq, int row, int half, unsigned char* dst,
-                                                 unsigned char* dst_lo) {
-    unsigned char* panel = dst + half * kPanelB;      // columns 64 half .. 64 half + 63
-    unsigned char* panel_lo = dst_lo + half * kPanelB;
-#pragma unroll 1
-    for (int c0 = 0; c0 < 64; c0 += 32) {
-        float v[32];
-        tmem_ld32(tmem_row_addr(tmem, wq, kColP + 64 * half + c0), v);
-#pragma unroll
-        for (int c = 0; c < 4; ++c) {
-            float x[8];
-#pragma unroll
-            for (int e = 0; e < 8; ++e) {
-                const int j = 64 * half + c0 + 8 * c + e;
-                const bool keep = REV ? (j >= row) : (j <= row);
-                x[e] = keep ? v[8 * c + e] : 0.f;
-            }
-            if (SPLIT) store_chunk_split(panel, panel_lo, row, (c0 >> 3) + c, x);
-            else store_chunk(panel, row, (c0 >> 3) + c, x);
-        }
-    }
-}
-
-// wait helper of the loops below: a wait that expires flags the CTA
-#define WAIT_OR_ABORT(bar, parity)                          \
-    do {                                                    \
-        if (!mbar_wait(bar, parity)) ctl->abort = 1;        \
-    } while (0)
 
 // Strong-decay chunk of value_side: this thread's 32 output slots of row `row`,
 //   out[s] = exp(+-..) * inter[s] + sum_j P_ij w_j[s] exp(-|G_i[s] - G_j[s]|),
@@ -266,9 +151,9 @@ value_side_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_cons
                      const __grid_constant__ CUtensorMap mapW, const __grid_constant__ CUtensorMap mapG,
                      const __grid_constant__ CUtensorMap mapO, ValueSideArgs a, const int* __restrict__ strong_flag,
                      int32_t* dev_status) {
-    // Two variants of this kernel are launched back to back: this CTA's (batch, head) belongs to
-    // the general one (with the strong-decay path) or to the lean one (moderate chunks only).
-    if ((strong_flag[blockIdx.x] != 0) != GENERAL) return;
+    // Two kernels are launched back to back: this general one (with the strong-decay path) takes
+    // the (batch, head) pairs flagged as having a strong-decay chunk, the pipelined one the others.
+    if (strong_flag[blockIdx.x] == 0) return;
     extern __shared__ unsigned char smem_raw[];
     // align by pointer arithmetic (not an integer round trip) so accesses stay in the shared window
     unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
@@ -615,8 +500,8 @@ key_side_tc_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_consta
                    const __grid_constant__ CUtensorMap mapUk, const __grid_constant__ CUtensorMap mapG,
                    const __grid_constant__ CUtensorMap mapO, KeySideArgs a, const int* __restrict__ strong_flag,
                    int32_t* dev_status) {
-    // (see value_side_tc_kernel: general or lean variant, by (batch, head))
-    if ((strong_flag[blockIdx.x] != 0) != GENERAL) return;
+    // (see value_side_tc_kernel: the flagged (batch, head) pairs only)
+    if (strong_flag[blockIdx.x] == 0) return;
     extern __shared__ unsigned char smem_raw[];
     // align by pointer arithmetic (not an integer round trip) so accesses stay in the shared window
     unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
@@ -882,17 +767,6 @@ key_side_tc_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_consta
 constexpr size_t kSmemValueSide = 1024 + 13 * kPanelB + sizeof(Ctl);
 constexpr size_t kSmemKeySide = 1024 + 13 * kPanelB + sizeof(Ctl);
 
-template <typename K>
-cudaError_t prepare(K kernel, size_t smem) {
-    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-    // each CTA takes the whole tensor memory of its SM: make sure no second CTA can be co-resident
-    int per_sm = 0;
-    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kThreads, smem);
-    if (e != cudaSuccess) return e;
-    return per_sm == 1 ? cudaSuccess : cudaErrorLaunchOutOfResources;
-}
-
 }  // namespace
 
 bool tc_supported(int d_k, int d_v, int M) {
@@ -912,14 +786,17 @@ cudaError_t launch_value_side_tc(const ValueSideArgs& a, int M, int reverse, con
     if (e == cudaSuccess) e = make_tensor_map_bthd(&mg, a.G, a.B, a.T, a.H, kM, kCT, 4);
     if (e != cudaSuccess) return e;
     dim3 grid(a.B * a.H, a.D / kDST);
-#define GSA_LAUNCH_VS(REVV, GEN)                                                                         \
-    e = prepare(value_side_tc_kernel<REVV, GEN>, kSmemValueSide);                                        \
+#define GSA_LAUNCH_VS(REVV, FLAGS)                                                                       \
+    e = prepare(value_side_tc_kernel<REVV, true>, kSmemValueSide);                                       \
     if (e != cudaSuccess) return e;                                                                      \
-    value_side_tc_kernel<REVV, GEN><<<grid, kThreads, kSmemValueSide, st>>>(mq, mk, mw, mg, mo, a, strong_flag, dev_status)
-    // lean variant for the (batch, head) pairs whose chunks all decay moderately, general
-    // variant for the others; each CTA of the variant that is not its own returns at once
-    if (reverse) { GSA_LAUNCH_VS(true, false); GSA_LAUNCH_VS(true, true); }
-    else { GSA_LAUNCH_VS(false, false); GSA_LAUNCH_VS(false, true); }
+    value_side_tc_kernel<REVV, true><<<grid, kThreads, kSmemValueSide, st>>>(mq, mk, mw, mg, mo, a, FLAGS, dev_status)
+    // the pipelined kernel for the (batch, head) pairs whose chunks all decay moderately, this
+    // general one for the others; each CTA of the kernel that is not its own returns at once
+    if (a.wd == nullptr) return cudaErrorInvalidValue;
+    e = launch_value_side_lean(a, reverse, strong_flag, st, dev_status);
+    if (e != cudaSuccess) return e;
+    if (reverse) { GSA_LAUNCH_VS(true, strong_flag); }
+    else { GSA_LAUNCH_VS(false, strong_flag); }
 #undef GSA_LAUNCH_VS
     return cudaGetLastError();
 }
@@ -935,12 +812,15 @@ cudaError_t launch_key_side_tc(const KeySideArgs& a, int M, int reverse, const i
     if (e == cudaSuccess) e = make_tensor_map_bthd(&mg, a.G, a.B, a.T, a.H, kM, kCT, 4);
     if (e != cudaSuccess) return e;
     dim3 grid(a.B * a.H, a.D / kDST);
-#define GSA_LAUNCH_KS(REVV, GEN)                                                                         \
-    e = prepare(key_side_tc_kernel<REVV, GEN>, kSmemKeySide);                                            \
+#define GSA_LAUNCH_KS(REVV, FLAGS)                                                                       \
+    e = prepare(key_side_tc_kernel<REVV, true>, kSmemKeySide);                                           \
     if (e != cudaSuccess) return e;                                                                      \
-    key_side_tc_kernel<REVV, GEN><<<grid, kThreads, kSmemKeySide, st>>>(mv, muq, muk, mg, mo, a, strong_flag, dev_status)
-    if (reverse) { GSA_LAUNCH_KS(true, false); GSA_LAUNCH_KS(true, true); }
-    else { GSA_LAUNCH_KS(false, false); GSA_LAUNCH_KS(false, true); }
+    key_side_tc_kernel<REVV, true><<<grid, kThreads, kSmemKeySide, st>>>(mv, muq, muk, mg, mo, a, FLAGS, dev_status)
+    if (a.uq_d == nullptr || a.uk_d == nullptr) return cudaErrorInvalidValue;
+    e = launch_key_side_lean(a, reverse, strong_flag, st, dev_status);
+    if (e != cudaSuccess) return e;
+    if (reverse) { GSA_LAUNCH_KS(true, strong_flag); }
+    else { GSA_LAUNCH_KS(false, strong_flag); }
 #undef GSA_LAUNCH_KS
     return cudaGetLastError();
 }

@@ -1,0 +1,648 @@
+// Pipelined ("lean") tcgen05 versions of the two chunk primitives of Algorithm 1, for the
+// (batch, head) pairs whose chunks all decay moderately (total log-decay of every chunk above
+// kFactorisedDecayMin), which is every pair of the paper's workloads except the strong-forgetting
+// stress case.
+//
+// Differences from the general kernels (chunk_tc.cu):
+//   * the slot-sized operands arrive by TMA already multiplied by their decay factor and already
+//     in bfloat16 -- w exp(-G) or w exp(G) as a high/low pair, written once per (batch, head) by
+//     the element-wise kernels that produce w (gate kernel, slot softmax forward / backward)
+//     instead of being rebuilt by each of the D/128 slices of every scan;
+//   * the per-chunk chain  product -> mask -> product -> read-out  is software-pipelined: the
+//     issuing lane queues the first product of chunk n+1 behind the last product of chunk n and
+//     requests every tile of chunk n+1 as soon as its buffer has been consumed, so the compute
+//     threads find their next accumulator ready when they finish a chunk.
+//   * tile copies and MMA issue are two lanes of two warps, so that a wait of one (for a store to
+//     drain, for a tile to land) never delays the other.
+// Tile geometry and the bounded waits are those of the general kernels.
+#include "chunk_tc_shared.cuh"
+
+namespace gsa {
+namespace {
+using namespace tc;
+using namespace tcchunk;
+
+// 8 compute warps, one warp whose lane 0 issues every MMA, one warp whose lane 0 requests every
+// tile copy (loads and stores)
+constexpr int kLeanThreads = kComputeThreads + 64;
+constexpr int kMmaThread = kComputeThreads, kCopyThread = kComputeThreads + 32;
+
+struct LeanCtl {
+    // filled by TMA
+    uint64_t bar_x;        // d-sized tiles of a chunk
+    uint64_t bar_x2[2];    // key_side: d-sized tiles, two stages
+    uint64_t bar_w[2];     // pre-decayed slot-sized operand tiles (value_side: two stages; key_side: [0] only)
+    // signalled by tcgen05.commit
+    uint64_t bar_p;        // first product of a chunk (P or A)
+    uint64_t bar_mma1;     // state products (U and the inter-chunk product)
+    uint64_t bar_mma2;     // intra-chunk product
+    uint64_t bar_free1;    // = bar_mma1, for the copy lane: tiles read by the state products may be overwritten
+    uint64_t bar_free2;    // = bar_mma2, for the copy lane: tiles read by the intra-chunk product may be overwritten
+    // signalled by the compute threads (one arrival after their barrier)
+    uint64_t bar_pm;       // masked P / A rows are in shared memory, the P / A accumulator is free
+    uint64_t bar_sb;       // state copy for the next chunk is written, the U accumulator is free
+    uint64_t bar_out;      // output rows are staged, the output accumulators are free
+    // signalled by the copy lane
+    uint64_t bar_free;     // the output staging buffer has been read by its store
+    uint32_t tmem_slot;
+    volatile int abort;
+    alignas(16) float egc[2][kM];   // exp(G of the chunk's last valid row), by chunk parity
+};
+
+// A wait that expires flags the CTA; once flagged, later waits return at once.  The compute
+// threads leave their loop only at the end-of-chunk barrier, on a vote, so that no thread is
+// left waiting at a barrier that others have abandoned.
+#define LEAN_WAIT(bar, parity)                                              \
+    do {                                                                    \
+        if (!ctl->abort && !mbar_wait(bar, parity)) ctl->abort = 1;         \
+    } while (0)
+
+__device__ __forceinline__ bool compute_sync_or(bool pred) {
+    uint32_t out;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.b32 q, %1, 0;\n\t"
+        "bar.red.or.pred p, 1, 256, q;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(out)
+        : "r"((uint32_t)pred)
+        : "memory");
+    return out != 0;
+}
+
+__device__ __forceinline__ void lean_ctl_init(LeanCtl* ctl, int tid, int warp) {
+    if (tid == 0) {
+        mbar_init(&ctl->bar_x, 1);
+        mbar_init(&ctl->bar_w[0], 1);
+        mbar_init(&ctl->bar_w[1], 1);
+        mbar_init(&ctl->bar_x2[0], 1);
+        mbar_init(&ctl->bar_x2[1], 1);
+        mbar_init(&ctl->bar_p, 1);
+        mbar_init(&ctl->bar_mma1, 1);
+        mbar_init(&ctl->bar_mma2, 1);
+        mbar_init(&ctl->bar_free1, 1);
+        mbar_init(&ctl->bar_free2, 1);
+        mbar_init(&ctl->bar_pm, 1);
+        mbar_init(&ctl->bar_sb, 1);
+        mbar_init(&ctl->bar_out, 1);
+        mbar_init(&ctl->bar_free, 1);
+        ctl->abort = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 0) {
+        __syncwarp();
+        tmem_alloc(&ctl->tmem_slot, kTmemCols);
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+}
+
+__device__ __forceinline__ void lean_finish(LeanCtl* ctl, int tid, int warp, uint32_t tmem, int32_t* dev_status) {
+    tc_fence_before_sync();
+    __syncthreads();
+    if (ctl->abort) {
+        if (tid == 0 && dev_status != nullptr) *dev_status = GSA_ERR_TIMEOUT;
+        // bounded grace period for tile copies still in flight before shared memory goes away
+        for (int i = 0; i < 200; ++i) __nanosleep(1000);
+    }
+    __syncthreads();
+    if (warp == 0) {
+        __syncwarp();
+        tmem_dealloc(tmem, kTmemCols);
+    }
+}
+
+// rows published and consumed: shared-memory writes to the async proxy, accumulator reads
+// ordered before the barrier, then one arrival for the issuing lane
+__device__ __forceinline__ void publish(uint64_t* bar, int tid) {
+    fence_async_smem();
+    tc_fence_before_sync();
+    compute_sync();
+    if (tid == 0) mbar_arrive(bar);
+}
+// the same at the end of a chunk, with the vote on leaving the loop
+__device__ __forceinline__ bool publish_and_vote(uint64_t* bar, int tid, bool stop) {
+    fence_async_smem();
+    tc_fence_before_sync();
+    const bool any = compute_sync_or(stop);
+    if (tid == 0) mbar_arrive(bar);
+    return any;
+}
+
+// accumulator columns of the lean kernels
+constexpr int kLvP = 0, kLvO = 128 /* two buffers of 64 */, kLvU = 256, kLvI = 384;     // value_side
+constexpr int kLkA = 0, kLkO = 128 /* two buffers of 128 */, kLkU = 384;                 // key_side
+
+// ======================================================================================
+// value_side: out_i[s] = sum_{j<=i} <xq_i, xk_j> w_j[s] decay_ij[s]  + decayed (xq_i S)[s]
+//   wd holds w exp(-G) (forward) or w exp(G) (reverse) as [hi | lo] bf16 rows of 128.
+//   The row factor -- exp(G_i) forward, exp(-G_i) reverse -- is NOT applied here: the kernel that
+//   sums the slices of `out` multiplies it in (see PendingDecay), so this kernel needs no G tile.
+// ======================================================================================
+template <bool REV>
+__global__ void __launch_bounds__(kLeanThreads, 1)
+value_side_lean_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK,
+                       const __grid_constant__ CUtensorMap mapWd, const __grid_constant__ CUtensorMap mapO,
+                       ValueSideArgs a, const int* __restrict__ strong_flag, int32_t* dev_status) {
+    if (strong_flag[blockIdx.x] != 0) return;       // the general kernel takes this (batch, head)
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
+    unsigned char* sXq = smem;                       // 2 panels                                  (32 KB)
+    unsigned char* sXk = sXq + 2 * kPanelB;          // 2 panels                                  (32 KB)
+    unsigned char* sWd = sXk + 2 * kPanelB;          // decayed weights, MN-major B [128][hi 64 | lo 64], 2 stages (64 KB)
+    unsigned char* sPm = sWd + 4 * kPanelB;          // masked P, K-major A, 2 panels             (32 KB)
+    unsigned char* sSb = sPm + 2 * kPanelB;          // state copy, MN-major B [128][64]          (16 KB)
+    unsigned char* sOut = sSb + kPanelB;             // output rows fp32, 2 panels of 32 slots    (32 KB)
+    LeanCtl* ctl = reinterpret_cast<LeanCtl*>(sOut + 2 * kPanelB);
+
+    const int tid = threadIdx.x, warp = tid >> 5, wq = warp & 3, half = (tid >> 7) & 1, row = tid & 127;
+    const int sb = kHS * half;          // this thread's first slot
+    const int bh = blockIdx.x, slice = blockIdx.y, b = bh / a.H, h = bh % a.H;
+    const int d0 = slice * kDST;
+
+    lean_ctl_init(ctl, tid, warp);
+    const uint32_t tmem = ctl->tmem_slot;
+    const int nchunks = (a.T + kCT - 1) / kCT;
+    auto chunk_t0 = [&](int n) { return (REV ? nchunks - 1 - n : n) * kCT; };
+
+    if (tid == kCopyThread) {
+        // =============================== copy lane: every tile load and store
+        auto load_x = [&](int n) {
+            const int t = chunk_t0(n);
+            mbar_expect_tx(&ctl->bar_x, 4 * kPanelB);
+            tma_load_4d(sXq, &mapQ, &ctl->bar_x, d0, h, t, b);
+            tma_load_4d(sXq + kPanelB, &mapQ, &ctl->bar_x, d0 + 64, h, t, b);
+            tma_load_4d(sXk, &mapK, &ctl->bar_x, d0, h, t, b);
+            tma_load_4d(sXk + kPanelB, &mapK, &ctl->bar_x, d0 + 64, h, t, b);
+        };
+        auto load_w = [&](int n) {
+            const int t = chunk_t0(n), st = n & 1;
+            mbar_expect_tx(&ctl->bar_w[st], 2 * kPanelB);
+            tma_load_4d(sWd + (2 * st) * kPanelB, &mapWd, &ctl->bar_w[st], 0, h, t, b);
+            tma_load_4d(sWd + (2 * st + 1) * kPanelB, &mapWd, &ctl->bar_w[st], 64, h, t, b);
+        };
+        auto store_out = [&](int n) {
+            const int t = chunk_t0(n);
+            tma_store_5d(&mapO, sOut, 0, h, t, b, slice);
+            tma_store_5d(&mapO, sOut + kPanelB, 32, h, t, b, slice);
+            bulk_commit();
+        };
+        prefetch_tmap(&mapQ); prefetch_tmap(&mapK); prefetch_tmap(&mapWd); prefetch_tmap(&mapO);
+        load_x(0);
+        load_w(0);
+        if (nchunks > 1) load_w(1);
+        for (int n = 0; n < nchunks && !ctl->abort; ++n) {
+            // the d-sized tiles are consumed once the state products are done: request the next chunk's
+            LEAN_WAIT(&ctl->bar_free1, n & 1);
+            if (n + 1 < nchunks) load_x(n + 1);
+            // output rows of the previous chunk
+            if (n >= 1) {
+                LEAN_WAIT(&ctl->bar_out, (n - 1) & 1);
+                if (ctl->abort) break;
+                store_out(n - 1);
+                bulk_wait_read();               // the staged rows have left: the buffer may be rewritten
+                mbar_arrive(&ctl->bar_free);
+            }
+            // the weights of chunk n make room for those of chunk n+2
+            LEAN_WAIT(&ctl->bar_free2, n & 1);
+            if (n + 2 < nchunks) load_w(n + 2);
+        }
+        if (!ctl->abort) {
+            LEAN_WAIT(&ctl->bar_out, (nchunks - 1) & 1);
+            if (!ctl->abort) store_out(nchunks - 1);
+        }
+        bulk_wait_read();      // staged output rows must have left before shared memory goes away
+    } else if (tid == kMmaThread) {
+        // =============================== MMA lane
+        constexpr uint32_t idescP = make_idesc(128, 128, false, false);    // xq xk^T
+        constexpr uint32_t idescO = make_idesc(128, kM, false, true);      // xq x state copy (MN-major B)
+        constexpr uint32_t idescU = make_idesc(128, 2 * kM, true, true);   // xk^T (MN-major A) x [W_hi | W_lo]
+        constexpr uint32_t idescI = make_idesc(128, 2 * kM, false, true);  // Pm x [W_hi | W_lo]
+        const uint64_t dQk = desc_kmajor(smem_u32(sXq), 0), dKk = desc_kmajor(smem_u32(sXk), 0);
+        const uint64_t dKm = desc_mnmajor(smem_u32(sXk), 0, kPanelB);
+        const uint64_t dS = desc_mnmajor(smem_u32(sSb), 0, kPanelB);
+        const uint64_t dP = desc_kmajor(smem_u32(sPm), 0);
+        auto kmaj = [](int kk) { return (uint32_t)((kk >> 2) * kPanelB + (kk & 3) * 32); };
+        auto mnmaj = [](int kk) { return (uint32_t)(kk * 2048); };
+        auto issue_p = [&]() {
+#pragma unroll
+            for (int kk = 0; kk < kDST / 16; ++kk)
+                mma_bf16(tmem + kLvP, desc_advance(dQk, kmaj(kk)), desc_advance(dKk, kmaj(kk)), idescP, kk > 0);
+            mma_commit(&ctl->bar_p);
+        };
+        LEAN_WAIT(&ctl->bar_x, 0);
+        tc_fence_after_sync();
+        issue_p();
+        PROF_DECL
+        for (int n = 0; n < nchunks && !ctl->abort; ++n) {
+            const int it = n;
+            (void)it;
+            const uint64_t dW = desc_mnmajor(smem_u32(sWd + 2 * (n & 1) * kPanelB), 0, kPanelB);
+            PROF_MARK();
+            // state products of chunk n: the state copy was written at the end of chunk n-1 (which also
+            // says that the accumulators they overwrite have been read)
+            LEAN_WAIT(&ctl->bar_w[n & 1], (n >> 1) & 1);
+            PROF_MARK();
+            LEAN_WAIT(&ctl->bar_sb, n & 1);
+            tc_fence_after_sync();
+            PROF_MARK();
+#pragma unroll
+            for (int kk = 0; kk < kCT / 16; ++kk)
+                mma_bf16(tmem + kLvU, desc_advance(dKm, mnmaj(kk)), desc_advance(dW, mnmaj(kk)), idescU, kk > 0);
+#pragma unroll
+            for (int kk = 0; kk < kDST / 16; ++kk)
+                mma_bf16(tmem + kLvO + 64 * (n & 1), desc_advance(dQk, kmaj(kk)), desc_advance(dS, mnmaj(kk)), idescO,
+                         kk > 0);
+            mma_commit(&ctl->bar_mma1);
+            mma_commit(&ctl->bar_free1);
+            PROF_MARK();
+            // intra-chunk product once the masked P rows are there
+            LEAN_WAIT(&ctl->bar_pm, n & 1);
+            tc_fence_after_sync();
+            PROF_MARK();
+#pragma unroll
+            for (int kk = 0; kk < kCT / 16; ++kk)
+                mma_bf16(tmem + kLvI, desc_advance(dP, kmaj(kk)), desc_advance(dW, mnmaj(kk)), idescI, kk > 0);
+            mma_commit(&ctl->bar_mma2);
+            mma_commit(&ctl->bar_free2);
+            PROF_MARK();
+            // the P accumulator is free: the next chunk's P queues right behind
+            if (n + 1 < nchunks) {
+                LEAN_WAIT(&ctl->bar_x, (n + 1) & 1);
+                tc_fence_after_sync();
+                PROF_MARK();
+                issue_p();
+            }
+            PROF_MARK();
+            PROF_DUMP("value_side lean mma");
+        }
+    } else if (tid < kComputeThreads) {
+        // =============================== compute threads
+        // state slice: S[c = row][s], slots sb .. sb+31
+        float S[kHS];
+#pragma unroll
+        for (int s = 0; s < kHS; ++s) S[s] = a.S0 ? a.S0[((size_t)bh * kM + sb + s) * a.D + d0 + row] : 0.f;
+        store_state_row<false>(sSb, row, sb, S, nullptr);
+
+        // G of the last valid row of chunk n (threads 0..63, one slot each), one chunk ahead
+        auto chunk_gc = [&](int n) {
+            const int last = min(chunk_t0(n) + kCT, a.T) - 1;
+            return a.G[(((size_t)b * a.T + last) * a.H + h) * kM + tid];
+        };
+        float g_next = 0.f;
+        if (tid < kM) {
+            ctl->egc[0][tid] = __expf(chunk_gc(0));
+            if (nchunks > 1) g_next = chunk_gc(1);
+        }
+        publish(&ctl->bar_sb, tid);
+
+        PROF_DECL
+        for (int n = 0; n < nchunks; ++n) {
+            const int it = n;
+            (void)it;
+            PROF_MARK();
+            const int valid = min(kCT, a.T - chunk_t0(n));
+            const float* egc = ctl->egc[n & 1];
+            if (tid < kM && n + 1 < nchunks) {
+                ctl->egc[(n + 1) & 1][tid] = __expf(g_next);
+                if (n + 2 < nchunks) g_next = chunk_gc(n + 2);
+            }
+            // ---- masked P rows (the barrier inside also publishes egc)
+            LEAN_WAIT(&ctl->bar_p, n & 1);
+            tc_fence_after_sync();
+            PROF_MARK();
+            store_masked_row<REV, false>(tmem, wq, row, half, sPm, sPm);
+            publish(&ctl->bar_pm, tid);
+            PROF_MARK();
+
+            // ---- state update from U: forward S <- exp(G_C) (S + U), reverse S <- exp(G_C) S + U
+            LEAN_WAIT(&ctl->bar_mma1, n & 1);
+            tc_fence_after_sync();
+            PROF_MARK();
+            {
+                float v[kHS], vl[kHS];
+                tmem_ld32(tmem_row_addr(tmem, wq, kLvU + sb), v);
+                tmem_ld32(tmem_row_addr(tmem, wq, kLvU + kM + sb), vl);
+#pragma unroll
+                for (int e = 0; e < kHS; e += 4) {
+                    const float4 ec = *reinterpret_cast<const float4*>(&egc[sb + e]);
+                    const float ecv[4] = {ec.x, ec.y, ec.z, ec.w};
+#pragma unroll
+                    for (int t = 0; t < 4; ++t) {
+                        const float u = v[e + t] + vl[e + t];
+                        S[e + t] = REV ? fmaf(S[e + t], ecv[t], u) : (S[e + t] + u) * ecv[t];
+                    }
+                }
+            }
+            store_state_row<false>(sSb, row, sb, S, nullptr);
+            publish(&ctl->bar_sb, tid);
+            PROF_MARK();
+
+            // ---- output rows without their row factor: inter + intra (reverse: exp(G_C) inter + intra),
+            // staged for one tiled store, clipped at the sequence end
+            LEAN_WAIT(&ctl->bar_mma2, n & 1);
+            tc_fence_after_sync();
+            if (n >= 1) LEAN_WAIT(&ctl->bar_free, (n - 1) & 1);
+            PROF_MARK();
+            {
+                float vo[kHS], vi[kHS];
+                tmem_ld32(tmem_row_addr(tmem, wq, kLvI + sb), vo);
+                tmem_ld32(tmem_row_addr(tmem, wq, kLvI + kM + sb), vi);
+#pragma unroll
+                for (int e = 0; e < kHS; ++e) vo[e] += vi[e];          // high + low weight parts
+                tmem_ld32(tmem_row_addr(tmem, wq, kLvO + 64 * (n & 1) + sb), vi);
+#pragma unroll
+                for (int e = 0; e < kHS; ++e) vo[e] = REV ? fmaf(vi[e], egc[sb + e], vo[e]) : vo[e] + vi[e];
+                unsigned char* panel = sOut + half * kPanelB;
+#pragma unroll
+                for (int c = 0; c < kHS / 4; ++c)
+                    *reinterpret_cast<float4*>(panel + swz128(row, c)) =
+                        make_float4(vo[4 * c], vo[4 * c + 1], vo[4 * c + 2], vo[4 * c + 3]);
+            }
+            (void)valid;
+            const bool stop = publish_and_vote(&ctl->bar_out, tid, ctl->abort != 0);
+            PROF_MARK();
+            PROF_DUMP("value_side lean compute");
+            if (stop) break;
+        }
+        if (!ctl->abort && a.Send) {
+#pragma unroll
+            for (int s = 0; s < kHS; ++s) a.Send[((size_t)bh * kM + sb + s) * a.D + d0 + row] = S[s];
+        }
+    }
+    lean_finish(ctl, tid, warp, tmem, dev_status);
+}
+
+// ======================================================================================
+// key_side: out_i = (uq_i * qscale_i) S + sum_j A_ij xv_j,  A_ij = sum_s uq_i[s] uk_j[s] decay_ij[s]
+//   uq_d / uk_d hold the decayed bf16 rows (first 64 of every 128): forward uq exp(G), uk exp(-G);
+//   reverse uq exp(-G), uk exp(G).
+// ======================================================================================
+template <bool REV>
+__global__ void __launch_bounds__(kLeanThreads, 1)
+key_side_lean_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_constant__ CUtensorMap mapUq,
+                     const __grid_constant__ CUtensorMap mapUk, const __grid_constant__ CUtensorMap mapO,
+                     KeySideArgs a, const int* __restrict__ strong_flag, int32_t* dev_status) {
+    if (strong_flag[blockIdx.x] != 0) return;       // the general kernel takes this (batch, head)
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
+    unsigned char* sXv = smem;                       // xv tile, 2 stages of 2 panels              (64 KB)
+    unsigned char* sQt = sXv + 4 * kPanelB;          // decayed uq, K-major A [128][64]            (16 KB)
+    unsigned char* sKt = sQt + kPanelB;              // decayed uk, K-major / MN-major B [128][64] (16 KB)
+    unsigned char* sAm = sKt + kPanelB;              // masked A, K-major A, 2 panels              (32 KB)
+    unsigned char* sAl = sAm + 2 * kPanelB;          // its rounding residual, 2 panels            (32 KB)
+    unsigned char* sSb = sAl + 2 * kPanelB;          // state copy, K-major B [128 (channel)][64]  (16 KB)
+    unsigned char* sOut = sSb + kPanelB;             // output rows, 2 panels                      (32 KB)
+    LeanCtl* ctl = reinterpret_cast<LeanCtl*>(sOut + 2 * kPanelB);
+
+    const int tid = threadIdx.x, warp = tid >> 5, wq = warp & 3, half = (tid >> 7) & 1, row = tid & 127;
+    const int sb = kHS * half;          // this thread's first slot
+    const int bh = blockIdx.x, slice = blockIdx.y, b = bh / a.H, h = bh % a.H;
+    const int d0 = slice * kDST;
+
+    lean_ctl_init(ctl, tid, warp);
+    const uint32_t tmem = ctl->tmem_slot;
+    const int nchunks = (a.T + kCT - 1) / kCT;
+    auto chunk_t0 = [&](int n) { return (REV ? nchunks - 1 - n : n) * kCT; };
+
+    if (tid == kCopyThread) {
+        // =============================== copy lane: every tile load and store
+        auto load_v = [&](int n) {
+            const int t = chunk_t0(n), st = n & 1;
+            mbar_expect_tx(&ctl->bar_x2[st], 2 * kPanelB);
+            tma_load_4d(sXv + (2 * st) * kPanelB, &mapV, &ctl->bar_x2[st], d0, h, t, b);
+            tma_load_4d(sXv + (2 * st + 1) * kPanelB, &mapV, &ctl->bar_x2[st], d0 + 64, h, t, b);
+        };
+        auto load_qk = [&](int n) {
+            const int t = chunk_t0(n);
+            mbar_expect_tx(&ctl->bar_w[0], 2 * kPanelB);
+            tma_load_4d(sQt, &mapUq, &ctl->bar_w[0], 0, h, t, b);
+            tma_load_4d(sKt, &mapUk, &ctl->bar_w[0], 0, h, t, b);
+        };
+        auto store_out = [&](int n) {
+            const int t = chunk_t0(n);
+            tma_store_4d(&mapO, sOut, d0, h, t, b);
+            tma_store_4d(&mapO, sOut + kPanelB, d0 + 64, h, t, b);
+            bulk_commit();
+        };
+        prefetch_tmap(&mapV); prefetch_tmap(&mapUq); prefetch_tmap(&mapUk); prefetch_tmap(&mapO);
+        load_qk(0);
+        load_v(0);
+        if (nchunks > 1) load_v(1);
+        for (int n = 0; n < nchunks && !ctl->abort; ++n) {
+            // the decayed uq / uk rows are consumed once the state products are done: request the next chunk's
+            LEAN_WAIT(&ctl->bar_free1, n & 1);
+            if (n + 1 < nchunks) load_qk(n + 1);
+            // output rows of the previous chunk
+            if (n >= 1) {
+                LEAN_WAIT(&ctl->bar_out, (n - 1) & 1);
+                if (ctl->abort) break;
+                store_out(n - 1);
+                bulk_wait_read();               // the staged rows have left: the buffer may be rewritten
+                mbar_arrive(&ctl->bar_free);
+            }
+            // the xv tile of chunk n makes room for that of chunk n+2
+            LEAN_WAIT(&ctl->bar_free2, n & 1);
+            if (n + 2 < nchunks) load_v(n + 2);
+        }
+        if (!ctl->abort) {
+            LEAN_WAIT(&ctl->bar_out, (nchunks - 1) & 1);
+            if (!ctl->abort) store_out(nchunks - 1);
+        }
+        bulk_wait_read();      // staged output rows must have left before shared memory goes away
+    } else if (tid == kMmaThread) {
+        // =============================== MMA lane
+        constexpr uint32_t idescA = make_idesc(128, 128, false, false);   // Q~ K~^T
+        constexpr uint32_t idescO = make_idesc(128, kDST, false, false);  // Q~ x state copy (K-major B)
+        constexpr uint32_t idescU = make_idesc(128, kM, true, true);      // xv^T (MN-major A) x K~ (MN-major B)
+        constexpr uint32_t idescV = make_idesc(128, kDST, false, true);   // A x xv (MN-major B)
+        const uint64_t dS = desc_kmajor(smem_u32(sSb), 0);
+        const uint64_t dA = desc_kmajor(smem_u32(sAm), 0), dAl = desc_kmajor(smem_u32(sAl), 0);
+        const uint64_t dQt = desc_kmajor(smem_u32(sQt), 0), dKt = desc_kmajor(smem_u32(sKt), 0);
+        const uint64_t dKtm = desc_mnmajor(smem_u32(sKt), 0, kPanelB);   // the decayed uk read MN-major
+        auto kmaj = [](int kk) { return (uint32_t)((kk >> 2) * kPanelB + (kk & 3) * 32); };
+        auto mnmaj = [](int kk) { return (uint32_t)(kk * 2048); };
+        auto issue_a = [&]() {
+#pragma unroll
+            for (int kk = 0; kk < kM / 16; ++kk)
+                mma_bf16(tmem + kLkA, desc_advance(dQt, kmaj(kk)), desc_advance(dKt, kmaj(kk)), idescA, kk > 0);
+            mma_commit(&ctl->bar_p);
+        };
+        LEAN_WAIT(&ctl->bar_w[0], 0);
+        tc_fence_after_sync();
+        issue_a();
+        PROF_DECL
+        for (int n = 0; n < nchunks && !ctl->abort; ++n) {
+            const int it = n;
+            (void)it;
+            const uint64_t dV = desc_mnmajor(smem_u32(sXv + 2 * (n & 1) * kPanelB), 0, kPanelB);
+            const uint32_t accO = tmem + kLkO + 128 * (n & 1);
+            PROF_MARK();
+            // state products of chunk n: the state copy was written at the end of chunk n-1 (which also
+            // says that the accumulators they overwrite have been read)
+            LEAN_WAIT(&ctl->bar_x2[n & 1], (n >> 1) & 1);
+            PROF_MARK();
+            LEAN_WAIT(&ctl->bar_sb, n & 1);
+            tc_fence_after_sync();
+            PROF_MARK();
+#pragma unroll
+            for (int kk = 0; kk < kCT / 16; ++kk)
+                mma_bf16(tmem + kLkU, desc_advance(dV, mnmaj(kk)), desc_advance(dKtm, mnmaj(kk)), idescU, kk > 0);
+#pragma unroll
+            for (int kk = 0; kk < kM / 16; ++kk)
+                mma_bf16(accO, desc_advance(dQt, kmaj(kk)), desc_advance(dS, kmaj(kk)), idescO, kk > 0);
+            mma_commit(&ctl->bar_mma1);
+            mma_commit(&ctl->bar_free1);
+            PROF_MARK();
+            // intra-chunk product (masked A and its rounding residual) on top of the inter-chunk one
+            LEAN_WAIT(&ctl->bar_pm, n & 1);
+            tc_fence_after_sync();
+            PROF_MARK();
+#pragma unroll
+            for (int kk = 0; kk < kCT / 16; ++kk)
+                mma_bf16(accO, desc_advance(dA, kmaj(kk)), desc_advance(dV, mnmaj(kk)), idescV, true);
+#pragma unroll
+            for (int kk = 0; kk < kCT / 16; ++kk)
+                mma_bf16(accO, desc_advance(dAl, kmaj(kk)), desc_advance(dV, mnmaj(kk)), idescV, true);
+            mma_commit(&ctl->bar_mma2);
+            mma_commit(&ctl->bar_free2);
+            PROF_MARK();
+            // the A accumulator is free: the next chunk's A queues right behind
+            if (n + 1 < nchunks) {
+                LEAN_WAIT(&ctl->bar_w[0], (n + 1) & 1);
+                tc_fence_after_sync();
+                PROF_MARK();
+                issue_a();
+            }
+            PROF_MARK();
+            PROF_DUMP("key_side lean mma");
+        }
+    } else if (tid < kComputeThreads) {
+        // =============================== compute threads
+        // state slice, transposed: S[c = row][s], slots sb .. sb+31
+        float S[kHS];
+#pragma unroll
+        for (int s = 0; s < kHS; ++s) S[s] = a.S0 ? a.S0[((size_t)bh * kM + sb + s) * a.D + d0 + row] : 0.f;
+
+        // G of the last valid row of chunk n (threads 0..63, one slot each)
+        auto chunk_gc = [&](int n) {
+            const int t0 = chunk_t0(n);
+            const int last = min(t0 + kCT, a.T) - 1;
+            return a.G[(((size_t)b * a.T + last) * a.H + h) * kM + tid];
+        };
+        float g_next = 0.f;      // gc of chunk n+1, loaded one chunk ahead
+        if (tid < kM) {
+            ctl->egc[0][tid] = __expf(chunk_gc(0));
+            if (nchunks > 1) g_next = chunk_gc(1);
+        }
+        compute_sync();
+        // bf16 copy of the state for the first chunk's inter-chunk product (reverse: scaled by the
+        // chunk's total decay, which the decayed uq rows leave out)
+        if (REV) store_state_row<true>(sSb, row, sb, S, ctl->egc[0]);
+        else store_state_row<false>(sSb, row, sb, S, nullptr);
+        publish(&ctl->bar_sb, tid);
+
+        for (int n = 0; n < nchunks; ++n) {
+            const float* egc = ctl->egc[n & 1];
+            if (tid < kM && n + 1 < nchunks) {
+                ctl->egc[(n + 1) & 1][tid] = __expf(g_next);
+                if (n + 2 < nchunks) g_next = chunk_gc(n + 2);
+            }
+            // ---- masked A rows as a bf16 high/low pair (the barrier inside also publishes egc)
+            LEAN_WAIT(&ctl->bar_p, n & 1);
+            tc_fence_after_sync();
+            store_masked_row<REV, true>(tmem, wq, row, half, sAm, sAl);
+            publish(&ctl->bar_pm, tid);
+
+            // ---- state update from U^T: forward S <- exp(G_C) (S + U^T), reverse S <- exp(G_C) S + U^T
+            LEAN_WAIT(&ctl->bar_mma1, n & 1);
+            tc_fence_after_sync();
+            {
+                float v[kHS];
+                tmem_ld32(tmem_row_addr(tmem, wq, kLkU + sb), v);
+#pragma unroll
+                for (int e = 0; e < kHS; e += 4) {
+                    const float4 ec = *reinterpret_cast<const float4*>(&egc[sb + e]);
+                    const float ecv[4] = {ec.x, ec.y, ec.z, ec.w};
+#pragma unroll
+                    for (int t = 0; t < 4; ++t)
+                        S[e + t] = REV ? fmaf(S[e + t], ecv[t], v[e + t]) : (S[e + t] + v[e + t]) * ecv[t];
+                }
+            }
+            if (REV) store_state_row<true>(sSb, row, sb, S, ctl->egc[(n + 1) & 1]);
+            else store_state_row<false>(sSb, row, sb, S, nullptr);
+            publish(&ctl->bar_sb, tid);
+
+            // ---- output rows -> bf16, staged for the tiled store (clipped at the sequence end)
+            LEAN_WAIT(&ctl->bar_mma2, n & 1);
+            tc_fence_after_sync();
+            if (n >= 1) LEAN_WAIT(&ctl->bar_free, (n - 1) & 1);
+#pragma unroll 1
+            for (int c0 = 0; c0 < 64; c0 += 32) {
+                float v[32];
+                tmem_ld32(tmem_row_addr(tmem, wq, kLkO + 128 * (n & 1) + 64 * half + c0), v);
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    const float x[8] = {v[8 * c], v[8 * c + 1], v[8 * c + 2], v[8 * c + 3],
+                                        v[8 * c + 4], v[8 * c + 5], v[8 * c + 6], v[8 * c + 7]};
+                    store_chunk(sOut + half * kPanelB, row, (c0 >> 3) + c, x);
+                }
+            }
+            if (publish_and_vote(&ctl->bar_out, tid, ctl->abort != 0)) break;
+        }
+        if (!ctl->abort && a.Send) {
+#pragma unroll
+            for (int s = 0; s < kHS; ++s) a.Send[((size_t)bh * kM + sb + s) * a.D + d0 + row] = S[s];
+        }
+    }
+    lean_finish(ctl, tid, warp, tmem, dev_status);
+}
+
+constexpr size_t kSmemLean = 1024 + 13 * kPanelB + sizeof(LeanCtl);
+
+}  // namespace
+
+cudaError_t launch_value_side_lean(const ValueSideArgs& a, int reverse, const int* strong_flag, cudaStream_t st,
+                                   int32_t* dev_status) {
+    CUtensorMap mq, mk, mw, mo;
+    cudaError_t e = make_tensor_map_bthd(&mq, a.xq, a.B, a.T, a.H, a.D, kCT, 2);
+    if (e == cudaSuccess) e = make_tensor_map_sliced(&mo, a.out, a.D / kDST, a.B, a.T, a.H, kM, kCT, 4);
+    if (e == cudaSuccess) e = make_tensor_map_bthd(&mk, a.xk, a.B, a.T, a.H, a.D, kCT, 2);
+    if (e == cudaSuccess) e = make_tensor_map_bthd(&mw, a.wd, a.B, a.T, a.H, 2 * kM, kCT, 2);
+    if (e != cudaSuccess) return e;
+    dim3 grid(a.B * a.H, a.D / kDST);
+    if (reverse) {
+        e = prepare(value_side_lean_kernel<true>, kSmemLean, kLeanThreads);
+        if (e != cudaSuccess) return e;
+        value_side_lean_kernel<true><<<grid, kLeanThreads, kSmemLean, st>>>(mq, mk, mw, mo, a, strong_flag, dev_status);
+    } else {
+        e = prepare(value_side_lean_kernel<false>, kSmemLean, kLeanThreads);
+        if (e != cudaSuccess) return e;
+        value_side_lean_kernel<false><<<grid, kLeanThreads, kSmemLean, st>>>(mq, mk, mw, mo, a, strong_flag, dev_status);
+    }
+    return cudaGetLastError();
+}
+
+cudaError_t launch_key_side_lean(const KeySideArgs& a, int reverse, const int* strong_flag, cudaStream_t st,
+                                 int32_t* dev_status) {
+    CUtensorMap mv, muq, muk, mo;
+    cudaError_t e = make_tensor_map_bthd(&mv, a.xv, a.B, a.T, a.H, a.D, kCT, 2);
+    if (e == cudaSuccess) e = make_tensor_map_bthd(&mo, a.out, a.B, a.T, a.H, a.D, kCT, 2);
+    if (e == cudaSuccess) e = make_tensor_map_bthd(&muq, a.uq_d, a.B, a.T, a.H, 2 * kM, kCT, 2);
+    if (e == cudaSuccess) e = make_tensor_map_bthd(&muk, a.uk_d, a.B, a.T, a.H, 2 * kM, kCT, 2);
+    if (e != cudaSuccess) return e;
+    dim3 grid(a.B * a.H, a.D / kDST);
+    if (reverse) {
+        e = prepare(key_side_lean_kernel<true>, kSmemLean, kLeanThreads);
+        if (e != cudaSuccess) return e;
+        key_side_lean_kernel<true><<<grid, kLeanThreads, kSmemLean, st>>>(mv, muq, muk, mo, a, strong_flag, dev_status);
+    } else {
+        e = prepare(key_side_lean_kernel<false>, kSmemLean, kLeanThreads);
+        if (e != cudaSuccess) return e;
+        key_side_lean_kernel<false><<<grid, kLeanThreads, kSmemLean, st>>>(mv, muq, muk, mo, a, strong_flag, dev_status);
+    }
+    return cudaGetLastError();
+}
+
+}  // namespace gsa

@@ -80,6 +80,9 @@ struct ValueSideArgs {
     float* Send;                      // nullable
     float* out;                       // [nslice][B,T,H,M]
     int B, T, H, D;
+    // tensor-core path: the weights already multiplied by their decay factor, bf16 rows of 2M
+    // [high part | rounding residual] of w exp(-G) (forward) or w exp(G) (reverse); nullable
+    const void* wd;
 };
 struct KeySideArgs {
     const float* uq; const float* uk; const float* G;
@@ -88,14 +91,38 @@ struct KeySideArgs {
     float* Send;                      // nullable
     void* out;                        // io [B,T,H,D]
     int B, T, H, D;
+    // tensor-core path: decayed bf16 rows of 2M (the first M are used): forward uq exp(G) and
+    // uk exp(-G), reverse uq exp(-G) and uk exp(G); nullable (both or neither)
+    const void* uq_d; const void* uk_d;
+};
+
+// The pipelined tensor-core value_side kernel leaves the row factor of its partial sums --
+// exp(G_i) of a forward run, exp(-G_i) of a time-reversed one -- to the element-wise kernel that
+// consumes them (slot softmax forward / backward, gate gradient), which sums the D/128 slices
+// anyway.  strong[(b * nseg + segment) * H + h] != 0 marks the (batch, head) pairs that the general
+// kernel wrote, with the factor already applied.  G == nullptr: nothing is pending.
+struct PendingDecay {
+    const float* G;
+    const int* strong;
+    int T, H, nseg;
+    // row = (b * T + t) * H + h of a [B,T,H,M] tensor
+    __host__ __device__ bool pending(size_t row) const {
+        if (G == nullptr) return false;
+        const int h = (int)(row % H);
+        const size_t bt = row / H;
+        const int t = (int)(bt % T), b = (int)(bt / T);
+        return strong[((size_t)b * nseg + t / (T / nseg)) * H + h] == 0;
+    }
 };
 
 // launchers (definitions in the .cu files); all return cudaGetLastError() of the launch
 // strong_flag (nullable, [B*H] ints, zeroed by the caller): set to 1 for every (b,h) that has a
 // chunk whose total log-decay is below kFactorisedDecayMin (nseg > 1: [B*nseg*H], per segment).
+// decayed (nullable, bf16 [B,T,H,2M]): rows [high part | rounding residual] of I exp(-G), the
+// input-gate operand of the pipelined tensor-core kernels.
 cudaError_t launch_gate_cumsum(const float* gate, int gate_is_log, float* G, float* I,
                                int B, int T, int H, int M, int chunk, int* strong_flag, int nseg,
-                               cudaStream_t st);
+                               void* decayed, cudaStream_t st);
 // Segment-parallel scheduling (T cut into nseg segments run as independent sequences): per-segment
 // log-decay [B,nseg,H,M] from G, and the start memories [B,nseg,H,M,D] of every segment from the
 // end memories of the segments run from empty memories.
@@ -104,17 +131,21 @@ cudaError_t launch_segment_logdecay(const float* G, float* seg_logdecay, int B, 
 cudaError_t launch_segment_combine(const float* seg_logdecay, const float* local_end, const float* S0,
                                    float* start, float* final_state, int B, int H, int M, int D, int nseg,
                                    cudaStream_t st);
+// G, p_decayed / dz_decayed (nullable together; bf16 [rows, 2M]): rows [high | residual] of
+// p exp(G) and dz exp(G), operands of the pipelined tensor-core kernels.
 cudaError_t launch_slot_softmax_fwd(const float* part, int nslice, float scale, float* ok,
-                                    float* p, size_t rows, int M, cudaStream_t st);
+                                    float* p, size_t rows, int M, const float* G, void* p_decayed,
+                                    PendingDecay pend, cudaStream_t st);
 cudaError_t launch_slot_softmax_bwd(const float* ok, const float* dp_part, int nslice,
                                     float scale, float* p, float* dz, float* u, size_t rows,
-                                    int M, cudaStream_t st);
+                                    int M, const float* G, void* p_decayed, void* dz_decayed,
+                                    PendingDecay pend, cudaStream_t st);
 cudaError_t launch_gate_grad(const float* u, const float* I, const float* dIk_part, int nsk,
                              const float* dIv_part, int nsv, const float* gate,
                              int gate_is_log, const float* dKT, const float* KT,
                              const float* dVT, const float* VT, int d_k, int d_v,
                              float* chunk_tot, float* dgate, int B, int T, int H, int M,
-                             cudaStream_t st);
+                             PendingDecay pend, cudaStream_t st);
 int gate_grad_blocks(int T);       // entries per (b,h,slot) of launch_gate_grad's scratch
 cudaError_t launch_value_side_simt(const ValueSideArgs& a, int io, int M, int reverse,
                                    cudaStream_t st);
@@ -128,6 +159,12 @@ cudaError_t launch_value_side_tc(const ValueSideArgs& a, int M, int reverse, con
                                  cudaStream_t st, int32_t* dev_status);
 cudaError_t launch_key_side_tc(const KeySideArgs& a, int M, int reverse, const int* strong_flag,
                                cudaStream_t st, int32_t* dev_status);
+// the pipelined kernels for the (batch, head) pairs without a strong-decay chunk (strong_flag 0);
+// they need the pre-decayed operands of the argument structs
+cudaError_t launch_value_side_lean(const ValueSideArgs& a, int reverse, const int* strong_flag, cudaStream_t st,
+                                   int32_t* dev_status);
+cudaError_t launch_key_side_lean(const KeySideArgs& a, int reverse, const int* strong_flag, cudaStream_t st,
+                                 int32_t* dev_status);
 cudaError_t launch_decode(const gsa_params_t& p, const void* q, const void* k, const void* v,
                           const float* gate, float* Ks, float* Vs, void* o, cudaStream_t st);
 

@@ -7,99 +7,180 @@
 namespace gsa {
 
 // ------------------------------------------------------------------ chunk_cumsum
-// One CTA per (b,h, chunk): M slots x (chunk / 16) row groups.  A thread takes the logs of
-// its 16 rows (16 independent loads in flight), sums them, the group sums are scanned through
-// shared memory, and the thread writes its 16 running sums.  `chunk` is the chunk length of
-// the kernels that will consume G (64 or 128).
+// One CTA per (b,h, chunk): M/2 slot pairs x (chunk / 16) row groups.  A thread takes the logs
+// of its 16 rows x 2 slots (16 independent 8-byte loads in flight), sums them, the group sums
+// are scanned through shared memory, and the thread writes its running sums.  `chunk` is the
+// chunk length of the kernels that will consume G (64 or 128).
 constexpr int kCumRows = 16;
 
+// x as a bf16 pair: the rounded value and the rounding residual
+__device__ __forceinline__ void split_bf16(float x, __nv_bfloat16& hi, __nv_bfloat16& lo) {
+    hi = __float2bfloat16_rn(x);
+    lo = __float2bfloat16_rn(x - __bfloat162float(hi));
+}
+// two adjacent columns (c, c+1; c even) of a decayed-operand row [hi(M) | lo(M)]
 template <int M>
-__global__ void __launch_bounds__(M * 8) gate_cumsum_kernel(const float* __restrict__ gate,
+__device__ __forceinline__ void store_split2(__nv_bfloat16* row, int c, float x0, float x1) {
+    __nv_bfloat162 hi, lo;
+    split_bf16(x0, hi.x, lo.x);
+    split_bf16(x1, hi.y, lo.y);
+    *reinterpret_cast<__nv_bfloat162*>(row + c) = hi;
+    *reinterpret_cast<__nv_bfloat162*>(row + M + c) = lo;
+}
+
+template <int M>
+__global__ void __launch_bounds__(M * 4) gate_cumsum_kernel(const float* __restrict__ gate,
                                                             int gate_is_log,
                                                             float* __restrict__ G,
                                                             float* __restrict__ I, int T, int H,
-                                                            int chunk, int* __restrict__ strong_flag, int nseg) {
+                                                            int chunk, int* __restrict__ strong_flag, int nseg,
+                                                            __nv_bfloat16* __restrict__ decayed) {
     __shared__ double group_sum[8][M];
-    const int s = threadIdx.x, grp = threadIdx.y;          // blockDim.y = chunk / 16 <= 8
+    const int s = 2 * threadIdx.x, grp = threadIdx.y;          // blockDim.y = chunk / 16 <= 8
     const int n = blockIdx.y;
     const int bh = blockIdx.x, b = bh / H, h = bh % H;
     const int t0 = n * chunk + grp * kCumRows;
     const int rows = max(0, min(kCumRows, min(T, (n + 1) * chunk) - t0));
     const size_t stride = (size_t)H * M;
     const size_t base = (((size_t)b * T + t0) * H + h) * M + s;
-    float g[kCumRows];
+    float2 g[kCumRows], inps[kCumRows];
 #pragma unroll
     for (int i = 0; i < kCumRows; ++i) {
-        float x = gate_is_log ? 0.f : 1.f;
-        if (i < rows) x = gate[base + (size_t)i * stride];
-        float inp;
+        const float neutral = gate_is_log ? 0.f : 1.f;
+        float2 x = make_float2(neutral, neutral);
+        if (i < rows) x = *reinterpret_cast<const float2*>(gate + base + (size_t)i * stride);
         if (gate_is_log) {
             g[i] = x;
-            inp = -expm1f(x);
+            inps[i] = make_float2(-expm1f(x.x), -expm1f(x.y));
         } else {
-            g[i] = logf(x);
-            inp = 1.f - x;
+            g[i] = make_float2(logf(x.x), logf(x.y));
+            inps[i] = make_float2(1.f - x.x, 1.f - x.y);
         }
-        g[i] = fmaxf(g[i], kLogGateMin);
-        if (i < rows) I[base + (size_t)i * stride] = inp;
+        g[i].x = fmaxf(g[i].x, kLogGateMin);
+        g[i].y = fmaxf(g[i].y, kLogGateMin);
+        if (i < rows) *reinterpret_cast<float2*>(I + base + (size_t)i * stride) = inps[i];
     }
     // running sums in fp64 (a handful of adds per thread): G is then the correctly rounded
     // cumulative sum, which matters when strong decay makes |G| reach the hundreds
-    double run[kCumRows], acc = 0.0;
+    double run0[kCumRows], run1[kCumRows], acc0 = 0.0, acc1 = 0.0;
 #pragma unroll
     for (int i = 0; i < kCumRows; ++i) {
-        acc += (i < rows) ? (double)g[i] : 0.0;
-        run[i] = acc;
+        acc0 += (i < rows) ? (double)g[i].x : 0.0;
+        acc1 += (i < rows) ? (double)g[i].y : 0.0;
+        run0[i] = acc0;
+        run1[i] = acc1;
     }
-    group_sum[grp][s] = acc;
+    group_sum[grp][s] = acc0;
+    group_sum[grp][s + 1] = acc1;
     __syncthreads();
-    double before = 0.0;
-    for (int q = 0; q < grp; ++q) before += group_sum[q][s];
-    // the chunk's total log-decay decides which variant of the chunk kernels takes this (b,h)
+    double before0 = 0.0, before1 = 0.0;
+    for (int q = 0; q < grp; ++q) {
+        before0 += group_sum[q][s];
+        before1 += group_sum[q][s + 1];
+    }
+    // the chunk's total log-decay decides which of the chunk kernels takes this (b,h)
     // (with segment-parallel scheduling the flags are per (batch, segment, head))
-    if (strong_flag != nullptr && grp == (int)blockDim.y - 1 && before + acc < (double)kFactorisedDecayMin) {
+    if (strong_flag != nullptr && grp == (int)blockDim.y - 1 &&
+        fmin(before0 + acc0, before1 + acc1) < (double)kFactorisedDecayMin) {
         const int seg = (int)(((long long)n * chunk) / (T / nseg));
         strong_flag[(b * nseg + seg) * H + h] = 1;
     }
 #pragma unroll
     for (int i = 0; i < kCumRows; ++i)
-        if (i < rows) G[base + (size_t)i * stride] = (float)(before + run[i]);
+        if (i < rows) {
+            const float G0 = (float)(before0 + run0[i]), G1 = (float)(before1 + run1[i]);
+            *reinterpret_cast<float2*>(G + base + (size_t)i * stride) = make_float2(G0, G1);
+            if (decayed != nullptr) {
+                // (meaningful for moderate decay only; pairs with a strong-decay chunk do not read it)
+                store_split2<M>(decayed + 2 * (base + (size_t)i * stride - s), s, inps[i].x * __expf(-G0),
+                                inps[i].y * __expf(-G1));
+            }
+        }
 }
 
 cudaError_t launch_gate_cumsum(const float* gate, int gate_is_log, float* G, float* I, int B,
-                               int T, int H, int M, int chunk, int* strong_flag, int nseg, cudaStream_t st) {
+                               int T, int H, int M, int chunk, int* strong_flag, int nseg, void* decayed, cudaStream_t st) {
     if (chunk % kCumRows != 0 || chunk / kCumRows > 8) return cudaErrorInvalidValue;
     const int nchunks = (T + chunk - 1) / chunk;
-    dim3 block(M, chunk / kCumRows);
+    dim3 block(M / 2, chunk / kCumRows);
     dim3 grid(B * H, nchunks);
     if (M == 64)
-        gate_cumsum_kernel<64><<<grid, block, 0, st>>>(gate, gate_is_log, G, I, T, H, chunk, strong_flag, nseg < 1 ? 1 : nseg);
+        gate_cumsum_kernel<64><<<grid, block, 0, st>>>(gate, gate_is_log, G, I, T, H, chunk, strong_flag, nseg < 1 ? 1 : nseg,
+                                                       static_cast<__nv_bfloat16*>(decayed));
     else
-        gate_cumsum_kernel<32><<<grid, block, 0, st>>>(gate, gate_is_log, G, I, T, H, chunk, strong_flag, nseg < 1 ? 1 : nseg);
+        gate_cumsum_kernel<32><<<grid, block, 0, st>>>(gate, gate_is_log, G, I, T, H, chunk, strong_flag, nseg < 1 ? 1 : nseg,
+                                                       static_cast<__nv_bfloat16*>(decayed));
     return cudaGetLastError();
 }
 
 // ------------------------------------------------------------------ slot softmax
-// One warp per token-head row of M slots (M/32 values per lane).
+// One warp per token-head row of M slots: lane l holds the R = M/32 adjacent slots l R .. l R + R-1
+// (one 8-byte access per tensor and lane for M = 64).
+template <int R>
+__device__ __forceinline__ void ld_vec(const float* p, float (&x)[R]) {
+    if constexpr (R == 2) {
+        const float2 v = *reinterpret_cast<const float2*>(p);
+        x[0] = v.x; x[1] = v.y;
+    } else {
+#pragma unroll
+        for (int r = 0; r < R; ++r) x[r] = p[r];
+    }
+}
+template <int R>
+__device__ __forceinline__ void st_vec(float* p, const float (&x)[R]) {
+    if constexpr (R == 2) {
+        *reinterpret_cast<float2*>(p) = make_float2(x[0], x[1]);
+    } else {
+#pragma unroll
+        for (int r = 0; r < R; ++r) p[r] = x[r];
+    }
+}
+// the lane's slots of a decayed-operand row [hi(M) | lo(M)]
+template <int M, int R>
+__device__ __forceinline__ void st_split(__nv_bfloat16* row, int c, const float (&x)[R]) {
+    if constexpr (R == 2) {
+        store_split2<M>(row, c, x[0], x[1]);
+    } else {
+#pragma unroll
+        for (int r = 0; r < R; ++r) split_bf16(x[r], row[c + r], row[M + c + r]);
+    }
+}
+
 template <int M>
 __global__ void __launch_bounds__(256) slot_softmax_fwd_kernel(const float* __restrict__ part,
                                                                int nslice, float scale,
                                                                float* __restrict__ ok,
                                                                float* __restrict__ p,
-                                                               size_t rows) {
+                                                               size_t rows, const float* __restrict__ G,
+                                                               __nv_bfloat16* __restrict__ p_decayed,
+                                                               PendingDecay pend) {
     constexpr int R = M / 32;
     const size_t row = (size_t)blockIdx.x * 8 + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
     if (row >= rows) return;
     const size_t total = rows * M;
-    float z[R];
+    const size_t idx = row * M + lane * R;
+    const bool pending = pend.pending(row);
+    float z[R], eg[R];
+#pragma unroll
+    for (int r = 0; r < R; ++r) { z[r] = 0.f; eg[r] = 1.f; }
+#pragma unroll 4
+    for (int sl = 0; sl < nslice; ++sl) {
+        float t[R];
+        ld_vec<R>(part + idx + (size_t)sl * total, t);
+#pragma unroll
+        for (int r = 0; r < R; ++r) z[r] += t[r];
+    }
+    if (G != nullptr) {
+        ld_vec<R>(G + idx, eg);
+#pragma unroll
+        for (int r = 0; r < R; ++r) eg[r] = __expf(eg[r]);
+    }
     float zmax = -INFINITY;
 #pragma unroll
     for (int r = 0; r < R; ++r) {
-        const size_t idx = row * M + lane + 32 * r;
-        float acc = 0.f;
-        for (int sl = 0; sl < nslice; ++sl) acc += part[idx + (size_t)sl * total];
-        z[r] = acc * scale;
+        if (pending) z[r] *= eg[r];
+        z[r] *= scale;
         zmax = fmaxf(zmax, z[r]);
     }
 #pragma unroll
@@ -111,20 +192,26 @@ __global__ void __launch_bounds__(256) slot_softmax_fwd_kernel(const float* __re
     for (int o = 16; o; o >>= 1) den += __shfl_xor_sync(0xffffffffu, den, o);
     const float inv = 1.f / den;
 #pragma unroll
-    for (int r = 0; r < R; ++r) {
-        const size_t idx = row * M + lane + 32 * r;
-        ok[idx] = z[r];
-        p[idx] = e[r] * inv;
+    for (int r = 0; r < R; ++r) e[r] *= inv;
+    st_vec<R>(ok + idx, z);
+    st_vec<R>(p + idx, e);
+    if (p_decayed != nullptr) {
+#pragma unroll
+        for (int r = 0; r < R; ++r) e[r] *= eg[r];
+        st_split<M, R>(p_decayed + row * 2 * M, lane * R, e);
     }
 }
 
 cudaError_t launch_slot_softmax_fwd(const float* part, int nslice, float scale, float* ok,
-                                    float* p, size_t rows, int M, cudaStream_t st) {
+                                    float* p, size_t rows, int M, const float* G, void* p_decayed,
+                                    PendingDecay pend, cudaStream_t st) {
     const unsigned grid = (unsigned)((rows + 7) / 8);
     if (M == 64)
-        slot_softmax_fwd_kernel<64><<<grid, 256, 0, st>>>(part, nslice, scale, ok, p, rows);
+        slot_softmax_fwd_kernel<64><<<grid, 256, 0, st>>>(part, nslice, scale, ok, p, rows, G,
+                                                          static_cast<__nv_bfloat16*>(p_decayed), pend);
     else
-        slot_softmax_fwd_kernel<32><<<grid, 256, 0, st>>>(part, nslice, scale, ok, p, rows);
+        slot_softmax_fwd_kernel<32><<<grid, 256, 0, st>>>(part, nslice, scale, ok, p, rows, G,
+                                                          static_cast<__nv_bfloat16*>(p_decayed), pend);
     return cudaGetLastError();
 }
 
@@ -140,22 +227,38 @@ __global__ void __launch_bounds__(256) slot_softmax_bwd_kernel(const float* __re
                                                                float* __restrict__ p,
                                                                float* __restrict__ dz,
                                                                float* __restrict__ u,
-                                                               size_t rows) {
+                                                               size_t rows, const float* __restrict__ G,
+                                                               __nv_bfloat16* __restrict__ p_decayed,
+                                                               __nv_bfloat16* __restrict__ dz_decayed,
+                                                               PendingDecay pend) {
     constexpr int R = M / 32;
     const size_t row = (size_t)blockIdx.x * 8 + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
     if (row >= rows) return;
     const size_t total = rows * M;
-    float z[R], dpv[R];
+    const size_t idx = row * M + lane * R;
+    const bool pending = pend.pending(row);
+    float z[R], dpv[R], eg[R];
+    ld_vec<R>(ok + idx, z);
+#pragma unroll
+    for (int r = 0; r < R; ++r) { dpv[r] = 0.f; eg[r] = 1.f; }
+#pragma unroll 4
+    for (int sl = 0; sl < nslice; ++sl) {
+        float t[R];
+        ld_vec<R>(dp_part + idx + (size_t)sl * total, t);
+#pragma unroll
+        for (int r = 0; r < R; ++r) dpv[r] += t[r];
+    }
+    if (G != nullptr) {
+        ld_vec<R>(G + idx, eg);
+#pragma unroll
+        for (int r = 0; r < R; ++r) eg[r] = __expf(eg[r]);
+    }
     float zmax = -INFINITY;
 #pragma unroll
     for (int r = 0; r < R; ++r) {
-        const size_t idx = row * M + lane + 32 * r;
-        z[r] = ok[idx];
+        if (pending) dpv[r] *= eg[r];
         zmax = fmaxf(zmax, z[r]);
-        float acc = 0.f;
-        for (int sl = 0; sl < nslice; ++sl) acc += dp_part[idx + (size_t)sl * total];
-        dpv[r] = acc;
     }
 #pragma unroll
     for (int o = 16; o; o >>= 1) zmax = fmaxf(zmax, __shfl_xor_sync(0xffffffffu, zmax, o));
@@ -170,24 +273,37 @@ __global__ void __launch_bounds__(256) slot_softmax_bwd_kernel(const float* __re
     for (int r = 0; r < R; ++r) { e[r] *= inv; pdp += e[r] * dpv[r]; }
 #pragma unroll
     for (int o = 16; o; o >>= 1) pdp += __shfl_xor_sync(0xffffffffu, pdp, o);
+    float dzv[R], uv[R];
 #pragma unroll
     for (int r = 0; r < R; ++r) {
-        const size_t idx = row * M + lane + 32 * r;
         const float dok = e[r] * (dpv[r] - pdp);
-        p[idx] = e[r];
-        dz[idx] = scale * dok;
-        u[idx] = e[r] * dpv[r] + z[r] * dok;
+        dzv[r] = scale * dok;
+        uv[r] = e[r] * dpv[r] + z[r] * dok;
+    }
+    st_vec<R>(p + idx, e);
+    st_vec<R>(dz + idx, dzv);
+    st_vec<R>(u + idx, uv);
+    if (p_decayed != nullptr) {
+#pragma unroll
+        for (int r = 0; r < R; ++r) { e[r] *= eg[r]; dzv[r] *= eg[r]; }
+        st_split<M, R>(p_decayed + row * 2 * M, lane * R, e);
+        st_split<M, R>(dz_decayed + row * 2 * M, lane * R, dzv);
     }
 }
 
 cudaError_t launch_slot_softmax_bwd(const float* ok, const float* dp_part, int nslice,
                                     float scale, float* p, float* dz, float* u, size_t rows,
-                                    int M, cudaStream_t st) {
+                                    int M, const float* G, void* p_decayed, void* dz_decayed,
+                                    PendingDecay pend, cudaStream_t st) {
     const unsigned grid = (unsigned)((rows + 7) / 8);
     if (M == 64)
-        slot_softmax_bwd_kernel<64><<<grid, 256, 0, st>>>(ok, dp_part, nslice, scale, p, dz, u, rows);
+        slot_softmax_bwd_kernel<64><<<grid, 256, 0, st>>>(ok, dp_part, nslice, scale, p, dz, u, rows, G,
+                                                          static_cast<__nv_bfloat16*>(p_decayed),
+                                                          static_cast<__nv_bfloat16*>(dz_decayed), pend);
     else
-        slot_softmax_bwd_kernel<32><<<grid, 256, 0, st>>>(ok, dp_part, nslice, scale, p, dz, u, rows);
+        slot_softmax_bwd_kernel<32><<<grid, 256, 0, st>>>(ok, dp_part, nslice, scale, p, dz, u, rows, G,
+                                                          static_cast<__nv_bfloat16*>(p_decayed),
+                                                          static_cast<__nv_bfloat16*>(dz_decayed), pend);
     return cudaGetLastError();
 }
 
@@ -262,10 +378,10 @@ __global__ void __launch_bounds__(M * 16) gate_grad_scan_kernel(
 // at the block's end, turned into the gate gradient as if nothing followed the block, plus
 // the block total for the scan.  One read of every input.
 template <int M>
-__global__ void __launch_bounds__(256) gate_grad_local_kernel(
+__global__ void __launch_bounds__(256, 2) gate_grad_local_kernel(
     const float* __restrict__ u, const float* __restrict__ I, const float* __restrict__ dIk, int nsk,
     const float* __restrict__ dIv, int nsv, const float* __restrict__ gate, int gate_is_log,
-    float* __restrict__ blk_tot, float* __restrict__ dgate, int B, int T, int H, int nblk) {
+    float* __restrict__ blk_tot, float* __restrict__ dgate, int B, int T, int H, int nblk, PendingDecay pend) {
     const int s = threadIdx.x;
     const int n = blockIdx.y * blockDim.y + threadIdx.y;
     if (n >= nblk) return;
@@ -274,16 +390,29 @@ __global__ void __launch_bounds__(256) gate_grad_local_kernel(
     const int rows = min(kGG, T - t0);
     const size_t stride = (size_t)H * M, total = (size_t)B * T * H * M;
     const size_t base = (((size_t)b * T + t0) * H + h) * M + s;
-    float x[kGG], dI[kGG], gt[kGG], ii[kGG];
-#pragma unroll
-    for (int i = 0; i < kGG; ++i) {
-        x[i] = (i < rows) ? u[base + (size_t)i * stride] : 0.f;
-        ii[i] = (i < rows) ? I[base + (size_t)i * stride] : 0.f;
-        gt[i] = (i < rows) ? gate[base + (size_t)i * stride] : 1.f;
-    }
+    float x[kGG], dI[kGG], gt[kGG];
     load_dI(dIk, nsk, dIv, nsv, base, stride, total, rows, dI);
+    if (pend.G != nullptr && pend.strong[bh] == 0) {
+        // the time-reversed value_side runs left their row factor exp(-G_i) to this kernel
+        float gg[kGG];
 #pragma unroll
-    for (int i = 0; i < kGG; ++i) x[i] -= ii[i] * dI[i];
+        for (int i = 0; i < kGG; ++i) gg[i] = (i < rows) ? pend.G[base + (size_t)i * stride] : 0.f;
+#pragma unroll
+        for (int i = 0; i < kGG; ++i) dI[i] *= __expf(-gg[i]);
+    }
+    {
+        float ii[kGG];
+#pragma unroll
+        for (int i = 0; i < kGG; ++i) ii[i] = (i < rows) ? I[base + (size_t)i * stride] : 0.f;
+#pragma unroll
+        for (int i = 0; i < kGG; ++i) x[i] = -ii[i] * dI[i];
+    }
+#pragma unroll
+    for (int i = 0; i < kGG; ++i) gt[i] = (i < rows) ? u[base + (size_t)i * stride] : 0.f;
+#pragma unroll
+    for (int i = 0; i < kGG; ++i) x[i] += gt[i];
+#pragma unroll
+    for (int i = 0; i < kGG; ++i) gt[i] = (i < rows) ? gate[base + (size_t)i * stride] : 1.f;
     float run = 0.f;
 #pragma unroll
     for (int i = kGG - 1; i >= 0; --i) {
@@ -334,18 +463,18 @@ cudaError_t launch_gate_grad(const float* u, const float* I, const float* dIk_pa
                              int gate_is_log, const float* dKT, const float* KT,
                              const float* dVT, const float* VT, int d_k, int d_v,
                              float* blk_tot, float* dgate, int B, int T, int H, int M,
-                             cudaStream_t st) {
+                             PendingDecay pend, cudaStream_t st) {
     const int nblk = gate_grad_blocks(T);
     dim3 block(M, 256 / M);
     dim3 grid(B * H, (nblk + block.y - 1) / block.y);
     if (M == 64) {
         gate_grad_local_kernel<64><<<grid, block, 0, st>>>(u, I, dIk_part, nsk, dIv_part, nsv, gate, gate_is_log,
-                                                           blk_tot, dgate, B, T, H, nblk);
+                                                           blk_tot, dgate, B, T, H, nblk, pend);
         gate_grad_scan_kernel<64><<<B * H, dim3(64, 16), 0, st>>>(blk_tot, dKT, KT, dVT, VT, d_k, d_v, nblk);
         gate_grad_carry_kernel<64><<<grid, block, 0, st>>>(gate, gate_is_log, blk_tot, dgate, T, H, nblk);
     } else {
         gate_grad_local_kernel<32><<<grid, block, 0, st>>>(u, I, dIk_part, nsk, dIv_part, nsv, gate, gate_is_log,
-                                                           blk_tot, dgate, B, T, H, nblk);
+                                                           blk_tot, dgate, B, T, H, nblk, pend);
         gate_grad_scan_kernel<32><<<B * H, dim3(32, 16), 0, st>>>(blk_tot, dKT, KT, dVT, VT, d_k, d_v, nblk);
         gate_grad_carry_kernel<32><<<grid, block, 0, st>>>(gate, gate_is_log, blk_tot, dgate, T, H, nblk);
     }
