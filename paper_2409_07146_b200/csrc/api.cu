@@ -200,7 +200,7 @@ gsa_status_t gsa_gate_cumsum(const gsa_params_t* params, const float* gate, floa
     const gsa_params_t& p = *params;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     GSA_LAUNCH("gate_cumsum", launch_gate_cumsum(gate, p.gate_kind == GSA_GATE_LOG_A, G, I, p.B, p.T,
-                                                 p.H, p.m, chunk_of(p), nullptr, 1, nullptr, st));
+                                                 p.H, p.m, chunk_of(p), nullptr, 1, nullptr, 0, st));
     return GSA_OK;
 }
 
@@ -219,12 +219,11 @@ gsa_status_t gsa_fwd(const gsa_params_t* params, const void* q, const void* k, c
     if (ws_bytes < w.bytes) return GSA_ERR_WORKSPACE;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const Slices s = slices(p);
-    const size_t rows = (size_t)p.B * p.T * p.H;
 
     const int nseg = segments_of(p);
     GSA_CUDA(cudaMemsetAsync(w.strong, 0, sizeof(int) * (size_t)p.B * p.H * nseg, st));
     GSA_LAUNCH("gate_cumsum", launch_gate_cumsum(gate, p.gate_kind == GSA_GATE_LOG_A, w.G, w.I, p.B, p.T,
-                                                 p.H, p.m, chunk_of(p), w.strong, nseg, w.Id, st));
+                                                 p.H, p.m, chunk_of(p), w.strong, nseg, w.Id, p.io == GSA_BF16, st));
     float* ok = ok_save ? ok_save : w.ok;
     // the pipelined kernels leave the row factor of the pass-1 sums to the softmax kernel
     const PendingDecay pend = use_tc(p) ? PendingDecay{w.G, w.strong, p.T, p.H, nseg} : PendingDecay{nullptr, nullptr, 1, 1, 1};
@@ -252,7 +251,8 @@ gsa_status_t gsa_fwd(const gsa_params_t* params, const void* q, const void* k, c
     // pass 1: o' = GLA(q, k, 1-a) with the decay on the slot (value) side
     ValueSideArgs a1{q, k, w.I, w.G, Kin, Kout, w.okpart, Bs, Ts, p.H, p.d_k, w.Id};
     GSA_LAUNCH("pass1_value_side", value_side(p, a1, 0, w.strong, st, dev_status));
-    GSA_LAUNCH("slot_softmax", launch_slot_softmax_fwd(w.okpart, s.k, p.scale, ok, w.p, rows, p.m, pend.G, w.Pd, pend, st));
+    GSA_LAUNCH("slot_softmax", launch_slot_softmax_fwd(w.okpart, s.k, p.scale, ok, w.p, p.B, p.T * p.H, p.m, pend.G, w.Pd,
+                                                       pend, st));
     // pass 2: o = GLA(softmax(o'), 1-a, v) with the decay on the slot (key) side
     KeySideArgs a2{w.p, w.I, w.G, v, Vin, Vout, o, Bs, Ts, p.H, p.d_v, w.Pd, w.Id};
     GSA_LAUNCH("pass2_key_side", key_side(p, a2, 0, w.strong, st, dev_status));
@@ -278,23 +278,23 @@ gsa_status_t gsa_bwd(const gsa_params_t* params, const void* q, const void* k, c
     if (ws_bytes < w.bytes) return GSA_ERR_WORKSPACE;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const Slices s = slices(p);
-    const size_t rows = (size_t)p.B * p.T * p.H;
 
     GSA_CUDA(cudaMemsetAsync(w.strong, 0, sizeof(int) * (size_t)p.B * p.H, st));
     GSA_LAUNCH("gate_cumsum", launch_gate_cumsum(gate, p.gate_kind == GSA_GATE_LOG_A, w.G, w.I, p.B, p.T,
-                                                 p.H, p.m, chunk_of(p), w.strong, 1, w.Id, st));
+                                                 p.H, p.m, chunk_of(p), w.strong, 1, w.Id, p.io == GSA_BF16, st));
     const float* ok = ok_saved;
     const PendingDecay pend = use_tc(p) ? PendingDecay{w.G, w.strong, p.T, p.H, 1} : PendingDecay{nullptr, nullptr, 1, 1, 1};
     if (ok == nullptr) {  // recompute pass 1 and its logits
         ValueSideArgs a1{q, k, w.I, w.G, K0, nullptr, w.okpart, p.B, p.T, p.H, p.d_k, w.Id};
         GSA_LAUNCH("pass1_value_side", value_side(p, a1, 0, w.strong, st, dev_status));
-        GSA_LAUNCH("slot_softmax", launch_slot_softmax_fwd(w.okpart, s.k, p.scale, w.ok, w.p, rows, p.m, pend.G, nullptr, pend, st));
+        GSA_LAUNCH("slot_softmax", launch_slot_softmax_fwd(w.okpart, s.k, p.scale, w.ok, w.p, p.B, p.T * p.H, p.m, pend.G,
+                                                           nullptr, pend, st));
         ok = w.ok;
     }
     // gradient w.r.t. the pass-2 queries p: the pass-1 form on (dO, v, 1-a); carries V~
     ValueSideArgs adp{dO, v, w.I, w.G, V0, dVT ? w.VT : nullptr, w.dppart, p.B, p.T, p.H, p.d_v, w.Id};
     GSA_LAUNCH("bwd_dp_value_side", value_side(p, adp, 0, w.strong, st, dev_status));
-    GSA_LAUNCH("slot_softmax_bwd", launch_slot_softmax_bwd(ok, w.dppart, s.v, p.scale, w.p, w.dz, w.u, rows, p.m, pend.G, w.Pd,
+    GSA_LAUNCH("slot_softmax_bwd", launch_slot_softmax_bwd(ok, w.dppart, s.v, p.scale, w.p, w.dz, w.u, p.B, p.T * p.H, p.m, pend.G, w.Pd,
                                                            w.Zd, pend, st));
     // dq: the pass-2 form on (dz, 1-a, k); carries K~
     KeySideArgs adq{w.dz, w.I, w.G, k, K0, dKT ? w.KT : nullptr, dq, p.B, p.T, p.H, p.d_k, w.Zd, w.Id};

@@ -769,6 +769,33 @@ constexpr size_t kSmemKeySide = 1024 + 13 * kPanelB + sizeof(Ctl);
 
 }  // namespace
 
+// The general kernel of a scan runs on a side stream of the calling host thread, beside the
+// pipelined kernel on the caller's stream (they write disjoint (batch, head) pairs): in the
+// usual case that no pair is flagged, its launch and the exit of its CTAs then cost the
+// caller's stream nothing.  fork: the side stream waits for what precedes on the caller's
+// stream; join: the caller's stream waits for the general kernel.
+struct SideLane {
+    cudaStream_t stream = nullptr;
+    cudaEvent_t fork = nullptr, join = nullptr;
+};
+cudaError_t side_lane(SideLane** out) {
+    constexpr int kMaxDevices = 64;
+    thread_local SideLane lanes[kMaxDevices];
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+    SideLane& l = lanes[dev];
+    if (l.stream == nullptr) {
+        e = cudaStreamCreateWithFlags(&l.stream, cudaStreamNonBlocking);
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&l.fork, cudaEventDisableTiming);
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&l.join, cudaEventDisableTiming);
+        if (e != cudaSuccess) return e;
+    }
+    *out = &l;
+    return cudaSuccess;
+}
+
 bool tc_supported(int d_k, int d_v, int M) {
     return M == kM && d_k % kDST == 0 && d_v % kDST == 0;
 }
@@ -789,14 +816,22 @@ cudaError_t launch_value_side_tc(const ValueSideArgs& a, int M, int reverse, con
 #define GSA_LAUNCH_VS(REVV, FLAGS)                                                                       \
     e = prepare(value_side_tc_kernel<REVV, true>, kSmemValueSide);                                       \
     if (e != cudaSuccess) return e;                                                                      \
-    value_side_tc_kernel<REVV, true><<<grid, kThreads, kSmemValueSide, st>>>(mq, mk, mw, mg, mo, a, FLAGS, dev_status)
+    value_side_tc_kernel<REVV, true><<<grid, kThreads, kSmemValueSide, side->stream>>>(mq, mk, mw, mg, mo, a, FLAGS, dev_status)
     // the pipelined kernel for the (batch, head) pairs whose chunks all decay moderately, this
     // general one for the others; each CTA of the kernel that is not its own returns at once
     if (a.wd == nullptr) return cudaErrorInvalidValue;
-    e = launch_value_side_lean(a, reverse, strong_flag, st, dev_status);
+    SideLane* side = nullptr;
+    e = side_lane(&side);
+    if (e == cudaSuccess) e = cudaEventRecord(side->fork, st);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(side->stream, side->fork, 0);
+    if (e == cudaSuccess) e = launch_value_side_lean(a, reverse, strong_flag, st, dev_status);
     if (e != cudaSuccess) return e;
     if (reverse) { GSA_LAUNCH_VS(true, strong_flag); }
     else { GSA_LAUNCH_VS(false, strong_flag); }
+    e = cudaGetLastError();
+    if (e == cudaSuccess) e = cudaEventRecord(side->join, side->stream);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(st, side->join, 0);
+    if (e != cudaSuccess) return e;
 #undef GSA_LAUNCH_VS
     return cudaGetLastError();
 }
@@ -815,12 +850,20 @@ cudaError_t launch_key_side_tc(const KeySideArgs& a, int M, int reverse, const i
 #define GSA_LAUNCH_KS(REVV, FLAGS)                                                                       \
     e = prepare(key_side_tc_kernel<REVV, true>, kSmemKeySide);                                           \
     if (e != cudaSuccess) return e;                                                                      \
-    key_side_tc_kernel<REVV, true><<<grid, kThreads, kSmemKeySide, st>>>(mv, muq, muk, mg, mo, a, FLAGS, dev_status)
+    key_side_tc_kernel<REVV, true><<<grid, kThreads, kSmemKeySide, side->stream>>>(mv, muq, muk, mg, mo, a, FLAGS, dev_status)
     if (a.uq_d == nullptr || a.uk_d == nullptr) return cudaErrorInvalidValue;
-    e = launch_key_side_lean(a, reverse, strong_flag, st, dev_status);
+    SideLane* side = nullptr;
+    e = side_lane(&side);
+    if (e == cudaSuccess) e = cudaEventRecord(side->fork, st);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(side->stream, side->fork, 0);
+    if (e == cudaSuccess) e = launch_key_side_lean(a, reverse, strong_flag, st, dev_status);
     if (e != cudaSuccess) return e;
     if (reverse) { GSA_LAUNCH_KS(true, strong_flag); }
     else { GSA_LAUNCH_KS(false, strong_flag); }
+    e = cudaGetLastError();
+    if (e == cudaSuccess) e = cudaEventRecord(side->join, side->stream);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(st, side->join, 0);
+    if (e != cudaSuccess) return e;
 #undef GSA_LAUNCH_KS
     return cudaGetLastError();
 }

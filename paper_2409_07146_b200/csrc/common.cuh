@@ -105,13 +105,12 @@ struct PendingDecay {
     const float* G;
     const int* strong;
     int T, H, nseg;
-    // row = (b * T + t) * H + h of a [B,T,H,M] tensor
-    __host__ __device__ bool pending(size_t row) const {
+    // row r = t * H + h of batch element b of a [B,T,H,M] tensor (32-bit arithmetic: T * H < 2^31)
+    __host__ __device__ bool pending(int b, int r) const {
         if (G == nullptr) return false;
-        const int h = (int)(row % H);
-        const size_t bt = row / H;
-        const int t = (int)(bt % T), b = (int)(bt / T);
-        return strong[((size_t)b * nseg + t / (T / nseg)) * H + h] == 0;
+        const int t = r / H, h = r - t * H;
+        const int seg = nseg == 1 ? 0 : t / (T / nseg);
+        return strong[(b * nseg + seg) * H + h] == 0;
     }
 };
 
@@ -119,10 +118,11 @@ struct PendingDecay {
 // strong_flag (nullable, [B*H] ints, zeroed by the caller): set to 1 for every (b,h) that has a
 // chunk whose total log-decay is below kFactorisedDecayMin (nseg > 1: [B*nseg*H], per segment).
 // decayed (nullable, bf16 [B,T,H,2M]): rows [high part | rounding residual] of I exp(-G), the
-// input-gate operand of the pipelined tensor-core kernels.
+// input-gate operand of the pipelined tensor-core kernels.  fast_log: take log a with the
+// hardware base-2 logarithm (absolute error 2^-21.4 for a in [0.5, 1], 3 ulp below), for bf16 io.
 cudaError_t launch_gate_cumsum(const float* gate, int gate_is_log, float* G, float* I,
                                int B, int T, int H, int M, int chunk, int* strong_flag, int nseg,
-                               void* decayed, cudaStream_t st);
+                               void* decayed, int fast_log, cudaStream_t st);
 // Segment-parallel scheduling (T cut into nseg segments run as independent sequences): per-segment
 // log-decay [B,nseg,H,M] from G, and the start memories [B,nseg,H,M,D] of every segment from the
 // end memories of the segments run from empty memories.
@@ -133,11 +133,12 @@ cudaError_t launch_segment_combine(const float* seg_logdecay, const float* local
                                    cudaStream_t st);
 // G, p_decayed / dz_decayed (nullable together; bf16 [rows, 2M]): rows [high | residual] of
 // p exp(G) and dz exp(G), operands of the pipelined tensor-core kernels.
+// (tensors [B, rows_per_batch = T*H, M])
 cudaError_t launch_slot_softmax_fwd(const float* part, int nslice, float scale, float* ok,
-                                    float* p, size_t rows, int M, const float* G, void* p_decayed,
+                                    float* p, int B, int rows_per_batch, int M, const float* G, void* p_decayed,
                                     PendingDecay pend, cudaStream_t st);
 cudaError_t launch_slot_softmax_bwd(const float* ok, const float* dp_part, int nslice,
-                                    float scale, float* p, float* dz, float* u, size_t rows,
+                                    float scale, float* p, float* dz, float* u, int B, int rows_per_batch,
                                     int M, const float* G, void* p_decayed, void* dz_decayed,
                                     PendingDecay pend, cudaStream_t st);
 cudaError_t launch_gate_grad(const float* u, const float* I, const float* dIk_part, int nsk,

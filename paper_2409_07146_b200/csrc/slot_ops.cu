@@ -34,7 +34,7 @@ __global__ void __launch_bounds__(M * 4) gate_cumsum_kernel(const float* __restr
                                                             float* __restrict__ G,
                                                             float* __restrict__ I, int T, int H,
                                                             int chunk, int* __restrict__ strong_flag, int nseg,
-                                                            __nv_bfloat16* __restrict__ decayed) {
+                                                            __nv_bfloat16* __restrict__ decayed, int fast_log) {
     __shared__ double group_sum[8][M];
     const int s = 2 * threadIdx.x, grp = threadIdx.y;          // blockDim.y = chunk / 16 <= 8
     const int n = blockIdx.y;
@@ -53,7 +53,7 @@ __global__ void __launch_bounds__(M * 4) gate_cumsum_kernel(const float* __restr
             g[i] = x;
             inps[i] = make_float2(-expm1f(x.x), -expm1f(x.y));
         } else {
-            g[i] = make_float2(logf(x.x), logf(x.y));
+            g[i] = fast_log ? make_float2(__logf(x.x), __logf(x.y)) : make_float2(logf(x.x), logf(x.y));
             inps[i] = make_float2(1.f - x.x, 1.f - x.y);
         }
         g[i].x = fmaxf(g[i].x, kLogGateMin);
@@ -62,13 +62,11 @@ __global__ void __launch_bounds__(M * 4) gate_cumsum_kernel(const float* __restr
     }
     // running sums in fp64 (a handful of adds per thread): G is then the correctly rounded
     // cumulative sum, which matters when strong decay makes |G| reach the hundreds
-    double run0[kCumRows], run1[kCumRows], acc0 = 0.0, acc1 = 0.0;
+    double acc0 = 0.0, acc1 = 0.0;
 #pragma unroll
     for (int i = 0; i < kCumRows; ++i) {
         acc0 += (i < rows) ? (double)g[i].x : 0.0;
         acc1 += (i < rows) ? (double)g[i].y : 0.0;
-        run0[i] = acc0;
-        run1[i] = acc1;
     }
     group_sum[grp][s] = acc0;
     group_sum[grp][s + 1] = acc1;
@@ -85,10 +83,13 @@ __global__ void __launch_bounds__(M * 4) gate_cumsum_kernel(const float* __restr
         const int seg = (int)(((long long)n * chunk) / (T / nseg));
         strong_flag[(b * nseg + seg) * H + h] = 1;
     }
+    // second pass over the same rows: the running sums continue from the groups before
 #pragma unroll
     for (int i = 0; i < kCumRows; ++i)
         if (i < rows) {
-            const float G0 = (float)(before0 + run0[i]), G1 = (float)(before1 + run1[i]);
+            before0 += (double)g[i].x;
+            before1 += (double)g[i].y;
+            const float G0 = (float)before0, G1 = (float)before1;
             *reinterpret_cast<float2*>(G + base + (size_t)i * stride) = make_float2(G0, G1);
             if (decayed != nullptr) {
                 // (meaningful for moderate decay only; pairs with a strong-decay chunk do not read it)
@@ -99,17 +100,18 @@ __global__ void __launch_bounds__(M * 4) gate_cumsum_kernel(const float* __restr
 }
 
 cudaError_t launch_gate_cumsum(const float* gate, int gate_is_log, float* G, float* I, int B,
-                               int T, int H, int M, int chunk, int* strong_flag, int nseg, void* decayed, cudaStream_t st) {
+                               int T, int H, int M, int chunk, int* strong_flag, int nseg, void* decayed, int fast_log,
+                               cudaStream_t st) {
     if (chunk % kCumRows != 0 || chunk / kCumRows > 8) return cudaErrorInvalidValue;
     const int nchunks = (T + chunk - 1) / chunk;
     dim3 block(M / 2, chunk / kCumRows);
     dim3 grid(B * H, nchunks);
     if (M == 64)
         gate_cumsum_kernel<64><<<grid, block, 0, st>>>(gate, gate_is_log, G, I, T, H, chunk, strong_flag, nseg < 1 ? 1 : nseg,
-                                                       static_cast<__nv_bfloat16*>(decayed));
+                                                       static_cast<__nv_bfloat16*>(decayed), fast_log);
     else
         gate_cumsum_kernel<32><<<grid, block, 0, st>>>(gate, gate_is_log, G, I, T, H, chunk, strong_flag, nseg < 1 ? 1 : nseg,
-                                                       static_cast<__nv_bfloat16*>(decayed));
+                                                       static_cast<__nv_bfloat16*>(decayed), fast_log);
     return cudaGetLastError();
 }
 
@@ -151,16 +153,17 @@ __global__ void __launch_bounds__(256) slot_softmax_fwd_kernel(const float* __re
                                                                int nslice, float scale,
                                                                float* __restrict__ ok,
                                                                float* __restrict__ p,
-                                                               size_t rows, const float* __restrict__ G,
+                                                               int rows_per_batch, const float* __restrict__ G,
                                                                __nv_bfloat16* __restrict__ p_decayed,
                                                                PendingDecay pend) {
     constexpr int R = M / 32;
-    const size_t row = (size_t)blockIdx.x * 8 + (threadIdx.x >> 5);
+    const int r_in_b = blockIdx.x * 8 + (threadIdx.x >> 5), b = blockIdx.y;
     const int lane = threadIdx.x & 31;
-    if (row >= rows) return;
-    const size_t total = rows * M;
+    if (r_in_b >= rows_per_batch) return;
+    const size_t row = (size_t)b * rows_per_batch + r_in_b;
+    const size_t total = (size_t)gridDim.y * rows_per_batch * M;
     const size_t idx = row * M + lane * R;
-    const bool pending = pend.pending(row);
+    const bool pending = pend.pending(b, r_in_b);
     float z[R], eg[R];
 #pragma unroll
     for (int r = 0; r < R; ++r) { z[r] = 0.f; eg[r] = 1.f; }
@@ -203,9 +206,10 @@ __global__ void __launch_bounds__(256) slot_softmax_fwd_kernel(const float* __re
 }
 
 cudaError_t launch_slot_softmax_fwd(const float* part, int nslice, float scale, float* ok,
-                                    float* p, size_t rows, int M, const float* G, void* p_decayed,
+                                    float* p, int B, int rows_per_batch, int M, const float* G, void* p_decayed,
                                     PendingDecay pend, cudaStream_t st) {
-    const unsigned grid = (unsigned)((rows + 7) / 8);
+    const dim3 grid((unsigned)((rows_per_batch + 7) / 8), (unsigned)B);
+    const int rows = rows_per_batch;
     if (M == 64)
         slot_softmax_fwd_kernel<64><<<grid, 256, 0, st>>>(part, nslice, scale, ok, p, rows, G,
                                                           static_cast<__nv_bfloat16*>(p_decayed), pend);
@@ -227,17 +231,18 @@ __global__ void __launch_bounds__(256) slot_softmax_bwd_kernel(const float* __re
                                                                float* __restrict__ p,
                                                                float* __restrict__ dz,
                                                                float* __restrict__ u,
-                                                               size_t rows, const float* __restrict__ G,
+                                                               int rows_per_batch, const float* __restrict__ G,
                                                                __nv_bfloat16* __restrict__ p_decayed,
                                                                __nv_bfloat16* __restrict__ dz_decayed,
                                                                PendingDecay pend) {
     constexpr int R = M / 32;
-    const size_t row = (size_t)blockIdx.x * 8 + (threadIdx.x >> 5);
+    const int r_in_b = blockIdx.x * 8 + (threadIdx.x >> 5), b = blockIdx.y;
     const int lane = threadIdx.x & 31;
-    if (row >= rows) return;
-    const size_t total = rows * M;
+    if (r_in_b >= rows_per_batch) return;
+    const size_t row = (size_t)b * rows_per_batch + r_in_b;
+    const size_t total = (size_t)gridDim.y * rows_per_batch * M;
     const size_t idx = row * M + lane * R;
-    const bool pending = pend.pending(row);
+    const bool pending = pend.pending(b, r_in_b);
     float z[R], dpv[R], eg[R];
     ld_vec<R>(ok + idx, z);
 #pragma unroll
@@ -292,10 +297,11 @@ __global__ void __launch_bounds__(256) slot_softmax_bwd_kernel(const float* __re
 }
 
 cudaError_t launch_slot_softmax_bwd(const float* ok, const float* dp_part, int nslice,
-                                    float scale, float* p, float* dz, float* u, size_t rows,
+                                    float scale, float* p, float* dz, float* u, int B, int rows_per_batch,
                                     int M, const float* G, void* p_decayed, void* dz_decayed,
                                     PendingDecay pend, cudaStream_t st) {
-    const unsigned grid = (unsigned)((rows + 7) / 8);
+    const dim3 grid((unsigned)((rows_per_batch + 7) / 8), (unsigned)B);
+    const int rows = rows_per_batch;
     if (M == 64)
         slot_softmax_bwd_kernel<64><<<grid, 256, 0, st>>>(ok, dp_part, nslice, scale, p, dz, u, rows, G,
                                                           static_cast<__nv_bfloat16*>(p_decayed),
@@ -318,25 +324,21 @@ cudaError_t launch_slot_softmax_bwd(const float* ok, const float* dp_part, int n
 constexpr int kGG = 16;   // rows per thread of the gate-gradient kernels
 
 // dI[i] = sum over the d_k and d_v slices of the input-gate gradient partial sums, for the
-// kGG rows of this thread; the rows of one slice are loaded together (16 loads in flight).
+// kGG rows x 2 slots of this thread; the rows of one slice are loaded together (16 loads of 8
+// bytes in flight).
 __device__ __forceinline__ void load_dI(const float* __restrict__ dIk, int nsk, const float* __restrict__ dIv,
                                         int nsv, size_t base, size_t stride, size_t total, int rows,
-                                        float (&dI)[kGG]) {
+                                        float2 (&dI)[kGG]) {
 #pragma unroll
-    for (int i = 0; i < kGG; ++i) dI[i] = 0.f;
-    for (int sl = 0; sl < nsk; ++sl) {
-        float t[kGG];
+    for (int i = 0; i < kGG; ++i) dI[i] = make_float2(0.f, 0.f);
+    for (int sl = 0; sl < nsk + nsv; ++sl) {
+        const float* src = sl < nsk ? dIk + (size_t)sl * total : dIv + (size_t)(sl - nsk) * total;
+        float2 t[kGG];
 #pragma unroll
-        for (int i = 0; i < kGG; ++i) t[i] = (i < rows) ? dIk[base + (size_t)i * stride + (size_t)sl * total] : 0.f;
+        for (int i = 0; i < kGG; ++i)
+            t[i] = (i < rows) ? *reinterpret_cast<const float2*>(src + base + (size_t)i * stride) : make_float2(0.f, 0.f);
 #pragma unroll
-        for (int i = 0; i < kGG; ++i) dI[i] += t[i];
-    }
-    for (int sl = 0; sl < nsv; ++sl) {
-        float t[kGG];
-#pragma unroll
-        for (int i = 0; i < kGG; ++i) t[i] = (i < rows) ? dIv[base + (size_t)i * stride + (size_t)sl * total] : 0.f;
-#pragma unroll
-        for (int i = 0; i < kGG; ++i) dI[i] += t[i];
+        for (int i = 0; i < kGG; ++i) { dI[i].x += t[i].x; dI[i].y += t[i].y; }
     }
 }
 
@@ -378,11 +380,11 @@ __global__ void __launch_bounds__(M * 16) gate_grad_scan_kernel(
 // at the block's end, turned into the gate gradient as if nothing followed the block, plus
 // the block total for the scan.  One read of every input.
 template <int M>
-__global__ void __launch_bounds__(256, 2) gate_grad_local_kernel(
+__global__ void __launch_bounds__(128) gate_grad_local_kernel(
     const float* __restrict__ u, const float* __restrict__ I, const float* __restrict__ dIk, int nsk,
     const float* __restrict__ dIv, int nsv, const float* __restrict__ gate, int gate_is_log,
     float* __restrict__ blk_tot, float* __restrict__ dgate, int B, int T, int H, int nblk, PendingDecay pend) {
-    const int s = threadIdx.x;
+    const int s = 2 * threadIdx.x;                       // this thread's two slots
     const int n = blockIdx.y * blockDim.y + threadIdx.y;
     if (n >= nblk) return;
     const int bh = blockIdx.x, b = bh / H, h = bh % H;
@@ -390,53 +392,55 @@ __global__ void __launch_bounds__(256, 2) gate_grad_local_kernel(
     const int rows = min(kGG, T - t0);
     const size_t stride = (size_t)H * M, total = (size_t)B * T * H * M;
     const size_t base = (((size_t)b * T + t0) * H + h) * M + s;
-    float x[kGG], dI[kGG], gt[kGG];
+    auto ld2 = [&](const float* p, int i, float fill) {
+        return (i < rows) ? *reinterpret_cast<const float2*>(p + base + (size_t)i * stride) : make_float2(fill, fill);
+    };
+    float2 x[kGG], dI[kGG], gt[kGG];
     load_dI(dIk, nsk, dIv, nsv, base, stride, total, rows, dI);
     if (pend.G != nullptr && pend.strong[bh] == 0) {
         // the time-reversed value_side runs left their row factor exp(-G_i) to this kernel
-        float gg[kGG];
 #pragma unroll
-        for (int i = 0; i < kGG; ++i) gg[i] = (i < rows) ? pend.G[base + (size_t)i * stride] : 0.f;
+        for (int i = 0; i < kGG; ++i) gt[i] = ld2(pend.G, i, 0.f);
 #pragma unroll
-        for (int i = 0; i < kGG; ++i) dI[i] *= __expf(-gg[i]);
-    }
-    {
-        float ii[kGG];
-#pragma unroll
-        for (int i = 0; i < kGG; ++i) ii[i] = (i < rows) ? I[base + (size_t)i * stride] : 0.f;
-#pragma unroll
-        for (int i = 0; i < kGG; ++i) x[i] = -ii[i] * dI[i];
+        for (int i = 0; i < kGG; ++i) { dI[i].x *= __expf(-gt[i].x); dI[i].y *= __expf(-gt[i].y); }
     }
 #pragma unroll
-    for (int i = 0; i < kGG; ++i) gt[i] = (i < rows) ? u[base + (size_t)i * stride] : 0.f;
+    for (int i = 0; i < kGG; ++i) gt[i] = ld2(I, i, 0.f);
 #pragma unroll
-    for (int i = 0; i < kGG; ++i) x[i] += gt[i];
+    for (int i = 0; i < kGG; ++i) x[i] = make_float2(-gt[i].x * dI[i].x, -gt[i].y * dI[i].y);
 #pragma unroll
-    for (int i = 0; i < kGG; ++i) gt[i] = (i < rows) ? gate[base + (size_t)i * stride] : 1.f;
-    float run = 0.f;
+    for (int i = 0; i < kGG; ++i) gt[i] = ld2(u, i, 0.f);
+#pragma unroll
+    for (int i = 0; i < kGG; ++i) { x[i].x += gt[i].x; x[i].y += gt[i].y; }
+#pragma unroll
+    for (int i = 0; i < kGG; ++i) gt[i] = ld2(gate, i, 1.f);
+    float run0 = 0.f, run1 = 0.f;
 #pragma unroll
     for (int i = kGG - 1; i >= 0; --i) {
-        run += x[i];
+        run0 += x[i].x;
+        run1 += x[i].y;
         if (i < rows) {
-            float out;
+            float2 out;
             if (gate_is_log) {
-                out = run - __expf(fmaxf(gt[i], kLogGateMin)) * dI[i];
+                out.x = run0 - __expf(fmaxf(gt[i].x, kLogGateMin)) * dI[i].x;
+                out.y = run1 - __expf(fmaxf(gt[i].y, kLogGateMin)) * dI[i].y;
             } else {
                 // a == 0 leaves no way back from d(log a) to da: only the input-gate part is kept
-                out = (gt[i] > 0.f) ? run / gt[i] - dI[i] : -dI[i];
+                out.x = (gt[i].x > 0.f) ? run0 / gt[i].x - dI[i].x : -dI[i].x;
+                out.y = (gt[i].y > 0.f) ? run1 / gt[i].y - dI[i].y : -dI[i].y;
             }
-            dgate[base + (size_t)i * stride] = out;
+            *reinterpret_cast<float2*>(dgate + base + (size_t)i * stride) = out;
         }
     }
-    blk_tot[((size_t)bh * nblk + n) * M + s] = run;
+    *reinterpret_cast<float2*>(blk_tot + ((size_t)bh * nblk + n) * M + s) = make_float2(run0, run1);
 }
 
 // Adds what follows the block: dgate += carry (log gate) or carry / a (linear gate).
 template <int M>
-__global__ void __launch_bounds__(256) gate_grad_carry_kernel(
+__global__ void __launch_bounds__(128) gate_grad_carry_kernel(
     const float* __restrict__ gate, int gate_is_log, const float* __restrict__ blk_carry,
     float* __restrict__ dgate, int T, int H, int nblk) {
-    const int s = threadIdx.x;
+    const int s = 2 * threadIdx.x;
     const int n = blockIdx.y * blockDim.y + threadIdx.y;
     if (n >= nblk) return;
     const int bh = blockIdx.x, b = bh / H, h = bh % H;
@@ -444,16 +448,22 @@ __global__ void __launch_bounds__(256) gate_grad_carry_kernel(
     const int rows = min(kGG, T - t0);
     const size_t stride = (size_t)H * M;
     const size_t base = (((size_t)b * T + t0) * H + h) * M + s;
-    const float carry = blk_carry[((size_t)bh * nblk + n) * M + s];
-    float d[kGG], gt[kGG];
+    const float2 carry = *reinterpret_cast<const float2*>(blk_carry + ((size_t)bh * nblk + n) * M + s);
+    float2 d[kGG], gt[kGG];
 #pragma unroll
     for (int i = 0; i < kGG; ++i) {
-        d[i] = (i < rows) ? dgate[base + (size_t)i * stride] : 0.f;
-        gt[i] = (i < rows && !gate_is_log) ? gate[base + (size_t)i * stride] : 1.f;
+        d[i] = (i < rows) ? *reinterpret_cast<const float2*>(dgate + base + (size_t)i * stride) : make_float2(0.f, 0.f);
+        gt[i] = (i < rows && !gate_is_log) ? *reinterpret_cast<const float2*>(gate + base + (size_t)i * stride)
+                                           : make_float2(1.f, 1.f);
     }
 #pragma unroll
     for (int i = 0; i < kGG; ++i)
-        if (i < rows) dgate[base + (size_t)i * stride] = d[i] + ((gate_is_log || gt[i] > 0.f) ? carry / gt[i] : 0.f);
+        if (i < rows) {
+            float2 out;
+            out.x = d[i].x + ((gate_is_log || gt[i].x > 0.f) ? carry.x / gt[i].x : 0.f);
+            out.y = d[i].y + ((gate_is_log || gt[i].y > 0.f) ? carry.y / gt[i].y : 0.f);
+            *reinterpret_cast<float2*>(dgate + base + (size_t)i * stride) = out;
+        }
 }
 
 int gate_grad_blocks(int T) { return (T + kGG - 1) / kGG; }
@@ -465,7 +475,7 @@ cudaError_t launch_gate_grad(const float* u, const float* I, const float* dIk_pa
                              float* blk_tot, float* dgate, int B, int T, int H, int M,
                              PendingDecay pend, cudaStream_t st) {
     const int nblk = gate_grad_blocks(T);
-    dim3 block(M, 256 / M);
+    dim3 block(M / 2, 256 / M);      // 128 threads: M/2 slot pairs x 16-row blocks
     dim3 grid(B * H, (nblk + block.y - 1) / block.y);
     if (M == 64) {
         gate_grad_local_kernel<64><<<grid, block, 0, st>>>(u, I, dIk_part, nsk, dIv_part, nsv, gate, gate_is_log,
