@@ -38,8 +38,11 @@ WORKLOAD = "train_1p3b"
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the tensor-core kernels on this
 # workload, from one `ncu --set full` capture (profiles/tc_chunk_kernels_train_1p3b_ncu_full.md).
 NCU_TRAFFIC = {
-    "pass1_value_side": 211809024, "bwd_dp_value_side": 211809024,
-    "pass2_key_side": 159327744, "bwd_dq_key_side": 159327744,
+    "pass1_value_side": 188711936, "bwd_dp_value_side": 187666432,
+    "bwd_dIv_value_side_rev": 190694912, "bwd_dIk_value_side_rev": 188507392,
+    "pass2_key_side": 106306560, "bwd_dq_key_side": 112874752,
+    "bwd_dv_key_side_rev": 108698624, "bwd_dk_key_side_rev": 112610560,
+    "gate_cumsum": 18426112, "slot_softmax": 102300416, "slot_softmax_bwd": 142108672,
 }
 
 
@@ -69,19 +72,21 @@ def kernel_algorithmic_bytes(label: str, w: W.Workload) -> int:
     R = w.B * w.T * w.H
     m = w.m
     nsk, nsv = w.d_k // 128, w.d_v // 128
+    # bytes per token-head row on the tensor-core path: fp32 [.., m] tensors are 4m, a decayed
+    # bf16 operand row [high | residual] is 4m too (the key_side kernels read its first half)
     table = {
-        "gate_cumsum": 12 * m,
-        "pass1_value_side": 2 * w.d_k * e + 8 * m + 4 * m * nsk,
-        "slot_softmax": 4 * m * nsk + 8 * m,
-        "pass2_key_side": 12 * m + 2 * w.d_v * e,
-        "bwd_dp_value_side": 2 * w.d_v * e + 8 * m + 4 * m * nsv,
-        "slot_softmax_bwd": 4 * m * (1 + nsv) + 12 * m,
-        "bwd_dq_key_side": 12 * m + 2 * w.d_k * e,
-        "bwd_dv_key_side_rev": 12 * m + 2 * w.d_v * e,
-        "bwd_dIv_value_side_rev": 2 * w.d_v * e + 8 * m + 4 * m * nsv,
-        "bwd_dk_key_side_rev": 12 * m + 2 * w.d_k * e,
-        "bwd_dIk_value_side_rev": 2 * w.d_k * e + 8 * m + 4 * m * nsk,
-        "gate_grad": 4 * m * (7 + nsk + nsv),   # one pass over u, I, gate, partials -> dgate; carry pass r/w
+        "gate_cumsum": 16 * m,                                       # gate -> G, I, I exp(-G)
+        "pass1_value_side": 2 * w.d_k * e + 4 * m + 4 * m * nsk,     # q, k, I exp(-G) -> slices of o'
+        "slot_softmax": 4 * m * nsk + 16 * m,                        # slices, G -> o', p, p exp(G)
+        "pass2_key_side": 2 * w.d_v * e + 4 * m,                     # v, two decayed half rows -> o
+        "bwd_dp_value_side": 2 * w.d_v * e + 4 * m + 4 * m * nsv,
+        "slot_softmax_bwd": 4 * m * nsv + 28 * m,                    # o', slices, G -> p, dz, u, p exp(G), dz exp(G)
+        "bwd_dq_key_side": 2 * w.d_k * e + 4 * m,
+        "bwd_dv_key_side_rev": 2 * w.d_v * e + 4 * m,
+        "bwd_dIv_value_side_rev": 2 * w.d_v * e + 4 * m + 4 * m * nsv,
+        "bwd_dk_key_side_rev": 2 * w.d_k * e + 4 * m,
+        "bwd_dIk_value_side_rev": 2 * w.d_k * e + 4 * m + 4 * m * nsk,
+        "gate_grad": 4 * m * (8 + nsk + nsv),   # u, I, gate, G, partials -> dgate; carry pass reads gate, r/w dgate
     }
     return R * table[label]
 
