@@ -148,13 +148,12 @@ value_side_lean_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_co
     if (strong_flag[blockIdx.x] != 0) return;       // the general kernel takes this (batch, head)
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
-    unsigned char* sXq = smem;                       // 2 panels                                  (32 KB)
-    unsigned char* sXk = sXq + 2 * kPanelB;          // 2 panels                                  (32 KB)
-    unsigned char* sWd = sXk + 2 * kPanelB;          // decayed weights, MN-major B [128][hi 64 | lo 64], 2 stages (64 KB)
-    unsigned char* sPm = sWd + 4 * kPanelB;          // masked P, K-major A, 2 panels             (32 KB)
+    unsigned char* sX = smem;                        // xq, xk tiles: 2 stages x (2 + 2 panels)  (128 KB)
+    unsigned char* sWd = sX + 8 * kPanelB;           // decayed weights, MN-major B [128][hi 64 | lo 64] (32 KB)
+    unsigned char* sPm = sWd + 2 * kPanelB;          // masked P, K-major A, 2 panels             (32 KB)
+    unsigned char* sOut = sPm;                       //   ... shared with the output rows fp32, 2 panels of 32 slots
     unsigned char* sSb = sPm + 2 * kPanelB;          // state copy, MN-major B [128][64]          (16 KB)
-    unsigned char* sOut = sSb + kPanelB;             // output rows fp32, 2 panels of 32 slots    (32 KB)
-    LeanCtl* ctl = reinterpret_cast<LeanCtl*>(sOut + 2 * kPanelB);
+    LeanCtl* ctl = reinterpret_cast<LeanCtl*>(sSb + kPanelB);
 
     const int tid = threadIdx.x, warp = tid >> 5, wq = warp & 3, half = (tid >> 7) & 1, row = tid & 127;
     const int sb = kHS * half;          // this thread's first slot
@@ -169,18 +168,20 @@ value_side_lean_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_co
     if (tid == kCopyThread) {
         // =============================== copy lane: every tile load and store
         auto load_x = [&](int n) {
-            const int t = chunk_t0(n);
-            mbar_expect_tx(&ctl->bar_x, 4 * kPanelB);
-            tma_load_4d(sXq, &mapQ, &ctl->bar_x, d0, h, t, b);
-            tma_load_4d(sXq + kPanelB, &mapQ, &ctl->bar_x, d0 + 64, h, t, b);
-            tma_load_4d(sXk, &mapK, &ctl->bar_x, d0, h, t, b);
-            tma_load_4d(sXk + kPanelB, &mapK, &ctl->bar_x, d0 + 64, h, t, b);
+            const int t = chunk_t0(n), st = n & 1;
+            unsigned char* sXq = sX + 4 * st * kPanelB;
+            unsigned char* sXk = sXq + 2 * kPanelB;
+            mbar_expect_tx(&ctl->bar_x2[st], 4 * kPanelB);
+            tma_load_4d(sXq, &mapQ, &ctl->bar_x2[st], d0, h, t, b);
+            tma_load_4d(sXq + kPanelB, &mapQ, &ctl->bar_x2[st], d0 + 64, h, t, b);
+            tma_load_4d(sXk, &mapK, &ctl->bar_x2[st], d0, h, t, b);
+            tma_load_4d(sXk + kPanelB, &mapK, &ctl->bar_x2[st], d0 + 64, h, t, b);
         };
         auto load_w = [&](int n) {
-            const int t = chunk_t0(n), st = n & 1;
-            mbar_expect_tx(&ctl->bar_w[st], 2 * kPanelB);
-            tma_load_4d(sWd + (2 * st) * kPanelB, &mapWd, &ctl->bar_w[st], 0, h, t, b);
-            tma_load_4d(sWd + (2 * st + 1) * kPanelB, &mapWd, &ctl->bar_w[st], 64, h, t, b);
+            const int t = chunk_t0(n);
+            mbar_expect_tx(&ctl->bar_w[0], 2 * kPanelB);
+            tma_load_4d(sWd, &mapWd, &ctl->bar_w[0], 0, h, t, b);
+            tma_load_4d(sWd + kPanelB, &mapWd, &ctl->bar_w[0], 64, h, t, b);
         };
         auto store_out = [&](int n) {
             const int t = chunk_t0(n);
@@ -191,58 +192,54 @@ value_side_lean_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_co
         prefetch_tmap(&mapQ); prefetch_tmap(&mapK); prefetch_tmap(&mapWd); prefetch_tmap(&mapO);
         load_x(0);
         load_w(0);
-        if (nchunks > 1) load_w(1);
+        if (nchunks > 1) load_x(1);
         for (int n = 0; n < nchunks && !ctl->abort; ++n) {
-            // the d-sized tiles are consumed once the state products are done: request the next chunk's
+            // the d-sized tiles of chunk n are consumed once its state products are done: their
+            // buffer takes the tiles of chunk n+2
             LEAN_WAIT(&ctl->bar_free1, n & 1);
-            if (n + 1 < nchunks) load_x(n + 1);
-            // output rows of the previous chunk
-            if (n >= 1) {
-                LEAN_WAIT(&ctl->bar_out, (n - 1) & 1);
-                if (ctl->abort) break;
-                store_out(n - 1);
-                bulk_wait_read();               // the staged rows have left: the buffer may be rewritten
-                mbar_arrive(&ctl->bar_free);
-            }
-            // the weights of chunk n make room for those of chunk n+2
+            if (n + 2 < nchunks) load_x(n + 2);
+            // the weights are consumed once the intra-chunk product is done
             LEAN_WAIT(&ctl->bar_free2, n & 1);
-            if (n + 2 < nchunks) load_w(n + 2);
+            if (n + 1 < nchunks) load_w(n + 1);
+            // output rows, staged over the masked P
+            LEAN_WAIT(&ctl->bar_out, n & 1);
+            if (ctl->abort) break;
+            store_out(n);
+            bulk_wait_read();               // the staged rows have left: the buffer may be rewritten
+            mbar_arrive(&ctl->bar_free);
         }
-        if (!ctl->abort) {
-            LEAN_WAIT(&ctl->bar_out, (nchunks - 1) & 1);
-            if (!ctl->abort) store_out(nchunks - 1);
-        }
-        bulk_wait_read();      // staged output rows must have left before shared memory goes away
     } else if (tid == kMmaThread) {
         // =============================== MMA lane
         constexpr uint32_t idescP = make_idesc(128, 128, false, false);    // xq xk^T
         constexpr uint32_t idescO = make_idesc(128, kM, false, true);      // xq x state copy (MN-major B)
         constexpr uint32_t idescU = make_idesc(128, 2 * kM, true, true);   // xk^T (MN-major A) x [W_hi | W_lo]
         constexpr uint32_t idescI = make_idesc(128, 2 * kM, false, true);  // Pm x [W_hi | W_lo]
-        const uint64_t dQk = desc_kmajor(smem_u32(sXq), 0), dKk = desc_kmajor(smem_u32(sXk), 0);
-        const uint64_t dKm = desc_mnmajor(smem_u32(sXk), 0, kPanelB);
+        const uint64_t dW = desc_mnmajor(smem_u32(sWd), 0, kPanelB);
         const uint64_t dS = desc_mnmajor(smem_u32(sSb), 0, kPanelB);
         const uint64_t dP = desc_kmajor(smem_u32(sPm), 0);
         auto kmaj = [](int kk) { return (uint32_t)((kk >> 2) * kPanelB + (kk & 3) * 32); };
         auto mnmaj = [](int kk) { return (uint32_t)(kk * 2048); };
-        auto issue_p = [&]() {
+        auto issue_p = [&](int n) {
+            const uint32_t xq = smem_u32(sX + 4 * (n & 1) * kPanelB);
+            const uint64_t dQk = desc_kmajor(xq, 0), dKk = desc_kmajor(xq + 2 * kPanelB, 0);
 #pragma unroll
             for (int kk = 0; kk < kDST / 16; ++kk)
                 mma_bf16(tmem + kLvP, desc_advance(dQk, kmaj(kk)), desc_advance(dKk, kmaj(kk)), idescP, kk > 0);
             mma_commit(&ctl->bar_p);
         };
-        LEAN_WAIT(&ctl->bar_x, 0);
+        LEAN_WAIT(&ctl->bar_x2[0], 0);
         tc_fence_after_sync();
-        issue_p();
+        issue_p(0);
         PROF_DECL
         for (int n = 0; n < nchunks && !ctl->abort; ++n) {
             const int it = n;
             (void)it;
-            const uint64_t dW = desc_mnmajor(smem_u32(sWd + 2 * (n & 1) * kPanelB), 0, kPanelB);
+            const uint32_t xq = smem_u32(sX + 4 * (n & 1) * kPanelB);
+            const uint64_t dQk = desc_kmajor(xq, 0), dKm = desc_mnmajor(xq + 2 * kPanelB, 0, kPanelB);
             PROF_MARK();
             // state products of chunk n: the state copy was written at the end of chunk n-1 (which also
             // says that the accumulators they overwrite have been read)
-            LEAN_WAIT(&ctl->bar_w[n & 1], (n >> 1) & 1);
+            LEAN_WAIT(&ctl->bar_w[0], n & 1);
             PROF_MARK();
             LEAN_WAIT(&ctl->bar_sb, n & 1);
             tc_fence_after_sync();
@@ -269,10 +266,10 @@ value_side_lean_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_co
             PROF_MARK();
             // the P accumulator is free: the next chunk's P queues right behind
             if (n + 1 < nchunks) {
-                LEAN_WAIT(&ctl->bar_x, (n + 1) & 1);
+                LEAN_WAIT(&ctl->bar_x2[(n + 1) & 1], ((n + 1) >> 1) & 1);
                 tc_fence_after_sync();
                 PROF_MARK();
-                issue_p();
+                issue_p(n + 1);
             }
             PROF_MARK();
             PROF_DUMP("value_side lean mma");
@@ -311,6 +308,7 @@ value_side_lean_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_co
             // ---- masked P rows (the barrier inside also publishes egc)
             LEAN_WAIT(&ctl->bar_p, n & 1);
             tc_fence_after_sync();
+            if (n >= 1) LEAN_WAIT(&ctl->bar_free, (n - 1) & 1);     // the staged rows of chunk n-1 have left
             PROF_MARK();
             store_masked_row<REV, false>(tmem, wq, row, half, sPm, sPm);
             publish(&ctl->bar_pm, tid);
@@ -343,7 +341,6 @@ value_side_lean_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_co
             // staged for one tiled store, clipped at the sequence end
             LEAN_WAIT(&ctl->bar_mma2, n & 1);
             tc_fence_after_sync();
-            if (n >= 1) LEAN_WAIT(&ctl->bar_free, (n - 1) & 1);
             PROF_MARK();
             {
                 float vo[kHS], vi[kHS];
@@ -388,13 +385,14 @@ key_side_lean_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_cons
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
     unsigned char* sXv = smem;                       // xv tile, 2 stages of 2 panels              (64 KB)
-    unsigned char* sQt = sXv + 4 * kPanelB;          // decayed uq, K-major A [128][64]            (16 KB)
-    unsigned char* sKt = sQt + kPanelB;              // decayed uk, K-major / MN-major B [128][64] (16 KB)
-    unsigned char* sAm = sKt + kPanelB;              // masked A, K-major A, 2 panels              (32 KB)
-    unsigned char* sAl = sAm + 2 * kPanelB;          // its rounding residual, 2 panels            (32 KB)
+                                                     //   ... a stage also holds the chunk's output rows once
+                                                     //   its tile is consumed
+    unsigned char* sQK = sXv + 4 * kPanelB;          // decayed uq (K-major A [128][64]) and uk (K-major /
+                                                     //   MN-major B [128][64]), 2 stages of 1 + 1 panels (64 KB)
+    unsigned char* sAm = sQK + 4 * kPanelB;          // masked A, K-major A, 2 panels              (32 KB)
+    unsigned char* sAl = sAm + 2 * kPanelB;          // rounding residual of the masked A, 2 panels (32 KB)
     unsigned char* sSb = sAl + 2 * kPanelB;          // state copy, K-major B [128 (channel)][64]  (16 KB)
-    unsigned char* sOut = sSb + kPanelB;             // output rows, 2 panels                      (32 KB)
-    LeanCtl* ctl = reinterpret_cast<LeanCtl*>(sOut + 2 * kPanelB);
+    LeanCtl* ctl = reinterpret_cast<LeanCtl*>(sSb + kPanelB);
 
     const int tid = threadIdx.x, warp = tid >> 5, wq = warp & 3, half = (tid >> 7) & 1, row = tid & 127;
     const int sb = kHS * half;          // this thread's first slot
@@ -415,13 +413,14 @@ key_side_lean_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_cons
             tma_load_4d(sXv + (2 * st + 1) * kPanelB, &mapV, &ctl->bar_x2[st], d0 + 64, h, t, b);
         };
         auto load_qk = [&](int n) {
-            const int t = chunk_t0(n);
-            mbar_expect_tx(&ctl->bar_w[0], 2 * kPanelB);
-            tma_load_4d(sQt, &mapUq, &ctl->bar_w[0], 0, h, t, b);
-            tma_load_4d(sKt, &mapUk, &ctl->bar_w[0], 0, h, t, b);
+            const int t = chunk_t0(n), st = n & 1;
+            mbar_expect_tx(&ctl->bar_w[st], 2 * kPanelB);
+            tma_load_4d(sQK + (2 * st) * kPanelB, &mapUq, &ctl->bar_w[st], 0, h, t, b);
+            tma_load_4d(sQK + (2 * st + 1) * kPanelB, &mapUk, &ctl->bar_w[st], 0, h, t, b);
         };
         auto store_out = [&](int n) {
             const int t = chunk_t0(n);
+            const unsigned char* sOut = sXv + 2 * (n & 1) * kPanelB;
             tma_store_4d(&mapO, sOut, d0, h, t, b);
             tma_store_4d(&mapO, sOut + kPanelB, d0 + 64, h, t, b);
             bulk_commit();
@@ -429,28 +428,24 @@ key_side_lean_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_cons
         prefetch_tmap(&mapV); prefetch_tmap(&mapUq); prefetch_tmap(&mapUk); prefetch_tmap(&mapO);
         load_qk(0);
         load_v(0);
-        if (nchunks > 1) load_v(1);
+        if (nchunks > 1) {
+            load_qk(1);
+            load_v(1);
+        }
         for (int n = 0; n < nchunks && !ctl->abort; ++n) {
-            // the decayed uq / uk rows are consumed once the state products are done: request the next chunk's
+            // the decayed uq / uk rows of chunk n are consumed once its state products are done: their
+            // buffer takes the rows of chunk n+2
             LEAN_WAIT(&ctl->bar_free1, n & 1);
-            if (n + 1 < nchunks) load_qk(n + 1);
-            // output rows of the previous chunk
-            if (n >= 1) {
-                LEAN_WAIT(&ctl->bar_out, (n - 1) & 1);
-                if (ctl->abort) break;
-                store_out(n - 1);
-                bulk_wait_read();               // the staged rows have left: the buffer may be rewritten
-                mbar_arrive(&ctl->bar_free);
-            }
-            // the xv tile of chunk n makes room for that of chunk n+2
-            LEAN_WAIT(&ctl->bar_free2, n & 1);
+            if (n + 2 < nchunks) load_qk(n + 2);
+            // the xv tile is consumed once the intra-chunk product is done; the compute threads then
+            // stage the output rows in its place, and when those have left the buffer takes the tile
+            // of chunk n+2
+            LEAN_WAIT(&ctl->bar_out, n & 1);
+            if (ctl->abort) break;
+            store_out(n);
+            bulk_wait_read();
             if (n + 2 < nchunks) load_v(n + 2);
         }
-        if (!ctl->abort) {
-            LEAN_WAIT(&ctl->bar_out, (nchunks - 1) & 1);
-            if (!ctl->abort) store_out(nchunks - 1);
-        }
-        bulk_wait_read();      // staged output rows must have left before shared memory goes away
     } else if (tid == kMmaThread) {
         // =============================== MMA lane
         constexpr uint32_t idescA = make_idesc(128, 128, false, false);   // Q~ K~^T
@@ -459,11 +454,11 @@ key_side_lean_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_cons
         constexpr uint32_t idescV = make_idesc(128, kDST, false, true);   // A x xv (MN-major B)
         const uint64_t dS = desc_kmajor(smem_u32(sSb), 0);
         const uint64_t dA = desc_kmajor(smem_u32(sAm), 0), dAl = desc_kmajor(smem_u32(sAl), 0);
-        const uint64_t dQt = desc_kmajor(smem_u32(sQt), 0), dKt = desc_kmajor(smem_u32(sKt), 0);
-        const uint64_t dKtm = desc_mnmajor(smem_u32(sKt), 0, kPanelB);   // the decayed uk read MN-major
         auto kmaj = [](int kk) { return (uint32_t)((kk >> 2) * kPanelB + (kk & 3) * 32); };
         auto mnmaj = [](int kk) { return (uint32_t)(kk * 2048); };
-        auto issue_a = [&]() {
+        auto issue_a = [&](int n) {
+            const uint32_t qk = smem_u32(sQK + 2 * (n & 1) * kPanelB);
+            const uint64_t dQt = desc_kmajor(qk, 0), dKt = desc_kmajor(qk + kPanelB, 0);
 #pragma unroll
             for (int kk = 0; kk < kM / 16; ++kk)
                 mma_bf16(tmem + kLkA, desc_advance(dQt, kmaj(kk)), desc_advance(dKt, kmaj(kk)), idescA, kk > 0);
@@ -471,13 +466,16 @@ key_side_lean_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_cons
         };
         LEAN_WAIT(&ctl->bar_w[0], 0);
         tc_fence_after_sync();
-        issue_a();
+        issue_a(0);
         PROF_DECL
         for (int n = 0; n < nchunks && !ctl->abort; ++n) {
             const int it = n;
             (void)it;
             const uint64_t dV = desc_mnmajor(smem_u32(sXv + 2 * (n & 1) * kPanelB), 0, kPanelB);
             const uint32_t accO = tmem + kLkO + 128 * (n & 1);
+            const uint32_t qk = smem_u32(sQK + 2 * (n & 1) * kPanelB);
+            const uint64_t dQt = desc_kmajor(qk, 0);
+            const uint64_t dKtm = desc_mnmajor(qk + kPanelB, 0, kPanelB);   // the decayed uk read MN-major
             PROF_MARK();
             // state products of chunk n: the state copy was written at the end of chunk n-1 (which also
             // says that the accumulators they overwrite have been read)
@@ -510,10 +508,10 @@ key_side_lean_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_cons
             PROF_MARK();
             // the A accumulator is free: the next chunk's A queues right behind
             if (n + 1 < nchunks) {
-                LEAN_WAIT(&ctl->bar_w[0], (n + 1) & 1);
+                LEAN_WAIT(&ctl->bar_w[(n + 1) & 1], ((n + 1) >> 1) & 1);
                 tc_fence_after_sync();
                 PROF_MARK();
-                issue_a();
+                issue_a(n + 1);
             }
             PROF_MARK();
             PROF_DUMP("key_side lean mma");
@@ -577,7 +575,6 @@ key_side_lean_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_cons
             // ---- output rows -> bf16, staged for the tiled store (clipped at the sequence end)
             LEAN_WAIT(&ctl->bar_mma2, n & 1);
             tc_fence_after_sync();
-            if (n >= 1) LEAN_WAIT(&ctl->bar_free, (n - 1) & 1);
 #pragma unroll 1
             for (int c0 = 0; c0 < 64; c0 += 32) {
                 float v[32];
@@ -586,7 +583,7 @@ key_side_lean_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_cons
                 for (int c = 0; c < 4; ++c) {
                     const float x[8] = {v[8 * c], v[8 * c + 1], v[8 * c + 2], v[8 * c + 3],
                                         v[8 * c + 4], v[8 * c + 5], v[8 * c + 6], v[8 * c + 7]};
-                    store_chunk(sOut + half * kPanelB, row, (c0 >> 3) + c, x);
+                    store_chunk(sXv + (2 * (n & 1) + half) * kPanelB, row, (c0 >> 3) + c, x);
                 }
             }
             if (publish_and_vote(&ctl->bar_out, tid, ctl->abort != 0)) break;
