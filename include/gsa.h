@@ -173,6 +173,7 @@ GSA_API gsa_status_t gsa_fwd_noalloc(const gsa_params_t* params, const void* q, 
  * row-major bf16 device matrices X, Y into D (fp32, row-major):
  *   mode 0: D[128x128] = X Y^T        mode 1: D[128x128] = X Y
  *   mode 2: D[128x64]  = X^T Y[:64]^T mode 3: D[128x64]  = X Y[:, :64]
+ *   mode 4: D[128x128] = X Y^T        mode 5: D[128x128] = X Y      (A operand in tensor memory)
  * dev_status (nullable) receives GSA_ERR_TIMEOUT if a bounded wait expired.
  */
 GSA_API gsa_status_t gsa_tc_selftest(int32_t mode, const void* X, const void* Y, float* D,

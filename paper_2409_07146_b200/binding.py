@@ -219,7 +219,7 @@ def gsa_decode_step(p: Params, q, k, v, gate, Kstate, Vstate, o=None):
 
 def gsa_tc_selftest(mode: int, X, Y, dev_status=None):
     """Tensor-core building-block self-test: X, Y 128 x 128 bf16; returns D (fp32)."""
-    n = 128 if mode <= 1 else 64
+    n = 128 if (mode <= 1 or mode >= 4) else 64
     D = torch.zeros(128, n, dtype=torch.float32, device=X.device)
     _check(load_library().gsa_tc_selftest(
         mode, _ptr(X, torch.bfloat16, (128, 128), "X"), _ptr(Y, torch.bfloat16, (128, 128), "Y"),

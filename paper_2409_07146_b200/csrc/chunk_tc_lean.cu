@@ -149,10 +149,10 @@ value_side_lean_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_co
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
     unsigned char* sX = smem;                        // xq, xk tiles: 2 stages x (2 + 2 panels)  (128 KB)
-    unsigned char* sWd = sX + 8 * kPanelB;           // decayed weights, MN-major B [128][hi 64 | lo 64] (32 KB)
-    unsigned char* sPm = sWd + 2 * kPanelB;          // masked P, K-major A, 2 panels             (32 KB)
-    unsigned char* sOut = sPm;                       //   ... shared with the output rows fp32, 2 panels of 32 slots
-    unsigned char* sSb = sPm + 2 * kPanelB;          // state copy, MN-major B [128][64]          (16 KB)
+    unsigned char* sWd = sX + 8 * kPanelB;           // decayed weights, MN-major B [128][hi 64 | lo 64], 2 stages (64 KB)
+                                                     //   ... a stage also holds the chunk's output rows (fp32, 2
+                                                     //   panels of 32 slots) once its weights are consumed
+    unsigned char* sSb = sWd + 4 * kPanelB;          // state copy, MN-major B [128][64]          (16 KB)
     LeanCtl* ctl = reinterpret_cast<LeanCtl*>(sSb + kPanelB);
 
     const int tid = threadIdx.x, warp = tid >> 5, wq = warp & 3, half = (tid >> 7) & 1, row = tid & 127;
@@ -178,13 +178,14 @@ value_side_lean_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_co
             tma_load_4d(sXk + kPanelB, &mapK, &ctl->bar_x2[st], d0 + 64, h, t, b);
         };
         auto load_w = [&](int n) {
-            const int t = chunk_t0(n);
-            mbar_expect_tx(&ctl->bar_w[0], 2 * kPanelB);
-            tma_load_4d(sWd, &mapWd, &ctl->bar_w[0], 0, h, t, b);
-            tma_load_4d(sWd + kPanelB, &mapWd, &ctl->bar_w[0], 64, h, t, b);
+            const int t = chunk_t0(n), st = n & 1;
+            mbar_expect_tx(&ctl->bar_w[st], 2 * kPanelB);
+            tma_load_4d(sWd + (2 * st) * kPanelB, &mapWd, &ctl->bar_w[st], 0, h, t, b);
+            tma_load_4d(sWd + (2 * st + 1) * kPanelB, &mapWd, &ctl->bar_w[st], 64, h, t, b);
         };
         auto store_out = [&](int n) {
             const int t = chunk_t0(n);
+            const unsigned char* sOut = sWd + 2 * (n & 1) * kPanelB;
             tma_store_5d(&mapO, sOut, 0, h, t, b, slice);
             tma_store_5d(&mapO, sOut + kPanelB, 32, h, t, b, slice);
             bulk_commit();
@@ -192,31 +193,31 @@ value_side_lean_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_co
         prefetch_tmap(&mapQ); prefetch_tmap(&mapK); prefetch_tmap(&mapWd); prefetch_tmap(&mapO);
         load_x(0);
         load_w(0);
-        if (nchunks > 1) load_x(1);
+        if (nchunks > 1) {
+            load_x(1);
+            load_w(1);
+        }
         for (int n = 0; n < nchunks && !ctl->abort; ++n) {
             // the d-sized tiles of chunk n are consumed once its state products are done: their
             // buffer takes the tiles of chunk n+2
             LEAN_WAIT(&ctl->bar_free1, n & 1);
             if (n + 2 < nchunks) load_x(n + 2);
-            // the weights are consumed once the intra-chunk product is done
-            LEAN_WAIT(&ctl->bar_free2, n & 1);
-            if (n + 1 < nchunks) load_w(n + 1);
-            // output rows, staged over the masked P
+            // the weights are consumed once the intra-chunk product is done; the compute threads then
+            // stage the output rows in their place, and when those have left the buffer takes the
+            // weights of chunk n+2
             LEAN_WAIT(&ctl->bar_out, n & 1);
             if (ctl->abort) break;
             store_out(n);
-            bulk_wait_read();               // the staged rows have left: the buffer may be rewritten
-            mbar_arrive(&ctl->bar_free);
+            bulk_wait_read();
+            if (n + 2 < nchunks) load_w(n + 2);
         }
     } else if (tid == kMmaThread) {
         // =============================== MMA lane
         constexpr uint32_t idescP = make_idesc(128, 128, false, false);    // xq xk^T
         constexpr uint32_t idescO = make_idesc(128, kM, false, true);      // xq x state copy (MN-major B)
         constexpr uint32_t idescU = make_idesc(128, 2 * kM, true, true);   // xk^T (MN-major A) x [W_hi | W_lo]
-        constexpr uint32_t idescI = make_idesc(128, 2 * kM, false, true);  // Pm x [W_hi | W_lo]
-        const uint64_t dW = desc_mnmajor(smem_u32(sWd), 0, kPanelB);
+        constexpr uint32_t idescI = make_idesc(128, 2 * kM, false, true);  // masked P (tensor memory) x [W_hi | W_lo]
         const uint64_t dS = desc_mnmajor(smem_u32(sSb), 0, kPanelB);
-        const uint64_t dP = desc_kmajor(smem_u32(sPm), 0);
         auto kmaj = [](int kk) { return (uint32_t)((kk >> 2) * kPanelB + (kk & 3) * 32); };
         auto mnmaj = [](int kk) { return (uint32_t)(kk * 2048); };
         auto issue_p = [&](int n) {
@@ -236,10 +237,11 @@ value_side_lean_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_co
             (void)it;
             const uint32_t xq = smem_u32(sX + 4 * (n & 1) * kPanelB);
             const uint64_t dQk = desc_kmajor(xq, 0), dKm = desc_mnmajor(xq + 2 * kPanelB, 0, kPanelB);
+            const uint64_t dW = desc_mnmajor(smem_u32(sWd + 2 * (n & 1) * kPanelB), 0, kPanelB);
             PROF_MARK();
             // state products of chunk n: the state copy was written at the end of chunk n-1 (which also
             // says that the accumulators they overwrite have been read)
-            LEAN_WAIT(&ctl->bar_w[0], n & 1);
+            LEAN_WAIT(&ctl->bar_w[n & 1], (n >> 1) & 1);
             PROF_MARK();
             LEAN_WAIT(&ctl->bar_sb, n & 1);
             tc_fence_after_sync();
@@ -254,13 +256,14 @@ value_side_lean_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_co
             mma_commit(&ctl->bar_mma1);
             mma_commit(&ctl->bar_free1);
             PROF_MARK();
-            // intra-chunk product once the masked P rows are there
+            // intra-chunk product once the masked P rows are there (bf16, in place in tensor memory)
             LEAN_WAIT(&ctl->bar_pm, n & 1);
             tc_fence_after_sync();
             PROF_MARK();
 #pragma unroll
             for (int kk = 0; kk < kCT / 16; ++kk)
-                mma_bf16(tmem + kLvI, desc_advance(dP, kmaj(kk)), desc_advance(dW, mnmaj(kk)), idescI, kk > 0);
+                mma_bf16_ta(tmem + kLvI, tmem + kLvP + 64 * (kk >> 2) + 8 * (kk & 3), desc_advance(dW, mnmaj(kk)), idescI,
+                            kk > 0);
             mma_commit(&ctl->bar_mma2);
             mma_commit(&ctl->bar_free2);
             PROF_MARK();
@@ -308,9 +311,8 @@ value_side_lean_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_co
             // ---- masked P rows (the barrier inside also publishes egc)
             LEAN_WAIT(&ctl->bar_p, n & 1);
             tc_fence_after_sync();
-            if (n >= 1) LEAN_WAIT(&ctl->bar_free, (n - 1) & 1);     // the staged rows of chunk n-1 have left
             PROF_MARK();
-            store_masked_row<REV, false>(tmem, wq, row, half, sPm, sPm);
+            mask_row_in_tmem<REV, false>(tmem, wq, row, half, kLvP);
             publish(&ctl->bar_pm, tid);
             PROF_MARK();
 
@@ -351,7 +353,7 @@ value_side_lean_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_co
                 tmem_ld32(tmem_row_addr(tmem, wq, kLvO + 64 * (n & 1) + sb), vi);
 #pragma unroll
                 for (int e = 0; e < kHS; ++e) vo[e] = REV ? fmaf(vi[e], egc[sb + e], vo[e]) : vo[e] + vi[e];
-                unsigned char* panel = sOut + half * kPanelB;
+                unsigned char* panel = sWd + (2 * (n & 1) + half) * kPanelB;
 #pragma unroll
                 for (int c = 0; c < kHS / 4; ++c)
                     *reinterpret_cast<float4*>(panel + swz128(row, c)) =
@@ -389,9 +391,7 @@ key_side_lean_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_cons
                                                      //   its tile is consumed
     unsigned char* sQK = sXv + 4 * kPanelB;          // decayed uq (K-major A [128][64]) and uk (K-major /
                                                      //   MN-major B [128][64]), 2 stages of 1 + 1 panels (64 KB)
-    unsigned char* sAm = sQK + 4 * kPanelB;          // masked A, K-major A, 2 panels              (32 KB)
-    unsigned char* sAl = sAm + 2 * kPanelB;          // rounding residual of the masked A, 2 panels (32 KB)
-    unsigned char* sSb = sAl + 2 * kPanelB;          // state copy, K-major B [128 (channel)][64]  (16 KB)
+    unsigned char* sSb = sQK + 4 * kPanelB;          // state copy, K-major B [128 (channel)][64]  (16 KB)
     LeanCtl* ctl = reinterpret_cast<LeanCtl*>(sSb + kPanelB);
 
     const int tid = threadIdx.x, warp = tid >> 5, wq = warp & 3, half = (tid >> 7) & 1, row = tid & 127;
@@ -453,7 +453,6 @@ key_side_lean_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_cons
         constexpr uint32_t idescU = make_idesc(128, kM, true, true);      // xv^T (MN-major A) x K~ (MN-major B)
         constexpr uint32_t idescV = make_idesc(128, kDST, false, true);   // A x xv (MN-major B)
         const uint64_t dS = desc_kmajor(smem_u32(sSb), 0);
-        const uint64_t dA = desc_kmajor(smem_u32(sAm), 0), dAl = desc_kmajor(smem_u32(sAl), 0);
         auto kmaj = [](int kk) { return (uint32_t)((kk >> 2) * kPanelB + (kk & 3) * 32); };
         auto mnmaj = [](int kk) { return (uint32_t)(kk * 2048); };
         auto issue_a = [&](int n) {
@@ -497,12 +496,14 @@ key_side_lean_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_cons
             LEAN_WAIT(&ctl->bar_pm, n & 1);
             tc_fence_after_sync();
             PROF_MARK();
+            // (the masked A and its rounding residual are bf16 rows in tensor memory, in place of A)
 #pragma unroll
             for (int kk = 0; kk < kCT / 16; ++kk)
-                mma_bf16(accO, desc_advance(dA, kmaj(kk)), desc_advance(dV, mnmaj(kk)), idescV, true);
+                mma_bf16_ta(accO, tmem + kLkA + 64 * (kk >> 2) + 8 * (kk & 3), desc_advance(dV, mnmaj(kk)), idescV, true);
 #pragma unroll
             for (int kk = 0; kk < kCT / 16; ++kk)
-                mma_bf16(accO, desc_advance(dAl, kmaj(kk)), desc_advance(dV, mnmaj(kk)), idescV, true);
+                mma_bf16_ta(accO, tmem + kLkA + 64 * (kk >> 2) + 32 + 8 * (kk & 3), desc_advance(dV, mnmaj(kk)), idescV,
+                            true);
             mma_commit(&ctl->bar_mma2);
             mma_commit(&ctl->bar_free2);
             PROF_MARK();
@@ -550,7 +551,7 @@ key_side_lean_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_cons
             // ---- masked A rows as a bf16 high/low pair (the barrier inside also publishes egc)
             LEAN_WAIT(&ctl->bar_p, n & 1);
             tc_fence_after_sync();
-            store_masked_row<REV, true>(tmem, wq, row, half, sAm, sAl);
+            mask_row_in_tmem<REV, true>(tmem, wq, row, half, kLkA);
             publish(&ctl->bar_pm, tid);
 
             // ---- state update from U^T: forward S <- exp(G_C) (S + U^T), reverse S <- exp(G_C) S + U^T
@@ -596,7 +597,8 @@ key_side_lean_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_cons
     lean_finish(ctl, tid, warp, tmem, dev_status);
 }
 
-constexpr size_t kSmemLean = 1024 + 13 * kPanelB + sizeof(LeanCtl);
+constexpr size_t kSmemLeanValue = 1024 + 13 * kPanelB + sizeof(LeanCtl);   // value_side: 8 + 4 + 1 panels
+constexpr size_t kSmemLeanKey = 1024 + 9 * kPanelB + sizeof(LeanCtl);      // key_side: 4 + 4 + 1 panels
 
 }  // namespace
 
@@ -610,13 +612,13 @@ cudaError_t launch_value_side_lean(const ValueSideArgs& a, int reverse, const in
     if (e != cudaSuccess) return e;
     dim3 grid(a.B * a.H, a.D / kDST);
     if (reverse) {
-        e = prepare(value_side_lean_kernel<true>, kSmemLean, kLeanThreads);
+        e = prepare(value_side_lean_kernel<true>, kSmemLeanValue, kLeanThreads);
         if (e != cudaSuccess) return e;
-        value_side_lean_kernel<true><<<grid, kLeanThreads, kSmemLean, st>>>(mq, mk, mw, mo, a, strong_flag, dev_status);
+        value_side_lean_kernel<true><<<grid, kLeanThreads, kSmemLeanValue, st>>>(mq, mk, mw, mo, a, strong_flag, dev_status);
     } else {
-        e = prepare(value_side_lean_kernel<false>, kSmemLean, kLeanThreads);
+        e = prepare(value_side_lean_kernel<false>, kSmemLeanValue, kLeanThreads);
         if (e != cudaSuccess) return e;
-        value_side_lean_kernel<false><<<grid, kLeanThreads, kSmemLean, st>>>(mq, mk, mw, mo, a, strong_flag, dev_status);
+        value_side_lean_kernel<false><<<grid, kLeanThreads, kSmemLeanValue, st>>>(mq, mk, mw, mo, a, strong_flag, dev_status);
     }
     return cudaGetLastError();
 }
@@ -631,13 +633,13 @@ cudaError_t launch_key_side_lean(const KeySideArgs& a, int reverse, const int* s
     if (e != cudaSuccess) return e;
     dim3 grid(a.B * a.H, a.D / kDST);
     if (reverse) {
-        e = prepare(key_side_lean_kernel<true>, kSmemLean, kLeanThreads);
+        e = prepare(key_side_lean_kernel<true>, kSmemLeanKey, kLeanThreads);
         if (e != cudaSuccess) return e;
-        key_side_lean_kernel<true><<<grid, kLeanThreads, kSmemLean, st>>>(mv, muq, muk, mo, a, strong_flag, dev_status);
+        key_side_lean_kernel<true><<<grid, kLeanThreads, kSmemLeanKey, st>>>(mv, muq, muk, mo, a, strong_flag, dev_status);
     } else {
-        e = prepare(key_side_lean_kernel<false>, kSmemLean, kLeanThreads);
+        e = prepare(key_side_lean_kernel<false>, kSmemLeanKey, kLeanThreads);
         if (e != cudaSuccess) return e;
-        key_side_lean_kernel<false><<<grid, kLeanThreads, kSmemLean, st>>>(mv, muq, muk, mo, a, strong_flag, dev_status);
+        key_side_lean_kernel<false><<<grid, kLeanThreads, kSmemLeanKey, st>>>(mv, muq, muk, mo, a, strong_flag, dev_status);
     }
     return cudaGetLastError();
 }

@@ -118,6 +118,47 @@ __device__ __forceinline__ void store_masked_row(uint32_t tmem, int wq, int row,
     }
 }
 
+// The same into tensor memory, in place: the thread's 64 fp32 columns (64 half .. 64 half + 63 from
+// `col0` on) become bf16 pairs in the first 32 of them -- the A operand of the next product, K step
+// kk at column col0 + 64 (kk >> 2) + 8 (kk & 3).  With SPLIT the rounding residual follows in the
+// other 32 columns (K step kk at + 32).  Every thread overwrites only columns it has read itself.
+template <bool REV, bool SPLIT>
+__device__ __forceinline__ void mask_row_in_tmem(uint32_t tmem, int wq, int row, int half, int col0) {
+    const int base = col0 + 64 * half;
+    uint32_t hi[32], lo[SPLIT ? 32 : 1];
+#pragma unroll
+    for (int c0 = 0; c0 < 64; c0 += 32) {
+        float v[32];
+        tmem_ld32(tmem_row_addr(tmem, wq, base + c0), v);
+#pragma unroll
+        for (int e = 0; e < 32; e += 2) {
+            const int j = 64 * half + c0 + e;
+            const float x0 = (REV ? (j >= row) : (j <= row)) ? v[e] : 0.f;
+            const float x1 = (REV ? (j + 1 >= row) : (j + 1 <= row)) ? v[e + 1] : 0.f;
+            hi[(c0 + e) >> 1] = pack_bf16(x0, x1);
+            if (SPLIT) {
+                const __nv_bfloat162 h = *reinterpret_cast<const __nv_bfloat162*>(&hi[(c0 + e) >> 1]);
+                lo[(c0 + e) >> 1] = pack_bf16(x0 - __bfloat162float(h.x), x1 - __bfloat162float(h.y));
+            }
+        }
+        if (!SPLIT) {
+            // the 16 packed columns of this batch land on columns already read
+            const uint32_t (&r)[16] = *reinterpret_cast<const uint32_t (*)[16]>(&hi[c0 >> 1]);
+            tmem_st16(tmem_row_addr(tmem, wq, base + (c0 >> 1)), r);
+        }
+    }
+    if (SPLIT) {
+#pragma unroll
+        for (int q = 0; q < 2; ++q) {
+            const uint32_t (&rh)[16] = *reinterpret_cast<const uint32_t (*)[16]>(&hi[16 * q]);
+            const uint32_t (&rl)[16] = *reinterpret_cast<const uint32_t (*)[16]>(&lo[SPLIT ? 16 * q : 0]);
+            tmem_st16(tmem_row_addr(tmem, wq, base + 16 * q), rh);
+            tmem_st16(tmem_row_addr(tmem, wq, base + 32 + 16 * q), rl);
+        }
+    }
+    tmem_st_wait();
+}
+
 // wait helper of the loops below: a wait that expires flags the CTA
 #define WAIT_OR_ABORT(bar, parity)                          \
     do {                                                    \

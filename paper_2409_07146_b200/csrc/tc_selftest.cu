@@ -77,7 +77,7 @@ __global__ void __launch_bounds__(128) tc_selftest_kernel(const __grid_constant_
     }
     if (warp == 0) {
         __syncwarp();
-        tmem_alloc(&tmem_slot, 128);
+        tmem_alloc(&tmem_slot, 256);
     }
     tc_fence_before_sync();
     __syncthreads();
@@ -108,10 +108,20 @@ __global__ void __launch_bounds__(128) tc_selftest_kernel(const __grid_constant_
             store_chunk(sW, tid, c, x);
         }
     }
+    else if (mode >= 4) {   // A = X in tensor memory: thread = row = lane, 64 packed columns from 128 on
+        for (int c0 = 0; c0 < 64; c0 += 16) {
+            uint32_t r[16];
+            for (int e = 0; e < 16; ++e)
+                r[e] = pack_bf16(__bfloat162float(X[tid * 128 + 2 * (c0 + e)]), __bfloat162float(X[tid * 128 + 2 * (c0 + e) + 1]));
+            tmem_st16(tmem_row_addr(tmem, warp, 128 + c0), r);
+        }
+        tmem_st_wait();
+        tc_fence_before_sync();
+    }
     fence_async_smem();
     __syncthreads();
     bool ok = mbar_wait(&bar_load, 0);
-    const int N = (mode <= 1) ? 128 : 64;
+    const int N = (mode <= 1 || mode >= 4) ? 128 : 64;
     if (ok && tid == 0) {
         tc_fence_after_sync();
         const uint32_t aX = smem_u32(sX), aY = smem_u32(sY), aW = smem_u32(sW);
@@ -130,10 +140,16 @@ __global__ void __launch_bounds__(128) tc_selftest_kernel(const __grid_constant_
                 da = desc_mnmajor(aX, kk, kPanel);
                 db = desc_kmajor(aW + (kk >> 2) * (64 * 128), kk);
                 idesc = make_idesc(128, 64, true, false);
-            } else {
+            } else if (mode == 3) {
                 da = desc_kmajor(aX + (kk >> 2) * kPanel, kk);
                 db = desc_mnmajor(aW, kk, kPanel);
                 idesc = make_idesc(128, 64, false, true);
+            } else {
+                // A from tensor memory; B = Y K-major (mode 4: X Y^T) or MN-major (mode 5: X Y)
+                db = mode == 4 ? desc_kmajor(aY + (kk >> 2) * kPanel, kk) : desc_mnmajor(aY, kk, kPanel);
+                idesc = make_idesc(128, 128, false, mode == 5);
+                mma_bf16_ta(tmem, tmem + 128 + 8 * kk, db, idesc, kk > 0);
+                continue;
             }
             mma_bf16(tmem, da, db, idesc, kk > 0);
         }
@@ -154,7 +170,7 @@ __global__ void __launch_bounds__(128) tc_selftest_kernel(const __grid_constant_
     __syncthreads();
     if (warp == 0) {
         __syncwarp();
-        tmem_dealloc(tmem, 128);
+        tmem_dealloc(tmem, 256);
     }
 }
 }  // namespace
@@ -163,7 +179,7 @@ __global__ void __launch_bounds__(128) tc_selftest_kernel(const __grid_constant_
 extern "C" GSA_API gsa_status_t gsa_tc_selftest(int32_t mode, const void* X, const void* Y, float* D, void* stream,
                                                 int32_t* dev_status) {
     using namespace gsa;
-    if (mode < 0 || mode > 3 || X == nullptr || Y == nullptr || D == nullptr) return GSA_ERR_INVALID_ARG;
+    if (mode < 0 || mode > 5 || X == nullptr || Y == nullptr || D == nullptr) return GSA_ERR_INVALID_ARG;
     CUtensorMap mx, my;
     if (make_tensor_map_bthd(&mx, X, 1, 128, 1, 128, 128, 2) != cudaSuccess) return GSA_ERR_CUDA;
     if (make_tensor_map_bthd(&my, Y, 1, 128, 1, 128, 128, 2) != cudaSuccess) return GSA_ERR_CUDA;

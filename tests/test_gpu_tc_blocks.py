@@ -9,7 +9,7 @@ import paper_2409_07146_b200 as gsa
 pytestmark = pytest.mark.gpu
 
 
-@pytest.mark.parametrize("mode", [0, 1, 2, 3])
+@pytest.mark.parametrize("mode", [0, 1, 2, 3, 4, 5])
 def test_tc_selftest_products(mode):
     g = torch.Generator().manual_seed(mode)
     X = torch.randn(128, 128, generator=g).to(torch.bfloat16)
@@ -19,6 +19,6 @@ def test_tc_selftest_products(mode):
     torch.cuda.synchronize()
     assert int(status.item()) == 0, "a bounded wait expired"
     x, y = X.double().numpy(), Y.double().numpy()
-    ref = {0: x @ y.T, 1: x @ y, 2: x.T @ y[:64].T, 3: x @ y[:, :64]}[mode]
+    ref = {0: x @ y.T, 1: x @ y, 2: x.T @ y[:64].T, 3: x @ y[:, :64], 4: x @ y.T, 5: x @ y}[mode]
     err = np.abs(D.cpu().double().numpy() - ref).max()
     assert err < 1e-3, err
