@@ -150,6 +150,35 @@ void timing_after(const char* label, cudaStream_t st) {
     }
 }
 
+// ---- the five scans of the backward that follow the softmax gradient are independent: on the
+// tensor-core path they run on five streams of the calling host thread (the caller's and four
+// of the library's), so that the CTAs of one start as those of another finish and the SMs that
+// one scan's 128 CTAs leave idle take CTAs of the next.  Forked and joined by events; with a
+// timing sink active they run one after the other instead, so that each is timed alone.
+struct ScanLanes {
+    cudaStream_t stream[4] = {nullptr, nullptr, nullptr, nullptr};
+    cudaEvent_t fork = nullptr, join[4] = {nullptr, nullptr, nullptr, nullptr};
+};
+cudaError_t scan_lanes(ScanLanes** out) {
+    constexpr int kMaxDevices = 64;
+    thread_local ScanLanes lanes[kMaxDevices];
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+    ScanLanes& l = lanes[dev];
+    if (l.fork == nullptr) {
+        for (int i = 0; i < 4 && e == cudaSuccess; ++i) {
+            e = cudaStreamCreateWithFlags(&l.stream[i], cudaStreamNonBlocking);
+            if (e == cudaSuccess) e = cudaEventCreateWithFlags(&l.join[i], cudaEventDisableTiming);
+        }
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&l.fork, cudaEventDisableTiming);
+        if (e != cudaSuccess) return e;
+    }
+    *out = &l;
+    return cudaSuccess;
+}
+
 #define GSA_CUDA(expr)                                  \
     do {                                                \
         cudaError_t e__ = (expr);                       \
@@ -298,16 +327,33 @@ gsa_status_t gsa_bwd(const gsa_params_t* params, const void* q, const void* k, c
                                                            w.Zd, pend, st));
     // dq: the pass-2 form on (dz, 1-a, k); carries K~
     KeySideArgs adq{w.dz, w.I, w.G, k, K0, dKT ? w.KT : nullptr, dq, p.B, p.T, p.H, p.d_k, w.Zd, w.Id};
-    GSA_LAUNCH("bwd_dq_key_side", key_side(p, adq, 0, w.strong, st, dev_status));
     // time-reversed runs: dv and dI^v share the state dV~; dk and dI^k share dK~
     KeySideArgs adv{w.I, w.p, w.G, dO, dVT, dV0, dv, p.B, p.T, p.H, p.d_v, w.Id, w.Pd};
-    GSA_LAUNCH("bwd_dv_key_side_rev", key_side(p, adv, 1, w.strong, st, dev_status));
     ValueSideArgs adIv{v, dO, w.p, w.G, dVT, nullptr, w.dIv, p.B, p.T, p.H, p.d_v, w.Pd};
-    GSA_LAUNCH("bwd_dIv_value_side_rev", value_side(p, adIv, 1, w.strong, st, dev_status));
     KeySideArgs adk{w.I, w.dz, w.G, q, dKT, dK0, dk, p.B, p.T, p.H, p.d_k, w.Id, w.Zd};
-    GSA_LAUNCH("bwd_dk_key_side_rev", key_side(p, adk, 1, w.strong, st, dev_status));
     ValueSideArgs adIk{k, q, w.dz, w.G, dKT, nullptr, w.dIk, p.B, p.T, p.H, p.d_k, w.Zd};
-    GSA_LAUNCH("bwd_dIk_value_side_rev", value_side(p, adIk, 1, w.strong, st, dev_status));
+    if (use_tc(p) && !g_sink.active) {
+        // the five scans side by side (see ScanLanes)
+        ScanLanes* lanes = nullptr;
+        GSA_CUDA(scan_lanes(&lanes));
+        GSA_CUDA(cudaEventRecord(lanes->fork, st));
+        for (int i = 0; i < 4; ++i) GSA_CUDA(cudaStreamWaitEvent(lanes->stream[i], lanes->fork, 0));
+        GSA_CUDA(key_side(p, adq, 0, w.strong, st, dev_status));
+        GSA_CUDA(key_side(p, adv, 1, w.strong, lanes->stream[0], dev_status));
+        GSA_CUDA(value_side(p, adIv, 1, w.strong, lanes->stream[1], dev_status));
+        GSA_CUDA(key_side(p, adk, 1, w.strong, lanes->stream[2], dev_status));
+        GSA_CUDA(value_side(p, adIk, 1, w.strong, lanes->stream[3], dev_status));
+        for (int i = 0; i < 4; ++i) {
+            GSA_CUDA(cudaEventRecord(lanes->join[i], lanes->stream[i]));
+            GSA_CUDA(cudaStreamWaitEvent(st, lanes->join[i], 0));
+        }
+    } else {
+        GSA_LAUNCH("bwd_dq_key_side", key_side(p, adq, 0, w.strong, st, dev_status));
+        GSA_LAUNCH("bwd_dv_key_side_rev", key_side(p, adv, 1, w.strong, st, dev_status));
+        GSA_LAUNCH("bwd_dIv_value_side_rev", value_side(p, adIv, 1, w.strong, st, dev_status));
+        GSA_LAUNCH("bwd_dk_key_side_rev", key_side(p, adk, 1, w.strong, st, dev_status));
+        GSA_LAUNCH("bwd_dIk_value_side_rev", value_side(p, adIk, 1, w.strong, st, dev_status));
+    }
     // forget-gate gradient: reversed cumulative sum over the whole sequence
     GSA_LAUNCH("gate_grad", launch_gate_grad(w.u, w.I, w.dIk, s.k, w.dIv, s.v, gate, p.gate_kind == GSA_GATE_LOG_A,
                               dKT, w.KT, dVT, w.VT, p.d_k, p.d_v, w.chunk_tot, dgate, p.B, p.T,

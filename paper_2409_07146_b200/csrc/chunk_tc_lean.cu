@@ -36,19 +36,21 @@ struct LeanCtl {
     uint64_t bar_p;        // first product of a chunk (P or A)
     uint64_t bar_mma1;     // state products (U and the inter-chunk product)
     uint64_t bar_mma2;     // intra-chunk product
-    uint64_t bar_free1;    // = bar_mma1, for the copy lane: tiles read by the state products may be overwritten
-    uint64_t bar_free2;    // = bar_mma2, for the copy lane: tiles read by the intra-chunk product may be overwritten
+    uint64_t bar_free1[2]; // = bar_mma1, for the copy lane (by chunk parity): tiles read by the state products
+                           // may be overwritten
     // signalled by the compute threads (one arrival after their barrier)
     uint64_t bar_pm;       // masked P / A rows are in shared memory, the P / A accumulator is free
     uint64_t bar_sb;       // state copy for the next chunk is written, the U accumulator is free
-    uint64_t bar_out;      // output rows are staged, the output accumulators are free
-    // signalled by the copy lane
-    uint64_t bar_free;     // the output staging buffer has been read by its store
+    uint64_t bar_out[2];   // (by chunk parity) output rows are staged, the output accumulators are free
     uint32_t tmem_slot;
     volatile int abort;
     alignas(16) float egc[2][kM];   // exp(G of the chunk's last valid row), by chunk parity
 };
 
+// Every mbarrier below has one producer and waiters that its producer cannot run two phases ahead
+// of: a barrier's next completion always needs something (a tile, a row, an accumulator) that a
+// waiter supplies only after it has seen the previous one.  Where a resource has two stages, so
+// has its barrier (indexed by chunk parity).
 // A wait that expires flags the CTA; once flagged, later waits return at once.  The compute
 // threads leave their loop only at the end-of-chunk barrier, on a vote, so that no thread is
 // left waiting at a barrier that others have abandoned.
@@ -80,12 +82,12 @@ __device__ __forceinline__ void lean_ctl_init(LeanCtl* ctl, int tid, int warp) {
         mbar_init(&ctl->bar_p, 1);
         mbar_init(&ctl->bar_mma1, 1);
         mbar_init(&ctl->bar_mma2, 1);
-        mbar_init(&ctl->bar_free1, 1);
-        mbar_init(&ctl->bar_free2, 1);
+        mbar_init(&ctl->bar_free1[0], 1);
+        mbar_init(&ctl->bar_free1[1], 1);
         mbar_init(&ctl->bar_pm, 1);
         mbar_init(&ctl->bar_sb, 1);
-        mbar_init(&ctl->bar_out, 1);
-        mbar_init(&ctl->bar_free, 1);
+        mbar_init(&ctl->bar_out[0], 1);
+        mbar_init(&ctl->bar_out[1], 1);
         ctl->abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -200,12 +202,12 @@ value_side_lean_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_co
         for (int n = 0; n < nchunks && !ctl->abort; ++n) {
             // the d-sized tiles of chunk n are consumed once its state products are done: their
             // buffer takes the tiles of chunk n+2
-            LEAN_WAIT(&ctl->bar_free1, n & 1);
+            LEAN_WAIT(&ctl->bar_free1[n & 1], (n >> 1) & 1);
             if (n + 2 < nchunks) load_x(n + 2);
             // the weights are consumed once the intra-chunk product is done; the compute threads then
             // stage the output rows in their place, and when those have left the buffer takes the
             // weights of chunk n+2
-            LEAN_WAIT(&ctl->bar_out, n & 1);
+            LEAN_WAIT(&ctl->bar_out[n & 1], (n >> 1) & 1);
             if (ctl->abort) break;
             store_out(n);
             bulk_wait_read();
@@ -254,7 +256,7 @@ value_side_lean_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_co
                 mma_bf16(tmem + kLvO + 64 * (n & 1), desc_advance(dQk, kmaj(kk)), desc_advance(dS, mnmaj(kk)), idescO,
                          kk > 0);
             mma_commit(&ctl->bar_mma1);
-            mma_commit(&ctl->bar_free1);
+            mma_commit(&ctl->bar_free1[n & 1]);
             PROF_MARK();
             // intra-chunk product once the masked P rows are there (bf16, in place in tensor memory)
             LEAN_WAIT(&ctl->bar_pm, n & 1);
@@ -265,7 +267,6 @@ value_side_lean_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_co
                 mma_bf16_ta(tmem + kLvI, tmem + kLvP + 64 * (kk >> 2) + 8 * (kk & 3), desc_advance(dW, mnmaj(kk)), idescI,
                             kk > 0);
             mma_commit(&ctl->bar_mma2);
-            mma_commit(&ctl->bar_free2);
             PROF_MARK();
             // the P accumulator is free: the next chunk's P queues right behind
             if (n + 1 < nchunks) {
@@ -360,7 +361,7 @@ value_side_lean_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_co
                         make_float4(vo[4 * c], vo[4 * c + 1], vo[4 * c + 2], vo[4 * c + 3]);
             }
             (void)valid;
-            const bool stop = publish_and_vote(&ctl->bar_out, tid, ctl->abort != 0);
+            const bool stop = publish_and_vote(&ctl->bar_out[n & 1], tid, ctl->abort != 0);
             PROF_MARK();
             PROF_DUMP("value_side lean compute");
             if (stop) break;
@@ -435,12 +436,12 @@ key_side_lean_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_cons
         for (int n = 0; n < nchunks && !ctl->abort; ++n) {
             // the decayed uq / uk rows of chunk n are consumed once its state products are done: their
             // buffer takes the rows of chunk n+2
-            LEAN_WAIT(&ctl->bar_free1, n & 1);
+            LEAN_WAIT(&ctl->bar_free1[n & 1], (n >> 1) & 1);
             if (n + 2 < nchunks) load_qk(n + 2);
             // the xv tile is consumed once the intra-chunk product is done; the compute threads then
             // stage the output rows in its place, and when those have left the buffer takes the tile
             // of chunk n+2
-            LEAN_WAIT(&ctl->bar_out, n & 1);
+            LEAN_WAIT(&ctl->bar_out[n & 1], (n >> 1) & 1);
             if (ctl->abort) break;
             store_out(n);
             bulk_wait_read();
@@ -490,7 +491,7 @@ key_side_lean_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_cons
             for (int kk = 0; kk < kM / 16; ++kk)
                 mma_bf16(accO, desc_advance(dQt, kmaj(kk)), desc_advance(dS, kmaj(kk)), idescO, kk > 0);
             mma_commit(&ctl->bar_mma1);
-            mma_commit(&ctl->bar_free1);
+            mma_commit(&ctl->bar_free1[n & 1]);
             PROF_MARK();
             // intra-chunk product (masked A and its rounding residual) on top of the inter-chunk one
             LEAN_WAIT(&ctl->bar_pm, n & 1);
@@ -505,7 +506,6 @@ key_side_lean_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_cons
                 mma_bf16_ta(accO, tmem + kLkA + 64 * (kk >> 2) + 32 + 8 * (kk & 3), desc_advance(dV, mnmaj(kk)), idescV,
                             true);
             mma_commit(&ctl->bar_mma2);
-            mma_commit(&ctl->bar_free2);
             PROF_MARK();
             // the A accumulator is free: the next chunk's A queues right behind
             if (n + 1 < nchunks) {
@@ -587,7 +587,7 @@ key_side_lean_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_cons
                     store_chunk(sXv + (2 * (n & 1) + half) * kPanelB, row, (c0 >> 3) + c, x);
                 }
             }
-            if (publish_and_vote(&ctl->bar_out, tid, ctl->abort != 0)) break;
+            if (publish_and_vote(&ctl->bar_out[n & 1], tid, ctl->abort != 0)) break;
         }
         if (!ctl->abort && a.Send) {
 #pragma unroll
