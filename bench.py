@@ -36,13 +36,14 @@ WORKLOAD = "train_1p3b"
 
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the tensor-core kernels on this
-# workload, from one `ncu --set full` capture (profiles/tc_chunk_kernels_train_1p3b_ncu_full.md).
+# workload, from one `ncu --set full` capture (profiles/step_kernels_train_1p3b_ncu_full.md).
 NCU_TRAFFIC = {
-    "pass1_value_side": 188711936, "bwd_dp_value_side": 187666432,
-    "bwd_dIv_value_side_rev": 190694912, "bwd_dIk_value_side_rev": 188507392,
-    "pass2_key_side": 106306560, "bwd_dq_key_side": 112874752,
-    "bwd_dv_key_side_rev": 108698624, "bwd_dk_key_side_rev": 112610560,
-    "gate_cumsum": 18426112, "slot_softmax": 102300416, "slot_softmax_bwd": 142108672,
+    "pass1_value_side": 187117048, "bwd_dp_value_side": 185888506,
+    "bwd_dIv_value_side_rev": 188052734, "bwd_dIk_value_side_rev": 186800636,
+    "pass2_key_side": 111426304, "bwd_dq_key_side": 117850112,
+    "bwd_dv_key_side_rev": 109418752, "bwd_dk_key_side_rev": 112322816,
+    "gate_cumsum": 18514432, "slot_softmax": 102231296, "slot_softmax_bwd": 140101630,
+    "gate_grad": 248593152,     # local + scan + carry
 }
 
 
