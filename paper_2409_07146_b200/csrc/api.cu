@@ -357,7 +357,7 @@ gsa_status_t gsa_bwd(const gsa_params_t* params, const void* q, const void* k, c
     // forget-gate gradient: reversed cumulative sum over the whole sequence
     GSA_LAUNCH("gate_grad", launch_gate_grad(w.u, w.I, w.dIk, s.k, w.dIv, s.v, gate, p.gate_kind == GSA_GATE_LOG_A,
                               dKT, w.KT, dVT, w.VT, p.d_k, p.d_v, w.chunk_tot, dgate, p.B, p.T,
-                              p.H, p.m, pend, st));
+                              p.H, p.m, pend, st, dev_status));
     return GSA_OK;
 }
 

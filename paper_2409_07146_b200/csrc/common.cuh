@@ -146,7 +146,7 @@ cudaError_t launch_gate_grad(const float* u, const float* I, const float* dIk_pa
                              int gate_is_log, const float* dKT, const float* KT,
                              const float* dVT, const float* VT, int d_k, int d_v,
                              float* chunk_tot, float* dgate, int B, int T, int H, int M,
-                             PendingDecay pend, cudaStream_t st);
+                             PendingDecay pend, cudaStream_t st, int32_t* dev_status);
 int gate_grad_blocks(int T);       // entries per (b,h,slot) of launch_gate_grad's scratch
 cudaError_t launch_value_side_simt(const ValueSideArgs& a, int io, int M, int reverse,
                                    cudaStream_t st);

@@ -3,6 +3,7 @@
 // backward, and the forget-gate gradient (reversed cumulative sum, App. B).
 // All of them stream [B,T,H,m] fp32 tensors once: they are HBM-bound.
 #include "common.cuh"
+#include "tc_common.cuh"
 
 namespace gsa {
 
@@ -435,6 +436,109 @@ __global__ void __launch_bounds__(128) gate_grad_local_kernel(
     *reinterpret_cast<float2*>(blk_tot + ((size_t)bh * nblk + n) * M + s) = make_float2(run0, run1);
 }
 
+// The same block-local pass with its inputs staged through shared memory by TMA (M = 64): one
+// CTA per (b,h) and 32 rows, every tile of every input stream (u, I, gate, G and the n_k + n_v
+// slices of the input-gate gradient: 12 x 8 KB at d = 512) requested at once by one thread --
+// 96 KB in flight per CTA, two CTAs per SM, several times what registers can hold as landing
+// space.  Thread = (slot pair, 16-row group), as above.
+constexpr int kGGTmaRows = 32;
+constexpr int kGGTmaMaxSlices = 8;
+constexpr int kGGTileB = kGGTmaRows * 64 * 4;      // bytes of one [32 x 64] fp32 tile (two swizzled panels)
+
+__global__ void __launch_bounds__(64) gate_grad_local_tma_kernel(
+    const __grid_constant__ CUtensorMap mapU, const __grid_constant__ CUtensorMap mapI,
+    const __grid_constant__ CUtensorMap mapGate, const __grid_constant__ CUtensorMap mapG,
+    const __grid_constant__ CUtensorMap mapDIk, const __grid_constant__ CUtensorMap mapDIv, int nsk, int nsv,
+    int gate_is_log, float* __restrict__ blk_tot, float* __restrict__ dgate, int T, int H, int nblk,
+    const int* __restrict__ strong, int32_t* dev_status) {
+    using namespace tc;
+    constexpr int M = 64;
+    extern __shared__ unsigned char gg_smem_raw[];
+    unsigned char* smem = gg_smem_raw + ((1024u - (smem_u32(gg_smem_raw) & 1023u)) & 1023u);
+    __shared__ uint64_t bar;
+    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;       // slot pair, 16-row group
+    const int bh = blockIdx.x, b = bh / H, h = bh % H;
+    const int t0 = blockIdx.y * kGGTmaRows;
+    const int nslices = nsk + nsv;
+    if (threadIdx.x == 0) {
+        mbar_init(&bar, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        mbar_expect_tx(&bar, (uint32_t)((4 + nslices) * kGGTileB));
+        const CUtensorMap* maps[4] = {&mapU, &mapI, &mapGate, &mapG};
+        for (int i = 0; i < 4; ++i) {
+            tma_load_4d(smem + i * kGGTileB, maps[i], &bar, 0, h, t0, b);
+            tma_load_4d(smem + i * kGGTileB + kGGTileB / 2, maps[i], &bar, 32, h, t0, b);
+        }
+        for (int sl = 0; sl < nslices; ++sl) {
+            const CUtensorMap* m = sl < nsk ? &mapDIk : &mapDIv;
+            const int z = sl < nsk ? sl : sl - nsk;
+            tma_load_5d(smem + (4 + sl) * kGGTileB, m, &bar, 0, h, t0, b, z);
+            tma_load_5d(smem + (4 + sl) * kGGTileB + kGGTileB / 2, m, &bar, 32, h, t0, b, z);
+        }
+    }
+    __syncthreads();
+    const bool landed = mbar_wait(&bar, 0);
+    if (!landed && threadIdx.x == 0 && dev_status != nullptr) *dev_status = GSA_ERR_TIMEOUT;
+    if (__syncthreads_or(!landed)) return;
+
+    const int n = blockIdx.y * (kGGTmaRows / kGG) + ty;           // 16-row block of the sequence
+    if (n >= nblk) return;
+    const int rows = min(kGG, T - n * kGG);
+    // row r (of this thread's 16), this thread's two slots, of tile `tile`
+    auto at = [&](int tile, int r) {
+        const int row = ty * kGG + r, c = 2 * tx;
+        const unsigned char* p = smem + tile * kGGTileB + (c >> 5) * (kGGTileB / 2) + swz128(row, (c & 31) >> 2) + (c & 3) * 4;
+        return *reinterpret_cast<const float2*>(p);
+    };
+    float2 x[kGG], dI[kGG];
+#pragma unroll
+    for (int i = 0; i < kGG; ++i) dI[i] = make_float2(0.f, 0.f);
+    for (int sl = 0; sl < nslices; ++sl) {
+#pragma unroll
+        for (int i = 0; i < kGG; ++i) {
+            const float2 t = at(4 + sl, i);
+            dI[i].x += t.x;
+            dI[i].y += t.y;
+        }
+    }
+    if (strong != nullptr && strong[bh] == 0) {
+        // the time-reversed value_side runs left their row factor exp(-G_i) to this kernel
+#pragma unroll
+        for (int i = 0; i < kGG; ++i) {
+            const float2 g = at(3, i);
+            dI[i].x *= __expf(-g.x);
+            dI[i].y *= __expf(-g.y);
+        }
+    }
+#pragma unroll
+    for (int i = 0; i < kGG; ++i) {
+        const float2 uu = at(0, i), ii = at(1, i);
+        x[i] = make_float2(uu.x - ii.x * dI[i].x, uu.y - ii.y * dI[i].y);       // rows past the end: all zero
+    }
+    const size_t stride = (size_t)H * M;
+    const size_t base = (((size_t)b * T + n * kGG) * H + h) * M + 2 * tx;
+    float run0 = 0.f, run1 = 0.f;
+#pragma unroll
+    for (int i = kGG - 1; i >= 0; --i) {
+        run0 += x[i].x;
+        run1 += x[i].y;
+        if (i < rows) {
+            const float2 gt = at(2, i);
+            float2 out;
+            if (gate_is_log) {
+                out.x = run0 - __expf(fmaxf(gt.x, kLogGateMin)) * dI[i].x;
+                out.y = run1 - __expf(fmaxf(gt.y, kLogGateMin)) * dI[i].y;
+            } else {
+                // a == 0 leaves no way back from d(log a) to da: only the input-gate part is kept
+                out.x = (gt.x > 0.f) ? run0 / gt.x - dI[i].x : -dI[i].x;
+                out.y = (gt.y > 0.f) ? run1 / gt.y - dI[i].y : -dI[i].y;
+            }
+            *reinterpret_cast<float2*>(dgate + base + (size_t)i * stride) = out;
+        }
+    }
+    *reinterpret_cast<float2*>(blk_tot + ((size_t)bh * nblk + n) * M + 2 * tx) = make_float2(run0, run1);
+}
+
 // Adds what follows the block: dgate += carry (log gate) or carry / a (linear gate).
 template <int M>
 __global__ void __launch_bounds__(128) gate_grad_carry_kernel(
@@ -473,13 +577,37 @@ cudaError_t launch_gate_grad(const float* u, const float* I, const float* dIk_pa
                              int gate_is_log, const float* dKT, const float* KT,
                              const float* dVT, const float* VT, int d_k, int d_v,
                              float* blk_tot, float* dgate, int B, int T, int H, int M,
-                             PendingDecay pend, cudaStream_t st) {
+                             PendingDecay pend, cudaStream_t st, int32_t* dev_status) {
     const int nblk = gate_grad_blocks(T);
     dim3 block(M / 2, 256 / M);      // 128 threads: M/2 slot pairs x 16-row blocks
     dim3 grid(B * H, (nblk + block.y - 1) / block.y);
     if (M == 64) {
-        gate_grad_local_kernel<64><<<grid, block, 0, st>>>(u, I, dIk_part, nsk, dIv_part, nsv, gate, gate_is_log,
-                                                           blk_tot, dgate, B, T, H, nblk, pend);
+        const int nsl = nsk + nsv;
+        bool staged = nsl <= kGGTmaMaxSlices;
+        CUtensorMap mu, mi, mg, mG, mk, mv;
+        if (staged) {
+            const float* Gp = pend.G != nullptr ? pend.G : u;      // (unused without a pending factor)
+            cudaError_t e = make_tensor_map_bthd(&mu, u, B, T, H, M, kGGTmaRows, 4);
+            if (e == cudaSuccess) e = make_tensor_map_bthd(&mi, I, B, T, H, M, kGGTmaRows, 4);
+            if (e == cudaSuccess) e = make_tensor_map_bthd(&mg, gate, B, T, H, M, kGGTmaRows, 4);
+            if (e == cudaSuccess) e = make_tensor_map_bthd(&mG, Gp, B, T, H, M, kGGTmaRows, 4);
+            if (e == cudaSuccess) e = make_tensor_map_sliced(&mk, dIk_part, nsk, B, T, H, M, kGGTmaRows, 4);
+            if (e == cudaSuccess) e = make_tensor_map_sliced(&mv, dIv_part, nsv, B, T, H, M, kGGTmaRows, 4);
+            staged = e == cudaSuccess;
+        }
+        if (staged) {
+            const size_t smem = 1024 + (size_t)(4 + nsl) * kGGTileB;
+            cudaError_t e = cudaFuncSetAttribute(gate_grad_local_tma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                 (int)smem);
+            if (e != cudaSuccess) return e;
+            dim3 tgrid(B * H, (T + kGGTmaRows - 1) / kGGTmaRows);
+            gate_grad_local_tma_kernel<<<tgrid, 64, smem, st>>>(mu, mi, mg, mG, mk, mv, nsk, nsv, gate_is_log, blk_tot,
+                                                                dgate, T, H, nblk, pend.G != nullptr ? pend.strong : nullptr,
+                                                                dev_status);
+        } else {
+            gate_grad_local_kernel<64><<<grid, block, 0, st>>>(u, I, dIk_part, nsk, dIv_part, nsv, gate, gate_is_log,
+                                                               blk_tot, dgate, B, T, H, nblk, pend);
+        }
         gate_grad_scan_kernel<64><<<B * H, dim3(64, 16), 0, st>>>(blk_tot, dKT, KT, dVT, VT, d_k, d_v, nblk);
         gate_grad_carry_kernel<64><<<grid, block, 0, st>>>(gate, gate_is_log, blk_tot, dgate, T, H, nblk);
     } else {
