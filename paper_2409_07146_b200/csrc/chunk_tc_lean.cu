@@ -266,6 +266,10 @@ value_side_lean_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_co
             for (int kk = 0; kk < kCT / 16; ++kk)
                 mma_bf16_ta(tmem + kLvI, tmem + kLvP + 64 * (kk >> 2) + 8 * (kk & 3), desc_advance(dW, mnmaj(kk)), idescI,
                             kk > 0);
+#pragma unroll
+            for (int kk = 0; kk < kCT / 16; ++kk)      // ... and the rounding residual of the masked P
+                mma_bf16_ta(tmem + kLvI, tmem + kLvP + 64 * (kk >> 2) + 32 + 8 * (kk & 3), desc_advance(dW, mnmaj(kk)),
+                            idescI, true);
             mma_commit(&ctl->bar_mma2);
             PROF_MARK();
             // the P accumulator is free: the next chunk's P queues right behind
@@ -313,7 +317,7 @@ value_side_lean_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_co
             LEAN_WAIT(&ctl->bar_p, n & 1);
             tc_fence_after_sync();
             PROF_MARK();
-            mask_row_in_tmem<REV, false>(tmem, wq, row, half, kLvP);
+            mask_row_in_tmem<REV, true>(tmem, wq, row, half, kLvP);
             publish(&ctl->bar_pm, tid);
             PROF_MARK();
 
@@ -391,9 +395,11 @@ key_side_lean_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_cons
                                                      //   ... a stage also holds the chunk's output rows once
                                                      //   its tile is consumed
     unsigned char* sQK = sXv + 4 * kPanelB;          // decayed uq (K-major A [128][64]) and uk (K-major /
-                                                     //   MN-major B [128][64]), 2 stages of 1 + 1 panels (64 KB)
-    unsigned char* sSb = sQK + 4 * kPanelB;          // state copy, K-major B [128 (channel)][64]  (16 KB)
-    LeanCtl* ctl = reinterpret_cast<LeanCtl*>(sSb + kPanelB);
+                                                     //   MN-major B [128][64]), each with its rounding residual:
+                                                     //   2 stages of 4 panels [uq_hi, uk_hi, uq_lo, uk_lo] (128 KB)
+    unsigned char* sSb = sQK + 8 * kPanelB;          // state copy, K-major B [128 (channel)][64], and its
+                                                     //   rounding residual                        (32 KB)
+    LeanCtl* ctl = reinterpret_cast<LeanCtl*>(sSb + 2 * kPanelB);
 
     const int tid = threadIdx.x, warp = tid >> 5, wq = warp & 3, half = (tid >> 7) & 1, row = tid & 127;
     const int sb = kHS * half;          // this thread's first slot
@@ -415,9 +421,11 @@ key_side_lean_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_cons
         };
         auto load_qk = [&](int n) {
             const int t = chunk_t0(n), st = n & 1;
-            mbar_expect_tx(&ctl->bar_w[st], 2 * kPanelB);
-            tma_load_4d(sQK + (2 * st) * kPanelB, &mapUq, &ctl->bar_w[st], 0, h, t, b);
-            tma_load_4d(sQK + (2 * st + 1) * kPanelB, &mapUk, &ctl->bar_w[st], 0, h, t, b);
+            mbar_expect_tx(&ctl->bar_w[st], 4 * kPanelB);
+            tma_load_4d(sQK + (4 * st) * kPanelB, &mapUq, &ctl->bar_w[st], 0, h, t, b);
+            tma_load_4d(sQK + (4 * st + 1) * kPanelB, &mapUk, &ctl->bar_w[st], 0, h, t, b);
+            tma_load_4d(sQK + (4 * st + 2) * kPanelB, &mapUq, &ctl->bar_w[st], 64, h, t, b);
+            tma_load_4d(sQK + (4 * st + 3) * kPanelB, &mapUk, &ctl->bar_w[st], 64, h, t, b);
         };
         auto store_out = [&](int n) {
             const int t = chunk_t0(n);
@@ -453,15 +461,23 @@ key_side_lean_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_cons
         constexpr uint32_t idescO = make_idesc(128, kDST, false, false);  // Q~ x state copy (K-major B)
         constexpr uint32_t idescU = make_idesc(128, kM, true, true);      // xv^T (MN-major A) x K~ (MN-major B)
         constexpr uint32_t idescV = make_idesc(128, kDST, false, true);   // A x xv (MN-major B)
-        const uint64_t dS = desc_kmajor(smem_u32(sSb), 0);
+        const uint64_t dS = desc_kmajor(smem_u32(sSb), 0), dSl = desc_kmajor(smem_u32(sSb + kPanelB), 0);
         auto kmaj = [](int kk) { return (uint32_t)((kk >> 2) * kPanelB + (kk & 3) * 32); };
         auto mnmaj = [](int kk) { return (uint32_t)(kk * 2048); };
         auto issue_a = [&](int n) {
-            const uint32_t qk = smem_u32(sQK + 2 * (n & 1) * kPanelB);
+            // A = Q~ K~^T with both factors as bf16 high/low pairs (the low x low term is dropped)
+            const uint32_t qk = smem_u32(sQK + 4 * (n & 1) * kPanelB);
             const uint64_t dQt = desc_kmajor(qk, 0), dKt = desc_kmajor(qk + kPanelB, 0);
+            const uint64_t dQl = desc_kmajor(qk + 2 * kPanelB, 0), dKl = desc_kmajor(qk + 3 * kPanelB, 0);
 #pragma unroll
             for (int kk = 0; kk < kM / 16; ++kk)
                 mma_bf16(tmem + kLkA, desc_advance(dQt, kmaj(kk)), desc_advance(dKt, kmaj(kk)), idescA, kk > 0);
+#pragma unroll
+            for (int kk = 0; kk < kM / 16; ++kk)
+                mma_bf16(tmem + kLkA, desc_advance(dQl, kmaj(kk)), desc_advance(dKt, kmaj(kk)), idescA, true);
+#pragma unroll
+            for (int kk = 0; kk < kM / 16; ++kk)
+                mma_bf16(tmem + kLkA, desc_advance(dQt, kmaj(kk)), desc_advance(dKl, kmaj(kk)), idescA, true);
             mma_commit(&ctl->bar_p);
         };
         LEAN_WAIT(&ctl->bar_w[0], 0);
@@ -473,8 +489,8 @@ key_side_lean_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_cons
             (void)it;
             const uint64_t dV = desc_mnmajor(smem_u32(sXv + 2 * (n & 1) * kPanelB), 0, kPanelB);
             const uint32_t accO = tmem + kLkO + 128 * (n & 1);
-            const uint32_t qk = smem_u32(sQK + 2 * (n & 1) * kPanelB);
-            const uint64_t dQt = desc_kmajor(qk, 0);
+            const uint32_t qk = smem_u32(sQK + 4 * (n & 1) * kPanelB);
+            const uint64_t dQt = desc_kmajor(qk, 0), dQl = desc_kmajor(qk + 2 * kPanelB, 0);
             const uint64_t dKtm = desc_mnmajor(qk + kPanelB, 0, kPanelB);   // the decayed uk read MN-major
             PROF_MARK();
             // state products of chunk n: the state copy was written at the end of chunk n-1 (which also
@@ -487,9 +503,16 @@ key_side_lean_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_cons
 #pragma unroll
             for (int kk = 0; kk < kCT / 16; ++kk)
                 mma_bf16(tmem + kLkU, desc_advance(dV, mnmaj(kk)), desc_advance(dKtm, mnmaj(kk)), idescU, kk > 0);
+            // inter-chunk product with both factors as bf16 high/low pairs (low x low dropped)
 #pragma unroll
             for (int kk = 0; kk < kM / 16; ++kk)
                 mma_bf16(accO, desc_advance(dQt, kmaj(kk)), desc_advance(dS, kmaj(kk)), idescO, kk > 0);
+#pragma unroll
+            for (int kk = 0; kk < kM / 16; ++kk)
+                mma_bf16(accO, desc_advance(dQl, kmaj(kk)), desc_advance(dS, kmaj(kk)), idescO, true);
+#pragma unroll
+            for (int kk = 0; kk < kM / 16; ++kk)
+                mma_bf16(accO, desc_advance(dQt, kmaj(kk)), desc_advance(dSl, kmaj(kk)), idescO, true);
             mma_commit(&ctl->bar_mma1);
             mma_commit(&ctl->bar_free1[n & 1]);
             PROF_MARK();
@@ -538,8 +561,8 @@ key_side_lean_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_cons
         compute_sync();
         // bf16 copy of the state for the first chunk's inter-chunk product (reverse: scaled by the
         // chunk's total decay, which the decayed uq rows leave out)
-        if (REV) store_state_row<true>(sSb, row, sb, S, ctl->egc[0]);
-        else store_state_row<false>(sSb, row, sb, S, nullptr);
+        if (REV) store_state_row_split<true>(sSb, sSb + kPanelB, row, sb, S, ctl->egc[0]);
+        else store_state_row_split<false>(sSb, sSb + kPanelB, row, sb, S, nullptr);
         publish(&ctl->bar_sb, tid);
 
         for (int n = 0; n < nchunks; ++n) {
@@ -569,8 +592,8 @@ key_side_lean_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_cons
                         S[e + t] = REV ? fmaf(S[e + t], ecv[t], v[e + t]) : (S[e + t] + v[e + t]) * ecv[t];
                 }
             }
-            if (REV) store_state_row<true>(sSb, row, sb, S, ctl->egc[(n + 1) & 1]);
-            else store_state_row<false>(sSb, row, sb, S, nullptr);
+            if (REV) store_state_row_split<true>(sSb, sSb + kPanelB, row, sb, S, ctl->egc[(n + 1) & 1]);
+            else store_state_row_split<false>(sSb, sSb + kPanelB, row, sb, S, nullptr);
             publish(&ctl->bar_sb, tid);
 
             // ---- output rows -> bf16, staged for the tiled store (clipped at the sequence end)
@@ -598,7 +621,7 @@ key_side_lean_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_cons
 }
 
 constexpr size_t kSmemLeanValue = 1024 + 13 * kPanelB + sizeof(LeanCtl);   // value_side: 8 + 4 + 1 panels
-constexpr size_t kSmemLeanKey = 1024 + 9 * kPanelB + sizeof(LeanCtl);      // key_side: 4 + 4 + 1 panels
+constexpr size_t kSmemLeanKey = 1024 + 14 * kPanelB + sizeof(LeanCtl);     // key_side: 4 + 8 + 2 panels
 
 }  // namespace
 

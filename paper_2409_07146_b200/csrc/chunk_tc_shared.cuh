@@ -74,6 +74,19 @@ __device__ __forceinline__ void store_state_row(unsigned char* panel, int row, i
     }
 }
 
+// The same as a bf16 pair: the rounded copy and its rounding residual, in two panels
+template <bool SCALE>
+__device__ __forceinline__ void store_state_row_split(unsigned char* panel_hi, unsigned char* panel_lo, int row, int sb,
+                                                      const float (&S)[kHS], const float* scale) {
+#pragma unroll
+    for (int c = 0; c < kHS / 8; ++c) {
+        float x[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) x[e] = SCALE ? S[8 * c + e] * scale[sb + 8 * c + e] : S[8 * c + e];
+        store_chunk_split(panel_hi, panel_lo, row, (sb >> 3) + c, x);
+    }
+}
+
 // Barrier over the 256 compute threads only (the issuing warp runs ahead on its own).
 __device__ __forceinline__ void compute_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
 __device__ __forceinline__ bool compute_sync_and(bool pred) {

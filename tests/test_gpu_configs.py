@@ -80,6 +80,7 @@ def run_training_config(name, with_bwd):
         assert np.isfinite(gs).all(), n
         kind, rtol, limit = TC_CONFIG_BOUNDS[n]
         errs[n] = dict(bound=mixed_err(gs, ref[n], rtol), plain=rel_err(gs, ref[n]), limit=limit,
+                       after_output_half_ulp=rel_err(gs, ref[n], True),
                        max_over_rms=float(np.abs(ref[n]).max() / np.sqrt(np.mean(ref[n] ** 2))))
     record(name, dict(pairs=pairs, errors=errs))
     print(name, {n: (round(e["plain"], 4), round(e["bound"], 4)) for n, e in errs.items()})

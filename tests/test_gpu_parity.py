@@ -282,21 +282,19 @@ def test_bwd_tc(T, log):
     B, H, dk, dv, m = 2, 2, 128, 256, 64
     d = rand_inputs(600 + T, B, T, H, dk, dv, m, "bf16", init=True)
     got, ref = run_bwd(d, B, T, H, dk, dv, m, "bf16", impl="tc", scale=1.1, log=log)
-    # short random sequences with non-zero initial memories have heavier-tailed gradients than
-    # the benchmark workloads (which are held to 2e-2): 3e-2 here
-    errs = check_bwd(got, ref, 1.5 * TOL["bf16"], tc=True)
+    errs = check_bwd(got, ref, TOL["bf16"], tc=True)
     print("tc bwd", T, log, errs)
 
 
 @pytest.mark.parametrize("T", [100, 256])
 def test_bwd_tc_final_memory_gradients(T):
     # Gradients w.r.t. the final memories enter dk, dv through single bf16 products
-    # (1 - a_j) * decay * dK_T whose terms cancel across slots: the error follows the size of
-    # the terms, not of the sums, hence the wider bound on this stress case.
+    # (1 - a_j) * decay * dK_T whose terms cancel across slots: the error of the gate gradient
+    # follows the size of the terms, not of the sums, hence 3e-2 on this stress case.
     B, H, dk, dv, m = 2, 2, 128, 256, 64
     d = rand_inputs(700 + T, B, T, H, dk, dv, m, "bf16", init=True, final_grads=True)
     got, ref = run_bwd(d, B, T, H, dk, dv, m, "bf16", impl="tc", scale=1.1)
-    errs = check_bwd(got, ref, 4 * TOL["bf16"], tc=True)
+    errs = check_bwd(got, ref, 1.5 * TOL["bf16"], tc=True)
     print("tc bwd final", T, errs)
 
 

@@ -25,25 +25,26 @@ def to_np(t):
 
 BF16_IO = {"o", "dq", "dk", "dv"}   # tensors stored in the io type (bf16 when io == "bf16")
 
-# Relative allowance of the tensor-core path (bf16 operands): besides the inputs, the chunk
-# kernels round five derived operands to bfloat16 on the way to a gradient (masked q.k
-# products, decayed gate weights, the state copy, the slot-space attention matrix, the
-# scaled softmax gradient), each good to 2^-9 relative; 2^-7 |ref| covers their chain.
-TC_RTOL = 2.0 ** -7
+# Relative allowance of the tensor-core path in the small-shape tests: the half-ulp of a bfloat16
+# output, 2^-9 |ref| (for the fp32 outputs -- logits, memories, gate gradient -- it stands for the
+# bf16 rounding of the operand that dominates them).
+TC_RTOL = 2.0 ** -9
 # Bounds of the tensor-core path at the size of the benchmark configurations, per tensor:
 # ("plain", 0, x)  = max|err| / rms <= x with no allowance (the stated bound where x = 2e-2);
 # ("mixed", r, x)  = the same after a relative allowance r |ref| per element.
-# The output o, the slot logits, the final memories, dv and the gate gradient meet the
-# stated 2e-2 as it stands (the decayed weights and the masked slot-space matrix are carried
-# as bf16 high/low pairs for that).  dq and dk still sit behind plain bf16 roundings of the
-# masked q.k products, the state copy and the decayed softmax gradient: 3.9-4.2e-2 at
-# train_1p3b, and where key channels carry outliers (t2r_7b: max|dq| / rms = 39) the error
-# follows the scale of the channel rather than of the element, 11.5e-2; after a 2^-6
-# allowance (eight bf16 roundings in a row) they are at 1.4-5.0e-2: known gaps.
+# The output o, the slot logits, the final memories, dv and the gate gradient meet the stated
+# 2e-2 as it stands.  dq and dk are stored as bfloat16 and heavy-tailed (max|ref| / rms = 10-11
+# at train_1p3b, 39 for dq at t2r_7b, where key channels carry outliers): the half-ulp of the
+# output format alone, 2^-9 |ref|, is then 2e-2 of the rms and more, so it is taken off first
+# (as for the CUDA-core kernels with bf16 io).  What is left: 1.2e-2 at train_1p3b for both,
+# dk 1.0e-2 and dq 2.5e-2 at t2r_7b (the one known gap: the error follows the scale of the
+# outlier channel rather than of the element).  Every operand that the kernels derive on the
+# way to these gradients -- decayed weights, masked products, decayed q / k rows of the
+# slot-space product, the state copy of the pass-2 form -- is carried as a bf16 high/low pair.
 TC_CONFIG_BOUNDS = {
     "o": ("plain", 0.0, 2e-2), "ok": ("plain", 0.0, 2e-2), "KT": ("plain", 0.0, 2e-2),
-    "VT": ("plain", 0.0, 2e-2), "dv": ("plain", 0.0, 2e-2), "dq": ("mixed", 2.0 ** -6, 6e-2),
-    "dk": ("mixed", 2.0 ** -6, 3.5e-2), "dgate": ("plain", 0.0, 3e-2),
+    "VT": ("plain", 0.0, 2e-2), "dv": ("plain", 0.0, 2e-2), "dq": ("mixed", 2.0 ** -9, 2.6e-2),
+    "dk": ("mixed", 2.0 ** -9, 2e-2), "dgate": ("plain", 0.0, 2e-2),
 }
 
 
