@@ -38,12 +38,12 @@ WORKLOAD = "train_1p3b"
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the tensor-core kernels on this
 # workload, from one `ncu --set full` capture (profiles/step_kernels_train_1p3b_ncu_full.md).
 NCU_TRAFFIC = {
-    "pass1_value_side": 187117048, "bwd_dp_value_side": 185888506,
-    "bwd_dIv_value_side_rev": 188052734, "bwd_dIk_value_side_rev": 186800636,
-    "pass2_key_side": 111426304, "bwd_dq_key_side": 117850112,
-    "bwd_dv_key_side_rev": 109418752, "bwd_dk_key_side_rev": 112322816,
-    "gate_cumsum": 18514432, "slot_softmax": 102231296, "slot_softmax_bwd": 140101630,
-    "gate_grad": 248593152,     # local + scan + carry
+    "pass1_value_side": 187083264, "bwd_dp_value_side": 186084344,
+    "bwd_dIv_value_side_rev": 188307968, "bwd_dIk_value_side_rev": 190506744,
+    "pass2_key_side": 129381884, "bwd_dq_key_side": 136861688,
+    "bwd_dv_key_side_rev": 130355960, "bwd_dk_key_side_rev": 132610046,
+    "gate_cumsum": 18483712, "slot_softmax": 101182208, "slot_softmax_bwd": 140176126,
+    "gate_grad": 251560184,     # local + scan + carry
 }
 
 
@@ -74,18 +74,18 @@ def kernel_algorithmic_bytes(label: str, w: W.Workload) -> int:
     m = w.m
     nsk, nsv = w.d_k // 128, w.d_v // 128
     # bytes per token-head row on the tensor-core path: fp32 [.., m] tensors are 4m, a decayed
-    # bf16 operand row [high | residual] is 4m too (the key_side kernels read its first half)
+    # bf16 operand row [high | residual] is 4m too
     table = {
         "gate_cumsum": 16 * m,                                       # gate -> G, I, I exp(-G)
         "pass1_value_side": 2 * w.d_k * e + 4 * m + 4 * m * nsk,     # q, k, I exp(-G) -> slices of o'
         "slot_softmax": 4 * m * nsk + 16 * m,                        # slices, G -> o', p, p exp(G)
-        "pass2_key_side": 2 * w.d_v * e + 4 * m,                     # v, two decayed half rows -> o
+        "pass2_key_side": 2 * w.d_v * e + 8 * m,                     # v, two decayed rows -> o
         "bwd_dp_value_side": 2 * w.d_v * e + 4 * m + 4 * m * nsv,
         "slot_softmax_bwd": 4 * m * nsv + 28 * m,                    # o', slices, G -> p, dz, u, p exp(G), dz exp(G)
-        "bwd_dq_key_side": 2 * w.d_k * e + 4 * m,
-        "bwd_dv_key_side_rev": 2 * w.d_v * e + 4 * m,
+        "bwd_dq_key_side": 2 * w.d_k * e + 8 * m,
+        "bwd_dv_key_side_rev": 2 * w.d_v * e + 8 * m,
         "bwd_dIv_value_side_rev": 2 * w.d_v * e + 4 * m + 4 * m * nsv,
-        "bwd_dk_key_side_rev": 2 * w.d_k * e + 4 * m,
+        "bwd_dk_key_side_rev": 2 * w.d_k * e + 8 * m,
         "bwd_dIk_value_side_rev": 2 * w.d_k * e + 4 * m + 4 * m * nsk,
         "gate_grad": 4 * m * (8 + nsk + nsv),   # u, I, gate, G, partials -> dgate; carry pass reads gate, r/w dgate
     }
