@@ -30,7 +30,7 @@ __device__ __forceinline__ void store_split2(__nv_bfloat16* row, int c, float x0
 }
 
 template <int M>
-__global__ void __launch_bounds__(M * 4) gate_cumsum_kernel(const float* __restrict__ gate,
+__global__ void __launch_bounds__(M * 4, 4) gate_cumsum_kernel(const float* __restrict__ gate,
                                                             int gate_is_log,
                                                             float* __restrict__ G,
                                                             float* __restrict__ I, int T, int H,
@@ -117,36 +117,38 @@ cudaError_t launch_gate_cumsum(const float* gate, int gate_is_log, float* G, flo
 }
 
 // ------------------------------------------------------------------ slot softmax
-// One warp per token-head row of M slots: lane l holds the R = M/32 adjacent slots l R .. l R + R-1
-// (one 8-byte access per tensor and lane for M = 64).
-template <int R>
-__device__ __forceinline__ void ld_vec(const float* p, float (&x)[R]) {
-    if constexpr (R == 2) {
-        const float2 v = *reinterpret_cast<const float2*>(p);
-        x[0] = v.x; x[1] = v.y;
-    } else {
-#pragma unroll
-        for (int r = 0; r < R; ++r) x[r] = p[r];
-    }
+// M/4 lanes per token-head row of M slots, four adjacent slots per lane (one 16-byte access per
+// tensor and lane), 128/M rows per warp; reductions run over the lanes of a row.
+constexpr int kSmR = 4;                                  // slots per lane
+__device__ __forceinline__ void ld_vec(const float* p, float (&x)[kSmR]) {
+    const float4 v = *reinterpret_cast<const float4*>(p);
+    x[0] = v.x; x[1] = v.y; x[2] = v.z; x[3] = v.w;
 }
-template <int R>
-__device__ __forceinline__ void st_vec(float* p, const float (&x)[R]) {
-    if constexpr (R == 2) {
-        *reinterpret_cast<float2*>(p) = make_float2(x[0], x[1]);
-    } else {
-#pragma unroll
-        for (int r = 0; r < R; ++r) p[r] = x[r];
-    }
+__device__ __forceinline__ void st_vec(float* p, const float (&x)[kSmR]) {
+    *reinterpret_cast<float4*>(p) = make_float4(x[0], x[1], x[2], x[3]);
 }
 // the lane's slots of a decayed-operand row [hi(M) | lo(M)]
-template <int M, int R>
-__device__ __forceinline__ void st_split(__nv_bfloat16* row, int c, const float (&x)[R]) {
-    if constexpr (R == 2) {
-        store_split2<M>(row, c, x[0], x[1]);
-    } else {
+template <int M>
+__device__ __forceinline__ void st_split(__nv_bfloat16* row, int c, const float (&x)[kSmR]) {
+    __nv_bfloat162 h0, h1, l0, l1;
+    split_bf16(x[0], h0.x, l0.x);
+    split_bf16(x[1], h0.y, l0.y);
+    split_bf16(x[2], h1.x, l1.x);
+    split_bf16(x[3], h1.y, l1.y);
+    *reinterpret_cast<uint2*>(row + c) = make_uint2(*reinterpret_cast<uint32_t*>(&h0), *reinterpret_cast<uint32_t*>(&h1));
+    *reinterpret_cast<uint2*>(row + M + c) = make_uint2(*reinterpret_cast<uint32_t*>(&l0), *reinterpret_cast<uint32_t*>(&l1));
+}
+template <int LPR>
+__device__ __forceinline__ float row_max(float x) {
 #pragma unroll
-        for (int r = 0; r < R; ++r) split_bf16(x[r], row[c + r], row[M + c + r]);
-    }
+    for (int o = LPR / 2; o; o >>= 1) x = fmaxf(x, __shfl_xor_sync(0xffffffffu, x, o));
+    return x;
+}
+template <int LPR>
+__device__ __forceinline__ float row_sum(float x) {
+#pragma unroll
+    for (int o = LPR / 2; o; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
+    return x;
 }
 
 template <int M>
@@ -157,26 +159,27 @@ __global__ void __launch_bounds__(256) slot_softmax_fwd_kernel(const float* __re
                                                                int rows_per_batch, const float* __restrict__ G,
                                                                __nv_bfloat16* __restrict__ p_decayed,
                                                                PendingDecay pend) {
-    constexpr int R = M / 32;
-    const int r_in_b = blockIdx.x * 8 + (threadIdx.x >> 5), b = blockIdx.y;
-    const int lane = threadIdx.x & 31;
-    if (r_in_b >= rows_per_batch) return;
-    const size_t row = (size_t)b * rows_per_batch + r_in_b;
+    constexpr int R = kSmR, LPR = M / R, RPW = 32 / LPR;       // lanes per row, rows per warp
+    const int lane = threadIdx.x & 31, sub = lane / LPR, l = lane % LPR;
+    const int r_in_b = (blockIdx.x * 8 + (threadIdx.x >> 5)) * RPW + sub, b = blockIdx.y;
+    const bool live = r_in_b < rows_per_batch;       // a row past the end repeats the last one (full-warp shuffles)
+    const int rr = live ? r_in_b : rows_per_batch - 1;
+    const size_t row = (size_t)b * rows_per_batch + rr;
     const size_t total = (size_t)gridDim.y * rows_per_batch * M;
-    const size_t idx = row * M + lane * R;
-    const bool pending = pend.pending(b, r_in_b);
+    const size_t idx = row * M + l * R;
+    const bool pending = pend.pending(b, rr);
     float z[R], eg[R];
 #pragma unroll
     for (int r = 0; r < R; ++r) { z[r] = 0.f; eg[r] = 1.f; }
 #pragma unroll 4
     for (int sl = 0; sl < nslice; ++sl) {
         float t[R];
-        ld_vec<R>(part + idx + (size_t)sl * total, t);
+        ld_vec(part + idx + (size_t)sl * total, t);
 #pragma unroll
         for (int r = 0; r < R; ++r) z[r] += t[r];
     }
     if (G != nullptr) {
-        ld_vec<R>(G + idx, eg);
+        ld_vec(G + idx, eg);
 #pragma unroll
         for (int r = 0; r < R; ++r) eg[r] = __expf(eg[r]);
     }
@@ -187,29 +190,29 @@ __global__ void __launch_bounds__(256) slot_softmax_fwd_kernel(const float* __re
         z[r] *= scale;
         zmax = fmaxf(zmax, z[r]);
     }
-#pragma unroll
-    for (int o = 16; o; o >>= 1) zmax = fmaxf(zmax, __shfl_xor_sync(0xffffffffu, zmax, o));
+    zmax = row_max<LPR>(zmax);
     float e[R], den = 0.f;
 #pragma unroll
     for (int r = 0; r < R; ++r) { e[r] = __expf(z[r] - zmax); den += e[r]; }
-#pragma unroll
-    for (int o = 16; o; o >>= 1) den += __shfl_xor_sync(0xffffffffu, den, o);
+    den = row_sum<LPR>(den);
     const float inv = 1.f / den;
 #pragma unroll
     for (int r = 0; r < R; ++r) e[r] *= inv;
-    st_vec<R>(ok + idx, z);
-    st_vec<R>(p + idx, e);
+    if (!live) return;
+    st_vec(ok + idx, z);
+    st_vec(p + idx, e);
     if (p_decayed != nullptr) {
 #pragma unroll
         for (int r = 0; r < R; ++r) e[r] *= eg[r];
-        st_split<M, R>(p_decayed + row * 2 * M, lane * R, e);
+        st_split<M>(p_decayed + row * 2 * M, l * R, e);
     }
 }
 
 cudaError_t launch_slot_softmax_fwd(const float* part, int nslice, float scale, float* ok,
                                     float* p, int B, int rows_per_batch, int M, const float* G, void* p_decayed,
                                     PendingDecay pend, cudaStream_t st) {
-    const dim3 grid((unsigned)((rows_per_batch + 7) / 8), (unsigned)B);
+    const int rpb = 8 * (128 / M);       // rows per block: 8 warps x 128/M rows
+    const dim3 grid((unsigned)((rows_per_batch + rpb - 1) / rpb), (unsigned)B);
     const int rows = rows_per_batch;
     if (M == 64)
         slot_softmax_fwd_kernel<64><<<grid, 256, 0, st>>>(part, nslice, scale, ok, p, rows, G,
@@ -236,27 +239,28 @@ __global__ void __launch_bounds__(256) slot_softmax_bwd_kernel(const float* __re
                                                                __nv_bfloat16* __restrict__ p_decayed,
                                                                __nv_bfloat16* __restrict__ dz_decayed,
                                                                PendingDecay pend) {
-    constexpr int R = M / 32;
-    const int r_in_b = blockIdx.x * 8 + (threadIdx.x >> 5), b = blockIdx.y;
-    const int lane = threadIdx.x & 31;
-    if (r_in_b >= rows_per_batch) return;
-    const size_t row = (size_t)b * rows_per_batch + r_in_b;
+    constexpr int R = kSmR, LPR = M / R, RPW = 32 / LPR;       // lanes per row, rows per warp
+    const int lane = threadIdx.x & 31, sub = lane / LPR, l = lane % LPR;
+    const int r_in_b = (blockIdx.x * 8 + (threadIdx.x >> 5)) * RPW + sub, b = blockIdx.y;
+    const bool live = r_in_b < rows_per_batch;       // a row past the end repeats the last one (full-warp shuffles)
+    const int rr = live ? r_in_b : rows_per_batch - 1;
+    const size_t row = (size_t)b * rows_per_batch + rr;
     const size_t total = (size_t)gridDim.y * rows_per_batch * M;
-    const size_t idx = row * M + lane * R;
-    const bool pending = pend.pending(b, r_in_b);
+    const size_t idx = row * M + l * R;
+    const bool pending = pend.pending(b, rr);
     float z[R], dpv[R], eg[R];
-    ld_vec<R>(ok + idx, z);
+    ld_vec(ok + idx, z);
 #pragma unroll
     for (int r = 0; r < R; ++r) { dpv[r] = 0.f; eg[r] = 1.f; }
 #pragma unroll 4
     for (int sl = 0; sl < nslice; ++sl) {
         float t[R];
-        ld_vec<R>(dp_part + idx + (size_t)sl * total, t);
+        ld_vec(dp_part + idx + (size_t)sl * total, t);
 #pragma unroll
         for (int r = 0; r < R; ++r) dpv[r] += t[r];
     }
     if (G != nullptr) {
-        ld_vec<R>(G + idx, eg);
+        ld_vec(G + idx, eg);
 #pragma unroll
         for (int r = 0; r < R; ++r) eg[r] = __expf(eg[r]);
     }
@@ -266,19 +270,17 @@ __global__ void __launch_bounds__(256) slot_softmax_bwd_kernel(const float* __re
         if (pending) dpv[r] *= eg[r];
         zmax = fmaxf(zmax, z[r]);
     }
-#pragma unroll
-    for (int o = 16; o; o >>= 1) zmax = fmaxf(zmax, __shfl_xor_sync(0xffffffffu, zmax, o));
+    zmax = row_max<LPR>(zmax);
     float e[R], den = 0.f;
 #pragma unroll
     for (int r = 0; r < R; ++r) { e[r] = __expf(z[r] - zmax); den += e[r]; }
-#pragma unroll
-    for (int o = 16; o; o >>= 1) den += __shfl_xor_sync(0xffffffffu, den, o);
+    den = row_sum<LPR>(den);
     const float inv = 1.f / den;
     float pdp = 0.f;
 #pragma unroll
     for (int r = 0; r < R; ++r) { e[r] *= inv; pdp += e[r] * dpv[r]; }
-#pragma unroll
-    for (int o = 16; o; o >>= 1) pdp += __shfl_xor_sync(0xffffffffu, pdp, o);
+    pdp = row_sum<LPR>(pdp);
+    if (!live) return;
     float dzv[R], uv[R];
 #pragma unroll
     for (int r = 0; r < R; ++r) {
@@ -286,14 +288,14 @@ __global__ void __launch_bounds__(256) slot_softmax_bwd_kernel(const float* __re
         dzv[r] = scale * dok;
         uv[r] = e[r] * dpv[r] + z[r] * dok;
     }
-    st_vec<R>(p + idx, e);
-    st_vec<R>(dz + idx, dzv);
-    st_vec<R>(u + idx, uv);
+    st_vec(p + idx, e);
+    st_vec(dz + idx, dzv);
+    st_vec(u + idx, uv);
     if (p_decayed != nullptr) {
 #pragma unroll
         for (int r = 0; r < R; ++r) { e[r] *= eg[r]; dzv[r] *= eg[r]; }
-        st_split<M, R>(p_decayed + row * 2 * M, lane * R, e);
-        st_split<M, R>(dz_decayed + row * 2 * M, lane * R, dzv);
+        st_split<M>(p_decayed + row * 2 * M, l * R, e);
+        st_split<M>(dz_decayed + row * 2 * M, l * R, dzv);
     }
 }
 
@@ -301,7 +303,8 @@ cudaError_t launch_slot_softmax_bwd(const float* ok, const float* dp_part, int n
                                     float scale, float* p, float* dz, float* u, int B, int rows_per_batch,
                                     int M, const float* G, void* p_decayed, void* dz_decayed,
                                     PendingDecay pend, cudaStream_t st) {
-    const dim3 grid((unsigned)((rows_per_batch + 7) / 8), (unsigned)B);
+    const int rpb = 8 * (128 / M);       // rows per block: 8 warps x 128/M rows
+    const dim3 grid((unsigned)((rows_per_batch + rpb - 1) / rpb), (unsigned)B);
     const int rows = rows_per_batch;
     if (M == 64)
         slot_softmax_bwd_kernel<64><<<grid, 256, 0, st>>>(ok, dp_part, nslice, scale, p, dz, u, rows, G,
