@@ -266,9 +266,9 @@ gsa_status_t gsa_fwd(const gsa_params_t* params, const void* q, const void* k, c
         // segments, and the final memories, by a scan over the segments
         GSA_LAUNCH("segment_logdecay", launch_segment_logdecay(w.G, w.seg_decay, p.B, p.T, p.H, p.m, nseg,
                                                                chunk_of(p), st));
-        ValueSideArgs s1{q, k, w.I, w.G, nullptr, w.Kloc, w.okpart, Bs, Ts, p.H, p.d_k, w.Id};
+        ValueSideArgs s1{q, k, w.I, w.G, nullptr, w.Kloc, w.okpart, Bs, Ts, p.H, p.d_k, w.Id, 1};
         GSA_LAUNCH("segment_pass1_states", value_side(p, s1, 0, w.strong, st, dev_status));
-        KeySideArgs s2{w.I, w.I, w.G, v, nullptr, w.Vloc, o, Bs, Ts, p.H, p.d_v, w.Id, w.Id};
+        KeySideArgs s2{w.I, w.I, w.G, v, nullptr, w.Vloc, o, Bs, Ts, p.H, p.d_v, w.Id, w.Id, 1};
         GSA_LAUNCH("segment_pass2_states", key_side(p, s2, 0, w.strong, st, dev_status));
         GSA_LAUNCH("segment_combine", launch_segment_combine(w.seg_decay, w.Kloc, K0, w.Kstart, KT, p.B, p.H, p.m,
                                                              p.d_k, nseg, st));

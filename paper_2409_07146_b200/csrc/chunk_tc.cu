@@ -363,8 +363,9 @@ value_side_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_cons
                 // cores (only the general variant of the kernel carries this path).
                 WAIT_OR_ABORT(&ctl->bar_mma1, it & 1);    // the inter-chunk product
                 tc_fence_after_sync();
-                value_side_explicit_rows<REV>(gt, sW, ctl->gc, tmem, wq, row, sb, grow, valid,
-                                              obase + (size_t)(t0 + row) * strideM);
+                if (!a.state_only)
+                    value_side_explicit_rows<REV>(gt, sW, ctl->gc, tmem, wq, row, sb, grow, valid,
+                                                  obase + (size_t)(t0 + row) * strideM);
             }
 
             // ---- state update from U: S <- S exp(G_C) + U  (forward moderate chunk: exp(G_C) (S + U))
@@ -695,7 +696,7 @@ key_side_tc_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_consta
             } else if constexpr (GENERAL) {
                 // Strong decay: A_ij with explicit exponent differences (only the general variant of
                 // the kernel carries this path).
-                key_side_explicit_rows<REV>(sG, sUq, sUk, sAm, sAl, row, half, grow, valid);
+                if (!a.state_only) key_side_explicit_rows<REV>(sG, sUq, sUk, sAm, sAl, row, half, grow, valid);
             }
             fence_async_smem();
             tc_fence_before_sync();

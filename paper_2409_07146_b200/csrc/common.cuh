@@ -83,6 +83,9 @@ struct ValueSideArgs {
     // tensor-core path: the weights already multiplied by their decay factor, bf16 rows of 2M
     // [high part | rounding residual] of w exp(-G) (forward) or w exp(G) (reverse); nullable
     const void* wd;
+    // only the end state matters to the caller (first run of the segment-parallel forward): kernels
+    // may leave `out` unwritten where computing it is expensive
+    int state_only;
 };
 struct KeySideArgs {
     const float* uq; const float* uk; const float* G;
@@ -94,6 +97,7 @@ struct KeySideArgs {
     // tensor-core path: decayed bf16 rows of 2M (the first M are used): forward uq exp(G) and
     // uk exp(-G), reverse uq exp(-G) and uk exp(G); nullable (both or neither)
     const void* uq_d; const void* uk_d;
+    int state_only;                   // as in ValueSideArgs
 };
 
 // The pipelined tensor-core value_side kernel leaves the row factor of its partial sums --
