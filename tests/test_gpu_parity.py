@@ -267,6 +267,40 @@ def test_fwd_tc_segment_parallel_schedule(gate, init):
     print("segment-parallel fwd", errs)
 
 
+def test_step_is_graph_capturable_and_replays_bitwise():
+    # fwd + bwd enqueue on the caller's stream and on the library's side streams with event
+    # fork / join only: a CUDA graph capture of one step must replay to the same bits
+    B, T, H, dk, dv, m = 2, 384, 2, 256, 128, 64
+    d = rand_inputs(77, B, T, H, dk, dv, m, "bf16")
+    p = gsa.Params(B, T, H, dk, dv, m, io="bf16")
+    q, k, v, dO = (to_dev(d[n], "bf16") for n in ("q", "k", "v", "dO"))
+    gate = to_dev(d["gate"])
+    ok = torch.empty(B, T, H, m, device="cuda")
+    o = torch.empty(B, T, H, dv, dtype=torch.bfloat16, device="cuda")
+    dq, dk_, dv_, dg = torch.empty_like(q), torch.empty_like(k), torch.empty_like(v), torch.empty_like(gate)
+    ws_f = torch.empty(gsa.gsa_workspace_bytes(p, 0), dtype=torch.uint8, device="cuda")
+    ws_b = torch.empty(gsa.gsa_workspace_bytes(p, 1), dtype=torch.uint8, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+
+    def step():
+        gsa.gsa_fwd(p, q, k, v, gate, o=o, ok_save=ok, ws=ws_f, dev_status=status)
+        gsa.gsa_bwd(p, q, k, v, gate, dO, ok_saved=ok, dq=dq, dk=dk_, dv=dv_, dgate=dg, ws=ws_b, dev_status=status)
+
+    step()
+    torch.cuda.synchronize()
+    eager = [t.clone() for t in (o, dq, dk_, dv_, dg)]
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        step()
+    for t in (o, dq, dk_, dv_, dg):
+        t.zero_()
+    graph.replay()
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    for a, b in zip(eager, (o, dq, dk_, dv_, dg)):
+        assert torch.equal(a, b)
+
+
 def test_fwd_tc_matches_simt_closely():
     # same inputs through both kernel families: they differ only by bf16 operand rounding
     B, T, H, dk, dv, m = 1, 256, 2, 128, 128, 64
