@@ -16,8 +16,10 @@
  *     gate,dgate,ok [B,T,H,m]; memories and their gradients [B,H,m,d].
  *   - q,k,v,o,dO,dq,dk,dv have the element type `io` (fp32 or bf16); gate, the
  *     slot logits and all memories are always fp32; accumulation is fp32.
- *   - The gate tensor holds a in [0,1] (GSA_GATE_A) or log a <= 0
- *     (GSA_GATE_LOG_A).  Internally log a is clamped to >= -100.
+ *   - The gate tensor holds a in [0,1] (GSA_GATE_A), log a <= 0 (GSA_GATE_LOG_A) or the
+ *     layer's gate pre-activation x with a = sigmoid(x)^(1/tau) (GSA_GATE_LOGITS: Sec. 3.3,
+ *     tau = 8 in the paper; the damped sigmoid is then fused into the gate kernel and
+ *     `dgate` is the gradient with respect to x).  Internally log a is clamped to >= -100.
  *   - `params` is a HOST pointer.  `stream` is a cudaStream_t passed as void*
  *     (NULL = the legacy default stream).  Work is only enqueued; nothing
  *     synchronises with the host, allocates or frees device memory.
@@ -57,7 +59,7 @@ typedef enum {
 } gsa_status_t;
 
 typedef enum { GSA_F32 = 0, GSA_BF16 = 1 } gsa_dtype_t;
-typedef enum { GSA_GATE_A = 0, GSA_GATE_LOG_A = 1 } gsa_gate_t;
+typedef enum { GSA_GATE_A = 0, GSA_GATE_LOG_A = 1, GSA_GATE_LOGITS = 2 } gsa_gate_t;
 
 /* Which kernels serve the d-sized contractions of the chunk passes. */
 typedef enum {
@@ -72,6 +74,7 @@ typedef struct {
     int32_t gate_kind;  /* gsa_gate_t */
     float scale;        /* multiplies the slot logits; 1.0f is the paper's layer */
     int32_t impl;       /* gsa_impl_t */
+    float tau;          /* GSA_GATE_LOGITS only: damping of the gate, a = sigmoid(x)^(1/tau); > 0 */
 } gsa_params_t;
 
 enum { GSA_WS_FWD = 0, GSA_WS_BWD = 1, GSA_WS_DECODE = 2 };

@@ -86,16 +86,28 @@ def _run_split(fn, n_items: int, threads: int | None):
     return nt
 
 
+def gate_from_logits(x, tau):
+    """The layer's damped forget gate (Sec. 3.3): a = sigmoid(x)^(1/tau), and da/dx =
+    a (1 - sigmoid(x)) / tau.  Returns (a, da_dx) in float64."""
+    x = np.asarray(x, dtype=np.float64)
+    sig = 1.0 / (1.0 + np.exp(-x))
+    a = np.power(sig, 1.0 / float(tau))
+    return a, a * (1.0 - sig) / float(tau)
+
+
 def fwd(q, k, v, gate, *, gate_is_log=False, scale=1.0, K0=None, V0=None,
-        bh_range=None, threads=None):
+        bh_range=None, threads=None, gate_is_logits=False, tau=8.0):
     """Eq. 6 over whole sequences.
 
     q,k [B,T,H,d_k]; v [B,T,H,d_v]; gate [B,T,H,m] (a, or log a when
     gate_is_log).  Returns dict(o, ok, KT, VT): outputs, scaled pre-softmax slot
     logits [B,T,H,m], final memories [B,H,m,d].  ``bh_range=(lo, hi)`` restricts
     the work to those flattened (b,h) pairs; the other entries stay zero.
+    With gate_is_logits the gate tensor holds x and a = sigmoid(x)^(1/tau) (Sec. 3.3).
     """
     lib = _load()
+    if gate_is_logits:
+        gate, gate_is_log = gate_from_logits(gate, tau)[0], False
     q = _f64(q); B, T, H, dk = q.shape
     k = _f64(k, (B, T, H, dk))
     v = _f64(v); dv = v.shape[-1]
@@ -116,9 +128,16 @@ def fwd(q, k, v, gate, *, gate_is_log=False, scale=1.0, K0=None, V0=None,
 
 
 def bwd(q, k, v, gate, dO, *, gate_is_log=False, scale=1.0, K0=None, V0=None,
-        dKT=None, dVT=None, bh_range=None, threads=None):
+        dKT=None, dVT=None, bh_range=None, threads=None, gate_is_logits=False, tau=8.0):
     """Reverse sweep of Eq. 6.  Returns dict(dq, dk, dv, dgate, dK0, dV0);
-    dgate is the total derivative w.r.t. the gate tensor as passed."""
+    dgate is the total derivative w.r.t. the gate tensor as passed (with gate_is_logits:
+    w.r.t. x, through a = sigmoid(x)^(1/tau))."""
+    if gate_is_logits:
+        a, da_dx = gate_from_logits(gate, tau)
+        r = bwd(q, k, v, a, dO, gate_is_log=False, scale=scale, K0=K0, V0=V0, dKT=dKT, dVT=dVT,
+                bh_range=bh_range, threads=threads)
+        r["dgate"] = r["dgate"] * da_dx
+        return r
     lib = _load()
     q = _f64(q); B, T, H, dk = q.shape
     k = _f64(k, (B, T, H, dk))
@@ -145,11 +164,13 @@ def bwd(q, k, v, gate, dO, *, gate_is_log=False, scale=1.0, K0=None, V0=None,
 
 
 def decode_step(q, k, v, gate, Kstate, Vstate, *, gate_is_log=False, scale=1.0,
-                threads=None):
+                threads=None, gate_is_logits=False, tau=8.0):
     """One recurrent step of Eq. 6 for S sequences; q,k [S,H,d_k], v [S,H,d_v],
     gate [S,H,m]; Kstate/Vstate [S,H,m,d] float64 C-contiguous arrays updated IN
     PLACE.  Returns o [S,H,d_v]."""
     lib = _load()
+    if gate_is_logits:
+        gate, gate_is_log = gate_from_logits(gate, tau)[0], False
     q = _f64(q); S, H, dk = q.shape
     k = _f64(k, (S, H, dk))
     v = _f64(v); dv = v.shape[-1]

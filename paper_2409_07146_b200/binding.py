@@ -12,7 +12,7 @@ _LIB_PATH = os.path.join(_HERE, "libgsa.so")
 _lib = None
 
 GSA_F32, GSA_BF16 = 0, 1
-GSA_GATE_A, GSA_GATE_LOG_A = 0, 1
+GSA_GATE_A, GSA_GATE_LOG_A, GSA_GATE_LOGITS = 0, 1, 2
 GSA_IMPL_AUTO, GSA_IMPL_SIMT, GSA_IMPL_TC = 0, 1, 2
 GSA_WS_FWD, GSA_WS_BWD, GSA_WS_DECODE = 0, 1, 2
 
@@ -30,7 +30,7 @@ class _CParams(ctypes.Structure):
     _fields_ = [("B", ctypes.c_int32), ("T", ctypes.c_int32), ("H", ctypes.c_int32),
                 ("d_k", ctypes.c_int32), ("d_v", ctypes.c_int32), ("m", ctypes.c_int32),
                 ("io", ctypes.c_int32), ("gate_kind", ctypes.c_int32),
-                ("scale", ctypes.c_float), ("impl", ctypes.c_int32)]
+                ("scale", ctypes.c_float), ("impl", ctypes.c_int32), ("tau", ctypes.c_float)]
 
 
 @dataclass(frozen=True)
@@ -46,12 +46,15 @@ class Params:
     gate_is_log: bool = False
     scale: float = 1.0
     impl: str = "auto"        # "auto" | "simt" | "tc"
+    gate_is_logits: bool = False   # the gate tensor holds x, a = sigmoid(x)^(1/tau)
+    tau: float = 8.0
 
     def c(self) -> _CParams:
         return _CParams(self.B, self.T, self.H, self.d_k, self.d_v, self.m,
                         GSA_BF16 if self.io == "bf16" else GSA_F32,
-                        GSA_GATE_LOG_A if self.gate_is_log else GSA_GATE_A,
-                        float(self.scale), _IMPL[self.impl])
+                        GSA_GATE_LOGITS if self.gate_is_logits else
+                        (GSA_GATE_LOG_A if self.gate_is_log else GSA_GATE_A),
+                        float(self.scale), _IMPL[self.impl], float(self.tau))
 
     @property
     def io_dtype(self) -> torch.dtype:

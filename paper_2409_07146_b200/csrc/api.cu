@@ -22,7 +22,9 @@ gsa_status_t check_params(const gsa_params_t* p, bool need_T) {
     if (p->B < 1 || p->H < 1 || p->d_k < 1 || p->d_v < 1 || p->m < 1) return GSA_ERR_INVALID_ARG;
     if (need_T && p->T < 1) return GSA_ERR_INVALID_ARG;
     if (p->io != GSA_F32 && p->io != GSA_BF16) return GSA_ERR_INVALID_ARG;
-    if (p->gate_kind != GSA_GATE_A && p->gate_kind != GSA_GATE_LOG_A) return GSA_ERR_INVALID_ARG;
+    if (p->gate_kind != GSA_GATE_A && p->gate_kind != GSA_GATE_LOG_A && p->gate_kind != GSA_GATE_LOGITS)
+        return GSA_ERR_INVALID_ARG;
+    if (p->gate_kind == GSA_GATE_LOGITS && !(p->tau > 0.f)) return GSA_ERR_INVALID_ARG;
     if (p->impl != GSA_IMPL_AUTO && p->impl != GSA_IMPL_SIMT && p->impl != GSA_IMPL_TC)
         return GSA_ERR_INVALID_ARG;
     if (!(p->scale == p->scale)) return GSA_ERR_INVALID_ARG;
@@ -38,6 +40,8 @@ bool use_tc(const gsa_params_t& p) {
     if (p.impl == GSA_IMPL_SIMT) return false;
     return p.io == GSA_BF16 && tc_supported(p.d_k, p.d_v, p.m);
 }
+
+float inv_tau(const gsa_params_t& p) { return p.tau > 0.f ? 1.f / p.tau : 0.f; }
 
 int chunk_of(const gsa_params_t& p) { return use_tc(p) ? tc_chunk() : kChunk; }
 
@@ -228,7 +232,7 @@ gsa_status_t gsa_gate_cumsum(const gsa_params_t* params, const float* gate, floa
     if (!ok_ptr(gate) || !ok_ptr(G) || !ok_ptr(I)) return GSA_ERR_INVALID_ARG;
     const gsa_params_t& p = *params;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    GSA_LAUNCH("gate_cumsum", launch_gate_cumsum(gate, p.gate_kind == GSA_GATE_LOG_A, G, I, p.B, p.T,
+    GSA_LAUNCH("gate_cumsum", launch_gate_cumsum(gate, p.gate_kind, inv_tau(p), G, I, p.B, p.T,
                                                  p.H, p.m, chunk_of(p), nullptr, 1, nullptr, 0, st));
     return GSA_OK;
 }
@@ -251,7 +255,7 @@ gsa_status_t gsa_fwd(const gsa_params_t* params, const void* q, const void* k, c
 
     const int nseg = segments_of(p);
     GSA_CUDA(cudaMemsetAsync(w.strong, 0, sizeof(int) * (size_t)p.B * p.H * nseg, st));
-    GSA_LAUNCH("gate_cumsum", launch_gate_cumsum(gate, p.gate_kind == GSA_GATE_LOG_A, w.G, w.I, p.B, p.T,
+    GSA_LAUNCH("gate_cumsum", launch_gate_cumsum(gate, p.gate_kind, inv_tau(p), w.G, w.I, p.B, p.T,
                                                  p.H, p.m, chunk_of(p), w.strong, nseg, w.Id, p.io == GSA_BF16, st));
     float* ok = ok_save ? ok_save : w.ok;
     // the pipelined kernels leave the row factor of the pass-1 sums to the softmax kernel
@@ -309,7 +313,7 @@ gsa_status_t gsa_bwd(const gsa_params_t* params, const void* q, const void* k, c
     const Slices s = slices(p);
 
     GSA_CUDA(cudaMemsetAsync(w.strong, 0, sizeof(int) * (size_t)p.B * p.H, st));
-    GSA_LAUNCH("gate_cumsum", launch_gate_cumsum(gate, p.gate_kind == GSA_GATE_LOG_A, w.G, w.I, p.B, p.T,
+    GSA_LAUNCH("gate_cumsum", launch_gate_cumsum(gate, p.gate_kind, inv_tau(p), w.G, w.I, p.B, p.T,
                                                  p.H, p.m, chunk_of(p), w.strong, 1, w.Id, p.io == GSA_BF16, st));
     const float* ok = ok_saved;
     const PendingDecay pend = use_tc(p) ? PendingDecay{w.G, w.strong, p.T, p.H, 1} : PendingDecay{nullptr, nullptr, 1, 1, 1};
@@ -355,7 +359,7 @@ gsa_status_t gsa_bwd(const gsa_params_t* params, const void* q, const void* k, c
         GSA_LAUNCH("bwd_dIk_value_side_rev", value_side(p, adIk, 1, w.strong, st, dev_status));
     }
     // forget-gate gradient: reversed cumulative sum over the whole sequence
-    GSA_LAUNCH("gate_grad", launch_gate_grad(w.u, w.I, w.dIk, s.k, w.dIv, s.v, gate, p.gate_kind == GSA_GATE_LOG_A,
+    GSA_LAUNCH("gate_grad", launch_gate_grad(w.u, w.I, w.dIk, s.k, w.dIv, s.v, gate, p.gate_kind, inv_tau(p),
                               dKT, w.KT, dVT, w.VT, p.d_k, p.d_v, w.chunk_tot, dgate, p.B, p.T,
                               p.H, p.m, pend, st, dev_status));
     return GSA_OK;

@@ -100,6 +100,15 @@ struct KeySideArgs {
     int state_only;                   // as in ValueSideArgs
 };
 
+// GSA_GATE_LOGITS: log a = -softplus(-x) / tau (a = sigmoid(x)^(1/tau), Sec. 3.3) and the factor
+// d(log a)/dx = sigmoid(-x) / tau of the gate gradient.
+__device__ __forceinline__ float log_gate_from_logit(float x, float inv_tau) {
+    return -(fmaxf(-x, 0.f) + log1pf(__expf(-fabsf(x)))) * inv_tau;
+}
+__device__ __forceinline__ float dlog_gate_dlogit(float x, float inv_tau) {
+    return inv_tau / (1.f + __expf(x));
+}
+
 // The pipelined tensor-core value_side kernel leaves the row factor of its partial sums --
 // exp(G_i) of a forward run, exp(-G_i) of a time-reversed one -- to the element-wise kernel that
 // consumes them (slot softmax forward / backward, gate gradient), which sums the D/128 slices
@@ -124,7 +133,8 @@ struct PendingDecay {
 // decayed (nullable, bf16 [B,T,H,2M]): rows [high part | rounding residual] of I exp(-G), the
 // input-gate operand of the pipelined tensor-core kernels.  fast_log: take log a with the
 // hardware base-2 logarithm (absolute error 2^-21.4 for a in [0.5, 1], 3 ulp below), for bf16 io.
-cudaError_t launch_gate_cumsum(const float* gate, int gate_is_log, float* G, float* I,
+// gate_kind: gsa_gate_t (a, log a, or logits with inv_tau = 1/tau)
+cudaError_t launch_gate_cumsum(const float* gate, int gate_kind, float inv_tau, float* G, float* I,
                                int B, int T, int H, int M, int chunk, int* strong_flag, int nseg,
                                void* decayed, int fast_log, cudaStream_t st);
 // Segment-parallel scheduling (T cut into nseg segments run as independent sequences): per-segment
@@ -147,7 +157,7 @@ cudaError_t launch_slot_softmax_bwd(const float* ok, const float* dp_part, int n
                                     PendingDecay pend, cudaStream_t st);
 cudaError_t launch_gate_grad(const float* u, const float* I, const float* dIk_part, int nsk,
                              const float* dIv_part, int nsv, const float* gate,
-                             int gate_is_log, const float* dKT, const float* KT,
+                             int gate_kind, float inv_tau, const float* dKT, const float* KT,
                              const float* dVT, const float* VT, int d_k, int d_v,
                              float* chunk_tot, float* dgate, int B, int T, int H, int M,
                              PendingDecay pend, cudaStream_t st, int32_t* dev_status);

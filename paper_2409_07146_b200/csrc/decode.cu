@@ -65,7 +65,7 @@ struct RowVec {
 template <typename IO, int DK, int DV, int M>
 __global__ void __launch_bounds__(kDecodeWarps * 32)
 decode_step_kernel(const IO* __restrict__ q, const IO* __restrict__ k, const IO* __restrict__ v,
-                   const float* __restrict__ gate, int gate_is_log, float scale,
+                   const float* __restrict__ gate, int gate_kind, float inv_tau, float scale,
                    float* __restrict__ Ks, float* __restrict__ Vs, IO* __restrict__ o) {
     constexpr int RPW = M / kDecodeWarps;  // memory rows per warp
     const size_t pair = blockIdx.x;
@@ -85,8 +85,9 @@ decode_step_kernel(const IO* __restrict__ q, const IO* __restrict__ k, const IO*
     float a[RPW], ia[RPW];
 #pragma unroll
     for (int r = 0; r < RPW; ++r) {
-        const float gt = gate[pair * M + warp * RPW + r];
-        if (gate_is_log) { a[r] = __expf(gt); ia[r] = -expm1f(gt); }
+        float gt = gate[pair * M + warp * RPW + r];
+        if (gate_kind == GSA_GATE_LOGITS) gt = log_gate_from_logit(gt, inv_tau);
+        if (gate_kind != GSA_GATE_A) { a[r] = __expf(gt); ia[r] = -expm1f(gt); }
         else { a[r] = gt; ia[r] = 1.f - gt; }
     }
 
@@ -174,11 +175,12 @@ template <typename IO, int DK, int DV>
 static cudaError_t launch_decode_m(const gsa_params_t& p, const IO* q, const IO* k, const IO* v,
                                    const float* gate, float* Ks, float* Vs, IO* o, cudaStream_t st) {
     const unsigned pairs = (unsigned)p.B * (unsigned)p.H;
-    const int is_log = p.gate_kind == GSA_GATE_LOG_A;
+    const int is_log = p.gate_kind;
+    const float inv_tau = p.tau > 0.f ? 1.f / p.tau : 0.f;
     if (p.m == 64)
-        decode_step_kernel<IO, DK, DV, 64><<<pairs, kDecodeWarps * 32, 0, st>>>(q, k, v, gate, is_log, p.scale, Ks, Vs, o);
+        decode_step_kernel<IO, DK, DV, 64><<<pairs, kDecodeWarps * 32, 0, st>>>(q, k, v, gate, is_log, inv_tau, p.scale, Ks, Vs, o);
     else
-        decode_step_kernel<IO, DK, DV, 32><<<pairs, kDecodeWarps * 32, 0, st>>>(q, k, v, gate, is_log, p.scale, Ks, Vs, o);
+        decode_step_kernel<IO, DK, DV, 32><<<pairs, kDecodeWarps * 32, 0, st>>>(q, k, v, gate, is_log, inv_tau, p.scale, Ks, Vs, o);
     return cudaGetLastError();
 }
 

@@ -31,7 +31,7 @@ __device__ __forceinline__ void store_split2(__nv_bfloat16* row, int c, float x0
 
 template <int M>
 __global__ void __launch_bounds__(M * 4, 4) gate_cumsum_kernel(const float* __restrict__ gate,
-                                                            int gate_is_log,
+                                                            int gate_kind, float inv_tau,
                                                             float* __restrict__ G,
                                                             float* __restrict__ I, int T, int H,
                                                             int chunk, int* __restrict__ strong_flag, int nseg,
@@ -47,10 +47,12 @@ __global__ void __launch_bounds__(M * 4, 4) gate_cumsum_kernel(const float* __re
     float2 g[kCumRows], inps[kCumRows];
 #pragma unroll
     for (int i = 0; i < kCumRows; ++i) {
-        const float neutral = gate_is_log ? 0.f : 1.f;
+        // (rows past the end: a = 1, log a = 0)
+        const float neutral = gate_kind == GSA_GATE_LOG_A ? 0.f : (gate_kind == GSA_GATE_LOGITS ? 80.f : 1.f);
         float2 x = make_float2(neutral, neutral);
         if (i < rows) x = *reinterpret_cast<const float2*>(gate + base + (size_t)i * stride);
-        if (gate_is_log) {
+        if (gate_kind == GSA_GATE_LOGITS) x = make_float2(log_gate_from_logit(x.x, inv_tau), log_gate_from_logit(x.y, inv_tau));
+        if (gate_kind != GSA_GATE_A) {
             g[i] = x;
             inps[i] = make_float2(-expm1f(x.x), -expm1f(x.y));
         } else {
@@ -100,7 +102,7 @@ __global__ void __launch_bounds__(M * 4, 4) gate_cumsum_kernel(const float* __re
         }
 }
 
-cudaError_t launch_gate_cumsum(const float* gate, int gate_is_log, float* G, float* I, int B,
+cudaError_t launch_gate_cumsum(const float* gate, int gate_kind, float inv_tau, float* G, float* I, int B,
                                int T, int H, int M, int chunk, int* strong_flag, int nseg, void* decayed, int fast_log,
                                cudaStream_t st) {
     if (chunk % kCumRows != 0 || chunk / kCumRows > 8) return cudaErrorInvalidValue;
@@ -108,10 +110,10 @@ cudaError_t launch_gate_cumsum(const float* gate, int gate_is_log, float* G, flo
     dim3 block(M / 2, chunk / kCumRows);
     dim3 grid(B * H, nchunks);
     if (M == 64)
-        gate_cumsum_kernel<64><<<grid, block, 0, st>>>(gate, gate_is_log, G, I, T, H, chunk, strong_flag, nseg < 1 ? 1 : nseg,
+        gate_cumsum_kernel<64><<<grid, block, 0, st>>>(gate, gate_kind, inv_tau, G, I, T, H, chunk, strong_flag, nseg < 1 ? 1 : nseg,
                                                        static_cast<__nv_bfloat16*>(decayed), fast_log);
     else
-        gate_cumsum_kernel<32><<<grid, block, 0, st>>>(gate, gate_is_log, G, I, T, H, chunk, strong_flag, nseg < 1 ? 1 : nseg,
+        gate_cumsum_kernel<32><<<grid, block, 0, st>>>(gate, gate_kind, inv_tau, G, I, T, H, chunk, strong_flag, nseg < 1 ? 1 : nseg,
                                                        static_cast<__nv_bfloat16*>(decayed), fast_log);
     return cudaGetLastError();
 }
@@ -327,6 +329,24 @@ cudaError_t launch_slot_softmax_bwd(const float* ok, const float* dp_part, int n
 
 constexpr int kGG = 16;   // rows per thread of the gate-gradient kernels
 
+// From the decay-path gradient d(log a) (`run`: what this block knows of it) and the input-gate
+// gradient dI to the gradient with respect to the gate tensor as passed (`gt`):
+//   a       : run / a - dI            (a == 0 leaves no way back from d(log a): only -dI is kept)
+//   log a   : run - a dI
+//   logits  : (run - a dI) sigmoid(-x) / tau
+__device__ __forceinline__ float gate_grad_out(float run, float dI, float gt, int gate_kind, float inv_tau) {
+    if (gate_kind == GSA_GATE_A) return (gt > 0.f) ? run / gt - dI : -dI;
+    if (gate_kind == GSA_GATE_LOG_A) return run - __expf(fmaxf(gt, kLogGateMin)) * dI;
+    const float a = __expf(fmaxf(log_gate_from_logit(gt, inv_tau), kLogGateMin));
+    return (run - a * dI) * dlog_gate_dlogit(gt, inv_tau);
+}
+// the carry of the blocks after this one, in the same units
+__device__ __forceinline__ float gate_grad_carry(float carry, float gt, int gate_kind, float inv_tau) {
+    if (gate_kind == GSA_GATE_A) return (gt > 0.f) ? carry / gt : 0.f;
+    if (gate_kind == GSA_GATE_LOG_A) return carry;
+    return carry * dlog_gate_dlogit(gt, inv_tau);
+}
+
 // dI[i] = sum over the d_k and d_v slices of the input-gate gradient partial sums, for the
 // kGG rows x 2 slots of this thread; the rows of one slice are loaded together (16 loads of 8
 // bytes in flight).
@@ -386,7 +406,7 @@ __global__ void __launch_bounds__(M * 16) gate_grad_scan_kernel(
 template <int M>
 __global__ void __launch_bounds__(128) gate_grad_local_kernel(
     const float* __restrict__ u, const float* __restrict__ I, const float* __restrict__ dIk, int nsk,
-    const float* __restrict__ dIv, int nsv, const float* __restrict__ gate, int gate_is_log,
+    const float* __restrict__ dIv, int nsv, const float* __restrict__ gate, int gate_kind, float inv_tau,
     float* __restrict__ blk_tot, float* __restrict__ dgate, int B, int T, int H, int nblk, PendingDecay pend) {
     const int s = 2 * threadIdx.x;                       // this thread's two slots
     const int n = blockIdx.y * blockDim.y + threadIdx.y;
@@ -424,15 +444,8 @@ __global__ void __launch_bounds__(128) gate_grad_local_kernel(
         run0 += x[i].x;
         run1 += x[i].y;
         if (i < rows) {
-            float2 out;
-            if (gate_is_log) {
-                out.x = run0 - __expf(fmaxf(gt[i].x, kLogGateMin)) * dI[i].x;
-                out.y = run1 - __expf(fmaxf(gt[i].y, kLogGateMin)) * dI[i].y;
-            } else {
-                // a == 0 leaves no way back from d(log a) to da: only the input-gate part is kept
-                out.x = (gt[i].x > 0.f) ? run0 / gt[i].x - dI[i].x : -dI[i].x;
-                out.y = (gt[i].y > 0.f) ? run1 / gt[i].y - dI[i].y : -dI[i].y;
-            }
+            const float2 out = make_float2(gate_grad_out(run0, dI[i].x, gt[i].x, gate_kind, inv_tau),
+                                           gate_grad_out(run1, dI[i].y, gt[i].y, gate_kind, inv_tau));
             *reinterpret_cast<float2*>(dgate + base + (size_t)i * stride) = out;
         }
     }
@@ -452,7 +465,7 @@ __global__ void __launch_bounds__(64) gate_grad_local_tma_kernel(
     const __grid_constant__ CUtensorMap mapU, const __grid_constant__ CUtensorMap mapI,
     const __grid_constant__ CUtensorMap mapGate, const __grid_constant__ CUtensorMap mapG,
     const __grid_constant__ CUtensorMap mapDIk, const __grid_constant__ CUtensorMap mapDIv, int nsk, int nsv,
-    int gate_is_log, float* __restrict__ blk_tot, float* __restrict__ dgate, int T, int H, int nblk,
+    int gate_kind, float inv_tau, float* __restrict__ blk_tot, float* __restrict__ dgate, int T, int H, int nblk,
     const int* __restrict__ strong, int32_t* dev_status) {
     using namespace tc;
     constexpr int M = 64;
@@ -527,15 +540,8 @@ __global__ void __launch_bounds__(64) gate_grad_local_tma_kernel(
         run1 += x[i].y;
         if (i < rows) {
             const float2 gt = at(2, i);
-            float2 out;
-            if (gate_is_log) {
-                out.x = run0 - __expf(fmaxf(gt.x, kLogGateMin)) * dI[i].x;
-                out.y = run1 - __expf(fmaxf(gt.y, kLogGateMin)) * dI[i].y;
-            } else {
-                // a == 0 leaves no way back from d(log a) to da: only the input-gate part is kept
-                out.x = (gt.x > 0.f) ? run0 / gt.x - dI[i].x : -dI[i].x;
-                out.y = (gt.y > 0.f) ? run1 / gt.y - dI[i].y : -dI[i].y;
-            }
+            const float2 out = make_float2(gate_grad_out(run0, dI[i].x, gt.x, gate_kind, inv_tau),
+                                           gate_grad_out(run1, dI[i].y, gt.y, gate_kind, inv_tau));
             *reinterpret_cast<float2*>(dgate + base + (size_t)i * stride) = out;
         }
     }
@@ -545,7 +551,7 @@ __global__ void __launch_bounds__(64) gate_grad_local_tma_kernel(
 // Adds what follows the block: dgate += carry (log gate) or carry / a (linear gate).
 template <int M>
 __global__ void __launch_bounds__(128) gate_grad_carry_kernel(
-    const float* __restrict__ gate, int gate_is_log, const float* __restrict__ blk_carry,
+    const float* __restrict__ gate, int gate_kind, float inv_tau, const float* __restrict__ blk_carry,
     float* __restrict__ dgate, int T, int H, int nblk) {
     const int s = 2 * threadIdx.x;
     const int n = blockIdx.y * blockDim.y + threadIdx.y;
@@ -560,15 +566,15 @@ __global__ void __launch_bounds__(128) gate_grad_carry_kernel(
 #pragma unroll
     for (int i = 0; i < kGG; ++i) {
         d[i] = (i < rows) ? *reinterpret_cast<const float2*>(dgate + base + (size_t)i * stride) : make_float2(0.f, 0.f);
-        gt[i] = (i < rows && !gate_is_log) ? *reinterpret_cast<const float2*>(gate + base + (size_t)i * stride)
-                                           : make_float2(1.f, 1.f);
+        gt[i] = (i < rows && gate_kind != GSA_GATE_LOG_A) ? *reinterpret_cast<const float2*>(gate + base + (size_t)i * stride)
+                                                          : make_float2(1.f, 1.f);
     }
 #pragma unroll
     for (int i = 0; i < kGG; ++i)
         if (i < rows) {
             float2 out;
-            out.x = d[i].x + ((gate_is_log || gt[i].x > 0.f) ? carry.x / gt[i].x : 0.f);
-            out.y = d[i].y + ((gate_is_log || gt[i].y > 0.f) ? carry.y / gt[i].y : 0.f);
+            out.x = d[i].x + gate_grad_carry(carry.x, gt[i].x, gate_kind, inv_tau);
+            out.y = d[i].y + gate_grad_carry(carry.y, gt[i].y, gate_kind, inv_tau);
             *reinterpret_cast<float2*>(dgate + base + (size_t)i * stride) = out;
         }
 }
@@ -577,7 +583,7 @@ int gate_grad_blocks(int T) { return (T + kGG - 1) / kGG; }
 
 cudaError_t launch_gate_grad(const float* u, const float* I, const float* dIk_part, int nsk,
                              const float* dIv_part, int nsv, const float* gate,
-                             int gate_is_log, const float* dKT, const float* KT,
+                             int gate_kind, float inv_tau, const float* dKT, const float* KT,
                              const float* dVT, const float* VT, int d_k, int d_v,
                              float* blk_tot, float* dgate, int B, int T, int H, int M,
                              PendingDecay pend, cudaStream_t st, int32_t* dev_status) {
@@ -604,20 +610,20 @@ cudaError_t launch_gate_grad(const float* u, const float* I, const float* dIk_pa
                                                  (int)smem);
             if (e != cudaSuccess) return e;
             dim3 tgrid(B * H, (T + kGGTmaRows - 1) / kGGTmaRows);
-            gate_grad_local_tma_kernel<<<tgrid, 64, smem, st>>>(mu, mi, mg, mG, mk, mv, nsk, nsv, gate_is_log, blk_tot,
+            gate_grad_local_tma_kernel<<<tgrid, 64, smem, st>>>(mu, mi, mg, mG, mk, mv, nsk, nsv, gate_kind, inv_tau, blk_tot,
                                                                 dgate, T, H, nblk, pend.G != nullptr ? pend.strong : nullptr,
                                                                 dev_status);
         } else {
-            gate_grad_local_kernel<64><<<grid, block, 0, st>>>(u, I, dIk_part, nsk, dIv_part, nsv, gate, gate_is_log,
+            gate_grad_local_kernel<64><<<grid, block, 0, st>>>(u, I, dIk_part, nsk, dIv_part, nsv, gate, gate_kind, inv_tau,
                                                                blk_tot, dgate, B, T, H, nblk, pend);
         }
         gate_grad_scan_kernel<64><<<B * H, dim3(64, 16), 0, st>>>(blk_tot, dKT, KT, dVT, VT, d_k, d_v, nblk);
-        gate_grad_carry_kernel<64><<<grid, block, 0, st>>>(gate, gate_is_log, blk_tot, dgate, T, H, nblk);
+        gate_grad_carry_kernel<64><<<grid, block, 0, st>>>(gate, gate_kind, inv_tau, blk_tot, dgate, T, H, nblk);
     } else {
-        gate_grad_local_kernel<32><<<grid, block, 0, st>>>(u, I, dIk_part, nsk, dIv_part, nsv, gate, gate_is_log,
+        gate_grad_local_kernel<32><<<grid, block, 0, st>>>(u, I, dIk_part, nsk, dIv_part, nsv, gate, gate_kind, inv_tau,
                                                            blk_tot, dgate, B, T, H, nblk, pend);
         gate_grad_scan_kernel<32><<<B * H, dim3(32, 16), 0, st>>>(blk_tot, dKT, KT, dVT, VT, d_k, d_v, nblk);
-        gate_grad_carry_kernel<32><<<grid, block, 0, st>>>(gate, gate_is_log, blk_tot, dgate, T, H, nblk);
+        gate_grad_carry_kernel<32><<<grid, block, 0, st>>>(gate, gate_kind, inv_tau, blk_tot, dgate, T, H, nblk);
     }
     return cudaGetLastError();
 }

@@ -340,3 +340,49 @@ def test_bwd_tc_strong_forgetting_saved_logits():
     # (p dp + o' do' - (1-a) dI) cancel almost completely: the bf16 roundings of their factors
     # are what is left, hence the wider bound on this stress case
     check_bwd(got, ref, 4 * TOL["bf16"], tc=True)
+
+
+# ------------------------------------------------------------------ gate from logits (Sec. 3.3)
+@pytest.mark.parametrize("io,impl", [("f32", "auto"), ("bf16", "simt"), ("bf16", "tc")])
+def test_logit_gate_fwd_bwd(io, impl):
+    # the gate tensor holds the pre-activation x; a = sigmoid(x)^(1/8) is formed in the gate kernel
+    # and dgate is the gradient w.r.t. x
+    B, T, H, dk, dv, m = 2, 200, 2, 128, 128, 64
+    d = rand_inputs(901, B, T, H, dk, dv, m, io, init=True)
+    x = (2.0 * np.random.default_rng(5).standard_normal((B, T, H, m))).astype(np.float32)
+    x[0, 3, 0, 0] = 60.0      # a = 1 to rounding
+    x[0, 4, 0, 1] = -60.0     # a = e^-7.5
+    p = gsa.Params(B, T, H, dk, dv, m, io=io, impl=impl, gate_is_logits=True, tau=8.0)
+    q, k, v, dO = (to_dev(d[n], io) for n in ("q", "k", "v", "dO"))
+    K0, V0 = to_dev(d["K0"]), to_dev(d["V0"])
+    KT = torch.empty(B, H, m, dk, device="cuda"); VT = torch.empty(B, H, m, dv, device="cuda")
+    ok = torch.empty(B, T, H, m, device="cuda")
+    o = gsa.gsa_fwd(p, q, k, v, to_dev(x), K0, V0, ok_save=ok, KT=KT, VT=VT)
+    dq, dk_, dv_, dg = gsa.gsa_bwd(p, q, k, v, to_dev(x), dO, K0, V0, ok_saved=ok)
+    torch.cuda.synchronize()
+    rf = oracle.fwd(d["q"], d["k"], d["v"], x, K0=d["K0"], V0=d["V0"], gate_is_logits=True, tau=8.0)
+    rb = oracle.bwd(d["q"], d["k"], d["v"], x, d["dO"], K0=d["K0"], V0=d["V0"], gate_is_logits=True, tau=8.0)
+    got = dict(o=to_np(o), ok=to_np(ok), KT=to_np(KT), VT=to_np(VT), dq=to_np(dq), dk=to_np(dk_),
+               dv=to_np(dv_), dgate=to_np(dg))
+    ref = dict(rf, **rb)
+    tc = impl == "tc"
+    errs = {n: (mixed_err(got[n], ref[n], TC_RTOL) if tc else rel_err(got[n], ref[n], io == "bf16" and n in BF16_IO))
+            for n in got}
+    assert all(e <= TOL[io] for e in errs.values()), errs
+
+
+def test_logit_gate_decode():
+    S, H, dk, dv, m = 3, 4, 128, 128, 64
+    w = W.CONFIGS["decode"].scaled(B=S, H=H, d_k=dk, d_v=dv, m=m, io="bf16")
+    st = W.make_decode_states(w)
+    Ks, Vs = to_dev(st["K"]), to_dev(st["V"])
+    Kr, Vr = st["K"].astype(np.float64), st["V"].astype(np.float64)
+    p = gsa.Params(S, 1, H, dk, dv, m, io="bf16", gate_is_logits=True, tau=8.0)
+    for step in range(3):
+        x = W.make_decode_step_inputs(w, step)
+        logits = (3.0 * np.random.default_rng(step).standard_normal(x["gate"].shape)).astype(np.float32)
+        o = gsa.gsa_decode_step(p, to_dev(x["q"], "bf16"), to_dev(x["k"], "bf16"), to_dev(x["v"], "bf16"),
+                                to_dev(logits), Ks, Vs)
+        ro = oracle.decode_step(x["q"], x["k"], x["v"], logits, Kr, Vr, gate_is_logits=True, tau=8.0)
+        assert rel_err(to_np(o), ro, True) <= TOL["bf16"]
+    assert rel_err(to_np(Ks), Kr) <= 1e-5 and rel_err(to_np(Vs), Vr) <= 1e-5

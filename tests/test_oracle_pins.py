@@ -255,3 +255,52 @@ def test_chunkwise_backward_and_gate_identity_equal_sweep(C, with_final):
     np.testing.assert_allclose(ch["dg"], glog["dgate"][0, :, 0], atol=1e-10)
     np.testing.assert_allclose(ch["dK0"], g["dK0"][0, 0], atol=1e-11)
     np.testing.assert_allclose(ch["dV0"], g["dV0"][0, 0], atol=1e-11)
+
+
+# ------------------------------------------------------------------ gate from logits (Sec. 3.3)
+def test_logit_gate_equals_explicit_damped_sigmoid_and_chain_rule():
+    # a = sigmoid(x)^(1/tau): the logits mode must equal the linear-gate mode fed with that a, and
+    # its gate gradient the linear one times da/dx; tau = 1 is the plain sigmoid
+    r = np.random.default_rng(11)
+    B, T, H, d, m = 2, 9, 2, 4, 3
+    q, k, v, dO = (r.standard_normal((B, T, H, d)) for _ in range(4))
+    x = 2.0 * r.standard_normal((B, T, H, m))
+    for tau in (1.0, 8.0):
+        sig = 1.0 / (1.0 + np.exp(-x))
+        a = sig ** (1.0 / tau)
+        f_log, f_lin = oracle.fwd(q, k, v, x, gate_is_logits=True, tau=tau), oracle.fwd(q, k, v, a)
+        for n in ("o", "ok", "KT", "VT"):
+            assert np.abs(f_log[n] - f_lin[n]).max() < 1e-13
+        b_log = oracle.bwd(q, k, v, x, dO, gate_is_logits=True, tau=tau)
+        b_lin = oracle.bwd(q, k, v, a, dO)
+        for n in ("dq", "dk", "dv"):
+            assert np.abs(b_log[n] - b_lin[n]).max() < 1e-13
+        assert np.abs(b_log["dgate"] - b_lin["dgate"] * a * (1 - sig) / tau).max() < 1e-12
+
+
+def test_logit_gate_gradient_matches_central_finite_differences():
+    r = np.random.default_rng(12)
+    B, T, H, d, m = 1, 7, 1, 3, 2
+    q, k, v, dO = (r.standard_normal((B, T, H, d)) for _ in range(4))
+    x = r.standard_normal((B, T, H, m))
+    f = lambda x_: float((oracle.fwd(q, k, v, x_, gate_is_logits=True, tau=8.0)["o"] * dO).sum())
+    g = oracle.bwd(q, k, v, x, dO, gate_is_logits=True, tau=8.0)["dgate"]
+    eps = 1e-6
+    for idx in np.ndindex(*x.shape):
+        xp, xm = x.copy(), x.copy()
+        xp[idx] += eps
+        xm[idx] -= eps
+        assert abs((f(xp) - f(xm)) / (2 * eps) - g[idx]) < 1e-7
+
+
+def test_logit_gate_decode_steps_reproduce_forward():
+    r = np.random.default_rng(13)
+    S, T, H, d, m = 2, 5, 2, 4, 3
+    q, k, v = (r.standard_normal((S, T, H, d)) for _ in range(3))
+    x = r.standard_normal((S, T, H, m))
+    ref = oracle.fwd(q, k, v, x, gate_is_logits=True, tau=8.0)
+    Ks, Vs = np.zeros((S, H, m, d)), np.zeros((S, H, m, d))
+    for t in range(T):
+        o = oracle.decode_step(q[:, t], k[:, t], v[:, t], x[:, t], Ks, Vs, gate_is_logits=True, tau=8.0)
+        assert np.abs(o - ref["o"][:, t]).max() < 1e-13
+    assert np.abs(Ks - ref["KT"]).max() < 1e-13
