@@ -456,12 +456,12 @@ __global__ void __launch_bounds__(128) gate_grad_local_kernel(
 // CTA per (b,h) and 32 rows, every tile of every input stream (u, I, gate, G and the n_k + n_v
 // slices of the input-gate gradient: 12 x 8 KB at d = 512) requested at once by one thread --
 // 96 KB in flight per CTA, two CTAs per SM, several times what registers can hold as landing
-// space.  Thread = (slot pair, 16-row group), as above.
+// space.  Thread = (slot, 16-row group, early or late half of the group).
 constexpr int kGGTmaRows = 32;
 constexpr int kGGTmaMaxSlices = 8;
 constexpr int kGGTileB = kGGTmaRows * 64 * 4;      // bytes of one [32 x 64] fp32 tile (two swizzled panels)
 
-__global__ void __launch_bounds__(64) gate_grad_local_tma_kernel(
+__global__ void __launch_bounds__(256) gate_grad_local_tma_kernel(
     const __grid_constant__ CUtensorMap mapU, const __grid_constant__ CUtensorMap mapI,
     const __grid_constant__ CUtensorMap mapGate, const __grid_constant__ CUtensorMap mapG,
     const __grid_constant__ CUtensorMap mapDIk, const __grid_constant__ CUtensorMap mapDIv, int nsk, int nsv,
@@ -472,7 +472,9 @@ __global__ void __launch_bounds__(64) gate_grad_local_tma_kernel(
     extern __shared__ unsigned char gg_smem_raw[];
     unsigned char* smem = gg_smem_raw + ((1024u - (smem_u32(gg_smem_raw) & 1023u)) & 1023u);
     __shared__ uint64_t bar;
-    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;       // slot pair, 16-row group
+    __shared__ float late_half[kGGTmaRows / kGG][M];
+    // slot, 16-row group, early (0) or late (1) 8 rows of the group
+    const int tx = threadIdx.x & 63, ty = (threadIdx.x >> 6) & 1, hh = threadIdx.x >> 7;
     const int bh = blockIdx.x, b = bh / H, h = bh % H;
     const int t0 = blockIdx.y * kGGTmaRows;
     const int nslices = nsk + nsv;
@@ -497,55 +499,45 @@ __global__ void __launch_bounds__(64) gate_grad_local_tma_kernel(
     if (!landed && threadIdx.x == 0 && dev_status != nullptr) *dev_status = GSA_ERR_TIMEOUT;
     if (__syncthreads_or(!landed)) return;
 
+    constexpr int kHalf = kGG / 2;
     const int n = blockIdx.y * (kGGTmaRows / kGG) + ty;           // 16-row block of the sequence
-    if (n >= nblk) return;
-    const int rows = min(kGG, T - n * kGG);
-    // row r (of this thread's 16), this thread's two slots, of tile `tile`
+    const int rows = n < nblk ? min(kGG, T - n * kGG) : 0;
+    // row r (of this thread's 16), this thread's slot, of tile `tile`
     auto at = [&](int tile, int r) {
-        const int row = ty * kGG + r, c = 2 * tx;
+        const int row = ty * kGG + hh * kHalf + r, c = tx;
         const unsigned char* p = smem + tile * kGGTileB + (c >> 5) * (kGGTileB / 2) + swz128(row, (c & 31) >> 2) + (c & 3) * 4;
-        return *reinterpret_cast<const float2*>(p);
+        return *reinterpret_cast<const float*>(p);
     };
-    float2 x[kGG], dI[kGG];
+    float x[kHalf], dI[kHalf];
 #pragma unroll
-    for (int i = 0; i < kGG; ++i) dI[i] = make_float2(0.f, 0.f);
+    for (int i = 0; i < kHalf; ++i) dI[i] = 0.f;
     for (int sl = 0; sl < nslices; ++sl) {
 #pragma unroll
-        for (int i = 0; i < kGG; ++i) {
-            const float2 t = at(4 + sl, i);
-            dI[i].x += t.x;
-            dI[i].y += t.y;
-        }
+        for (int i = 0; i < kHalf; ++i) dI[i] += at(4 + sl, i);
     }
     if (strong != nullptr && strong[bh] == 0) {
         // the time-reversed value_side runs left their row factor exp(-G_i) to this kernel
 #pragma unroll
-        for (int i = 0; i < kGG; ++i) {
-            const float2 g = at(3, i);
-            dI[i].x *= __expf(-g.x);
-            dI[i].y *= __expf(-g.y);
-        }
+        for (int i = 0; i < kHalf; ++i) dI[i] *= __expf(-at(3, i));
     }
 #pragma unroll
-    for (int i = 0; i < kGG; ++i) {
-        const float2 uu = at(0, i), ii = at(1, i);
-        x[i] = make_float2(uu.x - ii.x * dI[i].x, uu.y - ii.y * dI[i].y);       // rows past the end: all zero
-    }
+    for (int i = 0; i < kHalf; ++i) x[i] = at(0, i) - at(1, i) * dI[i];       // rows past the end: all zero
     const size_t stride = (size_t)H * M;
-    const size_t base = (((size_t)b * T + n * kGG) * H + h) * M + 2 * tx;
-    float run0 = 0.f, run1 = 0.f;
+    const size_t base = (((size_t)b * T + n * kGG + hh * kHalf) * H + h) * M + tx;
+    // the early half starts from the total of the late half of its group
+    float tot = 0.f;
 #pragma unroll
-    for (int i = kGG - 1; i >= 0; --i) {
-        run0 += x[i].x;
-        run1 += x[i].y;
-        if (i < rows) {
-            const float2 gt = at(2, i);
-            const float2 out = make_float2(gate_grad_out(run0, dI[i].x, gt.x, gate_kind, inv_tau),
-                                           gate_grad_out(run1, dI[i].y, gt.y, gate_kind, inv_tau));
-            *reinterpret_cast<float2*>(dgate + base + (size_t)i * stride) = out;
-        }
+    for (int i = 0; i < kHalf; ++i) tot += x[i];
+    if (hh == 1) late_half[ty][tx] = tot;
+    __syncthreads();
+    float run = hh == 0 ? late_half[ty][tx] : 0.f;
+#pragma unroll
+    for (int i = kHalf - 1; i >= 0; --i) {
+        run += x[i];
+        if (hh * kHalf + i < rows)
+            dgate[base + (size_t)i * stride] = gate_grad_out(run, dI[i], at(2, i), gate_kind, inv_tau);
     }
-    *reinterpret_cast<float2*>(blk_tot + ((size_t)bh * nblk + n) * M + 2 * tx) = make_float2(run0, run1);
+    if (hh == 0 && n < nblk) blk_tot[((size_t)bh * nblk + n) * M + tx] = run;
 }
 
 // Adds what follows the block: dgate += carry (log gate) or carry / a (linear gate).
@@ -610,7 +602,7 @@ cudaError_t launch_gate_grad(const float* u, const float* I, const float* dIk_pa
                                                  (int)smem);
             if (e != cudaSuccess) return e;
             dim3 tgrid(B * H, (T + kGGTmaRows - 1) / kGGTmaRows);
-            gate_grad_local_tma_kernel<<<tgrid, 64, smem, st>>>(mu, mi, mg, mG, mk, mv, nsk, nsv, gate_kind, inv_tau, blk_tot,
+            gate_grad_local_tma_kernel<<<tgrid, 256, smem, st>>>(mu, mi, mg, mG, mk, mv, nsk, nsv, gate_kind, inv_tau, blk_tot,
                                                                 dgate, T, H, nblk, pend.G != nullptr ? pend.strong : nullptr,
                                                                 dev_status);
         } else {
