@@ -42,8 +42,8 @@ NCU_TRAFFIC = {
     "bwd_dIv_value_side_rev": 188307968, "bwd_dIk_value_side_rev": 190506744,
     "pass2_key_side": 129381884, "bwd_dq_key_side": 136861688,
     "bwd_dv_key_side_rev": 130355960, "bwd_dk_key_side_rev": 132610046,
-    "gate_cumsum": 18483712, "slot_softmax": 101182208, "slot_softmax_bwd": 140176126,
-    "gate_grad": 251560184,     # local + scan + carry
+    "gate_cumsum": 27124480, "slot_softmax": 100435968, "slot_softmax_bwd": 137995774,
+    "gate_grad": 250950394,     # local + scan + carry
 }
 
 
