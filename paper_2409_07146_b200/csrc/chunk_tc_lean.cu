@@ -459,7 +459,7 @@ key_side_lean_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_cons
         // =============================== MMA lane
         constexpr uint32_t idescA = make_idesc(128, 128, false, false);   // Q~ K~^T
         constexpr uint32_t idescO = make_idesc(128, kDST, false, false);  // Q~ x state copy (K-major B)
-        constexpr uint32_t idescU = make_idesc(128, kM, true, true);      // xv^T (MN-major A) x K~ (MN-major B)
+        constexpr uint32_t idescU = make_idesc(128, 2 * kM, true, true);  // xv^T (MN-major A) x [K~_hi | K~_lo] (MN-major B)
         constexpr uint32_t idescV = make_idesc(128, kDST, false, true);   // A x xv (MN-major B)
         const uint64_t dS = desc_kmajor(smem_u32(sSb), 0), dSl = desc_kmajor(smem_u32(sSb + kPanelB), 0);
         auto kmaj = [](int kk) { return (uint32_t)((kk >> 2) * kPanelB + (kk & 3) * 32); };
@@ -491,7 +491,9 @@ key_side_lean_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_cons
             const uint32_t accO = tmem + kLkO + 128 * (n & 1);
             const uint32_t qk = smem_u32(sQK + 4 * (n & 1) * kPanelB);
             const uint64_t dQt = desc_kmajor(qk, 0), dQl = desc_kmajor(qk + 2 * kPanelB, 0);
-            const uint64_t dKtm = desc_mnmajor(qk + kPanelB, 0, kPanelB);   // the decayed uk read MN-major
+            // the decayed uk read MN-major, its high and low parts as one N = 128 operand (the panels
+            // of a stage are [uq_hi, uk_hi, uq_lo, uk_lo]: the low part is two panels on)
+            const uint64_t dKtm = desc_mnmajor(qk + kPanelB, 0, 2 * kPanelB);
             PROF_MARK();
             // state products of chunk n: the state copy was written at the end of chunk n-1 (which also
             // says that the accumulators they overwrite have been read)
@@ -581,8 +583,11 @@ key_side_lean_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_cons
             LEAN_WAIT(&ctl->bar_mma1, n & 1);
             tc_fence_after_sync();
             {
-                float v[kHS];
+                float v[kHS], vl[kHS];
                 tmem_ld32(tmem_row_addr(tmem, wq, kLkU + sb), v);
+                tmem_ld32(tmem_row_addr(tmem, wq, kLkU + kM + sb), vl);
+#pragma unroll
+                for (int e = 0; e < kHS; ++e) v[e] += vl[e];          // high + low part of the decayed uk
 #pragma unroll
                 for (int e = 0; e < kHS; e += 4) {
                     const float4 ec = *reinterpret_cast<const float4*>(&egc[sb + e]);
