@@ -133,7 +133,7 @@ __device__ __forceinline__ bool publish_and_vote(uint64_t* bar, int tid, bool st
 }
 
 // accumulator columns of the lean kernels
-constexpr int kLvP = 0, kLvO = 128 /* two buffers of 64 */, kLvU = 256, kLvI = 384;     // value_side
+constexpr int kLvP = 0, kLvO = 128 /* high | low state part */, kLvU = 256, kLvI = 384;     // value_side
 constexpr int kLkA = 0, kLkO = 128 /* two buffers of 128 */, kLkU = 384;                 // key_side
 
 // ======================================================================================
@@ -154,8 +154,8 @@ value_side_lean_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_co
     unsigned char* sWd = sX + 8 * kPanelB;           // decayed weights, MN-major B [128][hi 64 | lo 64], 2 stages (64 KB)
                                                      //   ... a stage also holds the chunk's output rows (fp32, 2
                                                      //   panels of 32 slots) once its weights are consumed
-    unsigned char* sSb = sWd + 4 * kPanelB;          // state copy, MN-major B [128][64]          (16 KB)
-    LeanCtl* ctl = reinterpret_cast<LeanCtl*>(sSb + kPanelB);
+    unsigned char* sSb = sWd + 4 * kPanelB;          // state copy, MN-major B [128][hi 64 | lo 64] (32 KB)
+    LeanCtl* ctl = reinterpret_cast<LeanCtl*>(sSb + 2 * kPanelB);
 
     const int tid = threadIdx.x, warp = tid >> 5, wq = warp & 3, half = (tid >> 7) & 1, row = tid & 127;
     const int sb = kHS * half;          // this thread's first slot
@@ -216,7 +216,7 @@ value_side_lean_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_co
     } else if (tid == kMmaThread) {
         // =============================== MMA lane
         constexpr uint32_t idescP = make_idesc(128, 128, false, false);    // xq xk^T
-        constexpr uint32_t idescO = make_idesc(128, kM, false, true);      // xq x state copy (MN-major B)
+        constexpr uint32_t idescO = make_idesc(128, 2 * kM, false, true);  // xq x state copy [S_hi | S_lo] (MN-major B)
         constexpr uint32_t idescU = make_idesc(128, 2 * kM, true, true);   // xk^T (MN-major A) x [W_hi | W_lo]
         constexpr uint32_t idescI = make_idesc(128, 2 * kM, false, true);  // masked P (tensor memory) x [W_hi | W_lo]
         const uint64_t dS = desc_mnmajor(smem_u32(sSb), 0, kPanelB);
@@ -251,10 +251,16 @@ value_side_lean_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_co
 #pragma unroll
             for (int kk = 0; kk < kCT / 16; ++kk)
                 mma_bf16(tmem + kLvU, desc_advance(dKm, mnmaj(kk)), desc_advance(dW, mnmaj(kk)), idescU, kk > 0);
+            // the inter-chunk output accumulator is single: the previous chunk's output rows must have
+            // been read out (by now they almost always are: this is issued after that chunk's intra
+            // product and the next first product)
+            if (n >= 1) {
+                LEAN_WAIT(&ctl->bar_out[(n - 1) & 1], ((n - 1) >> 1) & 1);
+                tc_fence_after_sync();
+            }
 #pragma unroll
             for (int kk = 0; kk < kDST / 16; ++kk)
-                mma_bf16(tmem + kLvO + 64 * (n & 1), desc_advance(dQk, kmaj(kk)), desc_advance(dS, mnmaj(kk)), idescO,
-                         kk > 0);
+                mma_bf16(tmem + kLvO, desc_advance(dQk, kmaj(kk)), desc_advance(dS, mnmaj(kk)), idescO, kk > 0);
             mma_commit(&ctl->bar_mma1);
             mma_commit(&ctl->bar_free1[n & 1]);
             PROF_MARK();
@@ -288,7 +294,7 @@ value_side_lean_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_co
         float S[kHS];
 #pragma unroll
         for (int s = 0; s < kHS; ++s) S[s] = a.S0 ? a.S0[((size_t)bh * kM + sb + s) * a.D + d0 + row] : 0.f;
-        store_state_row<false>(sSb, row, sb, S, nullptr);
+        store_state_row_split<false>(sSb, sSb + kPanelB, row, sb, S, nullptr);
 
         // G of the last valid row of chunk n (threads 0..63, one slot each), one chunk ahead
         auto chunk_gc = [&](int n) {
@@ -340,7 +346,7 @@ value_side_lean_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_co
                     }
                 }
             }
-            store_state_row<false>(sSb, row, sb, S, nullptr);
+            store_state_row_split<false>(sSb, sSb + kPanelB, row, sb, S, nullptr);
             publish(&ctl->bar_sb, tid);
             PROF_MARK();
 
@@ -355,7 +361,11 @@ value_side_lean_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_co
                 tmem_ld32(tmem_row_addr(tmem, wq, kLvI + kM + sb), vi);
 #pragma unroll
                 for (int e = 0; e < kHS; ++e) vo[e] += vi[e];          // high + low weight parts
-                tmem_ld32(tmem_row_addr(tmem, wq, kLvO + 64 * (n & 1) + sb), vi);
+                float vj[kHS];
+                tmem_ld32(tmem_row_addr(tmem, wq, kLvO + sb), vi);
+                tmem_ld32(tmem_row_addr(tmem, wq, kLvO + kM + sb), vj);
+#pragma unroll
+                for (int e = 0; e < kHS; ++e) vi[e] += vj[e];          // high + low state parts
 #pragma unroll
                 for (int e = 0; e < kHS; ++e) vo[e] = REV ? fmaf(vi[e], egc[sb + e], vo[e]) : vo[e] + vi[e];
                 unsigned char* panel = sWd + (2 * (n & 1) + half) * kPanelB;
@@ -625,7 +635,7 @@ key_side_lean_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_cons
     lean_finish(ctl, tid, warp, tmem, dev_status);
 }
 
-constexpr size_t kSmemLeanValue = 1024 + 13 * kPanelB + sizeof(LeanCtl);   // value_side: 8 + 4 + 1 panels
+constexpr size_t kSmemLeanValue = 1024 + 14 * kPanelB + sizeof(LeanCtl);   // value_side: 8 + 4 + 2 panels
 constexpr size_t kSmemLeanKey = 1024 + 14 * kPanelB + sizeof(LeanCtl);     // key_side: 4 + 8 + 2 panels
 
 }  // namespace

@@ -32,18 +32,18 @@ TC_RTOL = 2.0 ** -9
 # Bounds of the tensor-core path at the size of the benchmark configurations, per tensor:
 # ("plain", 0, x)  = max|err| / rms <= x with no allowance (the stated bound where x = 2e-2);
 # ("mixed", r, x)  = the same after a relative allowance r |ref| per element.
-# The output o, the slot logits, the final memories, dv and the gate gradient meet the stated
-# 2e-2 as it stands.  dq and dk are stored as bfloat16 and heavy-tailed (max|ref| / rms = 10-11
-# at train_1p3b, 39 for dq at t2r_7b, where key channels carry outliers): the half-ulp of the
-# output format alone, 2^-9 |ref|, is then 2e-2 of the rms and more, so it is taken off first
-# (as for the CUDA-core kernels with bf16 io).  What is left: 1.2e-2 at train_1p3b for both,
-# dk 1.0e-2 and dq 2.5e-2 at t2r_7b (the one known gap: the error follows the scale of the
-# outlier channel rather than of the element).  Every operand that the kernels derive on the
-# way to these gradients -- decayed weights, masked products, decayed q / k rows of the
-# slot-space product, the state copy of the pass-2 form -- is carried as a bf16 high/low pair.
+# Every tensor meets the stated 2e-2; the logits, the final memories and the gate gradient (fp32)
+# by two orders of magnitude (1e-4), o and dv at 1.4-1.8e-2 (0.5-0.9e-2 after the half-ulp of
+# their bfloat16 storage).  dq and dk are stored as bfloat16 and heavy-tailed (max|ref| / rms =
+# 10-11 at train_1p3b, 39 for dq at t2r_7b, where key channels carry outliers): the half-ulp of
+# the output format alone, 2^-9 |ref|, is then 2e-2 of the rms and more, so it is taken off
+# first (as for the CUDA-core kernels with bf16 io).  What is left: 1.2e-2 at train_1p3b for
+# both, dk 0.9e-2 and dq 1.8e-2 at t2r_7b.  Every operand that the kernels derive on the way to
+# a result -- decayed weights, masked products, decayed q / k rows, the state copies -- is
+# carried as a bf16 high/low pair.
 TC_CONFIG_BOUNDS = {
     "o": ("plain", 0.0, 2e-2), "ok": ("plain", 0.0, 2e-2), "KT": ("plain", 0.0, 2e-2),
-    "VT": ("plain", 0.0, 2e-2), "dv": ("plain", 0.0, 2e-2), "dq": ("mixed", 2.0 ** -9, 2.6e-2),
+    "VT": ("plain", 0.0, 2e-2), "dv": ("plain", 0.0, 2e-2), "dq": ("mixed", 2.0 ** -9, 2e-2),
     "dk": ("mixed", 2.0 ** -9, 2e-2), "dgate": ("plain", 0.0, 2e-2),
 }
 
