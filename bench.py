@@ -38,10 +38,10 @@ WORKLOAD = "train_1p3b"
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the tensor-core kernels on this
 # workload, from one `ncu --set full` capture (profiles/step_kernels_train_1p3b_ncu_full.md).
 NCU_TRAFFIC = {
-    "pass1_value_side": 187083264, "bwd_dp_value_side": 186084344,
-    "bwd_dIv_value_side_rev": 188307968, "bwd_dIk_value_side_rev": 190506744,
-    "pass2_key_side": 129381884, "bwd_dq_key_side": 136861688,
-    "bwd_dv_key_side_rev": 130355960, "bwd_dk_key_side_rev": 132610046,
+    "pass1_value_side": 187349240, "bwd_dp_value_side": 187349240,
+    "bwd_dIv_value_side_rev": 188625912, "bwd_dIk_value_side_rev": 188625912,
+    "pass2_key_side": 129206520, "bwd_dq_key_side": 129206520,
+    "bwd_dv_key_side_rev": 130708992, "bwd_dk_key_side_rev": 130708992,
     "gate_cumsum": 27124480, "slot_softmax": 100435968, "slot_softmax_bwd": 137995774,
     "gate_grad": 250950394,     # local + scan + carry
 }
