@@ -78,10 +78,10 @@ def kernel_algorithmic_bytes(label: str, w: W.Workload) -> int:
     table = {
         "gate_cumsum": 16 * m,                                       # gate -> G, I, I exp(-G)
         "pass1_value_side": 2 * w.d_k * e + 4 * m + 4 * m * nsk,     # q, k, I exp(-G) -> slices of o'
-        "slot_softmax": 4 * m * nsk + 16 * m,                        # slices, G -> o', p, p exp(G)
+        "slot_softmax": 4 * m * nsk + 12 * m,                        # slices, G -> o', p exp(G)
         "pass2_key_side": 2 * w.d_v * e + 8 * m,                     # v, two decayed rows -> o
         "bwd_dp_value_side": 2 * w.d_v * e + 4 * m + 4 * m * nsv,
-        "slot_softmax_bwd": 4 * m * nsv + 28 * m,                    # o', slices, G -> p, dz, u, p exp(G), dz exp(G)
+        "slot_softmax_bwd": 4 * m * nsv + 20 * m,                    # o', slices, G -> u, p exp(G), dz exp(G)
         "bwd_dq_key_side": 2 * w.d_k * e + 8 * m,
         "bwd_dv_key_side_rev": 2 * w.d_v * e + 8 * m,
         "bwd_dIv_value_side_rev": 2 * w.d_v * e + 4 * m + 4 * m * nsv,

@@ -202,7 +202,9 @@ __global__ void __launch_bounds__(256) slot_softmax_fwd_kernel(const float* __re
     for (int r = 0; r < R; ++r) e[r] *= inv;
     if (!live) return;
     st_vec(ok + idx, z);
-    st_vec(p + idx, e);
+    // fp32 p is read by the general chunk kernels and the CUDA-core kernels only: rows of a pair
+    // that the pipelined kernels serve (pending) get the decayed bf16 rows alone
+    if (!pending) st_vec(p + idx, e);
     if (p_decayed != nullptr) {
 #pragma unroll
         for (int r = 0; r < R; ++r) e[r] *= eg[r];
@@ -290,8 +292,10 @@ __global__ void __launch_bounds__(256) slot_softmax_bwd_kernel(const float* __re
         dzv[r] = scale * dok;
         uv[r] = e[r] * dpv[r] + z[r] * dok;
     }
-    st_vec(p + idx, e);
-    st_vec(dz + idx, dzv);
+    if (!pending) {       // (as in the forward: fp32 p and dz only where a non-pipelined kernel reads them)
+        st_vec(p + idx, e);
+        st_vec(dz + idx, dzv);
+    }
     st_vec(u + idx, uv);
     if (p_decayed != nullptr) {
 #pragma unroll
