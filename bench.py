@@ -87,7 +87,7 @@ def kernel_algorithmic_bytes(label: str, w: W.Workload) -> int:
         "bwd_dIv_value_side_rev": 2 * w.d_v * e + 4 * m + 4 * m * nsv,
         "bwd_dk_key_side_rev": 2 * w.d_k * e + 8 * m,
         "bwd_dIk_value_side_rev": 2 * w.d_k * e + 4 * m + 4 * m * nsk,
-        "gate_grad": 4 * m * (8 + nsk + nsv),   # u, I, gate, G, partials -> dgate; carry pass reads gate, r/w dgate
+        "gate_grad": 4 * m * (7 + nsk + nsv),   # u, gate, G, partials -> dgate; carry pass reads gate, r/w dgate
     }
     return R * table[label]
 

@@ -485,9 +485,15 @@ __global__ void __launch_bounds__(256) gate_grad_local_tma_kernel(
     if (threadIdx.x == 0) {
         mbar_init(&bar, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        mbar_expect_tx(&bar, (uint32_t)((4 + nslices) * kGGTileB));
+        // tiles 0..3 = u, I, gate, G; I is not read when the gate tensor holds a itself (1 - a is one
+        // subtraction), G only when a row factor is pending
+        const bool need[4] = {true, gate_kind != GSA_GATE_A, true, strong != nullptr};
+        int ntiles = nslices;
+        for (int i = 0; i < 4; ++i) ntiles += need[i] ? 1 : 0;
+        mbar_expect_tx(&bar, (uint32_t)(ntiles * kGGTileB));
         const CUtensorMap* maps[4] = {&mapU, &mapI, &mapGate, &mapG};
         for (int i = 0; i < 4; ++i) {
+            if (!need[i]) continue;
             tma_load_4d(smem + i * kGGTileB, maps[i], &bar, 0, h, t0, b);
             tma_load_4d(smem + i * kGGTileB + kGGTileB / 2, maps[i], &bar, 32, h, t0, b);
         }
@@ -525,7 +531,10 @@ __global__ void __launch_bounds__(256) gate_grad_local_tma_kernel(
         for (int i = 0; i < kHalf; ++i) dI[i] *= __expf(-at(3, i));
     }
 #pragma unroll
-    for (int i = 0; i < kHalf; ++i) x[i] = at(0, i) - at(1, i) * dI[i];       // rows past the end: all zero
+    for (int i = 0; i < kHalf; ++i) {
+        const float ii = gate_kind == GSA_GATE_A ? 1.f - at(2, i) : at(1, i);      // 1 - a as the gate kernel formed it
+        x[i] = at(0, i) - ii * dI[i];                                              // rows past the end: u = dI = 0
+    }
     const size_t stride = (size_t)H * M;
     const size_t base = (((size_t)b * T + n * kGG + hh * kHalf) * H + h) * M + tx;
     // the early half starts from the total of the late half of its group
