@@ -23,6 +23,13 @@
  *   - `params` is a HOST pointer.  `stream` is a cudaStream_t passed as void*
  *     (NULL = the legacy default stream).  Work is only enqueued; nothing
  *     synchronises with the host, allocates or frees device memory.
+ *   - Kernels that are independent of one another (the five scans of the backward
+ *     after the softmax gradient; the general and the pipelined kernel of a scan)
+ *     run on internal streams: up to five per calling host thread and device,
+ *     with their events, created on first use and kept for the life of the
+ *     process.  They are forked from `stream` and joined back into it by events
+ *     inside the call, so ordering with respect to `stream` is that of a plain
+ *     in-stream call, and a call can be captured into a CUDA graph.
  *   - `ws` is caller-provided device scratch of at least
  *     gsa_workspace_bytes() bytes, 256-byte aligned; its contents are
  *     undefined afterwards.  Calls that run concurrently need distinct
