@@ -8,11 +8,11 @@
 namespace gsa {
 
 // ------------------------------------------------------------------ chunk_cumsum
-// One CTA per (b,h, chunk): M/2 slot pairs x (chunk / 16) row groups.  A thread takes the logs
-// of its 16 rows x 2 slots (16 independent 8-byte loads in flight), sums them, the group sums
+// One CTA per (b,h, chunk): M/2 slot pairs x (chunk / 8) row groups.  A thread takes the logs
+// of its 8 rows x 2 slots (8 independent 8-byte loads in flight), sums them, the group sums
 // are scanned through shared memory, and the thread writes its running sums.  `chunk` is the
 // chunk length of the kernels that will consume G (64 or 128).
-constexpr int kCumRows = 16;
+constexpr int kCumRows = 8;
 
 // x as a bf16 pair: the rounded value and the rounding residual
 __device__ __forceinline__ void split_bf16(float x, __nv_bfloat16& hi, __nv_bfloat16& lo) {
@@ -30,14 +30,14 @@ __device__ __forceinline__ void store_split2(__nv_bfloat16* row, int c, float x0
 }
 
 template <int M>
-__global__ void __launch_bounds__(M * 4, 4) gate_cumsum_kernel(const float* __restrict__ gate,
+__global__ void __launch_bounds__(M * 8, 2) gate_cumsum_kernel(const float* __restrict__ gate,
                                                             int gate_kind, float inv_tau,
                                                             float* __restrict__ G,
                                                             float* __restrict__ I, int T, int H,
                                                             int chunk, int* __restrict__ strong_flag, int nseg,
                                                             __nv_bfloat16* __restrict__ decayed, int fast_log) {
-    __shared__ double group_sum[8][M];
-    const int s = 2 * threadIdx.x, grp = threadIdx.y;          // blockDim.y = chunk / 16 <= 8
+    __shared__ double group_sum[16][M];
+    const int s = 2 * threadIdx.x, grp = threadIdx.y;          // blockDim.y = chunk / 8 <= 16
     const int n = blockIdx.y;
     const int bh = blockIdx.x, b = bh / H, h = bh % H;
     const int t0 = n * chunk + grp * kCumRows;
@@ -105,7 +105,7 @@ __global__ void __launch_bounds__(M * 4, 4) gate_cumsum_kernel(const float* __re
 cudaError_t launch_gate_cumsum(const float* gate, int gate_kind, float inv_tau, float* G, float* I, int B,
                                int T, int H, int M, int chunk, int* strong_flag, int nseg, void* decayed, int fast_log,
                                cudaStream_t st) {
-    if (chunk % kCumRows != 0 || chunk / kCumRows > 8) return cudaErrorInvalidValue;
+    if (chunk % kCumRows != 0 || chunk / kCumRows > 16) return cudaErrorInvalidValue;
     const int nchunks = (T + chunk - 1) / chunk;
     dim3 block(M / 2, chunk / kCumRows);
     dim3 grid(B * H, nchunks);
