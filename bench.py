@@ -42,8 +42,8 @@ NCU_TRAFFIC = {
     "bwd_dIv_value_side_rev": 188625912, "bwd_dIk_value_side_rev": 188625912,
     "pass2_key_side": 129206520, "bwd_dq_key_side": 129206520,
     "bwd_dv_key_side_rev": 130708992, "bwd_dk_key_side_rev": 130708992,
-    "gate_cumsum": 27124480, "slot_softmax": 100435968, "slot_softmax_bwd": 137995774,
-    "gate_grad": 250950394,     # local + scan + carry
+    "gate_cumsum": 18406144, "slot_softmax": 93043712, "slot_softmax_bwd": 122202876,
+    "gate_grad": 232713984,     # local + scan + carry
 }
 
 
