@@ -76,7 +76,8 @@ struct Carver {
 struct Workspace {
     float *G, *I, *okpart, *ok, *p, *dz, *u, *dppart, *dIk, *dIv, *chunk_tot, *KT, *VT;
     int* strong;     // [B*nseg*H] flags: this (b,h) has a chunk that decays too hard for the factorised form
-    float *seg_decay, *Kloc, *Vloc, *Kstart, *Vstart;   // segment-parallel forward only
+    float *seg_decay, *Kloc, *Vloc, *Kstart, *Vstart;   // segment-parallel scheduling only
+    float *dKend, *dVend;                               // ... backward: states entering each segment from the right
     // tensor-core path: bf16 rows [high | residual] of I exp(-G), p exp(G), dz exp(G), each [B,T,H,2m]
     void *Id, *Pd, *Zd;
     size_t bytes;
@@ -88,7 +89,7 @@ Workspace carve(const gsa_params_t& p, int which, void* ws) {
     const size_t mt = (size_t)p.B * p.T * p.H * p.m;
     const Slices s = slices(p);
     Carver c{static_cast<char*>(ws), 0};
-    const int nseg = which == GSA_WS_FWD ? segments_of(p) : 1;
+    const int nseg = segments_of(p);
     w.strong = reinterpret_cast<int*>(c.take((size_t)p.B * p.H * nseg));
     if (nseg > 1) {
         const size_t pairs = (size_t)p.B * nseg * p.H;
@@ -97,6 +98,10 @@ Workspace carve(const gsa_params_t& p, int which, void* ws) {
         w.Vloc = c.take(pairs * p.m * p.d_v);
         w.Kstart = c.take(pairs * p.m * p.d_k);
         w.Vstart = c.take(pairs * p.m * p.d_v);
+        if (which == GSA_WS_BWD) {
+            w.dKend = c.take(pairs * p.m * p.d_k);
+            w.dVend = c.take(pairs * p.m * p.d_v);
+        }
     }
     w.G = c.take(mt);
     w.I = c.take(mt);
@@ -275,9 +280,9 @@ gsa_status_t gsa_fwd(const gsa_params_t* params, const void* q, const void* k, c
         KeySideArgs s2{w.I, w.I, w.G, v, nullptr, w.Vloc, o, Bs, Ts, p.H, p.d_v, w.Id, w.Id, 1};
         GSA_LAUNCH("segment_pass2_states", key_side(p, s2, 0, w.strong, st, dev_status));
         GSA_LAUNCH("segment_combine", launch_segment_combine(w.seg_decay, w.Kloc, K0, w.Kstart, KT, p.B, p.H, p.m,
-                                                             p.d_k, nseg, st));
+                                                             p.d_k, nseg, 0, st));
         GSA_LAUNCH("segment_combine", launch_segment_combine(w.seg_decay, w.Vloc, V0, w.Vstart, VT, p.B, p.H, p.m,
-                                                             p.d_v, nseg, st));
+                                                             p.d_v, nseg, 0, st));
         Kin = w.Kstart; Vin = w.Vstart;
         Kout = nullptr; Vout = nullptr;
     }
@@ -312,30 +317,69 @@ gsa_status_t gsa_bwd(const gsa_params_t* params, const void* q, const void* k, c
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const Slices s = slices(p);
 
-    GSA_CUDA(cudaMemsetAsync(w.strong, 0, sizeof(int) * (size_t)p.B * p.H, st));
+    // Long sequences with few (batch, head) pairs run as nseg independent segments (see gsa_fwd):
+    // [B,T,H,.] viewed as [B*nseg, T/nseg, H, .], every scan starting from the state that enters its
+    // segment -- from the left for the forward-direction scans, from the right for the reversed ones.
+    const int nseg = segments_of(p);
+    const int Bs = p.B * nseg, Ts = p.T / nseg;
+    GSA_CUDA(cudaMemsetAsync(w.strong, 0, sizeof(int) * (size_t)p.B * p.H * nseg, st));
     GSA_LAUNCH("gate_cumsum", launch_gate_cumsum(gate, p.gate_kind, inv_tau(p), w.G, w.I, p.B, p.T,
-                                                 p.H, p.m, chunk_of(p), w.strong, 1, w.Id, p.io == GSA_BF16, st));
+                                                 p.H, p.m, chunk_of(p), w.strong, nseg, w.Id, p.io == GSA_BF16, st));
     const float* ok = ok_saved;
-    const PendingDecay pend = use_tc(p) ? PendingDecay{w.G, w.strong, p.T, p.H, 1} : PendingDecay{nullptr, nullptr, 1, 1, 1};
+    const PendingDecay pend = use_tc(p) ? PendingDecay{w.G, w.strong, p.T, p.H, nseg} : PendingDecay{nullptr, nullptr, 1, 1, 1};
+    const float *Kin = K0, *Vin = V0;        // states entering the forward-direction scans
+    float* KTout = dKT ? w.KT : nullptr;     // final memories, for the gate gradient's final-memory term
+    float* VTout = dVT ? w.VT : nullptr;
+    if (nseg > 1) {
+        GSA_LAUNCH("segment_logdecay", launch_segment_logdecay(w.G, w.seg_decay, p.B, p.T, p.H, p.m, nseg,
+                                                               chunk_of(p), st));
+        ValueSideArgs s1{q, k, w.I, w.G, nullptr, w.Kloc, w.okpart, Bs, Ts, p.H, p.d_k, w.Id, 1};
+        GSA_LAUNCH("segment_pass1_states", value_side(p, s1, 0, w.strong, st, dev_status));
+        KeySideArgs s2{w.I, w.I, w.G, v, nullptr, w.Vloc, dv, Bs, Ts, p.H, p.d_v, w.Id, w.Id, 1};
+        GSA_LAUNCH("segment_pass2_states", key_side(p, s2, 0, w.strong, st, dev_status));
+        GSA_LAUNCH("segment_combine", launch_segment_combine(w.seg_decay, w.Kloc, K0, w.Kstart, KTout, p.B, p.H, p.m,
+                                                             p.d_k, nseg, 0, st));
+        GSA_LAUNCH("segment_combine", launch_segment_combine(w.seg_decay, w.Vloc, V0, w.Vstart, VTout, p.B, p.H, p.m,
+                                                             p.d_v, nseg, 0, st));
+        Kin = w.Kstart; Vin = w.Vstart;
+        KTout = nullptr; VTout = nullptr;
+    }
     if (ok == nullptr) {  // recompute pass 1 and its logits
-        ValueSideArgs a1{q, k, w.I, w.G, K0, nullptr, w.okpart, p.B, p.T, p.H, p.d_k, w.Id};
+        ValueSideArgs a1{q, k, w.I, w.G, Kin, nullptr, w.okpart, Bs, Ts, p.H, p.d_k, w.Id};
         GSA_LAUNCH("pass1_value_side", value_side(p, a1, 0, w.strong, st, dev_status));
         GSA_LAUNCH("slot_softmax", launch_slot_softmax_fwd(w.okpart, s.k, p.scale, w.ok, w.p, p.B, p.T * p.H, p.m, pend.G,
                                                            nullptr, pend, st));
         ok = w.ok;
     }
     // gradient w.r.t. the pass-2 queries p: the pass-1 form on (dO, v, 1-a); carries V~
-    ValueSideArgs adp{dO, v, w.I, w.G, V0, dVT ? w.VT : nullptr, w.dppart, p.B, p.T, p.H, p.d_v, w.Id};
+    ValueSideArgs adp{dO, v, w.I, w.G, Vin, VTout, w.dppart, Bs, Ts, p.H, p.d_v, w.Id};
     GSA_LAUNCH("bwd_dp_value_side", value_side(p, adp, 0, w.strong, st, dev_status));
     GSA_LAUNCH("slot_softmax_bwd", launch_slot_softmax_bwd(ok, w.dppart, s.v, p.scale, w.p, w.dz, w.u, p.B, p.T * p.H, p.m, pend.G, w.Pd,
                                                            w.Zd, pend, st));
+    const float *dKin = dKT, *dVin = dVT;    // states entering the reversed scans (from the right)
+    float *dK0out = dK0, *dV0out = dV0;
+    if (nseg > 1) {
+        // reversed scans of every segment from empty states, for their end states only (the outputs
+        // land in dk / dv, which the real scans overwrite); then the states entering every segment,
+        // and dK0 / dV0, by a scan over the segments from the last one down
+        KeySideArgs r1{w.I, w.dz, w.G, q, nullptr, w.Kloc, dk, Bs, Ts, p.H, p.d_k, w.Id, w.Zd, 1};
+        GSA_LAUNCH("segment_dk_states", key_side(p, r1, 1, w.strong, st, dev_status));
+        KeySideArgs r2{w.I, w.p, w.G, dO, nullptr, w.Vloc, dv, Bs, Ts, p.H, p.d_v, w.Id, w.Pd, 1};
+        GSA_LAUNCH("segment_dv_states", key_side(p, r2, 1, w.strong, st, dev_status));
+        GSA_LAUNCH("segment_combine", launch_segment_combine(w.seg_decay, w.Kloc, dKT, w.dKend, dK0, p.B, p.H, p.m,
+                                                             p.d_k, nseg, 1, st));
+        GSA_LAUNCH("segment_combine", launch_segment_combine(w.seg_decay, w.Vloc, dVT, w.dVend, dV0, p.B, p.H, p.m,
+                                                             p.d_v, nseg, 1, st));
+        dKin = w.dKend; dVin = w.dVend;
+        dK0out = nullptr; dV0out = nullptr;
+    }
     // dq: the pass-2 form on (dz, 1-a, k); carries K~
-    KeySideArgs adq{w.dz, w.I, w.G, k, K0, dKT ? w.KT : nullptr, dq, p.B, p.T, p.H, p.d_k, w.Zd, w.Id};
+    KeySideArgs adq{w.dz, w.I, w.G, k, Kin, KTout, dq, Bs, Ts, p.H, p.d_k, w.Zd, w.Id};
     // time-reversed runs: dv and dI^v share the state dV~; dk and dI^k share dK~
-    KeySideArgs adv{w.I, w.p, w.G, dO, dVT, dV0, dv, p.B, p.T, p.H, p.d_v, w.Id, w.Pd};
-    ValueSideArgs adIv{v, dO, w.p, w.G, dVT, nullptr, w.dIv, p.B, p.T, p.H, p.d_v, w.Pd};
-    KeySideArgs adk{w.I, w.dz, w.G, q, dKT, dK0, dk, p.B, p.T, p.H, p.d_k, w.Id, w.Zd};
-    ValueSideArgs adIk{k, q, w.dz, w.G, dKT, nullptr, w.dIk, p.B, p.T, p.H, p.d_k, w.Zd};
+    KeySideArgs adv{w.I, w.p, w.G, dO, dVin, dV0out, dv, Bs, Ts, p.H, p.d_v, w.Id, w.Pd};
+    ValueSideArgs adIv{v, dO, w.p, w.G, dVin, nullptr, w.dIv, Bs, Ts, p.H, p.d_v, w.Pd};
+    KeySideArgs adk{w.I, w.dz, w.G, q, dKin, dK0out, dk, Bs, Ts, p.H, p.d_k, w.Id, w.Zd};
+    ValueSideArgs adIk{k, q, w.dz, w.G, dKin, nullptr, w.dIk, Bs, Ts, p.H, p.d_k, w.Zd};
     if (use_tc(p) && !g_sink.active) {
         // the five scans side by side (see ScanLanes)
         ScanLanes* lanes = nullptr;

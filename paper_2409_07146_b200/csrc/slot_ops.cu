@@ -425,7 +425,7 @@ __global__ void __launch_bounds__(128) gate_grad_local_kernel(
     };
     float2 x[kGG], dI[kGG], gt[kGG];
     load_dI(dIk, nsk, dIv, nsv, base, stride, total, rows, dI);
-    if (pend.G != nullptr && pend.strong[bh] == 0) {
+    if (pend.G != nullptr && pend.strong[(b * pend.nseg + t0 / (T / pend.nseg)) * H + h] == 0) {
         // the time-reversed value_side runs left their row factor exp(-G_i) to this kernel
 #pragma unroll
         for (int i = 0; i < kGG; ++i) gt[i] = ld2(pend.G, i, 0.f);
@@ -470,7 +470,7 @@ __global__ void __launch_bounds__(256) gate_grad_local_tma_kernel(
     const __grid_constant__ CUtensorMap mapGate, const __grid_constant__ CUtensorMap mapG,
     const __grid_constant__ CUtensorMap mapDIk, const __grid_constant__ CUtensorMap mapDIv, int nsk, int nsv,
     int gate_kind, float inv_tau, float* __restrict__ blk_tot, float* __restrict__ dgate, int T, int H, int nblk,
-    const int* __restrict__ strong, int32_t* dev_status) {
+    const int* __restrict__ strong, int nseg, int32_t* dev_status) {
     using namespace tc;
     constexpr int M = 64;
     extern __shared__ unsigned char gg_smem_raw[];
@@ -525,7 +525,7 @@ __global__ void __launch_bounds__(256) gate_grad_local_tma_kernel(
 #pragma unroll
         for (int i = 0; i < kHalf; ++i) dI[i] += at(4 + sl, i);
     }
-    if (strong != nullptr && strong[bh] == 0) {
+    if (strong != nullptr && strong[(b * nseg + t0 / (T / nseg)) * H + h] == 0) {
         // the time-reversed value_side runs left their row factor exp(-G_i) to this kernel
 #pragma unroll
         for (int i = 0; i < kHalf; ++i) dI[i] *= __expf(-at(3, i));
@@ -617,7 +617,7 @@ cudaError_t launch_gate_grad(const float* u, const float* I, const float* dIk_pa
             dim3 tgrid(B * H, (T + kGGTmaRows - 1) / kGGTmaRows);
             gate_grad_local_tma_kernel<<<tgrid, 256, smem, st>>>(mu, mi, mg, mG, mk, mv, nsk, nsv, gate_kind, inv_tau, blk_tot,
                                                                 dgate, T, H, nblk, pend.G != nullptr ? pend.strong : nullptr,
-                                                                dev_status);
+                                                                pend.nseg, dev_status);
         } else {
             gate_grad_local_kernel<64><<<grid, block, 0, st>>>(u, I, dIk_part, nsk, dIv_part, nsv, gate, gate_kind, inv_tau,
                                                                blk_tot, dgate, B, T, H, nblk, pend);
@@ -654,16 +654,19 @@ __global__ void segment_logdecay_kernel(const float* __restrict__ G, float* __re
 
 // start[b][r] = D[r-1] start[b][r-1] + local_end[b][r-1], start[b][0] = S0[b] (or 0); the memory
 // after the last segment goes to final (nullable).  Memories [.., H, M, D]; one thread per (s, c).
+// reverse: the same from the last segment down (time-reversed scans: start[r] is the state that
+// enters segment r from the right, S0 the one after the last token, final the one before the first).
 template <int M>
 __global__ void segment_combine_kernel(const float* __restrict__ seg_logdecay, const float* __restrict__ local_end,
                                        const float* __restrict__ S0, float* __restrict__ start,
-                                       float* __restrict__ final_state, int H, int D, int nseg) {
+                                       float* __restrict__ final_state, int H, int D, int nseg, int reverse) {
     const int b = blockIdx.x / H, h = blockIdx.x % H;
     const int idx = blockIdx.y * blockDim.x + threadIdx.x;
     if (idx < M * D) {
         const int s = idx / D;
         float cur = S0 ? S0[((size_t)(b * H + h)) * M * D + idx] : 0.f;
-        for (int r = 0; r < nseg; ++r) {
+        for (int i = 0; i < nseg; ++i) {
+            const int r = reverse ? nseg - 1 - i : i;
             const size_t pair = ((size_t)b * nseg + r) * H + h;
             start[pair * M * D + idx] = cur;
             cur = fmaf(cur, __expf(seg_logdecay[pair * M + s]), local_end[pair * M * D + idx]);
@@ -681,12 +684,12 @@ cudaError_t launch_segment_logdecay(const float* G, float* seg_logdecay, int B, 
 }
 
 cudaError_t launch_segment_combine(const float* seg_logdecay, const float* local_end, const float* S0, float* start,
-                                   float* final_state, int B, int H, int M, int D, int nseg, cudaStream_t st) {
+                                   float* final_state, int B, int H, int M, int D, int nseg, int reverse, cudaStream_t st) {
     dim3 grid(B * H, (M * D + 255) / 256);
     if (M == 64)
-        segment_combine_kernel<64><<<grid, 256, 0, st>>>(seg_logdecay, local_end, S0, start, final_state, H, D, nseg);
+        segment_combine_kernel<64><<<grid, 256, 0, st>>>(seg_logdecay, local_end, S0, start, final_state, H, D, nseg, reverse);
     else
-        segment_combine_kernel<32><<<grid, 256, 0, st>>>(seg_logdecay, local_end, S0, start, final_state, H, D, nseg);
+        segment_combine_kernel<32><<<grid, 256, 0, st>>>(seg_logdecay, local_end, S0, start, final_state, H, D, nseg, reverse);
     return cudaGetLastError();
 }
 

@@ -31,7 +31,7 @@ BF16_IO = {"o", "dq", "dk", "dv"}   # tensors stored in the io type (bf16 when i
 TC_RTOL = 2.0 ** -9
 # Bounds of the tensor-core path at the size of the benchmark configurations, per tensor:
 # ("plain", 0, x)  = max|err| / rms <= x with no allowance (the stated bound where x = 2e-2);
-# ("mixed", r, x)  = the same after a relative allowance r |ref| per element.
+# ("bf16out", 0, x) = the same after the half-ulp of the tensor's bfloat16 storage (bf16_half_ulp).
 # Every tensor meets the stated 2e-2; the logits, the final memories and the gate gradient (fp32)
 # by two orders of magnitude (1e-4), o and dv at 1.4-1.8e-2 (0.5-0.9e-2 after the half-ulp of
 # their bfloat16 storage).  dq and dk are stored as bfloat16 and heavy-tailed (max|ref| / rms =
@@ -43,8 +43,8 @@ TC_RTOL = 2.0 ** -9
 # carried as a bf16 high/low pair.
 TC_CONFIG_BOUNDS = {
     "o": ("plain", 0.0, 2e-2), "ok": ("plain", 0.0, 2e-2), "KT": ("plain", 0.0, 2e-2),
-    "VT": ("plain", 0.0, 2e-2), "dv": ("plain", 0.0, 2e-2), "dq": ("mixed", 2.0 ** -9, 2e-2),
-    "dk": ("mixed", 2.0 ** -9, 2e-2), "dgate": ("plain", 0.0, 2e-2),
+    "VT": ("plain", 0.0, 2e-2), "dv": ("plain", 0.0, 2e-2), "dq": ("bf16out", 0.0, 2e-2),
+    "dk": ("bf16out", 0.0, 2e-2), "dgate": ("plain", 0.0, 2e-2),
 }
 
 
@@ -58,18 +58,26 @@ def mixed_err(x, ref, rtol):
     return float(diff.max() / (rms if rms > 0 else 1.0))
 
 
+def bf16_half_ulp(ref):
+    """Half the spacing of bfloat16 numbers (8 significant bits) at |ref|: the largest error that
+    rounding an exact result to bfloat16 can make.  Between 2^-9 |ref| and 2^-8 |ref|."""
+    a = np.abs(np.asarray(ref, dtype=np.float64))
+    e = np.floor(np.log2(np.maximum(a, 1e-300)))
+    return np.where(a > 0, 2.0 ** (e - 8), 0.0)
+
+
 def rel_err(x, ref, stored_bf16=False):
     """max |x - ref| / rms(ref): the normalisation used for every tolerance.
 
     For a tensor that the library stores as bfloat16, the half-ulp rounding of the result
-    itself (2^-9 |ref| per element) is taken off first: with heavy-tailed gradients
-    max|ref| / rms reaches 15-20, and the output format alone would then exceed the 2e-2
+    itself (bf16_half_ulp(ref) per element) is taken off first: with heavy-tailed gradients
+    max|ref| / rms reaches 15-40, and the output format alone would then exceed the 2e-2
     bound however exact the arithmetic."""
     x = np.asarray(x, dtype=np.float64)
     ref = np.asarray(ref, dtype=np.float64)
     diff = np.abs(x - ref)
     if stored_bf16:
-        diff = np.maximum(diff - 2.0 ** -9 * np.abs(ref), 0.0)
+        diff = np.maximum(diff - bf16_half_ulp(ref), 0.0)
     rms = np.sqrt(np.mean(ref ** 2))
     if rms == 0:
         return float(diff.max())
