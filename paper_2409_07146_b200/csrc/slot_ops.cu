@@ -383,18 +383,27 @@ __global__ void __launch_bounds__(M * 16) gate_grad_scan_kernel(
     double sum = 0.0;
     for (int n = lo; n < hi; ++n) sum += (double)blk_tot[((size_t)bh * nblk + n) * M + s];
     seg_sum[seg][s] = sum;
+    // final-memory term <dK~_T[s], K~_T[s]> + <dV~_T[s], V~_T[s]>: a warp per slot, lanes along the row
+    __shared__ double final_term[M];
+    const int warp = (seg * M + s) >> 5, lane = (seg * M + s) & 31, nwarp = (M * 16) >> 5;
+    for (int slot = warp; slot < M; slot += nwarp) {
+        double dot = 0.0;
+        if (dKT != nullptr) {
+            const float* a = dKT + ((size_t)bh * M + slot) * d_k;
+            const float* bb = KT + ((size_t)bh * M + slot) * d_k;
+            for (int c = lane; c < d_k; c += 32) dot += (double)a[c] * (double)bb[c];
+        }
+        if (dVT != nullptr) {
+            const float* a = dVT + ((size_t)bh * M + slot) * d_v;
+            const float* bb = VT + ((size_t)bh * M + slot) * d_v;
+            for (int c = lane; c < d_v; c += 32) dot += (double)a[c] * (double)bb[c];
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
+        if (lane == 0) final_term[slot] = dot;
+    }
     __syncthreads();
-    double carry = 0.0;
-    if (dKT != nullptr) {
-        const float* a = dKT + ((size_t)bh * M + s) * d_k;
-        const float* bb = KT + ((size_t)bh * M + s) * d_k;
-        for (int c = 0; c < d_k; ++c) carry += (double)a[c] * (double)bb[c];
-    }
-    if (dVT != nullptr) {
-        const float* a = dVT + ((size_t)bh * M + s) * d_v;
-        const float* bb = VT + ((size_t)bh * M + s) * d_v;
-        for (int c = 0; c < d_v; ++c) carry += (double)a[c] * (double)bb[c];
-    }
+    double carry = final_term[s];
     for (int g = seg + 1; g < 16; ++g) carry += seg_sum[g][s];
     for (int n = hi - 1; n >= lo; --n) {
         const size_t idx = ((size_t)bh * nblk + n) * M + s;
