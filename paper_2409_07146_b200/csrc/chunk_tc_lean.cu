@@ -100,7 +100,8 @@ __device__ __forceinline__ void lean_ctl_init(LeanCtl* ctl, int tid, int warp) {
     tc_fence_after_sync();
 }
 
-__device__ __forceinline__ void lean_finish(LeanCtl* ctl, int tid, int warp, uint32_t tmem, int32_t* dev_status) {
+template <class Ctl>
+__device__ __forceinline__ void lean_finish(Ctl* ctl, int tid, int warp, uint32_t tmem, int32_t* dev_status) {
     tc_fence_before_sync();
     __syncthreads();
     if (ctl->abort) {
@@ -635,13 +636,185 @@ key_side_lean_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_cons
     lean_finish(ctl, tid, warp, tmem, dev_status);
 }
 
+// ======================================================================================
+// End state only (segment-parallel scheduling runs every segment once from empty memories just
+// for its end memories).  Both primitives update their state the same way,
+//     U_n = X_n^T [W_hi | W_lo]_n,   forward S <- exp(G_C) (S + U_n),   reverse S <- exp(G_C) S + U_n,
+// with X the d-sized tile that enters the state (xk of value_side, xv of key_side) and W the
+// decayed slot-sized rows beside it (wd, uk_d), and no product depends on the state: the chunk
+// chain is copy -> product -> read-out, with three tile stages and two accumulators, and reads
+// each of the two streams once.
+// ======================================================================================
+constexpr int kScanStages = 3;
+
+struct ScanCtl {
+    uint64_t bar_x[kScanStages];      // (TMA) the tiles of a chunk have landed
+    uint64_t bar_free[kScanStages];   // (tcgen05.commit) ... and have been consumed by the chunk's product
+    uint64_t bar_u[2];                // (tcgen05.commit) the product of a chunk is complete, by chunk parity
+    uint64_t bar_acc[2];              // (compute threads) ... and has been read out
+    uint32_t tmem_slot;
+    volatile int abort;
+    alignas(16) float egc[2][kM];     // exp(G of the chunk's last valid row), by chunk parity
+};
+
+template <bool REV>
+__global__ void __launch_bounds__(kLeanThreads, 1)
+state_scan_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUtensorMap mapW,
+                  const float* __restrict__ G, const float* __restrict__ S0, float* __restrict__ Send, int T, int H,
+                  int D, const int* __restrict__ strong_flag, int32_t* dev_status) {
+    if (strong_flag[blockIdx.x] != 0) return;       // the general kernel takes this (batch, head)
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
+    // a stage: X tile (2 panels of 64 channels) and the decayed rows [hi 64 | lo 64] (2 panels)
+    ScanCtl* ctl = reinterpret_cast<ScanCtl*>(smem + kScanStages * 4 * kPanelB);
+
+    const int tid = threadIdx.x, warp = tid >> 5, wq = warp & 3, half = (tid >> 7) & 1, row = tid & 127;
+    const int sb = kHS * half;          // this thread's first slot
+    const int bh = blockIdx.x, slice = blockIdx.y, b = bh / H, h = bh % H;
+    const int d0 = slice * kDST;
+
+    if (tid == 0) {
+        for (int i = 0; i < kScanStages; ++i) {
+            mbar_init(&ctl->bar_x[i], 1);
+            mbar_init(&ctl->bar_free[i], 1);
+        }
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(&ctl->bar_u[i], 1);
+            mbar_init(&ctl->bar_acc[i], 1);
+        }
+        ctl->abort = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 0) {
+        __syncwarp();
+        tmem_alloc(&ctl->tmem_slot, kTmemCols);
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem = ctl->tmem_slot;
+    const int nchunks = (T + kCT - 1) / kCT;
+    auto chunk_t0 = [&](int n) { return (REV ? nchunks - 1 - n : n) * kCT; };
+
+    if (tid == kCopyThread) {
+        // =============================== copy lane
+        auto load = [&](int n) {
+            const int t = chunk_t0(n), st = n % kScanStages;
+            unsigned char* sX = smem + 4 * st * kPanelB;
+            mbar_expect_tx(&ctl->bar_x[st], 4 * kPanelB);
+            tma_load_4d(sX, &mapX, &ctl->bar_x[st], d0, h, t, b);
+            tma_load_4d(sX + kPanelB, &mapX, &ctl->bar_x[st], d0 + 64, h, t, b);
+            tma_load_4d(sX + 2 * kPanelB, &mapW, &ctl->bar_x[st], 0, h, t, b);
+            tma_load_4d(sX + 3 * kPanelB, &mapW, &ctl->bar_x[st], 64, h, t, b);
+        };
+        prefetch_tmap(&mapX); prefetch_tmap(&mapW);
+        for (int n = 0; n < kScanStages && n < nchunks; ++n) load(n);
+        for (int n = 0; n + kScanStages < nchunks && !ctl->abort; ++n) {
+            LEAN_WAIT(&ctl->bar_free[n % kScanStages], (n / kScanStages) & 1);
+            if (ctl->abort) break;
+            load(n + kScanStages);
+        }
+    } else if (tid == kMmaThread) {
+        // =============================== MMA lane
+        constexpr uint32_t idescU = make_idesc(128, 2 * kM, true, true);   // X^T (MN-major A) x [W_hi | W_lo] (MN-major B)
+        auto mnmaj = [](int kk) { return (uint32_t)(kk * 2048); };
+        for (int n = 0; n < nchunks && !ctl->abort; ++n) {
+            const int st = n % kScanStages;
+            const uint32_t sX = smem_u32(smem + 4 * st * kPanelB);
+            const uint64_t dX = desc_mnmajor(sX, 0, kPanelB), dW = desc_mnmajor(sX + 2 * kPanelB, 0, kPanelB);
+            LEAN_WAIT(&ctl->bar_x[st], (n / kScanStages) & 1);
+            // the accumulator of chunk n-2 must have been read out
+            if (n >= 2) LEAN_WAIT(&ctl->bar_acc[n & 1], ((n - 2) >> 1) & 1);
+            if (ctl->abort) break;
+            tc_fence_after_sync();
+#pragma unroll
+            for (int kk = 0; kk < kCT / 16; ++kk)
+                mma_bf16(tmem + 128 * (n & 1), desc_advance(dX, mnmaj(kk)), desc_advance(dW, mnmaj(kk)), idescU, kk > 0);
+            mma_commit(&ctl->bar_u[n & 1]);
+            mma_commit(&ctl->bar_free[st]);
+        }
+    } else if (tid < kComputeThreads) {
+        // =============================== compute threads: S[c = row][s], slots sb .. sb+31
+        float S[kHS];
+#pragma unroll
+        for (int s = 0; s < kHS; ++s) S[s] = S0 ? S0[((size_t)bh * kM + sb + s) * D + d0 + row] : 0.f;
+        // G of the last valid row of chunk n (threads 0..63, one slot each), one chunk ahead
+        auto chunk_gc = [&](int n) {
+            const int last = min(chunk_t0(n) + kCT, T) - 1;
+            return G[(((size_t)b * T + last) * H + h) * kM + tid];
+        };
+        float g_next = 0.f;
+        if (tid < kM) {
+            ctl->egc[0][tid] = __expf(chunk_gc(0));
+            if (nchunks > 1) g_next = chunk_gc(1);
+        }
+        compute_sync();
+        for (int n = 0; n < nchunks; ++n) {
+            const float* egc = ctl->egc[n & 1];
+            if (tid < kM && n + 1 < nchunks) {
+                ctl->egc[(n + 1) & 1][tid] = __expf(g_next);
+                if (n + 2 < nchunks) g_next = chunk_gc(n + 2);
+            }
+            LEAN_WAIT(&ctl->bar_u[n & 1], (n >> 1) & 1);
+            tc_fence_after_sync();
+            {
+                float v[kHS], vl[kHS];
+                tmem_ld32(tmem_row_addr(tmem, wq, 128 * (n & 1) + sb), v);
+                tmem_ld32(tmem_row_addr(tmem, wq, 128 * (n & 1) + kM + sb), vl);
+#pragma unroll
+                for (int e = 0; e < kHS; e += 4) {
+                    const float4 ec = *reinterpret_cast<const float4*>(&egc[sb + e]);
+                    const float ecv[4] = {ec.x, ec.y, ec.z, ec.w};
+#pragma unroll
+                    for (int t = 0; t < 4; ++t) {
+                        const float u = v[e + t] + vl[e + t];
+                        S[e + t] = REV ? fmaf(S[e + t], ecv[t], u) : (S[e + t] + u) * ecv[t];
+                    }
+                }
+            }
+            // (the barrier inside also publishes the next chunk's egc)
+            if (publish_and_vote(&ctl->bar_acc[n & 1], tid, ctl->abort != 0)) break;
+        }
+        if (!ctl->abort && Send) {
+#pragma unroll
+            for (int s = 0; s < kHS; ++s) Send[((size_t)bh * kM + sb + s) * D + d0 + row] = S[s];
+        }
+    }
+    lean_finish(ctl, tid, warp, tmem, dev_status);
+}
+
+constexpr size_t kSmemStateScan = 1024 + kScanStages * 4 * kPanelB + sizeof(ScanCtl);
 constexpr size_t kSmemLeanValue = 1024 + 14 * kPanelB + sizeof(LeanCtl);   // value_side: 8 + 4 + 2 panels
 constexpr size_t kSmemLeanKey = 1024 + 14 * kPanelB + sizeof(LeanCtl);     // key_side: 4 + 8 + 2 panels
 
 }  // namespace
 
+namespace {
+// X: [B,T,H,D] bf16, the tile that enters the state; W: [B,T,H,2M] bf16 decayed rows [hi | lo]
+cudaError_t launch_state_scan(const void* X, const void* W, const float* G, const float* S0, float* Send, int B, int T,
+                              int H, int D, int reverse, const int* strong_flag, cudaStream_t st, int32_t* dev_status) {
+    CUtensorMap mx, mw;
+    cudaError_t e = make_tensor_map_bthd(&mx, X, B, T, H, D, kCT, 2);
+    if (e == cudaSuccess) e = make_tensor_map_bthd(&mw, W, B, T, H, 2 * kM, kCT, 2);
+    if (e != cudaSuccess) return e;
+    dim3 grid(B * H, D / kDST);
+    if (reverse) {
+        e = prepare(state_scan_kernel<true>, kSmemStateScan, kLeanThreads);
+        if (e != cudaSuccess) return e;
+        state_scan_kernel<true><<<grid, kLeanThreads, kSmemStateScan, st>>>(mx, mw, G, S0, Send, T, H, D, strong_flag, dev_status);
+    } else {
+        e = prepare(state_scan_kernel<false>, kSmemStateScan, kLeanThreads);
+        if (e != cudaSuccess) return e;
+        state_scan_kernel<false><<<grid, kLeanThreads, kSmemStateScan, st>>>(mx, mw, G, S0, Send, T, H, D, strong_flag, dev_status);
+    }
+    return cudaGetLastError();
+}
+}  // namespace
+
 cudaError_t launch_value_side_lean(const ValueSideArgs& a, int reverse, const int* strong_flag, cudaStream_t st,
                                    int32_t* dev_status) {
+    if (a.state_only)
+        return launch_state_scan(a.xk, a.wd, a.G, a.S0, a.Send, a.B, a.T, a.H, a.D, reverse, strong_flag, st, dev_status);
     CUtensorMap mq, mk, mw, mo;
     cudaError_t e = make_tensor_map_bthd(&mq, a.xq, a.B, a.T, a.H, a.D, kCT, 2);
     if (e == cudaSuccess) e = make_tensor_map_sliced(&mo, a.out, a.D / kDST, a.B, a.T, a.H, kM, kCT, 4);
@@ -663,6 +836,8 @@ cudaError_t launch_value_side_lean(const ValueSideArgs& a, int reverse, const in
 
 cudaError_t launch_key_side_lean(const KeySideArgs& a, int reverse, const int* strong_flag, cudaStream_t st,
                                  int32_t* dev_status) {
+    if (a.state_only)
+        return launch_state_scan(a.xv, a.uk_d, a.G, a.S0, a.Send, a.B, a.T, a.H, a.D, reverse, strong_flag, st, dev_status);
     CUtensorMap mv, muq, muk, mo;
     cudaError_t e = make_tensor_map_bthd(&mv, a.xv, a.B, a.T, a.H, a.D, kCT, 2);
     if (e == cudaSuccess) e = make_tensor_map_bthd(&mo, a.out, a.B, a.T, a.H, a.D, kCT, 2);
