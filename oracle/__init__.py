@@ -45,11 +45,11 @@ def _load():
     if _lib is None:
         lib = ctypes.CDLL(build())
         i, d = ctypes.c_int, ctypes.c_double
-        lib.gsa_oracle_fwd.argtypes = [i] * 7 + [d] + [_D] * 10 + [i, i]
+        lib.gsa_oracle_fwd.argtypes = [i] * 8 + [d] + [_D] * 10 + [i, i]
         lib.gsa_oracle_fwd.restype = i
-        lib.gsa_oracle_decode_step.argtypes = [i] * 6 + [d] + [_D] * 7 + [i, i]
+        lib.gsa_oracle_decode_step.argtypes = [i] * 7 + [d] + [_D] * 7 + [i, i]
         lib.gsa_oracle_decode_step.restype = i
-        lib.gsa_oracle_bwd.argtypes = [i] * 7 + [d] + [_D] * 15 + [i, i]
+        lib.gsa_oracle_bwd.argtypes = [i] * 8 + [d] + [_D] * 15 + [i, i]
         lib.gsa_oracle_bwd.restype = i
         _lib = lib
     return _lib
@@ -86,6 +86,12 @@ def _run_split(fn, n_items: int, threads: int | None):
     return nt
 
 
+# The non-linearity between the two passes: Eq. 6's softmax over the slots, or one of the
+# element-wise replacements of the paper's ablation (Table "ablations": no softmax, Swish, ReLU,
+# squared ReLU).
+ACTS = {"softmax": 0, "none": 1, "relu": 2, "swish": 3, "relu2": 4}
+
+
 def gate_from_logits(x, tau):
     """The layer's damped forget gate (Sec. 3.3): a = sigmoid(x)^(1/tau), and da/dx =
     a (1 - sigmoid(x)) / tau.  Returns (a, da_dx) in float64."""
@@ -96,7 +102,7 @@ def gate_from_logits(x, tau):
 
 
 def fwd(q, k, v, gate, *, gate_is_log=False, scale=1.0, K0=None, V0=None,
-        bh_range=None, threads=None, gate_is_logits=False, tau=8.0):
+        bh_range=None, threads=None, gate_is_logits=False, tau=8.0, act="softmax"):
     """Eq. 6 over whole sequences.
 
     q,k [B,T,H,d_k]; v [B,T,H,d_v]; gate [B,T,H,m] (a, or log a when
@@ -104,6 +110,7 @@ def fwd(q, k, v, gate, *, gate_is_log=False, scale=1.0, K0=None, V0=None,
     logits [B,T,H,m], final memories [B,H,m,d].  ``bh_range=(lo, hi)`` restricts
     the work to those flattened (b,h) pairs; the other entries stay zero.
     With gate_is_logits the gate tensor holds x and a = sigmoid(x)^(1/tau) (Sec. 3.3).
+    ``act`` (a key of ACTS) replaces the softmax over the slots.
     """
     lib = _load()
     if gate_is_logits:
@@ -119,7 +126,7 @@ def fwd(q, k, v, gate, *, gate_is_log=False, scale=1.0, K0=None, V0=None,
     lo, hi = bh_range if bh_range is not None else (0, B * H)
 
     def run(b0, b1):
-        return lib.gsa_oracle_fwd(B, T, H, dk, dv, m, int(gate_is_log), float(scale),
+        return lib.gsa_oracle_fwd(B, T, H, dk, dv, m, int(gate_is_log), ACTS[act], float(scale),
                                   _p(q), _p(k), _p(v), _p(gate), _p(K0), _p(V0),
                                   _p(o), _p(ok), _p(KT), _p(VT), lo + b0, lo + b1)
 
@@ -128,14 +135,15 @@ def fwd(q, k, v, gate, *, gate_is_log=False, scale=1.0, K0=None, V0=None,
 
 
 def bwd(q, k, v, gate, dO, *, gate_is_log=False, scale=1.0, K0=None, V0=None,
-        dKT=None, dVT=None, bh_range=None, threads=None, gate_is_logits=False, tau=8.0):
+        dKT=None, dVT=None, bh_range=None, threads=None, gate_is_logits=False, tau=8.0,
+        act="softmax"):
     """Reverse sweep of Eq. 6.  Returns dict(dq, dk, dv, dgate, dK0, dV0);
     dgate is the total derivative w.r.t. the gate tensor as passed (with gate_is_logits:
     w.r.t. x, through a = sigmoid(x)^(1/tau))."""
     if gate_is_logits:
         a, da_dx = gate_from_logits(gate, tau)
         r = bwd(q, k, v, a, dO, gate_is_log=False, scale=scale, K0=K0, V0=V0, dKT=dKT, dVT=dVT,
-                bh_range=bh_range, threads=threads)
+                bh_range=bh_range, threads=threads, act=act)
         r["dgate"] = r["dgate"] * da_dx
         return r
     lib = _load()
@@ -154,7 +162,7 @@ def bwd(q, k, v, gate, dO, *, gate_is_log=False, scale=1.0, K0=None, V0=None,
     lo, hi = bh_range if bh_range is not None else (0, B * H)
 
     def run(b0, b1):
-        return lib.gsa_oracle_bwd(B, T, H, dk, dv, m, int(gate_is_log), float(scale),
+        return lib.gsa_oracle_bwd(B, T, H, dk, dv, m, int(gate_is_log), ACTS[act], float(scale),
                                   _p(q), _p(k), _p(v), _p(gate), _p(K0), _p(V0),
                                   _p(dO), _p(dKT), _p(dVT), _p(dq), _p(dk_), _p(dv_),
                                   _p(dgate), _p(dK0), _p(dV0), lo + b0, lo + b1)
@@ -164,7 +172,7 @@ def bwd(q, k, v, gate, dO, *, gate_is_log=False, scale=1.0, K0=None, V0=None,
 
 
 def decode_step(q, k, v, gate, Kstate, Vstate, *, gate_is_log=False, scale=1.0,
-                threads=None, gate_is_logits=False, tau=8.0):
+                threads=None, gate_is_logits=False, tau=8.0, act="softmax"):
     """One recurrent step of Eq. 6 for S sequences; q,k [S,H,d_k], v [S,H,d_v],
     gate [S,H,m]; Kstate/Vstate [S,H,m,d] float64 C-contiguous arrays updated IN
     PLACE.  Returns o [S,H,d_v]."""
@@ -182,7 +190,7 @@ def decode_step(q, k, v, gate, Kstate, Vstate, *, gate_is_log=False, scale=1.0,
     o = np.zeros((S, H, dv))
 
     def run(s0, s1):
-        return lib.gsa_oracle_decode_step(S, H, dk, dv, m, int(gate_is_log), float(scale),
+        return lib.gsa_oracle_decode_step(S, H, dk, dv, m, int(gate_is_log), ACTS[act], float(scale),
                                           _p(q), _p(k), _p(v), _p(gate), _p(Kstate),
                                           _p(Vstate), _p(o), s0, s1)
 

@@ -19,7 +19,23 @@ from __future__ import annotations
 import torch
 
 
-def gsa_unrolled(q, k, v, a, K0=None, V0=None, scale=1.0):
+def _slot_weights(logits, act):
+    """softmax over the slots (Eq. 6) or its element-wise replacements in the paper's ablation
+    on the non-linearity, each by the library's own routine."""
+    if act == "softmax":
+        return torch.softmax(logits, dim=-1)
+    if act == "none":
+        return logits
+    if act == "relu":
+        return torch.nn.functional.relu(logits)
+    if act == "swish":
+        return torch.nn.functional.silu(logits)
+    if act == "relu2":
+        return torch.nn.functional.relu(logits).square()
+    raise ValueError(act)
+
+
+def gsa_unrolled(q, k, v, a, K0=None, V0=None, scale=1.0, act="softmax"):
     """One head.  q,k [T,d_k]; v [T,d_v]; a [T,m] linear gate in [0,1];
     K0 [m,d_k], V0 [m,d_v] or None.  Returns (o [T,d_v], logits [T,m],
     K_T [m,d_k], V_T [m,d_v]) as float64 torch tensors (differentiable)."""
@@ -55,6 +71,6 @@ def gsa_unrolled(q, k, v, a, K0=None, V0=None, scale=1.0):
         V0 = torch.as_tensor(V0, dtype=torch.float64)
         Vmem = Vmem + D0[:, :, None] * V0[None]
     logits = scale * logits
-    p = torch.softmax(logits, dim=-1)
+    p = _slot_weights(logits, act)
     o = torch.einsum("ts,tsc->tc", p, Vmem)
     return o, logits, Kmem[-1], Vmem[-1]

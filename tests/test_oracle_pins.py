@@ -304,3 +304,68 @@ def test_logit_gate_decode_steps_reproduce_forward():
         o = oracle.decode_step(q[:, t], k[:, t], v[:, t], x[:, t], Ks, Vs, gate_is_logits=True, tau=8.0)
         assert np.abs(o - ref["o"][:, t]).max() < 1e-13
     assert np.abs(Ks - ref["KT"]).max() < 1e-13
+
+
+# ------------------------------------- the ablation's replacements of the slot softmax
+ACTS = ["none", "relu", "swish", "relu2"]
+
+
+@pytest.mark.parametrize("act", ACTS)
+def test_slot_activation_variants_match_unrolled_form_and_its_autograd(act):
+    """Forward against the unrolled two-pass form with the library's activation routine, every
+    gradient against autograd of that form (the paper's ablation on the non-linearity)."""
+    T = 10
+    q, k, v, a, K0, V0 = rand_problem(31, B=1, T=T, H=1, dk=5, dv=4, m=3, init=True)
+    r = np.random.default_rng(32)
+    dO = r.standard_normal(v.shape)
+    dKT = r.standard_normal(K0.shape); dVT = r.standard_normal(V0.shape)
+    f = oracle.fwd(q, k, v, a, K0=K0, V0=V0, scale=0.9, act=act)
+    g = oracle.bwd(q, k, v, a, dO, K0=K0, V0=V0, dKT=dKT, dVT=dVT, scale=0.9, act=act)
+    ts = [torch.tensor(x[0, :, 0] if x.ndim == 4 and x.shape[1] == T else x[0, 0],
+                       requires_grad=True) for x in (q, k, v, a, K0, V0)]
+    o, logits, KT, VT = unrolled.gsa_unrolled(*ts, scale=0.9, act=act)
+    np.testing.assert_allclose(f["o"][0, :, 0], o.detach().numpy(), rtol=0, atol=1e-12)
+    np.testing.assert_allclose(f["ok"][0, :, 0], logits.detach().numpy(), rtol=0, atol=1e-12)
+    if act in ("relu", "relu2"):      # both signs occur, so the kink is exercised on either side
+        assert (logits.detach().numpy() > 0).any() and (logits.detach().numpy() < 0).any()
+    loss = (o * torch.tensor(dO[0, :, 0])).sum() + (KT * torch.tensor(dKT[0, 0])).sum() \
+        + (VT * torch.tensor(dVT[0, 0])).sum()
+    grads = torch.autograd.grad(loss, ts)
+    for name, gt, sel in zip(("dq", "dk", "dv", "dgate", "dK0", "dV0"), grads, (0, 0, 0, 0, 1, 1)):
+        mine = g[name][0, :, 0] if sel == 0 else g[name][0, 0]
+        np.testing.assert_allclose(mine, gt.numpy(), rtol=0, atol=1e-11, err_msg=name)
+
+
+def test_slot_activation_none_is_a_double_sum_without_memories():
+    """Without a non-linearity the layer is bilinear in the two passes:
+    o_t = scale * sum_{i,j<=t} (sum_s W[t,i,s] W[t,j,s]) <q_t, k_j> v_i."""
+    T, m = 9, 3
+    q, k, v, a, _, _ = rand_problem(33, B=1, T=T, H=1, dk=4, dv=3, m=m)
+    f = oracle.fwd(q, k, v, a, scale=0.6, act="none")
+    qq, kk, vv, aa = q[0, :, 0], k[0, :, 0], v[0, :, 0], a[0, :, 0]
+    for t in range(T):
+        W = np.zeros((t + 1, m))
+        for j in range(t + 1):
+            W[j] = (1 - aa[j]) * np.prod(aa[j + 1:t + 1], axis=0)
+        o = np.zeros(3)
+        for i in range(t + 1):
+            for j in range(t + 1):
+                o += 0.6 * (W[i] * W[j]).sum() * (qq[t] @ kk[j]) * vv[i]
+        np.testing.assert_allclose(f["o"][0, t, 0], o, rtol=0, atol=1e-12)
+
+
+def test_slot_activation_relations_and_decode():
+    """ReLU on all-positive logits is the identity; squared ReLU is ReLU with the logits as
+    weights once more; decode steps reproduce the forward for a replacement too."""
+    q, k, v, a, K0, V0 = rand_problem(34, B=2, T=8, H=2, init=True)
+    q, k, K0p = np.abs(q), np.abs(k), np.abs(K0)
+    none = oracle.fwd(q, k, v, a, K0=K0p, V0=V0, scale=0.5, act="none")
+    relu = oracle.fwd(q, k, v, a, K0=K0p, V0=V0, scale=0.5, act="relu")
+    assert (none["ok"] > 0).all()
+    np.testing.assert_allclose(relu["o"], none["o"], rtol=0, atol=1e-14)
+    full = oracle.fwd(q, k, v, a, K0=K0, V0=V0, scale=0.7, act="swish")
+    Ks, Vs = K0.copy(), V0.copy()
+    for t in range(8):
+        o = oracle.decode_step(q[:, t], k[:, t], v[:, t], a[:, t], Ks, Vs, scale=0.7, act="swish")
+        np.testing.assert_allclose(o, full["o"][:, t], atol=1e-14)
+    np.testing.assert_allclose(Ks, full["KT"], atol=1e-14)
