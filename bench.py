@@ -157,11 +157,11 @@ class ClockSampler:
 
 
 # ----------------------------------------------------------------------------- reference arm
-def oracle_step(x, w, pairs, threads):
+def oracle_step(x, w, pairs, threads, act="softmax"):
     import oracle
     rng = (0, pairs)
-    oracle.fwd(x["q"], x["k"], x["v"], x["gate"], bh_range=rng, threads=threads)
-    oracle.bwd(x["q"], x["k"], x["v"], x["gate"], x["dO"], bh_range=rng, threads=threads)
+    oracle.fwd(x["q"], x["k"], x["v"], x["gate"], bh_range=rng, threads=threads, act=act)
+    oracle.bwd(x["q"], x["k"], x["v"], x["gate"], x["dO"], bh_range=rng, threads=threads, act=act)
 
 
 def run_reference(args):
@@ -175,10 +175,10 @@ def run_reference(args):
     threads = min(oracle.default_threads(), 16, w.B * w.H)
     pairs = threads
     for _ in range(args.warmup):
-        oracle_step(x, w, pairs, threads)
+        oracle_step(x, w, pairs, threads, args.slot_act)
     t0 = time.perf_counter()
     for _ in range(args.steps):
-        oracle_step(x, w, pairs, threads)
+        oracle_step(x, w, pairs, threads, args.slot_act)
     dt = (time.perf_counter() - t0) / args.steps
     tokens = pairs * w.T / w.H          # a token counts once all H heads are done
     val = tokens / dt
@@ -241,7 +241,7 @@ def run_ours(args):
 
     w = rank_workload(rank)
     x = W.make_inputs(w)
-    p = gsa.Params(w.B, w.T, w.H, w.d_k, w.d_v, w.m, io=w.io)
+    p = gsa.Params(w.B, w.T, w.H, w.d_k, w.d_v, w.m, io=w.io, slot_act=args.slot_act)
 
     def host(a, bf16):
         t = torch.from_numpy(np.ascontiguousarray(a))
@@ -426,7 +426,7 @@ def run_ours(args):
             threads = min(oracle.default_threads(), 16, w.B * w.H)
             pairs = min(w.B * w.H, 2 * threads)
             t0 = time.perf_counter()
-            oracle_step(x0, w, pairs, threads)
+            oracle_step(x0, w, pairs, threads, args.slot_act)
             dt = time.perf_counter() - t0
             cpu = {"value": pairs * w.T / w.H / dt, "unit": UNIT, "cores": threads, "kind": "oracle",
                    "sample": f"{pairs} of {w.B * w.H} (batch, head) pairs of one {WORKLOAD} step, "
@@ -440,6 +440,7 @@ def run_ours(args):
             "config": {"workload": WORKLOAD, "B": w.B, "T": w.T, "H": w.H, "d_k": w.d_k,
                        "d_v": w.d_v, "m": w.m, "io": w.io, "chunk": gsa.gsa_chunk_size(p),
                        "step": "gsa_fwd (logits saved) + gsa_bwd",
+                       "slot_act": args.slot_act,
                        "launch": launch_mode,
                        "l2": "inputs larger than L2 (1.1 GB touched per step vs 126 MB)",
                        "parallelism": f"dp{world} over batch, no collective"},
@@ -502,6 +503,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--slot-act", default="softmax", choices=["softmax", "none", "relu", "swish", "relu2"],
+                    help="the non-linearity between the two passes: the paper's softmax (the headline "
+                         "workload) or one of the replacements of its ablation")
     ap.add_argument("--no-graph", action="store_true", help="time plain library calls instead of a CUDA graph replay")
     ap.add_argument("--profile-case", action="store_true",
                     help="run warmup + steps bare (for ncu); prints no benchmark line")

@@ -68,6 +68,14 @@ typedef enum {
 typedef enum { GSA_F32 = 0, GSA_BF16 = 1 } gsa_dtype_t;
 typedef enum { GSA_GATE_A = 0, GSA_GATE_LOG_A = 1, GSA_GATE_LOGITS = 2 } gsa_gate_t;
 
+/* The non-linearity between the two passes: the softmax over the m slots of Eq. 6, or one of the
+ * element-wise replacements of the paper's ablation on it (Sec. 4, table of ablations,
+ * "Ablations on non-linearity": no softmax, Swish, ReLU, squared ReLU), applied to the scaled
+ * slot logits scale * K~_t q_t. */
+typedef enum {
+    GSA_ACT_SOFTMAX = 0, GSA_ACT_NONE = 1, GSA_ACT_RELU = 2, GSA_ACT_SWISH = 3, GSA_ACT_RELU2 = 4
+} gsa_act_t;
+
 /* Which kernels serve the d-sized contractions of the chunk passes. */
 typedef enum {
     GSA_IMPL_AUTO = 0,   /* bf16 io: tensor-core kernels; fp32 io: fp32 CUDA-core kernels */
@@ -82,6 +90,7 @@ typedef struct {
     float scale;        /* multiplies the slot logits; 1.0f is the paper's layer */
     int32_t impl;       /* gsa_impl_t */
     float tau;          /* GSA_GATE_LOGITS only: damping of the gate, a = sigmoid(x)^(1/tau); > 0 */
+    int32_t slot_act;   /* gsa_act_t; 0 = the paper's softmax */
 } gsa_params_t;
 
 enum { GSA_WS_FWD = 0, GSA_WS_BWD = 1, GSA_WS_DECODE = 2 };

@@ -17,6 +17,7 @@ GSA_IMPL_AUTO, GSA_IMPL_SIMT, GSA_IMPL_TC = 0, 1, 2
 GSA_WS_FWD, GSA_WS_BWD, GSA_WS_DECODE = 0, 1, 2
 
 _IMPL = {"auto": GSA_IMPL_AUTO, "simt": GSA_IMPL_SIMT, "tc": GSA_IMPL_TC}
+_ACT = {"softmax": 0, "none": 1, "relu": 2, "swish": 3, "relu2": 4}   # gsa_act_t
 
 
 class GsaError(RuntimeError):
@@ -30,7 +31,8 @@ class _CParams(ctypes.Structure):
     _fields_ = [("B", ctypes.c_int32), ("T", ctypes.c_int32), ("H", ctypes.c_int32),
                 ("d_k", ctypes.c_int32), ("d_v", ctypes.c_int32), ("m", ctypes.c_int32),
                 ("io", ctypes.c_int32), ("gate_kind", ctypes.c_int32),
-                ("scale", ctypes.c_float), ("impl", ctypes.c_int32), ("tau", ctypes.c_float)]
+                ("scale", ctypes.c_float), ("impl", ctypes.c_int32), ("tau", ctypes.c_float),
+                ("slot_act", ctypes.c_int32)]
 
 
 @dataclass(frozen=True)
@@ -48,13 +50,14 @@ class Params:
     impl: str = "auto"        # "auto" | "simt" | "tc"
     gate_is_logits: bool = False   # the gate tensor holds x, a = sigmoid(x)^(1/tau)
     tau: float = 8.0
+    slot_act: str = "softmax"      # "softmax" | "none" | "relu" | "swish" | "relu2"
 
     def c(self) -> _CParams:
         return _CParams(self.B, self.T, self.H, self.d_k, self.d_v, self.m,
                         GSA_BF16 if self.io == "bf16" else GSA_F32,
                         GSA_GATE_LOGITS if self.gate_is_logits else
                         (GSA_GATE_LOG_A if self.gate_is_log else GSA_GATE_A),
-                        float(self.scale), _IMPL[self.impl], float(self.tau))
+                        float(self.scale), _IMPL[self.impl], float(self.tau), _ACT[self.slot_act])
 
     @property
     def io_dtype(self) -> torch.dtype:

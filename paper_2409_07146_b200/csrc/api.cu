@@ -25,6 +25,7 @@ gsa_status_t check_params(const gsa_params_t* p, bool need_T) {
     if (p->gate_kind != GSA_GATE_A && p->gate_kind != GSA_GATE_LOG_A && p->gate_kind != GSA_GATE_LOGITS)
         return GSA_ERR_INVALID_ARG;
     if (p->gate_kind == GSA_GATE_LOGITS && !(p->tau > 0.f)) return GSA_ERR_INVALID_ARG;
+    if (p->slot_act < GSA_ACT_SOFTMAX || p->slot_act > GSA_ACT_RELU2) return GSA_ERR_INVALID_ARG;
     if (p->impl != GSA_IMPL_AUTO && p->impl != GSA_IMPL_SIMT && p->impl != GSA_IMPL_TC)
         return GSA_ERR_INVALID_ARG;
     if (!(p->scale == p->scale)) return GSA_ERR_INVALID_ARG;
@@ -289,7 +290,7 @@ gsa_status_t gsa_fwd(const gsa_params_t* params, const void* q, const void* k, c
     // pass 1: o' = GLA(q, k, 1-a) with the decay on the slot (value) side
     ValueSideArgs a1{q, k, w.I, w.G, Kin, Kout, w.okpart, Bs, Ts, p.H, p.d_k, w.Id};
     GSA_LAUNCH("pass1_value_side", value_side(p, a1, 0, w.strong, st, dev_status));
-    GSA_LAUNCH("slot_softmax", launch_slot_softmax_fwd(w.okpart, s.k, p.scale, ok, w.p, p.B, p.T * p.H, p.m, pend.G, w.Pd,
+    GSA_LAUNCH("slot_softmax", launch_slot_softmax_fwd(w.okpart, s.k, p.scale, p.slot_act, ok, w.p, p.B, p.T * p.H, p.m, pend.G, w.Pd,
                                                        pend, st));
     // pass 2: o = GLA(softmax(o'), 1-a, v) with the decay on the slot (key) side
     KeySideArgs a2{w.p, w.I, w.G, v, Vin, Vout, o, Bs, Ts, p.H, p.d_v, w.Pd, w.Id};
@@ -347,14 +348,14 @@ gsa_status_t gsa_bwd(const gsa_params_t* params, const void* q, const void* k, c
     if (ok == nullptr) {  // recompute pass 1 and its logits
         ValueSideArgs a1{q, k, w.I, w.G, Kin, nullptr, w.okpart, Bs, Ts, p.H, p.d_k, w.Id};
         GSA_LAUNCH("pass1_value_side", value_side(p, a1, 0, w.strong, st, dev_status));
-        GSA_LAUNCH("slot_softmax", launch_slot_softmax_fwd(w.okpart, s.k, p.scale, w.ok, w.p, p.B, p.T * p.H, p.m, pend.G,
+        GSA_LAUNCH("slot_softmax", launch_slot_softmax_fwd(w.okpart, s.k, p.scale, p.slot_act, w.ok, w.p, p.B, p.T * p.H, p.m, pend.G,
                                                            nullptr, pend, st));
         ok = w.ok;
     }
     // gradient w.r.t. the pass-2 queries p: the pass-1 form on (dO, v, 1-a); carries V~
     ValueSideArgs adp{dO, v, w.I, w.G, Vin, VTout, w.dppart, Bs, Ts, p.H, p.d_v, w.Id};
     GSA_LAUNCH("bwd_dp_value_side", value_side(p, adp, 0, w.strong, st, dev_status));
-    GSA_LAUNCH("slot_softmax_bwd", launch_slot_softmax_bwd(ok, w.dppart, s.v, p.scale, w.p, w.dz, w.u, p.B, p.T * p.H, p.m, pend.G, w.Pd,
+    GSA_LAUNCH("slot_softmax_bwd", launch_slot_softmax_bwd(ok, w.dppart, s.v, p.scale, p.slot_act, w.p, w.dz, w.u, p.B, p.T * p.H, p.m, pend.G, w.Pd,
                                                            w.Zd, pend, st));
     const float *dKin = dKT, *dVin = dVT;    // states entering the reversed scans (from the right)
     float *dK0out = dK0, *dV0out = dV0;

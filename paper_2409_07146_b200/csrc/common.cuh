@@ -100,6 +100,24 @@ struct KeySideArgs {
     int state_only;                   // as in ValueSideArgs
 };
 
+// Element-wise replacements of the slot softmax (gsa_act_t other than GSA_ACT_SOFTMAX): f(z) and f'(z).
+__device__ __forceinline__ float slot_act_value(float z, int act) {
+    const float r = fmaxf(z, 0.f);
+    if (act == GSA_ACT_NONE) return z;
+    if (act == GSA_ACT_RELU) return r;
+    if (act == GSA_ACT_SWISH) return z / (1.f + __expf(-z));
+    return r * r;
+}
+__device__ __forceinline__ float slot_act_slope(float z, int act) {
+    if (act == GSA_ACT_NONE) return 1.f;
+    if (act == GSA_ACT_RELU) return z > 0.f ? 1.f : 0.f;
+    if (act == GSA_ACT_SWISH) {
+        const float sg = 1.f / (1.f + __expf(-z));
+        return sg * (1.f + z * (1.f - sg));
+    }
+    return 2.f * fmaxf(z, 0.f);
+}
+
 // GSA_GATE_LOGITS: log a = -softplus(-x) / tau (a = sigmoid(x)^(1/tau), Sec. 3.3) and the factor
 // d(log a)/dx = sigmoid(-x) / tau of the gate gradient.
 __device__ __forceinline__ float log_gate_from_logit(float x, float inv_tau) {
@@ -148,11 +166,12 @@ cudaError_t launch_segment_combine(const float* seg_logdecay, const float* local
 // G, p_decayed / dz_decayed (nullable together; bf16 [rows, 2M]): rows [high | residual] of
 // p exp(G) and dz exp(G), operands of the pipelined tensor-core kernels.
 // (tensors [B, rows_per_batch = T*H, M])
-cudaError_t launch_slot_softmax_fwd(const float* part, int nslice, float scale, float* ok,
+// act: gsa_act_t (the softmax over the slots or an element-wise replacement)
+cudaError_t launch_slot_softmax_fwd(const float* part, int nslice, float scale, int act, float* ok,
                                     float* p, int B, int rows_per_batch, int M, const float* G, void* p_decayed,
                                     PendingDecay pend, cudaStream_t st);
 cudaError_t launch_slot_softmax_bwd(const float* ok, const float* dp_part, int nslice,
-                                    float scale, float* p, float* dz, float* u, int B, int rows_per_batch,
+                                    float scale, int act, float* p, float* dz, float* u, int B, int rows_per_batch,
                                     int M, const float* G, void* p_decayed, void* dz_decayed,
                                     PendingDecay pend, cudaStream_t st);
 cudaError_t launch_gate_grad(const float* u, const float* I, const float* dIk_part, int nsk,

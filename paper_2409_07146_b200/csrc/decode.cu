@@ -65,7 +65,7 @@ struct RowVec {
 template <typename IO, int DK, int DV, int M>
 __global__ void __launch_bounds__(kDecodeWarps * 32)
 decode_step_kernel(const IO* __restrict__ q, const IO* __restrict__ k, const IO* __restrict__ v,
-                   const float* __restrict__ gate, int gate_kind, float inv_tau, float scale,
+                   const float* __restrict__ gate, int gate_kind, float inv_tau, float scale, int act,
                    float* __restrict__ Ks, float* __restrict__ Vs, IO* __restrict__ o) {
     constexpr int RPW = M / kDecodeWarps;  // memory rows per warp
     const size_t pair = blockIdx.x;
@@ -117,8 +117,11 @@ decode_step_kernel(const IO* __restrict__ q, const IO* __restrict__ k, const IO*
         }
     }
     __syncthreads();
-    // softmax over the m slots
-    if (warp == 0) {
+    // softmax over the m slots, or its element-wise replacement
+    if (warp == 0 && act != GSA_ACT_SOFTMAX) {
+#pragma unroll
+        for (int r = 0; r < M / 32; ++r) s_p[lane + 32 * r] = slot_act_value(s_z[lane + 32 * r], act);
+    } else if (warp == 0) {
         float z[M / 32], zmax = -INFINITY;
 #pragma unroll
         for (int r = 0; r < M / 32; ++r) { z[r] = s_z[lane + 32 * r]; zmax = fmaxf(zmax, z[r]); }
@@ -178,9 +181,9 @@ static cudaError_t launch_decode_m(const gsa_params_t& p, const IO* q, const IO*
     const int is_log = p.gate_kind;
     const float inv_tau = p.tau > 0.f ? 1.f / p.tau : 0.f;
     if (p.m == 64)
-        decode_step_kernel<IO, DK, DV, 64><<<pairs, kDecodeWarps * 32, 0, st>>>(q, k, v, gate, is_log, inv_tau, p.scale, Ks, Vs, o);
+        decode_step_kernel<IO, DK, DV, 64><<<pairs, kDecodeWarps * 32, 0, st>>>(q, k, v, gate, is_log, inv_tau, p.scale, p.slot_act, Ks, Vs, o);
     else
-        decode_step_kernel<IO, DK, DV, 32><<<pairs, kDecodeWarps * 32, 0, st>>>(q, k, v, gate, is_log, inv_tau, p.scale, Ks, Vs, o);
+        decode_step_kernel<IO, DK, DV, 32><<<pairs, kDecodeWarps * 32, 0, st>>>(q, k, v, gate, is_log, inv_tau, p.scale, p.slot_act, Ks, Vs, o);
     return cudaGetLastError();
 }
 

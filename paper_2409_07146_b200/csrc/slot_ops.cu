@@ -155,7 +155,7 @@ __device__ __forceinline__ float row_sum(float x) {
 
 template <int M>
 __global__ void __launch_bounds__(256) slot_softmax_fwd_kernel(const float* __restrict__ part,
-                                                               int nslice, float scale,
+                                                               int nslice, float scale, int act,
                                                                float* __restrict__ ok,
                                                                float* __restrict__ p,
                                                                int rows_per_batch, const float* __restrict__ G,
@@ -192,14 +192,20 @@ __global__ void __launch_bounds__(256) slot_softmax_fwd_kernel(const float* __re
         z[r] *= scale;
         zmax = fmaxf(zmax, z[r]);
     }
-    zmax = row_max<LPR>(zmax);
-    float e[R], den = 0.f;
+    float e[R];
+    if (act == GSA_ACT_SOFTMAX) {
+        zmax = row_max<LPR>(zmax);
+        float den = 0.f;
 #pragma unroll
-    for (int r = 0; r < R; ++r) { e[r] = __expf(z[r] - zmax); den += e[r]; }
-    den = row_sum<LPR>(den);
-    const float inv = 1.f / den;
+        for (int r = 0; r < R; ++r) { e[r] = __expf(z[r] - zmax); den += e[r]; }
+        den = row_sum<LPR>(den);
+        const float inv = 1.f / den;
 #pragma unroll
-    for (int r = 0; r < R; ++r) e[r] *= inv;
+        for (int r = 0; r < R; ++r) e[r] *= inv;
+    } else {               // element-wise replacement of the softmax (uniform over the launch)
+#pragma unroll
+        for (int r = 0; r < R; ++r) e[r] = slot_act_value(z[r], act);
+    }
     if (!live) return;
     st_vec(ok + idx, z);
     // fp32 p is read by the general chunk kernels and the CUDA-core kernels only: rows of a pair
@@ -212,22 +218,22 @@ __global__ void __launch_bounds__(256) slot_softmax_fwd_kernel(const float* __re
     }
 }
 
-cudaError_t launch_slot_softmax_fwd(const float* part, int nslice, float scale, float* ok,
+cudaError_t launch_slot_softmax_fwd(const float* part, int nslice, float scale, int act, float* ok,
                                     float* p, int B, int rows_per_batch, int M, const float* G, void* p_decayed,
                                     PendingDecay pend, cudaStream_t st) {
     const int rpb = 8 * (128 / M);       // rows per block: 8 warps x 128/M rows
     const dim3 grid((unsigned)((rows_per_batch + rpb - 1) / rpb), (unsigned)B);
     const int rows = rows_per_batch;
     if (M == 64)
-        slot_softmax_fwd_kernel<64><<<grid, 256, 0, st>>>(part, nslice, scale, ok, p, rows, G,
+        slot_softmax_fwd_kernel<64><<<grid, 256, 0, st>>>(part, nslice, scale, act, ok, p, rows, G,
                                                           static_cast<__nv_bfloat16*>(p_decayed), pend);
     else
-        slot_softmax_fwd_kernel<32><<<grid, 256, 0, st>>>(part, nslice, scale, ok, p, rows, G,
+        slot_softmax_fwd_kernel<32><<<grid, 256, 0, st>>>(part, nslice, scale, act, ok, p, rows, G,
                                                           static_cast<__nv_bfloat16*>(p_decayed), pend);
     return cudaGetLastError();
 }
 
-// Softmax backward (dsoftmax of Algorithm 1): from the scaled logits ok and the gradient dp
+// Softmax backward (dsoftmax of Algorithm 1; f'(ok) dp for an element-wise replacement f): from the scaled logits ok and the gradient dp
 // w.r.t. the softmax output (summed over the d_v slices that produced it):
 //   p = softmax(ok); dok = p * (dp - <p,dp>); dz = scale * dok (gradient w.r.t. the unscaled
 //   pass-1 output); u = p*dp + ok*dok (the two "query x query-gradient" terms of the
@@ -235,7 +241,7 @@ cudaError_t launch_slot_softmax_fwd(const float* part, int nslice, float scale, 
 template <int M>
 __global__ void __launch_bounds__(256) slot_softmax_bwd_kernel(const float* __restrict__ ok,
                                                                const float* __restrict__ dp_part,
-                                                               int nslice, float scale,
+                                                               int nslice, float scale, int act,
                                                                float* __restrict__ p,
                                                                float* __restrict__ dz,
                                                                float* __restrict__ u,
@@ -274,24 +280,34 @@ __global__ void __launch_bounds__(256) slot_softmax_bwd_kernel(const float* __re
         if (pending) dpv[r] *= eg[r];
         zmax = fmaxf(zmax, z[r]);
     }
-    zmax = row_max<LPR>(zmax);
-    float e[R], den = 0.f;
+    float e[R], dzv[R], uv[R];
+    if (act == GSA_ACT_SOFTMAX) {
+        zmax = row_max<LPR>(zmax);
+        float den = 0.f;
 #pragma unroll
-    for (int r = 0; r < R; ++r) { e[r] = __expf(z[r] - zmax); den += e[r]; }
-    den = row_sum<LPR>(den);
-    const float inv = 1.f / den;
-    float pdp = 0.f;
+        for (int r = 0; r < R; ++r) { e[r] = __expf(z[r] - zmax); den += e[r]; }
+        den = row_sum<LPR>(den);
+        const float inv = 1.f / den;
+        float pdp = 0.f;
 #pragma unroll
-    for (int r = 0; r < R; ++r) { e[r] *= inv; pdp += e[r] * dpv[r]; }
-    pdp = row_sum<LPR>(pdp);
-    if (!live) return;
-    float dzv[R], uv[R];
+        for (int r = 0; r < R; ++r) { e[r] *= inv; pdp += e[r] * dpv[r]; }
+        pdp = row_sum<LPR>(pdp);
 #pragma unroll
-    for (int r = 0; r < R; ++r) {
-        const float dok = e[r] * (dpv[r] - pdp);
-        dzv[r] = scale * dok;
-        uv[r] = e[r] * dpv[r] + z[r] * dok;
+        for (int r = 0; r < R; ++r) {
+            const float dok = e[r] * (dpv[r] - pdp);
+            dzv[r] = scale * dok;
+            uv[r] = e[r] * dpv[r] + z[r] * dok;
+        }
+    } else {               // element-wise replacement f of the softmax: dok = f'(ok) dp
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+            e[r] = slot_act_value(z[r], act);
+            const float dok = slot_act_slope(z[r], act) * dpv[r];
+            dzv[r] = scale * dok;
+            uv[r] = e[r] * dpv[r] + z[r] * dok;
+        }
     }
+    if (!live) return;
     if (!pending) {       // (as in the forward: fp32 p and dz only where a non-pipelined kernel reads them)
         st_vec(p + idx, e);
         st_vec(dz + idx, dzv);
@@ -306,18 +322,18 @@ __global__ void __launch_bounds__(256) slot_softmax_bwd_kernel(const float* __re
 }
 
 cudaError_t launch_slot_softmax_bwd(const float* ok, const float* dp_part, int nslice,
-                                    float scale, float* p, float* dz, float* u, int B, int rows_per_batch,
+                                    float scale, int act, float* p, float* dz, float* u, int B, int rows_per_batch,
                                     int M, const float* G, void* p_decayed, void* dz_decayed,
                                     PendingDecay pend, cudaStream_t st) {
     const int rpb = 8 * (128 / M);       // rows per block: 8 warps x 128/M rows
     const dim3 grid((unsigned)((rows_per_batch + rpb - 1) / rpb), (unsigned)B);
     const int rows = rows_per_batch;
     if (M == 64)
-        slot_softmax_bwd_kernel<64><<<grid, 256, 0, st>>>(ok, dp_part, nslice, scale, p, dz, u, rows, G,
+        slot_softmax_bwd_kernel<64><<<grid, 256, 0, st>>>(ok, dp_part, nslice, scale, act, p, dz, u, rows, G,
                                                           static_cast<__nv_bfloat16*>(p_decayed),
                                                           static_cast<__nv_bfloat16*>(dz_decayed), pend);
     else
-        slot_softmax_bwd_kernel<32><<<grid, 256, 0, st>>>(ok, dp_part, nslice, scale, p, dz, u, rows, G,
+        slot_softmax_bwd_kernel<32><<<grid, 256, 0, st>>>(ok, dp_part, nslice, scale, act, p, dz, u, rows, G,
                                                           static_cast<__nv_bfloat16*>(p_decayed),
                                                           static_cast<__nv_bfloat16*>(dz_decayed), pend);
     return cudaGetLastError();

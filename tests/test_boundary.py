@@ -68,6 +68,12 @@ def test_validation_happens_before_any_launch(lib):
     # invalid sizes
     assert _call_fwd(lib, gsa.Params(1, 0, 1, 64, 64, 32, io="f32"), ok) == 1
     assert _call_fwd(lib, gsa.Params(0, 64, 1, 64, 64, 32, io="f32"), ok) == 1
+    # a non-linearity outside gsa_act_t
+    cp = good.c()
+    cp.slot_act = 5
+    assert lib.gsa_fwd(ctypes.byref(cp), *[ctypes.c_void_p(x) for x in ok], ctypes.c_void_p(0x1000), 1 << 40,
+                       None, None) == 1
+    assert _call_fwd(lib, gsa.Params(1, 64, 1, 64, 64, 32, io="f32", slot_act="relu2"), ok, ws=0) == 3
     # workspace: missing, misaligned, too small
     assert _call_fwd(lib, good, ok, ws=0) == 3
     assert _call_fwd(lib, good, ok, ws=0x1010) == 3

@@ -12,8 +12,8 @@ from util import BF16_IO, TC_RTOL, TOL, mixed_err, rand_inputs, rel_err, to_dev,
 pytestmark = pytest.mark.gpu
 
 
-def run_fwd(d, B, T, H, dk, dv, m, io, impl="auto", scale=1.0, log=False, want_states=True):
-    p = gsa.Params(B, T, H, dk, dv, m, io=io, impl=impl, scale=scale, gate_is_log=log)
+def run_fwd(d, B, T, H, dk, dv, m, io, impl="auto", scale=1.0, log=False, want_states=True, act="softmax"):
+    p = gsa.Params(B, T, H, dk, dv, m, io=io, impl=impl, scale=scale, gate_is_log=log, slot_act=act)
     gate = np.log(np.maximum(d["gate"].astype(np.float64), 1e-300)).astype(np.float32) if log else d["gate"]
     K0, V0 = to_dev(d.get("K0")), to_dev(d.get("V0"))
     KT = torch.empty(B, H, m, dk, device="cuda") if want_states else None
@@ -26,9 +26,9 @@ def run_fwd(d, B, T, H, dk, dv, m, io, impl="auto", scale=1.0, log=False, want_s
                 VT=None if VT is None else to_np(VT)), gate
 
 
-def check_fwd(d, got, gate, io, scale=1.0, log=False, tol=None, tc=False):
+def check_fwd(d, got, gate, io, scale=1.0, log=False, tol=None, tc=False, act="softmax"):
     ref = oracle.fwd(d["q"], d["k"], d["v"], gate, gate_is_log=log, scale=scale,
-                     K0=d.get("K0"), V0=d.get("V0"))
+                     K0=d.get("K0"), V0=d.get("V0"), act=act)
     tol = tol or TOL[io]
     if tc:      # bf16-stored o after the half-ulp of its format; fp32 tensors after the small-shape allowance
         errs = {n: (rel_err(got[n], ref[n], True) if n in BF16_IO else mixed_err(got[n], ref[n], TC_RTOL))
@@ -133,8 +133,8 @@ def test_fwd_state_carry_matches_one_call():
 
 
 # ------------------------------------------------------------------ backward
-def run_bwd(d, B, T, H, dk, dv, m, io, impl="auto", scale=1.0, log=False, saved=False):
-    p = gsa.Params(B, T, H, dk, dv, m, io=io, impl=impl, scale=scale, gate_is_log=log)
+def run_bwd(d, B, T, H, dk, dv, m, io, impl="auto", scale=1.0, log=False, saved=False, act="softmax"):
+    p = gsa.Params(B, T, H, dk, dv, m, io=io, impl=impl, scale=scale, gate_is_log=log, slot_act=act)
     gate = np.log(d["gate"].astype(np.float64)).astype(np.float32) if log else d["gate"]
     q, k, v, dO = (to_dev(d[n], io) for n in ("q", "k", "v", "dO"))
     K0, V0, dKT, dVT = (to_dev(d.get(n)) for n in ("K0", "V0", "dKT", "dVT"))
@@ -148,7 +148,7 @@ def run_bwd(d, B, T, H, dk, dv, m, io, impl="auto", scale=1.0, log=False, saved=
     torch.cuda.synchronize()
     got = dict(dq=to_np(dq), dk=to_np(dk_), dv=to_np(dv_), dgate=to_np(dg), dK0=to_np(dK0), dV0=to_np(dV0))
     ref = oracle.bwd(d["q"], d["k"], d["v"], gate, d["dO"], gate_is_log=log, scale=scale,
-                     K0=d.get("K0"), V0=d.get("V0"), dKT=d.get("dKT"), dVT=d.get("dVT"))
+                     K0=d.get("K0"), V0=d.get("V0"), dKT=d.get("dKT"), dVT=d.get("dVT"), act=act)
     return got, ref
 
 
@@ -405,3 +405,38 @@ def test_logit_gate_decode():
         ro = oracle.decode_step(x["q"], x["k"], x["v"], logits, Kr, Vr, gate_is_logits=True, tau=8.0)
         assert rel_err(to_np(o), ro, True) <= TOL["bf16"]
     assert rel_err(to_np(Ks), Kr) <= 1e-5 and rel_err(to_np(Vs), Vr) <= 1e-5
+
+
+# ------------------------------------------------------------------ replacements of the slot softmax
+# (the paper's ablation on the non-linearity between the two passes)
+ACTS = ["none", "relu", "swish", "relu2"]
+
+
+@pytest.mark.parametrize("act", ACTS)
+@pytest.mark.parametrize("io,impl,T", [("f32", "auto", 150), ("bf16", "tc", 300)])
+def test_slot_activation_variants_fwd_bwd(act, io, impl, T):
+    B, H, dk, dv, m = 2, 2, 128, 128, 64
+    d = rand_inputs(700 + T, B, T, H, dk, dv, m, io, init=True, final_grads=True)
+    tc = impl == "tc"
+    got, gate = run_fwd(d, B, T, H, dk, dv, m, io, impl=impl, scale=0.5, act=act)
+    ef = check_fwd(d, got, gate, io, scale=0.5, tc=tc, act=act)
+    gb, rb = run_bwd(d, B, T, H, dk, dv, m, io, impl=impl, scale=0.5, saved=True, act=act)
+    eb = check_bwd(gb, rb, TOL[io], tc=tc)
+    print("slot act", act, io, ef, eb)
+
+
+@pytest.mark.parametrize("act", ACTS)
+def test_slot_activation_variants_decode(act):
+    S, H, dk, dv, m = 3, 4, 128, 128, 64
+    w = W.CONFIGS["decode"].scaled(B=S, H=H, d_k=dk, d_v=dv, m=m, io="bf16")
+    st = W.make_decode_states(w)
+    Ks, Vs = to_dev(st["K"]), to_dev(st["V"])
+    Kr, Vr = st["K"].astype(np.float64), st["V"].astype(np.float64)
+    p = gsa.Params(S, 1, H, dk, dv, m, io="bf16", scale=0.8, slot_act=act)
+    for step in range(3):
+        x = W.make_decode_step_inputs(w, step)
+        o = gsa.gsa_decode_step(p, to_dev(x["q"], "bf16"), to_dev(x["k"], "bf16"), to_dev(x["v"], "bf16"),
+                                to_dev(x["gate"]), Ks, Vs)
+        ro = oracle.decode_step(x["q"], x["k"], x["v"], x["gate"], Kr, Vr, scale=0.8, act=act)
+        assert rel_err(to_np(o), ro, True) <= TOL["bf16"]
+
