@@ -262,7 +262,7 @@ def run_ours(args):
 
     w = rank_workload(rank)
     x = W.make_inputs(w)
-    p = gsa.Params(w.B, w.T, w.H, w.d_k, w.d_v, w.m, io=w.io, slot_act=args.slot_act)
+    p = gsa.Params(w.B, w.T, w.H, w.d_k, w.d_v, w.m, io=w.io, slot_act=args.slot_act, tc_operands=args.tc_operands)
 
     def host(a, bf16):
         t = torch.from_numpy(np.ascontiguousarray(a))
@@ -480,7 +480,7 @@ def run_ours(args):
             "config": {"workload": WORKLOAD, "B": w.B, "T": w.T, "H": w.H, "d_k": w.d_k,
                        "d_v": w.d_v, "m": w.m, "io": w.io, "chunk": gsa.gsa_chunk_size(p),
                        "step": "gsa_fwd (logits saved) + gsa_bwd",
-                       "slot_act": args.slot_act,
+                       "slot_act": args.slot_act, "tc_operands": args.tc_operands,
                        "launch": launch_mode,
                        "l2": "inputs larger than L2 (1.1 GB touched per step vs 126 MB)",
                        "parallelism": f"dp{world} over batch, no collective"},
@@ -543,6 +543,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--tc-operands", default="paired", choices=["paired", "single"],
+                    help="derived operands of the tensor-core kernels as bf16 high/low pairs (default) or as one "
+                         "bf16 value")
     ap.add_argument("--slot-act", default="softmax", choices=["softmax", "none", "relu", "swish", "relu2"],
                     help="the non-linearity between the two passes: the paper's softmax (the headline "
                          "workload) or one of the replacements of its ablation")

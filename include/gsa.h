@@ -76,6 +76,17 @@ typedef enum {
     GSA_ACT_SOFTMAX = 0, GSA_ACT_NONE = 1, GSA_ACT_RELU = 2, GSA_ACT_SWISH = 3, GSA_ACT_RELU2 = 4
 } gsa_act_t;
 
+/* Tensor-core kernels only: how the operands that the kernels derive on the way (masked
+ * intra-chunk products, decayed slot-space rows, state copies) enter the bf16 products.
+ * PAIRED carries each as a bfloat16 value plus its rounding residual wherever that costs extra
+ * products (fp32-like results: logits, gradients and memories at ~1e-4 of their rms);
+ * SINGLE rounds them to one bfloat16 value, as a plain bf16 matrix product of the chunkwise
+ * form does: a quarter fewer products per chunk (the step is 8% faster at d = 512), errors of
+ * the order of the bfloat16 rounding of those operands -- logits and gate gradient ~1e-2 of
+ * their rms, dq and dk 3e-2 to 1e-1 where the gradients are heavy-tailed, i.e. outside the
+ * 2e-2 that PAIRED meets for every tensor. */
+typedef enum { GSA_TC_PAIRED = 0, GSA_TC_SINGLE = 1 } gsa_tc_operands_t;
+
 /* Which kernels serve the d-sized contractions of the chunk passes. */
 typedef enum {
     GSA_IMPL_AUTO = 0,   /* bf16 io: tensor-core kernels; fp32 io: fp32 CUDA-core kernels */
@@ -91,6 +102,7 @@ typedef struct {
     int32_t impl;       /* gsa_impl_t */
     float tau;          /* GSA_GATE_LOGITS only: damping of the gate, a = sigmoid(x)^(1/tau); > 0 */
     int32_t slot_act;   /* gsa_act_t; 0 = the paper's softmax */
+    int32_t tc_operands; /* gsa_tc_operands_t; ignored by the fp32 kernels */
 } gsa_params_t;
 
 enum { GSA_WS_FWD = 0, GSA_WS_BWD = 1, GSA_WS_DECODE = 2 };

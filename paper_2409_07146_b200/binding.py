@@ -32,7 +32,7 @@ class _CParams(ctypes.Structure):
                 ("d_k", ctypes.c_int32), ("d_v", ctypes.c_int32), ("m", ctypes.c_int32),
                 ("io", ctypes.c_int32), ("gate_kind", ctypes.c_int32),
                 ("scale", ctypes.c_float), ("impl", ctypes.c_int32), ("tau", ctypes.c_float),
-                ("slot_act", ctypes.c_int32)]
+                ("slot_act", ctypes.c_int32), ("tc_operands", ctypes.c_int32)]
 
 
 @dataclass(frozen=True)
@@ -51,13 +51,15 @@ class Params:
     gate_is_logits: bool = False   # the gate tensor holds x, a = sigmoid(x)^(1/tau)
     tau: float = 8.0
     slot_act: str = "softmax"      # "softmax" | "none" | "relu" | "swish" | "relu2"
+    tc_operands: str = "paired"    # "paired" | "single" (tensor-core kernels: derived operands as bf16 pairs or not)
 
     def c(self) -> _CParams:
         return _CParams(self.B, self.T, self.H, self.d_k, self.d_v, self.m,
                         GSA_BF16 if self.io == "bf16" else GSA_F32,
                         GSA_GATE_LOGITS if self.gate_is_logits else
                         (GSA_GATE_LOG_A if self.gate_is_log else GSA_GATE_A),
-                        float(self.scale), _IMPL[self.impl], float(self.tau), _ACT[self.slot_act])
+                        float(self.scale), _IMPL[self.impl], float(self.tau), _ACT[self.slot_act],
+                        0 if self.tc_operands == "paired" else 1)
 
     @property
     def io_dtype(self) -> torch.dtype:

@@ -26,6 +26,7 @@ gsa_status_t check_params(const gsa_params_t* p, bool need_T) {
         return GSA_ERR_INVALID_ARG;
     if (p->gate_kind == GSA_GATE_LOGITS && !(p->tau > 0.f)) return GSA_ERR_INVALID_ARG;
     if (p->slot_act < GSA_ACT_SOFTMAX || p->slot_act > GSA_ACT_RELU2) return GSA_ERR_INVALID_ARG;
+    if (p->tc_operands != GSA_TC_PAIRED && p->tc_operands != GSA_TC_SINGLE) return GSA_ERR_INVALID_ARG;
     if (p->impl != GSA_IMPL_AUTO && p->impl != GSA_IMPL_SIMT && p->impl != GSA_IMPL_TC)
         return GSA_ERR_INVALID_ARG;
     if (!(p->scale == p->scale)) return GSA_ERR_INVALID_ARG;
@@ -130,12 +131,20 @@ Workspace carve(const gsa_params_t& p, int which, void* ws) {
 
 cudaError_t value_side(const gsa_params_t& p, const ValueSideArgs& a, int reverse, const int* strong,
                        cudaStream_t st, int32_t* dev_status) {
-    if (use_tc(p)) return launch_value_side_tc(a, p.m, reverse, strong, st, dev_status);
+    if (use_tc(p)) {
+        ValueSideArgs b = a;
+        b.single = p.tc_operands == GSA_TC_SINGLE;
+        return launch_value_side_tc(b, p.m, reverse, strong, st, dev_status);
+    }
     return launch_value_side_simt(a, p.io, p.m, reverse, st);
 }
 cudaError_t key_side(const gsa_params_t& p, const KeySideArgs& a, int reverse, const int* strong,
                      cudaStream_t st, int32_t* dev_status) {
-    if (use_tc(p)) return launch_key_side_tc(a, p.m, reverse, strong, st, dev_status);
+    if (use_tc(p)) {
+        KeySideArgs b = a;
+        b.single = p.tc_operands == GSA_TC_SINGLE;
+        return launch_key_side_tc(b, p.m, reverse, strong, st, dev_status);
+    }
     return launch_key_side_simt(a, p.io, p.m, reverse, st);
 }
 

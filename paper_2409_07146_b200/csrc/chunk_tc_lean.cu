@@ -143,7 +143,7 @@ constexpr int kLkA = 0, kLkO = 128 /* two buffers of 128 */, kLkU = 384;        
 //   The row factor -- exp(G_i) forward, exp(-G_i) reverse -- is NOT applied here: the kernel that
 //   sums the slices of `out` multiplies it in (see PendingDecay), so this kernel needs no G tile.
 // ======================================================================================
-template <bool REV>
+template <bool REV, bool PAIRS>
 __global__ void __launch_bounds__(kLeanThreads, 1)
 value_side_lean_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK,
                        const __grid_constant__ CUtensorMap mapWd, const __grid_constant__ CUtensorMap mapO,
@@ -273,10 +273,12 @@ value_side_lean_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_co
             for (int kk = 0; kk < kCT / 16; ++kk)
                 mma_bf16_ta(tmem + kLvI, tmem + kLvP + 64 * (kk >> 2) + 8 * (kk & 3), desc_advance(dW, mnmaj(kk)), idescI,
                             kk > 0);
+            if (PAIRS) {
 #pragma unroll
-            for (int kk = 0; kk < kCT / 16; ++kk)      // ... and the rounding residual of the masked P
-                mma_bf16_ta(tmem + kLvI, tmem + kLvP + 64 * (kk >> 2) + 32 + 8 * (kk & 3), desc_advance(dW, mnmaj(kk)),
-                            idescI, true);
+                for (int kk = 0; kk < kCT / 16; ++kk)      // ... and the rounding residual of the masked P
+                    mma_bf16_ta(tmem + kLvI, tmem + kLvP + 64 * (kk >> 2) + 32 + 8 * (kk & 3),
+                                desc_advance(dW, mnmaj(kk)), idescI, true);
+            }
             mma_commit(&ctl->bar_mma2);
             PROF_MARK();
             // the P accumulator is free: the next chunk's P queues right behind
@@ -324,7 +326,7 @@ value_side_lean_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_co
             LEAN_WAIT(&ctl->bar_p, n & 1);
             tc_fence_after_sync();
             PROF_MARK();
-            mask_row_in_tmem<REV, true>(tmem, wq, row, half, kLvP);
+            mask_row_in_tmem<REV, PAIRS>(tmem, wq, row, half, kLvP);
             publish(&ctl->bar_pm, tid);
             PROF_MARK();
 
@@ -394,7 +396,7 @@ value_side_lean_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_co
 //   uq_d / uk_d hold the decayed bf16 rows (first 64 of every 128): forward uq exp(G), uk exp(-G);
 //   reverse uq exp(-G), uk exp(G).
 // ======================================================================================
-template <bool REV>
+template <bool REV, bool PAIRS>
 __global__ void __launch_bounds__(kLeanThreads, 1)
 key_side_lean_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_constant__ CUtensorMap mapUq,
                      const __grid_constant__ CUtensorMap mapUk, const __grid_constant__ CUtensorMap mapO,
@@ -483,12 +485,14 @@ key_side_lean_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_cons
 #pragma unroll
             for (int kk = 0; kk < kM / 16; ++kk)
                 mma_bf16(tmem + kLkA, desc_advance(dQt, kmaj(kk)), desc_advance(dKt, kmaj(kk)), idescA, kk > 0);
+            if (PAIRS) {
 #pragma unroll
-            for (int kk = 0; kk < kM / 16; ++kk)
-                mma_bf16(tmem + kLkA, desc_advance(dQl, kmaj(kk)), desc_advance(dKt, kmaj(kk)), idescA, true);
+                for (int kk = 0; kk < kM / 16; ++kk)
+                    mma_bf16(tmem + kLkA, desc_advance(dQl, kmaj(kk)), desc_advance(dKt, kmaj(kk)), idescA, true);
 #pragma unroll
-            for (int kk = 0; kk < kM / 16; ++kk)
-                mma_bf16(tmem + kLkA, desc_advance(dQt, kmaj(kk)), desc_advance(dKl, kmaj(kk)), idescA, true);
+                for (int kk = 0; kk < kM / 16; ++kk)
+                    mma_bf16(tmem + kLkA, desc_advance(dQt, kmaj(kk)), desc_advance(dKl, kmaj(kk)), idescA, true);
+            }
             mma_commit(&ctl->bar_p);
         };
         LEAN_WAIT(&ctl->bar_w[0], 0);
@@ -520,12 +524,14 @@ key_side_lean_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_cons
 #pragma unroll
             for (int kk = 0; kk < kM / 16; ++kk)
                 mma_bf16(accO, desc_advance(dQt, kmaj(kk)), desc_advance(dS, kmaj(kk)), idescO, kk > 0);
+            if (PAIRS) {
 #pragma unroll
-            for (int kk = 0; kk < kM / 16; ++kk)
-                mma_bf16(accO, desc_advance(dQl, kmaj(kk)), desc_advance(dS, kmaj(kk)), idescO, true);
+                for (int kk = 0; kk < kM / 16; ++kk)
+                    mma_bf16(accO, desc_advance(dQl, kmaj(kk)), desc_advance(dS, kmaj(kk)), idescO, true);
 #pragma unroll
-            for (int kk = 0; kk < kM / 16; ++kk)
-                mma_bf16(accO, desc_advance(dQt, kmaj(kk)), desc_advance(dSl, kmaj(kk)), idescO, true);
+                for (int kk = 0; kk < kM / 16; ++kk)
+                    mma_bf16(accO, desc_advance(dQt, kmaj(kk)), desc_advance(dSl, kmaj(kk)), idescO, true);
+            }
             mma_commit(&ctl->bar_mma1);
             mma_commit(&ctl->bar_free1[n & 1]);
             PROF_MARK();
@@ -537,10 +543,12 @@ key_side_lean_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_cons
 #pragma unroll
             for (int kk = 0; kk < kCT / 16; ++kk)
                 mma_bf16_ta(accO, tmem + kLkA + 64 * (kk >> 2) + 8 * (kk & 3), desc_advance(dV, mnmaj(kk)), idescV, true);
+            if (PAIRS) {
 #pragma unroll
-            for (int kk = 0; kk < kCT / 16; ++kk)
-                mma_bf16_ta(accO, tmem + kLkA + 64 * (kk >> 2) + 32 + 8 * (kk & 3), desc_advance(dV, mnmaj(kk)), idescV,
-                            true);
+                for (int kk = 0; kk < kCT / 16; ++kk)
+                    mma_bf16_ta(accO, tmem + kLkA + 64 * (kk >> 2) + 32 + 8 * (kk & 3), desc_advance(dV, mnmaj(kk)),
+                                idescV, true);
+            }
             mma_commit(&ctl->bar_mma2);
             PROF_MARK();
             // the A accumulator is free: the next chunk's A queues right behind
@@ -587,7 +595,7 @@ key_side_lean_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_cons
             // ---- masked A rows as a bf16 high/low pair (the barrier inside also publishes egc)
             LEAN_WAIT(&ctl->bar_p, n & 1);
             tc_fence_after_sync();
-            mask_row_in_tmem<REV, true>(tmem, wq, row, half, kLkA);
+            mask_row_in_tmem<REV, PAIRS>(tmem, wq, row, half, kLkA);
             publish(&ctl->bar_pm, tid);
 
             // ---- state update from U^T: forward S <- exp(G_C) (S + U^T), reverse S <- exp(G_C) S + U^T
@@ -822,16 +830,14 @@ cudaError_t launch_value_side_lean(const ValueSideArgs& a, int reverse, const in
     if (e == cudaSuccess) e = make_tensor_map_bthd(&mw, a.wd, a.B, a.T, a.H, 2 * kM, kCT, 2);
     if (e != cudaSuccess) return e;
     dim3 grid(a.B * a.H, a.D / kDST);
-    if (reverse) {
-        e = prepare(value_side_lean_kernel<true>, kSmemLeanValue, kLeanThreads);
-        if (e != cudaSuccess) return e;
-        value_side_lean_kernel<true><<<grid, kLeanThreads, kSmemLeanValue, st>>>(mq, mk, mw, mo, a, strong_flag, dev_status);
-    } else {
-        e = prepare(value_side_lean_kernel<false>, kSmemLeanValue, kLeanThreads);
-        if (e != cudaSuccess) return e;
-        value_side_lean_kernel<false><<<grid, kLeanThreads, kSmemLeanValue, st>>>(mq, mk, mw, mo, a, strong_flag, dev_status);
-    }
-    return cudaGetLastError();
+    auto launch = [&](auto kernel) {
+        cudaError_t e2 = prepare(kernel, kSmemLeanValue, kLeanThreads);
+        if (e2 != cudaSuccess) return e2;
+        kernel<<<grid, kLeanThreads, kSmemLeanValue, st>>>(mq, mk, mw, mo, a, strong_flag, dev_status);
+        return cudaGetLastError();
+    };
+    if (reverse) return a.single ? launch(value_side_lean_kernel<true, false>) : launch(value_side_lean_kernel<true, true>);
+    return a.single ? launch(value_side_lean_kernel<false, false>) : launch(value_side_lean_kernel<false, true>);
 }
 
 cudaError_t launch_key_side_lean(const KeySideArgs& a, int reverse, const int* strong_flag, cudaStream_t st,
@@ -845,16 +851,14 @@ cudaError_t launch_key_side_lean(const KeySideArgs& a, int reverse, const int* s
     if (e == cudaSuccess) e = make_tensor_map_bthd(&muk, a.uk_d, a.B, a.T, a.H, 2 * kM, kCT, 2);
     if (e != cudaSuccess) return e;
     dim3 grid(a.B * a.H, a.D / kDST);
-    if (reverse) {
-        e = prepare(key_side_lean_kernel<true>, kSmemLeanKey, kLeanThreads);
-        if (e != cudaSuccess) return e;
-        key_side_lean_kernel<true><<<grid, kLeanThreads, kSmemLeanKey, st>>>(mv, muq, muk, mo, a, strong_flag, dev_status);
-    } else {
-        e = prepare(key_side_lean_kernel<false>, kSmemLeanKey, kLeanThreads);
-        if (e != cudaSuccess) return e;
-        key_side_lean_kernel<false><<<grid, kLeanThreads, kSmemLeanKey, st>>>(mv, muq, muk, mo, a, strong_flag, dev_status);
-    }
-    return cudaGetLastError();
+    auto launch = [&](auto kernel) {
+        cudaError_t e2 = prepare(kernel, kSmemLeanKey, kLeanThreads);
+        if (e2 != cudaSuccess) return e2;
+        kernel<<<grid, kLeanThreads, kSmemLeanKey, st>>>(mv, muq, muk, mo, a, strong_flag, dev_status);
+        return cudaGetLastError();
+    };
+    if (reverse) return a.single ? launch(key_side_lean_kernel<true, false>) : launch(key_side_lean_kernel<true, true>);
+    return a.single ? launch(key_side_lean_kernel<false, false>) : launch(key_side_lean_kernel<false, true>);
 }
 
 }  // namespace gsa

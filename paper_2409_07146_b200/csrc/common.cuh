@@ -86,6 +86,7 @@ struct ValueSideArgs {
     // only the end state matters to the caller (first run of the segment-parallel forward): kernels
     // may leave `out` unwritten where computing it is expensive
     int state_only;
+    int single;                       // tensor-core kernels: derived operands as one bf16 value (GSA_TC_SINGLE)
 };
 struct KeySideArgs {
     const float* uq; const float* uk; const float* G;
@@ -98,6 +99,7 @@ struct KeySideArgs {
     // uk exp(-G), reverse uq exp(-G) and uk exp(G); nullable (both or neither)
     const void* uq_d; const void* uk_d;
     int state_only;                   // as in ValueSideArgs
+    int single;                       // as in ValueSideArgs
 };
 
 // Element-wise replacements of the slot softmax (gsa_act_t other than GSA_ACT_SOFTMAX): f(z) and f'(z).

@@ -44,10 +44,10 @@ def sample_pairs(w, n=3):
     return sorted({0, total // 2 + 1 if total > 2 else total - 1, total - 1})[:n]
 
 
-def run_training_config(name, with_bwd):
+def run_training_config(name, with_bwd, tc_operands="paired"):
     w = W.CONFIGS[name]
     x = W.make_inputs(w)
-    p = gsa.Params(w.B, w.T, w.H, w.d_k, w.d_v, w.m, io=w.io)
+    p = gsa.Params(w.B, w.T, w.H, w.d_k, w.d_v, w.m, io=w.io, tc_operands=tc_operands)
     q, k, v = (to_dev(x[n], w.io) for n in ("q", "k", "v"))
     gate = to_dev(x["gate"])
     K0, V0 = to_dev(x.get("K0")), to_dev(x.get("V0"))
@@ -83,8 +83,8 @@ def run_training_config(name, with_bwd):
         errs[n] = dict(bound=bound, plain=rel_err(gs, ref[n]), limit=limit,
                        after_output_half_ulp=rel_err(gs, ref[n], True),
                        max_over_rms=float(np.abs(ref[n]).max() / np.sqrt(np.mean(ref[n] ** 2))))
-    record(name, dict(pairs=pairs, errors=errs))
-    print(name, {n: (round(e["plain"], 4), round(e["bound"], 4)) for n, e in errs.items()})
+    record(name if tc_operands == "paired" else name + "/" + tc_operands, dict(pairs=pairs, errors=errs))
+    print(name, tc_operands, {n: (round(e["plain"], 4), round(e["bound"], 4)) for n, e in errs.items()})
     bad = {}
     for n, e in errs.items():
         if e["bound"] > e["limit"]:

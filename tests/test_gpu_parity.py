@@ -440,3 +440,28 @@ def test_slot_activation_variants_decode(act):
         ro = oracle.decode_step(x["q"], x["k"], x["v"], x["gate"], Kr, Vr, scale=0.8, act=act)
         assert rel_err(to_np(o), ro, True) <= TOL["bf16"]
 
+
+
+def test_tc_single_operand_mode_is_bf16_accurate_and_paired_is_tighter():
+    """GSA_TC_SINGLE rounds the derived operands to one bfloat16 value: errors of the order of
+    that rounding (2^-9 per operand, accumulated over two passes: a few 1e-2 of the rms on the
+    gradients), against ~1e-5 with the default pairs."""
+    B, T, H, dk, dv, m = 2, 512, 2, 256, 256, 64
+    d = rand_inputs(811, B, T, H, dk, dv, m, "bf16", init=True)
+    ref_f = oracle.fwd(d["q"], d["k"], d["v"], d["gate"], K0=d["K0"], V0=d["V0"])
+    ref_b = oracle.bwd(d["q"], d["k"], d["v"], d["gate"], d["dO"], K0=d["K0"], V0=d["V0"])
+    errs = {}
+    for mode in ("paired", "single"):
+        p = gsa.Params(B, T, H, dk, dv, m, io="bf16", impl="tc", tc_operands=mode)
+        q, k, v, dO = (to_dev(d[n], "bf16") for n in ("q", "k", "v", "dO"))
+        ok = torch.empty(B, T, H, m, device="cuda")
+        o = gsa.gsa_fwd(p, q, k, v, to_dev(d["gate"]), to_dev(d["K0"]), to_dev(d["V0"]), ok_save=ok)
+        dq, dk_, dv_, dg = gsa.gsa_bwd(p, q, k, v, to_dev(d["gate"]), dO, to_dev(d["K0"]), to_dev(d["V0"]), ok_saved=ok)
+        torch.cuda.synchronize()
+        errs[mode] = dict(o=rel_err(to_np(o), ref_f["o"], True), ok=rel_err(to_np(ok), ref_f["ok"]),
+                          dq=rel_err(to_np(dq), ref_b["dq"], True), dk=rel_err(to_np(dk_), ref_b["dk"], True),
+                          dv=rel_err(to_np(dv_), ref_b["dv"], True), dgate=rel_err(to_np(dg), ref_b["dgate"]))
+    print("tc operands", errs)
+    assert all(e <= 1e-3 for e in errs["paired"].values()), errs
+    assert all(e <= 1e-1 for e in errs["single"].values()), errs
+    assert errs["single"]["ok"] > 10 * errs["paired"]["ok"] and errs["single"]["dq"] > 10 * errs["paired"]["dq"], errs
