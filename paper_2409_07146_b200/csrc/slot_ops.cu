@@ -14,19 +14,19 @@ namespace gsa {
 // chunk length of the kernels that will consume G (64 or 128).
 constexpr int kCumRows = 8;
 
-// x as a bf16 pair: the rounded value and the rounding residual
-__device__ __forceinline__ void split_bf16(float x, __nv_bfloat16& hi, __nv_bfloat16& lo) {
-    hi = __float2bfloat16_rn(x);
-    lo = __float2bfloat16_rn(x - __bfloat162float(hi));
+// (x0, x1) as a packed bf16 pair and the packed rounding residuals: two packed conversions
+__device__ __forceinline__ void split_bf16x2(float x0, float x1, uint32_t& hi, uint32_t& lo) {
+    const __nv_bfloat162 h = __floats2bfloat162_rn(x0, x1);
+    hi = *reinterpret_cast<const uint32_t*>(&h);
+    const __nv_bfloat162 l = __floats2bfloat162_rn(x0 - __uint_as_float(hi << 16), x1 - __uint_as_float(hi & 0xffff0000u));
+    lo = *reinterpret_cast<const uint32_t*>(&l);
 }
-// two adjacent columns (c, c+1; c even) of a decayed-operand row [hi(M) | lo(M)]
 template <int M>
 __device__ __forceinline__ void store_split2(__nv_bfloat16* row, int c, float x0, float x1) {
-    __nv_bfloat162 hi, lo;
-    split_bf16(x0, hi.x, lo.x);
-    split_bf16(x1, hi.y, lo.y);
-    *reinterpret_cast<__nv_bfloat162*>(row + c) = hi;
-    *reinterpret_cast<__nv_bfloat162*>(row + M + c) = lo;
+    uint32_t hi, lo;
+    split_bf16x2(x0, x1, hi, lo);
+    *reinterpret_cast<uint32_t*>(row + c) = hi;
+    *reinterpret_cast<uint32_t*>(row + M + c) = lo;
 }
 
 template <int M>
@@ -63,14 +63,15 @@ __global__ void __launch_bounds__(M * 8, 2) gate_cumsum_kernel(const float* __re
         g[i].y = fmaxf(g[i].y, kLogGateMin);
         if (i < rows) *reinterpret_cast<float2*>(I + base + (size_t)i * stride) = inps[i];
     }
-    // running sums in fp64 (a handful of adds per thread): G is then the correctly rounded
-    // cumulative sum, which matters when strong decay makes |G| reach the hundreds
-    double acc0 = 0.0, acc1 = 0.0;
+    // running sums: fp32 inside the thread's 8 rows (g becomes the running sum), fp64 across the
+    // row groups -- G stays within an ulp of the exact cumulative sum also where strong decay
+    // makes |G| reach the hundreds, without a conversion per element
 #pragma unroll
-    for (int i = 0; i < kCumRows; ++i) {
-        acc0 += (i < rows) ? (double)g[i].x : 0.0;
-        acc1 += (i < rows) ? (double)g[i].y : 0.0;
+    for (int i = 1; i < kCumRows; ++i) {
+        g[i].x = (i < rows) ? g[i - 1].x + g[i].x : g[i - 1].x;
+        g[i].y = (i < rows) ? g[i - 1].y + g[i].y : g[i - 1].y;
     }
+    const double acc0 = rows > 0 ? (double)g[kCumRows - 1].x : 0.0, acc1 = rows > 0 ? (double)g[kCumRows - 1].y : 0.0;
     group_sum[grp][s] = acc0;
     group_sum[grp][s + 1] = acc1;
     __syncthreads();
@@ -86,13 +87,13 @@ __global__ void __launch_bounds__(M * 8, 2) gate_cumsum_kernel(const float* __re
         const int seg = (int)(((long long)n * chunk) / (T / nseg));
         strong_flag[(b * nseg + seg) * H + h] = 1;
     }
-    // second pass over the same rows: the running sums continue from the groups before
+    // second pass over the same rows: the sums of the groups before as a float pair (value, rest)
+    const float b0h = (float)before0, b0l = (float)(before0 - (double)b0h);
+    const float b1h = (float)before1, b1l = (float)(before1 - (double)b1h);
 #pragma unroll
     for (int i = 0; i < kCumRows; ++i)
         if (i < rows) {
-            before0 += (double)g[i].x;
-            before1 += (double)g[i].y;
-            const float G0 = (float)before0, G1 = (float)before1;
+            const float G0 = b0h + (b0l + g[i].x), G1 = b1h + (b1l + g[i].y);
             *reinterpret_cast<float2*>(G + base + (size_t)i * stride) = make_float2(G0, G1);
             if (decayed != nullptr) {
                 // (meaningful for moderate decay only; pairs with a strong-decay chunk do not read it)
@@ -132,13 +133,11 @@ __device__ __forceinline__ void st_vec(float* p, const float (&x)[kSmR]) {
 // the lane's slots of a decayed-operand row [hi(M) | lo(M)]
 template <int M>
 __device__ __forceinline__ void st_split(__nv_bfloat16* row, int c, const float (&x)[kSmR]) {
-    __nv_bfloat162 h0, h1, l0, l1;
-    split_bf16(x[0], h0.x, l0.x);
-    split_bf16(x[1], h0.y, l0.y);
-    split_bf16(x[2], h1.x, l1.x);
-    split_bf16(x[3], h1.y, l1.y);
-    *reinterpret_cast<uint2*>(row + c) = make_uint2(*reinterpret_cast<uint32_t*>(&h0), *reinterpret_cast<uint32_t*>(&h1));
-    *reinterpret_cast<uint2*>(row + M + c) = make_uint2(*reinterpret_cast<uint32_t*>(&l0), *reinterpret_cast<uint32_t*>(&l1));
+    uint32_t h0, h1, l0, l1;
+    split_bf16x2(x[0], x[1], h0, l0);
+    split_bf16x2(x[2], x[3], h1, l1);
+    *reinterpret_cast<uint2*>(row + c) = make_uint2(h0, h1);
+    *reinterpret_cast<uint2*>(row + M + c) = make_uint2(l0, l1);
 }
 template <int LPR>
 __device__ __forceinline__ float row_max(float x) {
