@@ -38,12 +38,12 @@ WORKLOAD = "train_1p3b"
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the tensor-core kernels on this
 # workload, from one `ncu --set full` capture (profiles/step_kernels_train_1p3b_ncu_full.md).
 NCU_TRAFFIC = {
-    "pass1_value_side": 187349240, "bwd_dp_value_side": 187349240,
-    "bwd_dIv_value_side_rev": 188625912, "bwd_dIk_value_side_rev": 188625912,
-    "pass2_key_side": 129206520, "bwd_dq_key_side": 129206520,
-    "bwd_dv_key_side_rev": 130708992, "bwd_dk_key_side_rev": 130708992,
-    "gate_cumsum": 18406144, "slot_softmax": 93043712, "slot_softmax_bwd": 122202876,
-    "gate_grad": 232713984,     # local + scan + carry
+    "pass1_value_side": 186965760, "bwd_dp_value_side": 185658112,
+    "bwd_dIv_value_side_rev": 188858112, "bwd_dIk_value_side_rev": 187463680,
+    "pass2_key_side": 129739520, "bwd_dq_key_side": 135778048,
+    "bwd_dv_key_side_rev": 130483200, "bwd_dk_key_side_rev": 132975616,
+    "gate_cumsum": 17926144, "slot_softmax": 92744448, "slot_softmax_bwd": 118787072,
+    "gate_grad": 233491456,     # local + scan + carry
 }
 
 
