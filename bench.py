@@ -287,11 +287,16 @@ def run_ours(args):
 
     outs = {"o": o, "dq": dq, "dk": dk, "dv": dv, "dgate": dg}
 
+    # the forward leaves the gate kernel's products (as it leaves the logits) for the backward of
+    # the same step: memory for time, 50 MB at this shape; --recompute-gate times the plain pair
+    gate_blk = None if args.recompute_gate else gsa.gate_block(p, dev)
+
     def step(src, dst=outs):
         gsa.gsa_fwd(p, src["q"], src["k"], src["v"], src["gate"], o=dst["o"], ok_save=ok, ws=ws_f,
-                    dev_status=status)
+                    dev_status=status, gate_save=gate_blk)
         gsa.gsa_bwd(p, src["q"], src["k"], src["v"], src["gate"], src["dO"], ok_saved=ok, dq=dst["dq"],
-                    dk=dst["dk"], dv=dst["dv"], dgate=dst["dgate"], ws=ws_b, dev_status=status)
+                    dk=dst["dk"], dv=dst["dv"], dgate=dst["dgate"], ws=ws_b, dev_status=status,
+                    gate_saved=gate_blk)
 
     def barrier():
         if world > 1:
@@ -322,7 +327,7 @@ def run_ours(args):
         sampler.start()
     for _ in range(max(args.warmup, 3)):
         step(d_in)
-    # One step = 23 kernels on six streams: it is captured once into a CUDA graph and the timed
+    # One step = 22 kernels on six streams: it is captured once into a CUDA graph and the timed
     # region replays that graph (the library calls are capture-safe: no allocation, no host
     # synchronisation).  --no-graph times the plain calls instead.
     run_step, launch_mode = (lambda: step(d_in)), "library calls, one step after the other"
@@ -479,7 +484,8 @@ def run_ours(args):
             "data": "synthetic (seeded N(0,1) q,k,v,dO; gate sigmoid(N(0,1))^(1/8))",
             "config": {"workload": WORKLOAD, "B": w.B, "T": w.T, "H": w.H, "d_k": w.d_k,
                        "d_v": w.d_v, "m": w.m, "io": w.io, "chunk": gsa.gsa_chunk_size(p),
-                       "step": "gsa_fwd (logits saved) + gsa_bwd",
+                       "step": ("gsa_fwd (logits saved) + gsa_bwd" if args.recompute_gate else
+                                "gsa_fwd_save_gate (logits and the gate kernel's products saved) + gsa_bwd_saved_gate"),
                        "slot_act": args.slot_act, "tc_operands": args.tc_operands,
                        "launch": launch_mode,
                        "l2": "inputs larger than L2 (1.1 GB touched per step vs 126 MB)",
@@ -543,6 +549,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--recompute-gate", action="store_true",
+                    help="plain gsa_fwd + gsa_bwd: the backward runs the gate kernel again instead of reading the "
+                         "forward's saved block")
     ap.add_argument("--tc-operands", default="paired", choices=["paired", "single"],
                     help="derived operands of the tensor-core kernels as bf16 high/low pairs (default) or as one "
                          "bf16 value")

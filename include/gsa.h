@@ -105,7 +105,7 @@ typedef struct {
     int32_t tc_operands; /* gsa_tc_operands_t; ignored by the fp32 kernels */
 } gsa_params_t;
 
-enum { GSA_WS_FWD = 0, GSA_WS_BWD = 1, GSA_WS_DECODE = 2 };
+enum { GSA_WS_FWD = 0, GSA_WS_BWD = 1, GSA_WS_DECODE = 2, GSA_WS_GATE = 3 };
 
 /* Chunk length C of the chunkwise form that these params select (Algorithm 1 leaves C
  * open): 128 for the tensor-core kernels, 64 for the fp32 CUDA-core kernels; 0 for
@@ -113,7 +113,8 @@ enum { GSA_WS_FWD = 0, GSA_WS_BWD = 1, GSA_WS_DECODE = 2 };
 GSA_API int32_t gsa_chunk_size(const gsa_params_t* params);
 
 /* Bytes of scratch `which` (GSA_WS_*) needs for these params; 0 for decode and
- * for invalid params. */
+ * for invalid params.  GSA_WS_GATE: the block that gsa_fwd_save_gate fills for
+ * gsa_bwd_saved_gate. */
 GSA_API size_t gsa_workspace_bytes(const gsa_params_t* params, int32_t which);
 
 GSA_API const char* gsa_status_string(gsa_status_t status);
@@ -161,6 +162,29 @@ GSA_API gsa_status_t gsa_bwd(const gsa_params_t* params, const void* q, const vo
                      const float* dKT, const float* dVT, void* dq, void* dk,
                      void* dv, float* dgate, float* dK0, float* dV0, void* ws,
                      size_t ws_bytes, void* stream, int32_t* dev_status);
+
+/*
+ * The same two calls for a training step that trades memory for the backward's gate kernel
+ * (the save-instead-of-recompute side of the trade-off the paper discusses in Sec. 4,
+ * "Efficiency"): gsa_fwd_save_gate leaves the products of chunk_cumsum (the cumulative log
+ * gate, the input gate, its decayed bf16 rows and the per-(batch, head) decay flags) in
+ * gate_save, a device block of gsa_workspace_bytes(params, GSA_WS_GATE) bytes, 256-byte
+ * aligned, owned by the caller; gsa_bwd_saved_gate reads them from there instead of running
+ * the gate kernel again.  Both calls must use the same params and the same gate tensor;
+ * nothing checks that.  A missing, misaligned or short block is GSA_ERR_WORKSPACE.
+ */
+GSA_API gsa_status_t gsa_fwd_save_gate(const gsa_params_t* params, const void* q, const void* k,
+                                       const void* v, const float* gate, const float* K0,
+                                       const float* V0, void* o, float* ok_save, float* KT,
+                                       float* VT, void* gate_save, size_t gate_save_bytes, void* ws,
+                                       size_t ws_bytes, void* stream, int32_t* dev_status);
+GSA_API gsa_status_t gsa_bwd_saved_gate(const gsa_params_t* params, const void* q, const void* k,
+                                        const void* v, const float* gate, const float* K0,
+                                        const float* V0, const float* ok_saved, const void* dO,
+                                        const float* dKT, const float* dVT, void* dq, void* dk,
+                                        void* dv, float* dgate, float* dK0, float* dV0,
+                                        const void* gate_saved, size_t gate_saved_bytes, void* ws,
+                                        size_t ws_bytes, void* stream, int32_t* dev_status);
 
 /*
  * One recurrent step of Eq. 6 for B independent sequences (params->T is

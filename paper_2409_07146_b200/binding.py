@@ -14,7 +14,7 @@ _lib = None
 GSA_F32, GSA_BF16 = 0, 1
 GSA_GATE_A, GSA_GATE_LOG_A, GSA_GATE_LOGITS = 0, 1, 2
 GSA_IMPL_AUTO, GSA_IMPL_SIMT, GSA_IMPL_TC = 0, 1, 2
-GSA_WS_FWD, GSA_WS_BWD, GSA_WS_DECODE = 0, 1, 2
+GSA_WS_FWD, GSA_WS_BWD, GSA_WS_DECODE, GSA_WS_GATE = 0, 1, 2, 3
 
 _IMPL = {"auto": GSA_IMPL_AUTO, "simt": GSA_IMPL_SIMT, "tc": GSA_IMPL_TC}
 _ACT = {"softmax": 0, "none": 1, "relu": 2, "swish": 3, "relu2": 4}   # gsa_act_t
@@ -73,7 +73,7 @@ def lib_path() -> str:
 def exported_symbols():
     return ["gsa_chunk_size", "gsa_workspace_bytes", "gsa_status_string", "gsa_gate_cumsum",
             "gsa_fwd", "gsa_bwd", "gsa_decode_step", "gsa_tc_selftest", "gsa_timing_begin",
-            "gsa_timing_end", "gsa_fwd_noalloc"]
+            "gsa_timing_end", "gsa_fwd_noalloc", "gsa_fwd_save_gate", "gsa_bwd_saved_gate"]
 
 
 def load_library():
@@ -100,6 +100,10 @@ def load_library():
     lib.gsa_fwd.restype = ctypes.c_int
     lib.gsa_bwd.argtypes = [pp] + [vp] * 16 + [vp, sz, vp, vp]
     lib.gsa_bwd.restype = ctypes.c_int
+    lib.gsa_fwd_save_gate.argtypes = [pp] + [vp] * 10 + [vp, sz, vp, sz, vp, vp]
+    lib.gsa_fwd_save_gate.restype = ctypes.c_int
+    lib.gsa_bwd_saved_gate.argtypes = [pp] + [vp] * 16 + [vp, sz, vp, sz, vp, vp]
+    lib.gsa_bwd_saved_gate.restype = ctypes.c_int
     lib.gsa_decode_step.argtypes = [pp] + [vp] * 8
     lib.gsa_decode_step.restype = ctypes.c_int
     lib.gsa_fwd_noalloc.argtypes = [pp] + [vp] * 10 + [vp, vp]
@@ -162,10 +166,16 @@ def gsa_gate_cumsum(p: Params, gate, G, I):
         _ptr(I, torch.float32, shp, "I"), _stream()), "gsa_gate_cumsum")
 
 
+def gate_block(p: Params, device):
+    """A device block of gsa_workspace_bytes(p, GSA_WS_GATE) bytes for gsa_fwd(gate_save=...) and
+    gsa_bwd(gate_saved=...)."""
+    return torch.empty(gsa_workspace_bytes(p, GSA_WS_GATE), dtype=torch.uint8, device=device)
+
+
 def gsa_fwd(p: Params, q, k, v, gate, K0=None, V0=None, o=None, ok_save=None, KT=None, VT=None,
-            ws=None, dev_status=None):
+            ws=None, dev_status=None, gate_save=None):
     """Enqueue the forward on the current stream.  `o` (and `ws`) are allocated with torch when
-    not given.  Returns o."""
+    not given.  With gate_save (see gate_block) the call is gsa_fwd_save_gate.  Returns o."""
     io = p.io_dtype
     qk, vv, mm = (p.B, p.T, p.H, p.d_k), (p.B, p.T, p.H, p.d_v), (p.B, p.T, p.H, p.m)
     sk, sv = (p.B, p.H, p.m, p.d_k), (p.B, p.H, p.m, p.d_v)
@@ -173,19 +183,26 @@ def gsa_fwd(p: Params, q, k, v, gate, K0=None, V0=None, o=None, ok_save=None, KT
         o = torch.empty(vv, dtype=io, device=q.device)
     ws, ws_bytes = _workspace(p, GSA_WS_FWD, ws, q.device)
     cp = p.c()
-    _check(load_library().gsa_fwd(
-        ctypes.byref(cp), _ptr(q, io, qk, "q"), _ptr(k, io, qk, "k"), _ptr(v, io, vv, "v"),
-        _ptr(gate, torch.float32, mm, "gate"), _ptr(K0, torch.float32, sk, "K0"),
-        _ptr(V0, torch.float32, sv, "V0"), _ptr(o, io, vv, "o"),
-        _ptr(ok_save, torch.float32, mm, "ok_save"), _ptr(KT, torch.float32, sk, "KT"),
-        _ptr(VT, torch.float32, sv, "VT"), _ptr(ws, None, None, "ws"), ws_bytes, _stream(),
-        _ptr(dev_status, torch.int32, None, "dev_status")), "gsa_fwd")
+    head = (ctypes.byref(cp), _ptr(q, io, qk, "q"), _ptr(k, io, qk, "k"), _ptr(v, io, vv, "v"),
+            _ptr(gate, torch.float32, mm, "gate"), _ptr(K0, torch.float32, sk, "K0"),
+            _ptr(V0, torch.float32, sv, "V0"), _ptr(o, io, vv, "o"),
+            _ptr(ok_save, torch.float32, mm, "ok_save"), _ptr(KT, torch.float32, sk, "KT"),
+            _ptr(VT, torch.float32, sv, "VT"))
+    tail = (_ptr(ws, None, None, "ws"), ws_bytes, _stream(), _ptr(dev_status, torch.int32, None, "dev_status"))
+    if gate_save is None:
+        _check(load_library().gsa_fwd(*head, *tail), "gsa_fwd")
+    else:
+        _check(load_library().gsa_fwd_save_gate(*head, _ptr(gate_save, None, None, "gate_save"),
+                                                gate_save.numel() * gate_save.element_size(), *tail),
+               "gsa_fwd_save_gate")
     return o
 
 
 def gsa_bwd(p: Params, q, k, v, gate, dO, K0=None, V0=None, ok_saved=None, dKT=None, dVT=None,
-            dq=None, dk=None, dv=None, dgate=None, dK0=None, dV0=None, ws=None, dev_status=None):
-    """Enqueue the backward on the current stream.  Returns (dq, dk, dv, dgate)."""
+            dq=None, dk=None, dv=None, dgate=None, dK0=None, dV0=None, ws=None, dev_status=None,
+            gate_saved=None):
+    """Enqueue the backward on the current stream.  With gate_saved (the block a forward with the
+    same params and gate filled) the call is gsa_bwd_saved_gate.  Returns (dq, dk, dv, dgate)."""
     io = p.io_dtype
     qk, vv, mm = (p.B, p.T, p.H, p.d_k), (p.B, p.T, p.H, p.d_v), (p.B, p.T, p.H, p.m)
     sk, sv = (p.B, p.H, p.m, p.d_k), (p.B, p.H, p.m, p.d_v)
@@ -196,16 +213,20 @@ def gsa_bwd(p: Params, q, k, v, gate, dO, K0=None, V0=None, ok_saved=None, dKT=N
     dgate = torch.empty(mm, dtype=torch.float32, device=dev) if dgate is None else dgate
     ws, ws_bytes = _workspace(p, GSA_WS_BWD, ws, dev)
     cp = p.c()
-    _check(load_library().gsa_bwd(
-        ctypes.byref(cp), _ptr(q, io, qk, "q"), _ptr(k, io, qk, "k"), _ptr(v, io, vv, "v"),
-        _ptr(gate, torch.float32, mm, "gate"), _ptr(K0, torch.float32, sk, "K0"),
-        _ptr(V0, torch.float32, sv, "V0"), _ptr(ok_saved, torch.float32, mm, "ok_saved"),
-        _ptr(dO, io, vv, "dO"), _ptr(dKT, torch.float32, sk, "dKT"),
-        _ptr(dVT, torch.float32, sv, "dVT"), _ptr(dq, io, qk, "dq"), _ptr(dk, io, qk, "dk"),
-        _ptr(dv, io, vv, "dv"), _ptr(dgate, torch.float32, mm, "dgate"),
-        _ptr(dK0, torch.float32, sk, "dK0"), _ptr(dV0, torch.float32, sv, "dV0"),
-        _ptr(ws, None, None, "ws"), ws_bytes, _stream(),
-        _ptr(dev_status, torch.int32, None, "dev_status")), "gsa_bwd")
+    head = (ctypes.byref(cp), _ptr(q, io, qk, "q"), _ptr(k, io, qk, "k"), _ptr(v, io, vv, "v"),
+            _ptr(gate, torch.float32, mm, "gate"), _ptr(K0, torch.float32, sk, "K0"),
+            _ptr(V0, torch.float32, sv, "V0"), _ptr(ok_saved, torch.float32, mm, "ok_saved"),
+            _ptr(dO, io, vv, "dO"), _ptr(dKT, torch.float32, sk, "dKT"),
+            _ptr(dVT, torch.float32, sv, "dVT"), _ptr(dq, io, qk, "dq"), _ptr(dk, io, qk, "dk"),
+            _ptr(dv, io, vv, "dv"), _ptr(dgate, torch.float32, mm, "dgate"),
+            _ptr(dK0, torch.float32, sk, "dK0"), _ptr(dV0, torch.float32, sv, "dV0"))
+    tail = (_ptr(ws, None, None, "ws"), ws_bytes, _stream(), _ptr(dev_status, torch.int32, None, "dev_status"))
+    if gate_saved is None:
+        _check(load_library().gsa_bwd(*head, *tail), "gsa_bwd")
+    else:
+        _check(load_library().gsa_bwd_saved_gate(*head, _ptr(gate_saved, None, None, "gate_saved"),
+                                                 gate_saved.numel() * gate_saved.element_size(), *tail),
+               "gsa_bwd_saved_gate")
     return dq, dk, dv, dgate
 
 

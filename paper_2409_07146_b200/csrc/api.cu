@@ -129,6 +129,29 @@ Workspace carve(const gsa_params_t& p, int which, void* ws) {
     return w;
 }
 
+// The gate kernel's products as a block of their own (GSA_WS_GATE): what the forward can leave for
+// the backward of the same call so that the backward does not run the gate kernel again.
+struct GateSums { int* strong; float *G, *I; void* Id; size_t bytes; };
+GateSums carve_gate(const gsa_params_t& p, void* base) {
+    GateSums g;
+    const size_t mt = (size_t)p.B * p.T * p.H * p.m;
+    Carver c{static_cast<char*>(base), 0};
+    g.strong = reinterpret_cast<int*>(c.take((size_t)p.B * p.H * segments_of(p)));
+    g.G = c.take(mt);
+    g.I = c.take(mt);
+    g.Id = use_tc(p) ? c.take(mt) : nullptr;
+    g.bytes = c.off;
+    return g;
+}
+// points the workspace's gate products at the block; false if the block is missing or too small
+bool use_gate_block(const gsa_params_t& p, Workspace* w, void* block, size_t block_bytes) {
+    if (block == nullptr || (reinterpret_cast<uintptr_t>(block) & 255u) != 0) return false;
+    const GateSums g = carve_gate(p, block);
+    if (block_bytes < g.bytes) return false;
+    w->strong = g.strong; w->G = g.G; w->I = g.I; w->Id = g.Id;
+    return true;
+}
+
 cudaError_t value_side(const gsa_params_t& p, const ValueSideArgs& a, int reverse, const int* strong,
                        cudaStream_t st, int32_t* dev_status) {
     if (use_tc(p)) {
@@ -235,8 +258,9 @@ const char* gsa_status_string(gsa_status_t status) {
 
 size_t gsa_workspace_bytes(const gsa_params_t* params, int32_t which) {
     if (which == GSA_WS_DECODE) return 0;
-    if (which != GSA_WS_FWD && which != GSA_WS_BWD) return 0;
+    if (which != GSA_WS_FWD && which != GSA_WS_BWD && which != GSA_WS_GATE) return 0;
     if (check_params(params, true) != GSA_OK) return 0;
+    if (which == GSA_WS_GATE) return carve_gate(*params, nullptr).bytes;
     return carve(*params, which, nullptr).bytes;
 }
 
@@ -252,10 +276,11 @@ gsa_status_t gsa_gate_cumsum(const gsa_params_t* params, const float* gate, floa
     return GSA_OK;
 }
 
-gsa_status_t gsa_fwd(const gsa_params_t* params, const void* q, const void* k, const void* v,
-                     const float* gate, const float* K0, const float* V0, void* o,
-                     float* ok_save, float* KT, float* VT, void* ws, size_t ws_bytes,
-                     void* stream, int32_t* dev_status) {
+namespace {
+gsa_status_t fwd_impl(const gsa_params_t* params, const void* q, const void* k, const void* v,
+                      const float* gate, const float* K0, const float* V0, void* o,
+                      float* ok_save, float* KT, float* VT, bool save_gate, void* gate_save, size_t gate_save_bytes,
+                      void* ws, size_t ws_bytes, void* stream, int32_t* dev_status) {
     gsa_status_t rc = check_params(params, true);
     if (rc != GSA_OK) return rc;
     if (!ok_ptr(q) || !ok_ptr(k) || !ok_ptr(v) || !ok_ptr(gate) || !ok_ptr(o)) return GSA_ERR_INVALID_ARG;
@@ -263,8 +288,10 @@ gsa_status_t gsa_fwd(const gsa_params_t* params, const void* q, const void* k, c
         return GSA_ERR_INVALID_ARG;
     const gsa_params_t& p = *params;
     if (ws == nullptr || (reinterpret_cast<uintptr_t>(ws) & 255u) != 0) return GSA_ERR_WORKSPACE;
-    const Workspace w = carve(p, GSA_WS_FWD, ws);
+    Workspace w = carve(p, GSA_WS_FWD, ws);
     if (ws_bytes < w.bytes) return GSA_ERR_WORKSPACE;
+    // the gate kernel's products go to the caller's block when the backward is to reuse them
+    if (save_gate && !use_gate_block(p, &w, gate_save, gate_save_bytes)) return GSA_ERR_WORKSPACE;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const Slices s = slices(p);
 
@@ -306,12 +333,30 @@ gsa_status_t gsa_fwd(const gsa_params_t* params, const void* q, const void* k, c
     GSA_LAUNCH("pass2_key_side", key_side(p, a2, 0, w.strong, st, dev_status));
     return GSA_OK;
 }
+}  // namespace
 
-gsa_status_t gsa_bwd(const gsa_params_t* params, const void* q, const void* k, const void* v,
-                     const float* gate, const float* K0, const float* V0, const float* ok_saved,
-                     const void* dO, const float* dKT, const float* dVT, void* dq, void* dk,
-                     void* dv, float* dgate, float* dK0, float* dV0, void* ws, size_t ws_bytes,
+gsa_status_t gsa_fwd(const gsa_params_t* params, const void* q, const void* k, const void* v,
+                     const float* gate, const float* K0, const float* V0, void* o,
+                     float* ok_save, float* KT, float* VT, void* ws, size_t ws_bytes,
                      void* stream, int32_t* dev_status) {
+    return fwd_impl(params, q, k, v, gate, K0, V0, o, ok_save, KT, VT, false, nullptr, 0, ws, ws_bytes, stream,
+                    dev_status);
+}
+
+gsa_status_t gsa_fwd_save_gate(const gsa_params_t* params, const void* q, const void* k, const void* v,
+                               const float* gate, const float* K0, const float* V0, void* o,
+                               float* ok_save, float* KT, float* VT, void* gate_save, size_t gate_save_bytes,
+                               void* ws, size_t ws_bytes, void* stream, int32_t* dev_status) {
+    return fwd_impl(params, q, k, v, gate, K0, V0, o, ok_save, KT, VT, true, gate_save, gate_save_bytes, ws,
+                    ws_bytes, stream, dev_status);
+}
+
+namespace {
+gsa_status_t bwd_impl(const gsa_params_t* params, const void* q, const void* k, const void* v,
+                      const float* gate, const float* K0, const float* V0, const float* ok_saved,
+                      const void* dO, const float* dKT, const float* dVT, void* dq, void* dk,
+                      void* dv, float* dgate, float* dK0, float* dV0, bool gate_is_saved, const void* gate_saved,
+                      size_t gate_saved_bytes, void* ws, size_t ws_bytes, void* stream, int32_t* dev_status) {
     gsa_status_t rc = check_params(params, true);
     if (rc != GSA_OK) return rc;
     if (!ok_ptr(q) || !ok_ptr(k) || !ok_ptr(v) || !ok_ptr(gate) || !ok_ptr(dO) || !ok_ptr(dq) ||
@@ -322,8 +367,9 @@ gsa_status_t gsa_bwd(const gsa_params_t* params, const void* q, const void* k, c
         return GSA_ERR_INVALID_ARG;
     const gsa_params_t& p = *params;
     if (ws == nullptr || (reinterpret_cast<uintptr_t>(ws) & 255u) != 0) return GSA_ERR_WORKSPACE;
-    const Workspace w = carve(p, GSA_WS_BWD, ws);
+    Workspace w = carve(p, GSA_WS_BWD, ws);
     if (ws_bytes < w.bytes) return GSA_ERR_WORKSPACE;
+    if (gate_is_saved && !use_gate_block(p, &w, const_cast<void*>(gate_saved), gate_saved_bytes)) return GSA_ERR_WORKSPACE;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const Slices s = slices(p);
 
@@ -332,9 +378,11 @@ gsa_status_t gsa_bwd(const gsa_params_t* params, const void* q, const void* k, c
     // segment -- from the left for the forward-direction scans, from the right for the reversed ones.
     const int nseg = segments_of(p);
     const int Bs = p.B * nseg, Ts = p.T / nseg;
-    GSA_CUDA(cudaMemsetAsync(w.strong, 0, sizeof(int) * (size_t)p.B * p.H * nseg, st));
-    GSA_LAUNCH("gate_cumsum", launch_gate_cumsum(gate, p.gate_kind, inv_tau(p), w.G, w.I, p.B, p.T,
-                                                 p.H, p.m, chunk_of(p), w.strong, nseg, w.Id, p.io == GSA_BF16, st));
+    if (!gate_is_saved) {      // (a forward of the same call left the gate kernel's products otherwise)
+        GSA_CUDA(cudaMemsetAsync(w.strong, 0, sizeof(int) * (size_t)p.B * p.H * nseg, st));
+        GSA_LAUNCH("gate_cumsum", launch_gate_cumsum(gate, p.gate_kind, inv_tau(p), w.G, w.I, p.B, p.T,
+                                                     p.H, p.m, chunk_of(p), w.strong, nseg, w.Id, p.io == GSA_BF16, st));
+    }
     const float* ok = ok_saved;
     const PendingDecay pend = use_tc(p) ? PendingDecay{w.G, w.strong, p.T, p.H, nseg} : PendingDecay{nullptr, nullptr, 1, 1, 1};
     const float *Kin = K0, *Vin = V0;        // states entering the forward-direction scans
@@ -417,6 +465,26 @@ gsa_status_t gsa_bwd(const gsa_params_t* params, const void* q, const void* k, c
                               dKT, w.KT, dVT, w.VT, p.d_k, p.d_v, w.chunk_tot, dgate, p.B, p.T,
                               p.H, p.m, pend, st, dev_status));
     return GSA_OK;
+}
+}  // namespace
+
+gsa_status_t gsa_bwd(const gsa_params_t* params, const void* q, const void* k, const void* v,
+                     const float* gate, const float* K0, const float* V0, const float* ok_saved,
+                     const void* dO, const float* dKT, const float* dVT, void* dq, void* dk,
+                     void* dv, float* dgate, float* dK0, float* dV0, void* ws, size_t ws_bytes,
+                     void* stream, int32_t* dev_status) {
+    return bwd_impl(params, q, k, v, gate, K0, V0, ok_saved, dO, dKT, dVT, dq, dk, dv, dgate, dK0, dV0, false,
+                    nullptr, 0, ws, ws_bytes, stream, dev_status);
+}
+
+gsa_status_t gsa_bwd_saved_gate(const gsa_params_t* params, const void* q, const void* k, const void* v,
+                                const float* gate, const float* K0, const float* V0, const float* ok_saved,
+                                const void* dO, const float* dKT, const float* dVT, void* dq, void* dk,
+                                void* dv, float* dgate, float* dK0, float* dV0, const void* gate_saved,
+                                size_t gate_saved_bytes, void* ws, size_t ws_bytes, void* stream,
+                                int32_t* dev_status) {
+    return bwd_impl(params, q, k, v, gate, K0, V0, ok_saved, dO, dKT, dVT, dq, dk, dv, dgate, dK0, dV0, true,
+                    gate_saved, gate_saved_bytes, ws, ws_bytes, stream, dev_status);
 }
 
 gsa_status_t gsa_decode_step(const gsa_params_t* params, const void* q, const void* k,

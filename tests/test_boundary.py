@@ -41,6 +41,8 @@ def test_chunk_and_workspace_queries(lib):
     f, b = gsa.gsa_workspace_bytes(p, binding.GSA_WS_FWD), gsa.gsa_workspace_bytes(p, binding.GSA_WS_BWD)
     assert f > 0 and b > f and f % 256 == 0
     assert gsa.gsa_workspace_bytes(p, binding.GSA_WS_DECODE) == 0
+    g = gsa.gsa_workspace_bytes(p, binding.GSA_WS_GATE)      # flags + G + I (fp32 kernels: no decayed rows)
+    assert g % 256 == 0 and 2 * 4 * 2 * 100 * 3 * 32 <= g < f
     bad = gsa.Params(B=2, T=100, H=3, d_k=96, d_v=128, m=32)
     assert gsa.gsa_workspace_bytes(bad, binding.GSA_WS_FWD) == 0
 
@@ -84,6 +86,13 @@ def test_validation_happens_before_any_launch(lib):
     assert lib.gsa_decode_step(ctypes.byref(cp), *([None] * 8)) == 1
     assert lib.gsa_bwd(ctypes.byref(cp), *([None] * 16), None, 0, None, None) == 1
     assert lib.gsa_fwd(None, *([None] * 10), None, 0, None, None) == 1
+    # the saved-gate pair: validated like the plain calls; a missing or short block is a workspace error
+    assert lib.gsa_fwd_save_gate(ctypes.byref(cp), *([None] * 10), None, 0, None, 0, None, None) == 1
+    assert lib.gsa_bwd_saved_gate(ctypes.byref(cp), *([None] * 16), None, 0, None, 0, None, None) == 1
+    okp = [ctypes.c_void_p(x) for x in ok]
+    assert lib.gsa_fwd_save_gate(ctypes.byref(cp), *okp, None, 0, ctypes.c_void_p(0x1000), 1 << 40, None, None) == 3
+    assert lib.gsa_fwd_save_gate(ctypes.byref(cp), *okp, ctypes.c_void_p(0x1000), 16, ctypes.c_void_p(0x1000), 1 << 40,
+                                 None, None) == 3
 
 
 def test_binding_refuses_cpu_tensors(lib):

@@ -465,3 +465,31 @@ def test_tc_single_operand_mode_is_bf16_accurate_and_paired_is_tighter():
     assert all(e <= 1e-3 for e in errs["paired"].values()), errs
     assert all(e <= 1e-1 for e in errs["single"].values()), errs
     assert errs["single"]["ok"] > 10 * errs["paired"]["ok"] and errs["single"]["dq"] > 10 * errs["paired"]["dq"], errs
+
+
+@pytest.mark.parametrize("io,impl,T,H", [("bf16", "tc", 300, 2), ("f32", "auto", 150, 2), ("bf16", "tc", 4096, 1)])
+def test_bwd_with_the_forwards_saved_gate_block_is_the_same_backward(io, impl, T, H):
+    """gsa_fwd_save_gate + gsa_bwd_saved_gate (the backward skips its gate kernel) against the plain
+    pair of calls: the same kernels on the same numbers, so the results are equal bit for bit."""
+    B, dk, dv, m = 1, 128, 128, 64
+    d = rand_inputs(901, B, T, H, dk, dv, m, io, init=True, final_grads=True)
+    p = gsa.Params(B, T, H, dk, dv, m, io=io, impl=impl, scale=0.8)
+    q, k, v, dO = (to_dev(d[n], io) for n in ("q", "k", "v", "dO"))
+    gate, K0, V0, dKT, dVT = (to_dev(d[n]) for n in ("gate", "K0", "V0", "dKT", "dVT"))
+    outs = []
+    for saved in (False, True):
+        blk = gsa.gate_block(p, q.device) if saved else None
+        if saved:
+            blk.fill_(0xFF)          # nothing is read from the block before the forward has written it
+        ok = torch.empty(B, T, H, m, device="cuda")
+        o = gsa.gsa_fwd(p, q, k, v, gate, K0, V0, ok_save=ok, gate_save=blk)
+        dK0 = torch.empty(B, H, m, dk, device="cuda"); dV0 = torch.empty(B, H, m, dv, device="cuda")
+        g = gsa.gsa_bwd(p, q, k, v, gate, dO, K0, V0, ok_saved=ok, dKT=dKT, dVT=dVT, dK0=dK0, dV0=dV0,
+                        gate_saved=blk)
+        torch.cuda.synchronize()
+        outs.append([to_np(o)] + [to_np(t) for t in g] + [to_np(dK0), to_np(dV0)])
+    for a, b in zip(*outs):
+        assert np.array_equal(a, b)
+    ref = oracle.bwd(d["q"], d["k"], d["v"], d["gate"], d["dO"], K0=d["K0"], V0=d["V0"], dKT=d["dKT"],
+                     dVT=d["dVT"], scale=0.8)
+    assert rel_err(outs[1][4], ref["dgate"]) <= TOL[io]
