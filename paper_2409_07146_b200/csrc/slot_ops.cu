@@ -577,29 +577,31 @@ __global__ void __launch_bounds__(256) gate_grad_local_tma_kernel(
     if (hh == 0 && n < nblk) blk_tot[((size_t)bh * nblk + n) * M + tx] = run;
 }
 
-// Adds what follows the block: dgate += carry (log gate) or carry / a (linear gate).
+// Adds what follows the block: dgate += carry (log gate) or carry / a (linear gate).  A thread
+// takes two slots of eight rows (half a block): threadIdx = (slot pair, block, half).
 template <int M>
-__global__ void __launch_bounds__(128) gate_grad_carry_kernel(
+__global__ void __launch_bounds__(256) gate_grad_carry_kernel(
     const float* __restrict__ gate, int gate_kind, float inv_tau, const float* __restrict__ blk_carry,
     float* __restrict__ dgate, int T, int H, int nblk) {
+    constexpr int kRows = kGG / 2;
     const int s = 2 * threadIdx.x;
     const int n = blockIdx.y * blockDim.y + threadIdx.y;
     if (n >= nblk) return;
     const int bh = blockIdx.x, b = bh / H, h = bh % H;
-    const int t0 = n * kGG;
-    const int rows = min(kGG, T - t0);
+    const int t0 = n * kGG + threadIdx.z * kRows;
+    const int rows = max(0, min(kRows, T - t0));
     const size_t stride = (size_t)H * M;
     const size_t base = (((size_t)b * T + t0) * H + h) * M + s;
     const float2 carry = *reinterpret_cast<const float2*>(blk_carry + ((size_t)bh * nblk + n) * M + s);
-    float2 d[kGG], gt[kGG];
+    float2 d[kRows], gt[kRows];
 #pragma unroll
-    for (int i = 0; i < kGG; ++i) {
+    for (int i = 0; i < kRows; ++i) {
         d[i] = (i < rows) ? *reinterpret_cast<const float2*>(dgate + base + (size_t)i * stride) : make_float2(0.f, 0.f);
         gt[i] = (i < rows && gate_kind != GSA_GATE_LOG_A) ? *reinterpret_cast<const float2*>(gate + base + (size_t)i * stride)
                                                           : make_float2(1.f, 1.f);
     }
 #pragma unroll
-    for (int i = 0; i < kGG; ++i)
+    for (int i = 0; i < kRows; ++i)
         if (i < rows) {
             float2 out;
             out.x = d[i].x + gate_grad_carry(carry.x, gt[i].x, gate_kind, inv_tau);
@@ -647,12 +649,12 @@ cudaError_t launch_gate_grad(const float* u, const float* I, const float* dIk_pa
                                                                blk_tot, dgate, B, T, H, nblk, pend);
         }
         gate_grad_scan_kernel<64><<<B * H, dim3(64, 16), 0, st>>>(blk_tot, dKT, KT, dVT, VT, d_k, d_v, nblk);
-        gate_grad_carry_kernel<64><<<grid, block, 0, st>>>(gate, gate_kind, inv_tau, blk_tot, dgate, T, H, nblk);
+        gate_grad_carry_kernel<64><<<grid, dim3(block.x, block.y, 2), 0, st>>>(gate, gate_kind, inv_tau, blk_tot, dgate, T, H, nblk);
     } else {
         gate_grad_local_kernel<32><<<grid, block, 0, st>>>(u, I, dIk_part, nsk, dIv_part, nsv, gate, gate_kind, inv_tau,
                                                            blk_tot, dgate, B, T, H, nblk, pend);
         gate_grad_scan_kernel<32><<<B * H, dim3(32, 16), 0, st>>>(blk_tot, dKT, KT, dVT, VT, d_k, d_v, nblk);
-        gate_grad_carry_kernel<32><<<grid, block, 0, st>>>(gate, gate_kind, inv_tau, blk_tot, dgate, T, H, nblk);
+        gate_grad_carry_kernel<32><<<grid, dim3(block.x, block.y, 2), 0, st>>>(gate, gate_kind, inv_tau, blk_tot, dgate, T, H, nblk);
     }
     return cudaGetLastError();
 }
