@@ -131,15 +131,31 @@ Workspace carve(const gsa_params_t& p, int which, void* ws) {
 
 // The gate kernel's products as a block of their own (GSA_WS_GATE): what the forward can leave for
 // the backward of the same call so that the backward does not run the gate kernel again.
-struct GateSums { int* strong; float *G, *I; void* Id; size_t bytes; };
+// With segment-parallel scheduling the block also carries what the forward's first run found: the
+// segments' decay, the memories entering every segment and the final memories.
+struct GateSums {
+    int* strong; float *G, *I; void* Id;
+    float *seg_decay, *Kstart, *Vstart, *KT, *VT;     // nseg > 1 only
+    size_t bytes;
+};
 GateSums carve_gate(const gsa_params_t& p, void* base) {
     GateSums g;
+    memset(&g, 0, sizeof(g));
     const size_t mt = (size_t)p.B * p.T * p.H * p.m;
+    const int nseg = segments_of(p);
     Carver c{static_cast<char*>(base), 0};
-    g.strong = reinterpret_cast<int*>(c.take((size_t)p.B * p.H * segments_of(p)));
+    g.strong = reinterpret_cast<int*>(c.take((size_t)p.B * p.H * nseg));
     g.G = c.take(mt);
     g.I = c.take(mt);
     g.Id = use_tc(p) ? c.take(mt) : nullptr;
+    if (nseg > 1) {
+        const size_t pairs = (size_t)p.B * nseg * p.H;
+        g.seg_decay = c.take(pairs * p.m);
+        g.Kstart = c.take(pairs * p.m * p.d_k);
+        g.Vstart = c.take(pairs * p.m * p.d_v);
+        g.KT = c.take((size_t)p.B * p.H * p.m * p.d_k);
+        g.VT = c.take((size_t)p.B * p.H * p.m * p.d_v);
+    }
     g.bytes = c.off;
     return g;
 }
@@ -149,6 +165,10 @@ bool use_gate_block(const gsa_params_t& p, Workspace* w, void* block, size_t blo
     const GateSums g = carve_gate(p, block);
     if (block_bytes < g.bytes) return false;
     w->strong = g.strong; w->G = g.G; w->I = g.I; w->Id = g.Id;
+    if (g.seg_decay != nullptr) {
+        w->seg_decay = g.seg_decay; w->Kstart = g.Kstart; w->Vstart = g.Vstart;
+        w->KT = g.KT; w->VT = g.VT;      // (the forward's workspace has no KT / VT of its own)
+    }
     return true;
 }
 
@@ -316,10 +336,17 @@ gsa_status_t fwd_impl(const gsa_params_t* params, const void* q, const void* k, 
         GSA_LAUNCH("segment_pass1_states", value_side(p, s1, 0, w.strong, st, dev_status));
         KeySideArgs s2{w.I, w.I, w.G, v, nullptr, w.Vloc, o, Bs, Ts, p.H, p.d_v, w.Id, w.Id, 1};
         GSA_LAUNCH("segment_pass2_states", key_side(p, s2, 0, w.strong, st, dev_status));
-        GSA_LAUNCH("segment_combine", launch_segment_combine(w.seg_decay, w.Kloc, K0, w.Kstart, KT, p.B, p.H, p.m,
+        // (when the backward is to reuse them, the final memories land in the saved block first)
+        float* KTc = save_gate ? w.KT : KT;
+        float* VTc = save_gate ? w.VT : VT;
+        GSA_LAUNCH("segment_combine", launch_segment_combine(w.seg_decay, w.Kloc, K0, w.Kstart, KTc, p.B, p.H, p.m,
                                                              p.d_k, nseg, 0, st));
-        GSA_LAUNCH("segment_combine", launch_segment_combine(w.seg_decay, w.Vloc, V0, w.Vstart, VT, p.B, p.H, p.m,
+        GSA_LAUNCH("segment_combine", launch_segment_combine(w.seg_decay, w.Vloc, V0, w.Vstart, VTc, p.B, p.H, p.m,
                                                              p.d_v, nseg, 0, st));
+        if (save_gate && KT != nullptr)
+            GSA_CUDA(cudaMemcpyAsync(KT, w.KT, sizeof(float) * (size_t)p.B * p.H * p.m * p.d_k, cudaMemcpyDeviceToDevice, st));
+        if (save_gate && VT != nullptr)
+            GSA_CUDA(cudaMemcpyAsync(VT, w.VT, sizeof(float) * (size_t)p.B * p.H * p.m * p.d_v, cudaMemcpyDeviceToDevice, st));
         Kin = w.Kstart; Vin = w.Vstart;
         Kout = nullptr; Vout = nullptr;
     }
@@ -388,7 +415,12 @@ gsa_status_t bwd_impl(const gsa_params_t* params, const void* q, const void* k, 
     const float *Kin = K0, *Vin = V0;        // states entering the forward-direction scans
     float* KTout = dKT ? w.KT : nullptr;     // final memories, for the gate gradient's final-memory term
     float* VTout = dVT ? w.VT : nullptr;
-    if (nseg > 1) {
+    if (nseg > 1 && gate_is_saved) {
+        // the forward of the same call left the segments' decay, the memories entering every
+        // segment and the final memories in the block
+        Kin = w.Kstart; Vin = w.Vstart;
+        KTout = nullptr; VTout = nullptr;
+    } else if (nseg > 1) {
         GSA_LAUNCH("segment_logdecay", launch_segment_logdecay(w.G, w.seg_decay, p.B, p.T, p.H, p.m, nseg,
                                                                chunk_of(p), st));
         ValueSideArgs s1{q, k, w.I, w.G, nullptr, w.Kloc, w.okpart, Bs, Ts, p.H, p.d_k, w.Id, 1};
