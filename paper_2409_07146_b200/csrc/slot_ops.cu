@@ -577,6 +577,146 @@ __global__ void __launch_bounds__(256) gate_grad_local_tma_kernel(
     if (hh == 0 && n < nblk) blk_tot[((size_t)bh * nblk + n) * M + tx] = run;
 }
 
+// The TMA-staged pass as a ring, for wide heads (n_k + n_v >= 6: a CTA per tile then keeps
+// only two tiles per SM in flight and the copies pause while it computes, leaves and the next
+// one starts).  A tile is 32 rows of one (b,h) with every input stream (u, I, gate, G and the n_k + n_v slices of the
+// input-gate gradient: 12 x 8 KB at d = 512).  One persistent CTA per SM walks the tiles
+// blockIdx.x, blockIdx.x + gridDim.x, ... through a ring of 2-4 stages: a ninth warp requests the
+// tiles of the stages ahead while the eight compute warps work on the current one, so copies
+// are in flight all the time.  Compute thread = (slot, 16-row group, early or late half of it).
+constexpr int kGGMaxStages = 4;
+constexpr int kGGRingMinSlices = 6;
+constexpr int kGGComputeThreads = 256;
+
+__global__ void __launch_bounds__(kGGComputeThreads + 32) gate_grad_local_ring_kernel(
+    const __grid_constant__ CUtensorMap mapU, const __grid_constant__ CUtensorMap mapI,
+    const __grid_constant__ CUtensorMap mapGate, const __grid_constant__ CUtensorMap mapG,
+    const __grid_constant__ CUtensorMap mapDIk, const __grid_constant__ CUtensorMap mapDIv, int nsk, int nsv,
+    int gate_kind, float inv_tau, float* __restrict__ blk_tot, float* __restrict__ dgate, int T, int H, int BH,
+    int ntile, int nstage, int nblk, const int* __restrict__ strong, int nseg, int32_t* dev_status) {
+    using namespace tc;
+    constexpr int M = 64;
+    extern __shared__ unsigned char gg_smem_raw[];
+    unsigned char* smem0 = gg_smem_raw + ((1024u - (smem_u32(gg_smem_raw) & 1023u)) & 1023u);
+    __shared__ uint64_t bar_full[kGGMaxStages], bar_empty[kGGMaxStages];
+    __shared__ float late_half[kGGTmaRows / kGG][M];
+    __shared__ volatile int failed_s, stop_s;
+    const int nslices = nsk + nsv;
+    const int stage_bytes = (4 + nslices) * kGGTileB;
+    const int total = BH * ntile;
+    if (threadIdx.x == 0) {
+        failed_s = 0;
+        for (int s = 0; s < nstage; ++s) {
+            mbar_init(&bar_full[s], 1);
+            mbar_init(&bar_empty[s], 1);
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+
+    if (threadIdx.x == kGGComputeThreads) {
+        // =============================== copy lane
+        // tiles 0..3 = u, I, gate, G; I is not read when the gate tensor holds a itself (1 - a is one
+        // subtraction), G only when a row factor is pending
+        const bool need[4] = {true, gate_kind != GSA_GATE_A, true, strong != nullptr};
+        int ntiles = nslices;
+        for (int i = 0; i < 4; ++i) ntiles += need[i] ? 1 : 0;
+        const CUtensorMap* maps[4] = {&mapU, &mapI, &mapGate, &mapG};
+        int it = 0;
+        for (int t = blockIdx.x; t < total; t += gridDim.x, ++it) {
+            const int s = it % nstage;
+            if (it >= nstage && !mbar_wait(&bar_empty[s], ((it / nstage) - 1) & 1)) {
+                failed_s = 1;
+                break;
+            }
+            const int bh = t % BH, b = bh / H, h = bh % H, t0 = (t / BH) * kGGTmaRows;
+            unsigned char* smem = smem0 + (size_t)s * stage_bytes;
+            mbar_expect_tx(&bar_full[s], (uint32_t)(ntiles * kGGTileB));
+            for (int i = 0; i < 4; ++i) {
+                if (!need[i]) continue;
+                tma_load_4d(smem + i * kGGTileB, maps[i], &bar_full[s], 0, h, t0, b);
+                tma_load_4d(smem + i * kGGTileB + kGGTileB / 2, maps[i], &bar_full[s], 32, h, t0, b);
+            }
+            for (int sl = 0; sl < nslices; ++sl) {
+                const CUtensorMap* m = sl < nsk ? &mapDIk : &mapDIv;
+                const int z = sl < nsk ? sl : sl - nsk;
+                tma_load_5d(smem + (4 + sl) * kGGTileB, m, &bar_full[s], 0, h, t0, b, z);
+                tma_load_5d(smem + (4 + sl) * kGGTileB + kGGTileB / 2, m, &bar_full[s], 32, h, t0, b, z);
+            }
+        }
+    } else if (threadIdx.x < kGGComputeThreads) {
+        // =============================== compute warps
+        // slot, 16-row group, early (0) or late (1) 8 rows of the group
+        const int tx = threadIdx.x & 63, ty = (threadIdx.x >> 6) & 1, hh = threadIdx.x >> 7;
+        constexpr int kHalf = kGG / 2;
+        const size_t stride = (size_t)H * M;
+        auto csync = [] { asm volatile("bar.sync 1, 256;" ::: "memory"); };
+        int it = 0;
+        for (int t = blockIdx.x; t < total; t += gridDim.x, ++it) {
+            const int s = it % nstage;
+            const int bh = t % BH, b = bh / H, h = bh % H, ty0 = t / BH, t0 = ty0 * kGGTmaRows;
+            const unsigned char* smem = smem0 + (size_t)s * stage_bytes;
+            const bool landed = mbar_wait(&bar_full[s], (it / nstage) & 1);
+            if (!landed) failed_s = 1;
+            const int n = ty0 * (kGGTmaRows / kGG) + ty;           // 16-row block of the sequence
+            const int rows = n < nblk ? min(kGG, T - n * kGG) : 0;
+            // row r (of this thread's 8), this thread's slot, of tile `tile`
+            auto at = [&](int tile, int r) {
+                const int row = ty * kGG + hh * kHalf + r, c = tx;
+                const unsigned char* p = smem + tile * kGGTileB + (c >> 5) * (kGGTileB / 2) + swz128(row, (c & 31) >> 2) + (c & 3) * 4;
+                return *reinterpret_cast<const float*>(p);
+            };
+            float x[kHalf], dI[kHalf], gt[kHalf];
+#pragma unroll
+            for (int i = 0; i < kHalf; ++i) { dI[i] = 0.f; x[i] = 0.f; gt[i] = 1.f; }
+            if (landed) {
+                for (int sl = 0; sl < nslices; ++sl) {
+#pragma unroll
+                    for (int i = 0; i < kHalf; ++i) dI[i] += at(4 + sl, i);
+                }
+                if (strong != nullptr && strong[(b * nseg + t0 / (T / nseg)) * H + h] == 0) {
+                    // the time-reversed value_side runs left their row factor exp(-G_i) to this kernel
+#pragma unroll
+                    for (int i = 0; i < kHalf; ++i) dI[i] *= __expf(-at(3, i));
+                }
+#pragma unroll
+                for (int i = 0; i < kHalf; ++i) {
+                    gt[i] = at(2, i);
+                    const float ii = gate_kind == GSA_GATE_A ? 1.f - gt[i] : at(1, i);      // 1 - a as the gate kernel formed it
+                    x[i] = at(0, i) - ii * dI[i];                                          // rows past the end: u = dI = 0
+                }
+            }
+            // the early half starts from the total of the late half of its group
+            float tot = 0.f;
+#pragma unroll
+            for (int i = 0; i < kHalf; ++i) tot += x[i];
+            if (hh == 1) late_half[ty][tx] = tot;
+            csync();                              // (also: every thread has read its part of the stage)
+            if (threadIdx.x == 0)
+                asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&bar_empty[s])) : "memory");
+            float run = hh == 0 ? late_half[ty][tx] : 0.f;
+            const size_t base = (((size_t)b * T + n * kGG + hh * kHalf) * H + h) * M + tx;
+#pragma unroll
+            for (int i = kHalf - 1; i >= 0; --i) {
+                run += x[i];
+                if (hh * kHalf + i < rows)
+                    dgate[base + (size_t)i * stride] = gate_grad_out(run, dI[i], gt[i], gate_kind, inv_tau);
+            }
+            if (hh == 0 && n < nblk) blk_tot[((size_t)bh * nblk + n) * M + tx] = run;
+            // (one thread reads the flag that the copy lane may raise at any time, so that all leave together)
+            if (threadIdx.x == 0) stop_s = failed_s;
+            csync();                              // late_half may be rewritten
+            if (stop_s) break;
+        }
+    }
+    __syncthreads();
+    if (failed_s) {
+        if (threadIdx.x == 0 && dev_status != nullptr) *dev_status = GSA_ERR_TIMEOUT;
+        // bounded grace period for tile copies still in flight before shared memory goes away
+        for (int i = 0; i < 200; ++i) __nanosleep(1000);
+    }
+}
+
 // Adds what follows the block: dgate += carry (log gate) or carry / a (linear gate).  A thread
 // takes two slots of eight rows (half a block): threadIdx = (slot pair, block, half).
 template <int M>
@@ -635,7 +775,27 @@ cudaError_t launch_gate_grad(const float* u, const float* I, const float* dIk_pa
             if (e == cudaSuccess) e = make_tensor_map_sliced(&mv, dIv_part, nsv, B, T, H, M, kGGTmaRows, 4);
             staged = e == cudaSuccess;
         }
-        if (staged) {
+        if (staged && nsl >= kGGRingMinSlices) {
+            const int stage_bytes = (4 + nsl) * kGGTileB;
+            const int nstage = 2;
+            const size_t smem = 1024 + (size_t)nstage * stage_bytes;
+            cudaError_t e = cudaFuncSetAttribute(gate_grad_local_ring_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                 (int)smem);
+            if (e != cudaSuccess) return e;
+            static int sm_count = 0;
+            if (sm_count == 0) {
+                int dev = 0;
+                if (cudaGetDevice(&dev) != cudaSuccess ||
+                    cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sm_count <= 0)
+                    return cudaErrorUnknown;
+            }
+            const int BH = B * H, ntile = (T + kGGTmaRows - 1) / kGGTmaRows;
+            const long long total = (long long)BH * ntile;
+            const int ctas = (int)(total < sm_count ? total : sm_count);      // one persistent CTA per SM
+            gate_grad_local_ring_kernel<<<ctas, kGGComputeThreads + 32, smem, st>>>(
+                mu, mi, mg, mG, mk, mv, nsk, nsv, gate_kind, inv_tau, blk_tot, dgate, T, H, BH, ntile, nstage, nblk,
+                pend.G != nullptr ? pend.strong : nullptr, pend.nseg, dev_status);
+        } else if (staged) {
             const size_t smem = 1024 + (size_t)(4 + nsl) * kGGTileB;
             cudaError_t e = cudaFuncSetAttribute(gate_grad_local_tma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                  (int)smem);
