@@ -43,7 +43,7 @@ NCU_TRAFFIC = {
     "pass2_key_side": 129739520, "bwd_dq_key_side": 135778048,
     "bwd_dv_key_side_rev": 130483200, "bwd_dk_key_side_rev": 132975616,
     "gate_cumsum": 17926144, "slot_softmax": 92744448, "slot_softmax_bwd": 118787072,
-    "gate_grad": 233491456,     # local + scan + carry
+    "gate_grad": 231503872,     # local + scan + carry
 }
 
 
