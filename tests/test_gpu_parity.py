@@ -286,10 +286,12 @@ def test_bwd_tc_segment_parallel_schedule(strong_segment, saved):
     print("segment-parallel bwd", strong_segment, saved, errs)
 
 
-def test_step_is_graph_capturable_and_replays_bitwise():
+@pytest.mark.parametrize("saved_gate,T,H", [(False, 384, 2), (True, 384, 2), (True, 4096, 1)])
+def test_step_is_graph_capturable_and_replays_bitwise(saved_gate, T, H):
     # fwd + bwd enqueue on the caller's stream and on the library's side streams with event
-    # fork / join only: a CUDA graph capture of one step must replay to the same bits
-    B, T, H, dk, dv, m = 2, 384, 2, 256, 128, 64
+    # fork / join only: a CUDA graph capture of one step must replay to the same bits (also
+    # the step that hands the gate kernel's products over, and with segment-parallel scheduling)
+    B, dk, dv, m = 2 if H == 2 else 1, 256, 128, 64
     d = rand_inputs(77, B, T, H, dk, dv, m, "bf16")
     p = gsa.Params(B, T, H, dk, dv, m, io="bf16")
     q, k, v, dO = (to_dev(d[n], "bf16") for n in ("q", "k", "v", "dO"))
@@ -300,10 +302,12 @@ def test_step_is_graph_capturable_and_replays_bitwise():
     ws_f = torch.empty(gsa.gsa_workspace_bytes(p, 0), dtype=torch.uint8, device="cuda")
     ws_b = torch.empty(gsa.gsa_workspace_bytes(p, 1), dtype=torch.uint8, device="cuda")
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    blk = gsa.gate_block(p, q.device) if saved_gate else None
 
     def step():
-        gsa.gsa_fwd(p, q, k, v, gate, o=o, ok_save=ok, ws=ws_f, dev_status=status)
-        gsa.gsa_bwd(p, q, k, v, gate, dO, ok_saved=ok, dq=dq, dk=dk_, dv=dv_, dgate=dg, ws=ws_b, dev_status=status)
+        gsa.gsa_fwd(p, q, k, v, gate, o=o, ok_save=ok, ws=ws_f, dev_status=status, gate_save=blk)
+        gsa.gsa_bwd(p, q, k, v, gate, dO, ok_saved=ok, dq=dq, dk=dk_, dv=dv_, dgate=dg, ws=ws_b, dev_status=status,
+                    gate_saved=blk)
 
     step()
     torch.cuda.synchronize()
