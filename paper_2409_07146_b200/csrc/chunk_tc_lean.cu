@@ -15,6 +15,8 @@
 //   * tile copies and MMA issue are two lanes of two warps, so that a wait of one (for a store to
 //     drain, for a tile to land) never delays the other.
 // Tile geometry and the bounded waits are those of the general kernels.
+// The file also holds the state-only scan that segment-parallel scheduling uses for the end
+// memories of every segment (state_scan_kernel, below the two chunk kernels).
 #include "chunk_tc_shared.cuh"
 
 namespace gsa {
