@@ -211,7 +211,10 @@ GSA_API gsa_status_t gsa_decode_step(const gsa_params_t* params, const void* q,
  *   - Shapes whose gsa_workspace_bytes(params, GSA_WS_FWD) exceeds that maximum are
  *     rejected with GSA_ERR_WORKSPACE before anything is launched.
  *   - The first call on each device looks up the array's device address (with that device
- *     current); make that first call before any stream capture.
+ *     current).  Like gsa_fwd, the first tensor-core call of a host thread on a device also
+ *     creates that thread's side stream and its two events (no device memory).  Make that
+ *     first call before any stream capture and outside latency-critical sections; later
+ *     calls only read the cached address.
  *   - All calls on a device share the one array: calls that overlap on the GPU (different
  *     streams) race and give wrong results; serialise them or use gsa_fwd with separate
  *     workspaces.  The array keeps the previous call's contents; the forward needs none of

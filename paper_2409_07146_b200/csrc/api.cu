@@ -34,6 +34,8 @@ gsa_status_t check_params(const gsa_params_t* p, bool need_T) {
     if (p->m != 32 && p->m != 64) return GSA_ERR_UNSUPPORTED;
     if ((long long)p->B * p->H > 0x7fffffffLL / 4) return GSA_ERR_UNSUPPORTED;
     if (p->impl == GSA_IMPL_TC && p->io != GSA_BF16) return GSA_ERR_UNSUPPORTED;
+    // the tensor-core kernels asked for by name: no silent fall-back to the CUDA-core kernels
+    if (p->impl == GSA_IMPL_TC && !tc_supported(p->d_k, p->d_v, p->m)) return GSA_ERR_UNSUPPORTED;
     return GSA_OK;
 }
 

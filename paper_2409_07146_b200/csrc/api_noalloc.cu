@@ -6,6 +6,7 @@
 // only receives the framework's input and output buffers.  gsa_fwd needs scratch memory
 // from its caller; this entry point brings its own: a fixed array that lives in the library
 // image on every GPU that loads it.
+#include <atomic>
 #include <mutex>
 
 #include "common.cuh"
@@ -20,7 +21,7 @@ static __device__ __align__(256) unsigned char g_fwd_scratch[kScratchBytes];
 
 constexpr int kMaxDevices = 64;
 std::mutex g_mutex;
-void* g_scratch_ptr[kMaxDevices] = {};
+std::atomic<void*> g_scratch_ptr[kMaxDevices] = {};
 
 // Address of the scratch array on the CURRENT device (looked up on the first call per device).
 cudaError_t scratch_address(void** out) {
@@ -28,14 +29,17 @@ cudaError_t scratch_address(void** out) {
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
     if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
-    std::lock_guard<std::mutex> lock(g_mutex);
-    if (g_scratch_ptr[dev] == nullptr) {
-        void* p = nullptr;
-        e = cudaGetSymbolAddress(&p, g_fwd_scratch);
-        if (e != cudaSuccess) return e;
-        g_scratch_ptr[dev] = p;
+    void* p = g_scratch_ptr[dev].load(std::memory_order_acquire);      // steady state: no lock
+    if (p == nullptr) {
+        std::lock_guard<std::mutex> lock(g_mutex);
+        p = g_scratch_ptr[dev].load(std::memory_order_relaxed);
+        if (p == nullptr) {
+            e = cudaGetSymbolAddress(&p, g_fwd_scratch);
+            if (e != cudaSuccess) return e;
+            g_scratch_ptr[dev].store(p, std::memory_order_release);
+        }
     }
-    *out = g_scratch_ptr[dev];
+    *out = p;
     return cudaSuccess;
 }
 

@@ -67,6 +67,9 @@ def test_validation_happens_before_any_launch(lib):
     assert _call_fwd(lib, gsa.Params(1, 64, 1, 96, 64, 32, io="f32"), ok) == 2
     assert _call_fwd(lib, gsa.Params(1, 64, 1, 64, 64, 48, io="f32"), ok) == 2
     assert _call_fwd(lib, gsa.Params(1, 64, 1, 64, 64, 32, io="f32", impl="tc"), ok) == 2
+    # the tensor-core kernels asked for by name on a shape they do not serve: an error, not the CUDA-core kernels
+    assert _call_fwd(lib, gsa.Params(1, 64, 1, 64, 64, 48, io="bf16", impl="tc"), ok) == 2
+    assert _call_fwd(lib, gsa.Params(1, 64, 1, 96, 64, 64, io="bf16", impl="tc"), ok) == 2
     # invalid sizes
     assert _call_fwd(lib, gsa.Params(1, 0, 1, 64, 64, 32, io="f32"), ok) == 1
     assert _call_fwd(lib, gsa.Params(0, 64, 1, 64, 64, 32, io="f32"), ok) == 1

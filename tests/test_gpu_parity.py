@@ -7,9 +7,16 @@ import torch
 import gsa_workloads as W
 import oracle
 import paper_2409_07146_b200 as gsa
-from util import BF16_IO, TC_RTOL, TOL, mixed_err, rand_inputs, rel_err, to_dev, to_np
+from util import BF16_IO, TOL, bf16_storage_check, rand_inputs, rel_err, to_dev, to_np
 
 pytestmark = pytest.mark.gpu
+
+# A bfloat16-stored result must be the oracle's value rounded to bfloat16 or a neighbour of it
+# (bf16_storage_check).  At the size of the benchmark configurations the largest distance measured
+# is one ulp; the small stress shapes here (initial and final memories with their gradients) reach
+# two.  Not asserted where strong forgetting sends a (batch, head) pair to the general kernels,
+# whose derived operands are single bfloat16 values: those are held to the stated tolerance only.
+STORAGE_ULPS = 2.0
 
 
 def run_fwd(d, B, T, H, dk, dv, m, io, impl="auto", scale=1.0, log=False, want_states=True, act="softmax"):
@@ -26,18 +33,19 @@ def run_fwd(d, B, T, H, dk, dv, m, io, impl="auto", scale=1.0, log=False, want_s
                 VT=None if VT is None else to_np(VT)), gate
 
 
-def check_fwd(d, got, gate, io, scale=1.0, log=False, tol=None, tc=False, act="softmax"):
+def check_fwd(d, got, gate, io, scale=1.0, log=False, tol=None, tc=False, act="softmax", storage=True):
     ref = oracle.fwd(d["q"], d["k"], d["v"], gate, gate_is_log=log, scale=scale,
                      K0=d.get("K0"), V0=d.get("V0"), act=act)
     tol = tol or TOL[io]
-    if tc:      # bf16-stored o after the half-ulp of its format; fp32 tensors after the small-shape allowance
-        errs = {n: (rel_err(got[n], ref[n], True) if n in BF16_IO else mixed_err(got[n], ref[n], TC_RTOL))
-                for n in ("o", "ok", "KT", "VT") if got[n] is not None}
-    else:
-        errs = {n: rel_err(got[n], ref[n], io == "bf16" and n in BF16_IO)
-                for n in ("o", "ok", "KT", "VT") if got[n] is not None}
+    # fp32 tensors (logits, final memories): the plain metric.  Tensors stored as bfloat16: after the
+    # half-ulp of that storage, and within one bfloat16 ulp of the rounded oracle value
+    errs = {n: rel_err(got[n], ref[n], io == "bf16" and n in BF16_IO)
+            for n in ("o", "ok", "KT", "VT") if got[n] is not None}
     assert all(np.isfinite(got[n]).all() for n in errs), "non-finite output"
     assert all(e <= tol for e in errs.values()), errs
+    if io == "bf16" and storage:
+        ulps, equal = bf16_storage_check(got["o"], ref["o"])
+        assert ulps <= STORAGE_ULPS and equal >= 0.95, ("o", ulps, equal)
     return errs
 
 
@@ -93,7 +101,7 @@ def test_fwd_strong_forgetting_and_exact_zero_one_gates(impl, gate, log):
     d = rand_inputs(11, B, T, H, dk, dv, m, io, init=True, gate=gate)
     got, g = run_fwd(d, B, T, H, dk, dv, m, io, impl=impl, log=log)
     gref = np.maximum(g.astype(np.float64), -100.0) if log else g
-    check_fwd(d, got, gref, io, log=log)
+    check_fwd(d, got, gref, io, log=log, storage=False)
 
 
 def test_fwd_tiny_config_fp32():
@@ -152,13 +160,14 @@ def run_bwd(d, B, T, H, dk, dv, m, io, impl="auto", scale=1.0, log=False, saved=
     return got, ref
 
 
-def check_bwd(got, ref, tol, tc=False):
-    if tc:      # (as in check_fwd)
-        errs = {n: (rel_err(got[n], ref[n], True) if n in BF16_IO else mixed_err(got[n], ref[n], TC_RTOL)) for n in got}
-    else:
-        errs = {n: rel_err(got[n], ref[n], tol == TOL["bf16"] and n in BF16_IO) for n in got}
+def check_bwd(got, ref, tol, tc=False, storage=True):
+    bf16 = tc or tol == TOL["bf16"]
+    errs = {n: rel_err(got[n], ref[n], bf16 and n in BF16_IO) for n in got}
     assert all(np.isfinite(got[n]).all() for n in got), "non-finite gradient"
     assert all(e <= tol for e in errs.values()), errs
+    if bf16 and storage:
+        st = {n: bf16_storage_check(got[n], ref[n]) for n in ("dq", "dk", "dv")}
+        assert all(u <= STORAGE_ULPS and eq >= 0.95 for u, eq in st.values()), st
     return errs
 
 
@@ -184,9 +193,11 @@ def test_bwd_strong_forgetting():
     B, T, H, dk, dv, m = 1, 160, 1, 64, 64, 32
     d = rand_inputs(43, B, T, H, dk, dv, m, "f32", init=True, gate="strong")
     got, ref = run_bwd(d, B, T, H, dk, dv, m, "f32", log=True)
-    # cumulative log gates reach -200 here: in fp32 their differences carry an absolute
-    # rounding of ~1e-5, i.e. a relative 1e-5..1e-4 on every decay factor, hence 3e-4
-    check_bwd(got, ref, 3 * TOL["f32"])
+    # cumulative log gates reach -200 inside a chunk here: stored in fp32 they carry an absolute
+    # rounding of 200 * 2^-24 = 1.2e-5, which is a relative error of that size on every decay factor
+    # exp(G_i - G_j).  Measured 1.25e-4 on the gate gradient; the stated 1e-4 is read for gates in
+    # the layer's range (tau = 8: |G| <= 10 per chunk), where the same kernels measure 1e-6.
+    print("bwd strong f32", check_bwd(got, ref, 1.5 * TOL["f32"]))
 
 
 # ------------------------------------------------------------------ decode
@@ -250,7 +261,7 @@ def test_fwd_tc_strong_forgetting(gate, log):
     d = rand_inputs(13, B, T, H, dk, dv, m, "bf16", init=True, gate=gate)
     got, g = run_fwd(d, B, T, H, dk, dv, m, "bf16", impl="tc", log=log)
     gref = np.maximum(g.astype(np.float64), -100.0) if log else g
-    check_fwd(d, got, gref, "bf16", log=log, tc=True)
+    check_fwd(d, got, gref, "bf16", log=log, tc=True, storage=False)
 
 
 @pytest.mark.parametrize("gate", ["tau8", "mixed"])
@@ -264,7 +275,7 @@ def test_fwd_tc_segment_parallel_schedule(gate, init):
         d["gate"][:, :2048, :, 2] = 0.99
         d["gate"][:, 3072:, :, 2] = 0.99
     got, g = run_fwd(d, B, T, H, dk, dv, m, "bf16", impl="tc", scale=0.7)
-    errs = check_fwd(d, got, g, "bf16", scale=0.7, tc=True)
+    errs = check_fwd(d, got, g, "bf16", scale=0.7, tc=True, storage=gate != "mixed")
     print("segment-parallel fwd", errs)
 
 
@@ -282,7 +293,7 @@ def test_bwd_tc_segment_parallel_schedule(strong_segment, saved):
     # (gates of 1e-3 are passed as log a: the gradient w.r.t. a itself is d(log a) / a - dI, and the
     # division amplifies the fp32 noise of the whole-sequence sum by 1 / a)
     got, ref = run_bwd(d, B, T, H, dk, dv, m, "bf16", impl="tc", scale=0.7, saved=saved, log=strong_segment)
-    errs = check_bwd(got, ref, TOL["bf16"], tc=True)
+    errs = check_bwd(got, ref, TOL["bf16"], tc=True, storage=not strong_segment)
     print("segment-parallel bwd", strong_segment, saved, errs)
 
 
@@ -351,7 +362,7 @@ def test_bwd_tc_final_memory_gradients(T):
     B, H, dk, dv, m = 2, 2, 128, 256, 64
     d = rand_inputs(700 + T, B, T, H, dk, dv, m, "bf16", init=True, final_grads=True)
     got, ref = run_bwd(d, B, T, H, dk, dv, m, "bf16", impl="tc", scale=1.1)
-    errs = check_bwd(got, ref, 1.5 * TOL["bf16"], tc=True)
+    errs = check_bwd(got, ref, TOL["bf16"], tc=True)
     print("tc bwd final", T, errs)
 
 
@@ -360,9 +371,11 @@ def test_bwd_tc_strong_forgetting_saved_logits():
     d = rand_inputs(45, B, T, H, dk, dv, m, "bf16", gate="strong")
     got, ref = run_bwd(d, B, T, H, dk, dv, m, "bf16", impl="tc", log=True, saved=True)
     # with a ~ 0.05 the input gate 1 - a is ~ 1 and the three terms of the gate gradient
-    # (p dp + o' do' - (1-a) dI) cancel almost completely: the bf16 roundings of their factors
-    # are what is left, hence the wider bound on this stress case
-    check_bwd(got, ref, 4 * TOL["bf16"], tc=True)
+    # (p dp + o' do' - (1-a) dI) cancel almost completely; the general kernels, which take pairs
+    # with strong-decay chunks, carry their derived operands as single bfloat16 values, and their
+    # roundings are what is left: dq, dk 1.3e-2, gate gradient 4.8e-2 measured.  Held to 3x the
+    # stated bound on this stress case only.
+    print("bwd tc strong saved", check_bwd(got, ref, 3 * TOL["bf16"], tc=True, storage=False))
 
 
 # ------------------------------------------------------------------ gate from logits (Sec. 3.3)
@@ -388,9 +401,7 @@ def test_logit_gate_fwd_bwd(io, impl):
     got = dict(o=to_np(o), ok=to_np(ok), KT=to_np(KT), VT=to_np(VT), dq=to_np(dq), dk=to_np(dk_),
                dv=to_np(dv_), dgate=to_np(dg))
     ref = dict(rf, **rb)
-    tc = impl == "tc"
-    errs = {n: (mixed_err(got[n], ref[n], TC_RTOL) if (tc and n not in BF16_IO) else rel_err(got[n], ref[n], io == "bf16" and n in BF16_IO))
-            for n in got}
+    errs = {n: rel_err(got[n], ref[n], io == "bf16" and n in BF16_IO) for n in got}
     assert all(e <= TOL[io] for e in errs.values()), errs
 
 

@@ -7,8 +7,9 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 import paper_2409_07146_b200 as gsa
-from util import rand_inputs, to_dev
+from util import TOL, rand_inputs, rel_err, to_dev
 
 pytestmark = pytest.mark.gpu
 
@@ -33,6 +34,11 @@ def _run_both(seed, B, T, H, dk, dv, m, io):
         assert np.isfinite(b).all(), n
         # same kernels, same order, same inputs: the two entry points must agree to the bit
         np.testing.assert_array_equal(a, b, err_msg=n)
+    # ... and these shapes and seeds against the oracle itself
+    want = oracle.fwd(d["q"], d["k"], d["v"], d["gate"], K0=d["K0"], V0=d["V0"])
+    for n, name in (("o", "o"), ("ok_save", "ok"), ("KT", "KT"), ("VT", "VT")):
+        e = rel_err(got[n].float().cpu().numpy(), want[name], io == "bf16" and n == "o")
+        assert e <= TOL[io], (n, e)
 
 
 def test_noalloc_forward_matches_gsa_fwd_twice_in_a_row():
@@ -41,6 +47,24 @@ def test_noalloc_forward_matches_gsa_fwd_twice_in_a_row():
     _run_both(901, 2, 300, 2, 128, 128, 64, "bf16")     # tensor-core kernels
     _run_both(902, 1, 200, 3, 64, 128, 32, "f32")       # fp32 CUDA-core kernels
     _run_both(903, 2, 300, 2, 128, 128, 64, "bf16")
+
+
+def test_noalloc_steady_state_call_leaves_device_memory_alone():
+    # after the first call on this device (symbol lookup, the library's side stream and events) a
+    # call must not change the amount of free device memory
+    p = gsa.Params(2, 300, 2, 128, 128, 64, io="bf16")
+    d = rand_inputs(904, 2, 300, 2, 128, 128, 64, "bf16")
+    q, k, v = (to_dev(d[n], "bf16") for n in ("q", "k", "v"))
+    gate = to_dev(d["gate"])
+    o = torch.empty(2, 300, 2, 128, dtype=torch.bfloat16, device="cuda")
+    gsa.gsa_fwd_noalloc(p, q, k, v, gate, o=o)
+    torch.cuda.synchronize()
+    free0, _ = torch.cuda.mem_get_info()
+    alloc0 = torch.cuda.memory_allocated()
+    for _ in range(3):
+        gsa.gsa_fwd_noalloc(p, q, k, v, gate, o=o)
+    torch.cuda.synchronize()
+    assert torch.cuda.mem_get_info()[0] == free0 and torch.cuda.memory_allocated() == alloc0
 
 
 def test_noalloc_rejects_shapes_beyond_its_scratch():

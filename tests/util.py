@@ -25,37 +25,28 @@ def to_np(t):
 
 BF16_IO = {"o", "dq", "dk", "dv"}   # tensors stored in the io type (bf16 when io == "bf16")
 
-# Relative allowance of the tensor-core path in the small-shape tests: the half-ulp of a bfloat16
-# output, 2^-9 |ref| (for the fp32 outputs -- logits, memories, gate gradient -- it stands for the
-# bf16 rounding of the operand that dominates them).
-TC_RTOL = 2.0 ** -9
-# Bounds of the tensor-core path at the size of the benchmark configurations, per tensor:
-# ("plain", 0, x)  = max|err| / rms <= x with no allowance (the stated bound where x = 2e-2);
-# ("bf16out", 0, x) = the same after the half-ulp of the tensor's bfloat16 storage (bf16_half_ulp).
-# Every tensor meets the stated 2e-2; the logits, the final memories and the gate gradient (fp32)
-# by two orders of magnitude (1e-4), o and dv at 1.4-1.8e-2, all of it the rounding of their
-# bfloat16 storage.  dq and dk are stored as bfloat16 and heavy-tailed (max|ref| / rms = 10-11 at
-# train_1p3b, 39 for dq at t2r_7b, where key channels carry outliers): the half-ulp of the
-# output format alone (2^-9 to 2^-8 of |ref|) is then 2.6-6.8e-2 of the rms, so it is taken off
-# first (as for the CUDA-core kernels with bf16 io).  What is left is 1e-4 and less: the
-# arithmetic is as exact as that of the fp32 outputs.  Every operand that the kernels derive on
-# the way to a result -- decayed weights, masked products, decayed q / k rows, the state copies
-# -- is carried as a bf16 high/low pair.
+# Bounds of the tensor-core path at the size of the benchmark configurations, per tensor, on
+# max|err| / rms(ref):  ("plain", x) = no allowance;  ("bf16out", x) = after the half-ulp of the
+# tensor's bfloat16 storage (bf16_half_ulp).  The fp32 outputs (logits, final memories, gate
+# gradient) measure 1e-4, o and dv 1.4-1.8e-2 (the rounding of their bfloat16 storage), all on the
+# plain metric.  dq and dk are stored as bfloat16 and heavy-tailed (max|ref| / rms = 10-11 at
+# train_1p3b, 39 for dq at t2r_7b, where key channels carry outliers): the half-ulp of the output
+# format alone (2^-9 to 2^-8 of |ref|) is then 2.6-6.8e-2 of the rms, above the stated 2e-2 on the
+# plain metric, so these two meet the bound only after that half-ulp is taken off (what is left is
+# 1e-4 and less).  Their plain figures are held under the ceilings of TC_PLAIN_CEILING, and every
+# bfloat16-stored tensor is checked against the oracle's value rounded to bfloat16
+# (bf16_storage_check).
 TC_CONFIG_BOUNDS = {
-    "o": ("plain", 0.0, 2e-2), "ok": ("plain", 0.0, 2e-2), "KT": ("plain", 0.0, 2e-2),
-    "VT": ("plain", 0.0, 2e-2), "dv": ("plain", 0.0, 2e-2), "dq": ("bf16out", 0.0, 2e-2),
-    "dk": ("bf16out", 0.0, 2e-2), "dgate": ("plain", 0.0, 2e-2),
+    "o": ("plain", 2e-2), "ok": ("plain", 2e-2), "KT": ("plain", 2e-2),
+    "VT": ("plain", 2e-2), "dv": ("plain", 2e-2), "dq": ("bf16out", 2e-2),
+    "dk": ("bf16out", 2e-2), "dgate": ("plain", 2e-2),
 }
-
-
-def mixed_err(x, ref, rtol):
-    """max (|x - ref| - rtol |ref|)+ / rms(ref): the rms-normalised error that is left after
-    a relative allowance rtol per element (see TC_RTOL)."""
-    x = np.asarray(x, dtype=np.float64)
-    ref = np.asarray(ref, dtype=np.float64)
-    diff = np.maximum(np.abs(x - ref) - rtol * np.abs(ref), 0.0)
-    rms = np.sqrt(np.mean(ref ** 2))
-    return float(diff.max() / (rms if rms > 0 else 1.0))
+# plain max|err| / rms of dq and dk as measured (train_1p3b 2.6e-2 / 3.3e-2, t2r_7b 6.8e-2 / 1.9e-2)
+# plus 10%: the half-ulp of bfloat16 at the largest elements
+TC_PLAIN_CEILING = {
+    ("train_1p3b", "dq"): 2.9e-2, ("train_1p3b", "dk"): 3.7e-2,
+    ("t2r_7b", "dq"): 7.5e-2, ("t2r_7b", "dk"): 2.1e-2,
+}
 
 
 def bf16_half_ulp(ref):
@@ -64,6 +55,26 @@ def bf16_half_ulp(ref):
     a = np.abs(np.asarray(ref, dtype=np.float64))
     e = np.floor(np.log2(np.maximum(a, 1e-300)))
     return np.where(a > 0, 2.0 ** (e - 8), 0.0)
+
+
+def bf16_storage_check(x, ref):
+    """Direct check of the reading that a bfloat16-stored result differs from the oracle by the
+    rounding of its storage format and nothing else: every element of x must lie within one
+    bfloat16 ulp (2^-7 of the binade) of the oracle value rounded to nearest-even bfloat16.  The
+    ulp is taken at max(|ref|, 2e-2 rms(ref)): below that size an ulp is finer than the fp32
+    arithmetic behind the result.  Returns (largest distance in such ulps, fraction of elements
+    that are bit-equal to the rounded oracle value)."""
+    x = np.asarray(x, dtype=np.float64)
+    ref = np.asarray(ref, dtype=np.float64)
+    rms = np.sqrt(np.mean(ref ** 2))
+    a = np.abs(ref)
+    e = np.floor(np.log2(np.maximum(a, 1e-300)))
+    ulp = np.where(a > 0, 2.0 ** (e - 7), 0.0)
+    rne = np.where(a > 0, np.rint(ref / np.where(ulp > 0, ulp, 1.0)) * ulp, 0.0)
+    floor = max(2e-2 * rms, 1e-300)
+    ulp_eff = 2.0 ** (np.floor(np.log2(np.maximum(a, floor))) - 7)
+    worst = float((np.abs(x - rne) / ulp_eff).max())
+    return worst, float(np.mean(x == rne))
 
 
 def rel_err(x, ref, stored_bf16=False):
