@@ -89,6 +89,9 @@ def kernel_algorithmic_bytes(label: str, w: W.Workload) -> int:
         "bwd_dk_key_side_rev": 2 * w.d_k * e + 8 * m,
         "bwd_dIk_value_side_rev": 2 * w.d_k * e + 4 * m + 4 * m * nsk,
         "gate_grad": 4 * m * (7 + nsk + nsv),   # u, gate, G, partials -> dgate; carry pass reads gate, r/w dgate
+        # fused chunk kernels: the slot rows between the passes stay on chip
+        "fused_fwd": e * (2 * w.d_k + 2 * w.d_v) + 12 * m,           # q, k, v, I exp(-G), G -> o, o'
+        "fused_bwd": e * (2 * w.d_k + 2 * w.d_v) + 24 * m,           # dO, v, k, I exp(-G), G, o' -> dq, u, p exp(G), dz exp(G)
     }
     return R * table[label]
 
@@ -96,6 +99,8 @@ def kernel_algorithmic_bytes(label: str, w: W.Workload) -> int:
 def kernel_function(label: str) -> str:
     """The kernel that serves a timing label: the four value_side scans of a step are launches
     of one kernel, and so are the four key_side scans."""
+    if label.startswith("fused"):
+        return "fused_pair_kernel"
     if "key_side" in label:
         return "key_side_lean_kernel"
     if "value_side" in label:
@@ -109,7 +114,9 @@ def kernel_algorithmic_flops(fn: str, w: W.Workload, d: int) -> float:
     slot-space or head-space product, the intra-chunk product, the inter-chunk product and
     the state update."""
     C, m = 128, w.m
-    per_row = 2 * C * (m + d) + 4 * m * d if fn == "key_side_lean_kernel" else 2 * C * (d + m) + 4 * m * d
+    per_row = 2 * C * (m + d) + 4 * m * d      # (the same count for either primitive)
+    if fn == "fused_pair_kernel":
+        per_row *= 2                           # a value_side and a key_side scan
     return float(per_row) * w.B * w.T * w.H
 
 
@@ -262,7 +269,8 @@ def run_ours(args):
 
     w = rank_workload(rank)
     x = W.make_inputs(w)
-    p = gsa.Params(w.B, w.T, w.H, w.d_k, w.d_v, w.m, io=w.io, slot_act=args.slot_act, tc_operands=args.tc_operands)
+    p = gsa.Params(w.B, w.T, w.H, w.d_k, w.d_v, w.m, io=w.io, slot_act=args.slot_act, tc_operands=args.tc_operands,
+                   fuse=args.fuse)
 
     def host(a, bf16):
         t = torch.from_numpy(np.ascontiguousarray(a))
@@ -344,17 +352,25 @@ def run_ours(args):
             launch_mode += f" (graph capture failed: {type(exc).__name__})"
             torch.cuda.synchronize()
     total_ms = timed(run_step, args.steps)
-    # The timed region lasts a few tens of milliseconds, shorter than nvidia-smi's sampling
-    # period: keep the same steps running (untimed) for about a second so that the sampler
-    # sees the clocks of exactly this load.
-    t_end = time.perf_counter() + 1.2
+    # The timed region lasts a few milliseconds, shorter than nvidia-smi's sampling period and too short
+    # for the power limiter to settle: keep the same steps running for at least 1.5 s more, timed with
+    # CUDA events as well, so that the clock samples and the `sustained` figure describe the same load.
+    sust_steps, sust_ms = 0, 0.0
+    t_end = time.perf_counter() + 1.5
     while time.perf_counter() < t_end:
-        for _ in range(20):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(100):
             run_step()
+        e1.record()
         torch.cuda.synchronize()
+        sust_ms += float(e0.elapsed_time(e1))
+        sust_steps += 100
+    sust_ms = max_over_ranks(sust_ms, world, dev)
     clocks = sampler.stop() if rank == 0 else {}
     if rank == 0:
-        clocks["note"] = "nvidia-smi samples (50 ms period, utilisation >= 50%) over warm-up, the timed steps and 1.2 s more of the same steps"
+        clocks["note"] = ("nvidia-smi samples (50 ms period, utilisation >= 50%) over warm-up, the timed steps and "
+                          "the sustained loop of the same steps that follows them")
     ms_step = total_ms / args.steps
     value = aggregate_tokens_per_s(world, w.tokens, ms_step)
     if int(status.item()) != 0:
@@ -418,7 +434,9 @@ def run_ours(args):
         # kernels behind one label: gate_grad is three; every chunk pass is two (the lean and the
         # general variant of the kernel are both launched, each CTA runs in one of them)
         two = sum(len(v) for lab, v in per.items() if lab.endswith("_side") or lab.endswith("_side_rev"))
-        launches = (len(recs) + 2 * len(per.get("gate_grad", [])) + two) // reps
+        # a fused label is the fused kernel plus the three kernels that serve the flagged pairs
+        fusedl = sum(len(v) for lab, v in per.items() if lab.startswith("fused"))
+        launches = (len(recs) + 2 * len(per.get("gate_grad", [])) + two + 3 * fusedl) // reps
         kernels = []
         tot = sum(sum(v) for v in per.values())
         for lab, v in per.items():
@@ -446,7 +464,7 @@ def run_ours(args):
                     "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": alg / (avg_ms * 1e-3) / 1e9 / pk["hbm_gbs"],
                     "traffic": traffic, "peak_source": pk["source"],
                     "share_of_step": sum(k_["share"] for k_ in members)}
-        if fn.endswith("_side_lean_kernel"):
+        if fn.endswith("_side_lean_kernel") or fn == "fused_pair_kernel":
             d = w.d_v if fn.startswith("key") else w.d_k     # (d_k == d_v in the benchmark workload)
             fl = kernel_algorithmic_flops(fn, w, d)
             roofline["alg_tflops"] = fl / (avg_ms * 1e-3) / 1e12
@@ -462,6 +480,7 @@ def run_ours(args):
 
         # ---- decode step (the recurrent form), reported beside the training number
         decode = bench_decode(gsa, torch, dev, pk)
+        others = [] if args.no_other_configs else bench_other_configs(gsa, torch, dev, pk, args)
 
         # ---- the oracle on the host cores, bounded sample
         cpu = None
@@ -487,10 +506,15 @@ def run_ours(args):
                        "step": ("gsa_fwd (logits saved) + gsa_bwd" if args.recompute_gate else
                                 "gsa_fwd_save_gate (logits and the gate kernel's products saved) + gsa_bwd_saved_gate"),
                        "slot_act": args.slot_act, "tc_operands": args.tc_operands,
+                       "fused_slot_softmax": bool(args.fuse),
                        "launch": launch_mode,
                        "l2": "inputs larger than L2 (1.1 GB touched per step vs 126 MB)",
                        "parallelism": f"dp{world} over batch, no collective"},
             "clocks": clocks,
+            "sustained": {"ms_per_step": sust_ms / sust_steps, "tokens_per_s": aggregate_tokens_per_s(world, w.tokens, sust_ms / sust_steps),
+                          "steps": sust_steps, "seconds": sust_ms * 1e-3, "sm_mhz_median": clocks.get("sm_mhz"),
+                          "ms_x_mhz": (sust_ms / sust_steps) * clocks["sm_mhz"] if clocks.get("sm_mhz") else None,
+                          "note": "the same step replayed back to back for >= 1.5 s (power-capped clocks), CUDA events"},
             "e2e": {"value": world * w.tokens / (e2e_ms * 1e-3), "unit": UNIT,
                     "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms,
                     "overlap": "every step copies its inputs up and its results down; copies of "
@@ -501,6 +525,7 @@ def run_ours(args):
             "whole_step": whole,
             "kernels": kernels,
             "decode": decode,
+            "configs": others,
             "cpu_baseline": cpu,
         }
     if world > 1:
@@ -508,6 +533,82 @@ def run_ours(args):
         dist.destroy_process_group()
     if line is not None:
         print(json.dumps(line), flush=True)
+
+
+def forward_algorithmic_bytes(w: W.Workload) -> int:
+    """q, k, v, gate in; o out (no saved logits)."""
+    e = 2 if w.io == "bf16" else 4
+    return w.B * w.T * w.H * (e * (2 * w.d_k + 2 * w.d_v) + 4 * w.m)
+
+
+def bench_other_configs(gsa, torch, dev, pk, args):
+    """The other configurations, outside the headline region: plain library calls, CUDA events,
+    whole-call time and the fraction of the HBM bound on the bytes every tensor must cross HBM once."""
+    out = []
+    plan = [("t2r_7b", True, 10), ("long_keep", False, 10), ("long_forget", False, 5), ("tiny_f32", False, 50)]
+    for name, with_bwd, reps in plan:
+        w = W.CONFIGS[name]
+        x = W.make_inputs(w)
+        p = gsa.Params(w.B, w.T, w.H, w.d_k, w.d_v, w.m, io=w.io, fuse=args.fuse)
+
+        def dev_t(a, io_typed):
+            t = torch.from_numpy(np.ascontiguousarray(a)).to(dev)
+            return t.to(torch.bfloat16) if (io_typed and w.io == "bf16") else t
+
+        q, k, v = (dev_t(x[n], True) for n in ("q", "k", "v"))
+        gate = dev_t(x["gate"], False)
+        K0 = dev_t(x["K0"], False) if "K0" in x else None
+        V0 = dev_t(x["V0"], False) if "V0" in x else None
+        dO = dev_t(x["dO"], True) if with_bwd else None
+        o = torch.empty(w.B, w.T, w.H, w.d_v, dtype=p.io_dtype, device=dev)
+        ok = torch.empty(w.B, w.T, w.H, w.m, device=dev) if with_bwd else None
+        KT = torch.empty(w.B, w.H, w.m, w.d_k, device=dev) if K0 is not None else None
+        VT = torch.empty(w.B, w.H, w.m, w.d_v, device=dev) if V0 is not None else None
+        ws_f = torch.empty(max(gsa.gsa_workspace_bytes(p, 0), 256), dtype=torch.uint8, device=dev)
+        status = torch.zeros(1, dtype=torch.int32, device=dev)
+        blk = gsa.gate_block(p, dev) if with_bwd else None
+        if with_bwd:
+            ws_b = torch.empty(gsa.gsa_workspace_bytes(p, 1), dtype=torch.uint8, device=dev)
+            dq, dk, dv, dg = torch.empty_like(q), torch.empty_like(k), torch.empty_like(v), torch.empty_like(gate)
+
+        def fwd():
+            gsa.gsa_fwd(p, q, k, v, gate, K0, V0, o=o, ok_save=ok, KT=KT, VT=VT, ws=ws_f, dev_status=status, gate_save=blk)
+
+        def bwd():
+            gsa.gsa_bwd(p, q, k, v, gate, dO, K0, V0, ok_saved=ok, dq=dq, dk=dk, dv=dv, dgate=dg, ws=ws_b,
+                        dev_status=status, gate_saved=blk)
+
+        def time_ms(fn):
+            for _ in range(3):
+                fn()
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(reps):
+                fn()
+            e1.record()
+            torch.cuda.synchronize()
+            return float(e0.elapsed_time(e1)) / reps
+
+        f_ms = time_ms(fwd)
+        rec = {"workload": name, "B": w.B, "T": w.T, "H": w.H, "d": w.d_k, "m": w.m, "io": w.io,
+               "fwd_ms": f_ms, "fwd_tokens_per_s": w.tokens / (f_ms * 1e-3)}
+        by = forward_algorithmic_bytes(w)
+        if with_bwd:
+            b_ms = time_ms(bwd)
+            by = step_algorithmic_bytes(w)
+            rec.update(bwd_ms=b_ms, step_ms=f_ms + b_ms, step_tokens_per_s=w.tokens / ((f_ms + b_ms) * 1e-3))
+        t_ms = rec.get("step_ms", f_ms)
+        rec.update(alg_bytes=by, frac_of_hbm_peak=by / (t_ms * 1e-3) / 1e9 / pk["hbm_gbs"],
+                   launch="plain library calls" + (", gate kernel's products saved for the backward" if with_bwd else ""))
+        if name == "tiny_f32":
+            rec["note"] = "latency of one call (launch-bound); the fraction of the HBM bound means nothing at this size"
+        if int(status.item()) != 0:
+            rec["error"] = "a bounded device-side wait expired"
+        out.append(rec)
+        del q, k, v, gate, o
+        torch.cuda.empty_cache()
+    return out
 
 
 def bench_decode(gsa, torch, dev, pk):
@@ -558,6 +659,11 @@ def main():
     ap.add_argument("--slot-act", default="softmax", choices=["softmax", "none", "relu", "swish", "relu2"],
                     help="the non-linearity between the two passes: the paper's softmax (the headline "
                          "workload) or one of the replacements of its ablation")
+    ap.add_argument("--fuse", action="store_true",
+                    help="the fused chunk kernel (pass 1 -> slot softmax -> pass 2 in one kernel, and its backward "
+                         "twin) instead of the separate kernels; slower as measured, not the default")
+    ap.add_argument("--no-other-configs", action="store_true",
+                    help="skip the list of the other configurations (t2r_7b, long_keep, long_forget, tiny_f32)")
     ap.add_argument("--no-graph", action="store_true", help="time plain library calls instead of a CUDA graph replay")
     ap.add_argument("--profile-case", action="store_true",
                     help="run warmup + steps bare (for ncu); prints no benchmark line")

@@ -94,6 +94,19 @@ typedef enum {
     GSA_IMPL_TC = 2      /* tcgen05 bf16 tensor-core kernels (bf16 io only) */
 } gsa_impl_t;
 
+/* Tensor-core kernels only: whether the slot non-linearity runs inside the chunk kernel. */
+typedef enum {
+    GSA_FUSE_OFF = 0,    /* separate kernels: pass 1, slot softmax, pass 2 (and dp, dsoftmax, dq in the backward),
+                          * the slot-sized rows between them passed through the workspace; the faster form
+                          * on B200 as measured, hence the default */
+    GSA_FUSE_ON = 1      /* pass 1 -> softmax -> pass 2 (and dp -> dsoftmax -> dq) as ONE kernel wherever the
+                          * shape allows it (d_k == d_v in {128, 256, 512}, m = 64, paired operands): the slot
+                          * rows between the passes never leave the chip (a cluster of d / 128 CTAs per
+                          * (batch, head) exchanges them through distributed shared memory); with
+                          * ok_save == NULL the forward then writes nothing but o.  Other shapes fall back
+                          * to the separate kernels. */
+} gsa_fuse_t;
+
 typedef struct {
     int32_t B, T, H, d_k, d_v, m;
     int32_t io;         /* gsa_dtype_t */
@@ -103,6 +116,7 @@ typedef struct {
     float tau;          /* GSA_GATE_LOGITS only: damping of the gate, a = sigmoid(x)^(1/tau); > 0 */
     int32_t slot_act;   /* gsa_act_t; 0 = the paper's softmax */
     int32_t tc_operands; /* gsa_tc_operands_t; ignored by the fp32 kernels */
+    int32_t fuse;       /* gsa_fuse_t; ignored by the fp32 kernels */
 } gsa_params_t;
 
 enum { GSA_WS_FWD = 0, GSA_WS_BWD = 1, GSA_WS_DECODE = 2, GSA_WS_GATE = 3 };

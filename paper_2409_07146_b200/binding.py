@@ -32,7 +32,7 @@ class _CParams(ctypes.Structure):
                 ("d_k", ctypes.c_int32), ("d_v", ctypes.c_int32), ("m", ctypes.c_int32),
                 ("io", ctypes.c_int32), ("gate_kind", ctypes.c_int32),
                 ("scale", ctypes.c_float), ("impl", ctypes.c_int32), ("tau", ctypes.c_float),
-                ("slot_act", ctypes.c_int32), ("tc_operands", ctypes.c_int32)]
+                ("slot_act", ctypes.c_int32), ("tc_operands", ctypes.c_int32), ("fuse", ctypes.c_int32)]
 
 
 @dataclass(frozen=True)
@@ -52,6 +52,7 @@ class Params:
     tau: float = 8.0
     slot_act: str = "softmax"      # "softmax" | "none" | "relu" | "swish" | "relu2"
     tc_operands: str = "paired"    # "paired" | "single" (tensor-core kernels: derived operands as bf16 pairs or not)
+    fuse: bool = False             # tensor-core kernels: pass 1 -> softmax -> pass 2 as one kernel where the shape allows (gsa_fuse_t)
 
     def c(self) -> _CParams:
         return _CParams(self.B, self.T, self.H, self.d_k, self.d_v, self.m,
@@ -59,7 +60,7 @@ class Params:
                         GSA_GATE_LOGITS if self.gate_is_logits else
                         (GSA_GATE_LOG_A if self.gate_is_log else GSA_GATE_A),
                         float(self.scale), _IMPL[self.impl], float(self.tau), _ACT[self.slot_act],
-                        0 if self.tc_operands == "paired" else 1)
+                        0 if self.tc_operands == "paired" else 1, 1 if self.fuse else 0)
 
     @property
     def io_dtype(self) -> torch.dtype:

@@ -29,6 +29,7 @@ gsa_status_t check_params(const gsa_params_t* p, bool need_T) {
     if (p->tc_operands != GSA_TC_PAIRED && p->tc_operands != GSA_TC_SINGLE) return GSA_ERR_INVALID_ARG;
     if (p->impl != GSA_IMPL_AUTO && p->impl != GSA_IMPL_SIMT && p->impl != GSA_IMPL_TC)
         return GSA_ERR_INVALID_ARG;
+    if (p->fuse != GSA_FUSE_OFF && p->fuse != GSA_FUSE_ON) return GSA_ERR_INVALID_ARG;
     if (!(p->scale == p->scale)) return GSA_ERR_INVALID_ARG;
     if (!dim_ok(p->d_k) || !dim_ok(p->d_v)) return GSA_ERR_UNSUPPORTED;
     if (p->m != 32 && p->m != 64) return GSA_ERR_UNSUPPORTED;
@@ -43,6 +44,13 @@ gsa_status_t check_params(const gsa_params_t* p, bool need_T) {
 bool use_tc(const gsa_params_t& p) {
     if (p.impl == GSA_IMPL_SIMT) return false;
     return p.io == GSA_BF16 && tc_supported(p.d_k, p.d_v, p.m);
+}
+
+// Does this call run the slot non-linearity inside the fused chunk kernel?  (The operand pairs are
+// built into that kernel: GSA_TC_SINGLE keeps the separate kernels.)
+bool use_fused(const gsa_params_t& p) {
+    return use_tc(p) && p.fuse == GSA_FUSE_ON && p.tc_operands == GSA_TC_PAIRED &&
+           fused_pair_supported(p.d_k, p.d_v, p.m);
 }
 
 float inv_tau(const gsa_params_t& p) { return p.tau > 0.f ? 1.f / p.tau : 0.f; }
@@ -354,11 +362,36 @@ gsa_status_t fwd_impl(const gsa_params_t* params, const void* q, const void* k, 
     }
     // pass 1: o' = GLA(q, k, 1-a) with the decay on the slot (value) side
     ValueSideArgs a1{q, k, w.I, w.G, Kin, Kout, w.okpart, Bs, Ts, p.H, p.d_k, w.Id};
+    // pass 2: o = GLA(softmax(o'), 1-a, v) with the decay on the slot (key) side
+    KeySideArgs a2{w.p, w.I, w.G, v, Vin, Vout, o, Bs, Ts, p.H, p.d_v, w.Pd, w.Id};
+    if (use_fused(p)) {
+        // One kernel for pass 1 -> softmax -> pass 2; the logits are written only if the caller wants
+        // them.  The (batch, head) pairs flagged for strong decay take the general kernels and the
+        // slot kernel (restricted to those pairs) on the side stream, beside the fused kernel.
+        PendingDecay only = pend;
+        only.strong_only = 1;
+        SideLane* side = nullptr;
+        GSA_CUDA(side_lane(&side));
+        cudaStream_t ss = g_sink.active ? st : side->stream;
+        if (!g_sink.active) {
+            GSA_CUDA(cudaEventRecord(side->fork, st));
+            GSA_CUDA(cudaStreamWaitEvent(ss, side->fork, 0));
+        }
+        GSA_LAUNCH("fused_fwd", launch_fused_pair(0, q, k, w.Id, v, o, w.G, Kin, Vin, Kout, Vout, Bs, Ts, p.H, p.d_k,
+                                                  p.d_v, p.scale, p.slot_act, ok_save, nullptr, nullptr, nullptr, w.strong,
+                                                  st, dev_status));
+        GSA_CUDA(launch_value_side_general(a1, p.m, 0, w.strong, ss, dev_status));
+        GSA_CUDA(launch_slot_softmax_fwd(w.okpart, s.k, p.scale, p.slot_act, ok, w.p, p.B, p.T * p.H, p.m, pend.G, w.Pd, only, ss));
+        GSA_CUDA(launch_key_side_general(a2, p.m, 0, w.strong, ss, dev_status));
+        if (!g_sink.active) {
+            GSA_CUDA(cudaEventRecord(side->join, ss));
+            GSA_CUDA(cudaStreamWaitEvent(st, side->join, 0));
+        }
+        return GSA_OK;
+    }
     GSA_LAUNCH("pass1_value_side", value_side(p, a1, 0, w.strong, st, dev_status));
     GSA_LAUNCH("slot_softmax", launch_slot_softmax_fwd(w.okpart, s.k, p.scale, p.slot_act, ok, w.p, p.B, p.T * p.H, p.m, pend.G, w.Pd,
                                                        pend, st));
-    // pass 2: o = GLA(softmax(o'), 1-a, v) with the decay on the slot (key) side
-    KeySideArgs a2{w.p, w.I, w.G, v, Vin, Vout, o, Bs, Ts, p.H, p.d_v, w.Pd, w.Id};
     GSA_LAUNCH("pass2_key_side", key_side(p, a2, 0, w.strong, st, dev_status));
     return GSA_OK;
 }
@@ -445,9 +478,37 @@ gsa_status_t bwd_impl(const gsa_params_t* params, const void* q, const void* k, 
     }
     // gradient w.r.t. the pass-2 queries p: the pass-1 form on (dO, v, 1-a); carries V~
     ValueSideArgs adp{dO, v, w.I, w.G, Vin, VTout, w.dppart, Bs, Ts, p.H, p.d_v, w.Id};
-    GSA_LAUNCH("bwd_dp_value_side", value_side(p, adp, 0, w.strong, st, dev_status));
-    GSA_LAUNCH("slot_softmax_bwd", launch_slot_softmax_bwd(ok, w.dppart, s.v, p.scale, p.slot_act, w.p, w.dz, w.u, p.B, p.T * p.H, p.m, pend.G, w.Pd,
-                                                           w.Zd, pend, st));
+    // dq: the pass-2 form on (dz, 1-a, k); carries K~
+    KeySideArgs adq{w.dz, w.I, w.G, k, Kin, KTout, dq, Bs, Ts, p.H, p.d_k, w.Zd, w.Id};
+    const bool fused = use_fused(p);
+    if (fused) {
+        // One kernel for dp -> dsoftmax -> dq (it also leaves u and the decayed rows of p and dz for the
+        // reversed scans); the flagged pairs take the general kernels on the side stream.
+        PendingDecay only = pend;
+        only.strong_only = 1;
+        SideLane* side = nullptr;
+        GSA_CUDA(side_lane(&side));
+        cudaStream_t ss = g_sink.active ? st : side->stream;
+        if (!g_sink.active) {
+            GSA_CUDA(cudaEventRecord(side->fork, st));
+            GSA_CUDA(cudaStreamWaitEvent(ss, side->fork, 0));
+        }
+        GSA_LAUNCH("fused_bwd", launch_fused_pair(1, dO, v, w.Id, k, dq, w.G, Vin, Kin, VTout, KTout, Bs, Ts, p.H, p.d_v,
+                                                  p.d_k, p.scale, p.slot_act, const_cast<float*>(ok), w.u, w.Pd, w.Zd,
+                                                  w.strong, st, dev_status));
+        GSA_CUDA(launch_value_side_general(adp, p.m, 0, w.strong, ss, dev_status));
+        GSA_CUDA(launch_slot_softmax_bwd(ok, w.dppart, s.v, p.scale, p.slot_act, w.p, w.dz, w.u, p.B, p.T * p.H, p.m, pend.G,
+                                         w.Pd, w.Zd, only, ss));
+        GSA_CUDA(launch_key_side_general(adq, p.m, 0, w.strong, ss, dev_status));
+        if (!g_sink.active) {
+            GSA_CUDA(cudaEventRecord(side->join, ss));
+            GSA_CUDA(cudaStreamWaitEvent(st, side->join, 0));
+        }
+    } else {
+        GSA_LAUNCH("bwd_dp_value_side", value_side(p, adp, 0, w.strong, st, dev_status));
+        GSA_LAUNCH("slot_softmax_bwd", launch_slot_softmax_bwd(ok, w.dppart, s.v, p.scale, p.slot_act, w.p, w.dz, w.u, p.B, p.T * p.H, p.m, pend.G, w.Pd,
+                                                               w.Zd, pend, st));
+    }
     const float *dKin = dKT, *dVin = dVT;    // states entering the reversed scans (from the right)
     float *dK0out = dK0, *dV0out = dV0;
     if (nseg > 1) {
@@ -465,8 +526,6 @@ gsa_status_t bwd_impl(const gsa_params_t* params, const void* q, const void* k, 
         dKin = w.dKend; dVin = w.dVend;
         dK0out = nullptr; dV0out = nullptr;
     }
-    // dq: the pass-2 form on (dz, 1-a, k); carries K~
-    KeySideArgs adq{w.dz, w.I, w.G, k, Kin, KTout, dq, Bs, Ts, p.H, p.d_k, w.Zd, w.Id};
     // time-reversed runs: dv and dI^v share the state dV~; dk and dI^k share dK~
     KeySideArgs adv{w.I, w.p, w.G, dO, dVin, dV0out, dv, Bs, Ts, p.H, p.d_v, w.Id, w.Pd};
     ValueSideArgs adIv{v, dO, w.p, w.G, dVin, nullptr, w.dIv, Bs, Ts, p.H, p.d_v, w.Pd};
@@ -478,7 +537,7 @@ gsa_status_t bwd_impl(const gsa_params_t* params, const void* q, const void* k, 
         GSA_CUDA(scan_lanes(&lanes));
         GSA_CUDA(cudaEventRecord(lanes->fork, st));
         for (int i = 0; i < 4; ++i) GSA_CUDA(cudaStreamWaitEvent(lanes->stream[i], lanes->fork, 0));
-        GSA_CUDA(key_side(p, adq, 0, w.strong, st, dev_status));
+        if (!fused) GSA_CUDA(key_side(p, adq, 0, w.strong, st, dev_status));
         GSA_CUDA(key_side(p, adv, 1, w.strong, lanes->stream[0], dev_status));
         GSA_CUDA(value_side(p, adIv, 1, w.strong, lanes->stream[1], dev_status));
         GSA_CUDA(key_side(p, adk, 1, w.strong, lanes->stream[2], dev_status));
@@ -488,7 +547,7 @@ gsa_status_t bwd_impl(const gsa_params_t* params, const void* q, const void* k, 
             GSA_CUDA(cudaStreamWaitEvent(st, lanes->join[i], 0));
         }
     } else {
-        GSA_LAUNCH("bwd_dq_key_side", key_side(p, adq, 0, w.strong, st, dev_status));
+        if (!fused) GSA_LAUNCH("bwd_dq_key_side", key_side(p, adq, 0, w.strong, st, dev_status));
         GSA_LAUNCH("bwd_dv_key_side_rev", key_side(p, adv, 1, w.strong, st, dev_status));
         GSA_LAUNCH("bwd_dIv_value_side_rev", value_side(p, adIv, 1, w.strong, st, dev_status));
         GSA_LAUNCH("bwd_dk_key_side_rev", key_side(p, adk, 1, w.strong, st, dev_status));

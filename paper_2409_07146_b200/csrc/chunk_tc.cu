@@ -90,42 +90,93 @@ __device__ __forceinline__ void ctl_init(Ctl* ctl, int tid, int warp) {
     tc_fence_after_sync();
 }
 
+// Strong-decay chunks (App. A: a decay too strong for one reference point per chunk).  The decay
+// between two rows of a chunk is a product of per-step gates, prod_{r=j+1..i} a_r[s], every factor
+// <= 1: walking j away from the target row i, the product is carried along by ONE multiplication
+// per step and slot -- no exponential in the loop, nothing can overflow -- and the walk stops as
+// soon as the product has fallen below 2^-40 for all slots of the thread (what is left of the sum is
+// then below 1e-12 of its leading terms).  With strong forgetting that is after a dozen steps.
+// The per-step gates a_j = exp(G_j - G_{j-1}) are formed once per chunk, in place of the G tile.
+constexpr float kDecayFloor = 9.094947e-13f;      // 2^-40
+
+// Replace the G tile by the per-step gates (rows past the end: 1).  gi receives this thread's own
+// G row (slots sb .. sb+31) first.  Two compute-thread barriers inside.
+__device__ __forceinline__ void gates_in_place(unsigned char* gt, int row, int half, int sb, int valid, float (&gi)[kHS]) {
+    const int grow = min(row, valid - 1);
+    float aj[kHS];
+#pragma unroll
+    for (int c = 0; c < kHS / 8; ++c) {
+        float g[8], gp[8];
+        tile_row8(gt, grow, sb + 8 * c, g);
+        if (row > 0 && row < valid) tile_row8(gt, row - 1, sb + 8 * c, gp);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+            gi[8 * c + e] = g[e];
+            aj[8 * c + e] = row >= valid ? 1.f : __expf(row > 0 ? g[e] - gp[e] : g[e]);
+        }
+    }
+    compute_sync();           // every thread has read what it needs of G
+    unsigned char* panel = gt + half * kPanelB;
+#pragma unroll
+    for (int c = 0; c < kHS / 4; ++c)
+        *reinterpret_cast<float4*>(panel + swz128(row, c)) = make_float4(aj[4 * c], aj[4 * c + 1], aj[4 * c + 2], aj[4 * c + 3]);
+    compute_sync();
+}
+
+// 16 consecutive fp32 values (s0 % 16 == 0) of row `row` of a slot-sized fp32 tile
+__device__ __forceinline__ void tile_row16(const unsigned char* tile, int row, int s0, float (&x)[16]) {
+    const unsigned char* panel = tile + (s0 >> 5) * kPanelB;
+    const int c = (s0 & 31) >> 2;
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+        const float4 t = *reinterpret_cast<const float4*>(panel + swz128(row, c + q));
+        x[4 * q] = t.x; x[4 * q + 1] = t.y; x[4 * q + 2] = t.z; x[4 * q + 3] = t.w;
+    }
+}
+
 // Strong-decay chunk of value_side: this thread's 32 output slots of row `row`,
-//   out[s] = exp(+-..) * inter[s] + sum_j P_ij w_j[s] exp(-|G_i[s] - G_j[s]|),
-// with explicit exponent differences from the fp32 weight and G tiles; P and the inter-chunk
-// product are read from the accumulators; the row goes straight to global memory.
+//   out[s] = exp(+-..) * inter[s] + sum_j P_ij w_j[s] prod a_r[s]   (j <= i forward, j >= i reverse),
+// P and the inter-chunk product are read from the accumulators; the row goes straight to global
+// memory.  `gt` holds the per-step gates (gates_in_place), gi this thread's G row.
 template <bool REV>
 __device__ __forceinline__ void value_side_explicit_rows(const unsigned char* gt, const unsigned char* sW,
-                                                      const float* gc, uint32_t tmem, int wq, int row, int sb,
-                                                      int grow, int valid, float* out_row) {
-    const int jlo = REV ? row : 0, jhi = REV ? kCT - 1 : row;
-    // the accumulator loads are warp-collective: loop bounds are those of the whole warp
-    const int wlo = REV ? wq * 32 : 0, whi = REV ? kCT - 1 : wq * 32 + 31;
+                                                      const float* gc, const float (&gi)[kHS], uint32_t tmem, int wq,
+                                                      int row, int sb, int valid, float* out_row) {
+    // the accumulator loads are warp-collective: the 16-column segments are those of the whole warp,
+    // walked away from the diagonal
+    const int first = REV ? wq * 32 : wq * 32 + 16, last = REV ? kCT - 16 : 0, step = REV ? 16 : -16;
+#pragma unroll 1
     for (int s0 = sb; s0 < sb + kHS; s0 += 16) {
-        float gi[16], acc[16], tmp[8];
-        tile_row8(gt, grow, s0, tmp);
+        float acc[16], dec[16];
 #pragma unroll
-        for (int e = 0; e < 8; ++e) gi[e] = tmp[e];
-        tile_row8(gt, grow, s0 + 8, tmp);
-#pragma unroll
-        for (int e = 0; e < 8; ++e) gi[8 + e] = tmp[e];
-#pragma unroll
-        for (int e = 0; e < 16; ++e) acc[e] = 0.f;
-        for (int c0 = wlo; c0 <= whi; c0 += 16) {
+        for (int e = 0; e < 16; ++e) { acc[e] = 0.f; dec[e] = 1.f; }
+        bool live = true;
+#pragma unroll 1
+        for (int c0 = first; REV ? c0 <= last : c0 >= last; c0 += step) {
             float v[16];
             tmem_ld16(tmem_row_addr(tmem, wq, kColP + c0), v);
+            if (live) {
 #pragma unroll
-            for (int e = 0; e < 16; ++e) {
-                const int j = c0 + e;
-                if (j < jlo || j > jhi) continue;
-                const int jg = min(j, valid - 1);
+                for (int ee = 0; ee < 16; ++ee) {
+                    const int e = REV ? ee : 15 - ee;
+                    const int j = c0 + e;
+                    if (REV ? j < row : j > row) continue;
+                    float aj[16], wj[16];
+                    tile_row16(gt, j, s0, aj);
+                    tile_row16(sW, j, s0, wj);
 #pragma unroll
-                for (int u = 0; u < 16; ++u) {
-                    const float gj = tile_elem(gt, jg, s0 + u);
-                    const float ex = REV ? gj - gi[u] : gi[u] - gj;
-                    acc[u] = fmaf(v[e] * tile_elem(sW, j, s0 + u), __expf(fminf(ex, 0.f)), acc[u]);
+                    for (int u = 0; u < 16; ++u) {
+                        if (REV && j > row) dec[u] *= aj[u];            // prod_{r=i+1..j}
+                        acc[u] = fmaf(v[e] * wj[u], dec[u], acc[u]);
+                        if (!REV) dec[u] *= aj[u];                      // prod_{r=j..i} for the next (earlier) row
+                    }
                 }
+                float top = 0.f;
+#pragma unroll
+                for (int u = 0; u < 16; ++u) top = fmaxf(top, dec[u]);
+                live = top >= kDecayFloor;
             }
+            if (!__any_sync(0xffffffffu, live)) break;
         }
         float vi[16];
         tmem_ld16(tmem_row_addr(tmem, wq, kColO + s0), vi);
@@ -135,7 +186,7 @@ __device__ __forceinline__ void value_side_explicit_rows(const unsigned char* gt
                 float r[4];
 #pragma unroll
                 for (int u = 0; u < 4; ++u)
-                    r[u] = fmaf(vi[e + u], __expf(REV ? gc[s0 + e + u] - gi[e + u] : gi[e + u]), acc[e + u]);
+                    r[u] = fmaf(vi[e + u], __expf(REV ? gc[s0 + e + u] - gi[s0 - sb + e + u] : gi[s0 - sb + e + u]), acc[e + u]);
                 *reinterpret_cast<float4*>(out_row + s0 + e) = make_float4(r[0], r[1], r[2], r[3]);
             }
         }
@@ -363,9 +414,12 @@ value_side_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_cons
                 // cores (only the general variant of the kernel carries this path).
                 WAIT_OR_ABORT(&ctl->bar_mma1, it & 1);    // the inter-chunk product
                 tc_fence_after_sync();
-                if (!a.state_only)
-                    value_side_explicit_rows<REV>(gt, sW, ctl->gc, tmem, wq, row, sb, grow, valid,
+                if (!a.state_only) {
+                    float gi[kHS];
+                    gates_in_place(const_cast<unsigned char*>(gt), row, half, sb, valid, gi);
+                    value_side_explicit_rows<REV>(gt, sW, ctl->gc, gi, tmem, wq, row, sb, valid,
                                                   obase + (size_t)(t0 + row) * strideM);
+                }
             }
 
             // ---- state update from U: S <- S exp(G_C) + U  (forward moderate chunk: exp(G_C) (S + U))
@@ -452,43 +506,67 @@ value_side_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_cons
     }
 }
 
-// Strong-decay chunk of key_side: A_ij = sum_s uq_i[s] uk_j[s] exp(-|G_i[s] - G_j[s]|) on the kept
-// triangle, computed with explicit exponent differences from the fp32 uq / uk / G tiles, and
-// written as the bf16 operand rows of the masked matrix (which shares its buffer with the
-// uq tile: every thread first takes its uq row into registers).
+// Strong-decay chunk of key_side: A_ij = sum_s uq_i[s] uk_j[s] prod a_r[s] on the kept triangle, by
+// the same walk: the thread carries uq_i[s] times the running decay product for its 64 slots, one
+// multiplication per step and slot, and stops once every product is below 2^-40.  Written as the
+// bf16 operand rows of the masked matrix (which shares its buffer with the uq tile: every thread
+// first takes its uq row into registers).  `sG` is replaced by the per-step gates on the way.
 template <bool REV>
-__device__ __forceinline__ void key_side_explicit_rows(const unsigned char* sG, const unsigned char* sUq,
+__device__ __forceinline__ void key_side_explicit_rows(unsigned char* sG, const unsigned char* sUq,
                                                     const unsigned char* sUk, unsigned char* sAm,
-                                                    unsigned char* sAl, int row, int half, int grow, int valid) {
-    float gi[kM], qi[kM];
+                                                    unsigned char* sAl, int row, int half, int sb, int grow, int valid) {
+    // thread (row, half) fills columns j in [64 half, 64 half + 63]; its walk starts at the column nearest to
+    // the diagonal: j0 = min(row, 64 half + 63) forward, max(row, 64 half) reverse
+    const int jlo = 64 * half, jhi = jlo + 63;
+    const bool any = REV ? row <= jhi : row >= jlo;
+    const int j0 = REV ? max(row, jlo) : min(row, jhi);
+    float qd[kM];
+    {
+        // uq_i[s] exp(G_i[s] - G_j0[s]) (reverse: G_j0 - G_i): the product of the gates between the row and the
+        // start of the walk, 64 exponentials once (zero exponent when the walk starts on the diagonal)
+        const int g0 = min(j0, valid - 1);
 #pragma unroll
-    for (int s0 = 0; s0 < kM; s0 += 8) {
-        float g[8], uq[8];
-        tile_row8(sG, grow, s0, g);
-        tile_row8(sUq, row, s0, uq);
+        for (int s0 = 0; s0 < kM; s0 += 8) {
+            float g[8], gj[8], uq[8];
+            tile_row8(sG, grow, s0, g);
+            tile_row8(sG, g0, s0, gj);
+            tile_row8(sUq, row, s0, uq);
 #pragma unroll
-        for (int e = 0; e < 8; ++e) { gi[s0 + e] = g[e]; qi[s0 + e] = uq[e]; }
+            for (int e = 0; e < 8; ++e) qd[s0 + e] = uq[e] * __expf(fminf(REV ? gj[e] - g[e] : g[e] - gj[e], 0.f));
+        }
     }
-    compute_sync();           // every thread has its uq row in registers before sAm is written
-    for (int c0 = 64 * half; c0 < 64 * half + 64; c0 += 8) {
-        float x[8];
+    float gi[kHS];
+    gates_in_place(sG, row, half, sb, valid, gi);       // (its barriers also cover: every uq row is in registers)
+    (void)gi;
+    float x[64];
 #pragma unroll
-        for (int e = 0; e < 8; ++e) {
-            const int j = c0 + e;
-            const bool keep = REV ? (j >= row) : (j <= row);
-            float acc = 0.f;
-            if (keep) {
-                const int jg = min(j, valid - 1);
+    for (int e = 0; e < 64; ++e) x[e] = 0.f;
+    if (any) {
+#pragma unroll 1
+        for (int j = j0; REV ? j <= jhi : j >= jlo; j += REV ? 1 : -1) {
+            // reverse: the product up to column j includes a_j (prod_{r=i+1..j}); j0 itself is already covered
+            float acc = 0.f, top = 0.f;
 #pragma unroll
-                for (int s = 0; s < kM; ++s) {
-                    const float gj = tile_elem(sG, jg, s);
-                    const float ex = REV ? gj - gi[s] : gi[s] - gj;
-                    acc = fmaf(qi[s] * tile_elem(sUk, j, s), __expf(fminf(ex, 0.f)), acc);
+            for (int s0 = 0; s0 < kM; s0 += 16) {
+                float aj[16], uk[16];
+                tile_row16(sG, j, s0, aj);
+                tile_row16(sUk, j, s0, uk);
+#pragma unroll
+                for (int u = 0; u < 16; ++u) {
+                    if (REV && j > j0) qd[s0 + u] *= aj[u];
+                    acc = fmaf(qd[s0 + u], uk[u], acc);
+                    if (!REV) qd[s0 + u] *= aj[u];
+                    top = fmaxf(top, fabsf(qd[s0 + u]));
                 }
             }
-            x[e] = acc;
+            x[j - jlo] = acc;
+            if (top < 1e-30f) break;        // every later term is below 1e-30 |uk|
         }
-        store_chunk_split(sAm + (c0 >> 6) * kPanelB, sAl + (c0 >> 6) * kPanelB, row, (c0 & 63) >> 3, x);
+    }
+#pragma unroll
+    for (int c = 0; c < 8; ++c) {
+        const float xc[8] = {x[8 * c], x[8 * c + 1], x[8 * c + 2], x[8 * c + 3], x[8 * c + 4], x[8 * c + 5], x[8 * c + 6], x[8 * c + 7]};
+        store_chunk_split(sAm + half * kPanelB, sAl + half * kPanelB, row, c, xc);
     }
 }
 
@@ -696,7 +774,7 @@ key_side_tc_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_consta
             } else if constexpr (GENERAL) {
                 // Strong decay: A_ij with explicit exponent differences (only the general variant of
                 // the kernel carries this path).
-                if (!a.state_only) key_side_explicit_rows<REV>(sG, sUq, sUk, sAm, sAl, row, half, grow, valid);
+                if (!a.state_only) key_side_explicit_rows<REV>(sG, sUq, sUk, sAm, sAl, row, half, sb, grow, valid);
             }
             fence_async_smem();
             tc_fence_before_sync();
@@ -775,10 +853,6 @@ constexpr size_t kSmemKeySide = 1024 + 13 * kPanelB + sizeof(Ctl);
 // usual case that no pair is flagged, its launch and the exit of its CTAs then cost the
 // caller's stream nothing.  fork: the side stream waits for what precedes on the caller's
 // stream; join: the caller's stream waits for the general kernel.
-struct SideLane {
-    cudaStream_t stream = nullptr;
-    cudaEvent_t fork = nullptr, join = nullptr;
-};
 cudaError_t side_lane(SideLane** out) {
     constexpr int kMaxDevices = 64;
     thread_local SideLane lanes[kMaxDevices];
@@ -834,6 +908,52 @@ cudaError_t launch_value_side_tc(const ValueSideArgs& a, int M, int reverse, con
     if (e == cudaSuccess) e = cudaStreamWaitEvent(st, side->join, 0);
     if (e != cudaSuccess) return e;
 #undef GSA_LAUNCH_VS
+    return cudaGetLastError();
+}
+
+cudaError_t launch_value_side_general(const ValueSideArgs& a, int M, int reverse, const int* strong_flag,
+                                      cudaStream_t st, int32_t* dev_status) {
+    if (M != kM || a.D % kDST != 0 || strong_flag == nullptr) return cudaErrorNotSupported;
+    CUtensorMap mq, mk, mw, mg, mo;
+    cudaError_t e = make_tensor_map_bthd(&mq, a.xq, a.B, a.T, a.H, a.D, kCT, 2);
+    if (e == cudaSuccess) e = make_tensor_map_sliced(&mo, a.out, a.D / kDST, a.B, a.T, a.H, kM, kCT, 4);
+    if (e == cudaSuccess) e = make_tensor_map_bthd(&mk, a.xk, a.B, a.T, a.H, a.D, kCT, 2);
+    if (e == cudaSuccess) e = make_tensor_map_bthd(&mw, a.w, a.B, a.T, a.H, kM, kCT, 4);
+    if (e == cudaSuccess) e = make_tensor_map_bthd(&mg, a.G, a.B, a.T, a.H, kM, kCT, 4);
+    if (e != cudaSuccess) return e;
+    dim3 grid(a.B * a.H, a.D / kDST);
+    if (reverse) {
+        e = prepare(value_side_tc_kernel<true, true>, kSmemValueSide);
+        if (e != cudaSuccess) return e;
+        value_side_tc_kernel<true, true><<<grid, kThreads, kSmemValueSide, st>>>(mq, mk, mw, mg, mo, a, strong_flag, dev_status);
+    } else {
+        e = prepare(value_side_tc_kernel<false, true>, kSmemValueSide);
+        if (e != cudaSuccess) return e;
+        value_side_tc_kernel<false, true><<<grid, kThreads, kSmemValueSide, st>>>(mq, mk, mw, mg, mo, a, strong_flag, dev_status);
+    }
+    return cudaGetLastError();
+}
+
+cudaError_t launch_key_side_general(const KeySideArgs& a, int M, int reverse, const int* strong_flag,
+                                    cudaStream_t st, int32_t* dev_status) {
+    if (M != kM || a.D % kDST != 0 || strong_flag == nullptr) return cudaErrorNotSupported;
+    CUtensorMap mv, muq, muk, mg, mo;
+    cudaError_t e = make_tensor_map_bthd(&mv, a.xv, a.B, a.T, a.H, a.D, kCT, 2);
+    if (e == cudaSuccess) e = make_tensor_map_bthd(&mo, a.out, a.B, a.T, a.H, a.D, kCT, 2);
+    if (e == cudaSuccess) e = make_tensor_map_bthd(&muq, a.uq, a.B, a.T, a.H, kM, kCT, 4);
+    if (e == cudaSuccess) e = make_tensor_map_bthd(&muk, a.uk, a.B, a.T, a.H, kM, kCT, 4);
+    if (e == cudaSuccess) e = make_tensor_map_bthd(&mg, a.G, a.B, a.T, a.H, kM, kCT, 4);
+    if (e != cudaSuccess) return e;
+    dim3 grid(a.B * a.H, a.D / kDST);
+    if (reverse) {
+        e = prepare(key_side_tc_kernel<true, true>, kSmemKeySide);
+        if (e != cudaSuccess) return e;
+        key_side_tc_kernel<true, true><<<grid, kThreads, kSmemKeySide, st>>>(mv, muq, muk, mg, mo, a, strong_flag, dev_status);
+    } else {
+        e = prepare(key_side_tc_kernel<false, true>, kSmemKeySide);
+        if (e != cudaSuccess) return e;
+        key_side_tc_kernel<false, true><<<grid, kThreads, kSmemKeySide, st>>>(mv, muq, muk, mg, mo, a, strong_flag, dev_status);
+    }
     return cudaGetLastError();
 }
 

@@ -61,19 +61,6 @@ struct LeanCtl {
         if (!ctl->abort && !mbar_wait(bar, parity)) ctl->abort = 1;         \
     } while (0)
 
-__device__ __forceinline__ bool compute_sync_or(bool pred) {
-    uint32_t out;
-    asm volatile(
-        "{\n\t.reg .pred p, q;\n\t"
-        "setp.ne.b32 q, %1, 0;\n\t"
-        "bar.red.or.pred p, 1, 256, q;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(out)
-        : "r"((uint32_t)pred)
-        : "memory");
-    return out != 0;
-}
-
 __device__ __forceinline__ void lean_ctl_init(LeanCtl* ctl, int tid, int warp) {
     if (tid == 0) {
         mbar_init(&ctl->bar_x, 1);
@@ -116,23 +103,6 @@ __device__ __forceinline__ void lean_finish(Ctl* ctl, int tid, int warp, uint32_
         __syncwarp();
         tmem_dealloc(tmem, kTmemCols);
     }
-}
-
-// rows published and consumed: shared-memory writes to the async proxy, accumulator reads
-// ordered before the barrier, then one arrival for the issuing lane
-__device__ __forceinline__ void publish(uint64_t* bar, int tid) {
-    fence_async_smem();
-    tc_fence_before_sync();
-    compute_sync();
-    if (tid == 0) mbar_arrive(bar);
-}
-// the same at the end of a chunk, with the vote on leaving the loop
-__device__ __forceinline__ bool publish_and_vote(uint64_t* bar, int tid, bool stop) {
-    fence_async_smem();
-    tc_fence_before_sync();
-    const bool any = compute_sync_or(stop);
-    if (tid == 0) mbar_arrive(bar);
-    return any;
 }
 
 // accumulator columns of the lean kernels

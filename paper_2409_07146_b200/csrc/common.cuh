@@ -138,6 +138,9 @@ struct PendingDecay {
     const float* G;
     const int* strong;
     int T, H, nseg;
+    // != 0: the slot kernel serves ONLY the pairs flagged in `strong` (the fused chunk kernel has done
+    // the others on chip): rows with a pending factor are skipped
+    int strong_only;
     // row r = t * H + h of batch element b of a [B,T,H,M] tensor (32-bit arithmetic: T * H < 2^31)
     __host__ __device__ bool pending(int b, int r) const {
         if (G == nullptr) return false;
@@ -201,6 +204,26 @@ cudaError_t launch_value_side_lean(const ValueSideArgs& a, int reverse, const in
                                    int32_t* dev_status);
 cudaError_t launch_key_side_lean(const KeySideArgs& a, int reverse, const int* strong_flag, cudaStream_t st,
                                  int32_t* dev_status);
+// only the general kernel of a scan (the flagged pairs), on the given stream
+cudaError_t launch_value_side_general(const ValueSideArgs& a, int M, int reverse, const int* strong_flag,
+                                      cudaStream_t st, int32_t* dev_status);
+cudaError_t launch_key_side_general(const KeySideArgs& a, int M, int reverse, const int* strong_flag,
+                                    cudaStream_t st, int32_t* dev_status);
+// the side stream of the calling host thread on the current device, with its fork / join events
+struct SideLane {
+    cudaStream_t stream = nullptr;
+    cudaEvent_t fork = nullptr, join = nullptr;
+};
+cudaError_t side_lane(SideLane** out);
+// Fused chunk kernel: value_side scan -> slot non-linearity -> key_side scan in one kernel, for the
+// (batch, head) pairs without a strong-decay chunk (chunk_tc_fused.cu).
+//   mode 0 (forward):  xq1 = q,  xk1 = k, xv = v, out = o;   ok (nullable) receives the scaled logits
+//   mode 1 (backward): xq1 = dO, xk1 = v, xv = k, out = dq;  ok holds the scaled logits; u, Pd, Zd are written
+bool fused_pair_supported(int d_k, int d_v, int M);
+cudaError_t launch_fused_pair(int mode, const void* xq1, const void* xk1, const void* wd, const void* xv, void* out,
+                              const float* G, const float* S1_0, const float* S2_0, float* S1_end, float* S2_end, int B,
+                              int T, int H, int D1, int D2, float scale, int act, float* ok, float* u, void* Pd,
+                              void* Zd, const int* strong_flag, cudaStream_t st, int32_t* dev_status);
 cudaError_t launch_decode(const gsa_params_t& p, const void* q, const void* k, const void* v,
                           const float* gate, float* Ks, float* Vs, void* o, cudaStream_t st);
 

@@ -169,6 +169,9 @@ __global__ void __launch_bounds__(256) slot_softmax_fwd_kernel(const float* __re
     const size_t total = (size_t)gridDim.y * rows_per_batch * M;
     const size_t idx = row * M + l * R;
     const bool pending = pend.pending(b, rr);
+    // serving the flagged pairs only: a warp none of whose rows is flagged has nothing to do
+    const bool skip = pend.strong_only != 0 && pending;
+    if (__all_sync(0xffffffffu, skip)) return;
     float z[R], eg[R];
 #pragma unroll
     for (int r = 0; r < R; ++r) { z[r] = 0.f; eg[r] = 1.f; }
@@ -205,7 +208,7 @@ __global__ void __launch_bounds__(256) slot_softmax_fwd_kernel(const float* __re
 #pragma unroll
         for (int r = 0; r < R; ++r) e[r] = slot_act_value(z[r], act);
     }
-    if (!live) return;
+    if (!live || skip) return;
     st_vec(ok + idx, z);
     // fp32 p is read by the general chunk kernels and the CUDA-core kernels only: rows of a pair
     // that the pipelined kernels serve (pending) get the decayed bf16 rows alone
@@ -257,6 +260,8 @@ __global__ void __launch_bounds__(256) slot_softmax_bwd_kernel(const float* __re
     const size_t total = (size_t)gridDim.y * rows_per_batch * M;
     const size_t idx = row * M + l * R;
     const bool pending = pend.pending(b, rr);
+    const bool skip = pend.strong_only != 0 && pending;      // (as in the forward kernel)
+    if (__all_sync(0xffffffffu, skip)) return;
     float z[R], dpv[R], eg[R];
     ld_vec(ok + idx, z);
 #pragma unroll
@@ -306,7 +311,7 @@ __global__ void __launch_bounds__(256) slot_softmax_bwd_kernel(const float* __re
             uv[r] = e[r] * dpv[r] + z[r] * dok;
         }
     }
-    if (!live) return;
+    if (!live || skip) return;
     if (!pending) {       // (as in the forward: fp32 p and dz only where a non-pipelined kernel reads them)
         st_vec(p + idx, e);
         st_vec(dz + idx, dzv);
