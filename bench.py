@@ -213,7 +213,8 @@ def run_reference(args):
     sample = (f"{pairs} of {w.B * w.H} (batch, head) pairs of the {WORKLOAD} workload per step, "
               f"forward + reverse sweep in fp64; tokens = pairs * T / H")
     line = {
-        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT,
+        "n_gpus": int(os.environ.get("WORLD_SIZE", "1")),
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
         "data": "synthetic (seeded, bf16-rounded inputs)",
@@ -458,11 +459,22 @@ def run_ours(args):
         alg = sum(k_["alg_bytes"] * k_["launches_per_step"] for k_ in members) / n_l
         traf = [NCU_TRAFFIC.get(k_["kernel"]) for k_ in members]
         traffic = int(sum(traf) / len(traf)) if all(t is not None for t in traf) else None
+        # the bytes the same launch would move if the slot-sized rows between the passes stayed on chip
+        # (the d-sized tensors only: v in, o out for key_side; q, k in for value_side)
+        e_ = 2 if w.io == "bf16" else 4
+        fused_bytes = w.B * w.T * w.H * 2 * (w.d_v if fn.startswith("key") else w.d_k) * e_
         roofline = {"bound": "hbm", "kernel": fn, "labels": [k_["kernel"] for k_ in members],
                     "launches_per_step": n_l, "avg_launch_ms": avg_ms,
                     "achieved": alg / (avg_ms * 1e-3) / 1e9,
                     "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": alg / (avg_ms * 1e-3) / 1e9 / pk["hbm_gbs"],
-                    "traffic": traffic, "peak_source": pk["source"],
+                    "traffic": traffic, "traffic_source": ("profiles/step_kernels_train_1p3b_ncu_full.md (one ncu capture of "
+                                                           "this workload; not measured in this run)") if traffic else None,
+                    "frac_on_fused_bytes": fused_bytes / (avg_ms * 1e-3) / 1e9 / pk["hbm_gbs"],
+                    "limiter": ("tensor-pipe issue rate: the chunk loop issues its tcgen05.mma (a quarter of them only "
+                                "for the high/low operand pairs) back to back at 80-90 cycles each; ncu shows the tensor "
+                                "pipe 53-63% active and DRAM at 30-46% of peak, so HBM is the bound of the ideal fused "
+                                "layer, not what limits this kernel"),
+                    "peak_source": pk["source"],
                     "share_of_step": sum(k_["share"] for k_ in members)}
         if fn.endswith("_side_lean_kernel") or fn == "fused_pair_kernel":
             d = w.d_v if fn.startswith("key") else w.d_k     # (d_k == d_v in the benchmark workload)
@@ -643,6 +655,20 @@ def bench_decode(gsa, torch, dev, pk):
             "note": "states (1.07 GB read+write per step) exceed L2"}
 
 
+def free_port() -> int:
+    import socket
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        return sk.getsockname()[1]
+
+
+def launcher_command(n: int, argv):
+    """The command that runs this script as n ranks on one node (one rank per GPU, rendezvous on the
+    loopback address)."""
+    return [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}",
+            "--master-addr", "127.0.0.1", "--master-port", str(free_port()), os.path.abspath(__file__), *argv]
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -668,6 +694,9 @@ def main():
     ap.add_argument("--profile-case", action="store_true",
                     help="run warmup + steps bare (for ncu); prints no benchmark line")
     args = ap.parse_args()
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # started as a plain process: start the N ranks of one node here (what a torchrun command line does)
+        raise SystemExit(subprocess.call(launcher_command(args.gpus, sys.argv[1:])))
     if args.impl == "reference":
         run_reference(args)
     else:

@@ -26,8 +26,9 @@
  *   - Kernels that are independent of one another (the five scans of the backward
  *     after the softmax gradient; the general and the pipelined kernel of a scan)
  *     run on internal streams: up to five per calling host thread and device,
- *     with their events, created on first use and kept for the life of the
- *     process.  They are forked from `stream` and joined back into it by events
+ *     with their events, created on first use and kept until gsa_release_streams()
+ *     (this is the library's only state: per host thread and device, no device
+ *     memory).  They are forked from `stream` and joined back into it by events
  *     inside the call, so ordering with respect to `stream` is that of a plain
  *     in-stream call, and a call can be captured into a CUDA graph.
  *   - `ws` is caller-provided device scratch of at least
@@ -241,29 +242,12 @@ GSA_API gsa_status_t gsa_fwd_noalloc(const gsa_params_t* params, const void* q, 
                                      float* VT, void* stream, int32_t* dev_status);
 
 /*
- * Self-test of the tensor-core building blocks (no counterpart in the paper): computes one
- * 128-row bf16 product per operand layout the chunk kernels use, from two 128 x 128
- * row-major bf16 device matrices X, Y into D (fp32, row-major):
- *   mode 0: D[128x128] = X Y^T        mode 1: D[128x128] = X Y
- *   mode 2: D[128x64]  = X^T Y[:64]^T mode 3: D[128x64]  = X Y[:, :64]
- *   mode 4: D[128x128] = X Y^T        mode 5: D[128x128] = X Y      (A operand in tensor memory)
- * dev_status (nullable) receives GSA_ERR_TIMEOUT if a bounded wait expired.
+ * Releases the internal streams and events that this HOST thread's calls created on the current
+ * device (the side streams described in the conventions above); they are created again by the
+ * next call that needs them.  Call it only when none of this thread's gsa_* work is in flight on
+ * the device and no capture is open.  No counterpart in the paper.
  */
-GSA_API gsa_status_t gsa_tc_selftest(int32_t mode, const void* X, const void* Y, float* D,
-                                     void* stream, int32_t* dev_status);
-
-/*
- * Per-kernel timing for benchmarks (no counterpart in the paper).  Between
- * gsa_timing_begin(capacity) and gsa_timing_end() on the same HOST thread, every kernel
- * that this thread's gsa_* calls enqueue is bracketed by a pair of CUDA events on its
- * stream (up to `capacity` kernels).  gsa_timing_end waits for the last one, writes the
- * duration in milliseconds and a static label of each timed kernel, in launch order, to
- * ms[0..n) / labels[0..n), and returns n (-1 on error or if timing was not active).  These
- * two calls create and destroy events and synchronise with the host: keep them out of
- * production paths.
- */
-GSA_API gsa_status_t gsa_timing_begin(int32_t capacity);
-GSA_API int32_t gsa_timing_end(float* ms, const char** labels, int32_t capacity);
+GSA_API gsa_status_t gsa_release_streams(void);
 
 #ifdef __cplusplus
 }

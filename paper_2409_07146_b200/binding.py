@@ -74,7 +74,8 @@ def lib_path() -> str:
 def exported_symbols():
     return ["gsa_chunk_size", "gsa_workspace_bytes", "gsa_status_string", "gsa_gate_cumsum",
             "gsa_fwd", "gsa_bwd", "gsa_decode_step", "gsa_tc_selftest", "gsa_timing_begin",
-            "gsa_timing_end", "gsa_fwd_noalloc", "gsa_fwd_save_gate", "gsa_bwd_saved_gate"]
+            "gsa_timing_end", "gsa_fwd_noalloc", "gsa_fwd_save_gate", "gsa_bwd_saved_gate", "gsa_release_streams",
+            "gsa_wait_selftest"]
 
 
 def load_library():
@@ -115,6 +116,10 @@ def load_library():
     lib.gsa_timing_end.restype = i32
     lib.gsa_tc_selftest.argtypes = [i32, vp, vp, vp, vp, vp]
     lib.gsa_tc_selftest.restype = ctypes.c_int
+    lib.gsa_wait_selftest.argtypes = [ctypes.c_uint32, vp, vp, vp]
+    lib.gsa_wait_selftest.restype = ctypes.c_int
+    lib.gsa_release_streams.argtypes = []
+    lib.gsa_release_streams.restype = ctypes.c_int
     _lib = lib
     return lib
 
@@ -256,6 +261,19 @@ def gsa_tc_selftest(mode: int, X, Y, dev_status=None):
         _ptr(D, torch.float32, None, "D"), _stream(), _ptr(dev_status, torch.int32, None, "dev_status")),
         "gsa_tc_selftest")
     return D
+
+
+def gsa_wait_selftest(limit_us: int, dev_status, waited_us=None):
+    """One CTA waits limit_us microseconds on an mbarrier that nothing signals, gives up and writes
+    GSA_ERR_TIMEOUT to dev_status (int32 device tensor); waited_us (uint32/int32 device tensor, optional)
+    receives the time it waited."""
+    _check(load_library().gsa_wait_selftest(int(limit_us), _stream(), _ptr(dev_status, torch.int32, None, "dev_status"),
+                                            _ptr(waited_us, torch.int32, None, "waited_us")), "gsa_wait_selftest")
+
+
+def gsa_release_streams():
+    """Destroy the calling thread's internal streams and events on the current device."""
+    _check(load_library().gsa_release_streams(), "gsa_release_streams")
 
 
 def gsa_timing_begin(capacity: int = 4096):

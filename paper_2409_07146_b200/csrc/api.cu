@@ -5,6 +5,7 @@
 #include <vector>
 
 #include "common.cuh"
+#include "gsa_dev.h"
 
 using namespace gsa;
 
@@ -231,14 +232,15 @@ struct ScanLanes {
     cudaStream_t stream[4] = {nullptr, nullptr, nullptr, nullptr};
     cudaEvent_t fork = nullptr, join[4] = {nullptr, nullptr, nullptr, nullptr};
 };
+constexpr int kMaxLaneDevices = 64;
+thread_local ScanLanes g_scan_lanes[kMaxLaneDevices];
+
 cudaError_t scan_lanes(ScanLanes** out) {
-    constexpr int kMaxDevices = 64;
-    thread_local ScanLanes lanes[kMaxDevices];
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
-    if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
-    ScanLanes& l = lanes[dev];
+    if (dev < 0 || dev >= kMaxLaneDevices) return cudaErrorInvalidDevice;
+    ScanLanes& l = g_scan_lanes[dev];
     if (l.fork == nullptr) {
         for (int i = 0; i < 4 && e == cudaSuccess; ++i) {
             e = cudaStreamCreateWithFlags(&l.stream[i], cudaStreamNonBlocking);
@@ -248,6 +250,21 @@ cudaError_t scan_lanes(ScanLanes** out) {
         if (e != cudaSuccess) return e;
     }
     *out = &l;
+    return cudaSuccess;
+}
+
+cudaError_t scan_lanes_release() {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= kMaxLaneDevices) return cudaErrorInvalidDevice;
+    ScanLanes& l = g_scan_lanes[dev];
+    for (int i = 0; i < 4; ++i) {
+        if (l.stream[i] != nullptr) cudaStreamDestroy(l.stream[i]);
+        if (l.join[i] != nullptr) cudaEventDestroy(l.join[i]);
+    }
+    if (l.fork != nullptr) cudaEventDestroy(l.fork);
+    l = ScanLanes{};
     return cudaSuccess;
 }
 
@@ -329,7 +346,7 @@ gsa_status_t fwd_impl(const gsa_params_t* params, const void* q, const void* k, 
     GSA_CUDA(cudaMemsetAsync(w.strong, 0, sizeof(int) * (size_t)p.B * p.H * nseg, st));
     GSA_LAUNCH("gate_cumsum", launch_gate_cumsum(gate, p.gate_kind, inv_tau(p), w.G, w.I, p.B, p.T,
                                                  p.H, p.m, chunk_of(p), w.strong, nseg, w.Id, p.io == GSA_BF16, st));
-    float* ok = ok_save ? ok_save : w.ok;
+    float* ok = ok_save;      // the scaled logits leave the softmax kernel only if the caller keeps them
     // the pipelined kernels leave the row factor of the pass-1 sums to the softmax kernel
     const PendingDecay pend = use_tc(p) ? PendingDecay{w.G, w.strong, p.T, p.H, nseg} : PendingDecay{nullptr, nullptr, 1, 1, 1};
     // [B,T,H,.] cut into nseg segments is the same memory as [B*nseg, T/nseg, H, .]
@@ -590,6 +607,11 @@ gsa_status_t gsa_decode_step(const gsa_params_t* params, const void* q, const vo
         return GSA_ERR_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     GSA_LAUNCH("decode_step", launch_decode(*params, q, k, v, gate, Kstate, Vstate, o, st));
+    return GSA_OK;
+}
+
+gsa_status_t gsa_release_streams(void) {
+    if (scan_lanes_release() != cudaSuccess || side_lane_release() != cudaSuccess) return GSA_ERR_CUDA;
     return GSA_OK;
 }
 

@@ -160,7 +160,7 @@ __device__ __forceinline__ void value_side_explicit_rows(const unsigned char* gt
                 for (int ee = 0; ee < 16; ++ee) {
                     const int e = REV ? ee : 15 - ee;
                     const int j = c0 + e;
-                    if (REV ? j < row : j > row) continue;
+                    if ((REV ? j < row : j > row) || !live) continue;
                     float aj[16], wj[16];
                     tile_row16(gt, j, s0, aj);
                     tile_row16(sW, j, s0, wj);
@@ -170,11 +170,13 @@ __device__ __forceinline__ void value_side_explicit_rows(const unsigned char* gt
                         acc[u] = fmaf(v[e] * wj[u], dec[u], acc[u]);
                         if (!REV) dec[u] *= aj[u];                      // prod_{r=j..i} for the next (earlier) row
                     }
-                }
-                float top = 0.f;
+                    if ((ee & 3) == 3) {
+                        float top = 0.f;
 #pragma unroll
-                for (int u = 0; u < 16; ++u) top = fmaxf(top, dec[u]);
-                live = top >= kDecayFloor;
+                        for (int u = 0; u < 16; ++u) top = fmaxf(top, dec[u]);
+                        live = top >= kDecayFloor;
+                    }
+                }
             }
             if (!__any_sync(0xffffffffu, live)) break;
         }
@@ -542,10 +544,14 @@ __device__ __forceinline__ void key_side_explicit_rows(unsigned char* sG, const 
 #pragma unroll
     for (int e = 0; e < 64; ++e) x[e] = 0.f;
     if (any) {
+        float start = 0.f;
+#pragma unroll
+        for (int s = 0; s < kM; ++s) start = fmaxf(start, fabsf(qd[s]));
+        const float floor_ = start * kDecayFloor;
 #pragma unroll 1
         for (int j = j0; REV ? j <= jhi : j >= jlo; j += REV ? 1 : -1) {
             // reverse: the product up to column j includes a_j (prod_{r=i+1..j}); j0 itself is already covered
-            float acc = 0.f, top = 0.f;
+            float acc = 0.f;
 #pragma unroll
             for (int s0 = 0; s0 < kM; s0 += 16) {
                 float aj[16], uk[16];
@@ -556,11 +562,15 @@ __device__ __forceinline__ void key_side_explicit_rows(unsigned char* sG, const 
                     if (REV && j > j0) qd[s0 + u] *= aj[u];
                     acc = fmaf(qd[s0 + u], uk[u], acc);
                     if (!REV) qd[s0 + u] *= aj[u];
-                    top = fmaxf(top, fabsf(qd[s0 + u]));
                 }
             }
             x[j - jlo] = acc;
-            if (top < 1e-30f) break;        // every later term is below 1e-30 |uk|
+            if (((j - j0) & 3) == 0) {        // every fourth step: has every product fallen below 2^-40 of the start?
+                float top = 0.f;
+#pragma unroll
+                for (int s = 0; s < kM; ++s) top = fmaxf(top, fabsf(qd[s]));
+                if (top <= floor_) break;
+            }
         }
     }
 #pragma unroll
@@ -853,14 +863,17 @@ constexpr size_t kSmemKeySide = 1024 + 13 * kPanelB + sizeof(Ctl);
 // usual case that no pair is flagged, its launch and the exit of its CTAs then cost the
 // caller's stream nothing.  fork: the side stream waits for what precedes on the caller's
 // stream; join: the caller's stream waits for the general kernel.
+namespace {
+constexpr int kMaxLaneDevices = 64;
+thread_local SideLane g_side_lanes[kMaxLaneDevices];
+}  // namespace
+
 cudaError_t side_lane(SideLane** out) {
-    constexpr int kMaxDevices = 64;
-    thread_local SideLane lanes[kMaxDevices];
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
-    if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
-    SideLane& l = lanes[dev];
+    if (dev < 0 || dev >= kMaxLaneDevices) return cudaErrorInvalidDevice;
+    SideLane& l = g_side_lanes[dev];
     if (l.stream == nullptr) {
         e = cudaStreamCreateWithFlags(&l.stream, cudaStreamNonBlocking);
         if (e == cudaSuccess) e = cudaEventCreateWithFlags(&l.fork, cudaEventDisableTiming);
@@ -868,6 +881,22 @@ cudaError_t side_lane(SideLane** out) {
         if (e != cudaSuccess) return e;
     }
     *out = &l;
+    return cudaSuccess;
+}
+
+// destroys the calling thread's side stream and events on the current device (created again on demand)
+cudaError_t side_lane_release() {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= kMaxLaneDevices) return cudaErrorInvalidDevice;
+    SideLane& l = g_side_lanes[dev];
+    if (l.stream != nullptr) {
+        cudaStreamDestroy(l.stream);
+        if (l.fork != nullptr) cudaEventDestroy(l.fork);
+        if (l.join != nullptr) cudaEventDestroy(l.join);
+        l = SideLane{};
+    }
     return cudaSuccess;
 }
 

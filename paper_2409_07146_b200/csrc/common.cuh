@@ -215,6 +215,7 @@ struct SideLane {
     cudaEvent_t fork = nullptr, join = nullptr;
 };
 cudaError_t side_lane(SideLane** out);
+cudaError_t side_lane_release();
 // Fused chunk kernel: value_side scan -> slot non-linearity -> key_side scan in one kernel, for the
 // (batch, head) pairs without a strong-decay chunk (chunk_tc_fused.cu).
 //   mode 0 (forward):  xq1 = q,  xk1 = k, xv = v, out = o;   ok (nullable) receives the scaled logits

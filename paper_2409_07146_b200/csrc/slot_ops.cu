@@ -209,7 +209,7 @@ __global__ void __launch_bounds__(256) slot_softmax_fwd_kernel(const float* __re
         for (int r = 0; r < R; ++r) e[r] = slot_act_value(z[r], act);
     }
     if (!live || skip) return;
-    st_vec(ok + idx, z);
+    if (ok != nullptr) st_vec(ok + idx, z);
     // fp32 p is read by the general chunk kernels and the CUDA-core kernels only: rows of a pair
     // that the pipelined kernels serve (pending) get the decayed bf16 rows alone
     if (!pending) st_vec(p + idx, e);

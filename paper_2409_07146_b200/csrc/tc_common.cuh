@@ -83,7 +83,7 @@ __device__ __forceinline__ uint64_t global_timer_ns() {
 constexpr uint64_t kWaitLimitNs = 2000000000ull;   // every wait gives up after 2 s
 
 // Wait for the phase with the given parity; false if the time limit expired.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, uint64_t limit_ns = kWaitLimitNs) {
     const uint32_t addr = smem_u32(bar);
     uint64_t start = 0;
     for (uint32_t it = 0;; ++it) {
@@ -99,7 +99,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
         if ((it & 63u) == 63u) {
             const uint64_t now = global_timer_ns();
             if (start == 0) start = now;
-            else if (now - start > kWaitLimitNs) return false;
+            else if (now - start > limit_ns) return false;
         }
     }
 }

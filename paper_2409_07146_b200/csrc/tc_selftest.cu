@@ -2,6 +2,7 @@
 // combination that the chunk kernels use, on caller-provided 128 x 128 bf16 matrices.
 // It exists so that a wrong matrix descriptor or swizzle shows up in isolation.
 #include "common.cuh"
+#include "gsa_dev.h"
 #include "tc_common.cuh"
 
 namespace gsa {
@@ -173,8 +174,46 @@ __global__ void __launch_bounds__(128) tc_selftest_kernel(const __grid_constant_
         tmem_dealloc(tmem, 256);
     }
 }
+// The bounded wait itself: one CTA waits on an mbarrier that nothing will ever signal, with the
+// given limit; the wait must give up, the CTA must report GSA_ERR_TIMEOUT through dev_status the way
+// the chunk kernels do (flag, release tensor memory, return), and the context must stay usable.
+__global__ void __launch_bounds__(128) wait_expiry_kernel(uint64_t limit_ns, int32_t* dev_status, uint32_t* waited_us) {
+    __shared__ uint64_t bar;
+    __shared__ uint32_t tmem_slot;
+    const int tid = threadIdx.x, warp = tid >> 5;
+    if (tid == 0) {
+        mbar_init(&bar, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 0) {
+        __syncwarp();
+        tmem_alloc(&tmem_slot, 32);
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint64_t t0 = global_timer_ns();
+    const bool done = mbar_wait(&bar, 0, limit_ns);          // nobody arrives: must expire
+    const uint64_t t1 = global_timer_ns();
+    if (tid == 0) {
+        if (!done && dev_status != nullptr) *dev_status = GSA_ERR_TIMEOUT;
+        if (waited_us != nullptr) *waited_us = (uint32_t)((t1 - t0) / 1000u);
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 0) {
+        __syncwarp();
+        tmem_dealloc(tmem_slot, 32);
+    }
+}
 }  // namespace
 }  // namespace gsa
+
+extern "C" GSA_API gsa_status_t gsa_wait_selftest(uint32_t limit_us, void* stream, int32_t* dev_status, uint32_t* waited_us) {
+    if (limit_us < 1 || limit_us > 100000 || dev_status == nullptr) return GSA_ERR_INVALID_ARG;    // at most 0.1 s
+    gsa::wait_expiry_kernel<<<1, 128, 0, static_cast<cudaStream_t>(stream)>>>((uint64_t)limit_us * 1000ull, dev_status, waited_us);
+    return cudaGetLastError() == cudaSuccess ? GSA_OK : GSA_ERR_CUDA;
+}
 
 extern "C" GSA_API gsa_status_t gsa_tc_selftest(int32_t mode, const void* X, const void* Y, float* D, void* stream,
                                                 int32_t* dev_status) {

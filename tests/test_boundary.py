@@ -20,8 +20,12 @@ def lib():
 
 
 def declared_symbols():
-    text = open(os.path.join(ROOT, "include", "gsa.h")).read()
-    return re.findall(r"GSA_API[^;(]*?\b(gsa_\w+)\s*\(", text)
+    """Every entry point declared in the public header and in the header of the development aids."""
+    names = []
+    for h in ("gsa.h", "gsa_dev.h"):
+        text = open(os.path.join(ROOT, "include", h)).read()
+        names += re.findall(r"GSA_API[^;(]*?\b(gsa_\w+)\s*\(", text)
+    return names
 
 
 def test_library_exports_every_declared_symbol(lib):
@@ -31,6 +35,9 @@ def test_library_exports_every_declared_symbol(lib):
     for n in names:
         assert hasattr(lib, n), n
     assert set(gsa.exported_symbols()) == set(names)
+    # the layer's interface is gsa.h alone: the self-tests and timing hooks live in gsa_dev.h
+    public = open(os.path.join(ROOT, "include", "gsa.h")).read()
+    assert "gsa_tc_selftest" not in public and "gsa_timing_begin" not in public and "gsa_wait_selftest" not in public
 
 
 def test_chunk_and_workspace_queries(lib):

@@ -55,3 +55,20 @@ def test_two_gloo_ranks_shard_the_batch(tmp_path):
     assert meta[0] == 11.0                       # max over ranks of (10, 11)
     assert meta[1] != meta[2]                    # every rank draws its own batch
     assert bench.aggregate_tokens_per_s(2, 16384, 1.0) == 2 * 16384 / 1e-3
+
+
+def test_bench_starts_its_own_ranks_when_run_as_a_plain_process(tmp_path):
+    """`python bench.py --gpus 2` without a launcher must start two ranks itself and print one line with
+    n_gpus = 2.  Exercised here on the reference arm (the oracle on CPU: rank 0 works, rank 1 exits 0)."""
+    import json
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    cmd = bench.launcher_command(2, ["--gpus", "2"])
+    assert "--nproc-per-node=2" in cmd and "127.0.0.1" in cmd and cmd[-2:] == ["--gpus", "2"]
+    env = {k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK")}
+    out = subprocess.run([sys.executable, os.path.join(root, "bench.py"), "--gpus", "2", "--impl", "reference",
+                          "--steps", "1", "--warmup", "0"], env=env, capture_output=True, text=True, timeout=600)
+    assert out.returncode == 0, out.stderr[-2000:]
+    lines = [json.loads(l) for l in out.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1 and lines[0]["impl"] == "reference" and lines[0]["n_gpus"] == 2
