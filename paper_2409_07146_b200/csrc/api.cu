@@ -18,6 +18,8 @@ bool dim_ok(int d) { return d == 64 || d == 128 || d == 256 || d == 512; }
 
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
+constexpr int kPaddedSlots = 64;      // slot width of the tensor-core tiles (see pads_slots)
+
 gsa_status_t check_params(const gsa_params_t* p, bool need_T) {
     if (p == nullptr) return GSA_ERR_INVALID_ARG;
     if (p->B < 1 || p->H < 1 || p->d_k < 1 || p->d_v < 1 || p->m < 1) return GSA_ERR_INVALID_ARG;
@@ -37,7 +39,7 @@ gsa_status_t check_params(const gsa_params_t* p, bool need_T) {
     if ((long long)p->B * p->H > 0x7fffffffLL / 4) return GSA_ERR_UNSUPPORTED;
     if (p->impl == GSA_IMPL_TC && p->io != GSA_BF16) return GSA_ERR_UNSUPPORTED;
     // the tensor-core kernels asked for by name: no silent fall-back to the CUDA-core kernels
-    if (p->impl == GSA_IMPL_TC && !tc_supported(p->d_k, p->d_v, p->m)) return GSA_ERR_UNSUPPORTED;
+    if (p->impl == GSA_IMPL_TC && !tc_supported(p->d_k, p->d_v, p->m == 32 ? kPaddedSlots : p->m)) return GSA_ERR_UNSUPPORTED;
     return GSA_OK;
 }
 
@@ -45,6 +47,19 @@ gsa_status_t check_params(const gsa_params_t* p, bool need_T) {
 bool use_tc(const gsa_params_t& p) {
     if (p.impl == GSA_IMPL_SIMT) return false;
     return p.io == GSA_BF16 && tc_supported(p.d_k, p.d_v, p.m);
+}
+
+// A bf16 layer with 32 slots runs on the tensor-core kernels too: their tiles are 64 slots wide, so the
+// call is carried out with 64 slots of which the last 32 are padding -- a gate that keeps everything
+// and writes nothing (a = 1), empty memory rows, and a non-linearity that leaves the padding out.
+// The gate, the logits, the memories and their gradients are widened / narrowed at the boundary.
+bool pads_slots(const gsa_params_t& p) {
+    return p.impl != GSA_IMPL_SIMT && p.io == GSA_BF16 && p.m == 32 && tc_supported(p.d_k, p.d_v, kPaddedSlots);
+}
+gsa_params_t internal_params(const gsa_params_t& p) {
+    gsa_params_t q = p;
+    if (pads_slots(p)) q.m = kPaddedSlots;
+    return q;
 }
 
 // Does this call run the slot non-linearity inside the fused chunk kernel?  (The operand pairs are
@@ -71,7 +86,7 @@ Slices slices(const gsa_params_t& p) {
 int segments_of(const gsa_params_t& p) {
     if (!use_tc(p)) return 1;
     const int chunk = tc_chunk();
-    const long long ctas = (long long)p.B * p.H * (p.d_k < p.d_v ? p.d_k : p.d_v) / 128;
+    const long long ctas = (long long)p.B * p.H * tc_value_side_slices(p.d_k < p.d_v ? p.d_k : p.d_v);
     int nseg = 1;
     while (ctas * nseg * 2 <= 160 && p.T % (nseg * 2 * chunk) == 0 && p.T / (nseg * 2) >= 8 * chunk) nseg *= 2;
     return nseg;
@@ -268,6 +283,32 @@ cudaError_t scan_lanes_release() {
     return cudaSuccess;
 }
 
+// Buffers of the padded-slot mode, carved from the tail of the workspace (after the internal one).
+struct PadBuffers {
+    float *gate, *ok, *dgate;                    // [B,T,H,64]
+    float *K0, *V0, *KT, *VT;                    // [B,H,64,d]   (backward: K0, V0, dKT, dVT in; KT = dK0, VT = dV0 out)
+    float *dKT, *dVT;
+    size_t bytes;
+};
+PadBuffers carve_pad(const gsa_params_t& p, int which, void* base) {
+    PadBuffers b;
+    memset(&b, 0, sizeof(b));
+    if (!pads_slots(p)) return b;
+    const size_t mt = (size_t)p.B * p.T * p.H * kPaddedSlots;
+    const size_t sk = (size_t)p.B * p.H * kPaddedSlots * p.d_k, sv = (size_t)p.B * p.H * kPaddedSlots * p.d_v;
+    Carver c{static_cast<char*>(base), 0};
+    b.gate = c.take(mt);
+    b.ok = c.take(mt);
+    b.K0 = c.take(sk); b.V0 = c.take(sv); b.KT = c.take(sk); b.VT = c.take(sv);
+    if (which == GSA_WS_BWD) {
+        b.dgate = c.take(mt);
+        b.dKT = c.take(sk); b.dVT = c.take(sv);
+    }
+    b.bytes = c.off;
+    return b;
+}
+size_t pad_bytes(const gsa_params_t& p, int which) { return carve_pad(p, which, nullptr).bytes; }
+
 #define GSA_CUDA(expr)                                  \
     do {                                                \
         cudaError_t e__ = (expr);                       \
@@ -288,7 +329,7 @@ extern "C" {
 
 int32_t gsa_chunk_size(const gsa_params_t* params) {
     if (check_params(params, false) != GSA_OK) return 0;
-    return chunk_of(*params);
+    return chunk_of(internal_params(*params));
 }
 
 const char* gsa_status_string(gsa_status_t status) {
@@ -307,8 +348,9 @@ size_t gsa_workspace_bytes(const gsa_params_t* params, int32_t which) {
     if (which == GSA_WS_DECODE) return 0;
     if (which != GSA_WS_FWD && which != GSA_WS_BWD && which != GSA_WS_GATE) return 0;
     if (check_params(params, true) != GSA_OK) return 0;
-    if (which == GSA_WS_GATE) return carve_gate(*params, nullptr).bytes;
-    return carve(*params, which, nullptr).bytes;
+    const gsa_params_t pi = internal_params(*params);
+    if (which == GSA_WS_GATE) return carve_gate(pi, nullptr).bytes;
+    return carve(pi, which, nullptr).bytes + pad_bytes(*params, which);
 }
 
 gsa_status_t gsa_gate_cumsum(const gsa_params_t* params, const float* gate, float* G, float* I,
@@ -319,20 +361,15 @@ gsa_status_t gsa_gate_cumsum(const gsa_params_t* params, const float* gate, floa
     const gsa_params_t& p = *params;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     GSA_LAUNCH("gate_cumsum", launch_gate_cumsum(gate, p.gate_kind, inv_tau(p), G, I, p.B, p.T,
-                                                 p.H, p.m, chunk_of(p), nullptr, 1, nullptr, 0, st));
+                                                 p.H, p.m, chunk_of(internal_params(p)), nullptr, 1, nullptr, 0, st));
     return GSA_OK;
 }
 
 namespace {
-gsa_status_t fwd_impl(const gsa_params_t* params, const void* q, const void* k, const void* v,
+gsa_status_t fwd_core(const gsa_params_t* params, int m_active, const void* q, const void* k, const void* v,
                       const float* gate, const float* K0, const float* V0, void* o,
                       float* ok_save, float* KT, float* VT, bool save_gate, void* gate_save, size_t gate_save_bytes,
                       void* ws, size_t ws_bytes, void* stream, int32_t* dev_status) {
-    gsa_status_t rc = check_params(params, true);
-    if (rc != GSA_OK) return rc;
-    if (!ok_ptr(q) || !ok_ptr(k) || !ok_ptr(v) || !ok_ptr(gate) || !ok_ptr(o)) return GSA_ERR_INVALID_ARG;
-    if (!ok_opt(K0) || !ok_opt(V0) || !ok_opt(ok_save) || !ok_opt(KT) || !ok_opt(VT))
-        return GSA_ERR_INVALID_ARG;
     const gsa_params_t& p = *params;
     if (ws == nullptr || (reinterpret_cast<uintptr_t>(ws) & 255u) != 0) return GSA_ERR_WORKSPACE;
     Workspace w = carve(p, GSA_WS_FWD, ws);
@@ -398,7 +435,7 @@ gsa_status_t fwd_impl(const gsa_params_t* params, const void* q, const void* k, 
                                                   p.d_v, p.scale, p.slot_act, ok_save, nullptr, nullptr, nullptr, w.strong,
                                                   st, dev_status));
         GSA_CUDA(launch_value_side_general(a1, p.m, 0, w.strong, ss, dev_status));
-        GSA_CUDA(launch_slot_softmax_fwd(w.okpart, s.k, p.scale, p.slot_act, ok, w.p, p.B, p.T * p.H, p.m, pend.G, w.Pd, only, ss));
+        GSA_CUDA(launch_slot_softmax_fwd(w.okpart, s.k, p.scale, p.slot_act, ok, w.p, p.B, p.T * p.H, p.m, pend.G, w.Pd, only, ss, m_active));
         GSA_CUDA(launch_key_side_general(a2, p.m, 0, w.strong, ss, dev_status));
         if (!g_sink.active) {
             GSA_CUDA(cudaEventRecord(side->join, ss));
@@ -408,8 +445,45 @@ gsa_status_t fwd_impl(const gsa_params_t* params, const void* q, const void* k, 
     }
     GSA_LAUNCH("pass1_value_side", value_side(p, a1, 0, w.strong, st, dev_status));
     GSA_LAUNCH("slot_softmax", launch_slot_softmax_fwd(w.okpart, s.k, p.scale, p.slot_act, ok, w.p, p.B, p.T * p.H, p.m, pend.G, w.Pd,
-                                                       pend, st));
+                                                       pend, st, m_active));
     GSA_LAUNCH("pass2_key_side", key_side(p, a2, 0, w.strong, st, dev_status));
+    return GSA_OK;
+}
+
+// Validation, and the padded-slot mode around the core (see pads_slots).
+gsa_status_t fwd_impl(const gsa_params_t* params, const void* q, const void* k, const void* v,
+                      const float* gate, const float* K0, const float* V0, void* o,
+                      float* ok_save, float* KT, float* VT, bool save_gate, void* gate_save, size_t gate_save_bytes,
+                      void* ws, size_t ws_bytes, void* stream, int32_t* dev_status) {
+    gsa_status_t rc = check_params(params, true);
+    if (rc != GSA_OK) return rc;
+    if (!ok_ptr(q) || !ok_ptr(k) || !ok_ptr(v) || !ok_ptr(gate) || !ok_ptr(o)) return GSA_ERR_INVALID_ARG;
+    if (!ok_opt(K0) || !ok_opt(V0) || !ok_opt(ok_save) || !ok_opt(KT) || !ok_opt(VT))
+        return GSA_ERR_INVALID_ARG;
+    if (!pads_slots(*params))
+        return fwd_core(params, 0, q, k, v, gate, K0, V0, o, ok_save, KT, VT, save_gate, gate_save, gate_save_bytes, ws,
+                        ws_bytes, stream, dev_status);
+    const gsa_params_t& p = *params;
+    const gsa_params_t pi = internal_params(p);
+    if (ws == nullptr || (reinterpret_cast<uintptr_t>(ws) & 255u) != 0) return GSA_ERR_WORKSPACE;
+    const size_t core = carve(pi, GSA_WS_FWD, nullptr).bytes;
+    const PadBuffers pb = carve_pad(p, GSA_WS_FWD, static_cast<char*>(ws) + core);
+    if (ws_bytes < core + pb.bytes) return GSA_ERR_WORKSPACE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const size_t rows = (size_t)p.B * p.T * p.H, pairs = (size_t)p.B * p.H;
+    const int M = kPaddedSlots;
+    // a neutral gate for the padding: a = 1 (log a = 0; a logit whose sigmoid is 1 to rounding)
+    const float neutral = p.gate_kind == GSA_GATE_A ? 1.f : (p.gate_kind == GSA_GATE_LOG_A ? 0.f : 80.f);
+    GSA_CUDA(launch_resize_rows(gate, pb.gate, rows, p.m, M, neutral, st));
+    if (K0) GSA_CUDA(launch_resize_rows(K0, pb.K0, pairs, p.m * p.d_k, M * p.d_k, 0.f, st));
+    if (V0) GSA_CUDA(launch_resize_rows(V0, pb.V0, pairs, p.m * p.d_v, M * p.d_v, 0.f, st));
+    rc = fwd_core(&pi, p.m, q, k, v, pb.gate, K0 ? pb.K0 : nullptr, V0 ? pb.V0 : nullptr, o, ok_save ? pb.ok : nullptr,
+                  KT ? pb.KT : nullptr, VT ? pb.VT : nullptr, save_gate, gate_save, gate_save_bytes, ws, core, stream,
+                  dev_status);
+    if (rc != GSA_OK) return rc;
+    if (ok_save) GSA_CUDA(launch_resize_rows(pb.ok, ok_save, rows, M, p.m, 0.f, st));
+    if (KT) GSA_CUDA(launch_resize_rows(pb.KT, KT, pairs, M * p.d_k, p.m * p.d_k, 0.f, st));
+    if (VT) GSA_CUDA(launch_resize_rows(pb.VT, VT, pairs, M * p.d_v, p.m * p.d_v, 0.f, st));
     return GSA_OK;
 }
 }  // namespace
@@ -431,19 +505,11 @@ gsa_status_t gsa_fwd_save_gate(const gsa_params_t* params, const void* q, const 
 }
 
 namespace {
-gsa_status_t bwd_impl(const gsa_params_t* params, const void* q, const void* k, const void* v,
+gsa_status_t bwd_core(const gsa_params_t* params, int m_active, const void* q, const void* k, const void* v,
                       const float* gate, const float* K0, const float* V0, const float* ok_saved,
                       const void* dO, const float* dKT, const float* dVT, void* dq, void* dk,
                       void* dv, float* dgate, float* dK0, float* dV0, bool gate_is_saved, const void* gate_saved,
                       size_t gate_saved_bytes, void* ws, size_t ws_bytes, void* stream, int32_t* dev_status) {
-    gsa_status_t rc = check_params(params, true);
-    if (rc != GSA_OK) return rc;
-    if (!ok_ptr(q) || !ok_ptr(k) || !ok_ptr(v) || !ok_ptr(gate) || !ok_ptr(dO) || !ok_ptr(dq) ||
-        !ok_ptr(dk) || !ok_ptr(dv) || !ok_ptr(dgate))
-        return GSA_ERR_INVALID_ARG;
-    if (!ok_opt(K0) || !ok_opt(V0) || !ok_opt(ok_saved) || !ok_opt(dKT) || !ok_opt(dVT) ||
-        !ok_opt(dK0) || !ok_opt(dV0))
-        return GSA_ERR_INVALID_ARG;
     const gsa_params_t& p = *params;
     if (ws == nullptr || (reinterpret_cast<uintptr_t>(ws) & 255u) != 0) return GSA_ERR_WORKSPACE;
     Workspace w = carve(p, GSA_WS_BWD, ws);
@@ -490,7 +556,7 @@ gsa_status_t bwd_impl(const gsa_params_t* params, const void* q, const void* k, 
         ValueSideArgs a1{q, k, w.I, w.G, Kin, nullptr, w.okpart, Bs, Ts, p.H, p.d_k, w.Id};
         GSA_LAUNCH("pass1_value_side", value_side(p, a1, 0, w.strong, st, dev_status));
         GSA_LAUNCH("slot_softmax", launch_slot_softmax_fwd(w.okpart, s.k, p.scale, p.slot_act, w.ok, w.p, p.B, p.T * p.H, p.m, pend.G,
-                                                           nullptr, pend, st));
+                                                           nullptr, pend, st, m_active));
         ok = w.ok;
     }
     // gradient w.r.t. the pass-2 queries p: the pass-1 form on (dO, v, 1-a); carries V~
@@ -515,7 +581,7 @@ gsa_status_t bwd_impl(const gsa_params_t* params, const void* q, const void* k, 
                                                   w.strong, st, dev_status));
         GSA_CUDA(launch_value_side_general(adp, p.m, 0, w.strong, ss, dev_status));
         GSA_CUDA(launch_slot_softmax_bwd(ok, w.dppart, s.v, p.scale, p.slot_act, w.p, w.dz, w.u, p.B, p.T * p.H, p.m, pend.G,
-                                         w.Pd, w.Zd, only, ss));
+                                         w.Pd, w.Zd, only, ss, m_active));
         GSA_CUDA(launch_key_side_general(adq, p.m, 0, w.strong, ss, dev_status));
         if (!g_sink.active) {
             GSA_CUDA(cudaEventRecord(side->join, ss));
@@ -524,7 +590,7 @@ gsa_status_t bwd_impl(const gsa_params_t* params, const void* q, const void* k, 
     } else {
         GSA_LAUNCH("bwd_dp_value_side", value_side(p, adp, 0, w.strong, st, dev_status));
         GSA_LAUNCH("slot_softmax_bwd", launch_slot_softmax_bwd(ok, w.dppart, s.v, p.scale, p.slot_act, w.p, w.dz, w.u, p.B, p.T * p.H, p.m, pend.G, w.Pd,
-                                                               w.Zd, pend, st));
+                                                               w.Zd, pend, st, m_active));
     }
     const float *dKin = dKT, *dVin = dVT;    // states entering the reversed scans (from the right)
     float *dK0out = dK0, *dV0out = dV0;
@@ -574,6 +640,48 @@ gsa_status_t bwd_impl(const gsa_params_t* params, const void* q, const void* k, 
     GSA_LAUNCH("gate_grad", launch_gate_grad(w.u, w.I, w.dIk, s.k, w.dIv, s.v, gate, p.gate_kind, inv_tau(p),
                               dKT, w.KT, dVT, w.VT, p.d_k, p.d_v, w.chunk_tot, dgate, p.B, p.T,
                               p.H, p.m, pend, st, dev_status));
+    return GSA_OK;
+}
+
+gsa_status_t bwd_impl(const gsa_params_t* params, const void* q, const void* k, const void* v,
+                      const float* gate, const float* K0, const float* V0, const float* ok_saved,
+                      const void* dO, const float* dKT, const float* dVT, void* dq, void* dk,
+                      void* dv, float* dgate, float* dK0, float* dV0, bool gate_is_saved, const void* gate_saved,
+                      size_t gate_saved_bytes, void* ws, size_t ws_bytes, void* stream, int32_t* dev_status) {
+    gsa_status_t rc = check_params(params, true);
+    if (rc != GSA_OK) return rc;
+    if (!ok_ptr(q) || !ok_ptr(k) || !ok_ptr(v) || !ok_ptr(gate) || !ok_ptr(dO) || !ok_ptr(dq) ||
+        !ok_ptr(dk) || !ok_ptr(dv) || !ok_ptr(dgate))
+        return GSA_ERR_INVALID_ARG;
+    if (!ok_opt(K0) || !ok_opt(V0) || !ok_opt(ok_saved) || !ok_opt(dKT) || !ok_opt(dVT) ||
+        !ok_opt(dK0) || !ok_opt(dV0))
+        return GSA_ERR_INVALID_ARG;
+    if (!pads_slots(*params))
+        return bwd_core(params, 0, q, k, v, gate, K0, V0, ok_saved, dO, dKT, dVT, dq, dk, dv, dgate, dK0, dV0, gate_is_saved,
+                        gate_saved, gate_saved_bytes, ws, ws_bytes, stream, dev_status);
+    const gsa_params_t& p = *params;
+    const gsa_params_t pi = internal_params(p);
+    if (ws == nullptr || (reinterpret_cast<uintptr_t>(ws) & 255u) != 0) return GSA_ERR_WORKSPACE;
+    const size_t core = carve(pi, GSA_WS_BWD, nullptr).bytes;
+    const PadBuffers pb = carve_pad(p, GSA_WS_BWD, static_cast<char*>(ws) + core);
+    if (ws_bytes < core + pb.bytes) return GSA_ERR_WORKSPACE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const size_t rows = (size_t)p.B * p.T * p.H, pairs = (size_t)p.B * p.H;
+    const int M = kPaddedSlots;
+    const float neutral = p.gate_kind == GSA_GATE_A ? 1.f : (p.gate_kind == GSA_GATE_LOG_A ? 0.f : 80.f);
+    GSA_CUDA(launch_resize_rows(gate, pb.gate, rows, p.m, M, neutral, st));
+    if (ok_saved) GSA_CUDA(launch_resize_rows(ok_saved, pb.ok, rows, p.m, M, 0.f, st));
+    if (K0) GSA_CUDA(launch_resize_rows(K0, pb.K0, pairs, p.m * p.d_k, M * p.d_k, 0.f, st));
+    if (V0) GSA_CUDA(launch_resize_rows(V0, pb.V0, pairs, p.m * p.d_v, M * p.d_v, 0.f, st));
+    if (dKT) GSA_CUDA(launch_resize_rows(dKT, pb.dKT, pairs, p.m * p.d_k, M * p.d_k, 0.f, st));
+    if (dVT) GSA_CUDA(launch_resize_rows(dVT, pb.dVT, pairs, p.m * p.d_v, M * p.d_v, 0.f, st));
+    rc = bwd_core(&pi, p.m, q, k, v, pb.gate, K0 ? pb.K0 : nullptr, V0 ? pb.V0 : nullptr, ok_saved ? pb.ok : nullptr, dO,
+                  dKT ? pb.dKT : nullptr, dVT ? pb.dVT : nullptr, dq, dk, dv, pb.dgate, dK0 ? pb.KT : nullptr,
+                  dV0 ? pb.VT : nullptr, gate_is_saved, gate_saved, gate_saved_bytes, ws, core, stream, dev_status);
+    if (rc != GSA_OK) return rc;
+    GSA_CUDA(launch_resize_rows(pb.dgate, dgate, rows, M, p.m, 0.f, st));
+    if (dK0) GSA_CUDA(launch_resize_rows(pb.KT, dK0, pairs, M * p.d_k, p.m * p.d_k, 0.f, st));
+    if (dV0) GSA_CUDA(launch_resize_rows(pb.VT, dV0, pairs, M * p.d_v, p.m * p.d_v, 0.f, st));
     return GSA_OK;
 }
 }  // namespace

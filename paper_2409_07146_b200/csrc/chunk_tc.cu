@@ -351,7 +351,7 @@ value_side_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_cons
         // state slice: S[c = row][s], slots sb .. sb+31
         float S[kHS];
 #pragma unroll
-        for (int s = 0; s < kHS; ++s) S[s] = a.S0 ? a.S0[((size_t)bh * kM + sb + s) * a.D + d0 + row] : 0.f;
+        for (int s = 0; s < kHS; ++s) S[s] = (a.S0 && d0 + row < a.D) ? a.S0[((size_t)bh * kM + sb + s) * a.D + d0 + row] : 0.f;
 
         // bf16 copy of the state for the first chunk's inter-chunk product
         store_state_row<false>(sSb, row, sb, S, nullptr);
@@ -488,7 +488,7 @@ value_side_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_cons
             PROF_DUMP("value_side compute");
             if (ctl->abort) break;
         }
-        if (!ctl->abort && a.Send) {
+        if (!ctl->abort && a.Send && d0 + row < a.D) {
 #pragma unroll
             for (int s = 0; s < kHS; ++s) a.Send[((size_t)bh * kM + sb + s) * a.D + d0 + row] = S[s];
         }
@@ -698,7 +698,7 @@ key_side_tc_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_consta
                 WAIT_OR_ABORT(&ctl->bar_out, it & 1);
                 if (ctl->abort) break;
                 tma_store_4d(&mapO, sQt, d0, h, t0, b);
-                tma_store_4d(&mapO, sQt + kPanelB, d0 + 64, h, t0, b);
+                if (d0 + 64 < a.D) tma_store_4d(&mapO, sQt + kPanelB, d0 + 64, h, t0, b);
                 bulk_commit();
                 bulk_wait_read();
                 mbar_arrive(&ctl->bar_sb);
@@ -709,7 +709,7 @@ key_side_tc_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_consta
         // state slice, transposed: S[c = row][s], slots sb .. sb+31
         float S[kHS];
 #pragma unroll
-        for (int s = 0; s < kHS; ++s) S[s] = a.S0 ? a.S0[((size_t)bh * kM + sb + s) * a.D + d0 + row] : 0.f;
+        for (int s = 0; s < kHS; ++s) S[s] = (a.S0 && d0 + row < a.D) ? a.S0[((size_t)bh * kM + sb + s) * a.D + d0 + row] : 0.f;
 
         int n_mod = 0;     // moderate chunks so far (phases of bar_p)
         PROF_DECL
@@ -834,7 +834,7 @@ key_side_tc_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_consta
             PROF_DUMP("key_side compute");
             if (ctl->abort) break;
         }
-        if (!ctl->abort && a.Send) {
+        if (!ctl->abort && a.Send && d0 + row < a.D) {
 #pragma unroll
             for (int s = 0; s < kHS; ++s) a.Send[((size_t)bh * kM + sb + s) * a.D + d0 + row] = S[s];
         }
@@ -900,23 +900,26 @@ cudaError_t side_lane_release() {
     return cudaSuccess;
 }
 
+// Head dimensions the tensor-core kernels serve: multiples of the 128-wide slice, and 64 (half a
+// slice: the tile copies zero-fill the channels beyond the head, stores are clipped).
+bool tc_dim_ok(int D) { return D == 64 || (D > 0 && D % kDST == 0); }
 bool tc_supported(int d_k, int d_v, int M) {
-    return M == kM && d_k % kDST == 0 && d_v % kDST == 0;
+    return M == kM && tc_dim_ok(d_k) && tc_dim_ok(d_v);
 }
-int tc_value_side_slices(int D) { return D / kDST; }
+int tc_value_side_slices(int D) { return (D + kDST - 1) / kDST; }
 int tc_chunk() { return kCT; }
 
 cudaError_t launch_value_side_tc(const ValueSideArgs& a, int M, int reverse, const int* strong_flag,
                                  cudaStream_t st, int32_t* dev_status) {
-    if (M != kM || a.D % kDST != 0 || strong_flag == nullptr) return cudaErrorNotSupported;
+    if (M != kM || !tc_dim_ok(a.D) || strong_flag == nullptr) return cudaErrorNotSupported;
     CUtensorMap mq, mk, mw, mg, mo;
     cudaError_t e = make_tensor_map_bthd(&mq, a.xq, a.B, a.T, a.H, a.D, kCT, 2);
-    if (e == cudaSuccess) e = make_tensor_map_sliced(&mo, a.out, a.D / kDST, a.B, a.T, a.H, kM, kCT, 4);
+    if (e == cudaSuccess) e = make_tensor_map_sliced(&mo, a.out, tc_value_side_slices(a.D), a.B, a.T, a.H, kM, kCT, 4);
     if (e == cudaSuccess) e = make_tensor_map_bthd(&mk, a.xk, a.B, a.T, a.H, a.D, kCT, 2);
     if (e == cudaSuccess) e = make_tensor_map_bthd(&mw, a.w, a.B, a.T, a.H, kM, kCT, 4);
     if (e == cudaSuccess) e = make_tensor_map_bthd(&mg, a.G, a.B, a.T, a.H, kM, kCT, 4);
     if (e != cudaSuccess) return e;
-    dim3 grid(a.B * a.H, a.D / kDST);
+    dim3 grid(a.B * a.H, tc_value_side_slices(a.D));
 #define GSA_LAUNCH_VS(REVV, FLAGS)                                                                       \
     e = prepare(value_side_tc_kernel<REVV, true>, kSmemValueSide);                                       \
     if (e != cudaSuccess) return e;                                                                      \
@@ -942,15 +945,15 @@ cudaError_t launch_value_side_tc(const ValueSideArgs& a, int M, int reverse, con
 
 cudaError_t launch_value_side_general(const ValueSideArgs& a, int M, int reverse, const int* strong_flag,
                                       cudaStream_t st, int32_t* dev_status) {
-    if (M != kM || a.D % kDST != 0 || strong_flag == nullptr) return cudaErrorNotSupported;
+    if (M != kM || !tc_dim_ok(a.D) || strong_flag == nullptr) return cudaErrorNotSupported;
     CUtensorMap mq, mk, mw, mg, mo;
     cudaError_t e = make_tensor_map_bthd(&mq, a.xq, a.B, a.T, a.H, a.D, kCT, 2);
-    if (e == cudaSuccess) e = make_tensor_map_sliced(&mo, a.out, a.D / kDST, a.B, a.T, a.H, kM, kCT, 4);
+    if (e == cudaSuccess) e = make_tensor_map_sliced(&mo, a.out, tc_value_side_slices(a.D), a.B, a.T, a.H, kM, kCT, 4);
     if (e == cudaSuccess) e = make_tensor_map_bthd(&mk, a.xk, a.B, a.T, a.H, a.D, kCT, 2);
     if (e == cudaSuccess) e = make_tensor_map_bthd(&mw, a.w, a.B, a.T, a.H, kM, kCT, 4);
     if (e == cudaSuccess) e = make_tensor_map_bthd(&mg, a.G, a.B, a.T, a.H, kM, kCT, 4);
     if (e != cudaSuccess) return e;
-    dim3 grid(a.B * a.H, a.D / kDST);
+    dim3 grid(a.B * a.H, tc_value_side_slices(a.D));
     if (reverse) {
         e = prepare(value_side_tc_kernel<true, true>, kSmemValueSide);
         if (e != cudaSuccess) return e;
@@ -965,7 +968,7 @@ cudaError_t launch_value_side_general(const ValueSideArgs& a, int M, int reverse
 
 cudaError_t launch_key_side_general(const KeySideArgs& a, int M, int reverse, const int* strong_flag,
                                     cudaStream_t st, int32_t* dev_status) {
-    if (M != kM || a.D % kDST != 0 || strong_flag == nullptr) return cudaErrorNotSupported;
+    if (M != kM || !tc_dim_ok(a.D) || strong_flag == nullptr) return cudaErrorNotSupported;
     CUtensorMap mv, muq, muk, mg, mo;
     cudaError_t e = make_tensor_map_bthd(&mv, a.xv, a.B, a.T, a.H, a.D, kCT, 2);
     if (e == cudaSuccess) e = make_tensor_map_bthd(&mo, a.out, a.B, a.T, a.H, a.D, kCT, 2);
@@ -973,7 +976,7 @@ cudaError_t launch_key_side_general(const KeySideArgs& a, int M, int reverse, co
     if (e == cudaSuccess) e = make_tensor_map_bthd(&muk, a.uk, a.B, a.T, a.H, kM, kCT, 4);
     if (e == cudaSuccess) e = make_tensor_map_bthd(&mg, a.G, a.B, a.T, a.H, kM, kCT, 4);
     if (e != cudaSuccess) return e;
-    dim3 grid(a.B * a.H, a.D / kDST);
+    dim3 grid(a.B * a.H, tc_value_side_slices(a.D));
     if (reverse) {
         e = prepare(key_side_tc_kernel<true, true>, kSmemKeySide);
         if (e != cudaSuccess) return e;
@@ -988,7 +991,7 @@ cudaError_t launch_key_side_general(const KeySideArgs& a, int M, int reverse, co
 
 cudaError_t launch_key_side_tc(const KeySideArgs& a, int M, int reverse, const int* strong_flag,
                                cudaStream_t st, int32_t* dev_status) {
-    if (M != kM || a.D % kDST != 0 || strong_flag == nullptr) return cudaErrorNotSupported;
+    if (M != kM || !tc_dim_ok(a.D) || strong_flag == nullptr) return cudaErrorNotSupported;
     CUtensorMap mv, muq, muk, mg, mo;
     cudaError_t e = make_tensor_map_bthd(&mv, a.xv, a.B, a.T, a.H, a.D, kCT, 2);
     if (e == cudaSuccess) e = make_tensor_map_bthd(&mo, a.out, a.B, a.T, a.H, a.D, kCT, 2);
@@ -996,7 +999,7 @@ cudaError_t launch_key_side_tc(const KeySideArgs& a, int M, int reverse, const i
     if (e == cudaSuccess) e = make_tensor_map_bthd(&muk, a.uk, a.B, a.T, a.H, kM, kCT, 4);
     if (e == cudaSuccess) e = make_tensor_map_bthd(&mg, a.G, a.B, a.T, a.H, kM, kCT, 4);
     if (e != cudaSuccess) return e;
-    dim3 grid(a.B * a.H, a.D / kDST);
+    dim3 grid(a.B * a.H, tc_value_side_slices(a.D));
 #define GSA_LAUNCH_KS(REVV, FLAGS)                                                                       \
     e = prepare(key_side_tc_kernel<REVV, true>, kSmemKeySide);                                           \
     if (e != cudaSuccess) return e;                                                                      \

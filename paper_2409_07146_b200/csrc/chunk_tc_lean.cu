@@ -268,7 +268,7 @@ value_side_lean_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_co
         // state slice: S[c = row][s], slots sb .. sb+31
         float S[kHS];
 #pragma unroll
-        for (int s = 0; s < kHS; ++s) S[s] = a.S0 ? a.S0[((size_t)bh * kM + sb + s) * a.D + d0 + row] : 0.f;
+        for (int s = 0; s < kHS; ++s) S[s] = (a.S0 && d0 + row < a.D) ? a.S0[((size_t)bh * kM + sb + s) * a.D + d0 + row] : 0.f;
         store_state_row_split<false>(sSb, sSb + kPanelB, row, sb, S, nullptr);
 
         // G of the last valid row of chunk n (threads 0..63, one slot each), one chunk ahead
@@ -355,7 +355,7 @@ value_side_lean_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_co
             PROF_DUMP("value_side lean compute");
             if (stop) break;
         }
-        if (!ctl->abort && a.Send) {
+        if (!ctl->abort && a.Send && d0 + row < a.D) {
 #pragma unroll
             for (int s = 0; s < kHS; ++s) a.Send[((size_t)bh * kM + sb + s) * a.D + d0 + row] = S[s];
         }
@@ -416,7 +416,7 @@ key_side_lean_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_cons
             const int t = chunk_t0(n);
             const unsigned char* sOut = sXv + 2 * (n & 1) * kPanelB;
             tma_store_4d(&mapO, sOut, d0, h, t, b);
-            tma_store_4d(&mapO, sOut + kPanelB, d0 + 64, h, t, b);
+            if (d0 + 64 < a.D) tma_store_4d(&mapO, sOut + kPanelB, d0 + 64, h, t, b);
             bulk_commit();
         };
         prefetch_tmap(&mapV); prefetch_tmap(&mapUq); prefetch_tmap(&mapUk); prefetch_tmap(&mapO);
@@ -538,7 +538,7 @@ key_side_lean_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_cons
         // state slice, transposed: S[c = row][s], slots sb .. sb+31
         float S[kHS];
 #pragma unroll
-        for (int s = 0; s < kHS; ++s) S[s] = a.S0 ? a.S0[((size_t)bh * kM + sb + s) * a.D + d0 + row] : 0.f;
+        for (int s = 0; s < kHS; ++s) S[s] = (a.S0 && d0 + row < a.D) ? a.S0[((size_t)bh * kM + sb + s) * a.D + d0 + row] : 0.f;
 
         // G of the last valid row of chunk n (threads 0..63, one slot each)
         auto chunk_gc = [&](int n) {
@@ -608,7 +608,7 @@ key_side_lean_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_cons
             }
             if (publish_and_vote(&ctl->bar_out[n & 1], tid, ctl->abort != 0)) break;
         }
-        if (!ctl->abort && a.Send) {
+        if (!ctl->abort && a.Send && d0 + row < a.D) {
 #pragma unroll
             for (int s = 0; s < kHS; ++s) a.Send[((size_t)bh * kM + sb + s) * a.D + d0 + row] = S[s];
         }
@@ -717,7 +717,7 @@ state_scan_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
         // =============================== compute threads: S[c = row][s], slots sb .. sb+31
         float S[kHS];
 #pragma unroll
-        for (int s = 0; s < kHS; ++s) S[s] = S0 ? S0[((size_t)bh * kM + sb + s) * D + d0 + row] : 0.f;
+        for (int s = 0; s < kHS; ++s) S[s] = (S0 && d0 + row < D) ? S0[((size_t)bh * kM + sb + s) * D + d0 + row] : 0.f;
         // G of the last valid row of chunk n (threads 0..63, one slot each), one chunk ahead
         auto chunk_gc = [&](int n) {
             const int last = min(chunk_t0(n) + kCT, T) - 1;
@@ -755,7 +755,7 @@ state_scan_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
             // (the barrier inside also publishes the next chunk's egc)
             if (publish_and_vote(&ctl->bar_acc[n & 1], tid, ctl->abort != 0)) break;
         }
-        if (!ctl->abort && Send) {
+        if (!ctl->abort && Send && d0 + row < D) {
 #pragma unroll
             for (int s = 0; s < kHS; ++s) Send[((size_t)bh * kM + sb + s) * D + d0 + row] = S[s];
         }
@@ -777,7 +777,7 @@ cudaError_t launch_state_scan(const void* X, const void* W, const float* G, cons
     cudaError_t e = make_tensor_map_bthd(&mx, X, B, T, H, D, kCT, 2);
     if (e == cudaSuccess) e = make_tensor_map_bthd(&mw, W, B, T, H, 2 * kM, kCT, 2);
     if (e != cudaSuccess) return e;
-    dim3 grid(B * H, D / kDST);
+    dim3 grid(B * H, tc_value_side_slices(D));
     if (reverse) {
         e = prepare(state_scan_kernel<true>, kSmemStateScan, kLeanThreads);
         if (e != cudaSuccess) return e;
@@ -797,11 +797,11 @@ cudaError_t launch_value_side_lean(const ValueSideArgs& a, int reverse, const in
         return launch_state_scan(a.xk, a.wd, a.G, a.S0, a.Send, a.B, a.T, a.H, a.D, reverse, strong_flag, st, dev_status);
     CUtensorMap mq, mk, mw, mo;
     cudaError_t e = make_tensor_map_bthd(&mq, a.xq, a.B, a.T, a.H, a.D, kCT, 2);
-    if (e == cudaSuccess) e = make_tensor_map_sliced(&mo, a.out, a.D / kDST, a.B, a.T, a.H, kM, kCT, 4);
+    if (e == cudaSuccess) e = make_tensor_map_sliced(&mo, a.out, tc_value_side_slices(a.D), a.B, a.T, a.H, kM, kCT, 4);
     if (e == cudaSuccess) e = make_tensor_map_bthd(&mk, a.xk, a.B, a.T, a.H, a.D, kCT, 2);
     if (e == cudaSuccess) e = make_tensor_map_bthd(&mw, a.wd, a.B, a.T, a.H, 2 * kM, kCT, 2);
     if (e != cudaSuccess) return e;
-    dim3 grid(a.B * a.H, a.D / kDST);
+    dim3 grid(a.B * a.H, tc_value_side_slices(a.D));
     auto launch = [&](auto kernel) {
         cudaError_t e2 = prepare(kernel, kSmemLeanValue, kLeanThreads);
         if (e2 != cudaSuccess) return e2;
@@ -822,7 +822,7 @@ cudaError_t launch_key_side_lean(const KeySideArgs& a, int reverse, const int* s
     if (e == cudaSuccess) e = make_tensor_map_bthd(&muq, a.uq_d, a.B, a.T, a.H, 2 * kM, kCT, 2);
     if (e == cudaSuccess) e = make_tensor_map_bthd(&muk, a.uk_d, a.B, a.T, a.H, 2 * kM, kCT, 2);
     if (e != cudaSuccess) return e;
-    dim3 grid(a.B * a.H, a.D / kDST);
+    dim3 grid(a.B * a.H, tc_value_side_slices(a.D));
     auto launch = [&](auto kernel) {
         cudaError_t e2 = prepare(kernel, kSmemLeanKey, kLeanThreads);
         if (e2 != cudaSuccess) return e2;

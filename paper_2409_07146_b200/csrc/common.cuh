@@ -174,11 +174,14 @@ cudaError_t launch_segment_combine(const float* seg_logdecay, const float* local
 // act: gsa_act_t (the softmax over the slots or an element-wise replacement)
 cudaError_t launch_slot_softmax_fwd(const float* part, int nslice, float scale, int act, float* ok,
                                     float* p, int B, int rows_per_batch, int M, const float* G, void* p_decayed,
-                                    PendingDecay pend, cudaStream_t st);
+                                    PendingDecay pend, cudaStream_t st, int m_active = 0);
 cudaError_t launch_slot_softmax_bwd(const float* ok, const float* dp_part, int nslice,
                                     float scale, int act, float* p, float* dz, float* u, int B, int rows_per_batch,
                                     int M, const float* G, void* p_decayed, void* dz_decayed,
-                                    PendingDecay pend, cudaStream_t st);
+                                    PendingDecay pend, cudaStream_t st, int m_active = 0);
+// m_active (0 = all M): slots from m_active on are padding and take no part in the non-linearity.
+// rows of n_in floats -> rows of n_out floats (tail filled with `fill`, or cut)
+cudaError_t launch_resize_rows(const float* in, float* out, size_t rows, int n_in, int n_out, float fill, cudaStream_t st);
 cudaError_t launch_gate_grad(const float* u, const float* I, const float* dIk_part, int nsk,
                              const float* dIv_part, int nsv, const float* gate,
                              int gate_kind, float inv_tau, const float* dKT, const float* KT,
@@ -192,6 +195,7 @@ cudaError_t launch_key_side_simt(const KeySideArgs& a, int io, int M, int revers
                                  cudaStream_t st);
 // tcgen05 (bf16 tensor-core) versions of the two primitives; bf16 io only.
 bool tc_supported(int d_k, int d_v, int M);
+bool tc_dim_ok(int D);
 int tc_value_side_slices(int D);
 int tc_chunk();                    // chunk length of the tensor-core kernels   // how many partial-sum slices value_side writes for width D
 cudaError_t launch_value_side_tc(const ValueSideArgs& a, int M, int reverse, const int* strong_flag,

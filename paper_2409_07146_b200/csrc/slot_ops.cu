@@ -159,7 +159,7 @@ __global__ void __launch_bounds__(256) slot_softmax_fwd_kernel(const float* __re
                                                                float* __restrict__ p,
                                                                int rows_per_batch, const float* __restrict__ G,
                                                                __nv_bfloat16* __restrict__ p_decayed,
-                                                               PendingDecay pend) {
+                                                               PendingDecay pend, int m_active) {
     constexpr int R = kSmR, LPR = M / R, RPW = 32 / LPR;       // lanes per row, rows per warp
     const int lane = threadIdx.x & 31, sub = lane / LPR, l = lane % LPR;
     const int r_in_b = (blockIdx.x * 8 + (threadIdx.x >> 5)) * RPW + sub, b = blockIdx.y;
@@ -169,6 +169,8 @@ __global__ void __launch_bounds__(256) slot_softmax_fwd_kernel(const float* __re
     const size_t total = (size_t)gridDim.y * rows_per_batch * M;
     const size_t idx = row * M + l * R;
     const bool pending = pend.pending(b, rr);
+    // slots from m_active on are padding (a layer with fewer slots than the kernels' tile): they take no part
+    const bool padded = l * R >= m_active;
     // serving the flagged pairs only: a warp none of whose rows is flagged has nothing to do
     const bool skip = pend.strong_only != 0 && pending;
     if (__all_sync(0xffffffffu, skip)) return;
@@ -192,21 +194,21 @@ __global__ void __launch_bounds__(256) slot_softmax_fwd_kernel(const float* __re
     for (int r = 0; r < R; ++r) {
         if (pending) z[r] *= eg[r];
         z[r] *= scale;
-        zmax = fmaxf(zmax, z[r]);
+        if (!padded) zmax = fmaxf(zmax, z[r]);
     }
     float e[R];
     if (act == GSA_ACT_SOFTMAX) {
         zmax = row_max<LPR>(zmax);
         float den = 0.f;
 #pragma unroll
-        for (int r = 0; r < R; ++r) { e[r] = __expf(z[r] - zmax); den += e[r]; }
+        for (int r = 0; r < R; ++r) { e[r] = padded ? 0.f : __expf(z[r] - zmax); den += e[r]; }
         den = row_sum<LPR>(den);
         const float inv = 1.f / den;
 #pragma unroll
         for (int r = 0; r < R; ++r) e[r] *= inv;
     } else {               // element-wise replacement of the softmax (uniform over the launch)
 #pragma unroll
-        for (int r = 0; r < R; ++r) e[r] = slot_act_value(z[r], act);
+        for (int r = 0; r < R; ++r) e[r] = padded ? 0.f : slot_act_value(z[r], act);
     }
     if (!live || skip) return;
     if (ok != nullptr) st_vec(ok + idx, z);
@@ -222,16 +224,17 @@ __global__ void __launch_bounds__(256) slot_softmax_fwd_kernel(const float* __re
 
 cudaError_t launch_slot_softmax_fwd(const float* part, int nslice, float scale, int act, float* ok,
                                     float* p, int B, int rows_per_batch, int M, const float* G, void* p_decayed,
-                                    PendingDecay pend, cudaStream_t st) {
+                                    PendingDecay pend, cudaStream_t st, int m_active) {
+    if (m_active <= 0 || m_active > M) m_active = M;
     const int rpb = 8 * (128 / M);       // rows per block: 8 warps x 128/M rows
     const dim3 grid((unsigned)((rows_per_batch + rpb - 1) / rpb), (unsigned)B);
     const int rows = rows_per_batch;
     if (M == 64)
         slot_softmax_fwd_kernel<64><<<grid, 256, 0, st>>>(part, nslice, scale, act, ok, p, rows, G,
-                                                          static_cast<__nv_bfloat16*>(p_decayed), pend);
+                                                          static_cast<__nv_bfloat16*>(p_decayed), pend, m_active);
     else
         slot_softmax_fwd_kernel<32><<<grid, 256, 0, st>>>(part, nslice, scale, act, ok, p, rows, G,
-                                                          static_cast<__nv_bfloat16*>(p_decayed), pend);
+                                                          static_cast<__nv_bfloat16*>(p_decayed), pend, m_active);
     return cudaGetLastError();
 }
 
@@ -250,7 +253,7 @@ __global__ void __launch_bounds__(256) slot_softmax_bwd_kernel(const float* __re
                                                                int rows_per_batch, const float* __restrict__ G,
                                                                __nv_bfloat16* __restrict__ p_decayed,
                                                                __nv_bfloat16* __restrict__ dz_decayed,
-                                                               PendingDecay pend) {
+                                                               PendingDecay pend, int m_active) {
     constexpr int R = kSmR, LPR = M / R, RPW = 32 / LPR;       // lanes per row, rows per warp
     const int lane = threadIdx.x & 31, sub = lane / LPR, l = lane % LPR;
     const int r_in_b = (blockIdx.x * 8 + (threadIdx.x >> 5)) * RPW + sub, b = blockIdx.y;
@@ -261,6 +264,7 @@ __global__ void __launch_bounds__(256) slot_softmax_bwd_kernel(const float* __re
     const size_t idx = row * M + l * R;
     const bool pending = pend.pending(b, rr);
     const bool skip = pend.strong_only != 0 && pending;      // (as in the forward kernel)
+    const bool padded = l * R >= m_active;                   // (likewise)
     if (__all_sync(0xffffffffu, skip)) return;
     float z[R], dpv[R], eg[R];
     ld_vec(ok + idx, z);
@@ -282,14 +286,15 @@ __global__ void __launch_bounds__(256) slot_softmax_bwd_kernel(const float* __re
 #pragma unroll
     for (int r = 0; r < R; ++r) {
         if (pending) dpv[r] *= eg[r];
-        zmax = fmaxf(zmax, z[r]);
+        if (padded) { z[r] = 0.f; dpv[r] = 0.f; }
+        else zmax = fmaxf(zmax, z[r]);
     }
     float e[R], dzv[R], uv[R];
     if (act == GSA_ACT_SOFTMAX) {
         zmax = row_max<LPR>(zmax);
         float den = 0.f;
 #pragma unroll
-        for (int r = 0; r < R; ++r) { e[r] = __expf(z[r] - zmax); den += e[r]; }
+        for (int r = 0; r < R; ++r) { e[r] = padded ? 0.f : __expf(z[r] - zmax); den += e[r]; }
         den = row_sum<LPR>(den);
         const float inv = 1.f / den;
         float pdp = 0.f;
@@ -305,7 +310,7 @@ __global__ void __launch_bounds__(256) slot_softmax_bwd_kernel(const float* __re
     } else {               // element-wise replacement f of the softmax: dok = f'(ok) dp
 #pragma unroll
         for (int r = 0; r < R; ++r) {
-            e[r] = slot_act_value(z[r], act);
+            e[r] = padded ? 0.f : slot_act_value(z[r], act);
             const float dok = slot_act_slope(z[r], act) * dpv[r];
             dzv[r] = scale * dok;
             uv[r] = e[r] * dpv[r] + z[r] * dok;
@@ -328,18 +333,19 @@ __global__ void __launch_bounds__(256) slot_softmax_bwd_kernel(const float* __re
 cudaError_t launch_slot_softmax_bwd(const float* ok, const float* dp_part, int nslice,
                                     float scale, int act, float* p, float* dz, float* u, int B, int rows_per_batch,
                                     int M, const float* G, void* p_decayed, void* dz_decayed,
-                                    PendingDecay pend, cudaStream_t st) {
+                                    PendingDecay pend, cudaStream_t st, int m_active) {
+    if (m_active <= 0 || m_active > M) m_active = M;
     const int rpb = 8 * (128 / M);       // rows per block: 8 warps x 128/M rows
     const dim3 grid((unsigned)((rows_per_batch + rpb - 1) / rpb), (unsigned)B);
     const int rows = rows_per_batch;
     if (M == 64)
         slot_softmax_bwd_kernel<64><<<grid, 256, 0, st>>>(ok, dp_part, nslice, scale, act, p, dz, u, rows, G,
                                                           static_cast<__nv_bfloat16*>(p_decayed),
-                                                          static_cast<__nv_bfloat16*>(dz_decayed), pend);
+                                                          static_cast<__nv_bfloat16*>(dz_decayed), pend, m_active);
     else
         slot_softmax_bwd_kernel<32><<<grid, 256, 0, st>>>(ok, dp_part, nslice, scale, act, p, dz, u, rows, G,
                                                           static_cast<__nv_bfloat16*>(p_decayed),
-                                                          static_cast<__nv_bfloat16*>(dz_decayed), pend);
+                                                          static_cast<__nv_bfloat16*>(dz_decayed), pend, m_active);
     return cudaGetLastError();
 }
 
@@ -821,6 +827,26 @@ cudaError_t launch_gate_grad(const float* u, const float* I, const float* dIk_pa
         gate_grad_scan_kernel<32><<<B * H, dim3(32, 16), 0, st>>>(blk_tot, dKT, KT, dVT, VT, d_k, d_v, nblk);
         gate_grad_carry_kernel<32><<<grid, dim3(block.x, block.y, 2), 0, st>>>(gate, gate_kind, inv_tau, blk_tot, dgate, T, H, nblk);
     }
+    return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------ slot padding
+// Rows of n_in floats copied into rows of n_out floats: widened rows get `fill` in their tail,
+// narrowed rows lose theirs.  Used when a layer with 32 slots runs on the 64-slot tiles of the
+// tensor-core kernels: gate rows are widened with a neutral gate, memories with empty slots.
+__global__ void resize_rows_kernel(const float* __restrict__ in, float* __restrict__ out, size_t rows, int n_in, int n_out,
+                                   float fill) {
+    const size_t total = rows * (size_t)n_out;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+        const size_t r = i / n_out;
+        const int c = (int)(i - r * n_out);
+        out[i] = c < n_in ? in[r * n_in + c] : fill;
+    }
+}
+cudaError_t launch_resize_rows(const float* in, float* out, size_t rows, int n_in, int n_out, float fill, cudaStream_t st) {
+    const size_t total = rows * (size_t)n_out;
+    const unsigned blocks = (unsigned)((total + 255) / 256 < 148 * 32 ? (total + 255) / 256 : 148 * 32);
+    resize_rows_kernel<<<blocks ? blocks : 1, 256, 0, st>>>(in, out, rows, n_in, n_out, fill);
     return cudaGetLastError();
 }
 

@@ -45,6 +45,9 @@ def test_chunk_and_workspace_queries(lib):
     assert gsa.gsa_chunk_size(p) == 64
     assert gsa.gsa_chunk_size(gsa.Params(1, 256, 1, 128, 128, 64, io="bf16")) == 128
     assert gsa.gsa_chunk_size(gsa.Params(1, 256, 1, 128, 128, 64, io="bf16", impl="simt")) == 64
+    # 64-wide heads and 32 slots run on the tensor-core kernels too (bf16 io)
+    assert gsa.gsa_chunk_size(gsa.Params(1, 256, 1, 64, 64, 32, io="bf16")) == 128
+    assert gsa.gsa_chunk_size(gsa.Params(1, 256, 1, 64, 64, 32, io="f32")) == 64
     f, b = gsa.gsa_workspace_bytes(p, binding.GSA_WS_FWD), gsa.gsa_workspace_bytes(p, binding.GSA_WS_BWD)
     assert f > 0 and b > f and f % 256 == 0
     assert gsa.gsa_workspace_bytes(p, binding.GSA_WS_DECODE) == 0

@@ -246,6 +246,37 @@ def test_fwd_tc_ragged_lengths(T):
     print("tc fwd", T, errs)
 
 
+@pytest.mark.parametrize("dk,dv,m", [(64, 64, 64), (64, 128, 64), (128, 64, 64), (512, 512, 32), (64, 128, 32)])
+@pytest.mark.parametrize("T", [100, 384])
+def test_tc_narrow_heads_and_32_slots_fwd_bwd(dk, dv, m, T):
+    """64-wide heads (half a 128-wide slice: the tile copies zero-fill the rest) and 32 slots (the last 32
+    of the kernels' 64 padded with a gate that keeps everything and writes nothing) on the tensor-core
+    kernels, asked for by name: forward and backward with carried memories and final-memory gradients."""
+    B, H = 2, 2
+    d = rand_inputs(40 + dk + dv + m + T, B, T, H, dk, dv, m, "bf16", init=True, final_grads=True)
+    assert gsa.gsa_chunk_size(gsa.Params(B, T, H, dk, dv, m, io="bf16", impl="tc")) == 128
+    got, gate = run_fwd(d, B, T, H, dk, dv, m, "bf16", impl="tc", scale=0.8)
+    ef = check_fwd(d, got, gate, "bf16", scale=0.8, tc=True)
+    for saved in (False, True):
+        gb, rb = run_bwd(d, B, T, H, dk, dv, m, "bf16", impl="tc", scale=0.8, saved=saved)
+        eb = check_bwd(gb, rb, TOL["bf16"], tc=True)
+    print("narrow tc", dk, dv, m, T, ef, eb)
+
+
+def test_tc_32_slots_other_gate_kinds_and_activations():
+    B, T, H, dk, dv, m = 1, 200, 2, 128, 128, 32
+    d = rand_inputs(63, B, T, H, dk, dv, m, "bf16", init=True)
+    for log in (False, True):
+        got, gate = run_fwd(d, B, T, H, dk, dv, m, "bf16", impl="tc", log=log)
+        check_fwd(d, got, gate, "bf16", log=log, tc=True)
+        gb, rb = run_bwd(d, B, T, H, dk, dv, m, "bf16", impl="tc", log=log, saved=True)
+        check_bwd(gb, rb, TOL["bf16"], tc=True)
+    got, gate = run_fwd(d, B, T, H, dk, dv, m, "bf16", impl="tc", act="relu")
+    check_fwd(d, got, gate, "bf16", tc=True, act="relu")
+    gb, rb = run_bwd(d, B, T, H, dk, dv, m, "bf16", impl="tc", saved=True, act="relu")
+    check_bwd(gb, rb, TOL["bf16"], tc=True)
+
+
 @pytest.mark.parametrize("dk,dv", [(256, 128), (128, 512), (512, 512)])
 def test_fwd_tc_shapes(dk, dv):
     B, T, H, m = 1, 384, 2, 64
