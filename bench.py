@@ -228,11 +228,13 @@ def run_reference(args):
 
 
 # ----------------------------------------------------------------------------- sharding
-def rank_workload(rank: int) -> W.Workload:
+def rank_workload(rank: int, m: int = 0) -> W.Workload:
     """Weak scaling over batch: rank r runs its own batch of the workload (its own seed);
-    (batch, head) pairs are independent recurrences, so no rank needs another's data."""
+    (batch, head) pairs are independent recurrences, so no rank needs another's data.
+    m (0 = the workload's own 64): another slot count on the same shape (the paper's ablation on the
+    number of slots: 32, 64, 128)."""
     base = W.CONFIGS[WORKLOAD]
-    return base.scaled(seed=base.seed + 1000 * rank)
+    return base.scaled(seed=base.seed + 1000 * rank, m=m or base.m)
 
 
 def max_over_ranks(ms: float, world: int, device=None) -> float:
@@ -268,7 +270,7 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     dev = torch.device("cuda", local)
 
-    w = rank_workload(rank)
+    w = rank_workload(rank, args.m)
     x = W.make_inputs(w)
     p = gsa.Params(w.B, w.T, w.H, w.d_k, w.d_v, w.m, io=w.io, slot_act=args.slot_act, tc_operands=args.tc_operands,
                    fuse=args.fuse)
@@ -458,7 +460,7 @@ def run_ours(args):
         avg_ms = sum(k_["avg_ms"] * k_["launches_per_step"] for k_ in members) / n_l
         alg = sum(k_["alg_bytes"] * k_["launches_per_step"] for k_ in members) / n_l
         traf = [NCU_TRAFFIC.get(k_["kernel"]) for k_ in members]
-        traffic = int(sum(traf) / len(traf)) if all(t is not None for t in traf) else None
+        traffic = int(sum(traf) / len(traf)) if (all(t is not None for t in traf) and w.m == 64) else None
         # the bytes the same launch would move if the slot-sized rows between the passes stayed on chip
         # (the d-sized tensors only: v in, o out for key_side; q, k in for value_side)
         e_ = 2 if w.io == "bf16" else 4
@@ -685,6 +687,9 @@ def main():
     ap.add_argument("--slot-act", default="softmax", choices=["softmax", "none", "relu", "swish", "relu2"],
                     help="the non-linearity between the two passes: the paper's softmax (the headline "
                          "workload) or one of the replacements of its ablation")
+    ap.add_argument("--m", type=int, default=0, choices=[0, 32, 64, 128],
+                    help="slot count on the benchmark shape (default: the workload's 64); 32 runs on the tensor-core "
+                         "kernels' 64-slot tiles, 128 on the fp32 CUDA-core kernels")
     ap.add_argument("--fuse", action="store_true",
                     help="the fused chunk kernel (pass 1 -> slot softmax -> pass 2 in one kernel, and its backward "
                          "twin) instead of the separate kernels; slower as measured, not the default")

@@ -35,8 +35,11 @@
  *     gsa_workspace_bytes() bytes, 256-byte aligned; its contents are
  *     undefined afterwards.  Calls that run concurrently need distinct
  *     workspaces.
- *   - Supported: d_k, d_v in {64,128,256,512}; m in {32,64}; B,T,H >= 1
- *     (T need not be a multiple of the chunk; the tail chunk is masked).
+ *   - Supported: d_k, d_v in {64,128,256,512}; m in {32,64,128}; B,T,H >= 1
+ *     (T need not be a multiple of the chunk; the tail chunk is masked).  bf16 io
+ *     with m in {32,64} runs on the tensor-core kernels (m = 32 on their 64-slot
+ *     tiles with the upper half padded; d = 64 on half a 128-wide slice); fp32 io
+ *     and m = 128 run on the fp32 CUDA-core kernels.
  *   - Errors are return codes; arguments are validated before anything is
  *     launched and outputs are untouched when a call fails validation.
  *     No entry point throws, aborts or prints.

@@ -35,7 +35,7 @@ gsa_status_t check_params(const gsa_params_t* p, bool need_T) {
     if (p->fuse != GSA_FUSE_OFF && p->fuse != GSA_FUSE_ON) return GSA_ERR_INVALID_ARG;
     if (!(p->scale == p->scale)) return GSA_ERR_INVALID_ARG;
     if (!dim_ok(p->d_k) || !dim_ok(p->d_v)) return GSA_ERR_UNSUPPORTED;
-    if (p->m != 32 && p->m != 64) return GSA_ERR_UNSUPPORTED;
+    if (p->m != 32 && p->m != 64 && p->m != 128) return GSA_ERR_UNSUPPORTED;
     if ((long long)p->B * p->H > 0x7fffffffLL / 4) return GSA_ERR_UNSUPPORTED;
     if (p->impl == GSA_IMPL_TC && p->io != GSA_BF16) return GSA_ERR_UNSUPPORTED;
     // the tensor-core kernels asked for by name: no silent fall-back to the CUDA-core kernels

@@ -35,7 +35,11 @@ __device__ __forceinline__ void mm_nn(const float* A, int lda, const float* B, i
 #pragma unroll
         for (int kk = 0; kk < 4; ++kk) {
             float b[NJ];
-            if constexpr (NJ == 4) {
+            if constexpr (NJ == 8) {
+                const float4 t = *reinterpret_cast<const float4*>(B + (k + kk) * ldb + 8 * tx);
+                const float4 t2 = *reinterpret_cast<const float4*>(B + (k + kk) * ldb + 8 * tx + 4);
+                b[0] = t.x; b[1] = t.y; b[2] = t.z; b[3] = t.w; b[4] = t2.x; b[5] = t2.y; b[6] = t2.z; b[7] = t2.w;
+            } else if constexpr (NJ == 4) {
                 const float4 t = *reinterpret_cast<const float4*>(B + (k + kk) * ldb + 4 * tx);
                 b[0] = t.x; b[1] = t.y; b[2] = t.z; b[3] = t.w;
             } else {
@@ -58,7 +62,11 @@ __device__ __forceinline__ void mm_tn(const float* A, int lda, const float* B, i
         const float4 t = *reinterpret_cast<const float4*>(A + k * lda + 4 * ty);
         const float a[4] = {t.x, t.y, t.z, t.w};
         float b[NJ];
-        if constexpr (NJ == 4) {
+        if constexpr (NJ == 8) {
+            const float4 u = *reinterpret_cast<const float4*>(B + k * ldb + 8 * tx);
+            const float4 u2 = *reinterpret_cast<const float4*>(B + k * ldb + 8 * tx + 4);
+            b[0] = u.x; b[1] = u.y; b[2] = u.z; b[3] = u.w; b[4] = u2.x; b[5] = u2.y; b[6] = u2.z; b[7] = u2.w;
+        } else if constexpr (NJ == 4) {
             const float4 u = *reinterpret_cast<const float4*>(B + k * ldb + 4 * tx);
             b[0] = u.x; b[1] = u.y; b[2] = u.z; b[3] = u.w;
         } else {
@@ -400,12 +408,14 @@ __global__ void __launch_bounds__(256) key_side_simt_kernel(KeySideArgs a) {
         }
         __syncthreads();
         // S <- exp(G_C)[:,None] S + K-^T Xv   (thread (ty,tx): slots 4ty.., channels 4tx..)
-        if (4 * ty < M) {
+        // (64 slots per sweep of the 16 x 16 thread grid)
+        for (int s0 = 0; s0 < M; s0 += 64) {
+            if (s0 + 4 * ty >= M) break;
             float acc[4][4] = {};
-            mm_tn<4>(sK, LM, sV, kLd, kC, ty, tx, acc);
+            mm_tn<4>(sK + s0, LM, sV, kLd, kC, ty, tx, acc);
 #pragma unroll
             for (int ii = 0; ii < 4; ++ii) {
-                const int s = 4 * ty + ii;
+                const int s = s0 + 4 * ty + ii;
                 const float e = __expf(sG[(kC - 1) * LM + s]);
 #pragma unroll
                 for (int jj = 0; jj < 4; ++jj)
@@ -452,9 +462,9 @@ cudaError_t launch_value_side_simt(const ValueSideArgs& a, int io, int M, int re
 #define GSA_VS(IO, MM)                                                                   \
     return reverse ? launch_vs<IO, MM, true>(a, st) : launch_vs<IO, MM, false>(a, st)
     if (io == GSA_BF16) {
-        if (M == 64) { GSA_VS(__nv_bfloat16, 64); } else { GSA_VS(__nv_bfloat16, 32); }
+        if (M == 128) { GSA_VS(__nv_bfloat16, 128); } else if (M == 64) { GSA_VS(__nv_bfloat16, 64); } else { GSA_VS(__nv_bfloat16, 32); }
     } else {
-        if (M == 64) { GSA_VS(float, 64); } else { GSA_VS(float, 32); }
+        if (M == 128) { GSA_VS(float, 128); } else if (M == 64) { GSA_VS(float, 64); } else { GSA_VS(float, 32); }
     }
 #undef GSA_VS
 }
@@ -463,9 +473,9 @@ cudaError_t launch_key_side_simt(const KeySideArgs& a, int io, int M, int revers
 #define GSA_KS(IO, MM)                                                                   \
     return reverse ? launch_ks<IO, MM, true>(a, st) : launch_ks<IO, MM, false>(a, st)
     if (io == GSA_BF16) {
-        if (M == 64) { GSA_KS(__nv_bfloat16, 64); } else { GSA_KS(__nv_bfloat16, 32); }
+        if (M == 128) { GSA_KS(__nv_bfloat16, 128); } else if (M == 64) { GSA_KS(__nv_bfloat16, 64); } else { GSA_KS(__nv_bfloat16, 32); }
     } else {
-        if (M == 64) { GSA_KS(float, 64); } else { GSA_KS(float, 32); }
+        if (M == 128) { GSA_KS(float, 128); } else if (M == 64) { GSA_KS(float, 64); } else { GSA_KS(float, 32); }
     }
 #undef GSA_KS
 }

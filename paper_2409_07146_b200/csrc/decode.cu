@@ -180,7 +180,9 @@ static cudaError_t launch_decode_m(const gsa_params_t& p, const IO* q, const IO*
     const unsigned pairs = (unsigned)p.B * (unsigned)p.H;
     const int is_log = p.gate_kind;
     const float inv_tau = p.tau > 0.f ? 1.f / p.tau : 0.f;
-    if (p.m == 64)
+    if (p.m == 128)
+        decode_step_kernel<IO, DK, DV, 128><<<pairs, kDecodeWarps * 32, 0, st>>>(q, k, v, gate, is_log, inv_tau, p.scale, p.slot_act, Ks, Vs, o);
+    else if (p.m == 64)
         decode_step_kernel<IO, DK, DV, 64><<<pairs, kDecodeWarps * 32, 0, st>>>(q, k, v, gate, is_log, inv_tau, p.scale, p.slot_act, Ks, Vs, o);
     else
         decode_step_kernel<IO, DK, DV, 32><<<pairs, kDecodeWarps * 32, 0, st>>>(q, k, v, gate, is_log, inv_tau, p.scale, p.slot_act, Ks, Vs, o);

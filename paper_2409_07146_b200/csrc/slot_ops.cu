@@ -30,7 +30,7 @@ __device__ __forceinline__ void store_split2(__nv_bfloat16* row, int c, float x0
 }
 
 template <int M>
-__global__ void __launch_bounds__(M * 8, 2) gate_cumsum_kernel(const float* __restrict__ gate,
+__global__ void __launch_bounds__(M * 8 > 1024 ? 1024 : M * 8, M > 64 ? 1 : 2) gate_cumsum_kernel(const float* __restrict__ gate,
                                                             int gate_kind, float inv_tau,
                                                             float* __restrict__ G,
                                                             float* __restrict__ I, int T, int H,
@@ -106,11 +106,14 @@ __global__ void __launch_bounds__(M * 8, 2) gate_cumsum_kernel(const float* __re
 cudaError_t launch_gate_cumsum(const float* gate, int gate_kind, float inv_tau, float* G, float* I, int B,
                                int T, int H, int M, int chunk, int* strong_flag, int nseg, void* decayed, int fast_log,
                                cudaStream_t st) {
-    if (chunk % kCumRows != 0 || chunk / kCumRows > 16) return cudaErrorInvalidValue;
+    if (chunk % kCumRows != 0 || chunk / kCumRows > 16 || (M / 2) * (chunk / kCumRows) > 1024) return cudaErrorInvalidValue;
     const int nchunks = (T + chunk - 1) / chunk;
     dim3 block(M / 2, chunk / kCumRows);
     dim3 grid(B * H, nchunks);
-    if (M == 64)
+    if (M == 128)
+        gate_cumsum_kernel<128><<<grid, block, 0, st>>>(gate, gate_kind, inv_tau, G, I, T, H, chunk, strong_flag, nseg < 1 ? 1 : nseg,
+                                                        static_cast<__nv_bfloat16*>(decayed), fast_log);
+    else if (M == 64)
         gate_cumsum_kernel<64><<<grid, block, 0, st>>>(gate, gate_kind, inv_tau, G, I, T, H, chunk, strong_flag, nseg < 1 ? 1 : nseg,
                                                        static_cast<__nv_bfloat16*>(decayed), fast_log);
     else
@@ -229,7 +232,10 @@ cudaError_t launch_slot_softmax_fwd(const float* part, int nslice, float scale, 
     const int rpb = 8 * (128 / M);       // rows per block: 8 warps x 128/M rows
     const dim3 grid((unsigned)((rows_per_batch + rpb - 1) / rpb), (unsigned)B);
     const int rows = rows_per_batch;
-    if (M == 64)
+    if (M == 128)
+        slot_softmax_fwd_kernel<128><<<grid, 256, 0, st>>>(part, nslice, scale, act, ok, p, rows, G,
+                                                           static_cast<__nv_bfloat16*>(p_decayed), pend, m_active);
+    else if (M == 64)
         slot_softmax_fwd_kernel<64><<<grid, 256, 0, st>>>(part, nslice, scale, act, ok, p, rows, G,
                                                           static_cast<__nv_bfloat16*>(p_decayed), pend, m_active);
     else
@@ -338,7 +344,11 @@ cudaError_t launch_slot_softmax_bwd(const float* ok, const float* dp_part, int n
     const int rpb = 8 * (128 / M);       // rows per block: 8 warps x 128/M rows
     const dim3 grid((unsigned)((rows_per_batch + rpb - 1) / rpb), (unsigned)B);
     const int rows = rows_per_batch;
-    if (M == 64)
+    if (M == 128)
+        slot_softmax_bwd_kernel<128><<<grid, 256, 0, st>>>(ok, dp_part, nslice, scale, act, p, dz, u, rows, G,
+                                                           static_cast<__nv_bfloat16*>(p_decayed),
+                                                           static_cast<__nv_bfloat16*>(dz_decayed), pend, m_active);
+    else if (M == 64)
         slot_softmax_bwd_kernel<64><<<grid, 256, 0, st>>>(ok, dp_part, nslice, scale, act, p, dz, u, rows, G,
                                                           static_cast<__nv_bfloat16*>(p_decayed),
                                                           static_cast<__nv_bfloat16*>(dz_decayed), pend, m_active);
@@ -399,19 +409,20 @@ __device__ __forceinline__ void load_dI(const float* __restrict__ dIk, int nsk, 
 // blk_tot[bh][n][s] <- sum over blocks n' > n of the totals, plus the final-memory term.
 // One CTA per (b,h): M slots x 16 segments of consecutive blocks; fp64 running sums.
 template <int M>
-__global__ void __launch_bounds__(M * 16) gate_grad_scan_kernel(
+__global__ void __launch_bounds__(M * (M > 64 ? 8 : 16)) gate_grad_scan_kernel(
     float* __restrict__ blk_tot, const float* __restrict__ dKT, const float* __restrict__ KT,
     const float* __restrict__ dVT, const float* __restrict__ VT, int d_k, int d_v, int nblk) {
-    __shared__ double seg_sum[16][M];
+    constexpr int kSeg = M > 64 ? 8 : 16;       // segments of consecutive blocks (threads: M slots x kSeg)
+    __shared__ double seg_sum[kSeg][M];
     const int s = threadIdx.x, seg = threadIdx.y, bh = blockIdx.x;
-    const int per = (nblk + 15) / 16;
+    const int per = (nblk + kSeg - 1) / kSeg;
     const int lo = seg * per, hi = min(nblk, lo + per);
     double sum = 0.0;
     for (int n = lo; n < hi; ++n) sum += (double)blk_tot[((size_t)bh * nblk + n) * M + s];
     seg_sum[seg][s] = sum;
     // final-memory term <dK~_T[s], K~_T[s]> + <dV~_T[s], V~_T[s]>: a warp per slot, lanes along the row
     __shared__ double final_term[M];
-    const int warp = (seg * M + s) >> 5, lane = (seg * M + s) & 31, nwarp = (M * 16) >> 5;
+    const int warp = (seg * M + s) >> 5, lane = (seg * M + s) & 31, nwarp = (M * kSeg) >> 5;
     for (int slot = warp; slot < M; slot += nwarp) {
         double dot = 0.0;
         if (dKT != nullptr) {
@@ -430,7 +441,7 @@ __global__ void __launch_bounds__(M * 16) gate_grad_scan_kernel(
     }
     __syncthreads();
     double carry = final_term[s];
-    for (int g = seg + 1; g < 16; ++g) carry += seg_sum[g][s];
+    for (int g = seg + 1; g < kSeg; ++g) carry += seg_sum[g][s];
     for (int n = hi - 1; n >= lo; --n) {
         const size_t idx = ((size_t)bh * nblk + n) * M + s;
         const float t = blk_tot[idx];
@@ -821,6 +832,11 @@ cudaError_t launch_gate_grad(const float* u, const float* I, const float* dIk_pa
         }
         gate_grad_scan_kernel<64><<<B * H, dim3(64, 16), 0, st>>>(blk_tot, dKT, KT, dVT, VT, d_k, d_v, nblk);
         gate_grad_carry_kernel<64><<<grid, dim3(block.x, block.y, 2), 0, st>>>(gate, gate_kind, inv_tau, blk_tot, dgate, T, H, nblk);
+    } else if (M == 128) {
+        gate_grad_local_kernel<128><<<grid, block, 0, st>>>(u, I, dIk_part, nsk, dIv_part, nsv, gate, gate_kind, inv_tau,
+                                                            blk_tot, dgate, B, T, H, nblk, pend);
+        gate_grad_scan_kernel<128><<<B * H, dim3(128, 8), 0, st>>>(blk_tot, dKT, KT, dVT, VT, d_k, d_v, nblk);
+        gate_grad_carry_kernel<128><<<grid, dim3(block.x, block.y, 2), 0, st>>>(gate, gate_kind, inv_tau, blk_tot, dgate, T, H, nblk);
     } else {
         gate_grad_local_kernel<32><<<grid, block, 0, st>>>(u, I, dIk_part, nsk, dIv_part, nsv, gate, gate_kind, inv_tau,
                                                            blk_tot, dgate, B, T, H, nblk, pend);

@@ -200,9 +200,22 @@ def test_bwd_strong_forgetting():
     print("bwd strong f32", check_bwd(got, ref, 1.5 * TOL["f32"]))
 
 
+@pytest.mark.parametrize("io", ["f32", "bf16"])
+def test_128_slots_fwd_bwd(io):
+    """m = 128 (the largest slot count of the paper's ablation on the number of slots) runs on the
+    CUDA-core kernels for either io type."""
+    B, T, H, dk, dv, m = 2, 150, 2, 128, 64, 128
+    d = rand_inputs(128 + len(io), B, T, H, dk, dv, m, io, init=True, final_grads=True)
+    got, gate = run_fwd(d, B, T, H, dk, dv, m, io, scale=0.9)
+    check_fwd(d, got, gate, io, scale=0.9)
+    for log in (False, True):
+        gb, rb = run_bwd(d, B, T, H, dk, dv, m, io, scale=0.9, log=log, saved=not log)
+        check_bwd(gb, rb, TOL[io])
+
+
 # ------------------------------------------------------------------ decode
 @pytest.mark.parametrize("io", ["f32", "bf16"])
-@pytest.mark.parametrize("dk,dv,m", [(64, 64, 32), (128, 128, 64), (256, 512, 64), (512, 64, 32)])
+@pytest.mark.parametrize("dk,dv,m", [(64, 64, 32), (128, 128, 64), (256, 512, 64), (512, 64, 32), (128, 256, 128)])
 def test_decode_steps(io, dk, dv, m):
     S, H, steps = 3, 5, 4
     w = W.CONFIGS["decode"].scaled(B=S, H=H, d_k=dk, d_v=dv, m=m, io=io)
