@@ -123,7 +123,7 @@ typedef struct {
     int32_t fuse;       /* gsa_fuse_t; ignored by the fp32 kernels */
 } gsa_params_t;
 
-enum { GSA_WS_FWD = 0, GSA_WS_BWD = 1, GSA_WS_DECODE = 2, GSA_WS_GATE = 3 };
+enum { GSA_WS_FWD = 0, GSA_WS_BWD = 1, GSA_WS_DECODE = 2, GSA_WS_GATE = 3, GSA_WS_SHARD = 4 };
 
 /* Chunk length C of the chunkwise form that these params select (Algorithm 1 leaves C
  * open): 128 for the tensor-core kernels, 64 for the fp32 CUDA-core kernels; 0 for
@@ -243,6 +243,34 @@ GSA_API gsa_status_t gsa_fwd_noalloc(const gsa_params_t* params, const void* q, 
                                      const void* v, const float* gate, const float* K0,
                                      const float* V0, void* o, float* ok_save, float* KT,
                                      float* VT, void* stream, int32_t* dev_status);
+
+/*
+ * Sequence sharding across GPUs (the memories of Eq. 6 are linear in (k, v): the memory after a
+ * stretch of tokens is D * (memory before) + (memory of the stretch run from empty memories), D =
+ * the product of the stretch's gates).  A sequence cut into R shards, one per GPU, therefore needs
+ * ONE exchange: every rank computes the end memories of its shard from empty memories and the
+ * shard's log-decay (gsa_shard_states), the R results are gathered on every rank by the caller
+ * (an all-gather of m (d_k + d_v + 1) floats per (batch, head) and rank, into local memory), every
+ * rank combines them into the memories that enter its shard (gsa_shard_combine) and runs the
+ * ordinary gsa_fwd with those as K0 / V0.  The backward uses the same two calls on the memory
+ * gradients that gsa_bwd returns for a shard (dK0 / dV0 with zero final-memory gradients are the
+ * shard's local contribution; combined from the last shard down with reverse = 1 they give the
+ * dKT / dVT of every shard).  Both calls work on this GPU's memory only.
+ *
+ * gsa_shard_states: k, v, gate of the shard ([B,T,H,.] with T the shard's length) -> KT, VT
+ *   [B,H,m,d] (end memories from EMPTY memories) and logdecay [B,H,m] (sum of log a over the shard).
+ *   ws: gsa_workspace_bytes(params, GSA_WS_SHARD).  32-slot bf16 layers: GSA_ERR_UNSUPPORTED.
+ * gsa_shard_combine: logdecay_all [R,B,H,m] and local_all [R,B,H,m,d] gathered in rank order, S0
+ *   (nullable [B,H,m,d]: the memories before the first shard; reverse: the gradient after the last)
+ *   -> start (nullable): what enters shard `rank` (reverse = 0: from the left; 1: from the right);
+ *   final_state (nullable): what leaves the last shard (reverse: the first).  d = d_k or d_v.
+ */
+GSA_API gsa_status_t gsa_shard_states(const gsa_params_t* params, const void* k, const void* v,
+                                      const float* gate, float* KT, float* VT, float* logdecay,
+                                      void* ws, size_t ws_bytes, void* stream, int32_t* dev_status);
+GSA_API gsa_status_t gsa_shard_combine(const gsa_params_t* params, int32_t d, int32_t nshard, int32_t rank,
+                                       int32_t reverse, const float* logdecay_all, const float* local_all,
+                                       const float* S0, float* start, float* final_state, void* stream);
 
 /*
  * Releases the internal streams and events that this HOST thread's calls created on the current

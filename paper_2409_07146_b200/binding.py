@@ -14,7 +14,7 @@ _lib = None
 GSA_F32, GSA_BF16 = 0, 1
 GSA_GATE_A, GSA_GATE_LOG_A, GSA_GATE_LOGITS = 0, 1, 2
 GSA_IMPL_AUTO, GSA_IMPL_SIMT, GSA_IMPL_TC = 0, 1, 2
-GSA_WS_FWD, GSA_WS_BWD, GSA_WS_DECODE, GSA_WS_GATE = 0, 1, 2, 3
+GSA_WS_FWD, GSA_WS_BWD, GSA_WS_DECODE, GSA_WS_GATE, GSA_WS_SHARD = 0, 1, 2, 3, 4
 
 _IMPL = {"auto": GSA_IMPL_AUTO, "simt": GSA_IMPL_SIMT, "tc": GSA_IMPL_TC}
 _ACT = {"softmax": 0, "none": 1, "relu": 2, "swish": 3, "relu2": 4}   # gsa_act_t
@@ -75,7 +75,7 @@ def exported_symbols():
     return ["gsa_chunk_size", "gsa_workspace_bytes", "gsa_status_string", "gsa_gate_cumsum",
             "gsa_fwd", "gsa_bwd", "gsa_decode_step", "gsa_tc_selftest", "gsa_timing_begin",
             "gsa_timing_end", "gsa_fwd_noalloc", "gsa_fwd_save_gate", "gsa_bwd_saved_gate", "gsa_release_streams",
-            "gsa_wait_selftest"]
+            "gsa_wait_selftest", "gsa_shard_states", "gsa_shard_combine"]
 
 
 def load_library():
@@ -118,6 +118,10 @@ def load_library():
     lib.gsa_tc_selftest.restype = ctypes.c_int
     lib.gsa_wait_selftest.argtypes = [ctypes.c_uint32, vp, vp, vp]
     lib.gsa_wait_selftest.restype = ctypes.c_int
+    lib.gsa_shard_states.argtypes = [pp] + [vp] * 6 + [vp, sz, vp, vp]
+    lib.gsa_shard_states.restype = ctypes.c_int
+    lib.gsa_shard_combine.argtypes = [pp, i32, i32, i32, i32] + [vp] * 5 + [vp]
+    lib.gsa_shard_combine.restype = ctypes.c_int
     lib.gsa_release_streams.argtypes = []
     lib.gsa_release_streams.restype = ctypes.c_int
     _lib = lib
@@ -269,6 +273,38 @@ def gsa_wait_selftest(limit_us: int, dev_status, waited_us=None):
     receives the time it waited."""
     _check(load_library().gsa_wait_selftest(int(limit_us), _stream(), _ptr(dev_status, torch.int32, None, "dev_status"),
                                             _ptr(waited_us, torch.int32, None, "waited_us")), "gsa_wait_selftest")
+
+
+def gsa_shard_states(p: Params, k, v, gate, ws=None, dev_status=None):
+    """End memories of a sequence shard run from empty memories, and the shard's log-decay.
+    Returns (KT [B,H,m,d_k], VT [B,H,m,d_v], logdecay [B,H,m])."""
+    io = p.io_dtype
+    KT = torch.empty(p.B, p.H, p.m, p.d_k, dtype=torch.float32, device=k.device)
+    VT = torch.empty(p.B, p.H, p.m, p.d_v, dtype=torch.float32, device=k.device)
+    ld = torch.empty(p.B, p.H, p.m, dtype=torch.float32, device=k.device)
+    ws, nbytes = _workspace(p, GSA_WS_SHARD, ws, k.device)
+    cp = p.c()
+    _check(load_library().gsa_shard_states(
+        ctypes.byref(cp), _ptr(k, io, (p.B, p.T, p.H, p.d_k), "k"), _ptr(v, io, (p.B, p.T, p.H, p.d_v), "v"),
+        _ptr(gate, torch.float32, (p.B, p.T, p.H, p.m), "gate"), _ptr(KT), _ptr(VT), _ptr(ld),
+        _ptr(ws, torch.uint8, None, "ws"), nbytes, _stream(), _ptr(dev_status, torch.int32, None, "dev_status")),
+        "gsa_shard_states")
+    return KT, VT, ld
+
+
+def gsa_shard_combine(p: Params, d: int, rank: int, logdecay_all, local_all, S0=None, reverse=False, want_final=False):
+    """From the gathered shard results (logdecay_all [R,B,H,m], local_all [R,B,H,m,d], rank order) to the
+    memories entering shard `rank` (and, with want_final, those leaving the last / first shard)."""
+    R = logdecay_all.shape[0]
+    start = torch.empty(p.B, p.H, p.m, d, dtype=torch.float32, device=local_all.device)
+    final = torch.empty_like(start) if want_final else None
+    cp = p.c()
+    _check(load_library().gsa_shard_combine(
+        ctypes.byref(cp), d, R, rank, 1 if reverse else 0,
+        _ptr(logdecay_all, torch.float32, (R, p.B, p.H, p.m), "logdecay_all"),
+        _ptr(local_all, torch.float32, (R, p.B, p.H, p.m, d), "local_all"),
+        _ptr(S0, torch.float32, (p.B, p.H, p.m, d), "S0"), _ptr(start), _ptr(final), _stream()), "gsa_shard_combine")
+    return (start, final) if want_final else start
 
 
 def gsa_release_streams():

@@ -346,8 +346,14 @@ const char* gsa_status_string(gsa_status_t status) {
 
 size_t gsa_workspace_bytes(const gsa_params_t* params, int32_t which) {
     if (which == GSA_WS_DECODE) return 0;
-    if (which != GSA_WS_FWD && which != GSA_WS_BWD && which != GSA_WS_GATE) return 0;
+    if (which != GSA_WS_FWD && which != GSA_WS_BWD && which != GSA_WS_GATE && which != GSA_WS_SHARD) return 0;
     if (check_params(params, true) != GSA_OK) return 0;
+    if (which == GSA_WS_SHARD) {
+        if (pads_slots(*params)) return 0;
+        const size_t esz = params->io == GSA_BF16 ? 2 : 4;
+        return carve(*params, GSA_WS_FWD, nullptr).bytes +
+               align_up((size_t)params->B * params->T * params->H * params->d_v * esz, 256);
+    }
     const gsa_params_t pi = internal_params(*params);
     if (which == GSA_WS_GATE) return carve_gate(pi, nullptr).bytes;
     return carve(pi, which, nullptr).bytes + pad_bytes(*params, which);
@@ -715,6 +721,49 @@ gsa_status_t gsa_decode_step(const gsa_params_t* params, const void* q, const vo
         return GSA_ERR_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     GSA_LAUNCH("decode_step", launch_decode(*params, q, k, v, gate, Kstate, Vstate, o, st));
+    return GSA_OK;
+}
+
+// ---- sequence sharding across GPUs: the two local steps around the exchange of shard memories
+gsa_status_t gsa_shard_states(const gsa_params_t* params, const void* k, const void* v, const float* gate,
+                              float* KT, float* VT, float* logdecay, void* ws, size_t ws_bytes, void* stream,
+                              int32_t* dev_status) {
+    gsa_status_t rc = check_params(params, true);
+    if (rc != GSA_OK) return rc;
+    if (pads_slots(*params)) return GSA_ERR_UNSUPPORTED;
+    if (!ok_ptr(k) || !ok_ptr(v) || !ok_ptr(gate) || !ok_ptr(KT) || !ok_ptr(VT) || !ok_ptr(logdecay)) return GSA_ERR_INVALID_ARG;
+    const gsa_params_t& p = *params;
+    if (ws == nullptr || (reinterpret_cast<uintptr_t>(ws) & 255u) != 0) return GSA_ERR_WORKSPACE;
+    Workspace w = carve(p, GSA_WS_FWD, ws);
+    const size_t esz = p.io == GSA_BF16 ? 2 : 4;
+    const size_t obytes = align_up((size_t)p.B * p.T * p.H * p.d_v * esz, 256);
+    if (ws_bytes < w.bytes + obytes) return GSA_ERR_WORKSPACE;
+    void* oscratch = static_cast<char*>(ws) + w.bytes;      // the scans' token outputs are not wanted: they land here
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // one "segment" per batch element: the whole shard from empty memories, end memories only
+    GSA_CUDA(cudaMemsetAsync(w.strong, 0, sizeof(int) * (size_t)p.B * p.H * segments_of(p), st));
+    GSA_LAUNCH("gate_cumsum", launch_gate_cumsum(gate, p.gate_kind, inv_tau(p), w.G, w.I, p.B, p.T, p.H, p.m, chunk_of(p),
+                                                 w.strong, 1, w.Id, p.io == GSA_BF16, st));
+    GSA_LAUNCH("segment_logdecay", launch_segment_logdecay(w.G, logdecay, p.B, p.T, p.H, p.m, 1, chunk_of(p), st));
+    ValueSideArgs s1{k, k, w.I, w.G, nullptr, KT, w.okpart, p.B, p.T, p.H, p.d_k, w.Id, 1};
+    GSA_LAUNCH("segment_pass1_states", value_side(p, s1, 0, w.strong, st, dev_status));
+    KeySideArgs s2{w.I, w.I, w.G, v, nullptr, VT, oscratch, p.B, p.T, p.H, p.d_v, w.Id, w.Id, 1};
+    GSA_LAUNCH("segment_pass2_states", key_side(p, s2, 0, w.strong, st, dev_status));
+    return GSA_OK;
+}
+
+gsa_status_t gsa_shard_combine(const gsa_params_t* params, int32_t d, int32_t nshard, int32_t rank, int32_t reverse,
+                               const float* logdecay_all, const float* local_all, const float* S0, float* start,
+                               float* final_state, void* stream) {
+    gsa_status_t rc = check_params(params, false);
+    if (rc != GSA_OK) return rc;
+    if (nshard < 1 || rank < 0 || rank >= nshard || d < 1) return GSA_ERR_INVALID_ARG;
+    if (!ok_ptr(logdecay_all) || !ok_ptr(local_all) || !ok_opt(S0) || !ok_opt(start) || !ok_opt(final_state))
+        return GSA_ERR_INVALID_ARG;
+    const gsa_params_t& p = *params;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    GSA_LAUNCH("shard_combine", launch_shard_combine(logdecay_all, local_all, S0, start, final_state, p.B, p.H, p.m, d, nshard,
+                                                     rank, reverse != 0, st));
     return GSA_OK;
 }
 

@@ -168,6 +168,9 @@ cudaError_t launch_segment_logdecay(const float* G, float* seg_logdecay, int B, 
 cudaError_t launch_segment_combine(const float* seg_logdecay, const float* local_end, const float* S0,
                                    float* start, float* final_state, int B, int H, int M, int D, int nseg,
                                    int reverse, cudaStream_t st);
+cudaError_t launch_shard_combine(const float* logdecay_all, const float* local_all, const float* S0, float* start,
+                                 float* final_state, int B, int H, int M, int D, int nshard, int rank, int reverse,
+                                 cudaStream_t st);
 // G, p_decayed / dz_decayed (nullable together; bf16 [rows, 2M]): rows [high | residual] of
 // p exp(G) and dz exp(G), operands of the pipelined tensor-core kernels.
 // (tensors [B, rows_per_batch = T*H, M])

@@ -882,6 +882,8 @@ __global__ void segment_logdecay_kernel(const float* __restrict__ G, float* __re
     double acc = 0.0;
     for (int t = r * Tseg + chunk - 1; t < (r + 1) * Tseg; t += chunk)
         acc += (double)G[(((size_t)b * T + t) * H + h) * M + s];
+    // (a ragged last chunk, possible only when the whole sequence is one segment)
+    if (((r + 1) * Tseg) % chunk != 0) acc += (double)G[(((size_t)b * T + (r + 1) * Tseg - 1) * H + h) * M + s];
     seg_logdecay[(((size_t)b * nseg + r) * H + h) * M + s] = (float)acc;
 }
 
@@ -908,10 +910,39 @@ __global__ void segment_combine_kernel(const float* __restrict__ seg_logdecay, c
     }
 }
 
+// Sequence sharding across GPUs (same linearity): the gathered per-shard log-decays [R,B,H,M] and
+// local end memories [R,B,H,M,D] of all R shards -> the memories entering shard `rank` (from the left;
+// reverse: from the right, for the reversed scans of the backward) and, optionally, the memories after
+// the last shard (reverse: before the first).  S0: what enters the first shard (reverse: the last).
+__global__ void shard_combine_kernel(const float* __restrict__ logdecay_all, const float* __restrict__ local_all,
+                                     const float* __restrict__ S0, float* __restrict__ start, float* __restrict__ final_state,
+                                     int BH, int M, int D, int nshard, int rank, int reverse) {
+    const int bh = blockIdx.x;
+    const int idx = blockIdx.y * blockDim.x + threadIdx.x;
+    if (idx >= M * D) return;
+    const int s = idx / D;
+    float cur = S0 ? S0[(size_t)bh * M * D + idx] : 0.f;
+    for (int i = 0; i < nshard; ++i) {
+        const int r = reverse ? nshard - 1 - i : i;
+        if (r == rank && start != nullptr) start[(size_t)bh * M * D + idx] = cur;
+        const size_t pair = (size_t)r * BH + bh;
+        cur = fmaf(cur, __expf(logdecay_all[pair * M + s]), local_all[pair * M * D + idx]);
+    }
+    if (final_state != nullptr) final_state[(size_t)bh * M * D + idx] = cur;
+}
+cudaError_t launch_shard_combine(const float* logdecay_all, const float* local_all, const float* S0, float* start,
+                                 float* final_state, int B, int H, int M, int D, int nshard, int rank, int reverse,
+                                 cudaStream_t st) {
+    dim3 grid(B * H, (M * D + 255) / 256);
+    shard_combine_kernel<<<grid, 256, 0, st>>>(logdecay_all, local_all, S0, start, final_state, B * H, M, D, nshard, rank, reverse);
+    return cudaGetLastError();
+}
+
 cudaError_t launch_segment_logdecay(const float* G, float* seg_logdecay, int B, int T, int H, int M, int nseg,
                                     int chunk, cudaStream_t st) {
     dim3 grid(B * nseg, H);
-    if (M == 64) segment_logdecay_kernel<64><<<grid, 64, 0, st>>>(G, seg_logdecay, T, H, nseg, chunk);
+    if (M == 128) segment_logdecay_kernel<128><<<grid, 128, 0, st>>>(G, seg_logdecay, T, H, nseg, chunk);
+    else if (M == 64) segment_logdecay_kernel<64><<<grid, 64, 0, st>>>(G, seg_logdecay, T, H, nseg, chunk);
     else segment_logdecay_kernel<32><<<grid, 32, 0, st>>>(G, seg_logdecay, T, H, nseg, chunk);
     return cudaGetLastError();
 }
