@@ -495,6 +495,7 @@ def run_ours(args):
         # ---- decode step (the recurrent form), reported beside the training number
         decode = bench_decode(gsa, torch, dev, pk)
         others = [] if args.no_other_configs else bench_other_configs(gsa, torch, dev, pk, args)
+        decode_loop = None if args.no_other_configs else bench_decode_loop(gsa, torch, dev)
 
         # ---- the oracle on the host cores, bounded sample
         cpu = None
@@ -539,6 +540,7 @@ def run_ours(args):
             "whole_step": whole,
             "kernels": kernels,
             "decode": decode,
+            "decode_loop": decode_loop,
             "configs": others,
             "cpu_baseline": cpu,
         }
@@ -547,6 +549,79 @@ def run_ours(args):
         dist.destroy_process_group()
     if line is not None:
         print(json.dumps(line), flush=True)
+
+
+def run_seq_sharded(args):
+    """--shard seq: every rank holds one T-shard of the same sequences (rank r: tokens [r T, (r+1) T) of a
+    sequence of N T tokens), the shards' end memories are exchanged by one all-gather per direction
+    (NCCL over NVLink; into local memory), everything else is the local step.  Weak scaling in T."""
+    import torch
+    import torch.distributed as dist
+    import __graft_entry__ as entry
+    entry.build()
+    import paper_2409_07146_b200 as gsa
+    from paper_2409_07146_b200 import seqshard
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the GSA library has no CPU path")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    w = rank_workload(rank, args.m)          # (its own seed per rank: a different stretch of the long sequence)
+    x = W.make_inputs(w)
+    p = gsa.Params(w.B, w.T, w.H, w.d_k, w.d_v, w.m, io=w.io)
+    xs = {n: torch.from_numpy(x[n]).to(dev).to(torch.bfloat16) for n in ("q", "k", "v")}
+    xs["gate"] = torch.from_numpy(x["gate"]).to(dev)
+    dO = torch.from_numpy(x["dO"]).to(dev).to(torch.bfloat16)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    eng = seqshard.CudaEngine(p, dev_status=status)
+    gather = seqshard.dist_gather if world > 1 else (lambda t: t.unsqueeze(0).contiguous())
+
+    def step():
+        o, saved = seqshard.sharded_forward(eng, gather, rank, xs, w.d_k, w.d_v)
+        return seqshard.sharded_backward(eng, gather, rank, xs, dO, saved, w.d_k, w.d_v)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    for _ in range(max(args.warmup, 3)):
+        step()
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        step()
+    e1.record()
+    barrier()
+    ms = max_over_ranks(float(e0.elapsed_time(e1)), world, dev) / args.steps
+    clocks = sampler.stop() if rank == 0 else {}
+    if int(status.item()) != 0:
+        raise SystemExit("a bounded device-side wait expired during the benchmark")
+    if rank == 0:
+        exch = 4 * w.B * w.H * w.m * (w.d_k + w.d_v + 1) * 2      # forward and backward all-gather payload per rank
+        print(json.dumps({
+            "metric": METRIC, "value": aggregate_tokens_per_s(world, w.tokens, ms), "unit": UNIT, "n_gpus": world,
+            "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic (seeded)",
+            "config": {"workload": WORKLOAD, "B": w.B, "T_per_rank": w.T, "T_total": w.T * world, "H": w.H, "d_k": w.d_k,
+                       "d_v": w.d_v, "m": w.m, "parallelism": f"sp{world}: sequence sharded over T, one all-gather of shard "
+                       "memories per direction, the backward's local step run twice",
+                       "launch": "plain library calls", "l2": "inputs larger than L2",
+                       "exchange_bytes_per_rank_per_step": exch,
+                       "note": "N > 1 is unmeasured on hardware in this build (single-GPU runs only)" if world == 1 else None},
+            "clocks": clocks, "gpu_launches": None}), flush=True)
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
 
 
 def forward_algorithmic_bytes(w: W.Workload) -> int:
@@ -559,7 +634,8 @@ def bench_other_configs(gsa, torch, dev, pk, args):
     """The other configurations, outside the headline region: plain library calls, CUDA events,
     whole-call time and the fraction of the HBM bound on the bytes every tensor must cross HBM once."""
     out = []
-    plan = [("t2r_7b", True, 10), ("long_keep", False, 10), ("long_forget", False, 5), ("tiny_f32", False, 50)]
+    plan = [("train_2p7b", True, 10), ("t2r_7b", True, 10), ("long_keep", False, 10), ("long_forget", False, 5),
+            ("tiny_f32", False, 50)]
     for name, with_bwd, reps in plan:
         w = W.CONFIGS[name]
         x = W.make_inputs(w)
@@ -671,6 +747,52 @@ def launcher_command(n: int, argv):
             "--master-addr", "127.0.0.1", "--master-port", str(free_port()), os.path.abspath(__file__), *argv]
 
 
+def bench_decode_loop(gsa, torch, dev):
+    """Token-by-token decoding through the GSA layers of the whole 1.3B model: 24 layers, each one
+    gsa_decode_step on its own memories (one sequence, 4 heads of width 512, 64 slots), the 24 steps of a
+    token captured once as a CUDA graph and replayed per token.  Only the GSA layers: no projections,
+    no GLU, no sampling.  The paper's 211 s for 16K tokens is the whole model on one H800 -- context."""
+    w = W.CONFIGS["decode_1p3b"]
+    layers = 24
+    p = gsa.Params(w.B, 1, w.H, w.d_k, w.d_v, w.m, io="bf16")
+    st = W.make_decode_states(w)
+    Ks = [torch.from_numpy(st["K"]).to(dev).clone() for _ in range(layers)]
+    Vs = [torch.from_numpy(st["V"]).to(dev).clone() for _ in range(layers)]
+    xs = W.make_decode_step_inputs(w, 0)
+    q, k, v = (torch.from_numpy(xs[n]).to(dev).to(torch.bfloat16) for n in ("q", "k", "v"))
+    gate = torch.from_numpy(xs["gate"]).to(dev)
+    o = torch.empty(w.B, w.H, w.d_v, dtype=torch.bfloat16, device=dev)
+
+    def token():
+        for l in range(layers):
+            gsa.gsa_decode_step(p, q, k, v, gate, Ks[l], Vs[l], o=o)
+
+    for _ in range(3):
+        token()
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        token()
+    tokens = 2048
+    for _ in range(20):
+        graph.replay()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(tokens):
+        graph.replay()
+    e1.record()
+    torch.cuda.synchronize()
+    us = float(e0.elapsed_time(e1)) * 1e3 / tokens
+    state_bytes = layers * w.H * w.m * (w.d_k + w.d_v) * 4
+    return {"workload": "decode_1p3b: 24 GSA layers x (1 sequence, 4 heads, d=512, m=64), one token at a time",
+            "us_per_token": us, "tokens_per_s": 1e6 / us, "seconds_for_16k_tokens": us * 16384 * 1e-6,
+            "state_bytes": state_bytes, "achieved_gbs": 2 * state_bytes / (us * 1e-6) / 1e9,
+            "launch": "CUDA graph of the 24 decode steps of a token, replayed per token",
+            "paper_context": "whole 1.3B model, 1 x H800, 2K prefix + 16K generated: 211.0 s (another metric: the "
+                             "model's projections, GLU layers and sampling are not in this figure)"}
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -687,6 +809,9 @@ def main():
     ap.add_argument("--slot-act", default="softmax", choices=["softmax", "none", "relu", "swish", "relu2"],
                     help="the non-linearity between the two passes: the paper's softmax (the headline "
                          "workload) or one of the replacements of its ablation")
+    ap.add_argument("--shard", default="batch", choices=["batch", "seq"],
+                    help="how N ranks share the work: batch (the default: every rank its own batch, no collective) or "
+                         "seq (every rank a T-shard of the same sequences, one all-gather of shard memories)")
     ap.add_argument("--m", type=int, default=0, choices=[0, 32, 64, 128],
                     help="slot count on the benchmark shape (default: the workload's 64); 32 runs on the tensor-core "
                          "kernels' 64-slot tiles, 128 on the fp32 CUDA-core kernels")
@@ -704,6 +829,8 @@ def main():
         raise SystemExit(subprocess.call(launcher_command(args.gpus, sys.argv[1:])))
     if args.impl == "reference":
         run_reference(args)
+    elif args.shard == "seq":
+        run_seq_sharded(args)
     else:
         run_ours(args)
 

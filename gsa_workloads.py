@@ -58,6 +58,11 @@ class Workload:
 CONFIGS = {
     "tiny_f32": Workload("tiny_f32", B=1, T=256, H=2, d_k=64, d_v=64, m=32, io="f32", seed=0),
     "train_1p3b": Workload("train_1p3b", B=8, T=2048, H=4, d_k=512, d_v=512, m=64, seed=1),
+    # the 2.7B model's layer: 5 heads of width 512 (model width 2560), otherwise as the 1.3B one
+    "train_2p7b": Workload("train_2p7b", B=8, T=2048, H=5, d_k=512, d_v=512, m=64, seed=5),
+    # decoding with the whole 1.3B model's stack of GSA layers: one sequence, 24 layers of 4 heads of width 512
+    "decode_1p3b": Workload("decode_1p3b", B=1, T=16384, H=4, d_k=512, d_v=512, m=64, seed=6,
+                            init_state=True, with_dO=False),
     "t2r_7b": Workload("t2r_7b", B=4, T=4096, H=32, d_k=128, d_v=128, m=64, seed=2,
                        k_channel_sigma=0.5),
     "long_keep": Workload("long_keep", B=1, T=32768, H=16, d_k=128, d_v=128, m=64, seed=3,
