@@ -121,6 +121,16 @@ typedef struct {
     int32_t slot_act;   /* gsa_act_t; 0 = the paper's softmax */
     int32_t tc_operands; /* gsa_tc_operands_t; ignored by the fp32 kernels */
     int32_t fuse;       /* gsa_fuse_t; ignored by the fp32 kernels */
+    int32_t gate_dtype; /* gsa_dtype_t of the gate tensor: GSA_F32 (0, the default) or GSA_BF16 (meant for
+                         * GSA_GATE_LOG_A and GSA_GATE_LOGITS: bfloat16 cannot tell a = 0.99 from 1, its
+                         * logarithm it can); dgate is fp32 either way */
+    int32_t nseq;       /* packed sequences: number of sequences along T, 0 = none (see cu_seqlens) */
+    const int32_t* cu_seqlens; /* DEVICE pointer to nseq + 1 ascending token offsets, cu_seqlens[0] = 0 and
+                         * cu_seqlens[nseq] = T, or NULL.  Every batch row then holds nseq sequences back
+                         * to back (variable-length batches packed as B = 1): the memories are emptied at
+                         * every offset, so each sequence is an independent recurrence; K0 / V0 enter the
+                         * first sequence, KT / VT leave the last.  gsa_fwd and gsa_bwd only.  The chunks
+                         * that hold an offset run on the strong-decay kernels. */
 } gsa_params_t;
 
 enum { GSA_WS_FWD = 0, GSA_WS_BWD = 1, GSA_WS_DECODE = 2, GSA_WS_GATE = 3, GSA_WS_SHARD = 4 };

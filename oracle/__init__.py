@@ -196,3 +196,35 @@ def decode_step(q, k, v, gate, Kstate, Vstate, *, gate_is_log=False, scale=1.0,
 
     _run_split(run, S * H, threads)
     return o
+
+
+def fwd_packed(q, k, v, gate, cu_seqlens, **kw):
+    """Variable-length batches packed along T: every batch row holds the sequences
+    [cu_seqlens[i], cu_seqlens[i+1]) back to back, each an independent recurrence of Eq. 6 from
+    empty memories (K0 / V0, if given, enter the first one).  Plain definition: one `fwd` call per
+    sequence on its slice.  Returns dict(o, ok, KT, VT) with KT / VT those of the last sequence."""
+    cu = [int(c) for c in cu_seqlens]
+    K0, V0 = kw.pop("K0", None), kw.pop("V0", None)
+    parts = []
+    for i in range(len(cu) - 1):
+        sl = slice(cu[i], cu[i + 1])
+        parts.append(fwd(q[:, sl], k[:, sl], v[:, sl], gate[:, sl], K0=K0 if i == 0 else None,
+                         V0=V0 if i == 0 else None, **kw))
+    return dict(o=np.concatenate([p["o"] for p in parts], axis=1), ok=np.concatenate([p["ok"] for p in parts], axis=1),
+                KT=parts[-1]["KT"], VT=parts[-1]["VT"])
+
+
+def bwd_packed(q, k, v, gate, dO, cu_seqlens, **kw):
+    """Gradients of `fwd_packed`: one `bwd` call per sequence (dKT / dVT, if given, act on the last
+    sequence's final memories; dK0 / dV0 are those of the first sequence's initial memories)."""
+    cu = [int(c) for c in cu_seqlens]
+    K0, V0, dKT, dVT = (kw.pop(n, None) for n in ("K0", "V0", "dKT", "dVT"))
+    n = len(cu) - 1
+    parts = []
+    for i in range(n):
+        sl = slice(cu[i], cu[i + 1])
+        parts.append(bwd(q[:, sl], k[:, sl], v[:, sl], gate[:, sl], dO[:, sl], K0=K0 if i == 0 else None,
+                         V0=V0 if i == 0 else None, dKT=dKT if i == n - 1 else None, dVT=dVT if i == n - 1 else None, **kw))
+    out = {name: np.concatenate([p[name] for p in parts], axis=1) for name in ("dq", "dk", "dv", "dgate")}
+    out["dK0"], out["dV0"] = parts[0]["dK0"], parts[0]["dV0"]
+    return out

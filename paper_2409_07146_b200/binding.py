@@ -32,7 +32,8 @@ class _CParams(ctypes.Structure):
                 ("d_k", ctypes.c_int32), ("d_v", ctypes.c_int32), ("m", ctypes.c_int32),
                 ("io", ctypes.c_int32), ("gate_kind", ctypes.c_int32),
                 ("scale", ctypes.c_float), ("impl", ctypes.c_int32), ("tau", ctypes.c_float),
-                ("slot_act", ctypes.c_int32), ("tc_operands", ctypes.c_int32), ("fuse", ctypes.c_int32)]
+                ("slot_act", ctypes.c_int32), ("tc_operands", ctypes.c_int32), ("fuse", ctypes.c_int32),
+                ("gate_dtype", ctypes.c_int32), ("nseq", ctypes.c_int32), ("cu_seqlens", ctypes.c_void_p)]
 
 
 @dataclass(frozen=True)
@@ -53,6 +54,8 @@ class Params:
     slot_act: str = "softmax"      # "softmax" | "none" | "relu" | "swish" | "relu2"
     tc_operands: str = "paired"    # "paired" | "single" (tensor-core kernels: derived operands as bf16 pairs or not)
     fuse: bool = False             # tensor-core kernels: pass 1 -> softmax -> pass 2 as one kernel where the shape allows (gsa_fuse_t)
+    gate_bf16: bool = False        # the gate tensor is bfloat16 (log a or logits)
+    cu_seqlens: object = None      # packed sequences: int32 CUDA tensor of nseq + 1 offsets along T (kept alive by Params)
 
     def c(self) -> _CParams:
         return _CParams(self.B, self.T, self.H, self.d_k, self.d_v, self.m,
@@ -60,11 +63,18 @@ class Params:
                         GSA_GATE_LOGITS if self.gate_is_logits else
                         (GSA_GATE_LOG_A if self.gate_is_log else GSA_GATE_A),
                         float(self.scale), _IMPL[self.impl], float(self.tau), _ACT[self.slot_act],
-                        0 if self.tc_operands == "paired" else 1, 1 if self.fuse else 0)
+                        0 if self.tc_operands == "paired" else 1, 1 if self.fuse else 0,
+                        GSA_BF16 if self.gate_bf16 else GSA_F32,
+                        0 if self.cu_seqlens is None else int(self.cu_seqlens.numel()) - 1,
+                        None if self.cu_seqlens is None else self.cu_seqlens.data_ptr())
 
     @property
     def io_dtype(self) -> torch.dtype:
         return torch.bfloat16 if self.io == "bf16" else torch.float32
+
+    @property
+    def gate_torch_dtype(self) -> torch.dtype:
+        return torch.bfloat16 if self.gate_bf16 else torch.float32
 
 
 def lib_path() -> str:
@@ -194,7 +204,7 @@ def gsa_fwd(p: Params, q, k, v, gate, K0=None, V0=None, o=None, ok_save=None, KT
     ws, ws_bytes = _workspace(p, GSA_WS_FWD, ws, q.device)
     cp = p.c()
     head = (ctypes.byref(cp), _ptr(q, io, qk, "q"), _ptr(k, io, qk, "k"), _ptr(v, io, vv, "v"),
-            _ptr(gate, torch.float32, mm, "gate"), _ptr(K0, torch.float32, sk, "K0"),
+            _ptr(gate, p.gate_torch_dtype, mm, "gate"), _ptr(K0, torch.float32, sk, "K0"),
             _ptr(V0, torch.float32, sv, "V0"), _ptr(o, io, vv, "o"),
             _ptr(ok_save, torch.float32, mm, "ok_save"), _ptr(KT, torch.float32, sk, "KT"),
             _ptr(VT, torch.float32, sv, "VT"))
@@ -224,7 +234,7 @@ def gsa_bwd(p: Params, q, k, v, gate, dO, K0=None, V0=None, ok_saved=None, dKT=N
     ws, ws_bytes = _workspace(p, GSA_WS_BWD, ws, dev)
     cp = p.c()
     head = (ctypes.byref(cp), _ptr(q, io, qk, "q"), _ptr(k, io, qk, "k"), _ptr(v, io, vv, "v"),
-            _ptr(gate, torch.float32, mm, "gate"), _ptr(K0, torch.float32, sk, "K0"),
+            _ptr(gate, p.gate_torch_dtype, mm, "gate"), _ptr(K0, torch.float32, sk, "K0"),
             _ptr(V0, torch.float32, sv, "V0"), _ptr(ok_saved, torch.float32, mm, "ok_saved"),
             _ptr(dO, io, vv, "dO"), _ptr(dKT, torch.float32, sk, "dKT"),
             _ptr(dVT, torch.float32, sv, "dVT"), _ptr(dq, io, qk, "dq"), _ptr(dk, io, qk, "dk"),
@@ -249,7 +259,7 @@ def gsa_decode_step(p: Params, q, k, v, gate, Kstate, Vstate, o=None):
     cp = p.c()
     _check(load_library().gsa_decode_step(
         ctypes.byref(cp), _ptr(q, io, qk, "q"), _ptr(k, io, qk, "k"), _ptr(v, io, vv, "v"),
-        _ptr(gate, torch.float32, mm, "gate"),
+        _ptr(gate, p.gate_torch_dtype, mm, "gate"),
         _ptr(Kstate, torch.float32, (p.B, p.H, p.m, p.d_k), "Kstate"),
         _ptr(Vstate, torch.float32, (p.B, p.H, p.m, p.d_v), "Vstate"), _ptr(o, io, vv, "o"),
         _stream()), "gsa_decode_step")
@@ -341,7 +351,7 @@ def gsa_fwd_noalloc(p: Params, q, k, v, gate, o, K0=None, V0=None, ok_save=None,
     cp = p.c()
     _check(load_library().gsa_fwd_noalloc(
         ctypes.byref(cp), _ptr(q, io, qk, "q"), _ptr(k, io, qk, "k"), _ptr(v, io, vv, "v"),
-        _ptr(gate, torch.float32, mm, "gate"), _ptr(K0, torch.float32, sk, "K0"),
+        _ptr(gate, p.gate_torch_dtype, mm, "gate"), _ptr(K0, torch.float32, sk, "K0"),
         _ptr(V0, torch.float32, sv, "V0"), _ptr(o, io, vv, "o"),
         _ptr(ok_save, torch.float32, mm, "ok_save"), _ptr(KT, torch.float32, sk, "KT"),
         _ptr(VT, torch.float32, sv, "VT"), _stream(),

@@ -33,6 +33,8 @@ gsa_status_t check_params(const gsa_params_t* p, bool need_T) {
     if (p->impl != GSA_IMPL_AUTO && p->impl != GSA_IMPL_SIMT && p->impl != GSA_IMPL_TC)
         return GSA_ERR_INVALID_ARG;
     if (p->fuse != GSA_FUSE_OFF && p->fuse != GSA_FUSE_ON) return GSA_ERR_INVALID_ARG;
+    if (p->gate_dtype != GSA_F32 && p->gate_dtype != GSA_BF16) return GSA_ERR_INVALID_ARG;
+    if (p->nseq < 0 || (p->nseq == 0) != (p->cu_seqlens == nullptr)) return GSA_ERR_INVALID_ARG;
     if (!(p->scale == p->scale)) return GSA_ERR_INVALID_ARG;
     if (!dim_ok(p->d_k) || !dim_ok(p->d_v)) return GSA_ERR_UNSUPPORTED;
     if (p->m != 32 && p->m != 64 && p->m != 128) return GSA_ERR_UNSUPPORTED;
@@ -308,6 +310,22 @@ PadBuffers carve_pad(const gsa_params_t& p, int which, void* base) {
     return b;
 }
 size_t pad_bytes(const gsa_params_t& p, int which) { return carve_pad(p, which, nullptr).bytes; }
+// a gate tensor given in bfloat16 is widened to fp32 once, into the last part of the workspace
+size_t gate_conv_bytes(const gsa_params_t& p) {
+    return p.gate_dtype == GSA_BF16 ? align_up((size_t)p.B * p.T * p.H * p.m * sizeof(float), 256) : 0;
+}
+// the fp32 gate tensor of this call (the caller's, or its widened copy behind `before` bytes of workspace)
+gsa_status_t gate_as_f32(const gsa_params_t& p, const float* gate, void* ws, size_t ws_bytes, size_t before,
+                         cudaStream_t st, const float** out) {
+    *out = gate;
+    if (p.gate_dtype != GSA_BF16) return GSA_OK;
+    if (ws == nullptr || (reinterpret_cast<uintptr_t>(ws) & 255u) != 0 || ws_bytes < before + gate_conv_bytes(p))
+        return GSA_ERR_WORKSPACE;
+    float* buf = reinterpret_cast<float*>(static_cast<char*>(ws) + before);
+    if (launch_widen_bf16(gate, buf, (size_t)p.B * p.T * p.H * p.m, st) != cudaSuccess) return GSA_ERR_CUDA;
+    *out = buf;
+    return GSA_OK;
+}
 
 #define GSA_CUDA(expr)                                  \
     do {                                                \
@@ -356,7 +374,7 @@ size_t gsa_workspace_bytes(const gsa_params_t* params, int32_t which) {
     }
     const gsa_params_t pi = internal_params(*params);
     if (which == GSA_WS_GATE) return carve_gate(pi, nullptr).bytes;
-    return carve(pi, which, nullptr).bytes + pad_bytes(*params, which);
+    return carve(pi, which, nullptr).bytes + pad_bytes(*params, which) + gate_conv_bytes(*params);
 }
 
 gsa_status_t gsa_gate_cumsum(const gsa_params_t* params, const float* gate, float* G, float* I,
@@ -364,10 +382,12 @@ gsa_status_t gsa_gate_cumsum(const gsa_params_t* params, const float* gate, floa
     gsa_status_t rc = check_params(params, true);
     if (rc != GSA_OK) return rc;
     if (!ok_ptr(gate) || !ok_ptr(G) || !ok_ptr(I)) return GSA_ERR_INVALID_ARG;
+    if (params->gate_dtype != GSA_F32) return GSA_ERR_UNSUPPORTED;      // (this query entry point has no workspace)
     const gsa_params_t& p = *params;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     GSA_LAUNCH("gate_cumsum", launch_gate_cumsum(gate, p.gate_kind, inv_tau(p), G, I, p.B, p.T,
-                                                 p.H, p.m, chunk_of(internal_params(p)), nullptr, 1, nullptr, 0, st));
+                                                 p.H, p.m, chunk_of(internal_params(p)), nullptr, 1, nullptr, 0, st,
+                                                 p.cu_seqlens, p.nseq));
     return GSA_OK;
 }
 
@@ -388,7 +408,8 @@ gsa_status_t fwd_core(const gsa_params_t* params, int m_active, const void* q, c
     const int nseg = segments_of(p);
     GSA_CUDA(cudaMemsetAsync(w.strong, 0, sizeof(int) * (size_t)p.B * p.H * nseg, st));
     GSA_LAUNCH("gate_cumsum", launch_gate_cumsum(gate, p.gate_kind, inv_tau(p), w.G, w.I, p.B, p.T,
-                                                 p.H, p.m, chunk_of(p), w.strong, nseg, w.Id, p.io == GSA_BF16, st));
+                                                 p.H, p.m, chunk_of(p), w.strong, nseg, w.Id, p.io == GSA_BF16, st,
+                                                 p.cu_seqlens, p.nseq));
     float* ok = ok_save;      // the scaled logits leave the softmax kernel only if the caller keeps them
     // the pipelined kernels leave the row factor of the pass-1 sums to the softmax kernel
     const PendingDecay pend = use_tc(p) ? PendingDecay{w.G, w.strong, p.T, p.H, nseg} : PendingDecay{nullptr, nullptr, 1, 1, 1};
@@ -466,6 +487,13 @@ gsa_status_t fwd_impl(const gsa_params_t* params, const void* q, const void* k, 
     if (!ok_ptr(q) || !ok_ptr(k) || !ok_ptr(v) || !ok_ptr(gate) || !ok_ptr(o)) return GSA_ERR_INVALID_ARG;
     if (!ok_opt(K0) || !ok_opt(V0) || !ok_opt(ok_save) || !ok_opt(KT) || !ok_opt(VT))
         return GSA_ERR_INVALID_ARG;
+    {
+        // a bfloat16 gate tensor is widened once; everything downstream reads fp32
+        const gsa_params_t pi0 = internal_params(*params);
+        const size_t before = carve(pi0, GSA_WS_FWD, nullptr).bytes + pad_bytes(*params, GSA_WS_FWD);
+        rc = gate_as_f32(*params, gate, ws, ws_bytes, before, static_cast<cudaStream_t>(stream), &gate);
+        if (rc != GSA_OK) return rc;
+    }
     if (!pads_slots(*params))
         return fwd_core(params, 0, q, k, v, gate, K0, V0, o, ok_save, KT, VT, save_gate, gate_save, gate_save_bytes, ws,
                         ws_bytes, stream, dev_status);
@@ -532,7 +560,8 @@ gsa_status_t bwd_core(const gsa_params_t* params, int m_active, const void* q, c
     if (!gate_is_saved) {      // (a forward of the same call left the gate kernel's products otherwise)
         GSA_CUDA(cudaMemsetAsync(w.strong, 0, sizeof(int) * (size_t)p.B * p.H * nseg, st));
         GSA_LAUNCH("gate_cumsum", launch_gate_cumsum(gate, p.gate_kind, inv_tau(p), w.G, w.I, p.B, p.T,
-                                                     p.H, p.m, chunk_of(p), w.strong, nseg, w.Id, p.io == GSA_BF16, st));
+                                                     p.H, p.m, chunk_of(p), w.strong, nseg, w.Id, p.io == GSA_BF16, st,
+                                                     p.cu_seqlens, p.nseq));
     }
     const float* ok = ok_saved;
     const PendingDecay pend = use_tc(p) ? PendingDecay{w.G, w.strong, p.T, p.H, nseg} : PendingDecay{nullptr, nullptr, 1, 1, 1};
@@ -662,6 +691,12 @@ gsa_status_t bwd_impl(const gsa_params_t* params, const void* q, const void* k, 
     if (!ok_opt(K0) || !ok_opt(V0) || !ok_opt(ok_saved) || !ok_opt(dKT) || !ok_opt(dVT) ||
         !ok_opt(dK0) || !ok_opt(dV0))
         return GSA_ERR_INVALID_ARG;
+    {
+        const gsa_params_t pi0 = internal_params(*params);
+        const size_t before = carve(pi0, GSA_WS_BWD, nullptr).bytes + pad_bytes(*params, GSA_WS_BWD);
+        rc = gate_as_f32(*params, gate, ws, ws_bytes, before, static_cast<cudaStream_t>(stream), &gate);
+        if (rc != GSA_OK) return rc;
+    }
     if (!pads_slots(*params))
         return bwd_core(params, 0, q, k, v, gate, K0, V0, ok_saved, dO, dKT, dVT, dq, dk, dv, dgate, dK0, dV0, gate_is_saved,
                         gate_saved, gate_saved_bytes, ws, ws_bytes, stream, dev_status);
@@ -730,7 +765,7 @@ gsa_status_t gsa_shard_states(const gsa_params_t* params, const void* k, const v
                               int32_t* dev_status) {
     gsa_status_t rc = check_params(params, true);
     if (rc != GSA_OK) return rc;
-    if (pads_slots(*params)) return GSA_ERR_UNSUPPORTED;
+    if (pads_slots(*params) || params->gate_dtype != GSA_F32 || params->cu_seqlens != nullptr) return GSA_ERR_UNSUPPORTED;
     if (!ok_ptr(k) || !ok_ptr(v) || !ok_ptr(gate) || !ok_ptr(KT) || !ok_ptr(VT) || !ok_ptr(logdecay)) return GSA_ERR_INVALID_ARG;
     const gsa_params_t& p = *params;
     if (ws == nullptr || (reinterpret_cast<uintptr_t>(ws) & 255u) != 0) return GSA_ERR_WORKSPACE;

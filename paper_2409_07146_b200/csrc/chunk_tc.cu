@@ -180,8 +180,11 @@ __device__ __forceinline__ void value_side_explicit_rows(const unsigned char* gt
             }
             if (!__any_sync(0xffffffffu, live)) break;
         }
-        float vi[16];
+        float vi[16], vj[16];
         tmem_ld16(tmem_row_addr(tmem, wq, kColO + s0), vi);
+        tmem_ld16(tmem_row_addr(tmem, wq, kColO + kM + s0), vj);       // (the state copy is a high/low pair)
+#pragma unroll
+        for (int e = 0; e < 16; ++e) vi[e] += vj[e];
         if (row < valid) {
 #pragma unroll
             for (int e = 0; e < 16; e += 4) {
@@ -213,12 +216,13 @@ value_side_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_cons
     unsigned char* sXq = smem;                       // 2 panels                                  (32 KB)
     unsigned char* sXk = sXq + 2 * kPanelB;          // 2 panels                                  (32 KB)
     unsigned char* sG = sXk + 2 * kPanelB;           // G tile fp32, [2 stages][2 panels]         (64 KB)
-    unsigned char* sPm = sG + 4 * kPanelB;           // masked P, K-major A, 2 panels             (32 KB)
-    unsigned char* sW = sPm;                         //   ... shared with the weight tile fp32, 2 panels
-    unsigned char* sWa = sPm + 2 * kPanelB;          // decayed weights, bf16 high part, MN-major B [128][64] (16 KB)
+    unsigned char* sW = sG + 4 * kPanelB;            // weight tile fp32, 2 panels                (32 KB)
+    unsigned char* sWa = sW + 2 * kPanelB;           // decayed weights, bf16 high part, MN-major B [128][64] (16 KB)
     unsigned char* sWb = sWa + kPanelB;              // ... their bf16 rounding residual (low part)           (16 KB)
-    unsigned char* sSb = sWb + kPanelB;              // state copy, MN-major B [128][64]          (16 KB)
-    Ctl* ctl = reinterpret_cast<Ctl*>(sSb + kPanelB);
+    unsigned char* sSb = sWb + kPanelB;              // state copy, MN-major B [128][hi 64 | lo 64]  (32 KB)
+    Ctl* ctl = reinterpret_cast<Ctl*>(sSb + 2 * kPanelB);
+    // (the masked P never goes through shared memory: it is rewritten in place in tensor memory as a bf16
+    // high/low pair and read from there as the A operand of the intra-chunk product)
 
     const int tid = threadIdx.x, warp = tid >> 5, wq = warp & 3, half = (tid >> 7) & 1, row = tid & 127;
     const int sb = kHS * half;          // this thread's first slot
@@ -260,16 +264,15 @@ value_side_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_cons
             load_w(0);
             load_x(0);
             constexpr uint32_t idescP = make_idesc(128, 128, false, false);  // xq xk^T
-            constexpr uint32_t idescO = make_idesc(128, kM, false, true);    // xq x state copy (MN-major B)
+            constexpr uint32_t idescO = make_idesc(128, 2 * kM, false, true);  // xq x state copy [S_hi | S_lo] (MN-major B)
             // the high and the low part of the weights are two adjacent 64-column panels of ONE
             // MN-major B operand (N = 128): one product yields [.. W_hi | .. W_lo]
             constexpr uint32_t idescU = make_idesc(128, 2 * kM, true, true);   // xk^T (MN-major A) x [W_hi | W_lo]
-            constexpr uint32_t idescI = make_idesc(128, 2 * kM, false, true);  // Pm x [W_hi | W_lo]
+            constexpr uint32_t idescI = make_idesc(128, 2 * kM, false, true);  // masked P (tensor memory) x [W_hi | W_lo]
             // base descriptors of every operand (K step 0); advancing along K is one add each
             const uint64_t dQk = desc_kmajor(smem_u32(sXq), 0), dKk = desc_kmajor(smem_u32(sXk), 0);
             const uint64_t dKm = desc_mnmajor(smem_u32(sXk), 0, kPanelB), dWa = desc_mnmajor(smem_u32(sWa), 0, kPanelB);
             const uint64_t dS = desc_mnmajor(smem_u32(sSb), 0, kPanelB);
-            const uint64_t dP = desc_kmajor(smem_u32(sPm), 0);
             // byte offset of K step kk: K-major operands walk 32 bytes inside a 64-column panel,
             // MN-major operands walk 16 rows (2048 bytes)
             auto kmaj = [](int kk) { return (uint32_t)((kk >> 2) * kPanelB + (kk & 3) * 32); };
@@ -317,7 +320,12 @@ value_side_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_cons
                     PROF_MARK();
 #pragma unroll
                     for (int kk = 0; kk < kCT / 16; ++kk)
-                        mma_bf16(tmem + kColO2, desc_advance(dP, kmaj(kk)), desc_advance(dWa, mnmaj(kk)), idescI, kk > 0);
+                        mma_bf16_ta(tmem + kColO2, tmem + kColP + 64 * (kk >> 2) + 8 * (kk & 3), desc_advance(dWa, mnmaj(kk)),
+                                    idescI, kk > 0);
+#pragma unroll
+                    for (int kk = 0; kk < kCT / 16; ++kk)      // ... and the rounding residual of the masked P
+                        mma_bf16_ta(tmem + kColO2, tmem + kColP + 64 * (kk >> 2) + 32 + 8 * (kk & 3),
+                                    desc_advance(dWa, mnmaj(kk)), idescI, true);
                     mma_commit(&ctl->bar_mma2);
                     PROF_MARK();
                 }
@@ -353,8 +361,8 @@ value_side_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_cons
 #pragma unroll
         for (int s = 0; s < kHS; ++s) S[s] = (a.S0 && d0 + row < a.D) ? a.S0[((size_t)bh * kM + sb + s) * a.D + d0 + row] : 0.f;
 
-        // bf16 copy of the state for the first chunk's inter-chunk product
-        store_state_row<false>(sSb, row, sb, S, nullptr);
+        // bf16 copy of the state (value + rounding residual) for the first chunk's inter-chunk product
+        store_state_row_split<false>(sSb, sSb + kPanelB, row, sb, S, nullptr);
         fence_async_smem();
         compute_sync();
         if (tid == 0) mbar_arrive(&ctl->bar_sb);
@@ -406,8 +414,7 @@ value_side_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_cons
             tc_fence_after_sync();
             PROF_MARK();
             if (moderate) {
-                store_masked_row<REV, false>(tmem, wq, row, half, sPm, sPm);    // overwrites the weight tile
-                fence_async_smem();
+                mask_row_in_tmem<REV, true>(tmem, wq, row, half, kColP);
                 tc_fence_before_sync();
                 compute_sync();
                 if (tid == 0) mbar_arrive(&ctl->bar_pm);
@@ -446,7 +453,7 @@ value_side_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_cons
             }
             // its bf16 copy feeds the next chunk's inter-chunk product (issued as soon as the next
             // tiles are there); the product of this chunk that read the old copy is complete
-            store_state_row<false>(sSb, row, sb, S, nullptr);
+            store_state_row_split<false>(sSb, sSb + kPanelB, row, sb, S, nullptr);
 
             // ---- output rows of a moderate chunk: exp(+-G_i) * (inter + intra)
             PROF_MARK();
@@ -462,7 +469,13 @@ value_side_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_cons
                 tmem_ld32(tmem_row_addr(tmem, wq, kColO2 + kM + sb), vi);
 #pragma unroll
                 for (int e = 0; e < kHS; ++e) vo[e] += vi[e];          // high + low weight parts
-                tmem_ld32(tmem_row_addr(tmem, wq, kColO + sb), vi);
+                {
+                    float vj[kHS];
+                    tmem_ld32(tmem_row_addr(tmem, wq, kColO + sb), vi);
+                    tmem_ld32(tmem_row_addr(tmem, wq, kColO + kM + sb), vj);
+#pragma unroll
+                    for (int e = 0; e < kHS; ++e) vi[e] += vj[e];      // high + low state parts
+                }
                 // forward: exp(G) (inter + intra); reverse: exp(-G) (exp(G_C) inter + intra)
 #pragma unroll
                 for (int e = 0; e < kHS; ++e) vo[e] = REV ? fmaf(vi[e], ctl->egc[sb + e], vo[e]) : vo[e] + vi[e];
@@ -510,13 +523,14 @@ value_side_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_cons
 
 // Strong-decay chunk of key_side: A_ij = sum_s uq_i[s] uk_j[s] prod a_r[s] on the kept triangle, by
 // the same walk: the thread carries uq_i[s] times the running decay product for its 64 slots, one
-// multiplication per step and slot, and stops once every product is below 2^-40.  Written as the
-// bf16 operand rows of the masked matrix (which shares its buffer with the uq tile: every thread
-// first takes its uq row into registers).  `sG` is replaced by the per-step gates on the way.
+// multiplication per step and slot, and stops once every product is below 2^-40.  Written into tensor
+// memory as the bf16 high/low operand rows of the masked matrix, in the layout mask_row_in_tmem leaves
+// (this thread's 64 columns: 32 packed high parts, then 32 packed residuals).  `sG` is replaced by the
+// per-step gates on the way.
 template <bool REV>
 __device__ __forceinline__ void key_side_explicit_rows(unsigned char* sG, const unsigned char* sUq,
-                                                    const unsigned char* sUk, unsigned char* sAm,
-                                                    unsigned char* sAl, int row, int half, int sb, int grow, int valid) {
+                                                    const unsigned char* sUk, uint32_t tmem, int wq, int row, int half,
+                                                    int sb, int grow, int valid) {
     // thread (row, half) fills columns j in [64 half, 64 half + 63]; its walk starts at the column nearest to
     // the diagonal: j0 = min(row, 64 half + 63) forward, max(row, 64 half) reverse
     const int jlo = 64 * half, jhi = jlo + 63;
@@ -573,11 +587,21 @@ __device__ __forceinline__ void key_side_explicit_rows(unsigned char* sG, const 
             }
         }
     }
+    const int base = kColP + 64 * half;
 #pragma unroll
-    for (int c = 0; c < 8; ++c) {
-        const float xc[8] = {x[8 * c], x[8 * c + 1], x[8 * c + 2], x[8 * c + 3], x[8 * c + 4], x[8 * c + 5], x[8 * c + 6], x[8 * c + 7]};
-        store_chunk_split(sAm + half * kPanelB, sAl + half * kPanelB, row, c, xc);
+    for (int q = 0; q < 2; ++q) {
+        uint32_t hi[16], lo[16];
+#pragma unroll
+        for (int e = 0; e < 16; ++e) {
+            const float x0 = x[32 * q + 2 * e], x1 = x[32 * q + 2 * e + 1];
+            hi[e] = pack_bf16(x0, x1);
+            const __nv_bfloat162 h = *reinterpret_cast<const __nv_bfloat162*>(&hi[e]);
+            lo[e] = pack_bf16(x0 - __bfloat162float(h.x), x1 - __bfloat162float(h.y));
+        }
+        tmem_st16(tmem_row_addr(tmem, wq, base + 16 * q), hi);
+        tmem_st16(tmem_row_addr(tmem, wq, base + 32 + 16 * q), lo);
     }
+    tmem_st_wait();
 }
 
 // ======================================================================================
@@ -597,14 +621,14 @@ key_side_tc_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_consta
     unsigned char* sXv = smem;                       // 2 panels                                   (32 KB)
     unsigned char* sUk = sXv + 2 * kPanelB;          // uk tile fp32, 2 panels                     (32 KB)
     unsigned char* sG = sUk + 2 * kPanelB;           // G tile fp32, 2 panels                      (32 KB)
-    unsigned char* sAm = sG + 2 * kPanelB;           // masked A, K-major A, 2 panels              (32 KB)
-    unsigned char* sUq = sAm;                        //   ... shared with the uq tile fp32, 2 panels
-    unsigned char* sQt = sAm + 2 * kPanelB;          // decayed uq, K-major A [128][64]            (16 KB)
-    unsigned char* sKt = sQt + kPanelB;              // decayed uk, K-major B / MN-major B [128][64] (16 KB)
-                                                     //   ... sQt + sKt also stage the output rows
-    unsigned char* sSb = sKt + kPanelB;              // state copy, K-major B [128 (channel)][64]  (16 KB)
-    unsigned char* sAl = sSb + kPanelB;              // rounding residual of the masked A, 2 panels (32 KB)
-    Ctl* ctl = reinterpret_cast<Ctl*>(sAl + 2 * kPanelB);
+    unsigned char* sUq = sG + 2 * kPanelB;           // uq tile fp32, 2 panels                     (32 KB)
+    unsigned char* sQt = sUq + 2 * kPanelB;          // decayed uq, K-major A [128][64]: value, rounding residual (32 KB)
+                                                     //   ... they also stage the output rows
+    unsigned char* sKt = sQt + 2 * kPanelB;          // decayed uk, K-major / MN-major B [128][64]: value, residual (32 KB)
+    unsigned char* sSb = sKt + 2 * kPanelB;          // state copy, K-major B [128 (channel)][64]: value, residual  (32 KB)
+    Ctl* ctl = reinterpret_cast<Ctl*>(sSb + 2 * kPanelB);
+    // (the masked A never goes through shared memory: it is rewritten in place in tensor memory as a bf16
+    // high/low pair and read from there as the A operand of the intra-chunk product)
 
     const int tid = threadIdx.x, warp = tid >> 5, wq = warp & 3, half = (tid >> 7) & 1, row = tid & 127;
     const int sb = kHS * half;          // this thread's first slot
@@ -645,14 +669,15 @@ key_side_tc_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_consta
             load_v(0);
             constexpr uint32_t idescA = make_idesc(128, 128, false, false);   // Q~ K~^T
             constexpr uint32_t idescO = make_idesc(128, kDST, false, false);  // Q- x state copy (K-major B)
-            constexpr uint32_t idescU = make_idesc(128, kM, true, true);      // xv^T (MN-major A) x K- (MN-major B)
-            constexpr uint32_t idescV = make_idesc(128, kDST, false, true);   // A x xv (MN-major B)
+            constexpr uint32_t idescU = make_idesc(128, 2 * kM, true, true);  // xv^T (MN-major A) x [K-_hi | K-_lo] (MN-major B)
+            constexpr uint32_t idescV = make_idesc(128, kDST, false, true);   // masked A (tensor memory) x xv (MN-major B)
             // base descriptors of every operand (K step 0); advancing along K is one add each
             const uint64_t dV = desc_mnmajor(smem_u32(sXv), 0, kPanelB);
             const uint64_t dQt = desc_kmajor(smem_u32(sQt), 0), dKt = desc_kmajor(smem_u32(sKt), 0);
-            const uint64_t dS = desc_kmajor(smem_u32(sSb), 0);
-            const uint64_t dA = desc_kmajor(smem_u32(sAm), 0), dAl = desc_kmajor(smem_u32(sAl), 0);
-            const uint64_t dKtm = desc_mnmajor(smem_u32(sKt), 0, kPanelB);   // the decayed uk read MN-major
+            const uint64_t dQl = desc_kmajor(smem_u32(sQt + kPanelB), 0), dKl = desc_kmajor(smem_u32(sKt + kPanelB), 0);
+            const uint64_t dS = desc_kmajor(smem_u32(sSb), 0), dSl = desc_kmajor(smem_u32(sSb + kPanelB), 0);
+            // the decayed uk read MN-major, its value and residual as one N = 128 operand
+            const uint64_t dKtm = desc_mnmajor(smem_u32(sKt), 0, kPanelB);
             auto kmaj = [](int kk) { return (uint32_t)((kk >> 2) * kPanelB + (kk & 3) * 32); };
             auto mnmaj = [](int kk) { return (uint32_t)(kk * 2048); };
             for (int it = 0; it < nchunks && !ctl->abort; ++it) {
@@ -662,9 +687,16 @@ key_side_tc_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_consta
                 tc_fence_after_sync();
                 const bool moderate = !GENERAL || ctl->moderate[it & 1] != 0;
                 if (moderate) {
+                    // A = Q- K-^T with both factors as bf16 high/low pairs (the low x low term is dropped)
 #pragma unroll
                     for (int kk = 0; kk < kM / 16; ++kk)
                         mma_bf16(tmem + kColP, desc_advance(dQt, kmaj(kk)), desc_advance(dKt, kmaj(kk)), idescA, kk > 0);
+#pragma unroll
+                    for (int kk = 0; kk < kM / 16; ++kk)
+                        mma_bf16(tmem + kColP, desc_advance(dQl, kmaj(kk)), desc_advance(dKt, kmaj(kk)), idescA, true);
+#pragma unroll
+                    for (int kk = 0; kk < kM / 16; ++kk)
+                        mma_bf16(tmem + kColP, desc_advance(dQt, kmaj(kk)), desc_advance(dKl, kmaj(kk)), idescA, true);
                     mma_commit(&ctl->bar_p);     // the state products below run under the read-out of A
                 }
                 // the decayed uk is read K-major by the intra product and MN-major by the state update
@@ -674,6 +706,12 @@ key_side_tc_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_consta
 #pragma unroll
                 for (int kk = 0; kk < kM / 16; ++kk)
                     mma_bf16(tmem + kColO, desc_advance(dQt, kmaj(kk)), desc_advance(dS, kmaj(kk)), idescO, kk > 0);
+#pragma unroll
+                for (int kk = 0; kk < kM / 16; ++kk)
+                    mma_bf16(tmem + kColO, desc_advance(dQl, kmaj(kk)), desc_advance(dS, kmaj(kk)), idescO, true);
+#pragma unroll
+                for (int kk = 0; kk < kM / 16; ++kk)
+                    mma_bf16(tmem + kColO, desc_advance(dQt, kmaj(kk)), desc_advance(dSl, kmaj(kk)), idescO, true);
                 mma_commit(&ctl->bar_mma1);
                 // a moderate chunk is done with the uk and G tiles: request the next chunk's
                 if (moderate && it + 1 < nchunks) load_kg(it + 1);
@@ -681,13 +719,15 @@ key_side_tc_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_consta
                 tc_fence_after_sync();
 #pragma unroll
                 for (int kk = 0; kk < kCT / 16; ++kk)
-                    mma_bf16(tmem + kColO, desc_advance(dA, kmaj(kk)), desc_advance(dV, mnmaj(kk)), idescV, true);
+                    mma_bf16_ta(tmem + kColO, tmem + kColP + 64 * (kk >> 2) + 8 * (kk & 3), desc_advance(dV, mnmaj(kk)), idescV,
+                                true);
 #pragma unroll
                 for (int kk = 0; kk < kCT / 16; ++kk)      // ... and the rounding residual of A
-                    mma_bf16(tmem + kColO, desc_advance(dAl, kmaj(kk)), desc_advance(dV, mnmaj(kk)), idescV, true);
+                    mma_bf16_ta(tmem + kColO, tmem + kColP + 64 * (kk >> 2) + 32 + 8 * (kk & 3), desc_advance(dV, mnmaj(kk)),
+                                idescV, true);
                 mma_commit(&ctl->bar_mma2);
                 if (!moderate && it + 1 < nchunks) load_kg(it + 1);
-                // the masked A is consumed: its buffer takes the next chunk's uq tile
+                // every product of the chunk is done: the uq and xv tiles may be refilled
                 WAIT_OR_ABORT(&ctl->bar_mma2, it & 1);
                 if (it + 1 < nchunks) {
                     load_q(it + 1);
@@ -745,7 +785,7 @@ key_side_tc_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_consta
                 if (!REV && !moderate) tile_free_row8(&ctl->gc[s0], gcv);
 #pragma unroll
                 for (int e = 0; e < 8; ++e) kd[e] = uk[e] * __expf(REV ? g[e] : gcv[e] - g[e]);
-                store_chunk(sKt, row, s0 >> 3, kd);
+                store_chunk_split(sKt, sKt + kPanelB, row, s0 >> 3, kd);
             }
             PROF_MARK();
             WAIT_OR_ABORT(&ctl->bar_w, it & 1);
@@ -765,10 +805,10 @@ key_side_tc_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_consta
                 if (REV && !moderate) tile_free_row8(&ctl->gc[s0], gcv);
 #pragma unroll
                 for (int e = 0; e < 8; ++e) qd[e] = uq[e] * __expf(REV ? gcv[e] - g[e] : g[e]);
-                store_chunk(sQt, row, s0 >> 3, qd);
+                store_chunk_split(sQt, sQt + kPanelB, row, s0 >> 3, qd);
             }
-            if (REV && moderate) store_state_row<true>(sSb, row, sb, S, ctl->egc);
-            else store_state_row<false>(sSb, row, sb, S, nullptr);
+            if (REV && moderate) store_state_row_split<true>(sSb, sSb + kPanelB, row, sb, S, ctl->egc);
+            else store_state_row_split<false>(sSb, sSb + kPanelB, row, sb, S, nullptr);
             fence_async_smem();
             if (tid == 0) ctl->moderate[it & 1] = moderate;
             compute_sync();
@@ -780,13 +820,12 @@ key_side_tc_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_consta
                 ++n_mod;
                 tc_fence_after_sync();
                 PROF_MARK();
-                store_masked_row<REV, true>(tmem, wq, row, half, sAm, sAl);    // overwrites the uq tile: all rows were read
+                mask_row_in_tmem<REV, true>(tmem, wq, row, half, kColP);
             } else if constexpr (GENERAL) {
-                // Strong decay: A_ij with explicit exponent differences (only the general variant of
-                // the kernel carries this path).
-                if (!a.state_only) key_side_explicit_rows<REV>(sG, sUq, sUk, sAm, sAl, row, half, sb, grow, valid);
+                // Strong decay: A_ij by the walk over the per-step gates (only the general variant of the
+                // kernel carries this path).
+                if (!a.state_only) key_side_explicit_rows<REV>(sG, sUq, sUk, tmem, wq, row, half, sb, grow, valid);
             }
-            fence_async_smem();
             tc_fence_before_sync();
             compute_sync();
             if (tid == 0) mbar_arrive(&ctl->bar_pm);
@@ -797,8 +836,11 @@ key_side_tc_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_consta
             tc_fence_after_sync();
             PROF_MARK();
             {
-                float v[kHS];
+                float v[kHS], vl[kHS];
                 tmem_ld32(tmem_row_addr(tmem, wq, kColU + sb), v);
+                tmem_ld32(tmem_row_addr(tmem, wq, kColU + kM + sb), vl);
+#pragma unroll
+                for (int e = 0; e < kHS; ++e) v[e] += vl[e];          // value + residual of the decayed uk
 #pragma unroll
                 for (int e = 0; e < kHS; e += 4) {
                     const float4 ec = *reinterpret_cast<const float4*>(&ctl->egc[sb + e]);
@@ -853,8 +895,8 @@ key_side_tc_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_consta
     }
 }
 
-constexpr size_t kSmemValueSide = 1024 + 13 * kPanelB + sizeof(Ctl);
-constexpr size_t kSmemKeySide = 1024 + 13 * kPanelB + sizeof(Ctl);
+constexpr size_t kSmemValueSide = 1024 + 14 * kPanelB + sizeof(Ctl);
+constexpr size_t kSmemKeySide = 1024 + 14 * kPanelB + sizeof(Ctl);
 
 }  // namespace
 

@@ -159,7 +159,10 @@ struct PendingDecay {
 // gate_kind: gsa_gate_t (a, log a, or logits with inv_tau = 1/tau)
 cudaError_t launch_gate_cumsum(const float* gate, int gate_kind, float inv_tau, float* G, float* I,
                                int B, int T, int H, int M, int chunk, int* strong_flag, int nseg,
-                               void* decayed, int fast_log, cudaStream_t st);
+                               void* decayed, int fast_log, cudaStream_t st, const int* cu_seqlens = nullptr,
+                               int nseq = 0);
+// n bfloat16 values -> fp32 (a gate tensor given in bfloat16)
+cudaError_t launch_widen_bf16(const void* in, float* out, size_t n, cudaStream_t st);
 // Segment-parallel scheduling (T cut into nseg segments run as independent sequences): per-segment
 // log-decay [B,nseg,H,M] from G, and the start memories [B,nseg,H,M,D] of every segment from the
 // end memories of the segments run from empty memories.

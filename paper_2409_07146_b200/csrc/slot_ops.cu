@@ -29,13 +29,27 @@ __device__ __forceinline__ void store_split2(__nv_bfloat16* row, int c, float x0
     *reinterpret_cast<uint32_t*>(row + M + c) = lo;
 }
 
+// Packed sequences: is token t the first token of a sequence other than the first?  cu holds the
+// nseq + 1 ascending sequence offsets along T (cu[0] = 0, cu[nseq] = T).
+__device__ __forceinline__ bool sequence_starts_at(const int* __restrict__ cu, int nseq, int t) {
+    if (cu == nullptr || t == 0) return false;
+    int lo = 1, hi = nseq - 1;
+    while (lo <= hi) {
+        const int mid = (lo + hi) >> 1, v = cu[mid];
+        if (v == t) return true;
+        if (v < t) lo = mid + 1; else hi = mid - 1;
+    }
+    return false;
+}
+
 template <int M>
 __global__ void __launch_bounds__(M * 8 > 1024 ? 1024 : M * 8, M > 64 ? 1 : 2) gate_cumsum_kernel(const float* __restrict__ gate,
                                                             int gate_kind, float inv_tau,
                                                             float* __restrict__ G,
                                                             float* __restrict__ I, int T, int H,
                                                             int chunk, int* __restrict__ strong_flag, int nseg,
-                                                            __nv_bfloat16* __restrict__ decayed, int fast_log) {
+                                                            __nv_bfloat16* __restrict__ decayed, int fast_log,
+                                                            const int* __restrict__ cu_seqlens, int nseq) {
     __shared__ double group_sum[16][M];
     const int s = 2 * threadIdx.x, grp = threadIdx.y;          // blockDim.y = chunk / 8 <= 16
     const int n = blockIdx.y;
@@ -61,6 +75,9 @@ __global__ void __launch_bounds__(M * 8 > 1024 ? 1024 : M * 8, M > 64 ? 1 : 2) g
         }
         g[i].x = fmaxf(g[i].x, kLogGateMin);
         g[i].y = fmaxf(g[i].y, kLogGateMin);
+        // the first token of a packed sequence drops what the memories carried (its decay is exp(-100) = 0 in
+        // fp32); its own write, 1 - a, is untouched.  The chunk is then flagged for the strong-decay kernels.
+        if (sequence_starts_at(cu_seqlens, nseq, t0 + i)) g[i] = make_float2(kLogGateMin, kLogGateMin);
         if (i < rows) *reinterpret_cast<float2*>(I + base + (size_t)i * stride) = inps[i];
     }
     // running sums: fp32 inside the thread's 8 rows (g becomes the running sum), fp64 across the
@@ -105,20 +122,20 @@ __global__ void __launch_bounds__(M * 8 > 1024 ? 1024 : M * 8, M > 64 ? 1 : 2) g
 
 cudaError_t launch_gate_cumsum(const float* gate, int gate_kind, float inv_tau, float* G, float* I, int B,
                                int T, int H, int M, int chunk, int* strong_flag, int nseg, void* decayed, int fast_log,
-                               cudaStream_t st) {
+                               cudaStream_t st, const int* cu_seqlens, int nseq) {
     if (chunk % kCumRows != 0 || chunk / kCumRows > 16 || (M / 2) * (chunk / kCumRows) > 1024) return cudaErrorInvalidValue;
     const int nchunks = (T + chunk - 1) / chunk;
     dim3 block(M / 2, chunk / kCumRows);
     dim3 grid(B * H, nchunks);
     if (M == 128)
         gate_cumsum_kernel<128><<<grid, block, 0, st>>>(gate, gate_kind, inv_tau, G, I, T, H, chunk, strong_flag, nseg < 1 ? 1 : nseg,
-                                                        static_cast<__nv_bfloat16*>(decayed), fast_log);
+                                                        static_cast<__nv_bfloat16*>(decayed), fast_log, cu_seqlens, nseq);
     else if (M == 64)
         gate_cumsum_kernel<64><<<grid, block, 0, st>>>(gate, gate_kind, inv_tau, G, I, T, H, chunk, strong_flag, nseg < 1 ? 1 : nseg,
-                                                       static_cast<__nv_bfloat16*>(decayed), fast_log);
+                                                       static_cast<__nv_bfloat16*>(decayed), fast_log, cu_seqlens, nseq);
     else
         gate_cumsum_kernel<32><<<grid, block, 0, st>>>(gate, gate_kind, inv_tau, G, I, T, H, chunk, strong_flag, nseg < 1 ? 1 : nseg,
-                                                       static_cast<__nv_bfloat16*>(decayed), fast_log);
+                                                       static_cast<__nv_bfloat16*>(decayed), fast_log, cu_seqlens, nseq);
     return cudaGetLastError();
 }
 
@@ -843,6 +860,24 @@ cudaError_t launch_gate_grad(const float* u, const float* I, const float* dIk_pa
         gate_grad_scan_kernel<32><<<B * H, dim3(32, 16), 0, st>>>(blk_tot, dKT, KT, dVT, VT, d_k, d_v, nblk);
         gate_grad_carry_kernel<32><<<grid, dim3(block.x, block.y, 2), 0, st>>>(gate, gate_kind, inv_tau, blk_tot, dgate, T, H, nblk);
     }
+    return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------ gate tensor in bfloat16
+__global__ void widen_bf16_kernel(const __nv_bfloat16* __restrict__ in, float* __restrict__ out, size_t n) {
+    for (size_t i = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) * 2; i < n; i += (size_t)gridDim.x * blockDim.x * 2) {
+        if (i + 1 < n) {
+            const float2 f = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(in + i));
+            *reinterpret_cast<float2*>(out + i) = f;
+        } else {
+            out[i] = __bfloat162float(in[i]);
+        }
+    }
+}
+cudaError_t launch_widen_bf16(const void* in, float* out, size_t n, cudaStream_t st) {
+    const size_t pairs = (n + 1) / 2;
+    const unsigned blocks = (unsigned)((pairs + 255) / 256 < 148 * 32 ? (pairs + 255) / 256 : 148 * 32);
+    widen_bf16_kernel<<<blocks ? blocks : 1, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(in), out, n);
     return cudaGetLastError();
 }
 

@@ -129,9 +129,7 @@ def run_training_config(name, with_bwd, tc_operands="paired", launch="plain"):
         if e["plain_ceiling"] is not None and e["plain"] > e["plain_ceiling"]:
             bad[n] = e
         # a bfloat16-stored tensor is the oracle's value rounded to bfloat16, or its neighbour
-        # (not asserted for long_forget: its pairs run in the general kernels, whose derived operands
-        # are single bfloat16 values -- 4 ulps measured there)
-        if n in BF16_IO and tc_operands == "paired" and name != "long_forget" and (
+        if n in BF16_IO and tc_operands == "paired" and (
                 e["ulps_from_rounded_oracle"] > 1.0 or e["bit_equal_to_rounded_oracle"] < 0.95):
             bad[n] = e
     assert not bad, bad

@@ -14,8 +14,7 @@ pytestmark = pytest.mark.gpu
 # A bfloat16-stored result must be the oracle's value rounded to bfloat16 or a neighbour of it
 # (bf16_storage_check).  At the size of the benchmark configurations the largest distance measured
 # is one ulp; the small stress shapes here (initial and final memories with their gradients) reach
-# two.  Not asserted where strong forgetting sends a (batch, head) pair to the general kernels,
-# whose derived operands are single bfloat16 values: those are held to the stated tolerance only.
+# two.  It holds on the strong-decay kernels too (they carry the same operand pairs).
 STORAGE_ULPS = 2.0
 
 
@@ -101,7 +100,7 @@ def test_fwd_strong_forgetting_and_exact_zero_one_gates(impl, gate, log):
     d = rand_inputs(11, B, T, H, dk, dv, m, io, init=True, gate=gate)
     got, g = run_fwd(d, B, T, H, dk, dv, m, io, impl=impl, log=log)
     gref = np.maximum(g.astype(np.float64), -100.0) if log else g
-    check_fwd(d, got, gref, io, log=log, storage=False)
+    check_fwd(d, got, gref, io, log=log)
 
 
 def test_fwd_tiny_config_fp32():
@@ -305,7 +304,7 @@ def test_fwd_tc_strong_forgetting(gate, log):
     d = rand_inputs(13, B, T, H, dk, dv, m, "bf16", init=True, gate=gate)
     got, g = run_fwd(d, B, T, H, dk, dv, m, "bf16", impl="tc", log=log)
     gref = np.maximum(g.astype(np.float64), -100.0) if log else g
-    check_fwd(d, got, gref, "bf16", log=log, tc=True, storage=False)
+    check_fwd(d, got, gref, "bf16", log=log, tc=True)
 
 
 @pytest.mark.parametrize("gate", ["tau8", "mixed"])
@@ -319,7 +318,7 @@ def test_fwd_tc_segment_parallel_schedule(gate, init):
         d["gate"][:, :2048, :, 2] = 0.99
         d["gate"][:, 3072:, :, 2] = 0.99
     got, g = run_fwd(d, B, T, H, dk, dv, m, "bf16", impl="tc", scale=0.7)
-    errs = check_fwd(d, got, g, "bf16", scale=0.7, tc=True, storage=gate != "mixed")
+    errs = check_fwd(d, got, g, "bf16", scale=0.7, tc=True)
     print("segment-parallel fwd", errs)
 
 
@@ -337,7 +336,7 @@ def test_bwd_tc_segment_parallel_schedule(strong_segment, saved):
     # (gates of 1e-3 are passed as log a: the gradient w.r.t. a itself is d(log a) / a - dI, and the
     # division amplifies the fp32 noise of the whole-sequence sum by 1 / a)
     got, ref = run_bwd(d, B, T, H, dk, dv, m, "bf16", impl="tc", scale=0.7, saved=saved, log=strong_segment)
-    errs = check_bwd(got, ref, TOL["bf16"], tc=True, storage=not strong_segment)
+    errs = check_bwd(got, ref, TOL["bf16"], tc=True)
     print("segment-parallel bwd", strong_segment, saved, errs)
 
 
@@ -415,11 +414,9 @@ def test_bwd_tc_strong_forgetting_saved_logits():
     d = rand_inputs(45, B, T, H, dk, dv, m, "bf16", gate="strong")
     got, ref = run_bwd(d, B, T, H, dk, dv, m, "bf16", impl="tc", log=True, saved=True)
     # with a ~ 0.05 the input gate 1 - a is ~ 1 and the three terms of the gate gradient
-    # (p dp + o' do' - (1-a) dI) cancel almost completely; the general kernels, which take pairs
-    # with strong-decay chunks, carry their derived operands as single bfloat16 values, and their
-    # roundings are what is left: dq, dk 1.3e-2, gate gradient 4.8e-2 measured.  Held to 3x the
-    # stated bound on this stress case only.
-    print("bwd tc strong saved", check_bwd(got, ref, 3 * TOL["bf16"], tc=True, storage=False))
+    # (p dp + o' do' - (1-a) dI) cancel almost completely: a stress case for the operand pairs of the
+    # kernels that take the strong-decay chunks (4e-4 measured on the gate gradient, 4e-5 on dq / dk)
+    print("bwd tc strong saved", check_bwd(got, ref, TOL["bf16"], tc=True))
 
 
 # ------------------------------------------------------------------ gate from logits (Sec. 3.3)
@@ -552,3 +549,73 @@ def test_bwd_with_the_forwards_saved_gate_block_is_the_same_backward(io, impl, T
     ref = oracle.bwd(d["q"], d["k"], d["v"], d["gate"], d["dO"], K0=d["K0"], V0=d["V0"], dKT=d["dKT"],
                      dVT=d["dVT"], scale=0.8)
     assert rel_err(outs[1][4], ref["dgate"]) <= TOL[io]
+
+
+# ------------------------------------------------------------------ packed sequences, bfloat16 gates
+@pytest.mark.parametrize("io,impl", [("f32", "auto"), ("bf16", "tc")])
+def test_packed_variable_length_sequences_fwd_bwd(io, impl):
+    """Several sequences back to back along T (offsets inside chunks, at a chunk boundary, a sequence of
+    one token): the memories are emptied at every offset, so every sequence matches its own recurrence."""
+    B, T, H, dk, dv, m = 2, 700, 2, 128, 128, 64
+    d = rand_inputs(333, B, T, H, dk, dv, m, io, init=True, final_grads=True)
+    cu_list = [0, 100, 101, 256, 300, 512, 700]
+    cu = torch.tensor(cu_list, dtype=torch.int32, device="cuda")
+    p = gsa.Params(B, T, H, dk, dv, m, io=io, impl=impl, scale=0.9, cu_seqlens=cu)
+    q, k, v, dO = (to_dev(d[n], io) for n in ("q", "k", "v", "dO"))
+    gate, K0, V0, dKT, dVT = (to_dev(d[n]) for n in ("gate", "K0", "V0", "dKT", "dVT"))
+    ok = torch.empty(B, T, H, m, device="cuda")
+    KT = torch.empty(B, H, m, dk, device="cuda"); VT = torch.empty(B, H, m, dv, device="cuda")
+    o = gsa.gsa_fwd(p, q, k, v, gate, K0, V0, ok_save=ok, KT=KT, VT=VT)
+    dK0 = torch.empty_like(KT); dV0 = torch.empty_like(VT)
+    dq, dk_, dv_, dg = gsa.gsa_bwd(p, q, k, v, gate, dO, K0, V0, ok_saved=ok, dKT=dKT, dVT=dVT, dK0=dK0, dV0=dV0)
+    torch.cuda.synchronize()
+    rf = oracle.fwd_packed(d["q"], d["k"], d["v"], d["gate"], cu_list, K0=d["K0"], V0=d["V0"], scale=0.9)
+    rb = oracle.bwd_packed(d["q"], d["k"], d["v"], d["gate"], d["dO"], cu_list, K0=d["K0"], V0=d["V0"], dKT=d["dKT"],
+                           dVT=d["dVT"], scale=0.9)
+    got = dict(o=to_np(o), ok=to_np(ok), KT=to_np(KT), VT=to_np(VT), dq=to_np(dq), dk=to_np(dk_), dv=to_np(dv_),
+               dgate=to_np(dg), dK0=to_np(dK0), dV0=to_np(dV0))
+    ref = dict(rf, **rb)
+    errs = {n: rel_err(got[n], ref[n], io == "bf16" and n in BF16_IO) for n in got}
+    print("packed", io, {n: float("%.2g" % e) for n, e in errs.items()})
+    assert all(np.isfinite(got[n]).all() for n in got)
+    assert all(e <= TOL[io] for e in errs.values()), errs
+
+
+@pytest.mark.parametrize("kind", ["log", "logits"])
+def test_gate_tensor_in_bfloat16(kind):
+    """The gate as a bfloat16 tensor (log a or the layer's logits): widened once at the boundary; the
+    oracle sees the same bfloat16-rounded values."""
+    B, T, H, dk, dv, m = 2, 300, 2, 128, 128, 64
+    d = rand_inputs(71, B, T, H, dk, dv, m, "bf16", init=True)
+    r = np.random.default_rng(2)
+    if kind == "log":
+        g32 = np.log(d["gate"].astype(np.float64)).astype(np.float32)
+    else:
+        g32 = (2.0 * r.standard_normal((B, T, H, m))).astype(np.float32)
+    g16 = W.round_to_bf16(g32)
+    p = gsa.Params(B, T, H, dk, dv, m, io="bf16", impl="tc", gate_is_log=kind == "log", gate_is_logits=kind == "logits",
+                   tau=8.0, gate_bf16=True)
+    q, k, v, dO = (to_dev(d[n], "bf16") for n in ("q", "k", "v", "dO"))
+    gate = to_dev(g16).to(torch.bfloat16)
+    K0, V0 = to_dev(d["K0"]), to_dev(d["V0"])
+    ok = torch.empty(B, T, H, m, device="cuda")
+    o = gsa.gsa_fwd(p, q, k, v, gate, K0, V0, ok_save=ok)
+    dq, dk_, dv_, dg = gsa.gsa_bwd(p, q, k, v, gate, dO, K0, V0, ok_saved=ok)
+    torch.cuda.synchronize()
+    assert dg.dtype == torch.float32
+    kw = dict(gate_is_log=kind == "log", gate_is_logits=kind == "logits", tau=8.0, K0=d["K0"], V0=d["V0"])
+    rf = oracle.fwd(d["q"], d["k"], d["v"], g16, **kw)
+    rb = oracle.bwd(d["q"], d["k"], d["v"], g16, d["dO"], **kw)
+    got = dict(o=to_np(o), ok=to_np(ok), dq=to_np(dq), dk=to_np(dk_), dv=to_np(dv_), dgate=to_np(dg))
+    ref = dict(rf, **rb)
+    errs = {n: rel_err(got[n], ref[n], n in BF16_IO) for n in got}
+    assert all(e <= TOL["bf16"] for e in errs.values()), errs
+    # decode reads the bfloat16 gate directly
+    pd = gsa.Params(B, 1, H, dk, dv, m, io="bf16", gate_is_log=kind == "log", gate_is_logits=kind == "logits", tau=8.0,
+                    gate_bf16=True)
+    Ks, Vs = to_dev(d["K0"]).clone(), to_dev(d["V0"]).clone()
+    Kr, Vr = d["K0"].astype(np.float64), d["V0"].astype(np.float64)
+    od = gsa.gsa_decode_step(pd, q[:, 0].contiguous(), k[:, 0].contiguous(), v[:, 0].contiguous(), gate[:, 0].contiguous(), Ks, Vs)
+    ro = oracle.decode_step(d["q"][:, 0], d["k"][:, 0], d["v"][:, 0], g16[:, 0], Kr, Vr, gate_is_log=kind == "log",
+                            gate_is_logits=kind == "logits", tau=8.0)
+    assert rel_err(to_np(od), ro, True) <= TOL["bf16"] and rel_err(to_np(Ks), Kr) <= 1e-5

@@ -369,3 +369,42 @@ def test_slot_activation_relations_and_decode():
         o = oracle.decode_step(q[:, t], k[:, t], v[:, t], a[:, t], Ks, Vs, scale=0.7, act="swish")
         np.testing.assert_allclose(o, full["o"][:, t], atol=1e-14)
     np.testing.assert_allclose(Ks, full["KT"], atol=1e-14)
+
+
+# ---------------------------------------------------------------- packed sequences
+def test_packed_sequences_match_the_unrolled_form_of_every_sequence_and_finite_differences():
+    """fwd_packed / bwd_packed (variable-length sequences back to back along T, memories emptied at
+    every offset): each sequence against the brute-force unrolled form on its own slice, and the
+    assembled gradients (which sequence receives K0 / dKT) against central finite differences."""
+    q, k, v, a, K0, V0 = rand_problem(31, T=19, H=2, dk=4, dv=3, m=3, init=True)
+    cu = [0, 5, 6, 14, 19]
+    r = oracle.fwd_packed(q, k, v, a, cu, K0=K0, V0=V0, scale=0.7)
+    for i in range(len(cu) - 1):
+        sl = slice(cu[i], cu[i + 1])
+        for h in range(2):
+            o, logits, KT, VT = unrolled.gsa_unrolled(q[0, sl, h], k[0, sl, h], v[0, sl, h], a[0, sl, h],
+                                                      K0[0, h] if i == 0 else None, V0[0, h] if i == 0 else None, 0.7)
+            np.testing.assert_allclose(r["o"][0, sl, h], o.numpy(), rtol=1e-10, atol=1e-12)
+            np.testing.assert_allclose(r["ok"][0, sl, h], logits.numpy(), rtol=1e-10, atol=1e-12)
+            if i == len(cu) - 2:
+                np.testing.assert_allclose(r["KT"][0, h], KT.numpy(), rtol=1e-10, atol=1e-12)
+    rng = np.random.default_rng(5)
+    dO = rng.standard_normal(v.shape)
+    dKT, dVT = rng.standard_normal(K0.shape), rng.standard_normal(V0.shape)
+
+    def loss(q_, k_, v_, a_, K0_, V0_):
+        f = oracle.fwd_packed(q_, k_, v_, a_, cu, K0=K0_, V0=V0_, scale=0.7)
+        return float((f["o"] * dO).sum() + (f["KT"] * dKT).sum() + (f["VT"] * dVT).sum())
+
+    g = oracle.bwd_packed(q, k, v, a, dO, cu, K0=K0, V0=V0, dKT=dKT, dVT=dVT, scale=0.7)
+    args = [q, k, v, a, K0, V0]
+    eps = 1e-6
+    for pos, name in ((0, "dq"), (1, "dk"), (2, "dv"), (3, "dgate"), (4, "dK0"), (5, "dV0")):
+        x = args[pos]
+        for _ in range(6):
+            idx = tuple(rng.integers(0, n) for n in x.shape)
+            hi, lo = [t.copy() for t in args], [t.copy() for t in args]
+            hi[pos][idx] += eps
+            lo[pos][idx] -= eps
+            fd = (loss(*hi) - loss(*lo)) / (2 * eps)
+            assert abs(fd - g[name][idx]) <= 1e-6 * max(1.0, abs(fd)), (name, idx, fd, g[name][idx])
