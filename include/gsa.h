@@ -111,6 +111,12 @@ typedef enum {
                           * to the separate kernels. */
 } gsa_fuse_t;
 
+/* The layer's feature map on q, k, v (Sec. 3.3: q, k, v = Swish(W x)): with GSA_FEAT_SWISH the q, k, v
+ * tensors hold the projections' outputs and Swish is applied by the library (one pass over q, k, v
+ * in gsa_fwd and gsa_bwd, whose dq, dk, dv are then gradients w.r.t. those pre-activations; at load
+ * in gsa_decode_step). */
+typedef enum { GSA_FEAT_NONE = 0, GSA_FEAT_SWISH = 1 } gsa_feature_map_t;
+
 typedef struct {
     int32_t B, T, H, d_k, d_v, m;
     int32_t io;         /* gsa_dtype_t */
@@ -124,6 +130,7 @@ typedef struct {
     int32_t gate_dtype; /* gsa_dtype_t of the gate tensor: GSA_F32 (0, the default) or GSA_BF16 (meant for
                          * GSA_GATE_LOG_A and GSA_GATE_LOGITS: bfloat16 cannot tell a = 0.99 from 1, its
                          * logarithm it can); dgate is fp32 either way */
+    int32_t feature_map; /* gsa_feature_map_t */
     int32_t nseq;       /* packed sequences: number of sequences along T, 0 = none (see cu_seqlens) */
     const int32_t* cu_seqlens; /* DEVICE pointer to nseq + 1 ascending token offsets, cu_seqlens[0] = 0 and
                          * cu_seqlens[nseq] = T, or NULL.  Every batch row then holds nseq sequences back
@@ -253,6 +260,20 @@ GSA_API gsa_status_t gsa_fwd_noalloc(const gsa_params_t* params, const void* q, 
                                      const void* v, const float* gate, const float* K0,
                                      const float* V0, void* o, float* ok_save, float* KT,
                                      float* VT, void* stream, int32_t* dev_status);
+
+/*
+ * The layer's output path (Sec. 3.3: y = W_o RMSNorm(Swish(concat_h o^h))), element-wise part:
+ *   y = w * x / sqrt(mean(x^2) + eps),  x = Swish(o),  mean over the H d_v values of a token.
+ * o, y, dy, d_o: [B,T,H,d_v] of the io type; weight (nullable = ones), dweight (nullable): [H d_v] fp32.
+ * H d_v must not exceed 4096 (bf16) / 2048 (fp32).  gsa_out_norm_bwd recomputes the norm from o; with
+ * dweight != NULL it needs ws of gsa_out_norm_workspace_bytes(params) bytes (256-byte aligned) for the
+ * per-block partial sums of the weight gradient, added in a fixed order (deterministic).
+ */
+GSA_API gsa_status_t gsa_out_norm_fwd(const gsa_params_t* params, const void* o, const float* weight, float eps,
+                                      void* y, void* stream);
+GSA_API size_t gsa_out_norm_workspace_bytes(const gsa_params_t* params);
+GSA_API gsa_status_t gsa_out_norm_bwd(const gsa_params_t* params, const void* o, const void* dy, const float* weight,
+                                      float eps, void* d_o, float* dweight, void* ws, size_t ws_bytes, void* stream);
 
 /*
  * Sequence sharding across GPUs (the memories of Eq. 6 are linear in (k, v): the memory after a

@@ -33,7 +33,8 @@ class _CParams(ctypes.Structure):
                 ("io", ctypes.c_int32), ("gate_kind", ctypes.c_int32),
                 ("scale", ctypes.c_float), ("impl", ctypes.c_int32), ("tau", ctypes.c_float),
                 ("slot_act", ctypes.c_int32), ("tc_operands", ctypes.c_int32), ("fuse", ctypes.c_int32),
-                ("gate_dtype", ctypes.c_int32), ("nseq", ctypes.c_int32), ("cu_seqlens", ctypes.c_void_p)]
+                ("gate_dtype", ctypes.c_int32), ("feature_map", ctypes.c_int32), ("nseq", ctypes.c_int32),
+                ("cu_seqlens", ctypes.c_void_p)]
 
 
 @dataclass(frozen=True)
@@ -55,6 +56,7 @@ class Params:
     tc_operands: str = "paired"    # "paired" | "single" (tensor-core kernels: derived operands as bf16 pairs or not)
     fuse: bool = False             # tensor-core kernels: pass 1 -> softmax -> pass 2 as one kernel where the shape allows (gsa_fuse_t)
     gate_bf16: bool = False        # the gate tensor is bfloat16 (log a or logits)
+    feature_map: str = "none"      # "none" | "swish": q, k, v hold pre-activations, Swish applied by the library
     cu_seqlens: object = None      # packed sequences: int32 CUDA tensor of nseq + 1 offsets along T (kept alive by Params)
 
     def c(self) -> _CParams:
@@ -64,7 +66,7 @@ class Params:
                         (GSA_GATE_LOG_A if self.gate_is_log else GSA_GATE_A),
                         float(self.scale), _IMPL[self.impl], float(self.tau), _ACT[self.slot_act],
                         0 if self.tc_operands == "paired" else 1, 1 if self.fuse else 0,
-                        GSA_BF16 if self.gate_bf16 else GSA_F32,
+                        GSA_BF16 if self.gate_bf16 else GSA_F32, 1 if self.feature_map == "swish" else 0,
                         0 if self.cu_seqlens is None else int(self.cu_seqlens.numel()) - 1,
                         None if self.cu_seqlens is None else self.cu_seqlens.data_ptr())
 
@@ -85,7 +87,8 @@ def exported_symbols():
     return ["gsa_chunk_size", "gsa_workspace_bytes", "gsa_status_string", "gsa_gate_cumsum",
             "gsa_fwd", "gsa_bwd", "gsa_decode_step", "gsa_tc_selftest", "gsa_timing_begin",
             "gsa_timing_end", "gsa_fwd_noalloc", "gsa_fwd_save_gate", "gsa_bwd_saved_gate", "gsa_release_streams",
-            "gsa_wait_selftest", "gsa_shard_states", "gsa_shard_combine"]
+            "gsa_wait_selftest", "gsa_shard_states", "gsa_shard_combine", "gsa_out_norm_fwd",
+            "gsa_out_norm_workspace_bytes", "gsa_out_norm_bwd"]
 
 
 def load_library():
@@ -132,6 +135,12 @@ def load_library():
     lib.gsa_shard_states.restype = ctypes.c_int
     lib.gsa_shard_combine.argtypes = [pp, i32, i32, i32, i32] + [vp] * 5 + [vp]
     lib.gsa_shard_combine.restype = ctypes.c_int
+    lib.gsa_out_norm_fwd.argtypes = [pp, vp, vp, ctypes.c_float, vp, vp]
+    lib.gsa_out_norm_fwd.restype = ctypes.c_int
+    lib.gsa_out_norm_workspace_bytes.argtypes = [pp]
+    lib.gsa_out_norm_workspace_bytes.restype = sz
+    lib.gsa_out_norm_bwd.argtypes = [pp, vp, vp, vp, ctypes.c_float, vp, vp, vp, sz, vp]
+    lib.gsa_out_norm_bwd.restype = ctypes.c_int
     lib.gsa_release_streams.argtypes = []
     lib.gsa_release_streams.restype = ctypes.c_int
     _lib = lib
@@ -315,6 +324,34 @@ def gsa_shard_combine(p: Params, d: int, rank: int, logdecay_all, local_all, S0=
         _ptr(local_all, torch.float32, (R, p.B, p.H, p.m, d), "local_all"),
         _ptr(S0, torch.float32, (p.B, p.H, p.m, d), "S0"), _ptr(start), _ptr(final), _stream()), "gsa_shard_combine")
     return (start, final) if want_final else start
+
+
+def gsa_out_norm_fwd(p: Params, o, weight=None, eps=1e-6, y=None):
+    """y = weight * Swish(o) / sqrt(mean(Swish(o)^2) + eps) over the H d_v values of every token."""
+    io = p.io_dtype
+    shp = (p.B, p.T, p.H, p.d_v)
+    if y is None:
+        y = torch.empty(shp, dtype=io, device=o.device)
+    cp = p.c()
+    _check(load_library().gsa_out_norm_fwd(ctypes.byref(cp), _ptr(o, io, shp, "o"),
+                                           _ptr(weight, torch.float32, (p.H * p.d_v,), "weight"), float(eps),
+                                           _ptr(y, io, shp, "y"), _stream()), "gsa_out_norm_fwd")
+    return y
+
+
+def gsa_out_norm_bwd(p: Params, o, dy, weight=None, eps=1e-6, want_dweight=True):
+    """Gradients of gsa_out_norm_fwd: returns (d_o, dweight or None)."""
+    io = p.io_dtype
+    shp = (p.B, p.T, p.H, p.d_v)
+    d_o = torch.empty(shp, dtype=io, device=o.device)
+    dw = torch.empty(p.H * p.d_v, dtype=torch.float32, device=o.device) if want_dweight else None
+    cp = p.c()
+    nbytes = int(load_library().gsa_out_norm_workspace_bytes(ctypes.byref(cp))) if want_dweight else 0
+    ws = torch.empty(max(nbytes, 256), dtype=torch.uint8, device=o.device)
+    _check(load_library().gsa_out_norm_bwd(ctypes.byref(cp), _ptr(o, io, shp, "o"), _ptr(dy, io, shp, "dy"),
+                                           _ptr(weight, torch.float32, (p.H * p.d_v,), "weight"), float(eps),
+                                           _ptr(d_o, io, shp, "d_o"), _ptr(dw), _ptr(ws), nbytes, _stream()), "gsa_out_norm_bwd")
+    return d_o, dw
 
 
 def gsa_release_streams():

@@ -34,6 +34,7 @@ gsa_status_t check_params(const gsa_params_t* p, bool need_T) {
         return GSA_ERR_INVALID_ARG;
     if (p->fuse != GSA_FUSE_OFF && p->fuse != GSA_FUSE_ON) return GSA_ERR_INVALID_ARG;
     if (p->gate_dtype != GSA_F32 && p->gate_dtype != GSA_BF16) return GSA_ERR_INVALID_ARG;
+    if (p->feature_map != GSA_FEAT_NONE && p->feature_map != GSA_FEAT_SWISH) return GSA_ERR_INVALID_ARG;
     if (p->nseq < 0 || (p->nseq == 0) != (p->cu_seqlens == nullptr)) return GSA_ERR_INVALID_ARG;
     if (!(p->scale == p->scale)) return GSA_ERR_INVALID_ARG;
     if (!dim_ok(p->d_k) || !dim_ok(p->d_v)) return GSA_ERR_UNSUPPORTED;
@@ -314,6 +315,35 @@ size_t pad_bytes(const gsa_params_t& p, int which) { return carve_pad(p, which, 
 size_t gate_conv_bytes(const gsa_params_t& p) {
     return p.gate_dtype == GSA_BF16 ? align_up((size_t)p.B * p.T * p.H * p.m * sizeof(float), 256) : 0;
 }
+// The layer's feature map: Swish(q), Swish(k), Swish(v) are formed once, in the part of the workspace
+// that follows everything else; the scans then read those copies.
+struct FeatureBuffers { void *q, *k, *v; size_t bytes; };
+FeatureBuffers carve_features(const gsa_params_t& p, void* base) {
+    FeatureBuffers f{nullptr, nullptr, nullptr, 0};
+    if (p.feature_map != GSA_FEAT_SWISH) return f;
+    const size_t e = p.io == GSA_BF16 ? 2 : 4, R = (size_t)p.B * p.T * p.H;
+    const size_t nk = align_up(R * p.d_k * e, 256), nv = align_up(R * p.d_v * e, 256);
+    char* b = static_cast<char*>(base);
+    f.q = b; f.k = b + nk; f.v = b + 2 * nk;
+    f.bytes = 2 * nk + nv;
+    return f;
+}
+gsa_status_t apply_feature_map(const gsa_params_t& p, int which, const void** q, const void** k, const void** v, void* ws,
+                               size_t ws_bytes, cudaStream_t st) {
+    if (p.feature_map != GSA_FEAT_SWISH) return GSA_OK;
+    if (ws == nullptr || (reinterpret_cast<uintptr_t>(ws) & 255u) != 0) return GSA_ERR_WORKSPACE;
+    const gsa_params_t pi = internal_params(p);
+    const size_t before = carve(pi, which, nullptr).bytes + pad_bytes(p, which) + gate_conv_bytes(p);
+    const FeatureBuffers f = carve_features(p, static_cast<char*>(ws) + before);
+    if (ws_bytes < before + f.bytes) return GSA_ERR_WORKSPACE;
+    const size_t R = (size_t)p.B * p.T * p.H;
+    if (launch_swish_fwd(*q, f.q, R * p.d_k, p.io, st) != cudaSuccess) return GSA_ERR_CUDA;
+    if (launch_swish_fwd(*k, f.k, R * p.d_k, p.io, st) != cudaSuccess) return GSA_ERR_CUDA;
+    if (launch_swish_fwd(*v, f.v, R * p.d_v, p.io, st) != cudaSuccess) return GSA_ERR_CUDA;
+    *q = f.q; *k = f.k; *v = f.v;
+    return GSA_OK;
+}
+
 // the fp32 gate tensor of this call (the caller's, or its widened copy behind `before` bytes of workspace)
 gsa_status_t gate_as_f32(const gsa_params_t& p, const float* gate, void* ws, size_t ws_bytes, size_t before,
                          cudaStream_t st, const float** out) {
@@ -374,7 +404,8 @@ size_t gsa_workspace_bytes(const gsa_params_t* params, int32_t which) {
     }
     const gsa_params_t pi = internal_params(*params);
     if (which == GSA_WS_GATE) return carve_gate(pi, nullptr).bytes;
-    return carve(pi, which, nullptr).bytes + pad_bytes(*params, which) + gate_conv_bytes(*params);
+    return carve(pi, which, nullptr).bytes + pad_bytes(*params, which) + gate_conv_bytes(*params) +
+           carve_features(*params, nullptr).bytes;
 }
 
 gsa_status_t gsa_gate_cumsum(const gsa_params_t* params, const float* gate, float* G, float* I,
@@ -492,6 +523,8 @@ gsa_status_t fwd_impl(const gsa_params_t* params, const void* q, const void* k, 
         const gsa_params_t pi0 = internal_params(*params);
         const size_t before = carve(pi0, GSA_WS_FWD, nullptr).bytes + pad_bytes(*params, GSA_WS_FWD);
         rc = gate_as_f32(*params, gate, ws, ws_bytes, before, static_cast<cudaStream_t>(stream), &gate);
+        if (rc != GSA_OK) return rc;
+        rc = apply_feature_map(*params, GSA_WS_FWD, &q, &k, &v, ws, ws_bytes, static_cast<cudaStream_t>(stream));
         if (rc != GSA_OK) return rc;
     }
     if (!pads_slots(*params))
@@ -691,15 +724,28 @@ gsa_status_t bwd_impl(const gsa_params_t* params, const void* q, const void* k, 
     if (!ok_opt(K0) || !ok_opt(V0) || !ok_opt(ok_saved) || !ok_opt(dKT) || !ok_opt(dVT) ||
         !ok_opt(dK0) || !ok_opt(dV0))
         return GSA_ERR_INVALID_ARG;
+    const void *q_raw = q, *k_raw = k, *v_raw = v;
     {
         const gsa_params_t pi0 = internal_params(*params);
         const size_t before = carve(pi0, GSA_WS_BWD, nullptr).bytes + pad_bytes(*params, GSA_WS_BWD);
         rc = gate_as_f32(*params, gate, ws, ws_bytes, before, static_cast<cudaStream_t>(stream), &gate);
         if (rc != GSA_OK) return rc;
+        rc = apply_feature_map(*params, GSA_WS_BWD, &q, &k, &v, ws, ws_bytes, static_cast<cudaStream_t>(stream));
+        if (rc != GSA_OK) return rc;
     }
+    // with the feature map, dq / dk / dv are turned into gradients w.r.t. the pre-activations at the end
+    auto finish = [&](gsa_status_t r) -> gsa_status_t {
+        if (r != GSA_OK || params->feature_map != GSA_FEAT_SWISH) return r;
+        cudaStream_t s2 = static_cast<cudaStream_t>(stream);
+        const size_t R = (size_t)params->B * params->T * params->H;
+        if (launch_swish_bwd(q_raw, dq, R * params->d_k, params->io, s2) != cudaSuccess) return GSA_ERR_CUDA;
+        if (launch_swish_bwd(k_raw, dk, R * params->d_k, params->io, s2) != cudaSuccess) return GSA_ERR_CUDA;
+        if (launch_swish_bwd(v_raw, dv, R * params->d_v, params->io, s2) != cudaSuccess) return GSA_ERR_CUDA;
+        return GSA_OK;
+    };
     if (!pads_slots(*params))
-        return bwd_core(params, 0, q, k, v, gate, K0, V0, ok_saved, dO, dKT, dVT, dq, dk, dv, dgate, dK0, dV0, gate_is_saved,
-                        gate_saved, gate_saved_bytes, ws, ws_bytes, stream, dev_status);
+        return finish(bwd_core(params, 0, q, k, v, gate, K0, V0, ok_saved, dO, dKT, dVT, dq, dk, dv, dgate, dK0, dV0,
+                               gate_is_saved, gate_saved, gate_saved_bytes, ws, ws_bytes, stream, dev_status));
     const gsa_params_t& p = *params;
     const gsa_params_t pi = internal_params(p);
     if (ws == nullptr || (reinterpret_cast<uintptr_t>(ws) & 255u) != 0) return GSA_ERR_WORKSPACE;
@@ -723,7 +769,7 @@ gsa_status_t bwd_impl(const gsa_params_t* params, const void* q, const void* k, 
     GSA_CUDA(launch_resize_rows(pb.dgate, dgate, rows, M, p.m, 0.f, st));
     if (dK0) GSA_CUDA(launch_resize_rows(pb.KT, dK0, pairs, M * p.d_k, p.m * p.d_k, 0.f, st));
     if (dV0) GSA_CUDA(launch_resize_rows(pb.VT, dV0, pairs, M * p.d_v, p.m * p.d_v, 0.f, st));
-    return GSA_OK;
+    return finish(GSA_OK);
 }
 }  // namespace
 
@@ -765,7 +811,9 @@ gsa_status_t gsa_shard_states(const gsa_params_t* params, const void* k, const v
                               int32_t* dev_status) {
     gsa_status_t rc = check_params(params, true);
     if (rc != GSA_OK) return rc;
-    if (pads_slots(*params) || params->gate_dtype != GSA_F32 || params->cu_seqlens != nullptr) return GSA_ERR_UNSUPPORTED;
+    if (pads_slots(*params) || params->gate_dtype != GSA_F32 || params->cu_seqlens != nullptr ||
+        params->feature_map != GSA_FEAT_NONE)
+        return GSA_ERR_UNSUPPORTED;
     if (!ok_ptr(k) || !ok_ptr(v) || !ok_ptr(gate) || !ok_ptr(KT) || !ok_ptr(VT) || !ok_ptr(logdecay)) return GSA_ERR_INVALID_ARG;
     const gsa_params_t& p = *params;
     if (ws == nullptr || (reinterpret_cast<uintptr_t>(ws) & 255u) != 0) return GSA_ERR_WORKSPACE;
@@ -799,6 +847,40 @@ gsa_status_t gsa_shard_combine(const gsa_params_t* params, int32_t d, int32_t ns
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     GSA_LAUNCH("shard_combine", launch_shard_combine(logdecay_all, local_all, S0, start, final_state, p.B, p.H, p.m, d, nshard,
                                                      rank, reverse != 0, st));
+    return GSA_OK;
+}
+
+gsa_status_t gsa_out_norm_fwd(const gsa_params_t* params, const void* o, const float* weight, float eps, void* y,
+                              void* stream) {
+    gsa_status_t rc = check_params(params, true);
+    if (rc != GSA_OK) return rc;
+    if (!ok_ptr(o) || !ok_ptr(y) || !ok_opt(weight) || !(eps >= 0.f)) return GSA_ERR_INVALID_ARG;
+    const gsa_params_t& p = *params;
+    if (p.H * p.d_v > out_norm_max_width(p.io)) return GSA_ERR_UNSUPPORTED;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    GSA_LAUNCH("out_norm", launch_out_norm_fwd(o, weight, eps, y, (size_t)p.B * p.T, p.H * p.d_v, p.io, st));
+    return GSA_OK;
+}
+
+size_t gsa_out_norm_workspace_bytes(const gsa_params_t* params) {
+    if (check_params(params, true) != GSA_OK) return 0;
+    return align_up(out_norm_bwd_parts((size_t)params->B * params->T) * params->H * params->d_v * sizeof(float), 256);
+}
+
+gsa_status_t gsa_out_norm_bwd(const gsa_params_t* params, const void* o, const void* dy, const float* weight, float eps,
+                              void* d_o, float* dweight, void* ws, size_t ws_bytes, void* stream) {
+    gsa_status_t rc = check_params(params, true);
+    if (rc != GSA_OK) return rc;
+    if (!ok_ptr(o) || !ok_ptr(dy) || !ok_ptr(d_o) || !ok_opt(weight) || !ok_opt(dweight) || !(eps >= 0.f))
+        return GSA_ERR_INVALID_ARG;
+    const gsa_params_t& p = *params;
+    if (p.H * p.d_v > out_norm_max_width(p.io)) return GSA_ERR_UNSUPPORTED;
+    if (dweight != nullptr && (ws == nullptr || (reinterpret_cast<uintptr_t>(ws) & 255u) != 0 ||
+                               ws_bytes < gsa_out_norm_workspace_bytes(params)))
+        return GSA_ERR_WORKSPACE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    GSA_LAUNCH("out_norm_bwd", launch_out_norm_bwd(o, dy, weight, eps, d_o, static_cast<float*>(ws), dweight,
+                                                   (size_t)p.B * p.T, p.H * p.d_v, p.io, st));
     return GSA_OK;
 }
 

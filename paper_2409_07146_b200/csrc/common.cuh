@@ -235,6 +235,15 @@ cudaError_t launch_fused_pair(int mode, const void* xq1, const void* xk1, const 
                               const float* G, const float* S1_0, const float* S2_0, float* S1_end, float* S2_end, int B,
                               int T, int H, int D1, int D2, float scale, int act, float* ok, float* u, void* Pd,
                               void* Zd, const int* strong_flag, cudaStream_t st, int32_t* dev_status);
+// layer pre- and post-operations (layer_ops.cu)
+cudaError_t launch_swish_fwd(const void* in, void* out, size_t n, int io, cudaStream_t st);
+cudaError_t launch_swish_bwd(const void* x, void* d, size_t n, int io, cudaStream_t st);
+int out_norm_max_width(int io);
+size_t out_norm_bwd_parts(size_t rows);
+cudaError_t launch_out_norm_fwd(const void* o, const float* weight, float eps, void* y, size_t rows, int N, int io,
+                                cudaStream_t st);
+cudaError_t launch_out_norm_bwd(const void* o, const void* dy, const float* weight, float eps, void* d_o, float* dw_part,
+                                float* dweight, size_t rows, int N, int io, cudaStream_t st);
 cudaError_t launch_decode(const gsa_params_t& p, const void* q, const void* k, const void* v,
                           const float* gate, float* Ks, float* Vs, void* o, cudaStream_t st);
 

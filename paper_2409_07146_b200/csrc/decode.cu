@@ -60,12 +60,19 @@ struct RowVec {
 #pragma unroll
             for (int w = 0; w < kW; ++w) v[r][w] = io_to_float<IO>(row[(lane + 32 * r) * kW + w]);
     }
+    // the layer's feature map (Sec. 3.3), applied as the token's q, k, v are loaded
+    __device__ __forceinline__ void swish() {
+#pragma unroll
+        for (int r = 0; r < kN; ++r)
+#pragma unroll
+            for (int w = 0; w < kW; ++w) v[r][w] = v[r][w] / (1.f + __expf(-v[r][w]));
+    }
 };
 
 template <typename IO, int DK, int DV, int M>
 __global__ void __launch_bounds__(kDecodeWarps * 32)
 decode_step_kernel(const IO* __restrict__ q, const IO* __restrict__ k, const IO* __restrict__ v,
-                   const void* __restrict__ gate_raw, int gate_bf16, int gate_kind, float inv_tau, float scale, int act,
+                   const void* __restrict__ gate_raw, int gate_bf16, int feature_map, int gate_kind, float inv_tau, float scale, int act,
                    float* __restrict__ Ks, float* __restrict__ Vs, IO* __restrict__ o) {
     constexpr int RPW = M / kDecodeWarps;  // memory rows per warp
     const size_t pair = blockIdx.x;
@@ -82,6 +89,7 @@ decode_step_kernel(const IO* __restrict__ q, const IO* __restrict__ k, const IO*
     qv.load_io(q + pair * DK, lane);
     kv.load_io(k + pair * DK, lane);
     vv.load_io(v + pair * DV, lane);
+    if (feature_map == GSA_FEAT_SWISH) { qv.swish(); kv.swish(); vv.swish(); }
     float a[RPW], ia[RPW];
 #pragma unroll
     for (int r = 0; r < RPW; ++r) {
@@ -183,11 +191,11 @@ static cudaError_t launch_decode_m(const gsa_params_t& p, const IO* q, const IO*
     const int is_log = p.gate_kind;
     const float inv_tau = p.tau > 0.f ? 1.f / p.tau : 0.f;
     if (p.m == 128)
-        decode_step_kernel<IO, DK, DV, 128><<<pairs, kDecodeWarps * 32, 0, st>>>(q, k, v, gate, p.gate_dtype == GSA_BF16, is_log, inv_tau, p.scale, p.slot_act, Ks, Vs, o);
+        decode_step_kernel<IO, DK, DV, 128><<<pairs, kDecodeWarps * 32, 0, st>>>(q, k, v, gate, p.gate_dtype == GSA_BF16, p.feature_map, is_log, inv_tau, p.scale, p.slot_act, Ks, Vs, o);
     else if (p.m == 64)
-        decode_step_kernel<IO, DK, DV, 64><<<pairs, kDecodeWarps * 32, 0, st>>>(q, k, v, gate, p.gate_dtype == GSA_BF16, is_log, inv_tau, p.scale, p.slot_act, Ks, Vs, o);
+        decode_step_kernel<IO, DK, DV, 64><<<pairs, kDecodeWarps * 32, 0, st>>>(q, k, v, gate, p.gate_dtype == GSA_BF16, p.feature_map, is_log, inv_tau, p.scale, p.slot_act, Ks, Vs, o);
     else
-        decode_step_kernel<IO, DK, DV, 32><<<pairs, kDecodeWarps * 32, 0, st>>>(q, k, v, gate, p.gate_dtype == GSA_BF16, is_log, inv_tau, p.scale, p.slot_act, Ks, Vs, o);
+        decode_step_kernel<IO, DK, DV, 32><<<pairs, kDecodeWarps * 32, 0, st>>>(q, k, v, gate, p.gate_dtype == GSA_BF16, p.feature_map, is_log, inv_tau, p.scale, p.slot_act, Ks, Vs, o);
     return cudaGetLastError();
 }
 

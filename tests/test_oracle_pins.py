@@ -408,3 +408,43 @@ def test_packed_sequences_match_the_unrolled_form_of_every_sequence_and_finite_d
             lo[pos][idx] -= eps
             fd = (loss(*hi) - loss(*lo)) / (2 * eps)
             assert abs(fd - g[name][idx]) <= 1e-6 * max(1.0, abs(fd)), (name, idx, fd, g[name][idx])
+
+
+# ---------------------------------------------------------------- layer pre- and post-operations
+def test_layer_elementwise_ops_against_library_routines_closed_form_and_autograd():
+    """Swish (feature map of q, k, v) and Swish -> RMSNorm (output path): against torch's silu and
+    rms_norm in fp64, a closed form on constant rows, autograd, and central finite differences."""
+    from oracle import layer
+    r = np.random.default_rng(12)
+    x = r.standard_normal((2, 5, 3, 8)) * 2.0
+    xt = torch.tensor(x, dtype=torch.float64, requires_grad=True)
+    np.testing.assert_allclose(layer.swish(x), torch.nn.functional.silu(xt).detach().numpy(), rtol=1e-13, atol=1e-15)
+    torch.nn.functional.silu(xt).sum().backward()
+    np.testing.assert_allclose(layer.swish_grad(x), xt.grad.numpy(), rtol=1e-12, atol=1e-14)
+
+    w = r.standard_normal(24) * 0.5 + 1.0
+    eps = 1e-5
+    y = layer.out_norm_fwd(x, w, eps)
+    ot = torch.tensor(x, dtype=torch.float64, requires_grad=True)
+    wt = torch.tensor(w, dtype=torch.float64, requires_grad=True)
+    yt = torch.nn.functional.rms_norm(torch.nn.functional.silu(ot).reshape(2, 5, 24), (24,), wt, eps).reshape(2, 5, 3, 8)
+    np.testing.assert_allclose(y, yt.detach().numpy(), rtol=1e-12, atol=1e-14)
+    dy = r.standard_normal(x.shape)
+    (yt * torch.tensor(dy)).sum().backward()
+    do, dw = layer.out_norm_bwd(x, dy, w, eps)
+    np.testing.assert_allclose(do, ot.grad.numpy(), rtol=1e-10, atol=1e-12)
+    np.testing.assert_allclose(dw, wt.grad.numpy(), rtol=1e-10, atol=1e-12)
+    # constant rows: every value of a token equal to c  ->  Swish(c) / sqrt(Swish(c)^2 + eps)
+    c = 1.7
+    sc = c / (1 + np.exp(-c))
+    yc = layer.out_norm_fwd(np.full((1, 2, 3, 8), c), None, eps)
+    np.testing.assert_allclose(yc, sc / np.sqrt(sc * sc + eps), rtol=1e-13)
+    # finite differences of a scalar loss through the forward
+    h = 1e-6
+    for _ in range(6):
+        idx = tuple(r.integers(0, n) for n in x.shape)
+        hi, lo = x.copy(), x.copy()
+        hi[idx] += h
+        lo[idx] -= h
+        fd = ((layer.out_norm_fwd(hi, w, eps) - layer.out_norm_fwd(lo, w, eps)) * dy).sum() / (2 * h)
+        assert abs(fd - do[idx]) <= 1e-6 * max(1.0, abs(fd))
