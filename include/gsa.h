@@ -70,7 +70,14 @@ typedef enum {
 } gsa_status_t;
 
 typedef enum { GSA_F32 = 0, GSA_BF16 = 1 } gsa_dtype_t;
-typedef enum { GSA_GATE_A = 0, GSA_GATE_LOG_A = 1, GSA_GATE_LOGITS = 2 } gsa_gate_t;
+typedef enum {
+    GSA_GATE_A = 0, GSA_GATE_LOG_A = 1, GSA_GATE_LOGITS = 2,
+    /* ABC, the ungated ancestor of the layer (Eq. 3-4; the "no decay" row of the table of ablations): the
+     * gate tensor holds the score logits s_t, the memories only accumulate (a = 1) and the write weights
+     * are the cumulative softmax over time phi_t = exp(s_t) / sum_{j<=t} exp(s_j) per slot, formed by the
+     * library; dgate is the gradient w.r.t. s.  gsa_fwd and gsa_bwd only; not with packed sequences. */
+    GSA_GATE_ABC = 3
+} gsa_gate_t;
 
 /* The non-linearity between the two passes: the softmax over the m slots of Eq. 6, or one of the
  * element-wise replacements of the paper's ablation on it (Sec. 4, table of ablations,
@@ -131,6 +138,9 @@ typedef struct {
                          * GSA_GATE_LOG_A and GSA_GATE_LOGITS: bfloat16 cannot tell a = 0.99 from 1, its
                          * logarithm it can); dgate is fp32 either way */
     int32_t feature_map; /* gsa_feature_map_t */
+    int32_t gate_broadcast; /* != 0: data-independent decay (table of ablations): the gate tensor is ONE row
+                         * [H, m] used for every token of every sequence (any gate_kind but GSA_GATE_ABC), and
+                         * dgate is [H, m], the sum of the per-token gate gradients */
     int32_t nseq;       /* packed sequences: number of sequences along T, 0 = none (see cu_seqlens) */
     const int32_t* cu_seqlens; /* DEVICE pointer to nseq + 1 ascending token offsets, cu_seqlens[0] = 0 and
                          * cu_seqlens[nseq] = T, or NULL.  Every batch row then holds nseq sequences back

@@ -12,7 +12,7 @@ _LIB_PATH = os.path.join(_HERE, "libgsa.so")
 _lib = None
 
 GSA_F32, GSA_BF16 = 0, 1
-GSA_GATE_A, GSA_GATE_LOG_A, GSA_GATE_LOGITS = 0, 1, 2
+GSA_GATE_A, GSA_GATE_LOG_A, GSA_GATE_LOGITS, GSA_GATE_ABC = 0, 1, 2, 3
 GSA_IMPL_AUTO, GSA_IMPL_SIMT, GSA_IMPL_TC = 0, 1, 2
 GSA_WS_FWD, GSA_WS_BWD, GSA_WS_DECODE, GSA_WS_GATE, GSA_WS_SHARD = 0, 1, 2, 3, 4
 
@@ -33,7 +33,8 @@ class _CParams(ctypes.Structure):
                 ("io", ctypes.c_int32), ("gate_kind", ctypes.c_int32),
                 ("scale", ctypes.c_float), ("impl", ctypes.c_int32), ("tau", ctypes.c_float),
                 ("slot_act", ctypes.c_int32), ("tc_operands", ctypes.c_int32), ("fuse", ctypes.c_int32),
-                ("gate_dtype", ctypes.c_int32), ("feature_map", ctypes.c_int32), ("nseq", ctypes.c_int32),
+                ("gate_dtype", ctypes.c_int32), ("feature_map", ctypes.c_int32), ("gate_broadcast", ctypes.c_int32),
+                ("nseq", ctypes.c_int32),
                 ("cu_seqlens", ctypes.c_void_p)]
 
 
@@ -57,16 +58,19 @@ class Params:
     fuse: bool = False             # tensor-core kernels: pass 1 -> softmax -> pass 2 as one kernel where the shape allows (gsa_fuse_t)
     gate_bf16: bool = False        # the gate tensor is bfloat16 (log a or logits)
     feature_map: str = "none"      # "none" | "swish": q, k, v hold pre-activations, Swish applied by the library
+    gate_is_abc: bool = False      # ABC (Eq. 3-4): the gate tensor holds score logits, no decay, cumulative-softmax writes
+    gate_broadcast: bool = False   # data-independent decay: the gate tensor (and dgate) is one row [H, m]
     cu_seqlens: object = None      # packed sequences: int32 CUDA tensor of nseq + 1 offsets along T (kept alive by Params)
 
     def c(self) -> _CParams:
         return _CParams(self.B, self.T, self.H, self.d_k, self.d_v, self.m,
                         GSA_BF16 if self.io == "bf16" else GSA_F32,
-                        GSA_GATE_LOGITS if self.gate_is_logits else
-                        (GSA_GATE_LOG_A if self.gate_is_log else GSA_GATE_A),
+                        GSA_GATE_ABC if self.gate_is_abc else (GSA_GATE_LOGITS if self.gate_is_logits else
+                                                              (GSA_GATE_LOG_A if self.gate_is_log else GSA_GATE_A)),
                         float(self.scale), _IMPL[self.impl], float(self.tau), _ACT[self.slot_act],
                         0 if self.tc_operands == "paired" else 1, 1 if self.fuse else 0,
                         GSA_BF16 if self.gate_bf16 else GSA_F32, 1 if self.feature_map == "swish" else 0,
+                        1 if self.gate_broadcast else 0,
                         0 if self.cu_seqlens is None else int(self.cu_seqlens.numel()) - 1,
                         None if self.cu_seqlens is None else self.cu_seqlens.data_ptr())
 
@@ -77,6 +81,11 @@ class Params:
     @property
     def gate_torch_dtype(self) -> torch.dtype:
         return torch.bfloat16 if self.gate_bf16 else torch.float32
+
+    def gate_shape(self, decode=False):
+        if self.gate_broadcast:
+            return (self.H, self.m)
+        return (self.B, self.H, self.m) if decode else (self.B, self.T, self.H, self.m)
 
 
 def lib_path() -> str:
@@ -213,7 +222,7 @@ def gsa_fwd(p: Params, q, k, v, gate, K0=None, V0=None, o=None, ok_save=None, KT
     ws, ws_bytes = _workspace(p, GSA_WS_FWD, ws, q.device)
     cp = p.c()
     head = (ctypes.byref(cp), _ptr(q, io, qk, "q"), _ptr(k, io, qk, "k"), _ptr(v, io, vv, "v"),
-            _ptr(gate, p.gate_torch_dtype, mm, "gate"), _ptr(K0, torch.float32, sk, "K0"),
+            _ptr(gate, p.gate_torch_dtype, p.gate_shape(), "gate"), _ptr(K0, torch.float32, sk, "K0"),
             _ptr(V0, torch.float32, sv, "V0"), _ptr(o, io, vv, "o"),
             _ptr(ok_save, torch.float32, mm, "ok_save"), _ptr(KT, torch.float32, sk, "KT"),
             _ptr(VT, torch.float32, sv, "VT"))
@@ -239,15 +248,15 @@ def gsa_bwd(p: Params, q, k, v, gate, dO, K0=None, V0=None, ok_saved=None, dKT=N
     dq = torch.empty(qk, dtype=io, device=dev) if dq is None else dq
     dk = torch.empty(qk, dtype=io, device=dev) if dk is None else dk
     dv = torch.empty(vv, dtype=io, device=dev) if dv is None else dv
-    dgate = torch.empty(mm, dtype=torch.float32, device=dev) if dgate is None else dgate
+    dgate = torch.empty(p.gate_shape(), dtype=torch.float32, device=dev) if dgate is None else dgate
     ws, ws_bytes = _workspace(p, GSA_WS_BWD, ws, dev)
     cp = p.c()
     head = (ctypes.byref(cp), _ptr(q, io, qk, "q"), _ptr(k, io, qk, "k"), _ptr(v, io, vv, "v"),
-            _ptr(gate, p.gate_torch_dtype, mm, "gate"), _ptr(K0, torch.float32, sk, "K0"),
+            _ptr(gate, p.gate_torch_dtype, p.gate_shape(), "gate"), _ptr(K0, torch.float32, sk, "K0"),
             _ptr(V0, torch.float32, sv, "V0"), _ptr(ok_saved, torch.float32, mm, "ok_saved"),
             _ptr(dO, io, vv, "dO"), _ptr(dKT, torch.float32, sk, "dKT"),
             _ptr(dVT, torch.float32, sv, "dVT"), _ptr(dq, io, qk, "dq"), _ptr(dk, io, qk, "dk"),
-            _ptr(dv, io, vv, "dv"), _ptr(dgate, torch.float32, mm, "dgate"),
+            _ptr(dv, io, vv, "dv"), _ptr(dgate, torch.float32, p.gate_shape(), "dgate"),
             _ptr(dK0, torch.float32, sk, "dK0"), _ptr(dV0, torch.float32, sv, "dV0"))
     tail = (_ptr(ws, None, None, "ws"), ws_bytes, _stream(), _ptr(dev_status, torch.int32, None, "dev_status"))
     if gate_saved is None:
@@ -268,7 +277,7 @@ def gsa_decode_step(p: Params, q, k, v, gate, Kstate, Vstate, o=None):
     cp = p.c()
     _check(load_library().gsa_decode_step(
         ctypes.byref(cp), _ptr(q, io, qk, "q"), _ptr(k, io, qk, "k"), _ptr(v, io, vv, "v"),
-        _ptr(gate, p.gate_torch_dtype, mm, "gate"),
+        _ptr(gate, p.gate_torch_dtype, p.gate_shape(decode=True), "gate"),
         _ptr(Kstate, torch.float32, (p.B, p.H, p.m, p.d_k), "Kstate"),
         _ptr(Vstate, torch.float32, (p.B, p.H, p.m, p.d_v), "Vstate"), _ptr(o, io, vv, "o"),
         _stream()), "gsa_decode_step")
@@ -388,7 +397,7 @@ def gsa_fwd_noalloc(p: Params, q, k, v, gate, o, K0=None, V0=None, ok_save=None,
     cp = p.c()
     _check(load_library().gsa_fwd_noalloc(
         ctypes.byref(cp), _ptr(q, io, qk, "q"), _ptr(k, io, qk, "k"), _ptr(v, io, vv, "v"),
-        _ptr(gate, p.gate_torch_dtype, mm, "gate"), _ptr(K0, torch.float32, sk, "K0"),
+        _ptr(gate, p.gate_torch_dtype, p.gate_shape(), "gate"), _ptr(K0, torch.float32, sk, "K0"),
         _ptr(V0, torch.float32, sv, "V0"), _ptr(o, io, vv, "o"),
         _ptr(ok_save, torch.float32, mm, "ok_save"), _ptr(KT, torch.float32, sk, "KT"),
         _ptr(VT, torch.float32, sv, "VT"), _stream(),

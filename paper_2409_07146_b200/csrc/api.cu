@@ -25,8 +25,10 @@ gsa_status_t check_params(const gsa_params_t* p, bool need_T) {
     if (p->B < 1 || p->H < 1 || p->d_k < 1 || p->d_v < 1 || p->m < 1) return GSA_ERR_INVALID_ARG;
     if (need_T && p->T < 1) return GSA_ERR_INVALID_ARG;
     if (p->io != GSA_F32 && p->io != GSA_BF16) return GSA_ERR_INVALID_ARG;
-    if (p->gate_kind != GSA_GATE_A && p->gate_kind != GSA_GATE_LOG_A && p->gate_kind != GSA_GATE_LOGITS)
+    if (p->gate_kind != GSA_GATE_A && p->gate_kind != GSA_GATE_LOG_A && p->gate_kind != GSA_GATE_LOGITS &&
+        p->gate_kind != GSA_GATE_ABC)
         return GSA_ERR_INVALID_ARG;
+    if (p->gate_kind == GSA_GATE_ABC && (p->cu_seqlens != nullptr || p->gate_broadcast != 0)) return GSA_ERR_UNSUPPORTED;
     if (p->gate_kind == GSA_GATE_LOGITS && !(p->tau > 0.f)) return GSA_ERR_INVALID_ARG;
     if (p->slot_act < GSA_ACT_SOFTMAX || p->slot_act > GSA_ACT_RELU2) return GSA_ERR_INVALID_ARG;
     if (p->tc_operands != GSA_TC_PAIRED && p->tc_operands != GSA_TC_SINGLE) return GSA_ERR_INVALID_ARG;
@@ -312,9 +314,27 @@ PadBuffers carve_pad(const gsa_params_t& p, int which, void* base) {
 }
 size_t pad_bytes(const gsa_params_t& p, int which) { return carve_pad(p, which, nullptr).bytes; }
 // a gate tensor given in bfloat16 is widened to fp32 once, into the last part of the workspace
-size_t gate_conv_bytes(const gsa_params_t& p) {
-    return p.gate_dtype == GSA_BF16 ? align_up((size_t)p.B * p.T * p.H * p.m * sizeof(float), 256) : 0;
+size_t gate_elems(const gsa_params_t& p) {       // elements of the gate tensor as the caller passes it
+    return p.gate_broadcast ? (size_t)p.H * p.m : (size_t)p.B * p.T * p.H * p.m;
 }
+// Workspace behind the padded-slot buffers: [ widened bf16 gate | gate row spread over all tokens |
+// per-token gate gradient | its column-sum scratch ]
+struct GateBoundary { size_t conv, spread, dfull, colsum, bytes; };
+GateBoundary gate_boundary(const gsa_params_t& p, int which) {
+    GateBoundary g{0, 0, 0, 0, 0};
+    const size_t mt = align_up((size_t)p.B * p.T * p.H * p.m * sizeof(float), 256);
+    if (p.gate_dtype == GSA_BF16) g.conv = align_up(gate_elems(p) * sizeof(float), 256);
+    if (p.gate_broadcast) {
+        g.spread = mt;
+        if (which == GSA_WS_BWD) {
+            g.dfull = mt;
+            g.colsum = align_up(column_sum_parts((size_t)p.B * p.T) * p.H * p.m * sizeof(float), 256);
+        }
+    }
+    g.bytes = g.conv + g.spread + g.dfull + g.colsum;
+    return g;
+}
+size_t gate_conv_bytes(const gsa_params_t& p, int which = GSA_WS_BWD) { return gate_boundary(p, which).bytes; }
 // The layer's feature map: Swish(q), Swish(k), Swish(v) are formed once, in the part of the workspace
 // that follows everything else; the scans then read those copies.
 struct FeatureBuffers { void *q, *k, *v; size_t bytes; };
@@ -333,7 +353,7 @@ gsa_status_t apply_feature_map(const gsa_params_t& p, int which, const void** q,
     if (p.feature_map != GSA_FEAT_SWISH) return GSA_OK;
     if (ws == nullptr || (reinterpret_cast<uintptr_t>(ws) & 255u) != 0) return GSA_ERR_WORKSPACE;
     const gsa_params_t pi = internal_params(p);
-    const size_t before = carve(pi, which, nullptr).bytes + pad_bytes(p, which) + gate_conv_bytes(p);
+    const size_t before = carve(pi, which, nullptr).bytes + pad_bytes(p, which) + gate_conv_bytes(p, which);
     const FeatureBuffers f = carve_features(p, static_cast<char*>(ws) + before);
     if (ws_bytes < before + f.bytes) return GSA_ERR_WORKSPACE;
     const size_t R = (size_t)p.B * p.T * p.H;
@@ -345,15 +365,23 @@ gsa_status_t apply_feature_map(const gsa_params_t& p, int which, const void** q,
 }
 
 // the fp32 gate tensor of this call (the caller's, or its widened copy behind `before` bytes of workspace)
-gsa_status_t gate_as_f32(const gsa_params_t& p, const float* gate, void* ws, size_t ws_bytes, size_t before,
+gsa_status_t gate_as_f32(const gsa_params_t& p, int which, const float* gate, void* ws, size_t ws_bytes, size_t before,
                          cudaStream_t st, const float** out) {
     *out = gate;
-    if (p.gate_dtype != GSA_BF16) return GSA_OK;
-    if (ws == nullptr || (reinterpret_cast<uintptr_t>(ws) & 255u) != 0 || ws_bytes < before + gate_conv_bytes(p))
-        return GSA_ERR_WORKSPACE;
-    float* buf = reinterpret_cast<float*>(static_cast<char*>(ws) + before);
-    if (launch_widen_bf16(gate, buf, (size_t)p.B * p.T * p.H * p.m, st) != cudaSuccess) return GSA_ERR_CUDA;
-    *out = buf;
+    const GateBoundary g = gate_boundary(p, which);
+    if (g.bytes == 0) return GSA_OK;
+    if (ws == nullptr || (reinterpret_cast<uintptr_t>(ws) & 255u) != 0 || ws_bytes < before + g.bytes) return GSA_ERR_WORKSPACE;
+    char* base = static_cast<char*>(ws) + before;
+    if (p.gate_dtype == GSA_BF16) {
+        float* buf = reinterpret_cast<float*>(base);
+        if (launch_widen_bf16(gate, buf, gate_elems(p), st) != cudaSuccess) return GSA_ERR_CUDA;
+        *out = buf;
+    }
+    if (p.gate_broadcast) {
+        float* buf = reinterpret_cast<float*>(base + g.conv);
+        if (launch_broadcast_rows(*out, buf, (size_t)p.B * p.T, p.H * p.m, st) != cudaSuccess) return GSA_ERR_CUDA;
+        *out = buf;
+    }
     return GSA_OK;
 }
 
@@ -404,7 +432,7 @@ size_t gsa_workspace_bytes(const gsa_params_t* params, int32_t which) {
     }
     const gsa_params_t pi = internal_params(*params);
     if (which == GSA_WS_GATE) return carve_gate(pi, nullptr).bytes;
-    return carve(pi, which, nullptr).bytes + pad_bytes(*params, which) + gate_conv_bytes(*params) +
+    return carve(pi, which, nullptr).bytes + pad_bytes(*params, which) + gate_conv_bytes(*params, which) +
            carve_features(*params, nullptr).bytes;
 }
 
@@ -413,7 +441,8 @@ gsa_status_t gsa_gate_cumsum(const gsa_params_t* params, const float* gate, floa
     gsa_status_t rc = check_params(params, true);
     if (rc != GSA_OK) return rc;
     if (!ok_ptr(gate) || !ok_ptr(G) || !ok_ptr(I)) return GSA_ERR_INVALID_ARG;
-    if (params->gate_dtype != GSA_F32) return GSA_ERR_UNSUPPORTED;      // (this query entry point has no workspace)
+    if (params->gate_dtype != GSA_F32 || params->gate_kind == GSA_GATE_ABC || params->gate_broadcast)
+        return GSA_ERR_UNSUPPORTED;      // (this query entry point has no workspace)
     const gsa_params_t& p = *params;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     GSA_LAUNCH("gate_cumsum", launch_gate_cumsum(gate, p.gate_kind, inv_tau(p), G, I, p.B, p.T,
@@ -438,9 +467,12 @@ gsa_status_t fwd_core(const gsa_params_t* params, int m_active, const void* q, c
 
     const int nseg = segments_of(p);
     GSA_CUDA(cudaMemsetAsync(w.strong, 0, sizeof(int) * (size_t)p.B * p.H * nseg, st));
-    GSA_LAUNCH("gate_cumsum", launch_gate_cumsum(gate, p.gate_kind, inv_tau(p), w.G, w.I, p.B, p.T,
-                                                 p.H, p.m, chunk_of(p), w.strong, nseg, w.Id, p.io == GSA_BF16, st,
-                                                 p.cu_seqlens, p.nseq));
+    if (p.gate_kind == GSA_GATE_ABC)      // no decay, write weights from the cumulative softmax of the scores
+        GSA_LAUNCH("abc_write", launch_abc_write(gate, w.G, w.I, w.Id, p.B, p.T, p.H, p.m, st));
+    else
+        GSA_LAUNCH("gate_cumsum", launch_gate_cumsum(gate, p.gate_kind, inv_tau(p), w.G, w.I, p.B, p.T,
+                                                     p.H, p.m, chunk_of(p), w.strong, nseg, w.Id, p.io == GSA_BF16, st,
+                                                     p.cu_seqlens, p.nseq));
     float* ok = ok_save;      // the scaled logits leave the softmax kernel only if the caller keeps them
     // the pipelined kernels leave the row factor of the pass-1 sums to the softmax kernel
     const PendingDecay pend = use_tc(p) ? PendingDecay{w.G, w.strong, p.T, p.H, nseg} : PendingDecay{nullptr, nullptr, 1, 1, 1};
@@ -522,7 +554,7 @@ gsa_status_t fwd_impl(const gsa_params_t* params, const void* q, const void* k, 
         // a bfloat16 gate tensor is widened once; everything downstream reads fp32
         const gsa_params_t pi0 = internal_params(*params);
         const size_t before = carve(pi0, GSA_WS_FWD, nullptr).bytes + pad_bytes(*params, GSA_WS_FWD);
-        rc = gate_as_f32(*params, gate, ws, ws_bytes, before, static_cast<cudaStream_t>(stream), &gate);
+        rc = gate_as_f32(*params, GSA_WS_FWD, gate, ws, ws_bytes, before, static_cast<cudaStream_t>(stream), &gate);
         if (rc != GSA_OK) return rc;
         rc = apply_feature_map(*params, GSA_WS_FWD, &q, &k, &v, ws, ws_bytes, static_cast<cudaStream_t>(stream));
         if (rc != GSA_OK) return rc;
@@ -592,9 +624,12 @@ gsa_status_t bwd_core(const gsa_params_t* params, int m_active, const void* q, c
     const int Bs = p.B * nseg, Ts = p.T / nseg;
     if (!gate_is_saved) {      // (a forward of the same call left the gate kernel's products otherwise)
         GSA_CUDA(cudaMemsetAsync(w.strong, 0, sizeof(int) * (size_t)p.B * p.H * nseg, st));
-        GSA_LAUNCH("gate_cumsum", launch_gate_cumsum(gate, p.gate_kind, inv_tau(p), w.G, w.I, p.B, p.T,
-                                                     p.H, p.m, chunk_of(p), w.strong, nseg, w.Id, p.io == GSA_BF16, st,
-                                                     p.cu_seqlens, p.nseq));
+        if (p.gate_kind == GSA_GATE_ABC)
+            GSA_LAUNCH("abc_write", launch_abc_write(gate, w.G, w.I, w.Id, p.B, p.T, p.H, p.m, st));
+        else
+            GSA_LAUNCH("gate_cumsum", launch_gate_cumsum(gate, p.gate_kind, inv_tau(p), w.G, w.I, p.B, p.T,
+                                                         p.H, p.m, chunk_of(p), w.strong, nseg, w.Id, p.io == GSA_BF16, st,
+                                                         p.cu_seqlens, p.nseq));
     }
     const float* ok = ok_saved;
     const PendingDecay pend = use_tc(p) ? PendingDecay{w.G, w.strong, p.T, p.H, nseg} : PendingDecay{nullptr, nullptr, 1, 1, 1};
@@ -704,6 +739,11 @@ gsa_status_t bwd_core(const gsa_params_t* params, int m_active, const void* q, c
         GSA_LAUNCH("bwd_dk_key_side_rev", key_side(p, adk, 1, w.strong, st, dev_status));
         GSA_LAUNCH("bwd_dIk_value_side_rev", value_side(p, adIk, 1, w.strong, st, dev_status));
     }
+    if (p.gate_kind == GSA_GATE_ABC) {
+        // no decay path: the scores' gradient follows from that of the write weights (G == 0: no row factor pending)
+        GSA_LAUNCH("abc_grad", launch_abc_grad(w.I, w.dIk, s.k, w.dIv, s.v, dgate, p.B, p.T, p.H, p.m, st));
+        return GSA_OK;
+    }
     // forget-gate gradient: reversed cumulative sum over the whole sequence
     GSA_LAUNCH("gate_grad", launch_gate_grad(w.u, w.I, w.dIk, s.k, w.dIv, s.v, gate, p.gate_kind, inv_tau(p),
                               dKT, w.KT, dVT, w.VT, p.d_k, p.d_v, w.chunk_tot, dgate, p.B, p.T,
@@ -725,18 +765,30 @@ gsa_status_t bwd_impl(const gsa_params_t* params, const void* q, const void* k, 
         !ok_opt(dK0) || !ok_opt(dV0))
         return GSA_ERR_INVALID_ARG;
     const void *q_raw = q, *k_raw = k, *v_raw = v;
+    float *dgate_row = nullptr, *colsum = nullptr;
     {
         const gsa_params_t pi0 = internal_params(*params);
         const size_t before = carve(pi0, GSA_WS_BWD, nullptr).bytes + pad_bytes(*params, GSA_WS_BWD);
-        rc = gate_as_f32(*params, gate, ws, ws_bytes, before, static_cast<cudaStream_t>(stream), &gate);
+        rc = gate_as_f32(*params, GSA_WS_BWD, gate, ws, ws_bytes, before, static_cast<cudaStream_t>(stream), &gate);
         if (rc != GSA_OK) return rc;
         rc = apply_feature_map(*params, GSA_WS_BWD, &q, &k, &v, ws, ws_bytes, static_cast<cudaStream_t>(stream));
         if (rc != GSA_OK) return rc;
+        if (params->gate_broadcast) {        // the per-token gate gradient lands in the workspace; its sum is returned
+            const GateBoundary g = gate_boundary(*params, GSA_WS_BWD);
+            char* base = static_cast<char*>(ws) + before;
+            dgate_row = dgate;
+            dgate = reinterpret_cast<float*>(base + g.conv + g.spread);
+            colsum = reinterpret_cast<float*>(base + g.conv + g.spread + g.dfull);
+        }
     }
     // with the feature map, dq / dk / dv are turned into gradients w.r.t. the pre-activations at the end
     auto finish = [&](gsa_status_t r) -> gsa_status_t {
-        if (r != GSA_OK || params->feature_map != GSA_FEAT_SWISH) return r;
+        if (r != GSA_OK) return r;
         cudaStream_t s2 = static_cast<cudaStream_t>(stream);
+        if (dgate_row != nullptr &&
+            launch_column_sum(dgate, colsum, dgate_row, (size_t)params->B * params->T, params->H * params->m, s2) != cudaSuccess)
+            return GSA_ERR_CUDA;
+        if (params->feature_map != GSA_FEAT_SWISH) return GSA_OK;
         const size_t R = (size_t)params->B * params->T * params->H;
         if (launch_swish_bwd(q_raw, dq, R * params->d_k, params->io, s2) != cudaSuccess) return GSA_ERR_CUDA;
         if (launch_swish_bwd(k_raw, dk, R * params->d_k, params->io, s2) != cudaSuccess) return GSA_ERR_CUDA;
@@ -801,6 +853,7 @@ gsa_status_t gsa_decode_step(const gsa_params_t* params, const void* q, const vo
         !ok_ptr(Vstate) || !ok_ptr(o))
         return GSA_ERR_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (params->gate_kind == GSA_GATE_ABC) return GSA_ERR_UNSUPPORTED;      // (the running normaliser is not a state here)
     GSA_LAUNCH("decode_step", launch_decode(*params, q, k, v, gate, Kstate, Vstate, o, st));
     return GSA_OK;
 }
@@ -812,7 +865,7 @@ gsa_status_t gsa_shard_states(const gsa_params_t* params, const void* k, const v
     gsa_status_t rc = check_params(params, true);
     if (rc != GSA_OK) return rc;
     if (pads_slots(*params) || params->gate_dtype != GSA_F32 || params->cu_seqlens != nullptr ||
-        params->feature_map != GSA_FEAT_NONE)
+        params->feature_map != GSA_FEAT_NONE || params->gate_kind == GSA_GATE_ABC || params->gate_broadcast)
         return GSA_ERR_UNSUPPORTED;
     if (!ok_ptr(k) || !ok_ptr(v) || !ok_ptr(gate) || !ok_ptr(KT) || !ok_ptr(VT) || !ok_ptr(logdecay)) return GSA_ERR_INVALID_ARG;
     const gsa_params_t& p = *params;

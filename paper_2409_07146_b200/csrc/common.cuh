@@ -161,6 +161,15 @@ cudaError_t launch_gate_cumsum(const float* gate, int gate_kind, float inv_tau, 
                                int B, int T, int H, int M, int chunk, int* strong_flag, int nseg,
                                void* decayed, int fast_log, cudaStream_t st, const int* cu_seqlens = nullptr,
                                int nseq = 0);
+// ABC (Eq. 3-4): write weights phi (cumulative softmax over time of the scores) into I, zeros into G, phi as the
+// decayed bf16 rows; and the gradient w.r.t. the scores from phi and the input-gate gradient partial sums
+cudaError_t launch_abc_write(const float* s_in, float* G, float* I, void* decayed, int B, int T, int H, int M, cudaStream_t st);
+cudaError_t launch_abc_grad(const float* phi, const float* dIk, int nsk, const float* dIv, int nsv, float* ds, int B, int T,
+                            int H, int M, cudaStream_t st);
+// a gate row [n] spread over `rows` rows; column sums of [rows, n] (scratch: column_sum_parts(rows) * n floats)
+cudaError_t launch_broadcast_rows(const float* row, float* out, size_t rows, int n, cudaStream_t st);
+size_t column_sum_parts(size_t rows);
+cudaError_t launch_column_sum(const float* in, float* part, float* out, size_t rows, int n, cudaStream_t st);
 // n bfloat16 values -> fp32 (a gate tensor given in bfloat16)
 cudaError_t launch_widen_bf16(const void* in, float* out, size_t n, cudaStream_t st);
 // Segment-parallel scheduling (T cut into nseg segments run as independent sequences): per-segment

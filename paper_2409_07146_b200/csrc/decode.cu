@@ -72,7 +72,7 @@ struct RowVec {
 template <typename IO, int DK, int DV, int M>
 __global__ void __launch_bounds__(kDecodeWarps * 32)
 decode_step_kernel(const IO* __restrict__ q, const IO* __restrict__ k, const IO* __restrict__ v,
-                   const void* __restrict__ gate_raw, int gate_bf16, int feature_map, int gate_kind, float inv_tau, float scale, int act,
+                   const void* __restrict__ gate_raw, int gate_bf16, int gate_row_of_head, int feature_map, int gate_kind, float inv_tau, float scale, int act,
                    float* __restrict__ Ks, float* __restrict__ Vs, IO* __restrict__ o) {
     constexpr int RPW = M / kDecodeWarps;  // memory rows per warp
     const size_t pair = blockIdx.x;
@@ -93,7 +93,8 @@ decode_step_kernel(const IO* __restrict__ q, const IO* __restrict__ k, const IO*
     float a[RPW], ia[RPW];
 #pragma unroll
     for (int r = 0; r < RPW; ++r) {
-        const size_t gi = pair * M + warp * RPW + r;
+        // (data-independent decay: one gate row per head, shared by all sequences; gate_row_of_head = H then)
+        const size_t gi = (gate_row_of_head ? pair % gate_row_of_head : pair) * M + warp * RPW + r;
         float gt = gate_bf16 ? __bfloat162float(static_cast<const __nv_bfloat16*>(gate_raw)[gi])
                              : static_cast<const float*>(gate_raw)[gi];
         if (gate_kind == GSA_GATE_LOGITS) gt = log_gate_from_logit(gt, inv_tau);
@@ -191,11 +192,11 @@ static cudaError_t launch_decode_m(const gsa_params_t& p, const IO* q, const IO*
     const int is_log = p.gate_kind;
     const float inv_tau = p.tau > 0.f ? 1.f / p.tau : 0.f;
     if (p.m == 128)
-        decode_step_kernel<IO, DK, DV, 128><<<pairs, kDecodeWarps * 32, 0, st>>>(q, k, v, gate, p.gate_dtype == GSA_BF16, p.feature_map, is_log, inv_tau, p.scale, p.slot_act, Ks, Vs, o);
+        decode_step_kernel<IO, DK, DV, 128><<<pairs, kDecodeWarps * 32, 0, st>>>(q, k, v, gate, p.gate_dtype == GSA_BF16, p.gate_broadcast ? p.H : 0, p.feature_map, is_log, inv_tau, p.scale, p.slot_act, Ks, Vs, o);
     else if (p.m == 64)
-        decode_step_kernel<IO, DK, DV, 64><<<pairs, kDecodeWarps * 32, 0, st>>>(q, k, v, gate, p.gate_dtype == GSA_BF16, p.feature_map, is_log, inv_tau, p.scale, p.slot_act, Ks, Vs, o);
+        decode_step_kernel<IO, DK, DV, 64><<<pairs, kDecodeWarps * 32, 0, st>>>(q, k, v, gate, p.gate_dtype == GSA_BF16, p.gate_broadcast ? p.H : 0, p.feature_map, is_log, inv_tau, p.scale, p.slot_act, Ks, Vs, o);
     else
-        decode_step_kernel<IO, DK, DV, 32><<<pairs, kDecodeWarps * 32, 0, st>>>(q, k, v, gate, p.gate_dtype == GSA_BF16, p.feature_map, is_log, inv_tau, p.scale, p.slot_act, Ks, Vs, o);
+        decode_step_kernel<IO, DK, DV, 32><<<pairs, kDecodeWarps * 32, 0, st>>>(q, k, v, gate, p.gate_dtype == GSA_BF16, p.gate_broadcast ? p.H : 0, p.feature_map, is_log, inv_tau, p.scale, p.slot_act, Ks, Vs, o);
     return cudaGetLastError();
 }
 

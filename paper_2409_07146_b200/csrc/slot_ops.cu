@@ -863,6 +863,141 @@ cudaError_t launch_gate_grad(const float* u, const float* I, const float* dIk_pa
     return cudaGetLastError();
 }
 
+// ------------------------------------------------------------------ ABC: no decay, cumulative-softmax write weights
+// Eq. 3-4 (the ungated ancestor of GSA, the "no decay" row of the ablations): the memories only
+// accumulate, K~_t = K~_{t-1} + phi_t (x) k_t, with write weights phi_t = exp(s_t) / sum_{j<=t} exp(s_j)
+// per slot.  In the layer's terms: log a = 0 everywhere and the input gate is phi.  The cumulative
+// softmax over time is a scan per (batch, head, slot): one thread each, the rows of eight time steps
+// requested together so that the loads overlap; running maximum and rescaled running sum as in any
+// streaming softmax.  The decayed bf16 rows of the tensor-core kernels are phi itself (exp(-G) = 1).
+constexpr int kAbcBatch = 8;
+
+template <int M>
+__global__ void __launch_bounds__(M) abc_write_kernel(const float* __restrict__ s_in, float* __restrict__ G,
+                                                      float* __restrict__ I, __nv_bfloat16* __restrict__ decayed, int T,
+                                                      int H) {
+    const int bh = blockIdx.x, b = bh / H, h = bh % H, s = threadIdx.x;
+    const size_t stride = (size_t)H * M;
+    size_t idx = ((size_t)b * T * H + h) * M + s;
+    float mx = -INFINITY, z = 0.f;
+    for (int t0 = 0; t0 < T; t0 += kAbcBatch) {
+        float x[kAbcBatch];
+#pragma unroll
+        for (int i = 0; i < kAbcBatch; ++i) x[i] = (t0 + i < T) ? s_in[idx + (size_t)i * stride] : 0.f;
+#pragma unroll
+        for (int i = 0; i < kAbcBatch; ++i) {
+            if (t0 + i >= T) break;
+            const float nm = fmaxf(mx, x[i]);
+            const float e = __expf(x[i] - nm);
+            z = z * __expf(mx - nm) + e;
+            mx = nm;
+            const float phi = e / z;
+            const size_t at = idx + (size_t)i * stride;
+            G[at] = 0.f;
+            I[at] = phi;
+            if (decayed != nullptr) {
+                const __nv_bfloat16 hi = __float2bfloat16_rn(phi);
+                __nv_bfloat16* row = decayed + 2 * (at - s);
+                row[s] = hi;
+                row[M + s] = __float2bfloat16_rn(phi - __bfloat162float(hi));
+            }
+        }
+        idx += (size_t)kAbcBatch * stride;
+    }
+}
+
+// Gradient w.r.t. the scores: with dphi_t the gradient w.r.t. the write weights (the sum of the input-gate
+// gradient partial sums of both passes),
+//     ds_j = phi_j (dphi_j - R_j),   R_j = dphi_j phi_j + (1 - phi_{j+1}) R_{j+1}
+// (Z_j / Z_t = prod_{r=j+1..t} (1 - phi_r): nothing but phi is needed).  A reverse scan, same thread layout.
+template <int M>
+__global__ void __launch_bounds__(M) abc_grad_kernel(const float* __restrict__ phi_in, const float* __restrict__ dIk, int nsk,
+                                                     const float* __restrict__ dIv, int nsv, float* __restrict__ ds, int T,
+                                                     int H, size_t total) {
+    const int bh = blockIdx.x, b = bh / H, h = bh % H, s = threadIdx.x;
+    const size_t stride = (size_t)H * M;
+    const size_t base = ((size_t)b * T * H + h) * M + s;
+    float R = 0.f, phi_next = 0.f;          // (1 - phi_{T}) R_{T} = 0
+    for (int t1 = T; t1 > 0; t1 -= kAbcBatch) {
+        float phi[kAbcBatch], dphi[kAbcBatch];
+#pragma unroll
+        for (int i = 0; i < kAbcBatch; ++i) {
+            const int t = t1 - 1 - i;
+            phi[i] = 0.f; dphi[i] = 0.f;
+            if (t >= 0) {
+                const size_t at = base + (size_t)t * stride;
+                phi[i] = phi_in[at];
+                for (int sl = 0; sl < nsk; ++sl) dphi[i] += dIk[at + (size_t)sl * total];
+                for (int sl = 0; sl < nsv; ++sl) dphi[i] += dIv[at + (size_t)sl * total];
+            }
+        }
+#pragma unroll
+        for (int i = 0; i < kAbcBatch; ++i) {
+            const int t = t1 - 1 - i;
+            if (t < 0) break;
+            R = dphi[i] * phi[i] + (1.f - phi_next) * R;
+            ds[base + (size_t)t * stride] = phi[i] * (dphi[i] - R);
+            phi_next = phi[i];
+        }
+    }
+}
+
+cudaError_t launch_abc_write(const float* s_in, float* G, float* I, void* decayed, int B, int T, int H, int M, cudaStream_t st) {
+    if (M == 128) abc_write_kernel<128><<<B * H, 128, 0, st>>>(s_in, G, I, static_cast<__nv_bfloat16*>(decayed), T, H);
+    else if (M == 64) abc_write_kernel<64><<<B * H, 64, 0, st>>>(s_in, G, I, static_cast<__nv_bfloat16*>(decayed), T, H);
+    else abc_write_kernel<32><<<B * H, 32, 0, st>>>(s_in, G, I, static_cast<__nv_bfloat16*>(decayed), T, H);
+    return cudaGetLastError();
+}
+cudaError_t launch_abc_grad(const float* phi, const float* dIk, int nsk, const float* dIv, int nsv, float* ds, int B, int T,
+                            int H, int M, cudaStream_t st) {
+    const size_t total = (size_t)B * T * H * M;
+    if (M == 128) abc_grad_kernel<128><<<B * H, 128, 0, st>>>(phi, dIk, nsk, dIv, nsv, ds, T, H, total);
+    else if (M == 64) abc_grad_kernel<64><<<B * H, 64, 0, st>>>(phi, dIk, nsk, dIv, nsv, ds, T, H, total);
+    else abc_grad_kernel<32><<<B * H, 32, 0, st>>>(phi, dIk, nsk, dIv, nsv, ds, T, H, total);
+    return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------ data-independent decay
+// A gate that does not depend on the input (the "data-independent decay" row of the ablations) is one
+// row [H, M] for all tokens: it is spread over [B,T,H,M] on the way in, and the gate gradient is
+// summed over the tokens on the way out (partial sums per block of rows, added in order).
+__global__ void broadcast_rows_kernel(const float* __restrict__ row, float* __restrict__ out, size_t rows, int n) {
+    const size_t total = rows * (size_t)n;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x)
+        out[i] = row[i % n];
+}
+constexpr int kColSumRows = 256;
+__global__ void column_partial_kernel(const float* __restrict__ in, float* __restrict__ part, size_t rows, int n) {
+    const int c = blockIdx.y * blockDim.x + threadIdx.x;
+    if (c >= n) return;
+    const size_t r0 = (size_t)blockIdx.x * kColSumRows;
+    const size_t r1 = r0 + kColSumRows < rows ? r0 + kColSumRows : rows;
+    float acc = 0.f;
+    for (size_t r = r0; r < r1; ++r) acc += in[r * n + c];
+    part[(size_t)blockIdx.x * n + c] = acc;
+}
+__global__ void column_final_kernel(const float* __restrict__ part, float* __restrict__ out, int nparts, int n) {
+    const int c = blockIdx.x * blockDim.x + threadIdx.x;
+    if (c >= n) return;
+    double acc = 0.0;
+    for (int p = 0; p < nparts; ++p) acc += (double)part[(size_t)p * n + c];
+    out[c] = (float)acc;
+}
+cudaError_t launch_broadcast_rows(const float* row, float* out, size_t rows, int n, cudaStream_t st) {
+    const size_t total = rows * (size_t)n;
+    const unsigned blocks = (unsigned)((total + 255) / 256 < 148 * 32 ? (total + 255) / 256 : 148 * 32);
+    broadcast_rows_kernel<<<blocks ? blocks : 1, 256, 0, st>>>(row, out, rows, n);
+    return cudaGetLastError();
+}
+size_t column_sum_parts(size_t rows) { return (rows + kColSumRows - 1) / kColSumRows; }
+// out[c] = sum over rows of in[r][c]; part: column_sum_parts(rows) * n floats of scratch
+cudaError_t launch_column_sum(const float* in, float* part, float* out, size_t rows, int n, cudaStream_t st) {
+    const unsigned parts = (unsigned)column_sum_parts(rows);
+    column_partial_kernel<<<dim3(parts, (n + 127) / 128), 128, 0, st>>>(in, part, rows, n);
+    column_final_kernel<<<(n + 127) / 128, 128, 0, st>>>(part, out, (int)parts, n);
+    return cudaGetLastError();
+}
+
 // ------------------------------------------------------------------ gate tensor in bfloat16
 __global__ void widen_bf16_kernel(const __nv_bfloat16* __restrict__ in, float* __restrict__ out, size_t n) {
     for (size_t i = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) * 2; i < n; i += (size_t)gridDim.x * blockDim.x * 2) {

@@ -619,3 +619,69 @@ def test_gate_tensor_in_bfloat16(kind):
     ro = oracle.decode_step(d["q"][:, 0], d["k"][:, 0], d["v"][:, 0], g16[:, 0], Kr, Vr, gate_is_log=kind == "log",
                             gate_is_logits=kind == "logits", tau=8.0)
     assert rel_err(to_np(od), ro, True) <= TOL["bf16"] and rel_err(to_np(Ks), Kr) <= 1e-5
+
+
+# ------------------------------------------------------------------ ablation variants of the gate
+@pytest.mark.parametrize("io,impl,T,d", [("f32", "auto", 150, 64), ("bf16", "tc", 300, 128), ("bf16", "tc", 200, 256)])
+def test_abc_no_decay_variant_fwd_bwd(io, impl, T, d):
+    """ABC (Eq. 3-4): no decay, write weights from the cumulative softmax over time of score logits."""
+    from oracle import abc
+    B, H, m = 2, 2, 64
+    x = rand_inputs(21 + T, B, T, H, d, d, m, io, init=True)
+    s = (1.5 * np.random.default_rng(4).standard_normal((B, T, H, m))).astype(np.float32)
+    p = gsa.Params(B, T, H, d, d, m, io=io, impl=impl, gate_is_abc=True, scale=0.7)
+    q, k, v, dO = (to_dev(x[n], io) for n in ("q", "k", "v", "dO"))
+    K0, V0 = to_dev(x["K0"]), to_dev(x["V0"])
+    ok = torch.empty(B, T, H, m, device="cuda")
+    KT = torch.empty(B, H, m, d, device="cuda"); VT = torch.empty(B, H, m, d, device="cuda")
+    o = gsa.gsa_fwd(p, q, k, v, to_dev(s), K0, V0, ok_save=ok, KT=KT, VT=VT)
+    dK0 = torch.empty_like(KT); dV0 = torch.empty_like(VT)
+    dq, dk_, dv_, dg = gsa.gsa_bwd(p, q, k, v, to_dev(s), dO, K0, V0, ok_saved=ok, dK0=dK0, dV0=dV0)
+    torch.cuda.synchronize()
+    rf = abc.fwd(x["q"], x["k"], x["v"], s, scale=0.7, K0=x["K0"], V0=x["V0"])
+    rb = abc.bwd(x["q"], x["k"], x["v"], s, x["dO"], scale=0.7, K0=x["K0"], V0=x["V0"])
+    got = dict(o=to_np(o), ok=to_np(ok), KT=to_np(KT), VT=to_np(VT), dq=to_np(dq), dk=to_np(dk_), dv=to_np(dv_),
+               dgate=to_np(dg), dK0=to_np(dK0), dV0=to_np(dV0))
+    ref = dict(rf, **rb)
+    errs = {n: rel_err(got[n], ref[n], io == "bf16" and n in BF16_IO) for n in got}
+    print("abc", io, T, d, {n: float("%.2g" % e) for n, e in errs.items()})
+    assert all(e <= TOL[io] for e in errs.values()), errs
+
+
+@pytest.mark.parametrize("io,impl,kind", [("f32", "auto", "a"), ("bf16", "tc", "logits"), ("bf16", "tc", "a")])
+def test_data_independent_decay_one_gate_row_for_all_tokens(io, impl, kind):
+    """The gate as one row [H, m] (data-independent decay of the ablations): same results as the row
+    repeated for every token, and dgate is the sum of the per-token gate gradients."""
+    B, T, H, d, m = 2, 260, 2, 128, 64
+    x = rand_inputs(57, B, T, H, d, d, m, io, init=True)
+    r = np.random.default_rng(6)
+    if kind == "a":
+        row = (1 / (1 + np.exp(-r.standard_normal((H, m))))) ** 0.125
+        kw = {}
+    else:
+        row = 2.0 * r.standard_normal((H, m))
+        kw = dict(gate_is_logits=True, tau=8.0)
+    row = row.astype(np.float32)
+    full = np.ascontiguousarray(np.broadcast_to(row, (B, T, H, m)))
+    p = gsa.Params(B, T, H, d, d, m, io=io, impl=impl, gate_broadcast=True, **kw)
+    q, k, v, dO = (to_dev(x[n], io) for n in ("q", "k", "v", "dO"))
+    K0, V0 = to_dev(x["K0"]), to_dev(x["V0"])
+    ok = torch.empty(B, T, H, m, device="cuda")
+    o = gsa.gsa_fwd(p, q, k, v, to_dev(row), K0, V0, ok_save=ok)
+    dq, dk_, dv_, dg = gsa.gsa_bwd(p, q, k, v, to_dev(row), dO, K0, V0, ok_saved=ok)
+    torch.cuda.synchronize()
+    assert tuple(dg.shape) == (H, m)
+    rf = oracle.fwd(x["q"], x["k"], x["v"], full, K0=x["K0"], V0=x["V0"], **kw)
+    rb = oracle.bwd(x["q"], x["k"], x["v"], full, x["dO"], K0=x["K0"], V0=x["V0"], **kw)
+    got = dict(o=to_np(o), ok=to_np(ok), dq=to_np(dq), dk=to_np(dk_), dv=to_np(dv_), dgate=to_np(dg))
+    ref = dict(o=rf["o"], ok=rf["ok"], dq=rb["dq"], dk=rb["dk"], dv=rb["dv"], dgate=rb["dgate"].sum(axis=(0, 1)))
+    errs = {n: rel_err(got[n], ref[n], io == "bf16" and n in BF16_IO) for n in got}
+    print("constant gate", io, kind, {n: float("%.2g" % e) for n, e in errs.items()})
+    assert all(e <= TOL[io] for e in errs.values()), errs
+    # decode with the one row
+    pd = gsa.Params(B, 1, H, d, d, m, io=io, impl=impl, gate_broadcast=True, **kw)
+    Ks, Vs = to_dev(x["K0"]).clone(), to_dev(x["V0"]).clone()
+    Kr, Vr = x["K0"].astype(np.float64), x["V0"].astype(np.float64)
+    od = gsa.gsa_decode_step(pd, q[:, 0].contiguous(), k[:, 0].contiguous(), v[:, 0].contiguous(), to_dev(row), Ks, Vs)
+    ro = oracle.decode_step(x["q"][:, 0], x["k"][:, 0], x["v"][:, 0], full[:, 0], Kr, Vr, **kw)
+    assert rel_err(to_np(od), ro, io == "bf16") <= TOL[io] and rel_err(to_np(Ks), Kr) <= 1e-5

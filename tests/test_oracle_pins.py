@@ -448,3 +448,43 @@ def test_layer_elementwise_ops_against_library_routines_closed_form_and_autograd
         lo[idx] -= h
         fd = ((layer.out_norm_fwd(hi, w, eps) - layer.out_norm_fwd(lo, w, eps)) * dy).sum() / (2 * h)
         assert abs(fd - do[idx]) <= 1e-6 * max(1.0, abs(fd))
+
+
+# ---------------------------------------------------------------- ABC (no decay) and constant decay
+def test_abc_oracle_against_its_linear_attention_form_and_uniform_scores():
+    """oracle/abc.py (Eq. 3-4): (i) with the cumulative softmax written out, o' = sum_{j<=t} (q_t . k_j) phi_j
+    is plain causal linear attention (Eq. 5's parallel form), evaluated here with a masked matrix
+    product; (ii) equal scores give phi_t = 1 / t, so the memories are running sums of k_t / t."""
+    from oracle import abc
+    r = np.random.default_rng(3)
+    B, T, H, dk, dv, m = 1, 9, 2, 4, 3, 5
+    q, k, v = r.standard_normal((B, T, H, dk)), r.standard_normal((B, T, H, dk)), r.standard_normal((B, T, H, dv))
+    s = r.standard_normal((B, T, H, m))
+    f = abc.fwd(q, k, v, s, scale=0.8)
+    e = np.exp(s)
+    phi = e / np.cumsum(e, axis=1)
+    mask = np.tril(np.ones((T, T)))
+    for h in range(H):
+        P = (q[0, :, h] @ k[0, :, h].T) * mask                    # [T,T]
+        logits = 0.8 * P @ phi[0, :, h]                            # [T,m]
+        np.testing.assert_allclose(f["ok"][0, :, h], logits, rtol=1e-12, atol=1e-13)
+        p = np.exp(logits - logits.max(-1, keepdims=True)); p /= p.sum(-1, keepdims=True)
+        A = (p @ phi[0, :, h].T) * mask                            # [T,T]
+        np.testing.assert_allclose(f["o"][0, :, h], A @ v[0, :, h], rtol=1e-12, atol=1e-13)
+    f1 = abc.fwd(q, k, v, np.zeros_like(s))
+    want = np.cumsum(k[0, :, 0] / np.arange(1, T + 1)[:, None], axis=0)[-1]
+    np.testing.assert_allclose(f1["KT"][0, 0, 2], want, rtol=1e-12)
+    # the gradients come from autograd of the definition; spot-check them with finite differences
+    dO = r.standard_normal(v.shape)
+    g = abc.bwd(q, k, v, s, dO, scale=0.8)
+    h_ = 1e-6
+    for name, x in (("dgate", s), ("dk", k)):
+        for _ in range(4):
+            idx = tuple(r.integers(0, n) for n in x.shape)
+            hi, lo = x.copy(), x.copy()
+            hi[idx] += h_; lo[idx] -= h_
+            a_hi = [q, k, v, s]; a_lo = [q, k, v, s]
+            pos = 3 if name == "dgate" else 1
+            a_hi[pos], a_lo[pos] = hi, lo
+            fd = ((abc.fwd(*a_hi, scale=0.8)["o"] - abc.fwd(*a_lo, scale=0.8)["o"]) * dO).sum() / (2 * h_)
+            assert abs(fd - g[name][idx]) <= 1e-6 * max(1.0, abs(fd))
