@@ -327,8 +327,23 @@ def run_ours(args):
     if args.profile_case:
         # bare steps for a profiler: no timing, no extras (the numbers of such a run are not
         # benchmark values)
-        for _ in range(args.warmup + args.steps):
-            step(d_in)
+        if args.profile_case == "decode":
+            wd = W.CONFIGS["decode"]
+            pdec = gsa.Params(wd.B, 1, wd.H, wd.d_k, wd.d_v, wd.m, io="bf16")
+            sd = W.make_decode_states(wd)
+            Ks, Vs = torch.from_numpy(sd["K"]).to(dev), torch.from_numpy(sd["V"]).to(dev)
+            xd = W.make_decode_step_inputs(wd, 0)
+            qd, kd, vd = (torch.from_numpy(xd[n]).to(dev).to(torch.bfloat16) for n in ("q", "k", "v"))
+            gd = torch.from_numpy(xd["gate"]).to(dev)
+            od = torch.empty(wd.B, wd.H, wd.d_v, dtype=torch.bfloat16, device=dev)
+            for _ in range(args.warmup + args.steps):
+                gsa.gsa_decode_step(pdec, qd, kd, vd, gd, Ks, Vs, o=od)
+        elif args.profile_case == "fwd":
+            for _ in range(args.warmup + args.steps):
+                gsa.gsa_fwd(p, d_in["q"], d_in["k"], d_in["v"], d_in["gate"], o=o, ws=ws_f, dev_status=status)
+        else:
+            for _ in range(args.warmup + args.steps):
+                step(d_in)
         torch.cuda.synchronize()
         if rank == 0:
             print(json.dumps({"profile_case": True, "steps": args.steps, "warmup": args.warmup}))
@@ -821,8 +836,10 @@ def main():
     ap.add_argument("--no-other-configs", action="store_true",
                     help="skip the list of the other configurations (t2r_7b, long_keep, long_forget, tiny_f32)")
     ap.add_argument("--no-graph", action="store_true", help="time plain library calls instead of a CUDA graph replay")
-    ap.add_argument("--profile-case", action="store_true",
-                    help="run warmup + steps bare (for ncu); prints no benchmark line")
+    ap.add_argument("--profile-case", nargs="?", const="step", default=None, choices=["step", "fwd", "decode"],
+                    help="run warmup + steps of one case bare (for ncu; prints no benchmark line): step = the "
+                         "benchmark's forward + backward, fwd = the forward alone without saved logits (with --fuse: "
+                         "the fused kernel), decode = gsa_decode_step on the decode workload")
     args = ap.parse_args()
     if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
         # started as a plain process: start the N ranks of one node here (what a torchrun command line does)
