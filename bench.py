@@ -88,6 +88,9 @@ def kernel_algorithmic_bytes(label: str, w: W.Workload) -> int:
         "bwd_dIv_value_side_rev": 2 * w.d_v * e + 4 * m + 4 * m * nsv,
         "bwd_dk_key_side_rev": 2 * w.d_k * e + 8 * m,
         "bwd_dIk_value_side_rev": 2 * w.d_k * e + 4 * m + 4 * m * nsk,
+        # a pair of reversed scans as one kernel: both d-sized tiles and both decayed rows once
+        "bwd_dv_dIv_pair_rev": 3 * w.d_v * e + 8 * m + 4 * m * nsv,  # dO, v, I exp(-G), p exp(G) -> dv, slices of dI^v
+        "bwd_dk_dIk_pair_rev": 3 * w.d_k * e + 8 * m + 4 * m * nsk,  # q, k, I exp(-G), dz exp(G) -> dk, slices of dI^k
         "gate_grad": 4 * m * (7 + nsk + nsv),   # u, gate, G, partials -> dgate; carry pass reads gate, r/w dgate
         # fused chunk kernels: the slot rows between the passes stay on chip
         "fused_fwd": e * (2 * w.d_k + 2 * w.d_v) + 12 * m,           # q, k, v, I exp(-G), G -> o, o'
@@ -101,6 +104,8 @@ def kernel_function(label: str) -> str:
     of one kernel, and so are the four key_side scans."""
     if label.startswith("fused"):
         return "fused_pair_kernel"
+    if "pair_rev" in label:
+        return "rev_pair_kernel"
     if "key_side" in label:
         return "key_side_lean_kernel"
     if "value_side" in label:
@@ -117,6 +122,8 @@ def kernel_algorithmic_flops(fn: str, w: W.Workload, d: int) -> float:
     per_row = 2 * C * (m + d) + 4 * m * d      # (the same count for either primitive)
     if fn == "fused_pair_kernel":
         per_row *= 2                           # a value_side and a key_side scan
+    if fn == "rev_pair_kernel":
+        per_row = 4 * C * (m + d) + 6 * m * d  # ... that share the state update
     return float(per_row) * w.B * w.T * w.H
 
 
@@ -454,7 +461,9 @@ def run_ours(args):
         two = sum(len(v) for lab, v in per.items() if lab.endswith("_side") or lab.endswith("_side_rev"))
         # a fused label is the fused kernel plus the three kernels that serve the flagged pairs
         fusedl = sum(len(v) for lab, v in per.items() if lab.startswith("fused"))
-        launches = (len(recs) + 2 * len(per.get("gate_grad", [])) + two + 3 * fusedl) // reps
+        # a pair label is the pair kernel plus the two general kernels that serve the flagged pairs
+        pairl = sum(len(v) for lab, v in per.items() if "pair_rev" in lab)
+        launches = (len(recs) + 2 * len(per.get("gate_grad", [])) + two + 3 * fusedl + 2 * pairl) // reps
         kernels = []
         tot = sum(sum(v) for v in per.values())
         for lab, v in per.items():
@@ -487,7 +496,7 @@ def run_ours(args):
         # the bytes the same launch would move if the slot-sized rows between the passes stayed on chip
         # (the d-sized tensors only: v in, o out for key_side; q, k in for value_side)
         e_ = 2 if w.io == "bf16" else 4
-        fused_bytes = w.B * w.T * w.H * 2 * (w.d_v if fn.startswith("key") else w.d_k) * e_
+        fused_bytes = w.B * w.T * w.H * (3 if fn == "rev_pair_kernel" else 2) * (w.d_v if fn.startswith("key") else w.d_k) * e_
         roofline = {"bound": "hbm", "kernel": fn, "labels": [k_["kernel"] for k_ in members],
                     "launches_per_step": n_l, "avg_launch_ms": avg_ms,
                     "achieved": alg / (avg_ms * 1e-3) / 1e9,
@@ -501,7 +510,7 @@ def run_ours(args):
                                 "layer, not what limits this kernel"),
                     "peak_source": pk["source"],
                     "share_of_step": sum(k_["share"] for k_ in members)}
-        if fn.endswith("_side_lean_kernel") or fn == "fused_pair_kernel":
+        if fn.endswith("_side_lean_kernel") or fn in ("fused_pair_kernel", "rev_pair_kernel"):
             d = w.d_v if fn.startswith("key") else w.d_k     # (d_k == d_v in the benchmark workload)
             fl = kernel_algorithmic_flops(fn, w, d)
             roofline["alg_tflops"] = fl / (avg_ms * 1e-3) / 1e12

@@ -46,6 +46,15 @@ GSA_API int32_t gsa_timing_end(float* ms, const char** labels, int32_t capacity)
  */
 GSA_API gsa_status_t gsa_wait_selftest(uint32_t limit_us, void* stream, int32_t* dev_status, uint32_t* waited_us);
 
+/*
+ * Development switch (no counterpart in the paper).  The backward's four time-reversed scans share
+ * their states in pairs (dv with dI^v, dk with dI^k; App. B) and by default run as two kernels that
+ * compute a pair each.  enable == 0 makes later gsa_bwd calls of this process run four single scans
+ * instead (same results up to the rounding order of a few fp32 additions); non-zero restores the
+ * default.  Returns the previous setting.  Process-wide; takes effect at the next call.
+ */
+GSA_API int32_t gsa_dev_pair_scans(int32_t enable);
+
 #ifdef __cplusplus
 }
 #endif

@@ -11,4 +11,5 @@ from .binding import (  # noqa: F401
     gsa_chunk_size, gsa_workspace_bytes, gsa_gate_cumsum, gsa_fwd, gsa_bwd, gsa_decode_step, gsa_tc_selftest,
     gsa_timing_begin, gsa_timing_end, gsa_fwd_noalloc, gate_block, GSA_NOALLOC_MAX_WORKSPACE_BYTES,
     gsa_wait_selftest, gsa_release_streams, gsa_shard_states, gsa_shard_combine, gsa_out_norm_fwd, gsa_out_norm_bwd,
+    gsa_dev_pair_scans,
 )

@@ -97,7 +97,7 @@ def exported_symbols():
             "gsa_fwd", "gsa_bwd", "gsa_decode_step", "gsa_tc_selftest", "gsa_timing_begin",
             "gsa_timing_end", "gsa_fwd_noalloc", "gsa_fwd_save_gate", "gsa_bwd_saved_gate", "gsa_release_streams",
             "gsa_wait_selftest", "gsa_shard_states", "gsa_shard_combine", "gsa_out_norm_fwd",
-            "gsa_out_norm_workspace_bytes", "gsa_out_norm_bwd"]
+            "gsa_out_norm_workspace_bytes", "gsa_out_norm_bwd", "gsa_dev_pair_scans"]
 
 
 def load_library():
@@ -140,6 +140,8 @@ def load_library():
     lib.gsa_tc_selftest.restype = ctypes.c_int
     lib.gsa_wait_selftest.argtypes = [ctypes.c_uint32, vp, vp, vp]
     lib.gsa_wait_selftest.restype = ctypes.c_int
+    lib.gsa_dev_pair_scans.argtypes = [i32]
+    lib.gsa_dev_pair_scans.restype = i32
     lib.gsa_shard_states.argtypes = [pp] + [vp] * 6 + [vp, sz, vp, vp]
     lib.gsa_shard_states.restype = ctypes.c_int
     lib.gsa_shard_combine.argtypes = [pp, i32, i32, i32, i32] + [vp] * 5 + [vp]
@@ -301,6 +303,12 @@ def gsa_wait_selftest(limit_us: int, dev_status, waited_us=None):
     receives the time it waited."""
     _check(load_library().gsa_wait_selftest(int(limit_us), _stream(), _ptr(dev_status, torch.int32, None, "dev_status"),
                                             _ptr(waited_us, torch.int32, None, "waited_us")), "gsa_wait_selftest")
+
+
+def gsa_dev_pair_scans(enable: bool) -> bool:
+    """Development switch: the backward's reversed scans as two pair kernels (True, the default) or as four
+    single ones (False), for later gsa_bwd calls of this process.  Returns the previous setting."""
+    return bool(load_library().gsa_dev_pair_scans(1 if enable else 0))
 
 
 def gsa_shard_states(p: Params, k, v, gate, ws=None, dev_status=None):

@@ -2,6 +2,7 @@
 // the kernels of one forward / backward call are enqueued.  No kernel lives here.
 #include <string.h>
 
+#include <atomic>
 #include <vector>
 
 #include "common.cuh"
@@ -166,6 +167,7 @@ Workspace carve(const gsa_params_t& p, int which, void* ws) {
 // segments' decay, the memories entering every segment and the final memories.
 struct GateSums {
     int* strong; float *G, *I; void* Id;
+    float* p; void* Pd;                               // slot weights of the forward (tensor-core path)
     float *seg_decay, *Kstart, *Vstart, *KT, *VT;     // nseg > 1 only
     size_t bytes;
 };
@@ -179,6 +181,11 @@ GateSums carve_gate(const gsa_params_t& p, void* base) {
     g.G = c.take(mt);
     g.I = c.take(mt);
     g.Id = use_tc(p) ? c.take(mt) : nullptr;
+    // the slot weights p (fp32 for the pairs flagged for strong decay, the decayed operand pair for
+    // the others) depend on the forward's logits only: kept, they let the backward's dv and dI^v
+    // scans start before the softmax gradient is known
+    g.p = use_tc(p) ? c.take(mt) : nullptr;
+    g.Pd = use_tc(p) ? c.take(mt) : nullptr;
     if (nseg > 1) {
         const size_t pairs = (size_t)p.B * nseg * p.H;
         g.seg_decay = c.take(pairs * p.m);
@@ -196,6 +203,7 @@ bool use_gate_block(const gsa_params_t& p, Workspace* w, void* block, size_t blo
     const GateSums g = carve_gate(p, block);
     if (block_bytes < g.bytes) return false;
     w->strong = g.strong; w->G = g.G; w->I = g.I; w->Id = g.Id;
+    if (g.p != nullptr) { w->p = g.p; w->Pd = g.Pd; }
     if (g.seg_decay != nullptr) {
         w->seg_decay = g.seg_decay; w->Kstart = g.Kstart; w->Vstart = g.Vstart;
         w->KT = g.KT; w->VT = g.VT;      // (the forward's workspace has no KT / VT of its own)
@@ -232,6 +240,10 @@ struct TimingSink {
 };
 thread_local TimingSink g_sink;
 
+// development switch (gsa_dev_pair_scans): the backward's reversed scans as two pair kernels (default)
+// or as four single ones
+std::atomic<int> g_pair_scans{1};
+
 void timing_before(cudaStream_t st) {
     if (g_sink.active && g_sink.count < g_sink.capacity) cudaEventRecord(g_sink.ev[2 * g_sink.count], st);
 }
@@ -250,7 +262,9 @@ void timing_after(const char* label, cudaStream_t st) {
 // timing sink active they run one after the other instead, so that each is timed alone.
 struct ScanLanes {
     cudaStream_t stream[4] = {nullptr, nullptr, nullptr, nullptr};
-    cudaEvent_t fork = nullptr, join[4] = {nullptr, nullptr, nullptr, nullptr};
+    cudaStream_t fast = nullptr;       // highest priority: the chain the other scans wait for
+    cudaEvent_t fast_done = nullptr;
+    cudaEvent_t fork = nullptr, fork_early = nullptr, join[4] = {nullptr, nullptr, nullptr, nullptr};
 };
 constexpr int kMaxLaneDevices = 64;
 thread_local ScanLanes g_scan_lanes[kMaxLaneDevices];
@@ -267,6 +281,11 @@ cudaError_t scan_lanes(ScanLanes** out) {
             if (e == cudaSuccess) e = cudaEventCreateWithFlags(&l.join[i], cudaEventDisableTiming);
         }
         if (e == cudaSuccess) e = cudaEventCreateWithFlags(&l.fork, cudaEventDisableTiming);
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&l.fork_early, cudaEventDisableTiming);
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&l.fast_done, cudaEventDisableTiming);
+        int least = 0, greatest = 0;
+        if (e == cudaSuccess) e = cudaDeviceGetStreamPriorityRange(&least, &greatest);
+        if (e == cudaSuccess) e = cudaStreamCreateWithPriority(&l.fast, cudaStreamNonBlocking, greatest);
         if (e != cudaSuccess) return e;
     }
     *out = &l;
@@ -284,6 +303,9 @@ cudaError_t scan_lanes_release() {
         if (l.join[i] != nullptr) cudaEventDestroy(l.join[i]);
     }
     if (l.fork != nullptr) cudaEventDestroy(l.fork);
+    if (l.fork_early != nullptr) cudaEventDestroy(l.fork_early);
+    if (l.fast_done != nullptr) cudaEventDestroy(l.fast_done);
+    if (l.fast != nullptr) cudaStreamDestroy(l.fast);
     l = ScanLanes{};
     return cudaSuccess;
 }
@@ -667,6 +689,20 @@ gsa_status_t bwd_core(const gsa_params_t* params, int m_active, const void* q, c
     // dq: the pass-2 form on (dz, 1-a, k); carries K~
     KeySideArgs adq{w.dz, w.I, w.G, k, Kin, KTout, dq, Bs, Ts, p.H, p.d_k, w.Zd, w.Id};
     const bool fused = use_fused(p);
+    // With the forward's slot weights in the saved block (and the logits saved, so that nothing here
+    // rewrites them), the dv and dI^v scans depend on nothing this call computes: they start at once,
+    // on two of the library's streams, beside the dp scan and the softmax gradient.
+    const bool early = gate_is_saved && ok_saved != nullptr && use_tc(p) && !fused && nseg == 1 && !g_sink.active;
+    ScanLanes* lanes = nullptr;
+    if (use_tc(p) && !g_sink.active) GSA_CUDA(scan_lanes(&lanes));
+    if (early) {
+        GSA_CUDA(cudaEventRecord(lanes->fork_early, st));
+        for (int i = 0; i < 2; ++i) GSA_CUDA(cudaStreamWaitEvent(lanes->stream[i], lanes->fork_early, 0));
+        GSA_CUDA(cudaStreamWaitEvent(lanes->fast, lanes->fork_early, 0));
+    }
+    // (the chain dp -> softmax gradient, which three more scans wait for, goes first wherever an SM is free:
+    // it runs on the library's high-priority stream, the early scans fill what it leaves)
+    cudaStream_t sc = early ? lanes->fast : st;
     if (fused) {
         // One kernel for dp -> dsoftmax -> dq (it also leaves u and the decayed rows of p and dz for the
         // reversed scans); the flagged pairs take the general kernels on the side stream.
@@ -691,9 +727,26 @@ gsa_status_t bwd_core(const gsa_params_t* params, int m_active, const void* q, c
             GSA_CUDA(cudaStreamWaitEvent(st, side->join, 0));
         }
     } else {
-        GSA_LAUNCH("bwd_dp_value_side", value_side(p, adp, 0, w.strong, st, dev_status));
-        GSA_LAUNCH("slot_softmax_bwd", launch_slot_softmax_bwd(ok, w.dppart, s.v, p.scale, p.slot_act, w.p, w.dz, w.u, p.B, p.T * p.H, p.m, pend.G, w.Pd,
-                                                               w.Zd, pend, st, m_active));
+        GSA_LAUNCH("bwd_dp_value_side", value_side(p, adp, 0, w.strong, sc, dev_status));
+        if (early) {
+            KeySideArgs adv{w.I, w.p, w.G, dO, dVT, dV0, dv, Bs, Ts, p.H, p.d_v, w.Id, w.Pd};
+            ValueSideArgs adIv{v, dO, w.p, w.G, dVT, nullptr, w.dIv, Bs, Ts, p.H, p.d_v, w.Pd};
+            adv.single = adIv.single = p.tc_operands == GSA_TC_SINGLE;
+            if (g_pair_scans.load(std::memory_order_relaxed) != 0 && rev_pair_supported(adIv, adv, p.m)) {
+                GSA_CUDA(launch_rev_pair_tc(adIv, adv, p.m, w.strong, lanes->stream[0], dev_status));
+            } else {
+                GSA_CUDA(key_side(p, adv, 1, w.strong, lanes->stream[0], dev_status));
+                GSA_CUDA(value_side(p, adIv, 1, w.strong, lanes->stream[1], dev_status));
+            }
+        }
+        // (started early, the dv / dI^v scans are reading the forward's p: it is not written again)
+        GSA_LAUNCH("slot_softmax_bwd", launch_slot_softmax_bwd(ok, w.dppart, s.v, p.scale, p.slot_act, early ? nullptr : w.p, w.dz, w.u,
+                                                               p.B, p.T * p.H, p.m, pend.G, early ? nullptr : w.Pd, w.Zd, pend, sc,
+                                                               m_active));
+        if (early) {
+            GSA_CUDA(cudaEventRecord(lanes->fast_done, sc));
+            GSA_CUDA(cudaStreamWaitEvent(st, lanes->fast_done, 0));
+        }
     }
     const float *dKin = dKT, *dVin = dVT;    // states entering the reversed scans (from the right)
     float *dK0out = dK0, *dV0out = dV0;
@@ -717,15 +770,35 @@ gsa_status_t bwd_core(const gsa_params_t* params, int m_active, const void* q, c
     ValueSideArgs adIv{v, dO, w.p, w.G, dVin, nullptr, w.dIv, Bs, Ts, p.H, p.d_v, w.Pd};
     KeySideArgs adk{w.I, w.dz, w.G, q, dKin, dK0out, dk, Bs, Ts, p.H, p.d_k, w.Id, w.Zd};
     ValueSideArgs adIk{k, q, w.dz, w.G, dKin, nullptr, w.dIk, Bs, Ts, p.H, p.d_k, w.Zd};
-    if (use_tc(p) && !g_sink.active) {
-        // the five scans side by side (see ScanLanes)
-        ScanLanes* lanes = nullptr;
-        GSA_CUDA(scan_lanes(&lanes));
+    // the reversed scans that share a state run as one kernel each (dv with dI^v, dk with dI^k)
+    ValueSideArgs pIv = adIv, pIk = adIk;
+    KeySideArgs pv = adv, pk = adk;
+    pIv.single = pIk.single = pv.single = pk.single = p.tc_operands == GSA_TC_SINGLE;
+    const bool paired = use_tc(p) && g_pair_scans.load(std::memory_order_relaxed) != 0 &&
+                        rev_pair_supported(pIv, pv, p.m) && rev_pair_supported(pIk, pk, p.m);
+    if (paired && !g_sink.active) {
         GSA_CUDA(cudaEventRecord(lanes->fork, st));
-        for (int i = 0; i < 4; ++i) GSA_CUDA(cudaStreamWaitEvent(lanes->stream[i], lanes->fork, 0));
+        for (int i = early ? 1 : 0; i < 2; ++i) GSA_CUDA(cudaStreamWaitEvent(lanes->stream[i], lanes->fork, 0));
         if (!fused) GSA_CUDA(key_side(p, adq, 0, w.strong, st, dev_status));
-        GSA_CUDA(key_side(p, adv, 1, w.strong, lanes->stream[0], dev_status));
-        GSA_CUDA(value_side(p, adIv, 1, w.strong, lanes->stream[1], dev_status));
+        if (!early) GSA_CUDA(launch_rev_pair_tc(pIv, pv, p.m, w.strong, lanes->stream[0], dev_status));
+        GSA_CUDA(launch_rev_pair_tc(pIk, pk, p.m, w.strong, lanes->stream[1], dev_status));
+        for (int i = 0; i < 2; ++i) {
+            GSA_CUDA(cudaEventRecord(lanes->join[i], lanes->stream[i]));
+            GSA_CUDA(cudaStreamWaitEvent(st, lanes->join[i], 0));
+        }
+    } else if (paired) {
+        if (!fused) GSA_LAUNCH("bwd_dq_key_side", key_side(p, adq, 0, w.strong, st, dev_status));
+        GSA_LAUNCH("bwd_dv_dIv_pair_rev", launch_rev_pair_tc(pIv, pv, p.m, w.strong, st, dev_status));
+        GSA_LAUNCH("bwd_dk_dIk_pair_rev", launch_rev_pair_tc(pIk, pk, p.m, w.strong, st, dev_status));
+    } else if (use_tc(p) && !g_sink.active) {
+        // the five scans side by side (see ScanLanes)
+        GSA_CUDA(cudaEventRecord(lanes->fork, st));
+        for (int i = early ? 2 : 0; i < 4; ++i) GSA_CUDA(cudaStreamWaitEvent(lanes->stream[i], lanes->fork, 0));
+        if (!fused) GSA_CUDA(key_side(p, adq, 0, w.strong, st, dev_status));
+        if (!early) {
+            GSA_CUDA(key_side(p, adv, 1, w.strong, lanes->stream[0], dev_status));
+            GSA_CUDA(value_side(p, adIv, 1, w.strong, lanes->stream[1], dev_status));
+        }
         GSA_CUDA(key_side(p, adk, 1, w.strong, lanes->stream[2], dev_status));
         GSA_CUDA(value_side(p, adIk, 1, w.strong, lanes->stream[3], dev_status));
         for (int i = 0; i < 4; ++i) {
@@ -941,6 +1014,8 @@ gsa_status_t gsa_release_streams(void) {
     if (scan_lanes_release() != cudaSuccess || side_lane_release() != cudaSuccess) return GSA_ERR_CUDA;
     return GSA_OK;
 }
+
+int32_t gsa_dev_pair_scans(int32_t enable) { return g_pair_scans.exchange(enable != 0 ? 1 : 0); }
 
 gsa_status_t gsa_timing_begin(int32_t capacity) {
     if (capacity < 1 || capacity > (1 << 20) || g_sink.active) return GSA_ERR_INVALID_ARG;

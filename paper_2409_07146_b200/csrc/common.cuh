@@ -228,6 +228,11 @@ cudaError_t launch_value_side_general(const ValueSideArgs& a, int M, int reverse
                                       cudaStream_t st, int32_t* dev_status);
 cudaError_t launch_key_side_general(const KeySideArgs& a, int M, int reverse, const int* strong_flag,
                                     cudaStream_t st, int32_t* dev_status);
+// The two reversed scans that share a state (dv with dI^v, dk with dI^k) as one kernel
+// (chunk_tc_pair.cu): av / ak are the arguments the single reversed scans would get.
+bool rev_pair_supported(const ValueSideArgs& av, const KeySideArgs& ak, int M);
+cudaError_t launch_rev_pair_tc(const ValueSideArgs& av, const KeySideArgs& ak, int M, const int* strong_flag,
+                               cudaStream_t st, int32_t* dev_status);
 // the side stream of the calling host thread on the current device, with its fork / join events
 struct SideLane {
     cudaStream_t stream = nullptr;

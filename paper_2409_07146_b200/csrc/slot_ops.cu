@@ -341,14 +341,14 @@ __global__ void __launch_bounds__(256) slot_softmax_bwd_kernel(const float* __re
     }
     if (!live || skip) return;
     if (!pending) {       // (as in the forward: fp32 p and dz only where a non-pipelined kernel reads them)
-        st_vec(p + idx, e);
+        if (p != nullptr) st_vec(p + idx, e);      // (p == NULL: the forward's p is kept and in use)
         st_vec(dz + idx, dzv);
     }
     st_vec(u + idx, uv);
-    if (p_decayed != nullptr) {
+    if (dz_decayed != nullptr) {
 #pragma unroll
         for (int r = 0; r < R; ++r) { e[r] *= eg[r]; dzv[r] *= eg[r]; }
-        st_split<M>(p_decayed + row * 2 * M, l * R, e);
+        if (p_decayed != nullptr) st_split<M>(p_decayed + row * 2 * M, l * R, e);
         st_split<M>(dz_decayed + row * 2 * M, l * R, dzv);
     }
 }

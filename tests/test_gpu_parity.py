@@ -419,6 +419,28 @@ def test_bwd_tc_strong_forgetting_saved_logits():
     print("bwd tc strong saved", check_bwd(got, ref, TOL["bf16"], tc=True))
 
 
+@pytest.mark.parametrize("T,final", [(128, False), (385, True), (1100, True)])
+def test_bwd_tc_pair_kernels_and_single_reversed_scans(T, final):
+    # The reversed scans of the backward run as two pair kernels (dv with dI^v, dk with dI^k; App. B) by
+    # default and as four single scans behind the development switch: both against the oracle, and
+    # against each other (same operand roundings; the order of a few fp32 additions differs).
+    B, H, dk, dv, m = 2, 2, 128, 256, 64
+    d = rand_inputs(1300 + T, B, T, H, dk, dv, m, "bf16", init=True, final_grads=final)
+    res = {}
+    try:
+        for pair in (True, False):
+            gsa.gsa_dev_pair_scans(pair)
+            got, ref = run_bwd(d, B, T, H, dk, dv, m, "bf16", impl="tc", scale=0.9)
+            check_bwd(got, ref, TOL["bf16"], tc=True)
+            res[pair] = got
+    finally:
+        gsa.gsa_dev_pair_scans(True)
+    for n in ("dk", "dv", "dgate", "dK0", "dV0"):
+        if n in res[True] and res[True][n] is not None:
+            # (bfloat16 outputs: the two roundings may fall on neighbouring values)
+            assert rel_err(res[True][n], res[False][n], n in BF16_IO) <= (2e-2 if n in BF16_IO else 1e-3), n
+
+
 # ------------------------------------------------------------------ gate from logits (Sec. 3.3)
 @pytest.mark.parametrize("io,impl", [("f32", "auto"), ("bf16", "simt"), ("bf16", "tc")])
 def test_logit_gate_fwd_bwd(io, impl):
