@@ -238,7 +238,7 @@ value_side_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_cons
 
     if (warp == kComputeThreads / 32) {
         // =============================== issuing warp: TMA loads / stores and all MMAs
-        if (tid == kComputeThreads) {
+        if (elect_one()) {
             auto load_x = [&](int it) {
                 const int t = chunk_t0(it);
                 mbar_expect_tx(&ctl->bar_x, 4 * kPanelB);
@@ -642,7 +642,7 @@ key_side_tc_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_consta
 
     if (warp == kComputeThreads / 32) {
         // =============================== issuing warp: TMA loads / stores and all MMAs
-        if (tid == kComputeThreads) {
+        if (elect_one()) {
             auto load_v = [&](int it) {
                 const int t = chunk_t0(it);
                 mbar_expect_tx(&ctl->bar_x, 2 * kPanelB);

@@ -198,7 +198,8 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
     const uint32_t tmem = ctl->tmem_slot;
     const int nchunks = (a.T + kCT - 1) / kCT;
 
-    if (tid == kFCopy) {
+    if (warp == kFCopy / 32) {
+        if (elect_one()) {
         // =============================== copy lane: every tile load and store
         auto load_xk = [&](int n) {      // (expects the whole first-pass tile pair)
             mbar_expect_tx(&ctl->bar_x1, 4 * kPanelB);
@@ -250,7 +251,9 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
             bulk_wait_read();
             if (more) load_xv(n + 1);
         }
-    } else if (tid == kFMma) {
+        }
+    } else if (warp == kFMma / 32) {
+        if (elect_one()) {
         // =============================== MMA lane
         constexpr uint32_t idescP = make_idesc(128, 128, false, false);     // xq xk^T
         constexpr uint32_t idescO1 = make_idesc(128, 2 * kM, false, true);  // xq x [S_hi | S_lo] (MN-major B)
@@ -366,6 +369,7 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
             mma_commit(&ctl->bar_o2);
             PROF_MARK();
             PROF_DUMP("fused mma");
+        }
         }
     } else if (tid < kComputeThreads) {
         // =============================== compute threads

@@ -27,7 +27,7 @@ using namespace tcchunk;
 // 8 compute warps, one warp whose lane 0 issues every MMA, one warp whose lane 0 requests every
 // tile copy (loads and stores)
 constexpr int kLeanThreads = kComputeThreads + 64;
-constexpr int kMmaThread = kComputeThreads, kCopyThread = kComputeThreads + 32;
+constexpr int kMmaWarp = kComputeThreads / 32, kCopyWarp = kMmaWarp + 1;   // (entered by one elected lane, see elect_one)
 
 struct LeanCtl {
     // filled by TMA
@@ -140,7 +140,8 @@ value_side_lean_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_co
     const int nchunks = (a.T + kCT - 1) / kCT;
     auto chunk_t0 = [&](int n) { return (REV ? nchunks - 1 - n : n) * kCT; };
 
-    if (tid == kCopyThread) {
+    if (warp == kCopyWarp) {
+        if (elect_one()) {
         // =============================== copy lane: every tile load and store
         auto load_x = [&](int n) {
             const int t = chunk_t0(n), st = n & 1;
@@ -186,7 +187,9 @@ value_side_lean_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_co
             bulk_wait_read();
             if (n + 2 < nchunks) load_w(n + 2);
         }
-    } else if (tid == kMmaThread) {
+        }
+    } else if (warp == kMmaWarp) {
+        if (elect_one()) {
         // =============================== MMA lane
         constexpr uint32_t idescP = make_idesc(128, 128, false, false);    // xq xk^T
         constexpr uint32_t idescO = make_idesc(128, 2 * kM, false, true);  // xq x state copy [S_hi | S_lo] (MN-major B)
@@ -262,6 +265,7 @@ value_side_lean_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_co
             }
             PROF_MARK();
             PROF_DUMP("value_side lean mma");
+        }
         }
     } else if (tid < kComputeThreads) {
         // =============================== compute threads
@@ -396,7 +400,8 @@ key_side_lean_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_cons
     const int nchunks = (a.T + kCT - 1) / kCT;
     auto chunk_t0 = [&](int n) { return (REV ? nchunks - 1 - n : n) * kCT; };
 
-    if (tid == kCopyThread) {
+    if (warp == kCopyWarp) {
+        if (elect_one()) {
         // =============================== copy lane: every tile load and store
         auto load_v = [&](int n) {
             const int t = chunk_t0(n), st = n & 1;
@@ -440,7 +445,9 @@ key_side_lean_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_cons
             bulk_wait_read();
             if (n + 2 < nchunks) load_v(n + 2);
         }
-    } else if (tid == kMmaThread) {
+        }
+    } else if (warp == kMmaWarp) {
+        if (elect_one()) {
         // =============================== MMA lane
         constexpr uint32_t idescA = make_idesc(128, 128, false, false);   // Q~ K~^T
         constexpr uint32_t idescO = make_idesc(128, kDST, false, false);  // Q~ x state copy (K-major B)
@@ -532,6 +539,7 @@ key_side_lean_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_cons
             }
             PROF_MARK();
             PROF_DUMP("key_side lean mma");
+        }
         }
     } else if (tid < kComputeThreads) {
         // =============================== compute threads
@@ -676,7 +684,8 @@ state_scan_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
     const int nchunks = (T + kCT - 1) / kCT;
     auto chunk_t0 = [&](int n) { return (REV ? nchunks - 1 - n : n) * kCT; };
 
-    if (tid == kCopyThread) {
+    if (warp == kCopyWarp) {
+        if (elect_one()) {
         // =============================== copy lane
         auto load = [&](int n) {
             const int t = chunk_t0(n), st = n % kScanStages;
@@ -694,7 +703,9 @@ state_scan_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
             if (ctl->abort) break;
             load(n + kScanStages);
         }
-    } else if (tid == kMmaThread) {
+        }
+    } else if (warp == kMmaWarp) {
+        if (elect_one()) {
         // =============================== MMA lane
         constexpr uint32_t idescU = make_idesc(128, 2 * kM, true, true);   // X^T (MN-major A) x [W_hi | W_lo] (MN-major B)
         auto mnmaj = [](int kk) { return (uint32_t)(kk * 2048); };
@@ -712,6 +723,7 @@ state_scan_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
                 mma_bf16(tmem + 128 * (n & 1), desc_advance(dX, mnmaj(kk)), desc_advance(dW, mnmaj(kk)), idescU, kk > 0);
             mma_commit(&ctl->bar_u[n & 1]);
             mma_commit(&ctl->bar_free[st]);
+        }
         }
     } else if (tid < kComputeThreads) {
         // =============================== compute threads: S[c = row][s], slots sb .. sb+31

@@ -25,7 +25,7 @@ using namespace tc;
 using namespace tcchunk;
 
 constexpr int kPairThreads = kComputeThreads + 64;   // 8 compute warps, an MMA lane, a copy lane
-constexpr int kMmaThread = kComputeThreads, kCopyThread = kComputeThreads + 32;
+constexpr int kMmaWarp = kComputeThreads / 32, kCopyWarp = kMmaWarp + 1;
 
 struct PairCtl {
     // filled by TMA
@@ -35,8 +35,8 @@ struct PairCtl {
     // signalled by tcgen05.commit
     uint64_t bar_p;        // P = Y X^T of a chunk
     uint64_t bar_a;        // A = Q W^T of a chunk
-    uint64_t bar_mma1;     // state product U and the two inter-chunk products
-    uint64_t bar_yqfree;   // (the same moment, for the copy lane) Y and Q are consumed
+    uint64_t bar_yqfree;   // the two inter-chunk products (for the copy lane: Y and Q are consumed)
+    uint64_t bar_mma1;     // state product U
     uint64_t bar_v4;       // value-side output accumulator complete
     uint64_t bar_k4;       // key-side output accumulator complete
     // signalled by the compute threads (one arrival after their barrier)
@@ -109,7 +109,8 @@ rev_pair_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant_
     const int nchunks = (T + kCT - 1) / kCT;
     auto chunk_t0 = [&](int n) { return (nchunks - 1 - n) * kCT; };     // from the last chunk down
 
-    if (tid == kCopyThread) {
+    if (warp == kCopyWarp) {
+        if (elect_one()) {
         // =============================== copy lane: every tile load and store
         auto load_x = [&](int n) {
             const int t = chunk_t0(n), st = n & 1;
@@ -142,7 +143,15 @@ rev_pair_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant_
         }
         for (int n = 0; n < nchunks && !ctl->abort; ++n) {
             const int t = chunk_t0(n), st = n & 1;
-            // Y and Q are consumed once the inter-chunk products of chunk n are done
+            // Y and Q are consumed once the inter-chunk products of chunk n are done; their next tiles are
+            // asked into L2 ahead of that, so that the copy itself is short
+            if (n + 1 < nchunks) {
+                const int tn = chunk_t0(n + 1);
+                tma_prefetch_4d(&mapY, d0, h, tn, b);
+                if (d0 + 64 < D) tma_prefetch_4d(&mapY, d0 + 64, h, tn, b);
+                tma_prefetch_4d(&mapQ, 0, h, tn, b);
+                tma_prefetch_4d(&mapQ, 64, h, tn, b);
+            }
             PAIR_WAIT(&ctl->bar_yqfree, n & 1);
             if (ctl->abort) break;
             if (n + 1 < nchunks) load_yq(n + 1);
@@ -166,7 +175,9 @@ rev_pair_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant_
                 load_w(n + 2);
             }
         }
-    } else if (tid == kMmaThread) {
+        }
+    } else if (warp == kMmaWarp) {
+        if (elect_one()) {
         // =============================== MMA lane
         constexpr uint32_t idescP = make_idesc(128, 128, false, false);    // Y X^T and Q W^T
         constexpr uint32_t idescU = make_idesc(128, kM, true, true);       // X^T (MN-major A) x W part (MN-major B)
@@ -214,24 +225,11 @@ rev_pair_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant_
             const uint64_t dXm = desc_mnmajor(xs, 0, kPanelB);
             const uint64_t dWh = desc_mnmajor(ws, 0, kPanelB), dWl = desc_mnmajor(ws + kPanelB, 0, kPanelB);
             PROF_MARK();
-            // ---- state product U = X^T W: the U accumulator was read, and the state copy written, in chunk n-1
+            // ---- inter-chunk products first (Y and Q, single-staged, are free for the next chunk's tiles behind
+            // them): the state copy was written in chunk n-1, whose rows have been read out of the accumulators
             PAIR_WAIT(&ctl->bar_sb, n & 1);
+            if (n >= 1) PAIR_WAIT(&ctl->bar_outv[(n - 1) & 1], ((n - 1) >> 1) & 1);
             tc_fence_after_sync();
-            PROF_MARK();
-#pragma unroll
-            for (int kk = 0; kk < kCT / 16; ++kk)
-                mma_bf16(tmem + kPcU, desc_advance(dXm, mnmaj(kk)), desc_advance(dWh, mnmaj(kk)), idescU, kk > 0);
-            if (PAIRS) {
-#pragma unroll
-                for (int kk = 0; kk < kCT / 16; ++kk)
-                    mma_bf16(tmem + kPcU, desc_advance(dXm, mnmaj(kk)), desc_advance(dWl, mnmaj(kk)), idescU, true);
-            }
-            PROF_MARK();
-            // ---- inter-chunk products, once the previous chunk's rows have been read out of their accumulators
-            if (n >= 1) {
-                PAIR_WAIT(&ctl->bar_outv[(n - 1) & 1], ((n - 1) >> 1) & 1);
-                tc_fence_after_sync();
-            }
             PROF_MARK();
 #pragma unroll
             for (int kk = 0; kk < kDST / 16; ++kk)
@@ -258,8 +256,18 @@ rev_pair_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant_
                 for (int kk = 0; kk < kM / 16; ++kk)
                     mma_bf16(tmem + kPcO2, desc_advance(dQh, kmaj(kk)), desc_advance(dSkl, kmaj(kk)), idescQS, true);
             }
-            mma_commit(&ctl->bar_mma1);
             mma_commit(&ctl->bar_yqfree);
+            PROF_MARK();
+            // ---- state product U = X^T W (its accumulator was read in chunk n-1, before the state copy was written)
+#pragma unroll
+            for (int kk = 0; kk < kCT / 16; ++kk)
+                mma_bf16(tmem + kPcU, desc_advance(dXm, mnmaj(kk)), desc_advance(dWh, mnmaj(kk)), idescU, kk > 0);
+            if (PAIRS) {
+#pragma unroll
+                for (int kk = 0; kk < kCT / 16; ++kk)
+                    mma_bf16(tmem + kPcU, desc_advance(dXm, mnmaj(kk)), desc_advance(dWl, mnmaj(kk)), idescU, true);
+            }
+            mma_commit(&ctl->bar_mma1);
             PROF_MARK();
             // ---- value-side intra-chunk product: masked P (bf16 pair, in place in tensor memory) x W
             PAIR_WAIT(&ctl->bar_pm, n & 1);
@@ -308,6 +316,7 @@ rev_pair_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant_
             }
             PROF_MARK();
             PROF_DUMP("rev_pair mma");
+        }
         }
     } else if (tid < kComputeThreads) {
         // =============================== compute threads

@@ -31,8 +31,13 @@ constexpr int kColO2 = 384;    // value_side: intra-chunk output [128 x 128], hi
 #ifdef GSA_TC_PROF
 #define PROF_DECL long long prof_t[32]; int prof_n = 0;
 #define PROF_MARK() do { if (prof_n < 32) prof_t[prof_n++] = clock64(); } while (0)
+#ifdef GSA_TC_PROF_ABS
+#define PROF_DUMP(name) do { if (blockIdx.x == 0 && blockIdx.y == 0 && (tid == 0 || tid == 256) && (it == 5 || it == 6)) { \
+    printf("%s it %d:", name, it); for (int i_ = 0; i_ < prof_n; ++i_) printf(" %lld", prof_t[i_] % 1000000); printf("\n"); } prof_n = 0; } while (0)
+#else
 #define PROF_DUMP(name) do { if (blockIdx.x == 0 && blockIdx.y == 0 && ((tid == 0 && it == 6) || (tid == 256 && it == 4))) { \
     printf("%s:", name); for (int i_ = 1; i_ < prof_n; ++i_) printf(" %lld", prof_t[i_] - prof_t[i_ - 1]); printf("\n"); } prof_n = 0; } while (0)
+#endif
 #else
 #define PROF_DECL
 #define PROF_MARK() do {} while (0)
