@@ -33,7 +33,12 @@ constexpr int kColO2 = 384;    // value_side: intra-chunk output [128 x 128], hi
 #define PROF_MARK() do { if (prof_n < 32) prof_t[prof_n++] = clock64(); } while (0)
 #ifdef GSA_TC_PROF_ABS
 #define PROF_DUMP(name) do { if (blockIdx.x == 0 && blockIdx.y == 0 && (tid == 0 || tid == 256) && (it == 5 || it == 6)) { \
-    printf("%s it %d:", name, it); for (int i_ = 0; i_ < prof_n; ++i_) printf(" %lld", prof_t[i_] % 1000000); printf("\n"); } prof_n = 0; } while (0)
+    long long b_ = prof_t[0] % 1000000; for (int i_ = prof_n; i_ < 16; ++i_) prof_t[i_] = prof_t[0]; \
+    printf("%s tid %d it %d base %lld: %lld %lld %lld %lld %lld %lld %lld %lld %lld %lld %lld %lld %lld %lld %lld\n", name, (int)tid, it, b_, \
+           prof_t[1] - prof_t[0], prof_t[2] - prof_t[0], prof_t[3] - prof_t[0], prof_t[4] - prof_t[0], prof_t[5] - prof_t[0], \
+           prof_t[6] - prof_t[0], prof_t[7] - prof_t[0], prof_t[8] - prof_t[0], prof_t[9] - prof_t[0], prof_t[10] - prof_t[0], \
+           prof_t[11] - prof_t[0], prof_t[12] - prof_t[0], prof_t[13] - prof_t[0], prof_t[14] - prof_t[0], prof_t[15] - prof_t[0]); } \
+    prof_n = 0; } while (0)
 #else
 #define PROF_DUMP(name) do { if (blockIdx.x == 0 && blockIdx.y == 0 && ((tid == 0 && it == 6) || (tid == 256 && it == 4))) { \
     printf("%s:", name); for (int i_ = 1; i_ < prof_n; ++i_) printf(" %lld", prof_t[i_] - prof_t[i_ - 1]); printf("\n"); } prof_n = 0; } while (0)
