@@ -38,10 +38,11 @@ WORKLOAD = "train_1p3b"
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the tensor-core kernels on this
 # workload, from one `ncu --set full` capture (profiles/step_kernels_train_1p3b_ncu_full.md).
 NCU_TRAFFIC = {
-    "pass1_value_side": 186965760, "bwd_dp_value_side": 185658112,
+    "pass1_value_side": 187423232, "bwd_dp_value_side": 186575872,
     "bwd_dIv_value_side_rev": 188858112, "bwd_dIk_value_side_rev": 187463680,
-    "pass2_key_side": 129739520, "bwd_dq_key_side": 135778048,
+    "pass2_key_side": 130322432, "bwd_dq_key_side": 135258368,
     "bwd_dv_key_side_rev": 130483200, "bwd_dk_key_side_rev": 132975616,
+    "bwd_dv_dIv_pair_rev": 258483968, "bwd_dk_dIk_pair_rev": 257145344,
     "gate_cumsum": 17926144, "slot_softmax": 92744448, "slot_softmax_bwd": 118787072,
     "gate_grad": 231503872,     # local + scan + carry
 }
@@ -504,10 +505,11 @@ def run_ours(args):
                     "traffic": traffic, "traffic_source": ("profiles/step_kernels_train_1p3b_ncu_full.md (one ncu capture of "
                                                            "this workload; not measured in this run)") if traffic else None,
                     "frac_on_fused_bytes": fused_bytes / (avg_ms * 1e-3) / 1e9 / pk["hbm_gbs"],
-                    "limiter": ("tensor-pipe issue rate: the chunk loop issues its tcgen05.mma (a quarter of them only "
-                                "for the high/low operand pairs) back to back at 80-90 cycles each; ncu shows the tensor "
-                                "pipe 53-63% active and DRAM at 30-46% of peak, so HBM is the bound of the ideal fused "
-                                "layer, not what limits this kernel"),
+                    "limiter": ("the chunk loop is a chain of tensor-pipe products and compute-thread phases (mask, state update, "
+                                "read-out) that wait for one another: per chunk of the pair kernel the pipe needs 5.4-5.8 k cycles "
+                                "(the issued tcgen05.mma sequence timed alone), the compute threads 5.1 k, and a chunk takes 6.7-6.9 k; "
+                                "ncu shows the tensor pipe 58-67% active and DRAM at 32-50% of peak, so HBM is the bound of the "
+                                "ideal fused layer, not what limits this kernel"),
                     "peak_source": pk["source"],
                     "share_of_step": sum(k_["share"] for k_ in members)}
         if fn.endswith("_side_lean_kernel") or fn in ("fused_pair_kernel", "rev_pair_kernel"):
@@ -516,8 +518,8 @@ def run_ours(args):
             roofline["alg_tflops"] = fl / (avg_ms * 1e-3) / 1e12
             roofline["frac_of_bf16_peak"] = roofline["alg_tflops"] / pk["bf16_tflops"]
             roofline["note"] = ("flops per byte of the launch %.0f against a machine balance of %.0f: the HBM side of "
-                                "the roofline bounds it; the kernel itself is limited by the tensor pipe's issue rate "
-                                "on high/low operand pairs" % (fl / alg, pk["bf16_tflops"] * 1e12 / (pk["hbm_gbs"] * 1e9)))
+                                "the roofline bounds it; a third to a half of the tcgen05.mma of a chunk exist only for "
+                                "the high/low operand pairs that keep every tensor within tolerance" % (fl / alg, pk["bf16_tflops"] * 1e12 / (pk["hbm_gbs"] * 1e9)))
         step_bytes = step_algorithmic_bytes(w)
         whole = {"alg_bytes_per_step": step_bytes,
                  "achieved_gbs": step_bytes / (ms_step * 1e-3) / 1e9,

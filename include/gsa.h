@@ -212,9 +212,11 @@ GSA_API gsa_status_t gsa_bwd(const gsa_params_t* params, const void* q, const vo
  * The same two calls for a training step that trades memory for the backward's gate kernel
  * (the save-instead-of-recompute side of the trade-off the paper discusses in Sec. 4,
  * "Efficiency"): gsa_fwd_save_gate leaves the products of chunk_cumsum (the cumulative log
- * gate, the input gate, its decayed bf16 rows and the per-(batch, head) decay flags) and, where
- * a long sequence is cut into segments, the segments' decay, the memories entering every
- * segment and the final memories in gate_save, a device block of gsa_workspace_bytes(params, GSA_WS_GATE) bytes, 256-byte
+ * gate, the input gate, its decayed bf16 rows and the per-(batch, head) decay flags), on the
+ * tensor-core path also the forward's slot weights p (as the backward's reversed scans read them:
+ * they depend on the saved logits only, and with them in hand the backward starts its dv scan at
+ * once) and, where a long sequence is cut into segments, the segments' decay, the memories entering
+ * every segment and the final memories in gate_save, a device block of gsa_workspace_bytes(params, GSA_WS_GATE) bytes, 256-byte
  * aligned, owned by the caller; gsa_bwd_saved_gate reads them from there instead of running
  * the gate kernel (and the segments' forward-direction state runs) again.  Both calls must use the same params and the same gate tensor;
  * nothing checks that.  A missing, misaligned or short block is GSA_ERR_WORKSPACE.
