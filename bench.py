@@ -505,11 +505,11 @@ def run_ours(args):
                     "traffic": traffic, "traffic_source": ("profiles/step_kernels_train_1p3b_ncu_full.md (one ncu capture of "
                                                            "this workload; not measured in this run)") if traffic else None,
                     "frac_on_fused_bytes": fused_bytes / (avg_ms * 1e-3) / 1e9 / pk["hbm_gbs"],
-                    "limiter": ("the chunk loop is a chain of tensor-pipe products and compute-thread phases (mask, state update, "
-                                "read-out) that wait for one another: per chunk of the pair kernel the pipe needs 5.4-5.8 k cycles "
-                                "(the issued tcgen05.mma sequence timed alone), the compute threads 5.1 k, and a chunk takes 6.7-6.9 k; "
-                                "ncu shows the tensor pipe 58-67% active and DRAM at 32-50% of peak, so HBM is the bound of the "
-                                "ideal fused layer, not what limits this kernel"),
+                    "limiter": ("tile-copy throughput per SM: a CTA of a scan moves 2-3 MB through two shared-memory stages and one "
+                                "SM sustains about 41 GB/s of TMA copies (knock-out builds: a value_side scan with nothing but its "
+                                "copies and barrier hand-shakes takes 36.6 of its 50.8 us; removing the masks, the state update, the "
+                                "read-out or any group of MMAs changes it by 1-3 us each); ncu: tensor pipe 58-67% active, DRAM at "
+                                "32-50% of peak, 128 CTAs on 148 SMs"),
                     "peak_source": pk["source"],
                     "share_of_step": sum(k_["share"] for k_ in members)}
         if fn.endswith("_side_lean_kernel") or fn in ("fused_pair_kernel", "rev_pair_kernel"):
