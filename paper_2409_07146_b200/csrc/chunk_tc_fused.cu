@@ -200,176 +200,176 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
 
     if (warp == kFCopy / 32) {
         if (elect_one()) {
-        // =============================== copy lane: every tile load and store
-        auto load_xk = [&](int n) {      // (expects the whole first-pass tile pair)
-            mbar_expect_tx(&ctl->bar_x1, 4 * kPanelB);
-            tma_load_4d(sXk, &mapK, &ctl->bar_x1, d0, h, n * kCT, b);
-            tma_load_4d(sXk + kPanelB, &mapK, &ctl->bar_x1, d0 + 64, h, n * kCT, b);
-        };
-        auto load_xq = [&](int n) {
-            tma_load_4d(sXq, &mapQ, &ctl->bar_x1, d0, h, n * kCT, b);
-            tma_load_4d(sXq + kPanelB, &mapQ, &ctl->bar_x1, d0 + 64, h, n * kCT, b);
-        };
-        auto load_w = [&](int n) {
-            mbar_expect_tx(&ctl->bar_w, 2 * kPanelB);
-            tma_load_4d(sW, &mapW, &ctl->bar_w, 0, h, n * kCT, b);
-            tma_load_4d(sW + kPanelB, &mapW, &ctl->bar_w, 64, h, n * kCT, b);
-        };
-        auto load_xv = [&](int n) {
-            mbar_expect_tx(&ctl->bar_xv, 2 * kPanelB);
-            tma_load_4d(sXv, &mapV, &ctl->bar_xv, d0, h, n * kCT, b);
-            tma_load_4d(sXv + kPanelB, &mapV, &ctl->bar_xv, d0 + 64, h, n * kCT, b);
-        };
-        prefetch_tmap(&mapQ); prefetch_tmap(&mapK); prefetch_tmap(&mapW); prefetch_tmap(&mapV); prefetch_tmap(&mapO);
-        load_xk(0);
-        load_xq(0);
-        load_w(0);
-        load_xv(0);
-        for (int n = 0; n < nchunks && !ctl->abort; ++n) {
-            const uint32_t ph = n & 1;
-            const bool more = n + 1 < nchunks;
-            // the first pass's tiles are consumed once its state products are done; their places then hold
-            // this CTA's staged partial sums (xk) and the peers' (xq): free again once the peers have copied
-            // theirs out and this CTA has summed its rows
-            FUSED_WAIT(&ctl->bar_fx1, ph);
-            if (NSL > 1) FUSED_WAIT(&ctl->bar_txdone, ph);
-            FUSED_WAIT(&ctl->bar_rxdone, ph);
-            if (more && !ctl->abort) {
-                load_xk(n + 1);
-                load_xq(n + 1);
+            // =============================== copy lane: every tile load and store
+            auto load_xk = [&](int n) {      // (expects the whole first-pass tile pair)
+                mbar_expect_tx(&ctl->bar_x1, 4 * kPanelB);
+                tma_load_4d(sXk, &mapK, &ctl->bar_x1, d0, h, n * kCT, b);
+                tma_load_4d(sXk + kPanelB, &mapK, &ctl->bar_x1, d0 + 64, h, n * kCT, b);
+            };
+            auto load_xq = [&](int n) {
+                tma_load_4d(sXq, &mapQ, &ctl->bar_x1, d0, h, n * kCT, b);
+                tma_load_4d(sXq + kPanelB, &mapQ, &ctl->bar_x1, d0 + 64, h, n * kCT, b);
+            };
+            auto load_w = [&](int n) {
+                mbar_expect_tx(&ctl->bar_w, 2 * kPanelB);
+                tma_load_4d(sW, &mapW, &ctl->bar_w, 0, h, n * kCT, b);
+                tma_load_4d(sW + kPanelB, &mapW, &ctl->bar_w, 64, h, n * kCT, b);
+            };
+            auto load_xv = [&](int n) {
+                mbar_expect_tx(&ctl->bar_xv, 2 * kPanelB);
+                tma_load_4d(sXv, &mapV, &ctl->bar_xv, d0, h, n * kCT, b);
+                tma_load_4d(sXv + kPanelB, &mapV, &ctl->bar_xv, d0 + 64, h, n * kCT, b);
+            };
+            prefetch_tmap(&mapQ); prefetch_tmap(&mapK); prefetch_tmap(&mapW); prefetch_tmap(&mapV); prefetch_tmap(&mapO);
+            load_xk(0);
+            load_xq(0);
+            load_w(0);
+            load_xv(0);
+            for (int n = 0; n < nchunks && !ctl->abort; ++n) {
+                const uint32_t ph = n & 1;
+                const bool more = n + 1 < nchunks;
+                // the first pass's tiles are consumed once its state products are done; their places then hold
+                // this CTA's staged partial sums (xk) and the peers' (xq): free again once the peers have copied
+                // theirs out and this CTA has summed its rows
+                FUSED_WAIT(&ctl->bar_fx1, ph);
+                if (NSL > 1) FUSED_WAIT(&ctl->bar_txdone, ph);
+                FUSED_WAIT(&ctl->bar_rxdone, ph);
+                if (more && !ctl->abort) {
+                    load_xk(n + 1);
+                    load_xq(n + 1);
+                }
+                // the decayed input gate is consumed once the second pass's state products are done
+                FUSED_WAIT(&ctl->bar_fw, ph);
+                if (more && !ctl->abort) load_w(n + 1);
+                // the xv tile is consumed once the second intra-chunk product is done; the output rows are
+                // staged in its place, and when those have left the buffer takes the next tile
+                FUSED_WAIT(&ctl->bar_out, ph);
+                if (ctl->abort) break;
+                tma_store_4d(&mapO, sXv, d0, h, n * kCT, b);
+                tma_store_4d(&mapO, sXv + kPanelB, d0 + 64, h, n * kCT, b);
+                bulk_commit();
+                bulk_wait_read();
+                if (more) load_xv(n + 1);
             }
-            // the decayed input gate is consumed once the second pass's state products are done
-            FUSED_WAIT(&ctl->bar_fw, ph);
-            if (more && !ctl->abort) load_w(n + 1);
-            // the xv tile is consumed once the second intra-chunk product is done; the output rows are
-            // staged in its place, and when those have left the buffer takes the next tile
-            FUSED_WAIT(&ctl->bar_out, ph);
-            if (ctl->abort) break;
-            tma_store_4d(&mapO, sXv, d0, h, n * kCT, b);
-            tma_store_4d(&mapO, sXv + kPanelB, d0 + 64, h, n * kCT, b);
-            bulk_commit();
-            bulk_wait_read();
-            if (more) load_xv(n + 1);
-        }
         }
     } else if (warp == kFMma / 32) {
         if (elect_one()) {
-        // =============================== MMA lane
-        constexpr uint32_t idescP = make_idesc(128, 128, false, false);     // xq xk^T
-        constexpr uint32_t idescO1 = make_idesc(128, 2 * kM, false, true);  // xq x [S_hi | S_lo] (MN-major B)
-        constexpr uint32_t idescU = make_idesc(128, 2 * kM, true, true);    // x^T (MN-major A) x [W_hi | W_lo]
-        constexpr uint32_t idescI = make_idesc(128, 2 * kM, false, true);   // masked P (tensor memory) x [W_hi | W_lo]
-        constexpr uint32_t idescA = make_idesc(128, 128, false, false);     // Q~ K~^T
-        constexpr uint32_t idescO2 = make_idesc(128, kDST, false, false);   // Q~ x state copy (K-major B)
-        constexpr uint32_t idescV = make_idesc(128, kDST, false, true);     // masked A x xv (MN-major B)
-        auto kmaj = [](int kk) { return (uint32_t)((kk >> 2) * kPanelB + (kk & 3) * 32); };
-        auto mnmaj = [](int kk) { return (uint32_t)(kk * 2048); };
-        const uint64_t dQk = desc_kmajor(smem_u32(sXq), 0), dKk = desc_kmajor(smem_u32(sXk), 0);
-        const uint64_t dKm = desc_mnmajor(smem_u32(sXk), 0, kPanelB);
-        const uint64_t dWm = desc_mnmajor(smem_u32(sW), 0, kPanelB);          // [W_hi | W_lo], N = 128
-        const uint64_t dWk = desc_kmajor(smem_u32(sW), 0), dWkl = desc_kmajor(smem_u32(sW + kPanelB), 0);
-        const uint64_t dS1 = desc_mnmajor(smem_u32(sS1), 0, kPanelB);
-        const uint64_t dV = desc_mnmajor(smem_u32(sXv), 0, kPanelB);
-        const uint64_t dPh = desc_kmajor(smem_u32(sP), 0), dPl = desc_kmajor(smem_u32(sP + kPanelB), 0);
-        const uint64_t dS2 = desc_kmajor(smem_u32(sS2), 0), dS2l = desc_kmajor(smem_u32(sS2 + kPanelB), 0);
-        FUSED_WAIT(&ctl->bar_init, 0);
-        PROF_DECL
-        for (int n = 0; n < nchunks && !ctl->abort; ++n) {
-            const int it = n;
-            (void)it;
-            const uint32_t ph = n & 1;
-            PROF_MARK();
-            // ---- first pass: P = xq xk^T
-            FUSED_WAIT(&ctl->bar_x1, ph);
-            tc_fence_after_sync();
-            PROF_MARK();
+            // =============================== MMA lane
+            constexpr uint32_t idescP = make_idesc(128, 128, false, false);     // xq xk^T
+            constexpr uint32_t idescO1 = make_idesc(128, 2 * kM, false, true);  // xq x [S_hi | S_lo] (MN-major B)
+            constexpr uint32_t idescU = make_idesc(128, 2 * kM, true, true);    // x^T (MN-major A) x [W_hi | W_lo]
+            constexpr uint32_t idescI = make_idesc(128, 2 * kM, false, true);   // masked P (tensor memory) x [W_hi | W_lo]
+            constexpr uint32_t idescA = make_idesc(128, 128, false, false);     // Q~ K~^T
+            constexpr uint32_t idescO2 = make_idesc(128, kDST, false, false);   // Q~ x state copy (K-major B)
+            constexpr uint32_t idescV = make_idesc(128, kDST, false, true);     // masked A x xv (MN-major B)
+            auto kmaj = [](int kk) { return (uint32_t)((kk >> 2) * kPanelB + (kk & 3) * 32); };
+            auto mnmaj = [](int kk) { return (uint32_t)(kk * 2048); };
+            const uint64_t dQk = desc_kmajor(smem_u32(sXq), 0), dKk = desc_kmajor(smem_u32(sXk), 0);
+            const uint64_t dKm = desc_mnmajor(smem_u32(sXk), 0, kPanelB);
+            const uint64_t dWm = desc_mnmajor(smem_u32(sW), 0, kPanelB);          // [W_hi | W_lo], N = 128
+            const uint64_t dWk = desc_kmajor(smem_u32(sW), 0), dWkl = desc_kmajor(smem_u32(sW + kPanelB), 0);
+            const uint64_t dS1 = desc_mnmajor(smem_u32(sS1), 0, kPanelB);
+            const uint64_t dV = desc_mnmajor(smem_u32(sXv), 0, kPanelB);
+            const uint64_t dPh = desc_kmajor(smem_u32(sP), 0), dPl = desc_kmajor(smem_u32(sP + kPanelB), 0);
+            const uint64_t dS2 = desc_kmajor(smem_u32(sS2), 0), dS2l = desc_kmajor(smem_u32(sS2 + kPanelB), 0);
+            FUSED_WAIT(&ctl->bar_init, 0);
+            PROF_DECL
+            for (int n = 0; n < nchunks && !ctl->abort; ++n) {
+                const int it = n;
+                (void)it;
+                const uint32_t ph = n & 1;
+                PROF_MARK();
+                // ---- first pass: P = xq xk^T
+                FUSED_WAIT(&ctl->bar_x1, ph);
+                tc_fence_after_sync();
+                PROF_MARK();
 #pragma unroll
-            for (int kk = 0; kk < kDST / 16; ++kk)
-                mma_bf16(tmem + cP, desc_advance(dQk, kmaj(kk)), desc_advance(dKk, kmaj(kk)), idescP, kk > 0);
-            mma_commit(&ctl->bar_p1);
-            // state products: U = xk^T [W], rows = xq [S] (the U accumulator is shared with the second
-            // pass: its previous contents were read when that pass's state copy was written)
-            PROF_MARK();
-            FUSED_WAIT(&ctl->bar_w, ph);
-            PROF_MARK();
-            if (n >= 1) FUSED_WAIT(&ctl->bar_sb2, (n - 1) & 1);
-            tc_fence_after_sync();
-            PROF_MARK();
+                for (int kk = 0; kk < kDST / 16; ++kk)
+                    mma_bf16(tmem + cP, desc_advance(dQk, kmaj(kk)), desc_advance(dKk, kmaj(kk)), idescP, kk > 0);
+                mma_commit(&ctl->bar_p1);
+                // state products: U = xk^T [W], rows = xq [S] (the U accumulator is shared with the second
+                // pass: its previous contents were read when that pass's state copy was written)
+                PROF_MARK();
+                FUSED_WAIT(&ctl->bar_w, ph);
+                PROF_MARK();
+                if (n >= 1) FUSED_WAIT(&ctl->bar_sb2, (n - 1) & 1);
+                tc_fence_after_sync();
+                PROF_MARK();
 #pragma unroll
-            for (int kk = 0; kk < kCT / 16; ++kk)
-                mma_bf16(tmem + cU, desc_advance(dKm, mnmaj(kk)), desc_advance(dWm, mnmaj(kk)), idescU, kk > 0);
+                for (int kk = 0; kk < kCT / 16; ++kk)
+                    mma_bf16(tmem + cU, desc_advance(dKm, mnmaj(kk)), desc_advance(dWm, mnmaj(kk)), idescU, kk > 0);
 #pragma unroll
-            for (int kk = 0; kk < kDST / 16; ++kk)
-                mma_bf16(tmem + cO1, desc_advance(dQk, kmaj(kk)), desc_advance(dS1, mnmaj(kk)), idescO1, kk > 0);
-            mma_commit(&ctl->bar_s1);
-            mma_commit(&ctl->bar_fx1);
-            // intra-chunk product on top: masked P (bf16 high, then low part, in tensor memory) x [W]
-            PROF_MARK();
-            FUSED_WAIT(&ctl->bar_pm1, ph);
-            tc_fence_after_sync();
-            PROF_MARK();
+                for (int kk = 0; kk < kDST / 16; ++kk)
+                    mma_bf16(tmem + cO1, desc_advance(dQk, kmaj(kk)), desc_advance(dS1, mnmaj(kk)), idescO1, kk > 0);
+                mma_commit(&ctl->bar_s1);
+                mma_commit(&ctl->bar_fx1);
+                // intra-chunk product on top: masked P (bf16 high, then low part, in tensor memory) x [W]
+                PROF_MARK();
+                FUSED_WAIT(&ctl->bar_pm1, ph);
+                tc_fence_after_sync();
+                PROF_MARK();
 #pragma unroll
-            for (int kk = 0; kk < kCT / 16; ++kk)
-                mma_bf16_ta(tmem + cO1, tmem + cP + 64 * (kk >> 2) + 8 * (kk & 3), desc_advance(dWm, mnmaj(kk)), idescI, true);
+                for (int kk = 0; kk < kCT / 16; ++kk)
+                    mma_bf16_ta(tmem + cO1, tmem + cP + 64 * (kk >> 2) + 8 * (kk & 3), desc_advance(dWm, mnmaj(kk)), idescI, true);
 #pragma unroll
-            for (int kk = 0; kk < kCT / 16; ++kk)
-                mma_bf16_ta(tmem + cO1, tmem + cP + 64 * (kk >> 2) + 32 + 8 * (kk & 3), desc_advance(dWm, mnmaj(kk)), idescI,
-                            true);
-            mma_commit(&ctl->bar_o1);
-            // ---- second pass: its state update needs no queries, U = xv^T [W] (the first pass's U has been
-            // read once that pass's state copy is written)
-            PROF_MARK();
-            FUSED_WAIT(&ctl->bar_xv, ph);
-            PROF_MARK();
-            FUSED_WAIT(&ctl->bar_sb1, ph);
-            tc_fence_after_sync();
-            PROF_MARK();
+                for (int kk = 0; kk < kCT / 16; ++kk)
+                    mma_bf16_ta(tmem + cO1, tmem + cP + 64 * (kk >> 2) + 32 + 8 * (kk & 3), desc_advance(dWm, mnmaj(kk)), idescI,
+                                true);
+                mma_commit(&ctl->bar_o1);
+                // ---- second pass: its state update needs no queries, U = xv^T [W] (the first pass's U has been
+                // read once that pass's state copy is written)
+                PROF_MARK();
+                FUSED_WAIT(&ctl->bar_xv, ph);
+                PROF_MARK();
+                FUSED_WAIT(&ctl->bar_sb1, ph);
+                tc_fence_after_sync();
+                PROF_MARK();
 #pragma unroll
-            for (int kk = 0; kk < kCT / 16; ++kk)
-                mma_bf16(tmem + cU, desc_advance(dV, mnmaj(kk)), desc_advance(dWm, mnmaj(kk)), idescU, kk > 0);
-            // A = Q~ K~^T and rows = Q~ [S] once the queries of the chunk have landed from every CTA
-            // (high/low pairs on both factors, low x low dropped)
-            PROF_MARK();
-            FUSED_WAIT_CLUSTER(&ctl->bar_pready, ph);
-            tc_fence_after_sync();
-            PROF_MARK();
+                for (int kk = 0; kk < kCT / 16; ++kk)
+                    mma_bf16(tmem + cU, desc_advance(dV, mnmaj(kk)), desc_advance(dWm, mnmaj(kk)), idescU, kk > 0);
+                // A = Q~ K~^T and rows = Q~ [S] once the queries of the chunk have landed from every CTA
+                // (high/low pairs on both factors, low x low dropped)
+                PROF_MARK();
+                FUSED_WAIT_CLUSTER(&ctl->bar_pready, ph);
+                tc_fence_after_sync();
+                PROF_MARK();
 #pragma unroll
-            for (int kk = 0; kk < kM / 16; ++kk)
-                mma_bf16(tmem + cP, desc_advance(dPh, kmaj(kk)), desc_advance(dWk, kmaj(kk)), idescA, kk > 0);
+                for (int kk = 0; kk < kM / 16; ++kk)
+                    mma_bf16(tmem + cP, desc_advance(dPh, kmaj(kk)), desc_advance(dWk, kmaj(kk)), idescA, kk > 0);
 #pragma unroll
-            for (int kk = 0; kk < kM / 16; ++kk)
-                mma_bf16(tmem + cP, desc_advance(dPl, kmaj(kk)), desc_advance(dWk, kmaj(kk)), idescA, true);
+                for (int kk = 0; kk < kM / 16; ++kk)
+                    mma_bf16(tmem + cP, desc_advance(dPl, kmaj(kk)), desc_advance(dWk, kmaj(kk)), idescA, true);
 #pragma unroll
-            for (int kk = 0; kk < kM / 16; ++kk)
-                mma_bf16(tmem + cP, desc_advance(dPh, kmaj(kk)), desc_advance(dWkl, kmaj(kk)), idescA, true);
-            mma_commit(&ctl->bar_p2);
+                for (int kk = 0; kk < kM / 16; ++kk)
+                    mma_bf16(tmem + cP, desc_advance(dPh, kmaj(kk)), desc_advance(dWkl, kmaj(kk)), idescA, true);
+                mma_commit(&ctl->bar_p2);
 #pragma unroll
-            for (int kk = 0; kk < kM / 16; ++kk)
-                mma_bf16(tmem + cO2, desc_advance(dPh, kmaj(kk)), desc_advance(dS2, kmaj(kk)), idescO2, kk > 0);
+                for (int kk = 0; kk < kM / 16; ++kk)
+                    mma_bf16(tmem + cO2, desc_advance(dPh, kmaj(kk)), desc_advance(dS2, kmaj(kk)), idescO2, kk > 0);
 #pragma unroll
-            for (int kk = 0; kk < kM / 16; ++kk)
-                mma_bf16(tmem + cO2, desc_advance(dPl, kmaj(kk)), desc_advance(dS2, kmaj(kk)), idescO2, true);
+                for (int kk = 0; kk < kM / 16; ++kk)
+                    mma_bf16(tmem + cO2, desc_advance(dPl, kmaj(kk)), desc_advance(dS2, kmaj(kk)), idescO2, true);
 #pragma unroll
-            for (int kk = 0; kk < kM / 16; ++kk)
-                mma_bf16(tmem + cO2, desc_advance(dPh, kmaj(kk)), desc_advance(dS2l, kmaj(kk)), idescO2, true);
-            mma_commit(&ctl->bar_s2);
-            mma_commit(&ctl->bar_fw);
-            // intra-chunk product on top: masked A (high, low) x xv
-            PROF_MARK();
-            FUSED_WAIT(&ctl->bar_pm2, ph);
-            tc_fence_after_sync();
-            PROF_MARK();
+                for (int kk = 0; kk < kM / 16; ++kk)
+                    mma_bf16(tmem + cO2, desc_advance(dPh, kmaj(kk)), desc_advance(dS2l, kmaj(kk)), idescO2, true);
+                mma_commit(&ctl->bar_s2);
+                mma_commit(&ctl->bar_fw);
+                // intra-chunk product on top: masked A (high, low) x xv
+                PROF_MARK();
+                FUSED_WAIT(&ctl->bar_pm2, ph);
+                tc_fence_after_sync();
+                PROF_MARK();
 #pragma unroll
-            for (int kk = 0; kk < kCT / 16; ++kk)
-                mma_bf16_ta(tmem + cO2, tmem + cP + 64 * (kk >> 2) + 8 * (kk & 3), desc_advance(dV, mnmaj(kk)), idescV, true);
+                for (int kk = 0; kk < kCT / 16; ++kk)
+                    mma_bf16_ta(tmem + cO2, tmem + cP + 64 * (kk >> 2) + 8 * (kk & 3), desc_advance(dV, mnmaj(kk)), idescV, true);
 #pragma unroll
-            for (int kk = 0; kk < kCT / 16; ++kk)
-                mma_bf16_ta(tmem + cO2, tmem + cP + 64 * (kk >> 2) + 32 + 8 * (kk & 3), desc_advance(dV, mnmaj(kk)), idescV,
-                            true);
-            mma_commit(&ctl->bar_o2);
-            PROF_MARK();
-            PROF_DUMP("fused mma");
-        }
+                for (int kk = 0; kk < kCT / 16; ++kk)
+                    mma_bf16_ta(tmem + cO2, tmem + cP + 64 * (kk >> 2) + 32 + 8 * (kk & 3), desc_advance(dV, mnmaj(kk)), idescV,
+                                true);
+                mma_commit(&ctl->bar_o2);
+                PROF_MARK();
+                PROF_DUMP("fused mma");
+            }
         }
     } else if (tid < kComputeThreads) {
         // =============================== compute threads

@@ -142,130 +142,130 @@ value_side_lean_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_co
 
     if (warp == kCopyWarp) {
         if (elect_one()) {
-        // =============================== copy lane: every tile load and store
-        auto load_x = [&](int n) {
-            const int t = chunk_t0(n), st = n & 1;
-            unsigned char* sXq = sX + 4 * st * kPanelB;
-            unsigned char* sXk = sXq + 2 * kPanelB;
-            mbar_expect_tx(&ctl->bar_x2[st], 4 * kPanelB);
-            tma_load_4d(sXq, &mapQ, &ctl->bar_x2[st], d0, h, t, b);
-            tma_load_4d(sXq + kPanelB, &mapQ, &ctl->bar_x2[st], d0 + 64, h, t, b);
-            tma_load_4d(sXk, &mapK, &ctl->bar_x2[st], d0, h, t, b);
-            tma_load_4d(sXk + kPanelB, &mapK, &ctl->bar_x2[st], d0 + 64, h, t, b);
-        };
-        auto load_w = [&](int n) {
-            const int t = chunk_t0(n), st = n & 1;
-            mbar_expect_tx(&ctl->bar_w[st], 2 * kPanelB);
-            tma_load_4d(sWd + (2 * st) * kPanelB, &mapWd, &ctl->bar_w[st], 0, h, t, b);
-            tma_load_4d(sWd + (2 * st + 1) * kPanelB, &mapWd, &ctl->bar_w[st], 64, h, t, b);
-        };
-        auto store_out = [&](int n) {
-            const int t = chunk_t0(n);
-            const unsigned char* sOut = sWd + 2 * (n & 1) * kPanelB;
-            tma_store_5d(&mapO, sOut, 0, h, t, b, slice);
-            tma_store_5d(&mapO, sOut + kPanelB, 32, h, t, b, slice);
-            bulk_commit();
-        };
-        prefetch_tmap(&mapQ); prefetch_tmap(&mapK); prefetch_tmap(&mapWd); prefetch_tmap(&mapO);
-        load_x(0);
-        load_w(0);
-        if (nchunks > 1) {
-            load_x(1);
-            load_w(1);
-        }
-        for (int n = 0; n < nchunks && !ctl->abort; ++n) {
-            // the d-sized tiles of chunk n are consumed once its state products are done: their
-            // buffer takes the tiles of chunk n+2
-            LEAN_WAIT(&ctl->bar_free1[n & 1], (n >> 1) & 1);
-            if (n + 2 < nchunks) load_x(n + 2);
-            // the weights are consumed once the intra-chunk product is done; the compute threads then
-            // stage the output rows in their place, and when those have left the buffer takes the
-            // weights of chunk n+2
-            LEAN_WAIT(&ctl->bar_out[n & 1], (n >> 1) & 1);
-            if (ctl->abort) break;
-            store_out(n);
-            bulk_wait_read();
-            if (n + 2 < nchunks) load_w(n + 2);
-        }
+            // =============================== copy lane: every tile load and store
+            auto load_x = [&](int n) {
+                const int t = chunk_t0(n), st = n & 1;
+                unsigned char* sXq = sX + 4 * st * kPanelB;
+                unsigned char* sXk = sXq + 2 * kPanelB;
+                mbar_expect_tx(&ctl->bar_x2[st], 4 * kPanelB);
+                tma_load_4d(sXq, &mapQ, &ctl->bar_x2[st], d0, h, t, b);
+                tma_load_4d(sXq + kPanelB, &mapQ, &ctl->bar_x2[st], d0 + 64, h, t, b);
+                tma_load_4d(sXk, &mapK, &ctl->bar_x2[st], d0, h, t, b);
+                tma_load_4d(sXk + kPanelB, &mapK, &ctl->bar_x2[st], d0 + 64, h, t, b);
+            };
+            auto load_w = [&](int n) {
+                const int t = chunk_t0(n), st = n & 1;
+                mbar_expect_tx(&ctl->bar_w[st], 2 * kPanelB);
+                tma_load_4d(sWd + (2 * st) * kPanelB, &mapWd, &ctl->bar_w[st], 0, h, t, b);
+                tma_load_4d(sWd + (2 * st + 1) * kPanelB, &mapWd, &ctl->bar_w[st], 64, h, t, b);
+            };
+            auto store_out = [&](int n) {
+                const int t = chunk_t0(n);
+                const unsigned char* sOut = sWd + 2 * (n & 1) * kPanelB;
+                tma_store_5d(&mapO, sOut, 0, h, t, b, slice);
+                tma_store_5d(&mapO, sOut + kPanelB, 32, h, t, b, slice);
+                bulk_commit();
+            };
+            prefetch_tmap(&mapQ); prefetch_tmap(&mapK); prefetch_tmap(&mapWd); prefetch_tmap(&mapO);
+            load_x(0);
+            load_w(0);
+            if (nchunks > 1) {
+                load_x(1);
+                load_w(1);
+            }
+            for (int n = 0; n < nchunks && !ctl->abort; ++n) {
+                // the d-sized tiles of chunk n are consumed once its state products are done: their
+                // buffer takes the tiles of chunk n+2
+                LEAN_WAIT(&ctl->bar_free1[n & 1], (n >> 1) & 1);
+                if (n + 2 < nchunks) load_x(n + 2);
+                // the weights are consumed once the intra-chunk product is done; the compute threads then
+                // stage the output rows in their place, and when those have left the buffer takes the
+                // weights of chunk n+2
+                LEAN_WAIT(&ctl->bar_out[n & 1], (n >> 1) & 1);
+                if (ctl->abort) break;
+                store_out(n);
+                bulk_wait_read();
+                if (n + 2 < nchunks) load_w(n + 2);
+            }
         }
     } else if (warp == kMmaWarp) {
         if (elect_one()) {
-        // =============================== MMA lane
-        constexpr uint32_t idescP = make_idesc(128, 128, false, false);    // xq xk^T
-        constexpr uint32_t idescO = make_idesc(128, 2 * kM, false, true);  // xq x state copy [S_hi | S_lo] (MN-major B)
-        constexpr uint32_t idescU = make_idesc(128, 2 * kM, true, true);   // xk^T (MN-major A) x [W_hi | W_lo]
-        constexpr uint32_t idescI = make_idesc(128, 2 * kM, false, true);  // masked P (tensor memory) x [W_hi | W_lo]
-        const uint64_t dS = desc_mnmajor(smem_u32(sSb), 0, kPanelB);
-        auto kmaj = [](int kk) { return (uint32_t)((kk >> 2) * kPanelB + (kk & 3) * 32); };
-        auto mnmaj = [](int kk) { return (uint32_t)(kk * 2048); };
-        auto issue_p = [&](int n) {
-            const uint32_t xq = smem_u32(sX + 4 * (n & 1) * kPanelB);
-            const uint64_t dQk = desc_kmajor(xq, 0), dKk = desc_kmajor(xq + 2 * kPanelB, 0);
+            // =============================== MMA lane
+            constexpr uint32_t idescP = make_idesc(128, 128, false, false);    // xq xk^T
+            constexpr uint32_t idescO = make_idesc(128, 2 * kM, false, true);  // xq x state copy [S_hi | S_lo] (MN-major B)
+            constexpr uint32_t idescU = make_idesc(128, 2 * kM, true, true);   // xk^T (MN-major A) x [W_hi | W_lo]
+            constexpr uint32_t idescI = make_idesc(128, 2 * kM, false, true);  // masked P (tensor memory) x [W_hi | W_lo]
+            const uint64_t dS = desc_mnmajor(smem_u32(sSb), 0, kPanelB);
+            auto kmaj = [](int kk) { return (uint32_t)((kk >> 2) * kPanelB + (kk & 3) * 32); };
+            auto mnmaj = [](int kk) { return (uint32_t)(kk * 2048); };
+            auto issue_p = [&](int n) {
+                const uint32_t xq = smem_u32(sX + 4 * (n & 1) * kPanelB);
+                const uint64_t dQk = desc_kmajor(xq, 0), dKk = desc_kmajor(xq + 2 * kPanelB, 0);
 #pragma unroll
-            for (int kk = 0; kk < kDST / 16; ++kk)
-                mma_bf16(tmem + kLvP, desc_advance(dQk, kmaj(kk)), desc_advance(dKk, kmaj(kk)), idescP, kk > 0);
-            mma_commit(&ctl->bar_p);
-        };
-        LEAN_WAIT(&ctl->bar_x2[0], 0);
-        tc_fence_after_sync();
-        issue_p(0);
-        PROF_DECL
-        for (int n = 0; n < nchunks && !ctl->abort; ++n) {
-            const int it = n;
-            (void)it;
-            const uint32_t xq = smem_u32(sX + 4 * (n & 1) * kPanelB);
-            const uint64_t dQk = desc_kmajor(xq, 0), dKm = desc_mnmajor(xq + 2 * kPanelB, 0, kPanelB);
-            const uint64_t dW = desc_mnmajor(smem_u32(sWd + 2 * (n & 1) * kPanelB), 0, kPanelB);
-            PROF_MARK();
-            // state products of chunk n: the state copy was written at the end of chunk n-1 (which also
-            // says that the accumulators they overwrite have been read)
-            LEAN_WAIT(&ctl->bar_w[n & 1], (n >> 1) & 1);
-            PROF_MARK();
-            LEAN_WAIT(&ctl->bar_sb, n & 1);
+                for (int kk = 0; kk < kDST / 16; ++kk)
+                    mma_bf16(tmem + kLvP, desc_advance(dQk, kmaj(kk)), desc_advance(dKk, kmaj(kk)), idescP, kk > 0);
+                mma_commit(&ctl->bar_p);
+            };
+            LEAN_WAIT(&ctl->bar_x2[0], 0);
             tc_fence_after_sync();
-            PROF_MARK();
-#pragma unroll
-            for (int kk = 0; kk < kCT / 16; ++kk)
-                mma_bf16(tmem + kLvU, desc_advance(dKm, mnmaj(kk)), desc_advance(dW, mnmaj(kk)), idescU, kk > 0);
-            // the inter-chunk output accumulator is single: the previous chunk's output rows must have
-            // been read out (by now they almost always are: this is issued after that chunk's intra
-            // product and the next first product)
-            if (n >= 1) {
-                LEAN_WAIT(&ctl->bar_out[(n - 1) & 1], ((n - 1) >> 1) & 1);
-                tc_fence_after_sync();
-            }
-#pragma unroll
-            for (int kk = 0; kk < kDST / 16; ++kk)
-                mma_bf16(tmem + kLvO, desc_advance(dQk, kmaj(kk)), desc_advance(dS, mnmaj(kk)), idescO, kk > 0);
-            mma_commit(&ctl->bar_mma1);
-            mma_commit(&ctl->bar_free1[n & 1]);
-            PROF_MARK();
-            // intra-chunk product once the masked P rows are there (bf16, in place in tensor memory)
-            LEAN_WAIT(&ctl->bar_pm, n & 1);
-            tc_fence_after_sync();
-            PROF_MARK();
-#pragma unroll
-            for (int kk = 0; kk < kCT / 16; ++kk)
-                mma_bf16_ta(tmem + kLvI, tmem + kLvP + 64 * (kk >> 2) + 8 * (kk & 3), desc_advance(dW, mnmaj(kk)), idescI,
-                            kk > 0);
-            if (PAIRS) {
-#pragma unroll
-                for (int kk = 0; kk < kCT / 16; ++kk)      // ... and the rounding residual of the masked P
-                    mma_bf16_ta(tmem + kLvI, tmem + kLvP + 64 * (kk >> 2) + 32 + 8 * (kk & 3),
-                                desc_advance(dW, mnmaj(kk)), idescI, true);
-            }
-            mma_commit(&ctl->bar_mma2);
-            PROF_MARK();
-            // the P accumulator is free: the next chunk's P queues right behind
-            if (n + 1 < nchunks) {
-                LEAN_WAIT(&ctl->bar_x2[(n + 1) & 1], ((n + 1) >> 1) & 1);
+            issue_p(0);
+            PROF_DECL
+            for (int n = 0; n < nchunks && !ctl->abort; ++n) {
+                const int it = n;
+                (void)it;
+                const uint32_t xq = smem_u32(sX + 4 * (n & 1) * kPanelB);
+                const uint64_t dQk = desc_kmajor(xq, 0), dKm = desc_mnmajor(xq + 2 * kPanelB, 0, kPanelB);
+                const uint64_t dW = desc_mnmajor(smem_u32(sWd + 2 * (n & 1) * kPanelB), 0, kPanelB);
+                PROF_MARK();
+                // state products of chunk n: the state copy was written at the end of chunk n-1 (which also
+                // says that the accumulators they overwrite have been read)
+                LEAN_WAIT(&ctl->bar_w[n & 1], (n >> 1) & 1);
+                PROF_MARK();
+                LEAN_WAIT(&ctl->bar_sb, n & 1);
                 tc_fence_after_sync();
                 PROF_MARK();
-                issue_p(n + 1);
+#pragma unroll
+                for (int kk = 0; kk < kCT / 16; ++kk)
+                    mma_bf16(tmem + kLvU, desc_advance(dKm, mnmaj(kk)), desc_advance(dW, mnmaj(kk)), idescU, kk > 0);
+                // the inter-chunk output accumulator is single: the previous chunk's output rows must have
+                // been read out (by now they almost always are: this is issued after that chunk's intra
+                // product and the next first product)
+                if (n >= 1) {
+                    LEAN_WAIT(&ctl->bar_out[(n - 1) & 1], ((n - 1) >> 1) & 1);
+                    tc_fence_after_sync();
+                }
+#pragma unroll
+                for (int kk = 0; kk < kDST / 16; ++kk)
+                    mma_bf16(tmem + kLvO, desc_advance(dQk, kmaj(kk)), desc_advance(dS, mnmaj(kk)), idescO, kk > 0);
+                mma_commit(&ctl->bar_mma1);
+                mma_commit(&ctl->bar_free1[n & 1]);
+                PROF_MARK();
+                // intra-chunk product once the masked P rows are there (bf16, in place in tensor memory)
+                LEAN_WAIT(&ctl->bar_pm, n & 1);
+                tc_fence_after_sync();
+                PROF_MARK();
+#pragma unroll
+                for (int kk = 0; kk < kCT / 16; ++kk)
+                    mma_bf16_ta(tmem + kLvI, tmem + kLvP + 64 * (kk >> 2) + 8 * (kk & 3), desc_advance(dW, mnmaj(kk)), idescI,
+                                kk > 0);
+                if (PAIRS) {
+#pragma unroll
+                    for (int kk = 0; kk < kCT / 16; ++kk)      // ... and the rounding residual of the masked P
+                        mma_bf16_ta(tmem + kLvI, tmem + kLvP + 64 * (kk >> 2) + 32 + 8 * (kk & 3),
+                                    desc_advance(dW, mnmaj(kk)), idescI, true);
+                }
+                mma_commit(&ctl->bar_mma2);
+                PROF_MARK();
+                // the P accumulator is free: the next chunk's P queues right behind
+                if (n + 1 < nchunks) {
+                    LEAN_WAIT(&ctl->bar_x2[(n + 1) & 1], ((n + 1) >> 1) & 1);
+                    tc_fence_after_sync();
+                    PROF_MARK();
+                    issue_p(n + 1);
+                }
+                PROF_MARK();
+                PROF_DUMP("value_side lean mma");
             }
-            PROF_MARK();
-            PROF_DUMP("value_side lean mma");
-        }
         }
     } else if (tid < kComputeThreads) {
         // =============================== compute threads
@@ -402,144 +402,144 @@ key_side_lean_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_cons
 
     if (warp == kCopyWarp) {
         if (elect_one()) {
-        // =============================== copy lane: every tile load and store
-        auto load_v = [&](int n) {
-            const int t = chunk_t0(n), st = n & 1;
-            mbar_expect_tx(&ctl->bar_x2[st], 2 * kPanelB);
-            tma_load_4d(sXv + (2 * st) * kPanelB, &mapV, &ctl->bar_x2[st], d0, h, t, b);
-            tma_load_4d(sXv + (2 * st + 1) * kPanelB, &mapV, &ctl->bar_x2[st], d0 + 64, h, t, b);
-        };
-        auto load_qk = [&](int n) {
-            const int t = chunk_t0(n), st = n & 1;
-            mbar_expect_tx(&ctl->bar_w[st], 4 * kPanelB);
-            tma_load_4d(sQK + (4 * st) * kPanelB, &mapUq, &ctl->bar_w[st], 0, h, t, b);
-            tma_load_4d(sQK + (4 * st + 1) * kPanelB, &mapUk, &ctl->bar_w[st], 0, h, t, b);
-            tma_load_4d(sQK + (4 * st + 2) * kPanelB, &mapUq, &ctl->bar_w[st], 64, h, t, b);
-            tma_load_4d(sQK + (4 * st + 3) * kPanelB, &mapUk, &ctl->bar_w[st], 64, h, t, b);
-        };
-        auto store_out = [&](int n) {
-            const int t = chunk_t0(n);
-            const unsigned char* sOut = sXv + 2 * (n & 1) * kPanelB;
-            tma_store_4d(&mapO, sOut, d0, h, t, b);
-            if (d0 + 64 < a.D) tma_store_4d(&mapO, sOut + kPanelB, d0 + 64, h, t, b);
-            bulk_commit();
-        };
-        prefetch_tmap(&mapV); prefetch_tmap(&mapUq); prefetch_tmap(&mapUk); prefetch_tmap(&mapO);
-        load_qk(0);
-        load_v(0);
-        if (nchunks > 1) {
-            load_qk(1);
-            load_v(1);
-        }
-        for (int n = 0; n < nchunks && !ctl->abort; ++n) {
-            // the decayed uq / uk rows of chunk n are consumed once its state products are done: their
-            // buffer takes the rows of chunk n+2
-            LEAN_WAIT(&ctl->bar_free1[n & 1], (n >> 1) & 1);
-            if (n + 2 < nchunks) load_qk(n + 2);
-            // the xv tile is consumed once the intra-chunk product is done; the compute threads then
-            // stage the output rows in its place, and when those have left the buffer takes the tile
-            // of chunk n+2
-            LEAN_WAIT(&ctl->bar_out[n & 1], (n >> 1) & 1);
-            if (ctl->abort) break;
-            store_out(n);
-            bulk_wait_read();
-            if (n + 2 < nchunks) load_v(n + 2);
-        }
+            // =============================== copy lane: every tile load and store
+            auto load_v = [&](int n) {
+                const int t = chunk_t0(n), st = n & 1;
+                mbar_expect_tx(&ctl->bar_x2[st], 2 * kPanelB);
+                tma_load_4d(sXv + (2 * st) * kPanelB, &mapV, &ctl->bar_x2[st], d0, h, t, b);
+                tma_load_4d(sXv + (2 * st + 1) * kPanelB, &mapV, &ctl->bar_x2[st], d0 + 64, h, t, b);
+            };
+            auto load_qk = [&](int n) {
+                const int t = chunk_t0(n), st = n & 1;
+                mbar_expect_tx(&ctl->bar_w[st], 4 * kPanelB);
+                tma_load_4d(sQK + (4 * st) * kPanelB, &mapUq, &ctl->bar_w[st], 0, h, t, b);
+                tma_load_4d(sQK + (4 * st + 1) * kPanelB, &mapUk, &ctl->bar_w[st], 0, h, t, b);
+                tma_load_4d(sQK + (4 * st + 2) * kPanelB, &mapUq, &ctl->bar_w[st], 64, h, t, b);
+                tma_load_4d(sQK + (4 * st + 3) * kPanelB, &mapUk, &ctl->bar_w[st], 64, h, t, b);
+            };
+            auto store_out = [&](int n) {
+                const int t = chunk_t0(n);
+                const unsigned char* sOut = sXv + 2 * (n & 1) * kPanelB;
+                tma_store_4d(&mapO, sOut, d0, h, t, b);
+                if (d0 + 64 < a.D) tma_store_4d(&mapO, sOut + kPanelB, d0 + 64, h, t, b);
+                bulk_commit();
+            };
+            prefetch_tmap(&mapV); prefetch_tmap(&mapUq); prefetch_tmap(&mapUk); prefetch_tmap(&mapO);
+            load_qk(0);
+            load_v(0);
+            if (nchunks > 1) {
+                load_qk(1);
+                load_v(1);
+            }
+            for (int n = 0; n < nchunks && !ctl->abort; ++n) {
+                // the decayed uq / uk rows of chunk n are consumed once its state products are done: their
+                // buffer takes the rows of chunk n+2
+                LEAN_WAIT(&ctl->bar_free1[n & 1], (n >> 1) & 1);
+                if (n + 2 < nchunks) load_qk(n + 2);
+                // the xv tile is consumed once the intra-chunk product is done; the compute threads then
+                // stage the output rows in its place, and when those have left the buffer takes the tile
+                // of chunk n+2
+                LEAN_WAIT(&ctl->bar_out[n & 1], (n >> 1) & 1);
+                if (ctl->abort) break;
+                store_out(n);
+                bulk_wait_read();
+                if (n + 2 < nchunks) load_v(n + 2);
+            }
         }
     } else if (warp == kMmaWarp) {
         if (elect_one()) {
-        // =============================== MMA lane
-        constexpr uint32_t idescA = make_idesc(128, 128, false, false);   // Q~ K~^T
-        constexpr uint32_t idescO = make_idesc(128, kDST, false, false);  // Q~ x state copy (K-major B)
-        constexpr uint32_t idescU = make_idesc(128, 2 * kM, true, true);  // xv^T (MN-major A) x [K~_hi | K~_lo] (MN-major B)
-        constexpr uint32_t idescV = make_idesc(128, kDST, false, true);   // A x xv (MN-major B)
-        const uint64_t dS = desc_kmajor(smem_u32(sSb), 0), dSl = desc_kmajor(smem_u32(sSb + kPanelB), 0);
-        auto kmaj = [](int kk) { return (uint32_t)((kk >> 2) * kPanelB + (kk & 3) * 32); };
-        auto mnmaj = [](int kk) { return (uint32_t)(kk * 2048); };
-        auto issue_a = [&](int n) {
-            // A = Q~ K~^T with both factors as bf16 high/low pairs (the low x low term is dropped)
-            const uint32_t qk = smem_u32(sQK + 4 * (n & 1) * kPanelB);
-            const uint64_t dQt = desc_kmajor(qk, 0), dKt = desc_kmajor(qk + kPanelB, 0);
-            const uint64_t dQl = desc_kmajor(qk + 2 * kPanelB, 0), dKl = desc_kmajor(qk + 3 * kPanelB, 0);
-#pragma unroll
-            for (int kk = 0; kk < kM / 16; ++kk)
-                mma_bf16(tmem + kLkA, desc_advance(dQt, kmaj(kk)), desc_advance(dKt, kmaj(kk)), idescA, kk > 0);
-            if (PAIRS) {
+            // =============================== MMA lane
+            constexpr uint32_t idescA = make_idesc(128, 128, false, false);   // Q~ K~^T
+            constexpr uint32_t idescO = make_idesc(128, kDST, false, false);  // Q~ x state copy (K-major B)
+            constexpr uint32_t idescU = make_idesc(128, 2 * kM, true, true);  // xv^T (MN-major A) x [K~_hi | K~_lo] (MN-major B)
+            constexpr uint32_t idescV = make_idesc(128, kDST, false, true);   // A x xv (MN-major B)
+            const uint64_t dS = desc_kmajor(smem_u32(sSb), 0), dSl = desc_kmajor(smem_u32(sSb + kPanelB), 0);
+            auto kmaj = [](int kk) { return (uint32_t)((kk >> 2) * kPanelB + (kk & 3) * 32); };
+            auto mnmaj = [](int kk) { return (uint32_t)(kk * 2048); };
+            auto issue_a = [&](int n) {
+                // A = Q~ K~^T with both factors as bf16 high/low pairs (the low x low term is dropped)
+                const uint32_t qk = smem_u32(sQK + 4 * (n & 1) * kPanelB);
+                const uint64_t dQt = desc_kmajor(qk, 0), dKt = desc_kmajor(qk + kPanelB, 0);
+                const uint64_t dQl = desc_kmajor(qk + 2 * kPanelB, 0), dKl = desc_kmajor(qk + 3 * kPanelB, 0);
 #pragma unroll
                 for (int kk = 0; kk < kM / 16; ++kk)
-                    mma_bf16(tmem + kLkA, desc_advance(dQl, kmaj(kk)), desc_advance(dKt, kmaj(kk)), idescA, true);
+                    mma_bf16(tmem + kLkA, desc_advance(dQt, kmaj(kk)), desc_advance(dKt, kmaj(kk)), idescA, kk > 0);
+                if (PAIRS) {
 #pragma unroll
-                for (int kk = 0; kk < kM / 16; ++kk)
-                    mma_bf16(tmem + kLkA, desc_advance(dQt, kmaj(kk)), desc_advance(dKl, kmaj(kk)), idescA, true);
-            }
-            mma_commit(&ctl->bar_p);
-        };
-        LEAN_WAIT(&ctl->bar_w[0], 0);
-        tc_fence_after_sync();
-        issue_a(0);
-        PROF_DECL
-        for (int n = 0; n < nchunks && !ctl->abort; ++n) {
-            const int it = n;
-            (void)it;
-            const uint64_t dV = desc_mnmajor(smem_u32(sXv + 2 * (n & 1) * kPanelB), 0, kPanelB);
-            const uint32_t accO = tmem + kLkO + 128 * (n & 1);
-            const uint32_t qk = smem_u32(sQK + 4 * (n & 1) * kPanelB);
-            const uint64_t dQt = desc_kmajor(qk, 0), dQl = desc_kmajor(qk + 2 * kPanelB, 0);
-            // the decayed uk read MN-major, its high and low parts as one N = 128 operand (the panels
-            // of a stage are [uq_hi, uk_hi, uq_lo, uk_lo]: the low part is two panels on)
-            const uint64_t dKtm = desc_mnmajor(qk + kPanelB, 0, 2 * kPanelB);
-            PROF_MARK();
-            // state products of chunk n: the state copy was written at the end of chunk n-1 (which also
-            // says that the accumulators they overwrite have been read)
-            LEAN_WAIT(&ctl->bar_x2[n & 1], (n >> 1) & 1);
-            PROF_MARK();
-            LEAN_WAIT(&ctl->bar_sb, n & 1);
+                    for (int kk = 0; kk < kM / 16; ++kk)
+                        mma_bf16(tmem + kLkA, desc_advance(dQl, kmaj(kk)), desc_advance(dKt, kmaj(kk)), idescA, true);
+#pragma unroll
+                    for (int kk = 0; kk < kM / 16; ++kk)
+                        mma_bf16(tmem + kLkA, desc_advance(dQt, kmaj(kk)), desc_advance(dKl, kmaj(kk)), idescA, true);
+                }
+                mma_commit(&ctl->bar_p);
+            };
+            LEAN_WAIT(&ctl->bar_w[0], 0);
             tc_fence_after_sync();
-            PROF_MARK();
-#pragma unroll
-            for (int kk = 0; kk < kCT / 16; ++kk)
-                mma_bf16(tmem + kLkU, desc_advance(dV, mnmaj(kk)), desc_advance(dKtm, mnmaj(kk)), idescU, kk > 0);
-            // inter-chunk product with both factors as bf16 high/low pairs (low x low dropped)
-#pragma unroll
-            for (int kk = 0; kk < kM / 16; ++kk)
-                mma_bf16(accO, desc_advance(dQt, kmaj(kk)), desc_advance(dS, kmaj(kk)), idescO, kk > 0);
-            if (PAIRS) {
-#pragma unroll
-                for (int kk = 0; kk < kM / 16; ++kk)
-                    mma_bf16(accO, desc_advance(dQl, kmaj(kk)), desc_advance(dS, kmaj(kk)), idescO, true);
-#pragma unroll
-                for (int kk = 0; kk < kM / 16; ++kk)
-                    mma_bf16(accO, desc_advance(dQt, kmaj(kk)), desc_advance(dSl, kmaj(kk)), idescO, true);
-            }
-            mma_commit(&ctl->bar_mma1);
-            mma_commit(&ctl->bar_free1[n & 1]);
-            PROF_MARK();
-            // intra-chunk product (masked A and its rounding residual) on top of the inter-chunk one
-            LEAN_WAIT(&ctl->bar_pm, n & 1);
-            tc_fence_after_sync();
-            PROF_MARK();
-            // (the masked A and its rounding residual are bf16 rows in tensor memory, in place of A)
-#pragma unroll
-            for (int kk = 0; kk < kCT / 16; ++kk)
-                mma_bf16_ta(accO, tmem + kLkA + 64 * (kk >> 2) + 8 * (kk & 3), desc_advance(dV, mnmaj(kk)), idescV, true);
-            if (PAIRS) {
-#pragma unroll
-                for (int kk = 0; kk < kCT / 16; ++kk)
-                    mma_bf16_ta(accO, tmem + kLkA + 64 * (kk >> 2) + 32 + 8 * (kk & 3), desc_advance(dV, mnmaj(kk)),
-                                idescV, true);
-            }
-            mma_commit(&ctl->bar_mma2);
-            PROF_MARK();
-            // the A accumulator is free: the next chunk's A queues right behind
-            if (n + 1 < nchunks) {
-                LEAN_WAIT(&ctl->bar_w[(n + 1) & 1], ((n + 1) >> 1) & 1);
+            issue_a(0);
+            PROF_DECL
+            for (int n = 0; n < nchunks && !ctl->abort; ++n) {
+                const int it = n;
+                (void)it;
+                const uint64_t dV = desc_mnmajor(smem_u32(sXv + 2 * (n & 1) * kPanelB), 0, kPanelB);
+                const uint32_t accO = tmem + kLkO + 128 * (n & 1);
+                const uint32_t qk = smem_u32(sQK + 4 * (n & 1) * kPanelB);
+                const uint64_t dQt = desc_kmajor(qk, 0), dQl = desc_kmajor(qk + 2 * kPanelB, 0);
+                // the decayed uk read MN-major, its high and low parts as one N = 128 operand (the panels
+                // of a stage are [uq_hi, uk_hi, uq_lo, uk_lo]: the low part is two panels on)
+                const uint64_t dKtm = desc_mnmajor(qk + kPanelB, 0, 2 * kPanelB);
+                PROF_MARK();
+                // state products of chunk n: the state copy was written at the end of chunk n-1 (which also
+                // says that the accumulators they overwrite have been read)
+                LEAN_WAIT(&ctl->bar_x2[n & 1], (n >> 1) & 1);
+                PROF_MARK();
+                LEAN_WAIT(&ctl->bar_sb, n & 1);
                 tc_fence_after_sync();
                 PROF_MARK();
-                issue_a(n + 1);
+#pragma unroll
+                for (int kk = 0; kk < kCT / 16; ++kk)
+                    mma_bf16(tmem + kLkU, desc_advance(dV, mnmaj(kk)), desc_advance(dKtm, mnmaj(kk)), idescU, kk > 0);
+                // inter-chunk product with both factors as bf16 high/low pairs (low x low dropped)
+#pragma unroll
+                for (int kk = 0; kk < kM / 16; ++kk)
+                    mma_bf16(accO, desc_advance(dQt, kmaj(kk)), desc_advance(dS, kmaj(kk)), idescO, kk > 0);
+                if (PAIRS) {
+#pragma unroll
+                    for (int kk = 0; kk < kM / 16; ++kk)
+                        mma_bf16(accO, desc_advance(dQl, kmaj(kk)), desc_advance(dS, kmaj(kk)), idescO, true);
+#pragma unroll
+                    for (int kk = 0; kk < kM / 16; ++kk)
+                        mma_bf16(accO, desc_advance(dQt, kmaj(kk)), desc_advance(dSl, kmaj(kk)), idescO, true);
+                }
+                mma_commit(&ctl->bar_mma1);
+                mma_commit(&ctl->bar_free1[n & 1]);
+                PROF_MARK();
+                // intra-chunk product (masked A and its rounding residual) on top of the inter-chunk one
+                LEAN_WAIT(&ctl->bar_pm, n & 1);
+                tc_fence_after_sync();
+                PROF_MARK();
+                // (the masked A and its rounding residual are bf16 rows in tensor memory, in place of A)
+#pragma unroll
+                for (int kk = 0; kk < kCT / 16; ++kk)
+                    mma_bf16_ta(accO, tmem + kLkA + 64 * (kk >> 2) + 8 * (kk & 3), desc_advance(dV, mnmaj(kk)), idescV, true);
+                if (PAIRS) {
+#pragma unroll
+                    for (int kk = 0; kk < kCT / 16; ++kk)
+                        mma_bf16_ta(accO, tmem + kLkA + 64 * (kk >> 2) + 32 + 8 * (kk & 3), desc_advance(dV, mnmaj(kk)),
+                                    idescV, true);
+                }
+                mma_commit(&ctl->bar_mma2);
+                PROF_MARK();
+                // the A accumulator is free: the next chunk's A queues right behind
+                if (n + 1 < nchunks) {
+                    LEAN_WAIT(&ctl->bar_w[(n + 1) & 1], ((n + 1) >> 1) & 1);
+                    tc_fence_after_sync();
+                    PROF_MARK();
+                    issue_a(n + 1);
+                }
+                PROF_MARK();
+                PROF_DUMP("key_side lean mma");
             }
-            PROF_MARK();
-            PROF_DUMP("key_side lean mma");
-        }
         }
     } else if (tid < kComputeThreads) {
         // =============================== compute threads
@@ -686,44 +686,44 @@ state_scan_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
 
     if (warp == kCopyWarp) {
         if (elect_one()) {
-        // =============================== copy lane
-        auto load = [&](int n) {
-            const int t = chunk_t0(n), st = n % kScanStages;
-            unsigned char* sX = smem + 4 * st * kPanelB;
-            mbar_expect_tx(&ctl->bar_x[st], 4 * kPanelB);
-            tma_load_4d(sX, &mapX, &ctl->bar_x[st], d0, h, t, b);
-            tma_load_4d(sX + kPanelB, &mapX, &ctl->bar_x[st], d0 + 64, h, t, b);
-            tma_load_4d(sX + 2 * kPanelB, &mapW, &ctl->bar_x[st], 0, h, t, b);
-            tma_load_4d(sX + 3 * kPanelB, &mapW, &ctl->bar_x[st], 64, h, t, b);
-        };
-        prefetch_tmap(&mapX); prefetch_tmap(&mapW);
-        for (int n = 0; n < kScanStages && n < nchunks; ++n) load(n);
-        for (int n = 0; n + kScanStages < nchunks && !ctl->abort; ++n) {
-            LEAN_WAIT(&ctl->bar_free[n % kScanStages], (n / kScanStages) & 1);
-            if (ctl->abort) break;
-            load(n + kScanStages);
-        }
+            // =============================== copy lane
+            auto load = [&](int n) {
+                const int t = chunk_t0(n), st = n % kScanStages;
+                unsigned char* sX = smem + 4 * st * kPanelB;
+                mbar_expect_tx(&ctl->bar_x[st], 4 * kPanelB);
+                tma_load_4d(sX, &mapX, &ctl->bar_x[st], d0, h, t, b);
+                tma_load_4d(sX + kPanelB, &mapX, &ctl->bar_x[st], d0 + 64, h, t, b);
+                tma_load_4d(sX + 2 * kPanelB, &mapW, &ctl->bar_x[st], 0, h, t, b);
+                tma_load_4d(sX + 3 * kPanelB, &mapW, &ctl->bar_x[st], 64, h, t, b);
+            };
+            prefetch_tmap(&mapX); prefetch_tmap(&mapW);
+            for (int n = 0; n < kScanStages && n < nchunks; ++n) load(n);
+            for (int n = 0; n + kScanStages < nchunks && !ctl->abort; ++n) {
+                LEAN_WAIT(&ctl->bar_free[n % kScanStages], (n / kScanStages) & 1);
+                if (ctl->abort) break;
+                load(n + kScanStages);
+            }
         }
     } else if (warp == kMmaWarp) {
         if (elect_one()) {
-        // =============================== MMA lane
-        constexpr uint32_t idescU = make_idesc(128, 2 * kM, true, true);   // X^T (MN-major A) x [W_hi | W_lo] (MN-major B)
-        auto mnmaj = [](int kk) { return (uint32_t)(kk * 2048); };
-        for (int n = 0; n < nchunks && !ctl->abort; ++n) {
-            const int st = n % kScanStages;
-            const uint32_t sX = smem_u32(smem + 4 * st * kPanelB);
-            const uint64_t dX = desc_mnmajor(sX, 0, kPanelB), dW = desc_mnmajor(sX + 2 * kPanelB, 0, kPanelB);
-            LEAN_WAIT(&ctl->bar_x[st], (n / kScanStages) & 1);
-            // the accumulator of chunk n-2 must have been read out
-            if (n >= 2) LEAN_WAIT(&ctl->bar_acc[n & 1], ((n - 2) >> 1) & 1);
-            if (ctl->abort) break;
-            tc_fence_after_sync();
+            // =============================== MMA lane
+            constexpr uint32_t idescU = make_idesc(128, 2 * kM, true, true);   // X^T (MN-major A) x [W_hi | W_lo] (MN-major B)
+            auto mnmaj = [](int kk) { return (uint32_t)(kk * 2048); };
+            for (int n = 0; n < nchunks && !ctl->abort; ++n) {
+                const int st = n % kScanStages;
+                const uint32_t sX = smem_u32(smem + 4 * st * kPanelB);
+                const uint64_t dX = desc_mnmajor(sX, 0, kPanelB), dW = desc_mnmajor(sX + 2 * kPanelB, 0, kPanelB);
+                LEAN_WAIT(&ctl->bar_x[st], (n / kScanStages) & 1);
+                // the accumulator of chunk n-2 must have been read out
+                if (n >= 2) LEAN_WAIT(&ctl->bar_acc[n & 1], ((n - 2) >> 1) & 1);
+                if (ctl->abort) break;
+                tc_fence_after_sync();
 #pragma unroll
-            for (int kk = 0; kk < kCT / 16; ++kk)
-                mma_bf16(tmem + 128 * (n & 1), desc_advance(dX, mnmaj(kk)), desc_advance(dW, mnmaj(kk)), idescU, kk > 0);
-            mma_commit(&ctl->bar_u[n & 1]);
-            mma_commit(&ctl->bar_free[st]);
-        }
+                for (int kk = 0; kk < kCT / 16; ++kk)
+                    mma_bf16(tmem + 128 * (n & 1), desc_advance(dX, mnmaj(kk)), desc_advance(dW, mnmaj(kk)), idescU, kk > 0);
+                mma_commit(&ctl->bar_u[n & 1]);
+                mma_commit(&ctl->bar_free[st]);
+            }
         }
     } else if (tid < kComputeThreads) {
         // =============================== compute threads: S[c = row][s], slots sb .. sb+31

@@ -111,212 +111,212 @@ rev_pair_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant_
 
     if (warp == kCopyWarp) {
         if (elect_one()) {
-        // =============================== copy lane: every tile load and store
-        auto load_x = [&](int n) {
-            const int t = chunk_t0(n), st = n & 1;
-            mbar_expect_tx(&ctl->bar_x[st], 2 * kPanelB);
-            tma_load_4d(sX + (2 * st) * kPanelB, &mapX, &ctl->bar_x[st], d0, h, t, b);
-            tma_load_4d(sX + (2 * st + 1) * kPanelB, &mapX, &ctl->bar_x[st], d0 + 64, h, t, b);
-        };
-        auto load_w = [&](int n) {
-            const int t = chunk_t0(n), st = n & 1;
-            mbar_expect_tx(&ctl->bar_w[st], 2 * kPanelB);
-            tma_load_4d(sW + (2 * st) * kPanelB, &mapW, &ctl->bar_w[st], 0, h, t, b);
-            tma_load_4d(sW + (2 * st + 1) * kPanelB, &mapW, &ctl->bar_w[st], 64, h, t, b);
-        };
-        auto load_yq = [&](int n) {
-            const int t = chunk_t0(n);
-            mbar_expect_tx(&ctl->bar_yq, 4 * kPanelB);
-            tma_load_4d(sY, &mapY, &ctl->bar_yq, d0, h, t, b);
-            tma_load_4d(sY + kPanelB, &mapY, &ctl->bar_yq, d0 + 64, h, t, b);
-            tma_load_4d(sQ, &mapQ, &ctl->bar_yq, 0, h, t, b);
-            tma_load_4d(sQ + kPanelB, &mapQ, &ctl->bar_yq, 64, h, t, b);
-        };
-        prefetch_tmap(&mapX); prefetch_tmap(&mapY); prefetch_tmap(&mapW); prefetch_tmap(&mapQ);
-        prefetch_tmap(&mapOv); prefetch_tmap(&mapOk);
-        load_x(0);
-        load_yq(0);
-        load_w(0);
-        if (nchunks > 1) {
-            load_x(1);
-            load_w(1);
-        }
-        for (int n = 0; n < nchunks && !ctl->abort; ++n) {
-            const int t = chunk_t0(n), st = n & 1;
-            // Y and Q are consumed once the inter-chunk products of chunk n are done; their next tiles are
-            // asked into L2 ahead of that, so that the copy itself is short
-            if (n + 1 < nchunks) {
-                const int tn = chunk_t0(n + 1);
-                tma_prefetch_4d(&mapY, d0, h, tn, b);
-                if (d0 + 64 < D) tma_prefetch_4d(&mapY, d0 + 64, h, tn, b);
-                tma_prefetch_4d(&mapQ, 0, h, tn, b);
-                tma_prefetch_4d(&mapQ, 64, h, tn, b);
+            // =============================== copy lane: every tile load and store
+            auto load_x = [&](int n) {
+                const int t = chunk_t0(n), st = n & 1;
+                mbar_expect_tx(&ctl->bar_x[st], 2 * kPanelB);
+                tma_load_4d(sX + (2 * st) * kPanelB, &mapX, &ctl->bar_x[st], d0, h, t, b);
+                tma_load_4d(sX + (2 * st + 1) * kPanelB, &mapX, &ctl->bar_x[st], d0 + 64, h, t, b);
+            };
+            auto load_w = [&](int n) {
+                const int t = chunk_t0(n), st = n & 1;
+                mbar_expect_tx(&ctl->bar_w[st], 2 * kPanelB);
+                tma_load_4d(sW + (2 * st) * kPanelB, &mapW, &ctl->bar_w[st], 0, h, t, b);
+                tma_load_4d(sW + (2 * st + 1) * kPanelB, &mapW, &ctl->bar_w[st], 64, h, t, b);
+            };
+            auto load_yq = [&](int n) {
+                const int t = chunk_t0(n);
+                mbar_expect_tx(&ctl->bar_yq, 4 * kPanelB);
+                tma_load_4d(sY, &mapY, &ctl->bar_yq, d0, h, t, b);
+                tma_load_4d(sY + kPanelB, &mapY, &ctl->bar_yq, d0 + 64, h, t, b);
+                tma_load_4d(sQ, &mapQ, &ctl->bar_yq, 0, h, t, b);
+                tma_load_4d(sQ + kPanelB, &mapQ, &ctl->bar_yq, 64, h, t, b);
+            };
+            prefetch_tmap(&mapX); prefetch_tmap(&mapY); prefetch_tmap(&mapW); prefetch_tmap(&mapQ);
+            prefetch_tmap(&mapOv); prefetch_tmap(&mapOk);
+            load_x(0);
+            load_yq(0);
+            load_w(0);
+            if (nchunks > 1) {
+                load_x(1);
+                load_w(1);
             }
-            PAIR_WAIT(&ctl->bar_yqfree, n & 1);
-            if (ctl->abort) break;
-            if (n + 1 < nchunks) load_yq(n + 1);
-            // W is consumed once the value-side output is complete; the compute threads then stage that
-            // output in its place (a tiled store from shared memory costs less than the compute threads'
-            // own stores to global memory: those were measured at 140 us a launch against 95).  Likewise X
-            // and the key-side output.  When both have left, the buffers take the tiles of chunk n+2.
-            PAIR_WAIT(&ctl->bar_outv[st], (n >> 1) & 1);
-            if (ctl->abort) break;
-            tma_store_5d(&mapOv, sW + (2 * st) * kPanelB, 0, h, t, b, slice);
-            tma_store_5d(&mapOv, sW + (2 * st + 1) * kPanelB, 32, h, t, b, slice);
-            bulk_commit();
-            PAIR_WAIT(&ctl->bar_outk[st], (n >> 1) & 1);
-            if (ctl->abort) break;
-            tma_store_4d(&mapOk, sX + (2 * st) * kPanelB, d0, h, t, b);
-            if (d0 + 64 < D) tma_store_4d(&mapOk, sX + (2 * st + 1) * kPanelB, d0 + 64, h, t, b);
-            bulk_commit();
-            bulk_wait_read();
-            if (n + 2 < nchunks) {
-                load_x(n + 2);
-                load_w(n + 2);
+            for (int n = 0; n < nchunks && !ctl->abort; ++n) {
+                const int t = chunk_t0(n), st = n & 1;
+                // Y and Q are consumed once the inter-chunk products of chunk n are done; their next tiles are
+                // asked into L2 ahead of that, so that the copy itself is short
+                if (n + 1 < nchunks) {
+                    const int tn = chunk_t0(n + 1);
+                    tma_prefetch_4d(&mapY, d0, h, tn, b);
+                    if (d0 + 64 < D) tma_prefetch_4d(&mapY, d0 + 64, h, tn, b);
+                    tma_prefetch_4d(&mapQ, 0, h, tn, b);
+                    tma_prefetch_4d(&mapQ, 64, h, tn, b);
+                }
+                PAIR_WAIT(&ctl->bar_yqfree, n & 1);
+                if (ctl->abort) break;
+                if (n + 1 < nchunks) load_yq(n + 1);
+                // W is consumed once the value-side output is complete; the compute threads then stage that
+                // output in its place (a tiled store from shared memory costs less than the compute threads'
+                // own stores to global memory: those were measured at 140 us a launch against 95).  Likewise X
+                // and the key-side output.  When both have left, the buffers take the tiles of chunk n+2.
+                PAIR_WAIT(&ctl->bar_outv[st], (n >> 1) & 1);
+                if (ctl->abort) break;
+                tma_store_5d(&mapOv, sW + (2 * st) * kPanelB, 0, h, t, b, slice);
+                tma_store_5d(&mapOv, sW + (2 * st + 1) * kPanelB, 32, h, t, b, slice);
+                bulk_commit();
+                PAIR_WAIT(&ctl->bar_outk[st], (n >> 1) & 1);
+                if (ctl->abort) break;
+                tma_store_4d(&mapOk, sX + (2 * st) * kPanelB, d0, h, t, b);
+                if (d0 + 64 < D) tma_store_4d(&mapOk, sX + (2 * st + 1) * kPanelB, d0 + 64, h, t, b);
+                bulk_commit();
+                bulk_wait_read();
+                if (n + 2 < nchunks) {
+                    load_x(n + 2);
+                    load_w(n + 2);
+                }
             }
-        }
         }
     } else if (warp == kMmaWarp) {
         if (elect_one()) {
-        // =============================== MMA lane
-        constexpr uint32_t idescP = make_idesc(128, 128, false, false);    // Y X^T and Q W^T
-        constexpr uint32_t idescU = make_idesc(128, kM, true, true);       // X^T (MN-major A) x W part (MN-major B)
-        constexpr uint32_t idescYS = make_idesc(128, kM, false, true);     // Y x state-copy part (MN-major B); masked P x W part
-        constexpr uint32_t idescQS = make_idesc(128, kDST, false, false);  // Q x state copy (K-major B)
-        constexpr uint32_t idescAX = make_idesc(128, kDST, false, true);   // masked A x X (MN-major B)
-        auto kmaj = [](int kk) { return (uint32_t)((kk >> 2) * kPanelB + (kk & 3) * 32); };
-        auto mnmaj = [](int kk) { return (uint32_t)(kk * 2048); };
-        const uint64_t dYk = desc_kmajor(smem_u32(sY), 0);
-        const uint64_t dQh = desc_kmajor(smem_u32(sQ), 0), dQl = desc_kmajor(smem_u32(sQ + kPanelB), 0);
-        const uint64_t dSh = desc_mnmajor(smem_u32(sSb), 0, kPanelB), dSl = desc_mnmajor(smem_u32(sSb + kPanelB), 0, kPanelB);
-        const uint64_t dSkh = desc_kmajor(smem_u32(sSb), 0), dSkl = desc_kmajor(smem_u32(sSb + kPanelB), 0);
-        auto issue_first = [&](int n) {
-            const uint32_t xs = smem_u32(sX + 2 * (n & 1) * kPanelB), ws = smem_u32(sW + 2 * (n & 1) * kPanelB);
-            const uint64_t dXk = desc_kmajor(xs, 0);
-            const uint64_t dWh = desc_kmajor(ws, 0), dWl = desc_kmajor(ws + kPanelB, 0);
-#pragma unroll
-            for (int kk = 0; kk < kDST / 16; ++kk)
-                mma_bf16(tmem + kPcP, desc_advance(dYk, kmaj(kk)), desc_advance(dXk, kmaj(kk)), idescP, kk > 0);
-            mma_commit(&ctl->bar_p);
-            // A = Q W^T with both factors as bf16 high/low pairs (the low x low term is dropped)
-#pragma unroll
-            for (int kk = 0; kk < kM / 16; ++kk)
-                mma_bf16(tmem + kPcA, desc_advance(dQh, kmaj(kk)), desc_advance(dWh, kmaj(kk)), idescP, kk > 0);
-            if (PAIRS) {
-#pragma unroll
-                for (int kk = 0; kk < kM / 16; ++kk)
-                    mma_bf16(tmem + kPcA, desc_advance(dQl, kmaj(kk)), desc_advance(dWh, kmaj(kk)), idescP, true);
-#pragma unroll
-                for (int kk = 0; kk < kM / 16; ++kk)
-                    mma_bf16(tmem + kPcA, desc_advance(dQh, kmaj(kk)), desc_advance(dWl, kmaj(kk)), idescP, true);
-            }
-            mma_commit(&ctl->bar_a);
-        };
-        PAIR_WAIT(&ctl->bar_x[0], 0);
-        PAIR_WAIT(&ctl->bar_yq, 0);
-        PAIR_WAIT(&ctl->bar_w[0], 0);
-        tc_fence_after_sync();
-        if (!ctl->abort) issue_first(0);
-        PROF_DECL
-        for (int n = 0; n < nchunks && !ctl->abort; ++n) {
-            const int it = n;
-            (void)it;
-            const uint32_t xs = smem_u32(sX + 2 * (n & 1) * kPanelB), ws = smem_u32(sW + 2 * (n & 1) * kPanelB);
-            const uint64_t dXm = desc_mnmajor(xs, 0, kPanelB);
-            const uint64_t dWh = desc_mnmajor(ws, 0, kPanelB), dWl = desc_mnmajor(ws + kPanelB, 0, kPanelB);
-            PROF_MARK();
-            // ---- inter-chunk products first (Y and Q, single-staged, are free for the next chunk's tiles behind
-            // them): the state copy was written in chunk n-1, whose rows have been read out of the accumulators
-            PAIR_WAIT(&ctl->bar_sb, n & 1);
-            if (n >= 1) PAIR_WAIT(&ctl->bar_outv[(n - 1) & 1], ((n - 1) >> 1) & 1);
-            tc_fence_after_sync();
-            PROF_MARK();
-#pragma unroll
-            for (int kk = 0; kk < kDST / 16; ++kk)
-                mma_bf16(tmem + kPcOI, desc_advance(dYk, kmaj(kk)), desc_advance(dSh, mnmaj(kk)), idescYS, kk > 0);
-            if (PAIRS) {
+            // =============================== MMA lane
+            constexpr uint32_t idescP = make_idesc(128, 128, false, false);    // Y X^T and Q W^T
+            constexpr uint32_t idescU = make_idesc(128, kM, true, true);       // X^T (MN-major A) x W part (MN-major B)
+            constexpr uint32_t idescYS = make_idesc(128, kM, false, true);     // Y x state-copy part (MN-major B); masked P x W part
+            constexpr uint32_t idescQS = make_idesc(128, kDST, false, false);  // Q x state copy (K-major B)
+            constexpr uint32_t idescAX = make_idesc(128, kDST, false, true);   // masked A x X (MN-major B)
+            auto kmaj = [](int kk) { return (uint32_t)((kk >> 2) * kPanelB + (kk & 3) * 32); };
+            auto mnmaj = [](int kk) { return (uint32_t)(kk * 2048); };
+            const uint64_t dYk = desc_kmajor(smem_u32(sY), 0);
+            const uint64_t dQh = desc_kmajor(smem_u32(sQ), 0), dQl = desc_kmajor(smem_u32(sQ + kPanelB), 0);
+            const uint64_t dSh = desc_mnmajor(smem_u32(sSb), 0, kPanelB), dSl = desc_mnmajor(smem_u32(sSb + kPanelB), 0, kPanelB);
+            const uint64_t dSkh = desc_kmajor(smem_u32(sSb), 0), dSkl = desc_kmajor(smem_u32(sSb + kPanelB), 0);
+            auto issue_first = [&](int n) {
+                const uint32_t xs = smem_u32(sX + 2 * (n & 1) * kPanelB), ws = smem_u32(sW + 2 * (n & 1) * kPanelB);
+                const uint64_t dXk = desc_kmajor(xs, 0);
+                const uint64_t dWh = desc_kmajor(ws, 0), dWl = desc_kmajor(ws + kPanelB, 0);
 #pragma unroll
                 for (int kk = 0; kk < kDST / 16; ++kk)
-                    mma_bf16(tmem + kPcOI, desc_advance(dYk, kmaj(kk)), desc_advance(dSl, mnmaj(kk)), idescYS, true);
-            }
-            PROF_MARK();
-            if (n >= 1) {
-                PAIR_WAIT(&ctl->bar_outk[(n - 1) & 1], ((n - 1) >> 1) & 1);
-                tc_fence_after_sync();
-            }
-            PROF_MARK();
-#pragma unroll
-            for (int kk = 0; kk < kM / 16; ++kk)
-                mma_bf16(tmem + kPcO2, desc_advance(dQh, kmaj(kk)), desc_advance(dSkh, kmaj(kk)), idescQS, kk > 0);
-            if (PAIRS) {
+                    mma_bf16(tmem + kPcP, desc_advance(dYk, kmaj(kk)), desc_advance(dXk, kmaj(kk)), idescP, kk > 0);
+                mma_commit(&ctl->bar_p);
+                // A = Q W^T with both factors as bf16 high/low pairs (the low x low term is dropped)
 #pragma unroll
                 for (int kk = 0; kk < kM / 16; ++kk)
-                    mma_bf16(tmem + kPcO2, desc_advance(dQl, kmaj(kk)), desc_advance(dSkh, kmaj(kk)), idescQS, true);
+                    mma_bf16(tmem + kPcA, desc_advance(dQh, kmaj(kk)), desc_advance(dWh, kmaj(kk)), idescP, kk > 0);
+                if (PAIRS) {
 #pragma unroll
-                for (int kk = 0; kk < kM / 16; ++kk)
-                    mma_bf16(tmem + kPcO2, desc_advance(dQh, kmaj(kk)), desc_advance(dSkl, kmaj(kk)), idescQS, true);
-            }
-            mma_commit(&ctl->bar_yqfree);
-            PROF_MARK();
-            // ---- state product U = X^T W (its accumulator was read in chunk n-1, before the state copy was written)
+                    for (int kk = 0; kk < kM / 16; ++kk)
+                        mma_bf16(tmem + kPcA, desc_advance(dQl, kmaj(kk)), desc_advance(dWh, kmaj(kk)), idescP, true);
 #pragma unroll
-            for (int kk = 0; kk < kCT / 16; ++kk)
-                mma_bf16(tmem + kPcU, desc_advance(dXm, mnmaj(kk)), desc_advance(dWh, mnmaj(kk)), idescU, kk > 0);
-            if (PAIRS) {
-#pragma unroll
-                for (int kk = 0; kk < kCT / 16; ++kk)
-                    mma_bf16(tmem + kPcU, desc_advance(dXm, mnmaj(kk)), desc_advance(dWl, mnmaj(kk)), idescU, true);
-            }
-            mma_commit(&ctl->bar_mma1);
-            PROF_MARK();
-            // ---- value-side intra-chunk product: masked P (bf16 pair, in place in tensor memory) x W
-            PAIR_WAIT(&ctl->bar_pm, n & 1);
+                    for (int kk = 0; kk < kM / 16; ++kk)
+                        mma_bf16(tmem + kPcA, desc_advance(dQh, kmaj(kk)), desc_advance(dWl, kmaj(kk)), idescP, true);
+                }
+                mma_commit(&ctl->bar_a);
+            };
+            PAIR_WAIT(&ctl->bar_x[0], 0);
+            PAIR_WAIT(&ctl->bar_yq, 0);
+            PAIR_WAIT(&ctl->bar_w[0], 0);
             tc_fence_after_sync();
-            PROF_MARK();
-#pragma unroll
-            for (int kk = 0; kk < kCT / 16; ++kk)
-                mma_bf16_ta(tmem + kPcOI, tmem + kPcP + 64 * (kk >> 2) + 8 * (kk & 3), desc_advance(dWh, mnmaj(kk)), idescYS,
-                            true);
-            if (PAIRS) {
-#pragma unroll
-                for (int kk = 0; kk < kCT / 16; ++kk)
-                    mma_bf16_ta(tmem + kPcOI, tmem + kPcP + 64 * (kk >> 2) + 8 * (kk & 3), desc_advance(dWl, mnmaj(kk)),
-                                idescYS, true);
-#pragma unroll
-                for (int kk = 0; kk < kCT / 16; ++kk)
-                    mma_bf16_ta(tmem + kPcOI, tmem + kPcP + 64 * (kk >> 2) + 32 + 8 * (kk & 3),
-                                desc_advance(dWh, mnmaj(kk)), idescYS, true);
-            }
-            mma_commit(&ctl->bar_v4);
-            PROF_MARK();
-            // ---- key-side intra-chunk product: masked A x X on top of the inter-chunk one
-            PAIR_WAIT(&ctl->bar_am, n & 1);
-            tc_fence_after_sync();
-            PROF_MARK();
-#pragma unroll
-            for (int kk = 0; kk < kCT / 16; ++kk)
-                mma_bf16_ta(tmem + kPcO2, tmem + kPcA + 64 * (kk >> 2) + 8 * (kk & 3), desc_advance(dXm, mnmaj(kk)), idescAX,
-                            true);
-            if (PAIRS) {
-#pragma unroll
-                for (int kk = 0; kk < kCT / 16; ++kk)
-                    mma_bf16_ta(tmem + kPcO2, tmem + kPcA + 64 * (kk >> 2) + 32 + 8 * (kk & 3),
-                                desc_advance(dXm, mnmaj(kk)), idescAX, true);
-            }
-            mma_commit(&ctl->bar_k4);
-            PROF_MARK();
-            // ---- both first-product accumulators are free behind these: the next chunk's queue up
-            if (n + 1 < nchunks) {
-                PAIR_WAIT(&ctl->bar_x[(n + 1) & 1], ((n + 1) >> 1) & 1);
-                PAIR_WAIT(&ctl->bar_yq, (n + 1) & 1);
-                PAIR_WAIT(&ctl->bar_w[(n + 1) & 1], ((n + 1) >> 1) & 1);
+            if (!ctl->abort) issue_first(0);
+            PROF_DECL
+            for (int n = 0; n < nchunks && !ctl->abort; ++n) {
+                const int it = n;
+                (void)it;
+                const uint32_t xs = smem_u32(sX + 2 * (n & 1) * kPanelB), ws = smem_u32(sW + 2 * (n & 1) * kPanelB);
+                const uint64_t dXm = desc_mnmajor(xs, 0, kPanelB);
+                const uint64_t dWh = desc_mnmajor(ws, 0, kPanelB), dWl = desc_mnmajor(ws + kPanelB, 0, kPanelB);
+                PROF_MARK();
+                // ---- inter-chunk products first (Y and Q, single-staged, are free for the next chunk's tiles behind
+                // them): the state copy was written in chunk n-1, whose rows have been read out of the accumulators
+                PAIR_WAIT(&ctl->bar_sb, n & 1);
+                if (n >= 1) PAIR_WAIT(&ctl->bar_outv[(n - 1) & 1], ((n - 1) >> 1) & 1);
                 tc_fence_after_sync();
                 PROF_MARK();
-                if (!ctl->abort) issue_first(n + 1);
+#pragma unroll
+                for (int kk = 0; kk < kDST / 16; ++kk)
+                    mma_bf16(tmem + kPcOI, desc_advance(dYk, kmaj(kk)), desc_advance(dSh, mnmaj(kk)), idescYS, kk > 0);
+                if (PAIRS) {
+#pragma unroll
+                    for (int kk = 0; kk < kDST / 16; ++kk)
+                        mma_bf16(tmem + kPcOI, desc_advance(dYk, kmaj(kk)), desc_advance(dSl, mnmaj(kk)), idescYS, true);
+                }
+                PROF_MARK();
+                if (n >= 1) {
+                    PAIR_WAIT(&ctl->bar_outk[(n - 1) & 1], ((n - 1) >> 1) & 1);
+                    tc_fence_after_sync();
+                }
+                PROF_MARK();
+#pragma unroll
+                for (int kk = 0; kk < kM / 16; ++kk)
+                    mma_bf16(tmem + kPcO2, desc_advance(dQh, kmaj(kk)), desc_advance(dSkh, kmaj(kk)), idescQS, kk > 0);
+                if (PAIRS) {
+#pragma unroll
+                    for (int kk = 0; kk < kM / 16; ++kk)
+                        mma_bf16(tmem + kPcO2, desc_advance(dQl, kmaj(kk)), desc_advance(dSkh, kmaj(kk)), idescQS, true);
+#pragma unroll
+                    for (int kk = 0; kk < kM / 16; ++kk)
+                        mma_bf16(tmem + kPcO2, desc_advance(dQh, kmaj(kk)), desc_advance(dSkl, kmaj(kk)), idescQS, true);
+                }
+                mma_commit(&ctl->bar_yqfree);
+                PROF_MARK();
+                // ---- state product U = X^T W (its accumulator was read in chunk n-1, before the state copy was written)
+#pragma unroll
+                for (int kk = 0; kk < kCT / 16; ++kk)
+                    mma_bf16(tmem + kPcU, desc_advance(dXm, mnmaj(kk)), desc_advance(dWh, mnmaj(kk)), idescU, kk > 0);
+                if (PAIRS) {
+#pragma unroll
+                    for (int kk = 0; kk < kCT / 16; ++kk)
+                        mma_bf16(tmem + kPcU, desc_advance(dXm, mnmaj(kk)), desc_advance(dWl, mnmaj(kk)), idescU, true);
+                }
+                mma_commit(&ctl->bar_mma1);
+                PROF_MARK();
+                // ---- value-side intra-chunk product: masked P (bf16 pair, in place in tensor memory) x W
+                PAIR_WAIT(&ctl->bar_pm, n & 1);
+                tc_fence_after_sync();
+                PROF_MARK();
+#pragma unroll
+                for (int kk = 0; kk < kCT / 16; ++kk)
+                    mma_bf16_ta(tmem + kPcOI, tmem + kPcP + 64 * (kk >> 2) + 8 * (kk & 3), desc_advance(dWh, mnmaj(kk)), idescYS,
+                                true);
+                if (PAIRS) {
+#pragma unroll
+                    for (int kk = 0; kk < kCT / 16; ++kk)
+                        mma_bf16_ta(tmem + kPcOI, tmem + kPcP + 64 * (kk >> 2) + 8 * (kk & 3), desc_advance(dWl, mnmaj(kk)),
+                                    idescYS, true);
+#pragma unroll
+                    for (int kk = 0; kk < kCT / 16; ++kk)
+                        mma_bf16_ta(tmem + kPcOI, tmem + kPcP + 64 * (kk >> 2) + 32 + 8 * (kk & 3),
+                                    desc_advance(dWh, mnmaj(kk)), idescYS, true);
+                }
+                mma_commit(&ctl->bar_v4);
+                PROF_MARK();
+                // ---- key-side intra-chunk product: masked A x X on top of the inter-chunk one
+                PAIR_WAIT(&ctl->bar_am, n & 1);
+                tc_fence_after_sync();
+                PROF_MARK();
+#pragma unroll
+                for (int kk = 0; kk < kCT / 16; ++kk)
+                    mma_bf16_ta(tmem + kPcO2, tmem + kPcA + 64 * (kk >> 2) + 8 * (kk & 3), desc_advance(dXm, mnmaj(kk)), idescAX,
+                                true);
+                if (PAIRS) {
+#pragma unroll
+                    for (int kk = 0; kk < kCT / 16; ++kk)
+                        mma_bf16_ta(tmem + kPcO2, tmem + kPcA + 64 * (kk >> 2) + 32 + 8 * (kk & 3),
+                                    desc_advance(dXm, mnmaj(kk)), idescAX, true);
+                }
+                mma_commit(&ctl->bar_k4);
+                PROF_MARK();
+                // ---- both first-product accumulators are free behind these: the next chunk's queue up
+                if (n + 1 < nchunks) {
+                    PAIR_WAIT(&ctl->bar_x[(n + 1) & 1], ((n + 1) >> 1) & 1);
+                    PAIR_WAIT(&ctl->bar_yq, (n + 1) & 1);
+                    PAIR_WAIT(&ctl->bar_w[(n + 1) & 1], ((n + 1) >> 1) & 1);
+                    tc_fence_after_sync();
+                    PROF_MARK();
+                    if (!ctl->abort) issue_first(n + 1);
+                }
+                PROF_MARK();
+                PROF_DUMP("rev_pair mma");
             }
-            PROF_MARK();
-            PROF_DUMP("rev_pair mma");
-        }
         }
     } else if (tid < kComputeThreads) {
         // =============================== compute threads
