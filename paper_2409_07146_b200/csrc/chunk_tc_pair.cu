@@ -10,9 +10,10 @@
 //     value-side:  out_v[i][s] = sum_{j>=i} <y_i, x_j> W_j[s]  +  exp(G_C)[s] (y_i S)[s]     (fp32 partial sums per slice)
 //     key-side:    out_k[i]    = sum_{j>=i} <Q_i, W_j> x_j     +  Q_i (exp(G_C) S)           (io dtype)
 // (row factors left out of out_v as in the single value_side kernel, see PendingDecay).  Per chunk
-// that is seven products on one tensor pipe, which they keep busy: while the compute threads mask
-// one first product, the pipe works on the other member's.  Compared with two single scans the
-// pair reads X, W and G once instead of twice and does not repeat the state product.
+// that is seven products on one tensor pipe: while the compute threads mask one first product, the
+// pipe works on the other member's.  Compared with two single scans the pair reads X, W and G once
+// instead of twice (a scan is bound by the rate at which its SM pulls tiles) and does not repeat the
+// state product.
 //
 // Only for (batch, head) pairs without a strong-decay chunk; the flagged ones take the two general
 // kernels.  Geometry, operand pairs (bf16 value + rounding residual) and bounded waits are those
