@@ -72,3 +72,19 @@ def test_bench_starts_its_own_ranks_when_run_as_a_plain_process(tmp_path):
     assert out.returncode == 0, out.stderr[-2000:]
     lines = [json.loads(l) for l in out.stdout.splitlines() if l.startswith("{")]
     assert len(lines) == 1 and lines[0]["impl"] == "reference" and lines[0]["n_gpus"] == 2
+
+
+def test_bench_byte_model_knows_every_step_label():
+    """Every timing label that a training step of the library can emit (the GSA_LAUNCH names of the forward
+    and backward cores) has an entry in bench.py's byte model: a new kernel must not break the bench line."""
+    import re
+    import gsa_workloads as W
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    src = open(os.path.join(root, "paper_2409_07146_b200", "csrc", "api.cu")).read()
+    labels = set(re.findall(r'GSA_LAUNCH\("([a-zA-Z0-9_]+)"', src))
+    step = {l for l in labels if l.startswith(("pass1", "pass2", "bwd_", "slot_softmax", "gate_cumsum", "gate_grad", "fused_"))}
+    assert {"pass1_value_side", "pass2_key_side", "bwd_dv_dIv_pair_rev", "bwd_dk_dIk_pair_rev", "gate_grad"} <= step
+    w = W.CONFIGS["train_1p3b"]
+    for lab in sorted(step):
+        assert bench.kernel_algorithmic_bytes(lab, w) > 0, lab
+        assert isinstance(bench.kernel_function(lab), str)
